@@ -1,0 +1,144 @@
+/*
+ * kvq.h -- C ABI of libkvq: fused int4 KV-cache quantizer for NVIDIA B200 (sm_100a).
+ *
+ * The library quantizes head-dim vectors x in R^D to 4-bit codes plus fp16 group
+ * scales and reconstructs them:
+ *
+ *   encode:  z = pack(F diag(s) x)            sign-randomized unitary DFT in its real
+ *                                             orthogonal form (Sec. 3.1, Eq. 1-2)
+ *            v = lambda (.) z                 per-channel rescale (Sec. 5.1 item 1, Sec. 7.1)
+ *            sigma_j = fp16(max_{c in group j} |v_c| / 7)          (Sec. 3.2 step 3, Sec. 5.6)
+ *            q_c = clamp(rint(v_c / sigma_j), -7, 7)               (Sec. 3.2 step 4)
+ *            byte_i = (q_{2i+1} << 4) | (q_{2i} & 0xF)             (Sec. 3.2, nibble pack)
+ *   decode:  x^ = diag(s) F^-1 unpack( q sigma / max(lambda, 1e-6) ) (Sec. 3.1; Sec. 5.1 item 1)
+ *
+ * Conventions
+ *   - DFT kernel e^{-2 pi i k n / D}; Eq. 2 packing: z_0 = Re Y_0, z_{D/2} = Re Y_{D/2},
+ *     z_k = sqrt2 Re Y_k and z_{D/2+k} = sqrt2 Im Y_k for 0 < k < D/2.
+ *   - groups are `group` consecutive coordinates of z; codes use the STORED fp16 scale;
+ *     rounding is half-to-even; a zero scale gives zero codes.
+ *   - every data pointer is a DEVICE pointer owned by the caller unless it says "host".
+ *     The library owns only the plan and the small device tables hanging off it.
+ *   - calls are asynchronous on the given CUDA stream (a cudaStream_t passed as void*,
+ *     NULL = default stream); they do not synchronize.  kvq_encode / kvq_decode /
+ *     kvq_append allocate nothing after the plan's first use on a device.
+ *   - every function returns a kvq_status_t; nothing throws across the boundary.
+ *     Arguments are validated on the host before any CUDA call is made.
+ *   - there is no CPU fallback: without a CUDA device the compute calls return KVQ_ERR_CUDA.
+ */
+#ifndef KVQ_H
+#define KVQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct kvq_plan kvq_plan_t; /* opaque, library-owned */
+
+typedef enum {
+    KVQ_OK = 0,
+    KVQ_ERR_INVALID_ARG = 1,     /* null pointer, negative size, lambda table too short, pos >= T_max ... */
+    KVQ_ERR_UNSUPPORTED_DIM = 2, /* D or group outside the supported set */
+    KVQ_ERR_ALIGNMENT = 3,       /* a base pointer is not 16-byte aligned */
+    KVQ_ERR_CUDA = 4,            /* a CUDA runtime call failed (no device, launch error ...) */
+    KVQ_ERR_TIMEOUT = 5,         /* a bounded device-side wait ran out (see kvq_plan_device_status) */
+    KVQ_ERR_NOMEM = 6
+} kvq_status_t;
+
+typedef enum { KVQ_F16 = 0, KVQ_BF16 = 1 } kvq_dtype_t;
+
+/* Which kernel family serves a call.  AUTO picks the fastest one that meets the
+ * tolerances for the plan's D and the call's dtype. */
+typedef enum {
+    KVQ_IMPL_AUTO = 0,
+    KVQ_IMPL_FFT = 1, /* fp32 register FFT, one thread per vector: every D and dtype */
+    KVQ_IMPL_GEMM = 2 /* tcgen05 DFT-as-GEMM; returns KVQ_ERR_UNSUPPORTED_DIM where not built */
+} kvq_impl_t;
+
+/*
+ * kvq_plan_create -- "kvq_plan(D, group, seed)": draws the sign diagonal s (Sec. 3.1: "a fixed
+ * random sign vector drawn at initialization") and fixes the radix plan of the length-D/2
+ * complex FFT (Sec. 3.2 step 2; mixed radix 3 / 5 for D = 96 / 160).
+ *   D      head dimension; supported: 64, 96, 128, 160, 256.
+ *   group  coordinates per scale; supported: 32 (must divide D).
+ *   seed   sign n is -1 when the top bit of the n-th SplitMix64 output for this seed is set.
+ *   out    host pointer receiving the plan.
+ * Touches no GPU: device tables are created on the first compute call, on the device that is
+ * current then.  Errors: INVALID_ARG (null out), UNSUPPORTED_DIM, NOMEM.
+ */
+kvq_status_t kvq_plan_create(int D, int group, uint64_t seed, kvq_plan_t **out);
+
+/* Frees the plan and its device tables.  NULL is a no-op.  The caller must make sure no call
+ * using the plan is still running on the GPU. */
+kvq_status_t kvq_plan_destroy(kvq_plan_t *plan);
+
+/* Copies the D signs (+1 / -1) to a HOST array, so that tests can hand the same diagonal to an
+ * independent implementation. */
+kvq_status_t kvq_plan_get_signs(const kvq_plan_t *plan, int8_t *host_signs /* [D] */);
+
+/* Describes the plan: the radices of the length-D/2 complex FFT in the order they are applied
+ * (host array of at least 8 ints), how many there are, and the bytes of device tables the plan
+ * holds once initialised.  Any output pointer may be NULL. */
+kvq_status_t kvq_plan_describe(const kvq_plan_t *plan, int *radices, int *n_radices, size_t *table_bytes);
+
+/* Selects the kernel family for later kvq_encode / kvq_append (encode_impl) and kvq_decode
+ * (decode_impl) calls on this plan.  Default: AUTO for both. */
+kvq_status_t kvq_plan_set_impl(kvq_plan_t *plan, kvq_impl_t encode_impl, kvq_impl_t decode_impl);
+
+/* Synchronizes the current device and returns the plan's device status word through *word
+ * (host): 0 when no kernel using this plan ever gave up a bounded wait.  Returns
+ * KVQ_ERR_TIMEOUT if the word is non-zero. */
+kvq_status_t kvq_plan_device_status(kvq_plan_t *plan, uint32_t *word);
+
+/*
+ * kvq_encode -- forward path (Sec. 3.2 steps 1-4 with the fused lambda and per-group scales of
+ * Sec. 7.1) on N vectors.
+ *   x        device, [N, D] row-major, fp16 or bf16 per `dtype`; 16-byte aligned.
+ *   lambda   device, fp32 [n_lambda, D]; row r of x uses lambda row r / rows_per_lambda
+ *            (row 0 for every r when n_lambda == 1).  Requires
+ *            n_lambda * rows_per_lambda >= N when n_lambda > 1.
+ *   packed   device out, [N, D/2] bytes, byte i of a row = (q[2i+1] << 4) | (q[2i] & 0xF);
+ *            16-byte aligned.
+ *   scales   device out, [N, D/group] fp16; 16-byte aligned.
+ * N == 0 is a no-op.  Errors: INVALID_ARG, ALIGNMENT, UNSUPPORTED_DIM, CUDA.
+ */
+kvq_status_t kvq_encode(kvq_plan_t *plan, const void *x, kvq_dtype_t dtype, int64_t N,
+                        const float *lambda, int64_t n_lambda, int64_t rows_per_lambda,
+                        uint8_t *packed, void *scales, void *cuda_stream);
+
+/*
+ * kvq_decode -- inverse path ("unpack, irfft, apply s", Sec. 3.1; lambda clamped at 1e-6,
+ * Sec. 5.1 item 1) on N stored vectors: the per-step full-prefix read.
+ *   packed, scales, lambda as in kvq_encode (inputs here);
+ *   out      device out, [N, D] row-major, fp16 or bf16 per `dtype` (round to nearest even);
+ *            16-byte aligned.
+ */
+kvq_status_t kvq_decode(kvq_plan_t *plan, const uint8_t *packed, const void *scales, int64_t N,
+                        const float *lambda, int64_t n_lambda, int64_t rows_per_lambda,
+                        void *out, kvq_dtype_t dtype, void *cuda_stream);
+
+/*
+ * kvq_append -- the decode-step write (Sec. 7.2: the cache stores K/V as int4 + scales between
+ * decode steps): quantizes S new vectors, one per stream, and writes them to row `pos` of
+ * caches laid out packed_cache [S, T_max, D/2] and scales_cache [S, T_max, D/group].
+ * Stream i uses lambda row i / streams_per_lambda (row 0 when n_lambda == 1).  No other row
+ * of the caches is touched.  Requires 0 <= pos < T_max.
+ */
+kvq_status_t kvq_append(kvq_plan_t *plan, const void *x_new /* [S, D] */, kvq_dtype_t dtype, int64_t S,
+                        const float *lambda, int64_t n_lambda, int64_t streams_per_lambda,
+                        uint8_t *packed_cache, void *scales_cache, int64_t T_max, int64_t pos,
+                        void *cuda_stream);
+
+/* Static, human-readable name of a status code. */
+const char *kvq_status_string(kvq_status_t status);
+
+/* Number of kernels the library has launched in this process (all plans, all streams). */
+uint64_t kvq_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KVQ_H */

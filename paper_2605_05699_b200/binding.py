@@ -1,0 +1,222 @@
+"""Thin ctypes binding over the C ABI of ``libkvq.so`` (``include/kvq.h``).
+
+Argument marshalling only: every step of the quantizer runs in the library's CUDA
+kernels.  PyTorch provides device memory and streams.  If the library has not
+been built the binding raises; there is no other code path.
+
+The functions carry the names of the C entry points: ``kvq_plan_create``,
+``kvq_encode``, ``kvq_decode``, ``kvq_append`` ...  ``Plan`` is a small
+convenience holder that frees the plan when collected.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libkvq.so")
+
+KVQ_OK = 0
+KVQ_ERR_INVALID_ARG = 1
+KVQ_ERR_UNSUPPORTED_DIM = 2
+KVQ_ERR_ALIGNMENT = 3
+KVQ_ERR_CUDA = 4
+KVQ_ERR_TIMEOUT = 5
+KVQ_ERR_NOMEM = 6
+
+KVQ_F16 = 0
+KVQ_BF16 = 1
+
+KVQ_IMPL_AUTO = 0
+KVQ_IMPL_FFT = 1
+KVQ_IMPL_GEMM = 2
+
+# every symbol include/kvq.h declares
+EXPORTS = (
+    "kvq_plan_create", "kvq_plan_destroy", "kvq_plan_get_signs", "kvq_plan_describe", "kvq_plan_set_impl",
+    "kvq_plan_device_status", "kvq_encode", "kvq_decode", "kvq_append", "kvq_status_string", "kvq_launch_count",
+)
+
+_lib = None
+
+
+class KvqError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s failed: %s" % (where, status_string(status)))
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libkvq.so (once).  Raises if it has not been built: there is no fallback."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                "libkvq.so is missing at %s; build it with `python -m paper_2605_05699_b200.build`" % LIB_PATH)
+        L = ctypes.CDLL(LIB_PATH)
+        i32, i64, u64, vp = ctypes.c_int, ctypes.c_int64, ctypes.c_uint64, ctypes.c_void_p
+        L.kvq_plan_create.restype = i32
+        L.kvq_plan_create.argtypes = [i32, i32, u64, ctypes.POINTER(vp)]
+        L.kvq_plan_destroy.restype = i32
+        L.kvq_plan_destroy.argtypes = [vp]
+        L.kvq_plan_get_signs.restype = i32
+        L.kvq_plan_get_signs.argtypes = [vp, vp]
+        L.kvq_plan_describe.restype = i32
+        L.kvq_plan_describe.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_size_t)]
+        L.kvq_plan_set_impl.restype = i32
+        L.kvq_plan_set_impl.argtypes = [vp, i32, i32]
+        L.kvq_plan_device_status.restype = i32
+        L.kvq_plan_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
+        L.kvq_encode.restype = i32
+        L.kvq_encode.argtypes = [vp, vp, i32, i64, vp, i64, i64, vp, vp, vp]
+        L.kvq_decode.restype = i32
+        L.kvq_decode.argtypes = [vp, vp, vp, i64, vp, i64, i64, vp, i32, vp]
+        L.kvq_append.restype = i32
+        L.kvq_append.argtypes = [vp, vp, i32, i64, vp, i64, i64, vp, vp, i64, i64, vp]
+        L.kvq_status_string.restype = ctypes.c_char_p
+        L.kvq_status_string.argtypes = [i32]
+        L.kvq_launch_count.restype = u64
+        L.kvq_launch_count.argtypes = []
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().kvq_status_string(int(status)).decode()
+
+
+def kvq_launch_count() -> int:
+    return int(lib().kvq_launch_count())
+
+
+def _check(status: int, where: str):
+    if status != KVQ_OK:
+        raise KvqError(status, where)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float16:
+        return KVQ_F16
+    if t.dtype == torch.bfloat16:
+        return KVQ_BF16
+    raise TypeError("expected a float16 or bfloat16 tensor, got %s" % t.dtype)
+
+
+def _dev(t: torch.Tensor, what: str) -> int:
+    if not t.is_cuda:
+        raise ValueError("%s must live on a CUDA device" % what)
+    if not t.is_contiguous():
+        raise ValueError("%s must be contiguous" % what)
+    return t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+# ---- C entry points, same names ---------------------------------------------------------
+
+def kvq_plan_create(D: int, group: int, seed: int) -> int:
+    h = ctypes.c_void_p()
+    _check(lib().kvq_plan_create(D, group, ctypes.c_uint64(seed & (2**64 - 1)), ctypes.byref(h)), "kvq_plan_create")
+    return h.value
+
+
+def kvq_plan_destroy(plan: int) -> None:
+    _check(lib().kvq_plan_destroy(plan), "kvq_plan_destroy")
+
+
+def kvq_plan_get_signs(plan: int, D: int):
+    import numpy as np
+
+    s = np.empty(D, dtype=np.int8)
+    _check(lib().kvq_plan_get_signs(plan, s.ctypes.data_as(ctypes.c_void_p)), "kvq_plan_get_signs")
+    return s
+
+
+def kvq_plan_describe(plan: int):
+    r = (ctypes.c_int * 8)()
+    n = ctypes.c_int()
+    tb = ctypes.c_size_t()
+    _check(lib().kvq_plan_describe(plan, r, ctypes.byref(n), ctypes.byref(tb)), "kvq_plan_describe")
+    return list(r[: n.value]), int(tb.value)
+
+
+def kvq_plan_set_impl(plan: int, encode_impl: int, decode_impl: int) -> None:
+    _check(lib().kvq_plan_set_impl(plan, encode_impl, decode_impl), "kvq_plan_set_impl")
+
+
+def kvq_plan_device_status(plan: int) -> int:
+    w = ctypes.c_uint32()
+    st = lib().kvq_plan_device_status(plan, ctypes.byref(w))
+    if st not in (KVQ_OK, KVQ_ERR_TIMEOUT):
+        raise KvqError(st, "kvq_plan_device_status")
+    return int(w.value)
+
+
+def kvq_encode(plan: int, x: torch.Tensor, lam: torch.Tensor, packed: torch.Tensor, scales: torch.Tensor,
+               rows_per_lambda: int = 0, stream=None) -> None:
+    D = x.shape[-1]
+    N = x.numel() // D
+    n_lambda = lam.numel() // D
+    with torch.cuda.device(x.device):
+        _check(lib().kvq_encode(plan, _dev(x, "x"), _dtype_code(x), N, _dev(lam, "lambda"), n_lambda,
+                                rows_per_lambda, _dev(packed, "packed"), _dev(scales, "scales"), _stream(stream)),
+               "kvq_encode")
+
+
+def kvq_decode(plan: int, packed: torch.Tensor, scales: torch.Tensor, lam: torch.Tensor, out: torch.Tensor,
+               rows_per_lambda: int = 0, stream=None) -> None:
+    D = out.shape[-1]
+    N = out.numel() // D
+    n_lambda = lam.numel() // D
+    with torch.cuda.device(out.device):
+        _check(lib().kvq_decode(plan, _dev(packed, "packed"), _dev(scales, "scales"), N, _dev(lam, "lambda"),
+                                n_lambda, rows_per_lambda, _dev(out, "out"), _dtype_code(out), _stream(stream)),
+               "kvq_decode")
+
+
+def kvq_append(plan: int, x_new: torch.Tensor, lam: torch.Tensor, packed_cache: torch.Tensor,
+               scales_cache: torch.Tensor, pos: int, streams_per_lambda: int = 0, stream=None) -> None:
+    D = x_new.shape[-1]
+    S = x_new.numel() // D
+    T_max = packed_cache.shape[-2]
+    n_lambda = lam.numel() // D
+    with torch.cuda.device(x_new.device):
+        _check(lib().kvq_append(plan, _dev(x_new, "x_new"), _dtype_code(x_new), S, _dev(lam, "lambda"), n_lambda,
+                                streams_per_lambda, _dev(packed_cache, "packed_cache"),
+                                _dev(scales_cache, "scales_cache"), T_max, pos, _stream(stream)),
+               "kvq_append")
+
+
+class Plan:
+    """Owns a ``kvq_plan_t`` handle: ``Plan(D, group, seed).handle`` goes to the kvq_* calls."""
+
+    def __init__(self, D: int, group: int = 32, seed: int = 0):
+        self.D, self.group, self.seed = D, group, seed
+        self.handle = kvq_plan_create(D, group, seed)
+
+    def signs(self):
+        return kvq_plan_get_signs(self.handle, self.D)
+
+    def close(self):
+        if getattr(self, "handle", None):
+            kvq_plan_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):  # pragma: no cover
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # allocation helpers for callers that do not bring their own buffers
+    def empty_packed(self, N: int, device="cuda") -> torch.Tensor:
+        return torch.empty(N, self.D // 2, dtype=torch.uint8, device=device)
+
+    def empty_scales(self, N: int, device="cuda") -> torch.Tensor:
+        return torch.empty(N, self.D // self.group, dtype=torch.float16, device=device)

@@ -1,0 +1,275 @@
+// C ABI of libkvq (see include/kvq.h): plan object, host-side validation, dispatch.
+#include <atomic>
+#include <cstring>
+#include <mutex>
+#include <new>
+
+#include "../../include/kvq.h"
+#include "kvq_internal.h"
+
+namespace kvq {
+
+static std::atomic<uint64_t> g_launches{0};
+void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+
+// SplitMix64 output function (Steele, Lea, Flood 2014); sign n uses the n-th output for `seed`.
+static inline uint64_t splitmix64_at(uint64_t seed, uint64_t n)
+{
+    uint64_t z = seed + (n + 1) * 0x9E3779B97F4A7C15ULL;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ULL;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBULL;
+    return z ^ (z >> 31);
+}
+
+static bool dim_supported(int D) { return D == 64 || D == 96 || D == 128 || D == 160 || D == 256; }
+
+// Radices of the length-n complex FFT in the order the recursion splits them off (4 first,
+// then 2, 3, 5), mirroring radix_of() on the device side.
+static int radix_plan(int n, int *out)
+{
+    int k = 0;
+    while (n > 1) {
+        int r = n % 4 == 0 ? 4 : n % 2 == 0 ? 2 : n % 3 == 0 ? 3 : n % 5 == 0 ? 5 : n;
+        out[k++] = r;
+        n /= r;
+    }
+    return k;
+}
+
+}  // namespace kvq
+
+struct kvq_plan {
+    int D, group;
+    uint64_t seed;
+    int8_t signs[256];
+    uint32_t sign_xor[128];
+    kvq_impl_t enc_impl, dec_impl;
+    // device state, created on first use
+    std::mutex mu;
+    int device;            // -1 until initialised
+    uint32_t *d_status;    // device status word
+    size_t table_bytes;
+};
+
+using namespace kvq;
+
+static kvq_status_t ensure_device(kvq_plan *p)
+{
+    std::lock_guard<std::mutex> lk(p->mu);
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return KVQ_ERR_CUDA;
+    }
+    if (p->device == dev) return KVQ_OK;
+    if (p->device >= 0) return KVQ_ERR_INVALID_ARG;   // a plan stays on the device of its first use
+    uint32_t *st = nullptr;
+    if (cudaMalloc(&st, 256) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return KVQ_ERR_NOMEM;
+    }
+    if (cudaMemset(st, 0, 256) != cudaSuccess) {
+        (void)cudaGetLastError();
+        cudaFree(st);
+        return KVQ_ERR_CUDA;
+    }
+    p->d_status = st;
+    p->table_bytes = 256;
+    p->device = dev;
+    return KVQ_OK;
+}
+
+static bool misaligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+static kvq_status_t check_lambda(int64_t N, const float *lambda, int64_t n_lambda, int64_t rows_per_lambda)
+{
+    if (!lambda || n_lambda < 1) return KVQ_ERR_INVALID_ARG;
+    if (n_lambda > 1) {
+        if (rows_per_lambda < 1) return KVQ_ERR_INVALID_ARG;
+        if ((N + rows_per_lambda - 1) / rows_per_lambda > n_lambda) return KVQ_ERR_INVALID_ARG;
+    }
+    if (misaligned16(lambda)) return KVQ_ERR_ALIGNMENT;
+    return KVQ_OK;
+}
+
+static void fill_params(const kvq_plan *p, FftParams &prm, int64_t N, const float *lambda, int64_t n_lambda,
+                        int64_t rows_per_lambda)
+{
+    std::memset(&prm, 0, sizeof(prm));
+    prm.N = N;
+    prm.lambda = lambda;
+    prm.n_lambda = n_lambda;
+    prm.rows_per_lambda = rows_per_lambda < 1 ? 1 : rows_per_lambda;
+    prm.out_mul = 1;
+    prm.out_add = 0;
+    prm.status = p->d_status;
+    std::memcpy(prm.sign_xor, p->sign_xor, sizeof(prm.sign_xor));
+}
+
+extern "C" {
+
+kvq_status_t kvq_plan_create(int D, int group, uint64_t seed, kvq_plan_t **out)
+{
+    if (!out) return KVQ_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!dim_supported(D) || group != 32 || D % group) return KVQ_ERR_UNSUPPORTED_DIM;
+    kvq_plan *p = new (std::nothrow) kvq_plan();
+    if (!p) return KVQ_ERR_NOMEM;
+    p->D = D;
+    p->group = group;
+    p->seed = seed;
+    p->enc_impl = p->dec_impl = KVQ_IMPL_AUTO;
+    p->device = -1;
+    p->d_status = nullptr;
+    p->table_bytes = 0;
+    std::memset(p->signs, 0, sizeof(p->signs));
+    std::memset(p->sign_xor, 0, sizeof(p->sign_xor));
+    for (int n = 0; n < D; ++n) {
+        bool neg = (splitmix64_at(seed, (uint64_t)n) >> 63) != 0;
+        p->signs[n] = neg ? -1 : 1;
+        if (neg) p->sign_xor[n / 2] |= (n & 1) ? 0x80000000u : 0x00008000u;
+    }
+    *out = p;
+    return KVQ_OK;
+}
+
+kvq_status_t kvq_plan_destroy(kvq_plan_t *plan)
+{
+    if (!plan) return KVQ_OK;
+    if (plan->d_status) {
+        if (cudaFree(plan->d_status) != cudaSuccess) (void)cudaGetLastError();
+    }
+    delete plan;
+    return KVQ_OK;
+}
+
+kvq_status_t kvq_plan_get_signs(const kvq_plan_t *plan, int8_t *host_signs)
+{
+    if (!plan || !host_signs) return KVQ_ERR_INVALID_ARG;
+    std::memcpy(host_signs, plan->signs, (size_t)plan->D);
+    return KVQ_OK;
+}
+
+kvq_status_t kvq_plan_describe(const kvq_plan_t *plan, int *radices, int *n_radices, size_t *table_bytes)
+{
+    if (!plan) return KVQ_ERR_INVALID_ARG;
+    int r[16];
+    int n = radix_plan(plan->D / 2, r);
+    if (radices)
+        for (int i = 0; i < n && i < 8; ++i) radices[i] = r[i];
+    if (n_radices) *n_radices = n;
+    if (table_bytes) *table_bytes = plan->table_bytes;
+    return KVQ_OK;
+}
+
+kvq_status_t kvq_plan_set_impl(kvq_plan_t *plan, kvq_impl_t encode_impl, kvq_impl_t decode_impl)
+{
+    if (!plan) return KVQ_ERR_INVALID_ARG;
+    if ((int)encode_impl < 0 || (int)encode_impl > 2 || (int)decode_impl < 0 || (int)decode_impl > 2)
+        return KVQ_ERR_INVALID_ARG;
+    plan->enc_impl = encode_impl;
+    plan->dec_impl = decode_impl;
+    return KVQ_OK;
+}
+
+kvq_status_t kvq_plan_device_status(kvq_plan_t *plan, uint32_t *word)
+{
+    if (!plan || !word) return KVQ_ERR_INVALID_ARG;
+    *word = 0;
+    if (!plan->d_status) return KVQ_OK;   // never used on a device
+    if (cudaDeviceSynchronize() != cudaSuccess) {
+        (void)cudaGetLastError();
+        return KVQ_ERR_CUDA;
+    }
+    if (cudaMemcpy(word, plan->d_status, sizeof(uint32_t), cudaMemcpyDeviceToHost) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return KVQ_ERR_CUDA;
+    }
+    return *word ? KVQ_ERR_TIMEOUT : KVQ_OK;
+}
+
+static kvq_status_t encode_common(kvq_plan_t *plan, const void *x, kvq_dtype_t dtype, int64_t N, const float *lambda,
+                                  int64_t n_lambda, int64_t rows_per_lambda, uint8_t *packed, void *scales,
+                                  int64_t out_mul, int64_t out_add, void *cuda_stream)
+{
+    if (!plan || N < 0) return KVQ_ERR_INVALID_ARG;
+    if (dtype != KVQ_F16 && dtype != KVQ_BF16) return KVQ_ERR_INVALID_ARG;
+    if (!x || !packed || !scales) return KVQ_ERR_INVALID_ARG;
+    kvq_status_t st = check_lambda(N, lambda, n_lambda, rows_per_lambda);
+    if (st != KVQ_OK) return st;
+    if (misaligned16(x) || misaligned16(packed) || misaligned16(scales)) return KVQ_ERR_ALIGNMENT;
+    if (plan->enc_impl == KVQ_IMPL_GEMM) return KVQ_ERR_UNSUPPORTED_DIM;
+    if (N == 0) return KVQ_OK;
+    if ((st = ensure_device(plan)) != KVQ_OK) return st;
+    FftParams prm;
+    fill_params(plan, prm, N, lambda, n_lambda, rows_per_lambda);
+    prm.in = x;
+    prm.packed = packed;
+    prm.scales = scales;
+    prm.out_mul = out_mul;
+    prm.out_add = out_add;
+    cudaError_t e = fft_encode(plan->D, dtype == KVQ_BF16, N, prm, static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        return KVQ_ERR_CUDA;
+    }
+    return KVQ_OK;
+}
+
+kvq_status_t kvq_encode(kvq_plan_t *plan, const void *x, kvq_dtype_t dtype, int64_t N, const float *lambda,
+                        int64_t n_lambda, int64_t rows_per_lambda, uint8_t *packed, void *scales, void *cuda_stream)
+{
+    return encode_common(plan, x, dtype, N, lambda, n_lambda, rows_per_lambda, packed, scales, 1, 0, cuda_stream);
+}
+
+kvq_status_t kvq_append(kvq_plan_t *plan, const void *x_new, kvq_dtype_t dtype, int64_t S, const float *lambda,
+                        int64_t n_lambda, int64_t streams_per_lambda, uint8_t *packed_cache, void *scales_cache,
+                        int64_t T_max, int64_t pos, void *cuda_stream)
+{
+    if (T_max < 1 || pos < 0 || pos >= T_max) return KVQ_ERR_INVALID_ARG;
+    return encode_common(plan, x_new, dtype, S, lambda, n_lambda, streams_per_lambda, packed_cache, scales_cache,
+                         T_max, pos, cuda_stream);
+}
+
+kvq_status_t kvq_decode(kvq_plan_t *plan, const uint8_t *packed, const void *scales, int64_t N, const float *lambda,
+                        int64_t n_lambda, int64_t rows_per_lambda, void *out, kvq_dtype_t dtype, void *cuda_stream)
+{
+    if (!plan || N < 0) return KVQ_ERR_INVALID_ARG;
+    if (dtype != KVQ_F16 && dtype != KVQ_BF16) return KVQ_ERR_INVALID_ARG;
+    if (!packed || !scales || !out) return KVQ_ERR_INVALID_ARG;
+    kvq_status_t st = check_lambda(N, lambda, n_lambda, rows_per_lambda);
+    if (st != KVQ_OK) return st;
+    if (misaligned16(packed) || misaligned16(scales) || misaligned16(out)) return KVQ_ERR_ALIGNMENT;
+    if (plan->dec_impl == KVQ_IMPL_GEMM) return KVQ_ERR_UNSUPPORTED_DIM;
+    if (N == 0) return KVQ_OK;
+    if ((st = ensure_device(plan)) != KVQ_OK) return st;
+    FftParams prm;
+    fill_params(plan, prm, N, lambda, n_lambda, rows_per_lambda);
+    prm.packed = const_cast<uint8_t *>(packed);
+    prm.scales = const_cast<void *>(scales);
+    prm.out = out;
+    cudaError_t e = fft_decode(plan->D, dtype == KVQ_BF16, N, prm, static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        return KVQ_ERR_CUDA;
+    }
+    return KVQ_OK;
+}
+
+const char *kvq_status_string(kvq_status_t status)
+{
+    switch (status) {
+        case KVQ_OK: return "KVQ_OK";
+        case KVQ_ERR_INVALID_ARG: return "KVQ_ERR_INVALID_ARG";
+        case KVQ_ERR_UNSUPPORTED_DIM: return "KVQ_ERR_UNSUPPORTED_DIM";
+        case KVQ_ERR_ALIGNMENT: return "KVQ_ERR_ALIGNMENT";
+        case KVQ_ERR_CUDA: return "KVQ_ERR_CUDA";
+        case KVQ_ERR_TIMEOUT: return "KVQ_ERR_TIMEOUT";
+        case KVQ_ERR_NOMEM: return "KVQ_ERR_NOMEM";
+    }
+    return "KVQ_ERR_UNKNOWN";
+}
+
+uint64_t kvq_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

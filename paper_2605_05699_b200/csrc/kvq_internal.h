@@ -1,0 +1,29 @@
+// Declarations shared by the translation units of libkvq (not part of the public ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace kvq {
+
+// Arguments of the register-FFT kernels.  Passed by value as a __grid_constant__
+// parameter, so the sign words are read straight from the constant bank.
+struct FftParams {
+    const void *in;        // encode: x [N, D] half precision
+    const float *lambda;   // [n_lambda, D] fp32
+    void *packed;          // [*, D/2] bytes (encode: out, decode: in)
+    void *scales;          // [*, D/group] fp16 (encode: out, decode: in)
+    void *out;             // decode: x^ [N, D] half precision
+    int64_t N;
+    int64_t n_lambda, rows_per_lambda;
+    int64_t out_mul, out_add;   // encode: output row of input row r is r * out_mul + out_add
+    uint32_t *status;           // per-plan device status word
+    uint32_t sign_xor[128];     // word m: bit 15 set if s_{2m} = -1, bit 31 set if s_{2m+1} = -1
+};
+
+cudaError_t fft_encode(int D, bool bf16, int64_t N, const FftParams &prm, cudaStream_t stream);
+cudaError_t fft_decode(int D, bool bf16, int64_t N, const FftParams &prm, cudaStream_t stream);
+
+void count_launch();
+
+}  // namespace kvq

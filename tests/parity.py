@@ -1,0 +1,91 @@
+"""Parity rules between the CUDA path and the fp64 oracle, written once.
+
+Tolerances (the benchmark spec's, with the readings the design notes list):
+  * nibble pack / unpack: bit-exact (GPU bytes unpack to the GPU's own codes and repack to the same bytes;
+    where codes agree the bytes agree).
+  * int4 codes: identical on >= 99.99 % of entries; every mismatch is off by exactly one and lies at a
+    rounding tie: with t = v_oracle / sigma in fp64, |t - boundary| <= 1e-3 for sigma = the GPU's or the
+    oracle's stored scale; or, when the two stored scales differ (by one fp16 ulp at most), the GPU code is
+    the correctly rounded code for the GPU's own stored scale.
+  * group scales: |sigma_gpu - sigma_oracle| <= 1 fp16 ulp everywhere, and relative L2 per vector <= 1e-3.
+  * reconstruction: relative L2 per vector <= 1e-3 against the oracle's output rounded to the same dtype.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+from oracle import kvq_oracle as ko
+
+CODE_AGREEMENT = 0.9999
+TIE_TOL = 1e-3
+REL_L2 = 1e-3
+
+
+def f16_bits_to_f64(b):
+    return np.ascontiguousarray(b).view(np.uint16).view(np.float16).astype(np.float64)
+
+
+def check_encode(gpu_packed, gpu_scales_bits, ora, group, label=""):
+    """gpu_packed [N,D/2] uint8, gpu_scales_bits [N,G] uint16, ora = oracle.encode(..., want_v=True)."""
+    gpu_packed = np.ascontiguousarray(gpu_packed)
+    gpu_scales_bits = np.ascontiguousarray(gpu_scales_bits).view(np.uint16)
+    N, Dh = gpu_packed.shape
+    D = 2 * Dh
+    G = D // group
+    q_gpu = ko.unpack_nibbles(gpu_packed)
+    # pack/unpack bit-exactness
+    assert np.array_equal(ko.pack_nibbles(q_gpu), gpu_packed), label + ": repacking the GPU codes changes bytes"
+    assert q_gpu.min(initial=0) >= -7 and q_gpu.max(initial=0) <= 7, label + ": code outside [-7, 7]"
+    q_or = ora["codes"]
+    same = q_gpu == q_or
+    byte_same = gpu_packed == ora["packed"]
+    assert np.array_equal(byte_same, same[:, 0::2] & same[:, 1::2]), label + ": byte layout disagrees with codes"
+
+    # scales
+    bg = gpu_scales_bits.astype(np.int64)
+    bo = ora["scales"].astype(np.int64)
+    assert np.abs(bg - bo).max(initial=0) <= 1, label + ": a scale differs by more than one fp16 ulp"
+    sg, so = f16_bits_to_f64(gpu_scales_bits), f16_bits_to_f64(ora["scales"])
+    den = np.linalg.norm(so, axis=1)
+    rel = np.linalg.norm(sg - so, axis=1) / np.where(den > 0, den, 1.0)
+    assert rel.max(initial=0) <= REL_L2, label + ": scales relative L2 %.3g" % rel.max()
+    scale_flip_frac = float((bg != bo).mean()) if bg.size else 0.0
+    assert scale_flip_frac < 0.01, label + ": %.3g of the scales differ" % scale_flip_frac
+
+    # codes
+    agree = float(same.mean()) if same.size else 1.0
+    assert agree >= CODE_AGREEMENT, label + ": only %.6f of the codes agree" % agree
+    rr, cc = np.nonzero(~same)
+    if rr.size:
+        v = ora["v"][rr, cc]
+        qg = q_gpu[rr, cc].astype(np.int64)
+        qo = q_or[rr, cc].astype(np.int64)
+        assert np.all(np.abs(qg - qo) == 1), label + ": a code differs by more than one"
+        boundary = (qg + qo) / 2.0
+        s_g, s_o = sg[rr, cc // group], so[rr, cc // group]
+        with np.errstate(divide="ignore", invalid="ignore"):
+            t_g, t_o = v / s_g, v / s_o
+        at_tie = (np.abs(t_g - boundary) <= TIE_TOL) | (np.abs(t_o - boundary) <= TIE_TOL)
+        own = (s_g != s_o) & (np.clip(np.rint(t_g), -7, 7) == qg)
+        bad = ~(at_tie | own)
+        assert not bad.any(), label + ": %d mismatched codes are not at a rounding tie (e.g. t=%r)" % (
+            bad.sum(), t_o[bad][:4])
+    return {"agree": agree, "mismatches": int(rr.size), "scale_flips": scale_flip_frac,
+            "scale_rel_l2": float(rel.max(initial=0))}
+
+
+def rel_l2_rows(a, b):
+    den = np.linalg.norm(b, axis=1)
+    num = np.linalg.norm(a - b, axis=1)
+    return np.where(den > 0, num / np.where(den > 0, den, 1.0), num)
+
+
+def check_decode(gpu_bits, ora_bits, dtype, label=""):
+    """Both are raw uint16 bits of the half-precision outputs, [N, D]."""
+    g = ko.widen(np.ascontiguousarray(gpu_bits).view(np.uint16), dtype)
+    o = ko.widen(ora_bits, dtype)
+    assert np.isfinite(g).all(), label + ": non-finite output"
+    rel = rel_l2_rows(g, o)
+    assert rel.max(initial=0) <= REL_L2, label + ": reconstruction relative L2 %.3g" % rel.max()
+    return {"rel_l2_max": float(rel.max(initial=0)), "rel_l2_mean": float(rel.mean()) if rel.size else 0.0,
+            "bit_equal": float((np.ascontiguousarray(gpu_bits).view(np.uint16) == ora_bits).mean()) if g.size else 1.0}

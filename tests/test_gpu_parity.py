@@ -1,0 +1,218 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import kvq_oracle as ko
+from paper_2605_05699_b200 import binding as kb
+from paper_2605_05699_b200 import workloads as wl
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+G = wl.GROUP
+DT = {"f16": ko.F16, "bf16": ko.BF16}
+
+
+def bits(t):
+    return wl.raw_bits(t)
+
+
+def gpu_encode(plan, x, lam, rows_per_lambda=0):
+    N = x.shape[0]
+    packed, scales = plan.empty_packed(N), plan.empty_scales(N)
+    kb.kvq_encode(plan.handle, x, lam, packed, scales, rows_per_lambda)
+    torch.cuda.synchronize()
+    assert kb.kvq_plan_device_status(plan.handle) == 0
+    return packed, scales
+
+
+def gpu_decode(plan, packed, scales, lam, dtype, rows_per_lambda=0):
+    N = packed.shape[0]
+    out = torch.empty(N, plan.D, dtype=wl.torch_dtype(dtype), device="cuda")
+    kb.kvq_decode(plan.handle, packed, scales, lam, out, rows_per_lambda)
+    torch.cuda.synchronize()
+    assert kb.kvq_plan_device_status(plan.handle) == 0
+    return out
+
+
+def run_case(D, dtype, N, kind, seed, n_lambda=1, rows_per_lambda=0, plan_seed=None):
+    """Encode on GPU vs oracle; decode the ORACLE's compressed data on GPU vs oracle; GPU round trip."""
+    plan = kb.Plan(D, G, seed if plan_seed is None else plan_seed)
+    sg = plan.signs()
+    assert np.array_equal(sg, ko.signs(D, plan.seed))  # two independent implementations of the sign stream
+    x = wl.make_vectors(N, D, dtype, kind, seed)
+    lam = wl.make_lambda(n_lambda, D, seed + 1)
+    ora = ko.encode(bits(x), DT[dtype], sg, lam.numpy(), G, rows_per_lambda, want_v=True)
+    xd, lamd = x.cuda(), lam.cuda()
+    packed, scales = gpu_encode(plan, xd, lamd, rows_per_lambda)
+    label = "D=%d %s N=%d" % (D, dtype, N)
+    enc = parity.check_encode(packed.cpu().numpy(), bits(scales), ora, G, label + " encode")
+    # decode parity on the oracle's own compressed representation
+    ob = ko.decode(ora["packed"], ora["scales"], sg, lam.numpy(), G, DT[dtype], rows_per_lambda)
+    pk_o = torch.from_numpy(ora["packed"]).cuda()
+    sc_o = torch.from_numpy(ora["scales"].view(np.int16)).view(torch.float16).cuda()
+    out = gpu_decode(plan, pk_o, sc_o, lamd, dtype, rows_per_lambda)
+    dec = parity.check_decode(bits(out), ob, DT[dtype], label + " decode")
+    # GPU round trip stays close to the input (4-bit noise level, sanity only)
+    rt = gpu_decode(plan, packed, scales, lamd, dtype, rows_per_lambda).float().cpu().numpy()
+    xin = x.float().numpy()
+    rel = parity.rel_l2_rows(rt, xin)
+    assert np.median(rel) < 0.2
+    plan.close()
+    return enc, dec
+
+
+# ---- config 1: one tensor, 4096 x 128 fp16, outlier channels, lambda U(0.5, 2) -------------
+
+def test_config1_single_tensor_d128_f16():
+    enc, dec = run_case(128, "f16", 4096, "c1", 1001)
+    assert enc["mismatches"] <= 52  # 99.99 % of 524288 codes
+
+
+# ---- every head dim and dtype, ragged N (several tiles plus a tail), lambda rows that straddle tiles
+
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("D", [64, 96, 128, 160, 256])
+def test_all_dims_ragged_with_straddling_lambda_rows(D, dtype):
+    run_case(D, dtype, 1000, "k_outlier", 2000 + D, n_lambda=4, rows_per_lambda=333)
+
+
+@pytest.mark.parametrize("N", [1, 31, 32, 33, 4100])
+def test_small_and_ragged_sizes(N):
+    run_case(128, "f16", N, "gaussian", 3000 + N)
+
+
+def test_empty_input_is_a_noop():
+    plan = kb.Plan(128, G, 1)
+    x = torch.empty(0, 128, dtype=torch.float16, device="cuda")
+    lam = torch.ones(128, device="cuda")
+    pk, sc = plan.empty_packed(0), plan.empty_scales(0)
+    kb.kvq_encode(plan.handle, x, lam, pk, sc)
+    kb.kvq_decode(plan.handle, pk, sc, lam, x)
+    torch.cuda.synchronize()
+
+
+# ---- config 4: mixed-radix head dims, 65536 vectors each ------------------------------------
+
+@pytest.mark.parametrize("D", [96, 160])
+def test_config4_mixed_radix(D):
+    run_case(D, "f16", 65536, "lognormal", 4000 + D)
+
+
+# ---- config 2: Qwen2.5-1.5B-shaped cache: prefill, appends, full-prefix decode -------------
+
+def test_config2_qwen_shaped_prefill_append_decode():
+    shp = wl.QWEN25_1P5B
+    D, T0, steps = shp.head_dim, shp.prefix, 4
+    S = shp.streams  # 112 streams: (layer, K/V, head)
+    T_max = T0 + steps
+    per_lambda = shp.kv_heads  # one lambda row per (layer, K/V): 56 rows
+    n_lambda = S // per_lambda
+    plan = kb.Plan(D, G, 77)
+    sg = plan.signs()
+    lam = wl.make_lambda(n_lambda, D, 21)
+    # stream i is K-like for even (layer, kv) index, V-like for odd
+    xs = []
+    for i in range(n_lambda):
+        kind = "k_outlier" if i % 2 == 0 else "gaussian"
+        xs.append(wl.make_vectors(per_lambda * T_max, D, shp.dtype, kind, 500 + i).view(per_lambda, T_max, D))
+    x_all = torch.cat(xs, 0)  # [S, T_max, D]
+    lamd = lam.cuda()
+    packed = torch.zeros(S, T_max, D // 2, dtype=torch.uint8, device="cuda")
+    scales = torch.zeros(S, T_max, D // G, dtype=torch.float16, device="cuda")
+    # prefill: one encode per stream block sharing a lambda row (rows of a stream are contiguous in the cache)
+    for i in range(n_lambda):
+        for h in range(per_lambda):
+            s = i * per_lambda + h
+            xp = x_all[s, :T0].contiguous().cuda()
+            kb.kvq_encode(plan.handle, xp, lamd[i], packed[s, :T0], scales[s, :T0])
+    # decode steps: append one vector per stream
+    for t in range(steps):
+        xn = x_all[:, T0 + t].contiguous().cuda()
+        kb.kvq_append(plan.handle, xn, lamd, packed, scales, T0 + t, per_lambda)
+    torch.cuda.synchronize()
+    assert kb.kvq_plan_device_status(plan.handle) == 0
+    # oracle on the whole cache [S*T_max rows, lambda row = stream // per_lambda]
+    ora = ko.encode(bits(x_all.reshape(-1, D)), ko.F16, sg, lam.numpy(), G, per_lambda * T_max, want_v=True)
+    parity.check_encode(packed.view(-1, D // 2).cpu().numpy(), bits(scales.view(-1, D // G)), ora, G, "qwen cache")
+    # full-prefix decode of the whole cache in one launch
+    out = gpu_decode(plan, packed.view(-1, D // 2), scales.view(-1, D // G), lamd, shp.dtype, per_lambda * T_max)
+    ob = ko.decode(packed.view(-1, D // 2).cpu().numpy(), bits(scales.view(-1, D // G)), sg, lam.numpy(), G, ko.F16,
+                   per_lambda * T_max)
+    parity.check_decode(bits(out), ob, ko.F16, "qwen full-prefix decode")
+    plan.close()
+
+
+def test_append_touches_only_row_pos():
+    D, S, T = 128, 37, 9
+    plan = kb.Plan(D, G, 5)
+    x = wl.make_vectors(S, D, "f16", "gaussian", 9).cuda()
+    lam = wl.make_lambda(S, D, 10).cuda()
+    packed = torch.full((S, T, D // 2), 0xAB, dtype=torch.uint8, device="cuda")
+    scales = torch.full((S, T, D // G), 1.25, dtype=torch.float16, device="cuda")
+    kb.kvq_append(plan.handle, x, lam, packed, scales, 4, 1)
+    torch.cuda.synchronize()
+    keep = [t for t in range(T) if t != 4]
+    assert bool((packed[:, keep] == 0xAB).all()) and bool((scales[:, keep] == 1.25).all())
+    pc = np.full((S, T, D // 2), 0xAB, dtype=np.uint8)
+    sc = np.full((S, T, D // G), np.float16(1.25).view(np.uint16), dtype=np.uint16)
+    ko.append(bits(x), ko.F16, plan.signs(), lam.cpu().numpy(), G, pc, sc, 4, 1)
+    assert (packed.cpu().numpy() == pc).mean() > 0.999
+    assert np.abs(bits(scales).astype(np.int64) - sc.astype(np.int64)).max() <= 1
+    plan.close()
+
+
+# ---- config 3: Gemma-3-1B-shaped, D = 256 bf16, prefix sweep ---------------------------------
+
+@pytest.mark.parametrize("prefix", [256, 1024])
+def test_config3_gemma_shaped_d256_bf16(prefix):
+    shp = wl.GEMMA3_1B
+    N = 2 * shp.layers * prefix  # K and V of every layer
+    run_case(256, "bf16", N, "c1", 6000 + prefix, n_lambda=2 * shp.layers, rows_per_lambda=prefix)
+
+
+def test_config3_gemma_shaped_prefix_4096_sampled():
+    _full_size_sampled(256, "bf16", 2 * wl.GEMMA3_1B.layers * 4096, "c1", 6100, 2 * wl.GEMMA3_1B.layers, 4096)
+
+
+# ---- config 5: Llama-3-70B-shaped: one layer's K (1,048,576 vectors) per launch, sampled rows -
+
+def _full_size_sampled(D, dtype, N, kind, seed, n_lambda, rows_per_lambda, n_random=4096):
+    plan = kb.Plan(D, G, seed)
+    sg = plan.signs()
+    x = wl.make_vectors(N, D, dtype, kind, seed, device="cuda")
+    lam = wl.make_lambda(n_lambda, D, seed + 1, device="cuda")
+    packed, scales = gpu_encode(plan, x, lam, rows_per_lambda)
+    out = gpu_decode(plan, packed, scales, lam, dtype, rows_per_lambda)
+    g = torch.Generator().manual_seed(seed)
+    idx = torch.cat([torch.arange(0, 2048), torch.arange(N - 2048, N), torch.randint(0, N, (n_random,), generator=g)])
+    idx = torch.unique(idx)
+    idx_d = idx.cuda()
+    lam_h = lam.cpu().numpy()
+    lrow = (idx // rows_per_lambda).numpy() if n_lambda > 1 else np.zeros(len(idx), dtype=np.int64)
+    xs, pk, sc, od = x[idx_d].cpu(), packed[idx_d].cpu().numpy(), bits(scales[idx_d]), bits(out[idx_d])
+    for l in np.unique(lrow):
+        m = lrow == l
+        ora = ko.encode(bits(xs)[m], DT[dtype], sg, lam_h[l], G, want_v=True)
+        parity.check_encode(pk[m], sc[m], ora, G, "full-size encode lambda row %d" % l)
+        ob = ko.decode(pk[m], sc[m], sg, lam_h[l], G, DT[dtype])
+        parity.check_decode(od[m], ob, DT[dtype], "full-size decode lambda row %d" % l)
+    # properties that hold at any size: codes in range everywhere, scales finite and non-negative
+    assert bool(torch.isfinite(scales).all()) and bool((scales >= 0).all())
+    lo, hi = packed & 0xF, packed >> 4
+    assert not bool((lo == 8).any()) and not bool((hi == 8).any())  # -8 is never produced
+    assert bool(torch.isfinite(out).all())
+    plan.close()
+
+
+def test_config5_llama70b_shaped_one_layer_k_full_size_sampled():
+    shp = wl.LLAMA3_70B
+    N = shp.kv_heads * shp.batch * shp.prefix  # 1,048,576 vectors: K of one layer
+    _full_size_sampled(128, "f16", N, "k_outlier", 7001, 1, 0)
+
+
+def test_config5_llama70b_shaped_one_layer_v_full_size_sampled():
+    shp = wl.LLAMA3_70B
+    N = shp.kv_heads * shp.batch * shp.prefix
+    _full_size_sampled(128, "f16", N, "gaussian", 7002, 1, 0)
