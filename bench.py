@@ -1,0 +1,376 @@
+#!/usr/bin/env python
+"""Benchmark of the fused int4 KV-cache quantizer hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Workload: BASELINE config 5, the Llama-3-70B-shaped cache (80 layers x 8 KV heads x D=128 fp16,
+batch 4, prefix 32768).  One STEP is one pass of the whole hot path over one layer of that cache:
+
+    kvq_encode   K and V of the layer: 2 x 1,048,576 vectors (bulk prefill encode, one launch)
+    kvq_append   one new vector per (K/V, head, batch) stream: 64 vectors written at the last row
+    kvq_decode   full-prefix read of the layer: 2,097,152 vectors back to fp16 (one launch)
+
+Successive steps rotate over distinct layer slots, so every buffer a kernel touches (0.15 - 0.54 GB)
+is far larger than L2 and was last touched several launches ago.  The 80-layer sweep of the paper-shaped
+model is 80 such steps.  With N > 1 ranks every rank runs its own layers (weak scaling, no collective:
+vectors are independent and (layer, head) sharding needs no exchange).
+
+Prints ONE JSON line.  `value` is algorithmic GB/s over the whole step (encode + append + decode
+bytes / device time); the per-kernel figures, including encode ns/vec and prefix-decode GB/s as a
+fraction of the measured HBM copy peak, are in `detail` and `roofline`.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+D = 128
+GROUP = 32
+BYTES_PER_VEC = 2 * D + D // 2 + 2 * (D // GROUP)   # 328: fp16 row + packed row + fp16 scales
+FALLBACK_HBM_GBS = 6650.0
+METRIC = "kvq_hot_path_algorithmic_GBps"
+UNIT = "GB/s"
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+def workload_shape():
+    from paper_2605_05699_b200 import workloads as wl
+
+    shp = wl.LLAMA3_70B
+    streams = 2 * shp.kv_heads * shp.batch          # K and V streams of one layer: 64
+    return shp, streams, shp.prefix                 # T = 32768 rows per stream
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.proc = None
+        self.idx = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.idx), "--query-gpu=" + self.Q, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons, pw = [], [], set(), []
+        for line in out.splitlines():
+            f = [t.strip() for t in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+                pw.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        busy = [s for s in sm if s > 0.5 * max(sm)] or sm
+        return {"sm_mhz": statistics.median(busy), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm), "power_w_max": max(pw)}
+
+
+# --------------------------------------------------------------------------------------------
+# our arm
+# --------------------------------------------------------------------------------------------
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2605_05699_b200 import binding as kb
+    from paper_2605_05699_b200 import workloads as wl
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the product path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    shp, S, T = workload_shape()
+    N = S * T                                        # 2,097,152 vectors per step
+    n_slots = 3
+    plan = kb.Plan(D, GROUP, 70 + rank)
+    lam = wl.make_lambda(2, D, 71 + rank, device=dev)             # one lambda row for K, one for V
+    slots = []
+    for s in range(n_slots):
+        seed = 5000 + 10 * (rank * n_slots + s)
+        xk = wl.make_vectors(N // 2, D, shp.dtype, "k_outlier", seed, device=dev)
+        xv = wl.make_vectors(N // 2, D, shp.dtype, "gaussian", seed + 1, device=dev)
+        x = torch.cat([xk, xv], 0)
+        del xk, xv
+        slots.append({
+            "x": x,
+            "x_new": wl.make_vectors(S, D, shp.dtype, "gaussian", seed + 2, device=dev),
+            "packed": torch.empty(S, T, D // 2, dtype=torch.uint8, device=dev),
+            "scales": torch.empty(S, T, D // GROUP, dtype=torch.float16, device=dev),
+            "out": torch.empty(N, D, dtype=torch.float16, device=dev),
+        })
+    h = plan.handle
+    rpl = N // 2                                     # rows per lambda row in the flat [N, D] view
+    spl = S // 2                                     # streams per lambda row
+
+    def step(sl, ev=None):
+        if ev:
+            ev[0].record()
+        kb.kvq_encode(h, sl["x"], lam, sl["packed"], sl["scales"], rpl)
+        if ev:
+            ev[1].record()
+        kb.kvq_append(h, sl["x_new"], lam, sl["packed"], sl["scales"], T - 1, spl)
+        if ev:
+            ev[2].record()
+        kb.kvq_decode(h, sl["packed"], sl["scales"], lam, sl["out"], rpl)
+        if ev:
+            ev[3].record()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(slots[i % n_slots])
+    barrier()
+
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    launches0 = kb.kvq_launch_count()
+    barrier()
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for i in range(args.steps):
+        step(slots[(args.warmup + i) % n_slots], evs[i])
+    t1.record()
+    barrier()
+    launches = kb.kvq_launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    ms_total = t0.elapsed_time(t1)
+    if world > 1:
+        tt = torch.tensor([ms_total], device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms_total = float(tt.item())
+    assert kb.kvq_plan_device_status(h) == 0, "a device-side wait timed out"
+
+    enc_ms = [e[0].elapsed_time(e[1]) for e in evs]
+    app_ms = [e[1].elapsed_time(e[2]) for e in evs]
+    dec_ms = [e[2].elapsed_time(e[3]) for e in evs]
+
+    # ---- end to end through the public API with HOST buffers (pinned), copies inside the timed region
+    e2e = None
+    if rank == 0 or world > 1:
+        e2e_steps = max(1, min(args.steps, 4))
+        sl = slots[0]
+        hx = torch.empty(N, D, dtype=torch.float16).pin_memory()
+        hx.copy_(sl["x"])
+        hnew = torch.empty(S, D, dtype=torch.float16).pin_memory()
+        hnew.copy_(sl["x_new"])
+        hout = torch.empty(N, D, dtype=torch.float16).pin_memory()
+
+        def e2e_step():
+            sl["x"].copy_(hx, non_blocking=True)
+            sl["x_new"].copy_(hnew, non_blocking=True)
+            step(sl)
+            hout.copy_(sl["out"], non_blocking=True)
+
+        e2e_step()
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(e2e_steps):
+            e2e_step()
+        b.record()
+        barrier()
+        ms_e2e = a.elapsed_time(b)
+        if world > 1:
+            tt = torch.tensor([ms_e2e], device=dev)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            ms_e2e = float(tt.item())
+        step_bytes = (2 * N + S) * BYTES_PER_VEC
+        e2e = {"value": world * e2e_steps * step_bytes / (ms_e2e * 1e-3) / 1e9, "unit": UNIT,
+               "h2d_bytes_per_step": hx.numel() * 2 + hnew.numel() * 2, "d2h_bytes_per_step": hout.numel() * 2,
+               "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps}
+        del hx, hout
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    step_bytes = (2 * N + S) * BYTES_PER_VEC
+    value = world * args.steps * step_bytes / (ms_total * 1e-3) / 1e9
+    peak, peak_src = measured_peak()
+    dec_avg = sum(dec_ms) / len(dec_ms)
+    enc_avg = sum(enc_ms) / len(enc_ms)
+    dec_gbs = N * BYTES_PER_VEC / (dec_avg * 1e-3) / 1e9
+    enc_gbs = N * BYTES_PER_VEC / (enc_avg * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "kvq_decode (full-prefix read, %d vectors per launch)" % N,
+                "achieved": dec_gbs, "peak": peak, "unit": "GB/s", "frac": dec_gbs / peak,
+                "peak_source": peak_src, "algorithmic_bytes_per_launch": N * BYTES_PER_VEC,
+                "avg_launch_ms": dec_avg, "traffic": TRAFFIC.get("decode")}
+    cpu = cpu_baseline_sample(target_seconds=12.0)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "llama-3-70b-shaped KV cache (config 5): one layer per step = encode 2x1,048,576 "
+                               "vectors + append 64 + full-prefix decode 2,097,152 vectors, D=128 fp16 g=32",
+                   "vectors_per_step": 2 * N + S, "bytes_per_vector": BYTES_PER_VEC, "io_dtype": "f16",
+                   "l2": "every buffer (151-537 MB) exceeds L2; steps rotate over %d layer slots" % n_slots,
+                   "parallelism": "layers sharded over ranks, no collective" if world > 1 else "single GPU"},
+        "detail": {
+            "encode_ns_per_vec": enc_avg * 1e6 / N, "encode_GBps": enc_gbs, "encode_frac_of_hbm_peak": enc_gbs / peak,
+            "decode_ns_per_vec": dec_avg * 1e6 / N, "prefix_decode_GBps": dec_gbs,
+            "prefix_decode_frac_of_hbm_peak": dec_gbs / peak, "prefix_decode_frac_of_8TBps": dec_gbs / 8000.0,
+            "append_us": 1e3 * sum(app_ms) / len(app_ms),
+            "encode_ms_min": min(enc_ms), "decode_ms_min": min(dec_ms),
+            "model_sweep_decode_ms_80_layers": 80 * dec_avg,
+            "paper_context": "paper: 24.6 ns/vec encode at D=128 on an Apple M1 GPU (fp32 in, Sec. 7.1)",
+        },
+        "roofline": roofline,
+        "cpu_baseline": cpu,
+        "e2e": e2e,
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# DRAM bytes per full launch from ncu (dram__bytes_read.sum + dram__bytes_write.sum), filled in from the
+# committed profile summaries under profiles/; None until a capture exists.
+TRAFFIC = {"decode": None, "encode": None}
+
+
+# --------------------------------------------------------------------------------------------
+# the oracle on the host cores: reported baseline and the reference arm
+# --------------------------------------------------------------------------------------------
+
+def _oracle_pass(n, seed):
+    """One pass of the hot path in the oracle on n vectors (K-like half, V-like half): encode, append, decode."""
+    import numpy as np
+
+    from oracle import kvq_oracle as ko
+    from paper_2605_05699_b200 import workloads as wl
+
+    half = n // 2
+    x = np.concatenate([wl.raw_bits(wl.make_vectors(half, D, "f16", "k_outlier", seed)),
+                        wl.raw_bits(wl.make_vectors(n - half, D, "f16", "gaussian", seed + 1))])
+    lam = wl.make_lambda(2, D, seed + 2).numpy()
+    sg = ko.signs(D, 70)
+    xn = wl.raw_bits(wl.make_vectors(64, D, "f16", "gaussian", seed + 3))
+    t0 = time.perf_counter()
+    e = ko.encode(x, ko.F16, sg, lam, GROUP, rows_per_lambda=max(half, 1))
+    pc = e["packed"][:64].reshape(64, 1, D // 2).copy()
+    sc = e["scales"][:64].reshape(64, 1, D // GROUP).copy()
+    ko.append(xn, ko.F16, sg, lam, GROUP, pc, sc, 0, 32)
+    ko.decode(e["packed"], e["scales"], sg, lam, GROUP, ko.F16, rows_per_lambda=max(half, 1))
+    dt = time.perf_counter() - t0
+    return dt, (2 * n + 64) * BYTES_PER_VEC
+
+
+def cpu_baseline_sample(target_seconds=12.0):
+    from oracle import kvq_oracle as ko
+
+    dt, nbytes = _oracle_pass(16384, 900)                      # calibration, also warms the library
+    n = int(max(16384, min(4_000_000, 16384 * target_seconds / max(dt, 1e-3))))
+    dt, nbytes = _oracle_pass(n, 901)
+    return {"value": nbytes / dt / 1e9, "unit": UNIT, "cores": ko.num_threads(), "kind": "oracle",
+            "sample": "%d of the step's 2,097,152 vectors (half K-like, half V-like) + 64 appended: "
+                      "oracle encode + append + decode, fp64 naive DFT, %.1f s" % (n, dt),
+            "ns_per_vec_encode_plus_decode": dt * 1e9 / n}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import kvq_oracle as ko
+
+    dt, _ = _oracle_pass(8192, 800)
+    per_step = 60.0 / max(1, args.steps + args.warmup)          # keep the whole run near a minute
+    n = int(max(8192, min(2_097_152, 8192 * per_step / max(dt, 1e-3))))
+    for i in range(args.warmup):
+        _oracle_pass(n, 810 + i)
+    total_t, total_b = 0.0, 0
+    for i in range(args.steps):
+        t, b = _oracle_pass(n, 820 + i)
+        total_t += t
+        total_b += b
+    value = total_b / total_t / 1e9
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": int(args.gpus),
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total_t / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "llama-3-70b-shaped KV cache (config 5): bounded sample of %d vectors of the "
+                               "step's 2,097,152 per step, D=128 fp16 g=32" % n},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": ko.num_threads(), "kind": "oracle",
+                         "sample": "%d vectors per step, encode + append + decode" % n},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

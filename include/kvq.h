@@ -103,7 +103,7 @@ kvq_status_t kvq_plan_device_status(kvq_plan_t *plan, uint32_t *word);
  *   packed   device out, [N, D/2] bytes, byte i of a row = (q[2i+1] << 4) | (q[2i] & 0xF);
  *            16-byte aligned.
  *   scales   device out, [N, D/group] fp16; 16-byte aligned.
- * N == 0 is a no-op.  Errors: INVALID_ARG, ALIGNMENT, UNSUPPORTED_DIM, CUDA.
+ * N == 0 is a no-op that returns KVQ_OK without looking at the data pointers.  Errors: INVALID_ARG, ALIGNMENT, UNSUPPORTED_DIM, CUDA.
  */
 kvq_status_t kvq_encode(kvq_plan_t *plan, const void *x, kvq_dtype_t dtype, int64_t N,
                         const float *lambda, int64_t n_lambda, int64_t rows_per_lambda,

@@ -194,12 +194,12 @@ static kvq_status_t encode_common(kvq_plan_t *plan, const void *x, kvq_dtype_t d
 {
     if (!plan || N < 0) return KVQ_ERR_INVALID_ARG;
     if (dtype != KVQ_F16 && dtype != KVQ_BF16) return KVQ_ERR_INVALID_ARG;
+    if (N == 0) return KVQ_OK;   // nothing to do; empty buffers may be null
     if (!x || !packed || !scales) return KVQ_ERR_INVALID_ARG;
     kvq_status_t st = check_lambda(N, lambda, n_lambda, rows_per_lambda);
     if (st != KVQ_OK) return st;
     if (misaligned16(x) || misaligned16(packed) || misaligned16(scales)) return KVQ_ERR_ALIGNMENT;
     if (plan->enc_impl == KVQ_IMPL_GEMM) return KVQ_ERR_UNSUPPORTED_DIM;
-    if (N == 0) return KVQ_OK;
     if ((st = ensure_device(plan)) != KVQ_OK) return st;
     FftParams prm;
     fill_params(plan, prm, N, lambda, n_lambda, rows_per_lambda);
@@ -236,12 +236,12 @@ kvq_status_t kvq_decode(kvq_plan_t *plan, const uint8_t *packed, const void *sca
 {
     if (!plan || N < 0) return KVQ_ERR_INVALID_ARG;
     if (dtype != KVQ_F16 && dtype != KVQ_BF16) return KVQ_ERR_INVALID_ARG;
+    if (N == 0) return KVQ_OK;   // nothing to do; empty buffers may be null
     if (!packed || !scales || !out) return KVQ_ERR_INVALID_ARG;
     kvq_status_t st = check_lambda(N, lambda, n_lambda, rows_per_lambda);
     if (st != KVQ_OK) return st;
     if (misaligned16(packed) || misaligned16(scales) || misaligned16(out)) return KVQ_ERR_ALIGNMENT;
     if (plan->dec_impl == KVQ_IMPL_GEMM) return KVQ_ERR_UNSUPPORTED_DIM;
-    if (N == 0) return KVQ_OK;
     if ((st = ensure_device(plan)) != KVQ_OK) return st;
     FftParams prm;
     fill_params(plan, prm, N, lambda, n_lambda, rows_per_lambda);
