@@ -298,6 +298,7 @@ def _oracle_pass(n, seed):
     from oracle import kvq_oracle as ko
     from paper_2605_05699_b200 import workloads as wl
 
+    n -= n % 2
     half = n // 2
     x = np.concatenate([wl.raw_bits(wl.make_vectors(half, D, "f16", "k_outlier", seed)),
                         wl.raw_bits(wl.make_vectors(n - half, D, "f16", "gaussian", seed + 1))])

@@ -49,11 +49,11 @@ def run_case(D, dtype, N, kind, seed, n_lambda=1, rows_per_lambda=0, plan_seed=N
     label = "D=%d %s N=%d" % (D, dtype, N)
     enc = parity.check_encode(packed.cpu().numpy(), bits(scales), ora, G, label + " encode")
     # decode parity on the oracle's own compressed representation
-    ob = ko.decode(ora["packed"], ora["scales"], sg, lam.numpy(), G, DT[dtype], rows_per_lambda)
+    ob, o64 = ko.decode(ora["packed"], ora["scales"], sg, lam.numpy(), G, DT[dtype], rows_per_lambda, want_f64=True)
     pk_o = torch.from_numpy(ora["packed"]).cuda()
     sc_o = torch.from_numpy(ora["scales"].view(np.int16)).view(torch.float16).cuda()
     out = gpu_decode(plan, pk_o, sc_o, lamd, dtype, rows_per_lambda)
-    dec = parity.check_decode(bits(out), ob, DT[dtype], label + " decode")
+    dec = parity.check_decode(bits(out), ob, o64, DT[dtype], label + " decode")
     # GPU round trip stays close to the input (4-bit noise level, sanity only)
     rt = gpu_decode(plan, packed, scales, lamd, dtype, rows_per_lambda).float().cpu().numpy()
     xin = x.float().numpy()
@@ -138,9 +138,9 @@ def test_config2_qwen_shaped_prefill_append_decode():
     parity.check_encode(packed.view(-1, D // 2).cpu().numpy(), bits(scales.view(-1, D // G)), ora, G, "qwen cache")
     # full-prefix decode of the whole cache in one launch
     out = gpu_decode(plan, packed.view(-1, D // 2), scales.view(-1, D // G), lamd, shp.dtype, per_lambda * T_max)
-    ob = ko.decode(packed.view(-1, D // 2).cpu().numpy(), bits(scales.view(-1, D // G)), sg, lam.numpy(), G, ko.F16,
-                   per_lambda * T_max)
-    parity.check_decode(bits(out), ob, ko.F16, "qwen full-prefix decode")
+    ob, o64 = ko.decode(packed.view(-1, D // 2).cpu().numpy(), bits(scales.view(-1, D // G)), sg, lam.numpy(), G,
+                        ko.F16, per_lambda * T_max, want_f64=True)
+    parity.check_decode(bits(out), ob, o64, ko.F16, "qwen full-prefix decode")
     plan.close()
 
 
@@ -196,8 +196,8 @@ def _full_size_sampled(D, dtype, N, kind, seed, n_lambda, rows_per_lambda, n_ran
         m = lrow == l
         ora = ko.encode(bits(xs)[m], DT[dtype], sg, lam_h[l], G, want_v=True)
         parity.check_encode(pk[m], sc[m], ora, G, "full-size encode lambda row %d" % l)
-        ob = ko.decode(pk[m], sc[m], sg, lam_h[l], G, DT[dtype])
-        parity.check_decode(od[m], ob, DT[dtype], "full-size decode lambda row %d" % l)
+        ob, o64 = ko.decode(pk[m], sc[m], sg, lam_h[l], G, DT[dtype], want_f64=True)
+        parity.check_decode(od[m], ob, o64, DT[dtype], "full-size decode lambda row %d" % l)
     # properties that hold at any size: codes in range everywhere, scales finite and non-negative
     assert bool(torch.isfinite(scales).all()) and bool((scales >= 0).all())
     lo, hi = packed & 0xF, packed >> 4
