@@ -1,5 +1,6 @@
 // C ABI of libkvq (see include/kvq.h): plan object, host-side validation, dispatch.
 #include <atomic>
+#include <cmath>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -48,8 +49,28 @@ struct kvq_plan {
     std::mutex mu;
     int device;            // -1 until initialised
     uint32_t *d_status;    // device status word
+    float *d_b0;           // [D, D] fp32 inverse-transform matrix with the signs folded in (GEMM decode), or null
     size_t table_bytes;
 };
+
+// b0[n][c] = s_n M[c][n] with z = M (s (.) x) the transform of Eq. 1-2: row c of M is
+//   D^-1/2                       (c = 0),        (-1)^n D^-1/2               (c = D/2),
+//   sqrt(2/D) cos(2 pi c n / D)  (0 < c < D/2),  -sqrt(2/D) sin(2 pi k n / D) (c = D/2 + k, 0 < k < D/2).
+// M is orthogonal, so the inverse transform is x^_n = s_n sum_c M[c][n] z^_c.
+static void build_b0(const kvq_plan *p, float *b0)
+{
+    const int D = p->D, H = D / 2;
+    const double pi = 3.14159265358979323846;
+    for (int n = 0; n < D; ++n)
+        for (int c = 0; c < D; ++c) {
+            double m;
+            if (c == 0) m = 1.0 / std::sqrt((double)D);
+            else if (c == H) m = ((n & 1) ? -1.0 : 1.0) / std::sqrt((double)D);
+            else if (c < H) m = std::sqrt(2.0 / D) * std::cos(2.0 * pi * (double)((long)c * n % D) / D);
+            else m = -std::sqrt(2.0 / D) * std::sin(2.0 * pi * (double)((long)(c - H) * n % D) / D);
+            b0[(size_t)n * D + c] = (float)(p->signs[n] * m);
+        }
+}
 
 using namespace kvq;
 
@@ -75,6 +96,30 @@ static kvq_status_t ensure_device(kvq_plan *p)
     }
     p->d_status = st;
     p->table_bytes = 256;
+    if (p->D == 128) {   // the GEMM decode kernel exists for D = 128
+        const size_t bytes = sizeof(float) * (size_t)p->D * p->D;
+        float *host = new (std::nothrow) float[(size_t)p->D * p->D];
+        float *devp = nullptr;
+        if (!host || cudaMalloc(&devp, bytes) != cudaSuccess) {
+            (void)cudaGetLastError();
+            delete[] host;
+            cudaFree(st);
+            p->d_status = nullptr;
+            return KVQ_ERR_NOMEM;
+        }
+        build_b0(p, host);
+        cudaError_t e = cudaMemcpy(devp, host, bytes, cudaMemcpyHostToDevice);
+        delete[] host;
+        if (e != cudaSuccess) {
+            (void)cudaGetLastError();
+            cudaFree(devp);
+            cudaFree(st);
+            p->d_status = nullptr;
+            return KVQ_ERR_CUDA;
+        }
+        p->d_b0 = devp;
+        p->table_bytes += bytes;
+    }
     p->device = dev;
     return KVQ_OK;
 }
@@ -121,6 +166,7 @@ kvq_status_t kvq_plan_create(int D, int group, uint64_t seed, kvq_plan_t **out)
     p->enc_impl = p->dec_impl = KVQ_IMPL_AUTO;
     p->device = -1;
     p->d_status = nullptr;
+    p->d_b0 = nullptr;
     p->table_bytes = 0;
     std::memset(p->signs, 0, sizeof(p->signs));
     std::memset(p->sign_xor, 0, sizeof(p->sign_xor));
@@ -138,6 +184,9 @@ kvq_status_t kvq_plan_destroy(kvq_plan_t *plan)
     if (!plan) return KVQ_OK;
     if (plan->d_status) {
         if (cudaFree(plan->d_status) != cudaSuccess) (void)cudaGetLastError();
+    }
+    if (plan->d_b0) {
+        if (cudaFree(plan->d_b0) != cudaSuccess) (void)cudaGetLastError();
     }
     delete plan;
     return KVQ_OK;
@@ -241,8 +290,26 @@ kvq_status_t kvq_decode(kvq_plan_t *plan, const uint8_t *packed, const void *sca
     kvq_status_t st = check_lambda(N, lambda, n_lambda, rows_per_lambda);
     if (st != KVQ_OK) return st;
     if (misaligned16(packed) || misaligned16(scales) || misaligned16(out)) return KVQ_ERR_ALIGNMENT;
-    if (plan->dec_impl == KVQ_IMPL_GEMM) return KVQ_ERR_UNSUPPORTED_DIM;
+    const bool gemm_ok = plan->D == 128 && dtype == KVQ_F16;
+    if (plan->dec_impl == KVQ_IMPL_GEMM && !gemm_ok) return KVQ_ERR_UNSUPPORTED_DIM;
     if ((st = ensure_device(plan)) != KVQ_OK) return st;
+    if (gemm_ok && plan->dec_impl != KVQ_IMPL_FFT) {
+        GemmParams g;
+        g.packed = packed;
+        g.scales = scales;
+        g.lambda = lambda;
+        g.out = out;
+        g.b0 = plan->d_b0;
+        g.N = N;
+        g.n_lambda = n_lambda;
+        g.rows_per_lambda = rows_per_lambda < 1 ? 1 : rows_per_lambda;
+        g.status = plan->d_status;
+        if (gemm_decode_d128(N, g, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return KVQ_ERR_CUDA;
+        }
+        return KVQ_OK;
+    }
     FftParams prm;
     fill_params(plan, prm, N, lambda, n_lambda, rows_per_lambda);
     prm.packed = const_cast<uint8_t *>(packed);

@@ -21,6 +21,20 @@ struct FftParams {
     uint32_t sign_xor[128];     // word m: bit 15 set if s_{2m} = -1, bit 31 set if s_{2m+1} = -1
 };
 
+// Arguments of the tcgen05 DFT-as-GEMM decode kernel.
+struct GemmParams {
+    const void *packed;    // [N, D/2] bytes
+    const void *scales;    // [N, D/group] fp16
+    const float *lambda;   // [n_lambda, D] fp32
+    void *out;             // [N, D] fp16
+    const float *b0;       // plan table [D, D] fp32: b0[n][c] = s_n M[c][n], M the real orthogonal DFT matrix of Eq. 1-2
+    int64_t N;
+    int64_t n_lambda, rows_per_lambda;
+    uint32_t *status;
+};
+
+cudaError_t gemm_decode_d128(int64_t N, const GemmParams &prm, cudaStream_t stream);
+
 cudaError_t fft_encode(int D, bool bf16, int64_t N, const FftParams &prm, cudaStream_t stream);
 cudaError_t fft_decode(int D, bool bf16, int64_t N, const FftParams &prm, cudaStream_t stream);
 

@@ -36,9 +36,13 @@ def gpu_decode(plan, packed, scales, lam, dtype, rows_per_lambda=0):
     return out
 
 
-def run_case(D, dtype, N, kind, seed, n_lambda=1, rows_per_lambda=0, plan_seed=None):
+IMPL = {"auto": kb.KVQ_IMPL_AUTO, "fft": kb.KVQ_IMPL_FFT, "gemm": kb.KVQ_IMPL_GEMM}
+
+
+def run_case(D, dtype, N, kind, seed, n_lambda=1, rows_per_lambda=0, plan_seed=None, enc_impl="auto", dec_impl="auto"):
     """Encode on GPU vs oracle; decode the ORACLE's compressed data on GPU vs oracle; GPU round trip."""
     plan = kb.Plan(D, G, seed if plan_seed is None else plan_seed)
+    kb.kvq_plan_set_impl(plan.handle, IMPL[enc_impl], IMPL[dec_impl])
     sg = plan.signs()
     assert np.array_equal(sg, ko.signs(D, plan.seed))  # two independent implementations of the sign stream
     x = wl.make_vectors(N, D, dtype, kind, seed)
@@ -68,6 +72,47 @@ def run_case(D, dtype, N, kind, seed, n_lambda=1, rows_per_lambda=0, plan_seed=N
 def test_config1_single_tensor_d128_f16():
     enc, dec = run_case(128, "f16", 4096, "c1", 1001)
     assert enc["mismatches"] <= 52  # 99.99 % of 524288 codes
+
+
+# ---- both decode kernel families at D = 128 fp16: the fp32 register FFT and the tcgen05 DFT-as-GEMM
+
+@pytest.mark.parametrize("dec_impl", ["fft", "gemm"])
+@pytest.mark.parametrize("N,n_lambda,rpl,kind", [(4096, 1, 0, "c1"), (1000, 4, 333, "k_outlier"), (1, 1, 0, "gaussian"),
+                                                 (129, 1, 0, "gaussian"), (70000, 7, 10000, "k_outlier")])
+def test_decode_kernel_families_d128_f16(dec_impl, N, n_lambda, rpl, kind):
+    enc, dec = run_case(128, "f16", N, kind, 8000 + N, n_lambda=n_lambda, rows_per_lambda=rpl, dec_impl=dec_impl)
+    if dec_impl == "fft":
+        assert dec["rel_l2_plain_max"] < 1e-3  # fp32 arithmetic: far inside the tolerance even without the tie rule
+
+
+def test_gemm_decode_is_refused_where_it_is_not_built():
+    for D, dtype in [(256, torch.float16), (128, torch.bfloat16), (96, torch.float16)]:
+        plan = kb.Plan(D, G, 1)
+        kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_AUTO, kb.KVQ_IMPL_GEMM)
+        pk, sc = plan.empty_packed(8), plan.empty_scales(8)
+        out = torch.empty(8, D, dtype=dtype, device="cuda")
+        with pytest.raises(kb.KvqError) as e:
+            kb.kvq_decode(plan.handle, pk, sc, torch.ones(D, device="cuda"), out)
+        assert e.value.status == kb.KVQ_ERR_UNSUPPORTED_DIM
+        plan.close()
+
+
+def test_lambda_scale_does_not_matter_to_the_gemm_decode():
+    # lambda rows far from 1 (all channels x 2^-12 or x 2^9): the power-of-two normalisation keeps fp16 operands in range
+    for shift in (-12, 9):
+        D, N = 128, 2048
+        plan = kb.Plan(D, G, 31)
+        kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_FFT, kb.KVQ_IMPL_GEMM)
+        sg = plan.signs()
+        x = wl.make_vectors(N, D, "f16", "k_outlier", 77)
+        lam = wl.make_lambda(1, D, 78) * (2.0 ** shift)
+        ora = ko.encode(bits(x), ko.F16, sg, lam.numpy(), G, want_v=True)
+        ob, o64 = ko.decode(ora["packed"], ora["scales"], sg, lam.numpy(), G, ko.F16, want_f64=True)
+        pk = torch.from_numpy(ora["packed"]).cuda()
+        sc = torch.from_numpy(ora["scales"].view(np.int16)).view(torch.float16).cuda()
+        out = gpu_decode(plan, pk, sc, lam.cuda(), "f16")
+        parity.check_decode(bits(out), ob, o64, ko.F16, "gemm decode, lambda x 2^%d" % shift)
+        plan.close()
 
 
 # ---- every head dim and dtype, ragged N (several tiles plus a tail), lambda rows that straddle tiles
@@ -178,8 +223,9 @@ def test_config3_gemma_shaped_prefix_4096_sampled():
 
 # ---- config 5: Llama-3-70B-shaped: one layer's K (1,048,576 vectors) per launch, sampled rows -
 
-def _full_size_sampled(D, dtype, N, kind, seed, n_lambda, rows_per_lambda, n_random=4096):
+def _full_size_sampled(D, dtype, N, kind, seed, n_lambda, rows_per_lambda, n_random=4096, dec_impl="auto"):
     plan = kb.Plan(D, G, seed)
+    kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_AUTO, IMPL[dec_impl])
     sg = plan.signs()
     x = wl.make_vectors(N, D, dtype, kind, seed, device="cuda")
     lam = wl.make_lambda(n_lambda, D, seed + 1, device="cuda")
@@ -206,13 +252,15 @@ def _full_size_sampled(D, dtype, N, kind, seed, n_lambda, rows_per_lambda, n_ran
     plan.close()
 
 
-def test_config5_llama70b_shaped_one_layer_k_full_size_sampled():
+@pytest.mark.parametrize("dec_impl", ["fft", "gemm"])
+def test_config5_llama70b_shaped_one_layer_full_size_sampled(dec_impl):
+    # the launch configuration bench.py times: K and V of one layer in one call, 2 x 1,048,576 vectors, two lambda rows
     shp = wl.LLAMA3_70B
-    N = shp.kv_heads * shp.batch * shp.prefix  # 1,048,576 vectors: K of one layer
-    _full_size_sampled(128, "f16", N, "k_outlier", 7001, 1, 0)
+    half = shp.kv_heads * shp.batch * shp.prefix
+    _full_size_sampled(128, "f16", 2 * half, "k_outlier", 7001, 2, half, dec_impl=dec_impl)
 
 
-def test_config5_llama70b_shaped_one_layer_v_full_size_sampled():
+def test_config5_llama70b_shaped_v_like_full_size_sampled():
     shp = wl.LLAMA3_70B
     N = shp.kv_heads * shp.batch * shp.prefix
     _full_size_sampled(128, "f16", N, "gaussian", 7002, 1, 0)
