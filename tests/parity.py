@@ -86,30 +86,36 @@ def check_decode(gpu_bits, ora_bits, ora_f64, dtype, label=""):
     """gpu_bits / ora_bits: raw uint16 bits of the half-precision outputs [N, D]; ora_f64: the oracle's
     reconstruction before its rounding to the output dtype.
 
-    The 16-bit output format decides a rounding, like the quantizer decides a code: two correct results can
-    differ by one output ulp on an element whose exact value sits at a rounding midpoint (for bfloat16 one
-    such flip on a dominant channel is already 4e-3 of the vector norm).  Such elements are excused when the
-    two outputs are neighbours in the format and the exact value lies within 1e-3 of the vector's rms from
-    their midpoint; everything else must agree within 1e-3 relative L2 per vector.
+    A vector passes if its relative L2 distance to the oracle's rounded output is <= 1e-3.  The 16-bit
+    output format decides a rounding, like the quantizer decides a code: two correct results can differ
+    by one output ulp on an element whose exact value sits at a rounding midpoint, and for bfloat16 one
+    such flip on a dominant channel is already 4e-3 of the vector norm.  A vector that fails the plain
+    comparison is therefore compared again without the elements where the two outputs are neighbours in
+    the format and the exact value lies within 1e-3 of the vector's rms from their midpoint; it must
+    then pass, and such vectors must be rare.
     """
     gb = np.ascontiguousarray(gpu_bits).view(np.uint16)
     g = ko.widen(gb, dtype)
     o = ko.widen(ora_bits, dtype)
     assert np.isfinite(g).all(), label + ": non-finite output"
     D = g.shape[1]
-    rms = np.linalg.norm(ora_f64, axis=1, keepdims=True) / np.sqrt(D)
-    differ = gb != ora_bits
-    # neighbours in the format: sign-magnitude bit patterns one apart (or +-0)
-    key = lambda b: np.where(b & 0x8000, -(b & 0x7FFF).astype(np.int64), (b & 0x7FFF).astype(np.int64))
-    adjacent = np.abs(key(gb) - key(ora_bits)) <= 1
-    at_tie = differ & adjacent & (np.abs(ora_f64 - (g + o) / 2) <= REL_L2 * rms)
-    diff = np.where(at_tie, 0.0, g - o)
-    den = np.linalg.norm(o, axis=1)
-    rel = np.linalg.norm(diff, axis=1) / np.where(den > 0, den, 1.0)
-    assert rel.max(initial=0) <= REL_L2, label + ": reconstruction relative L2 %.3g" % rel.max()
-    excused = float(at_tie.mean()) if g.size else 0.0
-    assert excused < 0.02, label + ": %.3g of the outputs sit at a rounding tie" % excused
     plain = rel_l2_rows(g, o)
-    return {"rel_l2_max": float(rel.max(initial=0)), "rel_l2_plain_max": float(plain.max(initial=0)),
-            "rel_l2_plain_mean": float(plain.mean()) if plain.size else 0.0, "excused_at_output_ties": excused,
-            "bit_equal": float((~differ).mean()) if g.size else 1.0}
+    need = plain > REL_L2
+    worst = float(plain[~need].max(initial=0))
+    if need.any():
+        gg, oo, x64 = g[need], o[need], ora_f64[need]
+        rms = np.linalg.norm(x64, axis=1, keepdims=True) / np.sqrt(D)
+        # neighbours in the format: sign-magnitude bit patterns one apart (or +-0)
+        key = lambda b: np.where(b & 0x8000, -(b & 0x7FFF).astype(np.int64), (b & 0x7FFF).astype(np.int64))
+        adjacent = np.abs(key(gb[need]) - key(ora_bits[need])) == 1
+        at_tie = adjacent & (np.abs(x64 - (gg + oo) / 2) <= REL_L2 * rms)
+        diff = np.where(at_tie, 0.0, gg - oo)
+        den = np.linalg.norm(oo, axis=1)
+        rel = np.linalg.norm(diff, axis=1) / np.where(den > 0, den, 1.0)
+        assert rel.max() <= REL_L2, label + ": reconstruction relative L2 %.3g (plain %.3g)" % (rel.max(), plain.max())
+        worst = max(worst, float(rel.max()))
+    frac = float(need.mean()) if need.size else 0.0
+    assert frac < 0.05, label + ": %.3g of the vectors pass only with the output-tie rule" % frac
+    return {"rel_l2_max": worst, "rel_l2_plain_max": float(plain.max(initial=0)),
+            "rel_l2_plain_mean": float(plain.mean()) if plain.size else 0.0, "rows_needing_tie_rule": frac,
+            "bit_equal": float((gb == ora_bits).mean()) if g.size else 1.0}
