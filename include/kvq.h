@@ -45,7 +45,8 @@ typedef enum {
     KVQ_ERR_ALIGNMENT = 3,       /* a base pointer is not 16-byte aligned */
     KVQ_ERR_CUDA = 4,            /* a CUDA runtime call failed (no device, launch error ...) */
     KVQ_ERR_TIMEOUT = 5,         /* a bounded device-side wait ran out (see kvq_plan_device_status) */
-    KVQ_ERR_NOMEM = 6
+    KVQ_ERR_NOMEM = 6,
+    KVQ_ERR_SCRATCH_LIMIT = 7    /* the plan needs more fixed scratch than kvq_decode_static holds */
 } kvq_status_t;
 
 typedef enum { KVQ_F16 = 0, KVQ_BF16 = 1 } kvq_dtype_t;
@@ -131,6 +132,36 @@ kvq_status_t kvq_append(kvq_plan_t *plan, const void *x_new /* [S, D] */, kvq_dt
                         const float *lambda, int64_t n_lambda, int64_t streams_per_lambda,
                         uint8_t *packed_cache, void *scales_cache, int64_t T_max, int64_t pos,
                         void *cuda_stream);
+
+/*
+ * kvq_decode_static -- kvq_decode for callers that may not allocate device memory.  (The paper has
+ * no counterpart: this entry point exists for how the library is embedded, not for the method.)
+ *
+ * kvq_decode calls cudaMalloc the first time a plan is used on a device (a status word, and the
+ * [D, D] fp32 table of the tensor-core kernel).  A server that gave all of HBM to its own pool, a
+ * decode loop that cannot take cudaMalloc's device-wide synchronisation, or a plug-in restricted to
+ * the buffers it was handed cannot make that call.  This variant runs the same tensor-core kernel
+ * with those two objects in a fixed 65,792-byte block that is part of the library image (every GPU
+ * context that loads the library holds it until the process exits).  It calls no cudaMalloc,
+ * cudaFree or other allocating routine, on any call.
+ *
+ *   plan         D = 128 only; a plan with D > 128 is refused with KVQ_ERR_SCRATCH_LIMIT (its table
+ *                does not fit the block), smaller D and bf16 output with KVQ_ERR_UNSUPPORTED_DIM.
+ *   packed, scales, N, lambda, n_lambda, rows_per_lambda, out, cuda_stream: as in kvq_decode;
+ *                dtype must be KVQ_F16.
+ *   status_word  optional DEVICE pointer (4-byte aligned) to a word the caller owns: cleared on the
+ *                stream, then non-zero if a bounded device-side wait ran out.  NULL keeps the word
+ *                inside the block, where this library version does not expose it.
+ *
+ * The first call on a device looks up the block's device address; make that call before any
+ * stream capture begins.  The block is shared: it keeps the last call's table, which belongs to
+ * one plan, and a call with a different plan rewrites it on the caller's stream before decoding.
+ * Calls that can overlap on the GPU (different streams, no ordering between them) race on the
+ * block and on the table: order them, or use kvq_decode.
+ */
+kvq_status_t kvq_decode_static(kvq_plan_t *plan, const uint8_t *packed, const void *scales, int64_t N,
+                               const float *lambda, int64_t n_lambda, int64_t rows_per_lambda,
+                               void *out, kvq_dtype_t dtype, uint32_t *status_word, void *cuda_stream);
 
 /* Static, human-readable name of a status code. */
 const char *kvq_status_string(kvq_status_t status);

@@ -25,6 +25,7 @@ KVQ_ERR_ALIGNMENT = 3
 KVQ_ERR_CUDA = 4
 KVQ_ERR_TIMEOUT = 5
 KVQ_ERR_NOMEM = 6
+KVQ_ERR_SCRATCH_LIMIT = 7
 
 KVQ_F16 = 0
 KVQ_BF16 = 1
@@ -36,7 +37,8 @@ KVQ_IMPL_GEMM = 2
 # every symbol include/kvq.h declares
 EXPORTS = (
     "kvq_plan_create", "kvq_plan_destroy", "kvq_plan_get_signs", "kvq_plan_describe", "kvq_plan_set_impl",
-    "kvq_plan_device_status", "kvq_encode", "kvq_decode", "kvq_append", "kvq_status_string", "kvq_launch_count",
+    "kvq_plan_device_status", "kvq_encode", "kvq_decode", "kvq_append", "kvq_decode_static", "kvq_status_string",
+    "kvq_launch_count",
 )
 
 _lib = None
@@ -75,6 +77,8 @@ def lib() -> ctypes.CDLL:
         L.kvq_decode.argtypes = [vp, vp, vp, i64, vp, i64, i64, vp, i32, vp]
         L.kvq_append.restype = i32
         L.kvq_append.argtypes = [vp, vp, i32, i64, vp, i64, i64, vp, vp, i64, i64, vp]
+        L.kvq_decode_static.restype = i32
+        L.kvq_decode_static.argtypes = [vp, vp, vp, i64, vp, i64, i64, vp, i32, vp, vp]
         L.kvq_status_string.restype = ctypes.c_char_p
         L.kvq_status_string.argtypes = [i32]
         L.kvq_launch_count.restype = u64
@@ -191,6 +195,24 @@ def kvq_append(plan: int, x_new: torch.Tensor, lam: torch.Tensor, packed_cache: 
                                 streams_per_lambda, _dev(packed_cache, "packed_cache"),
                                 _dev(scales_cache, "scales_cache"), T_max, pos, _stream(stream)),
                "kvq_append")
+
+
+def kvq_decode_static(plan: int, packed: torch.Tensor, scales: torch.Tensor, lam: torch.Tensor, out: torch.Tensor,
+                      rows_per_lambda: int = 0, status_word: torch.Tensor | None = None, stream=None) -> None:
+    """kvq_decode without any device allocation inside the library (D = 128, fp16 output only).
+
+    For embedders that own all device memory themselves or cannot take an allocation in their decode
+    loop: the kernel's table and status word live in a fixed block inside the library.  Calls must not
+    overlap on the GPU; ``status_word`` is an optional int32 device tensor of one element."""
+    D = out.shape[-1]
+    N = out.numel() // D
+    n_lambda = lam.numel() // D
+    sw = None if status_word is None else _dev(status_word, "status_word")
+    with torch.cuda.device(out.device):
+        _check(lib().kvq_decode_static(plan, _dev(packed, "packed"), _dev(scales, "scales"), N, _dev(lam, "lambda"),
+                                       n_lambda, rows_per_lambda, _dev(out, "out"), _dtype_code(out), sw,
+                                       _stream(stream)),
+               "kvq_decode_static")
 
 
 class Plan:

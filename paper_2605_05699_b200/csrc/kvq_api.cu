@@ -39,20 +39,6 @@ static int radix_plan(int n, int *out)
 
 }  // namespace kvq
 
-struct kvq_plan {
-    int D, group;
-    uint64_t seed;
-    int8_t signs[256];
-    uint32_t sign_xor[128];
-    kvq_impl_t enc_impl, dec_impl;
-    // device state, created on first use
-    std::mutex mu;
-    int device;            // -1 until initialised
-    uint32_t *d_status;    // device status word
-    float *d_b0;           // [D, D] fp32 inverse-transform matrix with the signs folded in (GEMM decode), or null
-    size_t table_bytes;
-};
-
 // b0[n][c] = s_n M[c][n] with z = M (s (.) x) the transform of Eq. 1-2: row c of M is
 //   D^-1/2                       (c = 0),        (-1)^n D^-1/2               (c = D/2),
 //   sqrt(2/D) cos(2 pi c n / D)  (0 < c < D/2),  -sqrt(2/D) sin(2 pi k n / D) (c = D/2 + k, 0 < k < D/2).
@@ -333,6 +319,7 @@ const char *kvq_status_string(kvq_status_t status)
         case KVQ_ERR_CUDA: return "KVQ_ERR_CUDA";
         case KVQ_ERR_TIMEOUT: return "KVQ_ERR_TIMEOUT";
         case KVQ_ERR_NOMEM: return "KVQ_ERR_NOMEM";
+        case KVQ_ERR_SCRATCH_LIMIT: return "KVQ_ERR_SCRATCH_LIMIT";
     }
     return "KVQ_ERR_UNKNOWN";
 }

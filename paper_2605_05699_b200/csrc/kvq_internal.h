@@ -4,6 +4,10 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
+#include "../../include/kvq.h"
+
 namespace kvq {
 
 // Arguments of the register-FFT kernels.  Passed by value as a __grid_constant__
@@ -41,3 +45,18 @@ cudaError_t fft_decode(int D, bool bf16, int64_t N, const FftParams &prm, cudaSt
 void count_launch();
 
 }  // namespace kvq
+
+// The plan behind the opaque kvq_plan_t handle.
+struct kvq_plan {
+    int D, group;
+    uint64_t seed;
+    int8_t signs[256];
+    uint32_t sign_xor[128];
+    kvq_impl_t enc_impl, dec_impl;
+    // device state, created on first use
+    std::mutex mu;
+    int device;            // -1 until initialised
+    uint32_t *d_status;    // device status word
+    float *d_b0;           // [D, D] fp32 inverse-transform matrix with the signs folded in (GEMM decode), or null
+    size_t table_bytes;
+};
