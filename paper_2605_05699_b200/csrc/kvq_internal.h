@@ -38,6 +38,7 @@ struct GemmParams {
 };
 
 cudaError_t gemm_decode_d128(int64_t N, const GemmParams &prm, cudaStream_t stream);
+cudaError_t umma_decode_d128(int64_t N, const GemmParams &prm, cudaStream_t stream);
 
 cudaError_t fft_encode(int D, bool bf16, int64_t N, const FftParams &prm, cudaStream_t stream);
 cudaError_t fft_decode(int D, bool bf16, int64_t N, const FftParams &prm, cudaStream_t stream);
