@@ -25,7 +25,7 @@ struct FftParams {
     uint32_t sign_xor[128];     // word m: bit 15 set if s_{2m} = -1, bit 31 set if s_{2m+1} = -1
 };
 
-// Arguments of the tcgen05 DFT-as-GEMM decode kernel.
+// Arguments of the tcgen05 DFT-as-GEMM decode kernel (kvq_umma_decode.cu).
 struct GemmParams {
     const void *packed;    // [N, D/2] bytes
     const void *scales;    // [N, D/group] fp16
@@ -37,7 +37,6 @@ struct GemmParams {
     uint32_t *status;
 };
 
-cudaError_t gemm_decode_d128(int64_t N, const GemmParams &prm, cudaStream_t stream);
 cudaError_t umma_decode_d128(int64_t N, const GemmParams &prm, cudaStream_t stream);
 
 cudaError_t fft_encode(int D, bool bf16, int64_t N, const FftParams &prm, cudaStream_t stream);

@@ -6,20 +6,22 @@
 // to cross HBM, so the kernel's job is to keep HBM busy: one persistent CTA per SM runs four roles that
 // hand tiles to one another through mbarriers and never wait for one another's latency.
 //
-//   warp 0       producer   one TMA tensor load per tile: 128 packed rows (8 KB) into a ring of
-//                           shared-memory stages (64-byte swizzle, so that row-per-thread reads
-//                           are free of bank conflicts)
-//   warps 2-5    dequant    thread t owns row t: nibbles -> fp16 codes -> times sigma * rho, two codes per
-//                           half2 instruction, stored straight into TENSOR MEMORY as the A
-//                           operand (tcgen05.st); the group scales come by plain loads, two tiles
-//                           ahead.  These warps also rebuild the B operand when the lambda row changes.
-//   warp 1       mma        one thread issues 8 K-steps of tcgen05.mma (A from tensor memory, B from
-//                           shared memory) into one of two accumulator stages and commits
-//   warps 6-9    epilogue   thread t reads accumulator row t (tcgen05.ld), rounds to fp16, writes a
-//                           128-byte-swizzled staging tile; one lane per warp issues two TMA tensor
-//                           stores (32 rows x 128 B each).  The output tensor map is three-dimensional
-//                           (column, row within lambda segment, segment), so the hardware clips a tile
-//                           that ends with its segment or with the tensor: no per-row tail code.
+//   warp 0        producer   one TMA tensor load per tile: 128 packed rows (8 KB) into a ring of
+//                            shared-memory stages (64-byte swizzle, so that row-per-thread reads
+//                            are free of bank conflicts)
+//   warps 2-9     dequant    two groups of four warps that take alternate tiles.  Thread t of a group
+//                            owns row t: nibbles -> fp16 codes -> times sigma * rho, two codes per
+//                            half2 instruction, stored straight into TENSOR MEMORY as the A operand
+//                            (tcgen05.st); the group scales come by plain loads, one tile ahead.
+//                            The group that meets the first tile of a new lambda row rebuilds B.
+//   warp 1        mma        one thread issues 8 K-steps of tcgen05.mma (A from tensor memory, B from
+//                            shared memory) into one of two accumulator stages and commits
+//   warps 10-17   epilogue   two groups of four warps, alternate tiles.  Thread t reads accumulator
+//                            row t (tcgen05.ld), rounds to fp16, writes a 128-byte-swizzled staging
+//                            tile; one lane per warp issues two TMA tensor stores (32 rows x 128 B
+//                            each).  The output tensor map is three-dimensional (column, row within
+//                            lambda segment, segment), so the hardware clips a tile that ends with
+//                            its segment or with the tensor: no per-row tail code.
 //
 //   A [128 vectors, K = 128]  fp16 in tensor memory: lane = vector, 64 columns of two codes each
 //   B [N = 128 outputs, K]    fp16 in shared memory, K-major, 128-byte swizzle:
@@ -47,15 +49,14 @@ constexpr int kTile = 128;                 // vectors per tile = MMA M
 constexpr int kInStages = 6;               // packed tiles in flight
 constexpr int kAStages = 4;                // A operands in tensor memory
 constexpr int kAccStages = 2;              // accumulators in tensor memory
-constexpr int kThreads = 320;              // producer, mma, 4 dequant, 4 epilogue warps
+constexpr int kThreads = 576;              // producer, mma, 2 x 4 dequant, 2 x 4 epilogue warps
 
 constexpr int kBBytes = 2 * kTile * 128;               // 32 KB: two K blocks of [128 rows x 128 B]
 constexpr int kInBytes = kTile * (kD / 2);             // 8 KB per packed tile
 constexpr int kOutWarpBytes = 2 * 32 * 128;            // 8 KB: two column halves of [32 rows x 128 B]
-constexpr int kOutBytes = 4 * 2 * kOutWarpBytes;       // 4 warps, double buffered
-constexpr int kRlBytes = kD * 4;
+constexpr int kOutBytes = 8 * kOutWarpBytes;           // one staging tile per epilogue warp
 constexpr int kCtrlBytes = 256;
-constexpr int kSmemBytes = kBBytes + kInStages * kInBytes + kOutBytes + kRlBytes + kCtrlBytes + 1024;
+constexpr int kSmemBytes = kBBytes + kInStages * kInBytes + kOutBytes + kCtrlBytes + 1024;
 
 constexpr uint32_t kAccCol0 = 0;                       // 2 x 128 accumulator columns
 constexpr uint32_t kACol0 = kAccStages * kD;           // then 4 x 64 columns of A
@@ -68,10 +69,8 @@ struct Ctrl {
     uint64_t in_full[kInStages], in_empty[kInStages];
     uint64_t a_full[kAStages], a_empty[kAStages];
     uint64_t acc_full[kAccStages], acc_empty[kAccStages];
-    uint64_t dq_sync;
     uint32_t tmem_base;
     volatile uint32_t abort;
-    float red[4];
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
 
@@ -157,7 +156,6 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap *tm, int c0, int 
                  : "memory");
 }
 
-__device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
 
 __device__ __forceinline__ uint32_t lop3_and_or(uint32_t a, uint32_t b, uint32_t c)
 {
@@ -170,6 +168,43 @@ __device__ __forceinline__ uint32_t lop3_and_or(uint32_t a, uint32_t b, uint32_t
 __device__ __forceinline__ uint32_t sw128_chunk(int r, int j)
 {
     return (uint32_t)((j >> 3) * (kTile * 128) + r * 128 + (((j & 7) ^ (r & 7)) << 4));
+}
+
+// 1 / max(lambda, 1e-6) for the four channels 4 lane .. 4 lane + 3 of lambda row `lam`, divided by rho, the
+// power of two that brings the row's largest reciprocal into [1, 2).  Every lane of the warp gets rho.
+__device__ __forceinline__ float4 recip_lambda4(const float *__restrict__ lam, int lane, float &rho)
+{
+    const float4 l = __ldg(reinterpret_cast<const float4 *>(lam) + lane);
+    float4 r = make_float4(__frcp_rn(fmaxf(l.x, 1e-6f)), __frcp_rn(fmaxf(l.y, 1e-6f)), __frcp_rn(fmaxf(l.z, 1e-6f)),
+                           __frcp_rn(fmaxf(l.w, 1e-6f)));
+    float mx = fmaxf(fmaxf(r.x, r.y), fmaxf(r.z, r.w));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+    rho = __uint_as_float(__float_as_uint(mx) & 0x7F800000u);   // 2^floor(log2 max): exact to divide by
+    r.x /= rho, r.y /= rho, r.z /= rho, r.w /= rho;
+    return r;
+}
+
+// Rows [n0, n1) of the B operand, by one warp: lane l reads the four table entries b0[n][4l .. 4l+3]
+// (one coalesced 512-byte row per step), scales them, trades two values with its neighbour so that each
+// lane holds two K-ordered pairs, and writes 8 bytes of the swizzled row.
+__device__ __forceinline__ void build_b_rows(unsigned char *sB, const float *__restrict__ b0, float4 rl, int n0, int n1, int lane)
+{
+    const bool odd = lane & 1;
+    const int w = lane >> 1;   // word of 8 codes = 16-byte chunk of the K-major row
+#pragma unroll 8
+    for (int n = n0; n < n1; ++n) {
+        const float4 m = __ldg(reinterpret_cast<const float4 *>(b0 + (size_t)n * kD) + lane);
+        auto sat = [](float v) { return fminf(fmaxf(v, -65504.0f), 65504.0f); };
+        const float vx = sat(m.x * rl.x), vy = sat(m.y * rl.y), vz = sat(m.z * rl.z), vw = sat(m.w * rl.w);
+        // even lane holds codes 8w .. 8w+3, odd lane 8w+4 .. 8w+7; K order of the word is (0,4,1,5,2,6,3,7)
+        const float r0 = __shfl_xor_sync(0xFFFFFFFFu, odd ? vx : vz, 1);
+        const float r1 = __shfl_xor_sync(0xFFFFFFFFu, odd ? vy : vw, 1);
+        uint2 o;
+        o.x = odd ? narrow2<false>(r0, vz) : narrow2<false>(vx, r0);   // odd: (2, 6)   even: (0, 4)
+        o.y = odd ? narrow2<false>(r1, vw) : narrow2<false>(vy, r1);   // odd: (3, 7)   even: (1, 5)
+        *reinterpret_cast<uint2 *>(sB + sw128_chunk(n, w) + (odd ? 8 : 0)) = o;
+    }
 }
 
 // Bounded wait that also gives up when another role of the CTA has raised the abort flag.
@@ -206,8 +241,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     unsigned char *sB = smem;
     unsigned char *sIn = sB + kBBytes;
     unsigned char *sOut = sIn + kInStages * kInBytes;
-    float *sRl = reinterpret_cast<float *>(sOut + kOutBytes);
-    Ctrl *ctrl = reinterpret_cast<Ctrl *>(reinterpret_cast<unsigned char *>(sRl) + kRlBytes);
+    Ctrl *ctrl = reinterpret_cast<Ctrl *>(sOut + kOutBytes);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -224,18 +258,10 @@ __global__ void __launch_bounds__(kThreads, 1)
             mbar_init(smem_u32(&ctrl->acc_full[s]), 1);
             mbar_init(smem_u32(&ctrl->acc_empty[s]), 4);
         }
-        mbar_init(smem_u32(&ctrl->dq_sync), 128);
         ctrl->abort = 0u;
         mbar_init_fence();
     }
     if (warp == 0) tmem_alloc(smem_u32(&ctrl->tmem_base), kTmemCols);
-    fence_proxy_async();
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = ctrl->tmem_base;
-    volatile uint32_t *abort_flag = &ctrl->abort;
-    uint32_t *status = prm.g.status;
 
     // ---- tiles: lambda segments of rpl rows, cut into tiles of 128 rows; a contiguous range of tiles
     // ---- per CTA, so that the B operand is rebuilt as rarely as possible
@@ -246,6 +272,22 @@ __global__ void __launch_bounds__(kThreads, 1)
     const int64_t tile_begin = (int64_t)blockIdx.x * per_cta;
     const int64_t tile_end = tile_begin + per_cta < n_tiles ? tile_begin + per_cta : n_tiles;
     const int n_my = tile_end > tile_begin ? (int)(tile_end - tile_begin) : 0;
+    auto seg_of = [&](int j) -> int64_t { return (tile_begin + j) / tps; };
+    auto lambda_row = [&](int64_t seg) -> const float * { return prm.g.lambda + (prm.g.n_lambda == 1 ? 0 : seg) * kD; };
+
+    // ---- B for the first tile's lambda row: every warp builds eight rows
+    if (n_my > 0 && warp < 16) {
+        float rho;
+        const float4 rl = recip_lambda4(lambda_row(seg_of(0)), lane, rho);
+        build_b_rows(sB, prm.g.b0, rl, warp * 8, warp * 8 + 8, lane);
+    }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctrl->tmem_base;
+    volatile uint32_t *abort_flag = &ctrl->abort;
+    uint32_t *status = prm.g.status;
 
     if (warp == 0) {
         // =========================== producer ===========================
@@ -293,77 +335,42 @@ __global__ void __launch_bounds__(kThreads, 1)
                 umma_commit(smem_u32(&ctrl->a_empty[sa]));
             }
         }
-    } else if (warp < 6) {
+    } else if (warp < 10) {
         // =========================== dequant: packed codes -> A in tensor memory ===========================
+        const int grp = (warp - 2) >> 2;        // this group takes tiles grp, grp + 2, ...
         const int q = warp & 3;                 // tensor-memory lane quarter this warp may touch
         const int r = q * 32 + lane;            // tile row and tensor-memory lane of this thread
-        const int t = (warp - 2) * 32 + lane;   // 0..127: B row this thread builds
         const uint2 *scales = static_cast<const uint2 *>(prm.g.scales);   // 4 fp16 scales per row
         const uint32_t swz = (uint32_t)((r >> 1) & 3);
-        uint32_t dq_phase = 0;
-        int64_t cached_seg = -1;
-        float rho = 1.0f;
+        int64_t cached_seg = n_my > 0 ? seg_of(0) : -1;   // B holds this row's table (built before the roles split)
+        float rho;
+        (void)recip_lambda4(lambda_row(n_my > 0 ? seg_of(0) : 0), lane, rho);
 
-        auto row0_of = [&](int j, int64_t &seg) -> int64_t {
-            const int64_t tile = tile_begin + j;
-            seg = tile / tps;
-            return seg * rpl + (tile - seg * tps) * kTile;
-        };
         auto load_scales = [&](int j) -> uint2 {
             if (j >= n_my) return make_uint2(0u, 0u);
-            int64_t seg;
-            const int64_t row = row0_of(j, seg) + r;
+            const int64_t tile = tile_begin + j;
+            const int64_t seg = tile / tps;
+            const int64_t row = seg * rpl + (tile - seg * tps) * kTile + r;
             return row < N ? __ldg(scales + row) : make_uint2(0u, 0u);
         };
-        auto dq_barrier = [&]() -> bool {   // all 128 dequant threads, bounded
-            const uint32_t bar = smem_u32(&ctrl->dq_sync);
-            mbar_arrive(bar);
-            const bool ok = wait_or_abort(bar, dq_phase, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT);
-            dq_phase ^= 1u;
-            return ok;
-        };
 
-        uint2 sc0 = load_scales(0), sc1 = load_scales(1);
-        for (int j = 0; j < n_my; ++j) {
-            const uint2 sc = sc0;
-            sc0 = sc1;
-            sc1 = load_scales(j + 2);
-            int64_t seg;
-            (void)row0_of(j, seg);
+        uint2 sc_next = load_scales(grp);
+        for (int j = grp; j < n_my; j += 2) {
+            const uint2 sc = sc_next;
+            sc_next = load_scales(j + 2);
+            const int64_t seg = seg_of(j);
 
-            // ---- B operand for this lambda row (rare)
+            // ---- a new lambda row: this group needs its rho; the group that meets the row's first tile rebuilds B
             if (seg != cached_seg) {
-                // every MMA issued so far has read B: the commit of the previous tile covers them all
-                if (j > 0 &&
-                    !wait_or_abort(smem_u32(&ctrl->a_empty[(j - 1) % kAStages]), (uint32_t)((j - 1) / kAStages) & 1u, abort_flag,
-                                   status, KVQ_DEV_MMA_TIMEOUT))
-                    break;
-                const int64_t lr = prm.g.n_lambda == 1 ? 0 : seg;
-                const float rl = __frcp_rn(fmaxf(__ldg(prm.g.lambda + lr * kD + t), 1e-6f));
-                float mx = rl;
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
-                if (!dq_barrier()) break;        // nobody still reads red / sRl from the previous rebuild
-                if (lane == 0) ctrl->red[warp - 2] = mx;
-                if (!dq_barrier()) break;
-                mx = fmaxf(fmaxf(ctrl->red[0], ctrl->red[1]), fmaxf(ctrl->red[2], ctrl->red[3]));
-                rho = __uint_as_float(__float_as_uint(mx) & 0x7F800000u);   // 2^floor(log2 max): exact to divide by
-                sRl[t] = rl / rho;
-                if (!dq_barrier()) break;
-                const float4 *b0 = reinterpret_cast<const float4 *>(prm.g.b0 + (size_t)t * kD);   // row n = t, canonical c order
-#pragma unroll 4
-                for (int w = 0; w < 16; ++w) {
-                    const float4 m0 = __ldg(b0 + 2 * w), m1 = __ldg(b0 + 2 * w + 1);
-                    const float4 l0 = reinterpret_cast<const float4 *>(sRl)[2 * w], l1 = reinterpret_cast<const float4 *>(sRl)[2 * w + 1];
-                    auto sat = [](float v) { return fminf(fmaxf(v, -65504.0f), 65504.0f); };
-                    uint4 ch;
-                    ch.x = narrow2<false>(sat(m0.x * l0.x), sat(m1.x * l1.x));   // K order (0,4,1,5,2,6,3,7) of the word
-                    ch.y = narrow2<false>(sat(m0.y * l0.y), sat(m1.y * l1.y));
-                    ch.z = narrow2<false>(sat(m0.z * l0.z), sat(m1.z * l1.z));
-                    ch.w = narrow2<false>(sat(m0.w * l0.w), sat(m1.w * l1.w));
-                    *reinterpret_cast<uint4 *>(sB + sw128_chunk(t, w)) = ch;
+                const float4 rl = recip_lambda4(lambda_row(seg), lane, rho);
+                if (seg_of(j - 1) != seg) {
+                    // every MMA issued so far has read B: the commit of the previous tile covers them all
+                    if (!wait_or_abort(smem_u32(&ctrl->a_empty[(j - 1) % kAStages]), (uint32_t)((j - 1) / kAStages) & 1u, abort_flag,
+                                       status, KVQ_DEV_MMA_TIMEOUT))
+                        break;
+                    build_b_rows(sB, prm.g.b0, rl, q * 32, q * 32 + 32, lane);
+                    fence_proxy_async();   // B is read by the tensor core through the async proxy
                 }
-                fence_proxy_async();   // B is read by the tensor core through the async proxy
                 cached_seg = seg;
             }
 
@@ -412,23 +419,22 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
     } else {
         // =========================== epilogue: accumulator -> fp16 -> TMA store ===========================
+        const int grp = (warp - 10) >> 2;
         const int q = warp & 3;
-        const int ew = warp - 6;                                    // staging slot of this warp
-        unsigned char *stage_base = sOut + ew * (2 * kOutWarpBytes);
+        unsigned char *stg = sOut + (warp - 10) * kOutWarpBytes;   // this warp's staging tile: two [32 rows x 128 B] halves
         const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16) + kAccCol0;
-        for (int j = 0; j < n_my; ++j) {
+        for (int j = grp; j < n_my; j += 2) {
             const int sc = j % kAccStages;
-            unsigned char *stg = stage_base + (j & 1) * kOutWarpBytes;
             if (!wait_or_abort(smem_u32(&ctrl->acc_full[sc]), (uint32_t)(j / kAccStages) & 1u, abort_flag, status, KVQ_DEV_MMA_TIMEOUT)) break;
             tc_fence_after();
-            if (lane == 0) bulk_wait_read_1();   // the store that used this staging buffer two tiles ago has read it
+            if (lane == 0) bulk_wait_read_all();   // this warp's previous stores have read the staging tile
             __syncwarp();
 #pragma unroll
-            for (int cc = 0; cc < 4; ++cc) {
+            for (int cc = 0; cc < 4; ++cc) {   // 32 accumulator columns = 64 bytes of the output row
                 uint32_t v[32];
                 tmem_ld32(lane_addr + (uint32_t)sc * kD + (uint32_t)cc * 32u, v);
                 tmem_ld_wait();
-                unsigned char *half_base = stg + (cc >> 1) * (32 * 128) + lane * 128;
+                unsigned char *half_base = stg + (cc >> 1) * (32 * 128) + lane * 128;   // column half = one store box
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     uint4 o;
