@@ -56,7 +56,7 @@ typedef enum { KVQ_F16 = 0, KVQ_BF16 = 1 } kvq_dtype_t;
 typedef enum {
     KVQ_IMPL_AUTO = 0,
     KVQ_IMPL_FFT = 1, /* fp32 register FFT, one thread per vector: every D and dtype */
-    KVQ_IMPL_GEMM = 2 /* tcgen05 DFT-as-GEMM; returns KVQ_ERR_UNSUPPORTED_DIM where not built */
+    KVQ_IMPL_GEMM = 2 /* tcgen05 DFT-as-GEMM (encode: D = 128; decode: D = 128, fp16); KVQ_ERR_UNSUPPORTED_DIM elsewhere */
 } kvq_impl_t;
 
 /*

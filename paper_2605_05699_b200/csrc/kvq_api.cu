@@ -22,6 +22,9 @@ static inline uint64_t splitmix64_at(uint64_t seed, uint64_t n)
     return z ^ (z >> 31);
 }
 
+// AUTO sends kvq_encode / kvq_append calls of at least this many rows to the tensor-core kernel.
+constexpr int64_t kGemmEncodeMinRows = 4096;
+
 static bool dim_supported(int D) { return D == 64 || D == 96 || D == 128 || D == 160 || D == 256; }
 
 // Radices of the length-n complex FFT in the order the recursion splits them off (4 first,
@@ -105,6 +108,33 @@ static kvq_status_t ensure_device(kvq_plan *p)
         }
         p->d_b0 = devp;
         p->table_bytes += bytes;
+        // the forward table is the transpose: e0[c][n] = b0[n][c]
+        float *hostT = new (std::nothrow) float[(size_t)p->D * p->D];
+        float *devT = nullptr;
+        bool okT = hostT && cudaMalloc(&devT, bytes) == cudaSuccess;
+        if (okT) {
+            float *tmp = new (std::nothrow) float[(size_t)p->D * p->D];
+            okT = tmp != nullptr;
+            if (okT) {
+                build_b0(p, tmp);
+                for (int n = 0; n < p->D; ++n)
+                    for (int c = 0; c < p->D; ++c) hostT[(size_t)c * p->D + n] = tmp[(size_t)n * p->D + c];
+                okT = cudaMemcpy(devT, hostT, bytes, cudaMemcpyHostToDevice) == cudaSuccess;
+            }
+            delete[] tmp;
+        }
+        delete[] hostT;
+        if (!okT) {
+            (void)cudaGetLastError();
+            if (devT) cudaFree(devT);
+            cudaFree(devp);
+            cudaFree(st);
+            p->d_b0 = nullptr;
+            p->d_status = nullptr;
+            return KVQ_ERR_NOMEM;
+        }
+        p->d_e0 = devT;
+        p->table_bytes += bytes;
     }
     p->device = dev;
     return KVQ_OK;
@@ -153,6 +183,7 @@ kvq_status_t kvq_plan_create(int D, int group, uint64_t seed, kvq_plan_t **out)
     p->device = -1;
     p->d_status = nullptr;
     p->d_b0 = nullptr;
+    p->d_e0 = nullptr;
     p->table_bytes = 0;
     std::memset(p->signs, 0, sizeof(p->signs));
     std::memset(p->sign_xor, 0, sizeof(p->sign_xor));
@@ -173,6 +204,9 @@ kvq_status_t kvq_plan_destroy(kvq_plan_t *plan)
     }
     if (plan->d_b0) {
         if (cudaFree(plan->d_b0) != cudaSuccess) (void)cudaGetLastError();
+    }
+    if (plan->d_e0) {
+        if (cudaFree(plan->d_e0) != cudaSuccess) (void)cudaGetLastError();
     }
     delete plan;
     return KVQ_OK;
@@ -234,7 +268,8 @@ static kvq_status_t encode_common(kvq_plan_t *plan, const void *x, kvq_dtype_t d
     kvq_status_t st = check_lambda(N, lambda, n_lambda, rows_per_lambda);
     if (st != KVQ_OK) return st;
     if (misaligned16(x) || misaligned16(packed) || misaligned16(scales)) return KVQ_ERR_ALIGNMENT;
-    if (plan->enc_impl == KVQ_IMPL_GEMM) return KVQ_ERR_UNSUPPORTED_DIM;
+    const bool gemm_ok = plan->D == 128;
+    if (plan->enc_impl == KVQ_IMPL_GEMM && !gemm_ok) return KVQ_ERR_UNSUPPORTED_DIM;
     if ((st = ensure_device(plan)) != KVQ_OK) return st;
     FftParams prm;
     fill_params(plan, prm, N, lambda, n_lambda, rows_per_lambda);
@@ -243,7 +278,10 @@ static kvq_status_t encode_common(kvq_plan_t *plan, const void *x, kvq_dtype_t d
     prm.scales = scales;
     prm.out_mul = out_mul;
     prm.out_add = out_add;
-    cudaError_t e = fft_encode(plan->D, dtype == KVQ_BF16, N, prm, static_cast<cudaStream_t>(cuda_stream));
+    // the tensor-core kernel pays a fixed set-up per launch (B operand build); small calls stay on the register FFT
+    const bool use_gemm = gemm_ok && (plan->enc_impl == KVQ_IMPL_GEMM || (plan->enc_impl == KVQ_IMPL_AUTO && N >= kGemmEncodeMinRows));
+    cudaError_t e = use_gemm ? umma_encode_d128(dtype == KVQ_BF16, N, prm, plan->d_e0, static_cast<cudaStream_t>(cuda_stream))
+                             : fft_encode(plan->D, dtype == KVQ_BF16, N, prm, static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
         return KVQ_ERR_CUDA;

@@ -38,6 +38,9 @@ struct GemmParams {
 };
 
 cudaError_t umma_decode_d128(int64_t N, const GemmParams &prm, cudaStream_t stream);
+// tcgen05 DFT-as-GEMM encode (kvq_umma_encode.cu): takes the register-FFT argument block (sign words unused) and
+// the plan table e0 [D, D] fp32, e0[c][n] = M[c][n] s_n.
+cudaError_t umma_encode_d128(bool bf16, int64_t N, const FftParams &prm, const float *e0, cudaStream_t stream);
 
 cudaError_t fft_encode(int D, bool bf16, int64_t N, const FftParams &prm, cudaStream_t stream);
 cudaError_t fft_decode(int D, bool bf16, int64_t N, const FftParams &prm, cudaStream_t stream);
@@ -58,5 +61,6 @@ struct kvq_plan {
     int device;            // -1 until initialised
     uint32_t *d_status;    // device status word
     float *d_b0;           // [D, D] fp32 inverse-transform matrix with the signs folded in (GEMM decode), or null
+    float *d_e0;           // [D, D] fp32 forward-transform matrix with the signs folded in (GEMM encode), or null
     size_t table_bytes;
 };

@@ -85,7 +85,51 @@ def test_decode_kernel_families_d128_f16(dec_impl, N, n_lambda, rpl, kind):
         assert dec["rel_l2_plain_max"] < 1e-3  # fp32 arithmetic: far inside the tolerance even without the tie rule
 
 
-def test_gemm_decode_is_refused_where_it_is_not_built():
+# ---- both encode kernel families at D = 128: the fp32 register FFT and the tcgen05 DFT-as-GEMM with split W
+
+@pytest.mark.parametrize("enc_impl", ["fft", "gemm"])
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("N,n_lambda,rpl,kind", [(4096, 1, 0, "c1"), (1000, 4, 333, "k_outlier"), (1, 1, 0, "gaussian"),
+                                                 (129, 1, 0, "gaussian"), (70000, 7, 10000, "k_outlier")])
+def test_encode_kernel_families_d128(enc_impl, dtype, N, n_lambda, rpl, kind):
+    enc, dec = run_case(128, dtype, N, kind, 9000 + N, n_lambda=n_lambda, rows_per_lambda=rpl, enc_impl=enc_impl, dec_impl="fft")
+    assert enc["mismatches"] <= max(2, int(1e-4 * N * 128))
+
+
+def test_lambda_scale_does_not_matter_to_the_gemm_encode():
+    # lambda rows far from 1: the power-of-two lift keeps the split terms of W inside fp16's normal range
+    for shift in (-12, 9):
+        D, N = 128, 2048
+        plan = kb.Plan(D, G, 31)
+        kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_GEMM, kb.KVQ_IMPL_FFT)
+        sg = plan.signs()
+        x = wl.make_vectors(N, D, "f16", "k_outlier", 77)
+        lam = wl.make_lambda(1, D, 78) * (2.0 ** shift)
+        ora = ko.encode(bits(x), ko.F16, sg, lam.numpy(), G, want_v=True)
+        packed, scales = gpu_encode(plan, x.cuda(), lam.cuda())
+        parity.check_encode(packed.cpu().numpy(), bits(scales), ora, G, "gemm encode, lambda x 2^%d" % shift)
+        plan.close()
+
+
+def test_gemm_encode_serves_large_appends():
+    # append of many streams goes through the same tensor-core kernel with scattered output rows
+    D, S, T = 128, 5000, 3
+    plan = kb.Plan(D, G, 6)
+    kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_GEMM, kb.KVQ_IMPL_AUTO)
+    x = wl.make_vectors(S, D, "f16", "k_outlier", 19)
+    lam = wl.make_lambda(5, D, 20)
+    packed = torch.full((S, T, D // 2), 0xAB, dtype=torch.uint8, device="cuda")
+    scales = torch.full((S, T, D // G), 1.25, dtype=torch.float16, device="cuda")
+    kb.kvq_append(plan.handle, x.cuda(), lam.cuda(), packed, scales, 1, 1000)
+    torch.cuda.synchronize()
+    assert kb.kvq_plan_device_status(plan.handle) == 0
+    assert bool((packed[:, [0, 2]] == 0xAB).all()) and bool((scales[:, [0, 2]] == 1.25).all())
+    ora = ko.encode(bits(x), ko.F16, plan.signs(), lam.numpy(), G, 1000, want_v=True)
+    parity.check_encode(packed[:, 1].contiguous().cpu().numpy(), bits(scales[:, 1].contiguous()), ora, G, "gemm append")
+    plan.close()
+
+
+def test_gemm_kernels_are_refused_where_they_are_not_built():
     for D, dtype in [(256, torch.float16), (128, torch.bfloat16), (96, torch.float16)]:
         plan = kb.Plan(D, G, 1)
         kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_AUTO, kb.KVQ_IMPL_GEMM)
@@ -93,6 +137,14 @@ def test_gemm_decode_is_refused_where_it_is_not_built():
         out = torch.empty(8, D, dtype=dtype, device="cuda")
         with pytest.raises(kb.KvqError) as e:
             kb.kvq_decode(plan.handle, pk, sc, torch.ones(D, device="cuda"), out)
+        assert e.value.status == kb.KVQ_ERR_UNSUPPORTED_DIM
+        plan.close()
+    for D in (96, 256):
+        plan = kb.Plan(D, G, 1)
+        kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_GEMM, kb.KVQ_IMPL_AUTO)
+        x = torch.zeros(8, D, dtype=torch.float16, device="cuda")
+        with pytest.raises(kb.KvqError) as e:
+            kb.kvq_encode(plan.handle, x, torch.ones(D, device="cuda"), plan.empty_packed(8), plan.empty_scales(8))
         assert e.value.status == kb.KVQ_ERR_UNSUPPORTED_DIM
         plan.close()
 
@@ -223,9 +275,9 @@ def test_config3_gemma_shaped_prefix_4096_sampled():
 
 # ---- config 5: Llama-3-70B-shaped: one layer's K (1,048,576 vectors) per launch, sampled rows -
 
-def _full_size_sampled(D, dtype, N, kind, seed, n_lambda, rows_per_lambda, n_random=4096, dec_impl="auto"):
+def _full_size_sampled(D, dtype, N, kind, seed, n_lambda, rows_per_lambda, n_random=4096, dec_impl="auto", enc_impl="auto"):
     plan = kb.Plan(D, G, seed)
-    kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_AUTO, IMPL[dec_impl])
+    kb.kvq_plan_set_impl(plan.handle, IMPL[enc_impl], IMPL[dec_impl])
     sg = plan.signs()
     x = wl.make_vectors(N, D, dtype, kind, seed, device="cuda")
     lam = wl.make_lambda(n_lambda, D, seed + 1, device="cuda")
@@ -252,12 +304,12 @@ def _full_size_sampled(D, dtype, N, kind, seed, n_lambda, rows_per_lambda, n_ran
     plan.close()
 
 
-@pytest.mark.parametrize("dec_impl", ["fft", "gemm"])
-def test_config5_llama70b_shaped_one_layer_full_size_sampled(dec_impl):
+@pytest.mark.parametrize("impl", ["fft", "gemm"])
+def test_config5_llama70b_shaped_one_layer_full_size_sampled(impl):
     # the launch configuration bench.py times: K and V of one layer in one call, 2 x 1,048,576 vectors, two lambda rows
     shp = wl.LLAMA3_70B
     half = shp.kv_heads * shp.batch * shp.prefix
-    _full_size_sampled(128, "f16", 2 * half, "k_outlier", 7001, 2, half, dec_impl=dec_impl)
+    _full_size_sampled(128, "f16", 2 * half, "k_outlier", 7001, 2, half, dec_impl=impl, enc_impl=impl)
 
 
 def test_config5_llama70b_shaped_v_like_full_size_sampled():
