@@ -162,6 +162,31 @@ __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wa
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // ---------------------------------------------------------------------------
+// Tiles of the tensor-core kernels.  Rows are cut into lambda segments of `rpl` rows, a segment into
+// tiles of 128 rows (the last one of a segment may be short), tiles are numbered segment by segment.
+// The cursor walks a CTA's tiles without a 64-bit division per step.
+// ---------------------------------------------------------------------------
+struct TileCursor {
+    int64_t seg;   // lambda segment of the current tile
+    int64_t tin;   // index of the tile within its segment
+    int64_t tps;   // tiles per segment
+    __device__ __forceinline__ TileCursor(int64_t tile, int64_t tiles_per_segment)
+        : seg(tile / tiles_per_segment), tin(tile - (tile / tiles_per_segment) * tiles_per_segment), tps(tiles_per_segment)
+    {
+    }
+    __device__ __forceinline__ void advance(int step)
+    {
+        tin += step;
+        while (tin >= tps) {
+            tin -= tps;
+            ++seg;
+        }
+    }
+    __device__ __forceinline__ bool first_of_segment() const { return tin == 0; }
+    __device__ __forceinline__ int64_t row_in_segment() const { return tin * 128; }
+};
+
+// ---------------------------------------------------------------------------
 // half-precision words: two 16-bit values per 32-bit word, low half first
 // ---------------------------------------------------------------------------
 template <bool BF16>

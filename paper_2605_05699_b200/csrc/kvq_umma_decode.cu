@@ -272,13 +272,13 @@ __global__ void __launch_bounds__(kThreads, 1)
     const int64_t tile_begin = (int64_t)blockIdx.x * per_cta;
     const int64_t tile_end = tile_begin + per_cta < n_tiles ? tile_begin + per_cta : n_tiles;
     const int n_my = tile_end > tile_begin ? (int)(tile_end - tile_begin) : 0;
-    auto seg_of = [&](int j) -> int64_t { return (tile_begin + j) / tps; };
+    const int64_t seg_first = n_my > 0 ? tile_begin / tps : 0;
     auto lambda_row = [&](int64_t seg) -> const float * { return prm.g.lambda + (prm.g.n_lambda == 1 ? 0 : seg) * kD; };
 
     // ---- B for the first tile's lambda row: every warp builds eight rows
     if (n_my > 0 && warp < 16) {
         float rho;
-        const float4 rl = recip_lambda4(lambda_row(seg_of(0)), lane, rho);
+        const float4 rl = recip_lambda4(lambda_row(seg_first), lane, rho);
         build_b_rows(sB, prm.g.b0, rl, warp * 8, warp * 8 + 8, lane);
     }
     fence_proxy_async();
@@ -294,14 +294,13 @@ __global__ void __launch_bounds__(kThreads, 1)
         if (lane == 0) {
             int issued = 0;
             bool ok = true;
-            for (int j = 0; j < n_my; ++j) {
+            TileCursor cur(tile_begin, tps);
+            for (int j = 0; j < n_my; ++j, cur.advance(1)) {
                 const int s = j % kInStages;
                 const uint32_t use = (uint32_t)(j / kInStages);
                 ok = wait_or_abort(smem_u32(&ctrl->in_empty[s]), (use & 1u) ^ 1u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT);
                 if (!ok) break;
-                const int64_t tile = tile_begin + j;
-                const int64_t seg = tile / tps;
-                const int64_t row0 = seg * rpl + (tile - seg * tps) * kTile;
+                const int64_t row0 = cur.seg * rpl + cur.row_in_segment();
                 const uint32_t bar = smem_u32(&ctrl->in_full[s]);
                 mbar_arrive_expect_tx(bar, kInBytes);
                 tma_load_2d(smem_u32(sIn + s * kInBytes), &tm_packed, 0, (int)row0, bar);
@@ -342,28 +341,28 @@ __global__ void __launch_bounds__(kThreads, 1)
         const int r = q * 32 + lane;            // tile row and tensor-memory lane of this thread
         const uint2 *scales = static_cast<const uint2 *>(prm.g.scales);   // 4 fp16 scales per row
         const uint32_t swz = (uint32_t)((r >> 1) & 3);
-        int64_t cached_seg = n_my > 0 ? seg_of(0) : -1;   // B holds this row's table (built before the roles split)
+        int64_t cached_seg = n_my > 0 ? seg_first : -1;   // B holds this row's table (built before the roles split)
         float rho;
-        (void)recip_lambda4(lambda_row(n_my > 0 ? seg_of(0) : 0), lane, rho);
+        (void)recip_lambda4(lambda_row(seg_first), lane, rho);
 
+        TileCursor cur(tile_begin + grp, tps), ahead(tile_begin + grp, tps);   // this tile; the tile whose scales are fetched
         auto load_scales = [&](int j) -> uint2 {
             if (j >= n_my) return make_uint2(0u, 0u);
-            const int64_t tile = tile_begin + j;
-            const int64_t seg = tile / tps;
-            const int64_t row = seg * rpl + (tile - seg * tps) * kTile + r;
+            const int64_t row = ahead.seg * rpl + ahead.row_in_segment() + r;
             return row < N ? __ldg(scales + row) : make_uint2(0u, 0u);
         };
 
         uint2 sc_next = load_scales(grp);
-        for (int j = grp; j < n_my; j += 2) {
+        for (int j = grp; j < n_my; j += 2, cur.advance(2)) {
             const uint2 sc = sc_next;
+            ahead.advance(2);
             sc_next = load_scales(j + 2);
-            const int64_t seg = seg_of(j);
+            const int64_t seg = cur.seg;
 
             // ---- a new lambda row: this group needs its rho; the group that meets the row's first tile rebuilds B
             if (seg != cached_seg) {
                 const float4 rl = recip_lambda4(lambda_row(seg), lane, rho);
-                if (seg_of(j - 1) != seg) {
+                if (cur.first_of_segment()) {
                     // every MMA issued so far has read B: the commit of the previous tile covers them all
                     if (!wait_or_abort(smem_u32(&ctrl->a_empty[(j - 1) % kAStages]), (uint32_t)((j - 1) / kAStages) & 1u, abort_flag,
                                        status, KVQ_DEV_MMA_TIMEOUT))
@@ -423,7 +422,8 @@ __global__ void __launch_bounds__(kThreads, 1)
         const int q = warp & 3;
         unsigned char *stg = sOut + (warp - 10) * kOutWarpBytes;   // this warp's staging tile: two [32 rows x 128 B] halves
         const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16) + kAccCol0;
-        for (int j = grp; j < n_my; j += 2) {
+        TileCursor cur(tile_begin + grp, tps);
+        for (int j = grp; j < n_my; j += 2, cur.advance(2)) {
             const int sc = j % kAccStages;
             if (!wait_or_abort(smem_u32(&ctrl->acc_full[sc]), (uint32_t)(j / kAccStages) & 1u, abort_flag, status, KVQ_DEV_MMA_TIMEOUT)) break;
             tc_fence_after();
@@ -451,9 +451,8 @@ __global__ void __launch_bounds__(kThreads, 1)
             __syncwarp();
             if (lane == 0) {
                 mbar_arrive(smem_u32(&ctrl->acc_empty[sc]));
-                const int64_t tile = tile_begin + j;
-                const int64_t seg = tile / tps;
-                const int row_in_seg = (int)((tile - seg * tps) * kTile) + q * 32;
+                const int64_t seg = cur.seg;
+                const int row_in_seg = (int)cur.row_in_segment() + q * 32;
                 const bool tail = seg >= prm.n_full;
                 const CUtensorMap *tm = tail ? &tm_out_tail : &tm_out;
                 const int segc = tail ? 0 : (int)seg;

@@ -15,13 +15,14 @@
 //                            canonical K-major layout, four tiles in flight, no thread touches it
 //   warp 1        mma        one thread issues 8 K-steps per split term into one of four accumulator
 //                            stages, then commits: once to the epilogue, once to free the x stage
-//   warps 2-17    epilogue   thread = (row, group of 32 channels): tcgen05.ld of its 32 accumulator
-//                            columns, abs-max, fp16 scale, round-to-nearest-even codes, nibble pack
-//                            (Sec. 3.2 steps 3-4, per-group scales of Sec. 5.6 / 7.1): no shuffle, no
-//                            shared memory; 16 bytes of codes and one scale per thread go straight
-//                            to global memory.  The accumulator stage is released as soon as the
-//                            values are in registers.  These warps also build the B operand when the
-//                            lambda row changes (the mma warp waits for it on an mbarrier).
+//   warps 2-17    epilogue   two sets of eight warps on alternate tiles; thread = (row, half row).  Per group
+//                            of 32 channels: tcgen05.ld of the 32 accumulator columns, abs-max, fp16 scale,
+//                            round-to-nearest-even codes, nibble pack (Sec. 3.2 steps 3-4, per-group scales
+//                            of Sec. 5.6 / 7.1): no shuffle, no shared memory; 32 bytes of codes and two
+//                            scales per thread go straight to global memory.  The accumulator stage is
+//                            released as soon as the values are in registers.  The set that meets the first
+//                            tile of a new lambda row rebuilds the B operand (the mma warp waits for it on
+//                            an mbarrier).
 //
 //   A [128 vectors, K = 128]   x in shared memory (TMA), K-major, 128-byte swizzle
 //   B [N = 128 channels, K]    split terms of W 2^k in shared memory, same layout, one region per term
@@ -43,6 +44,7 @@ constexpr int kTile = 128;                 // vectors per tile = MMA M
 constexpr int kGroup = 32;
 constexpr int kInStages = 4;               // x tiles in flight (32 KB each)
 constexpr int kAccStages = 4;              // accumulators in tensor memory
+static_assert(kInStages == kAccStages, "the x stage of tile j is released by the accumulator barrier of tile j");
 constexpr int kThreads = 576;              // producer, mma, 16 epilogue warps
 constexpr int kEpiWarps = 16;
 
@@ -64,7 +66,7 @@ struct Cfg {
 };
 
 struct Ctrl {
-    uint64_t in_full[kInStages], in_empty[kInStages];
+    uint64_t in_full[kInStages];
     uint64_t acc_full[kAccStages], acc_empty[kAccStages];
     uint64_t b_ready;
     uint32_t tmem_base;
@@ -226,13 +228,12 @@ __global__ void __launch_bounds__(kThreads, 1)
     if (threadIdx.x == 0) {
         for (int s = 0; s < kInStages; ++s) {
             mbar_init(smem_u32(&ctrl->in_full[s]), 1);
-            mbar_init(smem_u32(&ctrl->in_empty[s]), 1);
         }
         for (int s = 0; s < kAccStages; ++s) {
             mbar_init(smem_u32(&ctrl->acc_full[s]), 1);
-            mbar_init(smem_u32(&ctrl->acc_empty[s]), kEpiWarps);
+            mbar_init(smem_u32(&ctrl->acc_empty[s]), kEpiWarps / 2);
         }
-        mbar_init(smem_u32(&ctrl->b_ready), kEpiWarps);
+        mbar_init(smem_u32(&ctrl->b_ready), kEpiWarps / 2);
         ctrl->abort = 0u;
         mbar_init_fence();
     }
@@ -253,20 +254,20 @@ __global__ void __launch_bounds__(kThreads, 1)
     const int64_t tile_begin = (int64_t)blockIdx.x * per_cta;
     const int64_t tile_end = tile_begin + per_cta < n_tiles ? tile_begin + per_cta : n_tiles;
     const int n_my = tile_end > tile_begin ? (int)(tile_end - tile_begin) : 0;
-    auto seg_of = [&](int j) -> int64_t { return (tile_begin + j) / tps; };
 
     if (warp == 0) {
         // =========================== producer ===========================
         if (lane == 0) {
             int issued = 0;
             bool ok = true;
-            for (int j = 0; j < n_my; ++j) {
+            TileCursor cur(tile_begin, tps);
+            for (int j = 0; j < n_my; ++j, cur.advance(1)) {
                 const int s = j % kInStages;
-                ok = wait_or_abort(smem_u32(&ctrl->in_empty[s]), ((uint32_t)(j / kInStages) & 1u) ^ 1u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT);
+                // the x stage is free once the MMAs of the tile that used it last are complete: that tile's accumulator barrier
+                if (j >= kInStages)
+                    ok = wait_or_abort(smem_u32(&ctrl->acc_full[s]), (uint32_t)(j / kInStages - 1) & 1u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT);
                 if (!ok) break;
-                const int64_t tile = tile_begin + j;
-                const int64_t seg = tile / tps;
-                const int64_t row0 = seg * rpl + (tile - seg * tps) * kTile;
+                const int64_t row0 = cur.seg * rpl + cur.row_in_segment();
                 const uint32_t bar = smem_u32(&ctrl->in_full[s]);
                 mbar_arrive_expect_tx(bar, kOpBytes);
                 tma_load_2d(smem_u32(sIn + s * kOpBytes), &tm_x, 0, (int)row0, bar);
@@ -283,15 +284,13 @@ __global__ void __launch_bounds__(kThreads, 1)
         // =========================== mma issuer ===========================
         if (lane == 0) {
             const uint32_t b_addr = smem_u32(sB);
-            int64_t cur_seg = -1;
             uint32_t builds = 0;
-            for (int j = 0; j < n_my; ++j) {
+            TileCursor cur(tile_begin, tps);
+            for (int j = 0; j < n_my; ++j, cur.advance(1)) {
                 const int s = j % kInStages, sc = j % kAccStages;
-                const int64_t seg = seg_of(j);
-                if (seg != cur_seg) {   // the epilogue warps rebuild B for this lambda row
+                if (j == 0 || cur.first_of_segment()) {   // an epilogue set rebuilds B for this lambda row
                     if (!wait_or_abort(smem_u32(&ctrl->b_ready), builds & 1u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT)) break;
                     ++builds;
-                    cur_seg = seg;
                 }
                 if (!wait_or_abort(smem_u32(&ctrl->in_full[s]), (uint32_t)(j / kInStages) & 1u, abort_flag, status, KVQ_DEV_LOAD_TIMEOUT)) break;
                 if (!wait_or_abort(smem_u32(&ctrl->acc_empty[sc]), ((uint32_t)(j / kAccStages) & 1u) ^ 1u, abort_flag, status,
@@ -309,33 +308,42 @@ __global__ void __launch_bounds__(kThreads, 1)
                                     (t > 0 || ks > 0) ? 1u : 0u);
                     }
                 }
-                umma_commit(smem_u32(&ctrl->acc_full[sc]));
-                umma_commit(smem_u32(&ctrl->in_empty[s]));   // the tensor core has read the x tile
+                umma_commit(smem_u32(&ctrl->acc_full[sc]));   // to the epilogue; the producer takes it as "x stage free"
             }
         }
     } else {
         // =========================== epilogue: accumulator -> scales, codes, nibbles ===========================
+        // Two sets of eight warps take alternate tiles, so that one set's waits (barrier, tensor-memory load)
+        // hide behind the other set's arithmetic.  Thread = (row, half row): groups 2h and 2h + 1.
+        const int set = (warp - 2) >> 3;        // this set takes tiles set, set + 2, ...
         const int q = warp & 3;                 // tensor-memory lane quarter this warp may touch
-        const int g = (warp - 2) >> 2;          // group of 32 channels this warp quantizes
+        const int h = ((warp - 2) >> 2) & 1;    // half of the row: channels 64 h .. 64 h + 63
         const int r = q * 32 + lane;            // tile row of this thread
-        const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(g * kGroup);
+        const int bw = (warp - 2) & 7;          // position within the set: 16 rows of B per warp when the set rebuilds B
+        const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(h * 2 * kGroup);
         int64_t cached_seg = -1;
         float unlift = 1.0f;
-        for (int j = 0; j < n_my; ++j) {
+        TileCursor cur(tile_begin + set, tps);
+        for (int j = set; j < n_my; j += 2, cur.advance(2)) {
             __syncwarp();
-            const int64_t tile = tile_begin + j;
-            const int64_t seg = tile / tps;
-            const int64_t off = (tile - seg * tps) * kTile;
+            const int64_t seg = cur.seg;
+            const int64_t off = cur.row_in_segment();
 
-            // ---- a new lambda row: all MMAs that read the old B are complete (this warp has consumed their
-            // ---- accumulators), so the 16 epilogue warps rewrite B, eight rows each, and tell the mma warp
+            // ---- a new lambda row.  Every set needs its lift; the set that owns the row's first tile rebuilds B,
+            // ---- once every MMA that read the old B is complete (the previous tile's accumulator is full), and
+            // ---- tells the mma warp.
             if (seg != cached_seg) {
                 const float *lam = prm.lambda + (prm.n_lambda == 1 ? 0 : seg) * kD;
                 const float lift = lift_of(lam, lane);
-                build_b_rows<BF16>(sB, prm.e0, lam, lift, (warp - 2) * 8, (warp - 2) * 8 + 8, lane);
-                fence_proxy_async();   // B is read by the tensor core through the async proxy
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&ctrl->b_ready));
+                if (j == 0 || cur.first_of_segment()) {
+                    if (j > 0 && !wait_or_abort(smem_u32(&ctrl->acc_full[(j - 1) % kAccStages]), (uint32_t)((j - 1) / kAccStages) & 1u,
+                                                abort_flag, status, KVQ_DEV_MMA_TIMEOUT))
+                        break;
+                    build_b_rows<BF16>(sB, prm.e0, lam, lift, bw * 16, bw * 16 + 16, lane);
+                    fence_proxy_async();   // B is read by the tensor core through the async proxy
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&ctrl->b_ready));
+                }
                 unlift = 1.0f / lift;
                 cached_seg = seg;
             }
@@ -343,49 +351,57 @@ __global__ void __launch_bounds__(kThreads, 1)
             const int sc = j % kAccStages;
             if (!wait_or_abort(smem_u32(&ctrl->acc_full[sc]), (uint32_t)(j / kAccStages) & 1u, abort_flag, status, KVQ_DEV_MMA_TIMEOUT)) break;
             tc_fence_after();
-            uint32_t vb[32];
-            tmem_ld32(t_addr + (uint32_t)sc * kD, vb);
-            tmem_ld_wait();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&ctrl->acc_empty[sc]));   // the values are in registers
 
             // ---- rows of the tile that exist: the segment (and with it the tensor) may end inside the tile
             int64_t seg_rows = N - seg * rpl;
             if (seg_rows > rpl) seg_rows = rpl;
-            if (off + r < seg_rows) {
+            const bool live = off + r < seg_rows;
             const int64_t orow = (seg * rpl + off + r) * prm.out_mul + prm.out_add;
-
-            // ---- scale: sigma = fp16(absmax / 7); codes are taken against the stored value
-            float amax = 0.0f;
+            uint32_t sbits = 0;
 #pragma unroll
-            for (int i = 0; i < 32; ++i) amax = fmaxf(amax, fabsf(__uint_as_float(vb[i])));
-            amax *= unlift;
-            const float sig = fminf(__fdiv_rn(amax, 7.0f), 65504.0f);
-            const __half hs = __float2half_rn(sig);
-            const float sg = __half2float(hs);
-            const float rs1 = sg > 0.0f ? __frcp_rn(sg) : 0.0f;
-            const bool clamp = !(amax * rs1 < 7.25f);   // saturated or subnormal scale: codes could leave [-7, 7]
-            const float rs = rs1 * unlift;              // applies to the lifted accumulator values
-            prm.scales[orow * (kD / kGroup) + g] = __half_as_ushort(hs);
-
-            // ---- round, bias to unsigned nibbles, pack 8 codes per word
-            uint32_t words[4];
-#pragma unroll
-            for (int w = 0; w < 4; ++w) {
-                uint32_t acc = 0;
-                if (!clamp) {
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) acc += __float_as_uint(fmaf(__uint_as_float(vb[8 * w + e]), rs, kMagicRound)) << (4 * e);
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 8; ++e)
-                        acc += __float_as_uint(fminf(fmaxf(__uint_as_float(vb[8 * w + e]) * rs, -7.0f), 7.0f) + kMagicRound) << (4 * e);
+            for (int gg = 0; gg < 2; ++gg) {
+                uint32_t vb[32];
+                tmem_ld32(t_addr + (uint32_t)sc * kD + (uint32_t)(gg * kGroup), vb);
+                tmem_ld_wait();
+                if (gg == 1) {   // both groups are in registers: hand the accumulator back
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&ctrl->acc_empty[sc]));
                 }
-                words[w] = (acc - kMagicSum) ^ 0x88888888u;
+                // ---- scale: sigma = fp16(absmax / 7); codes are taken against the stored value
+                float amax = 0.0f;
+#pragma unroll
+                for (int i = 0; i < 32; ++i) amax = fmaxf(amax, fabsf(__uint_as_float(vb[i])));
+                amax *= unlift;
+                const float sig = fminf(__fdiv_rn(amax, 7.0f), 65504.0f);
+                const __half hs = __float2half_rn(sig);
+                const float sg = __half2float(hs);
+                const float rs1 = sg > 0.0f ? __frcp_rn(sg) : 0.0f;
+                const bool clamp = !(amax * rs1 < 7.25f);   // saturated or subnormal scale: codes could leave [-7, 7]
+                const float rs = rs1 * unlift;              // applies to the lifted accumulator values
+                sbits |= (uint32_t)__half_as_ushort(hs) << (16 * gg);
+
+                // ---- round, bias to unsigned nibbles, pack 8 codes per word
+                uint32_t words[4];
+#pragma unroll
+                for (int w = 0; w < 4; ++w) {
+                    uint32_t acc = 0;
+                    if (!clamp) {
+#pragma unroll
+                        for (int e = 0; e < 8; ++e)
+                            acc += __float_as_uint(fmaf(__uint_as_float(vb[8 * w + e]), rs, kMagicRound)) << (4 * e);
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 8; ++e)
+                            acc += __float_as_uint(fminf(fmaxf(__uint_as_float(vb[8 * w + e]) * rs, -7.0f), 7.0f) + kMagicRound) << (4 * e);
+                    }
+                    words[w] = (acc - kMagicSum) ^ 0x88888888u;
+                }
+                if (live)
+                    *reinterpret_cast<uint4 *>(prm.packed + orow * (kD / 2) + (2 * h + gg) * 16) =
+                        make_uint4(words[0], words[1], words[2], words[3]);
             }
-            *reinterpret_cast<uint4 *>(prm.packed + orow * (kD / 2) + g * 16) = make_uint4(words[0], words[1], words[2], words[3]);
-            }
+            if (live) *reinterpret_cast<uint32_t *>(prm.scales + orow * (kD / kGroup) + 2 * h) = sbits;
         }
     }
 
