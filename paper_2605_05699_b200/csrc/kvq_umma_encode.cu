@@ -14,7 +14,8 @@
 //                            128-byte swizzle): x lands in shared memory in the tensor core's
 //                            canonical K-major layout, four tiles in flight, no thread touches it
 //   warp 1        mma        one thread issues 8 K-steps per split term into one of four accumulator
-//                            stages, then commits: once to the epilogue, once to free the x stage
+//                            stages, then commits once: the epilogue reads it as "accumulator full",
+//                            the producer as "x stage free"
 //   warps 2-17    epilogue   two sets of eight warps on alternate tiles; thread = (row, half row).  Per group
 //                            of 32 channels: tcgen05.ld of the 32 accumulator columns, abs-max, fp16 scale,
 //                            round-to-nearest-even codes, nibble pack (Sec. 3.2 steps 3-4, per-group scales
@@ -95,13 +96,14 @@ __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence:
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
 // D[tmem] (+)= A[smem] * B[smem]
-__device__ __forceinline__ void umma_f16_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+template <bool ACCUMULATE>
+__device__ __forceinline__ void umma_f16_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc)
 {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
-        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        "l"(adesc), "l"(bdesc), "r"(idesc), "n"(ACCUMULATE ? 1 : 0)
         : "memory");
 }
 
@@ -283,7 +285,13 @@ __global__ void __launch_bounds__(kThreads, 1)
     } else if (warp == 1) {
         // =========================== mma issuer ===========================
         if (lane == 0) {
-            const uint32_t b_addr = smem_u32(sB);
+            // Descriptors differ only in their 14-bit start-address field (bytes >> 4): one base per operand, one add per MMA.
+            // The issuing thread is a single instruction stream: what it spends per MMA beyond the issue itself is time
+            // the tensor core idles.
+            const uint64_t b_desc = smem_desc_sw128(smem_u32(sB));
+            const uint64_t a_desc = smem_desc_sw128(smem_u32(sIn));
+            const uint32_t b_lo = (uint32_t)b_desc, b_hi = (uint32_t)(b_desc >> 32);
+            const uint32_t a_lo = (uint32_t)a_desc, a_hi = (uint32_t)(a_desc >> 32);
             uint32_t builds = 0;
             TileCursor cur(tile_begin, tps);
             for (int j = 0; j < n_my; ++j, cur.advance(1)) {
@@ -298,14 +306,17 @@ __global__ void __launch_bounds__(kThreads, 1)
                     break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)sc * kD;
-                const uint32_t a_addr = smem_u32(sIn + s * kOpBytes);
+                const uint32_t a_lo_s = a_lo + (uint32_t)s * (kOpBytes >> 4);
 #pragma unroll
                 for (int t = 0; t < C::kSplit; ++t) {
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks) {
-                        const uint32_t koff = (uint32_t)((ks >> 2) * (kTile * 128) + (ks & 3) * 32);
-                        umma_f16_ss(d_tmem, smem_desc_sw128(a_addr + koff), smem_desc_sw128(b_addr + t * kOpBytes + koff), C::kIdesc,
-                                    (t > 0 || ks > 0) ? 1u : 0u);
+                        constexpr uint32_t kBlk = (kTile * 128) >> 4;
+                        const uint32_t koff = (uint32_t)(ks >> 2) * kBlk + (uint32_t)(ks & 3) * 2u;   // (bytes >> 4) of K-step ks
+                        const uint64_t ad = ((uint64_t)a_hi << 32) | (uint64_t)(a_lo_s + koff);
+                        const uint64_t bd = ((uint64_t)b_hi << 32) | (uint64_t)(b_lo + (uint32_t)t * (kOpBytes >> 4) + koff);
+                        if (t > 0 || ks > 0) umma_f16_ss<true>(d_tmem, ad, bd, C::kIdesc);
+                        else umma_f16_ss<false>(d_tmem, ad, bd, C::kIdesc);
                     }
                 }
                 umma_commit(smem_u32(&ctrl->acc_full[sc]));   // to the epilogue; the producer takes it as "x stage free"
