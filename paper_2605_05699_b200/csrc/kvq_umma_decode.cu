@@ -69,6 +69,7 @@ struct Ctrl {
     uint64_t in_full[kInStages], in_empty[kInStages];
     uint64_t a_full[kAStages], a_empty[kAStages];
     uint64_t acc_full[kAccStages], acc_empty[kAccStages];
+    uint64_t b_first;
     uint32_t tmem_base;
     volatile uint32_t abort;
 };
@@ -258,6 +259,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             mbar_init(smem_u32(&ctrl->acc_full[s]), 1);
             mbar_init(smem_u32(&ctrl->acc_empty[s]), 4);
         }
+        mbar_init(smem_u32(&ctrl->b_first), 16);   // first B: the sixteen dequant and epilogue warps build it
         ctrl->abort = 0u;
         mbar_init_fence();
     }
@@ -275,12 +277,6 @@ __global__ void __launch_bounds__(kThreads, 1)
     const int64_t seg_first = n_my > 0 ? tile_begin / tps : 0;
     auto lambda_row = [&](int64_t seg) -> const float * { return prm.g.lambda + (prm.g.n_lambda == 1 ? 0 : seg) * kD; };
 
-    // ---- B for the first tile's lambda row: every warp builds eight rows
-    if (n_my > 0 && warp < 16) {
-        float rho;
-        const float4 rl = recip_lambda4(lambda_row(seg_first), lane, rho);
-        build_b_rows(sB, prm.g.b0, rl, warp * 8, warp * 8 + 8, lane);
-    }
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
@@ -288,6 +284,17 @@ __global__ void __launch_bounds__(kThreads, 1)
     const uint32_t tmem_base = ctrl->tmem_base;
     volatile uint32_t *abort_flag = &ctrl->abort;
     uint32_t *status = prm.g.status;
+
+    // ---- B for the first tile's lambda row: the sixteen dequant and epilogue warps build eight rows each while the
+    // ---- producer's first loads are in flight; the mma warp waits for all of them
+    if (n_my > 0 && warp >= 2) {
+        float rho;
+        const float4 rl = recip_lambda4(lambda_row(seg_first), lane, rho);
+        build_b_rows(sB, prm.g.b0, rl, (warp - 2) * 8, (warp - 2) * 8 + 8, lane);
+        fence_proxy_async();   // B is read by the tensor core through the async proxy
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&ctrl->b_first));
+    }
 
     if (warp == 0) {
         // =========================== producer ===========================
@@ -316,7 +323,9 @@ __global__ void __launch_bounds__(kThreads, 1)
         // =========================== mma issuer ===========================
         if (lane == 0) {
             const uint32_t b_addr = smem_u32(sB);
-            for (int j = 0; j < n_my; ++j) {
+            int n_mma = n_my;
+            if (n_my > 0 && !wait_or_abort(smem_u32(&ctrl->b_first), 0u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT)) n_mma = 0;
+            for (int j = 0; j < n_mma; ++j) {
                 const int sa = j % kAStages, sc = j % kAccStages;
                 if (!wait_or_abort(smem_u32(&ctrl->a_full[sa]), (uint32_t)(j / kAStages) & 1u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT)) break;
                 if (!wait_or_abort(smem_u32(&ctrl->acc_empty[sc]), ((uint32_t)(j / kAccStages) & 1u) ^ 1u, abort_flag, status,
@@ -341,7 +350,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         const int r = q * 32 + lane;            // tile row and tensor-memory lane of this thread
         const uint2 *scales = static_cast<const uint2 *>(prm.g.scales);   // 4 fp16 scales per row
         const uint32_t swz = (uint32_t)((r >> 1) & 3);
-        int64_t cached_seg = n_my > 0 ? seg_first : -1;   // B holds this row's table (built before the roles split)
+        int64_t cached_seg = n_my > 0 ? seg_first : -1;   // B holds this row's table (built above)
         float rho;
         (void)recip_lambda4(lambda_row(seg_first), lane, rho);
 
@@ -363,7 +372,14 @@ __global__ void __launch_bounds__(kThreads, 1)
             if (seg != cached_seg) {
                 const float4 rl = recip_lambda4(lambda_row(seg), lane, rho);
                 if (cur.first_of_segment()) {
-                    // every MMA issued so far has read B: the commit of the previous tile covers them all
+                    // Every MMA issued so far has read B: the commit of the previous tile (the other group's) covers them
+                    // all.  A parity wait can only tell a phase from its neighbours, and the other group may lag by more
+                    // than one of its tiles, so first wait for this group's own last tile (its barrier is at most one
+                    // phase behind, this group waited on it before writing that tile): MMAs complete in order, so after it
+                    // the previous tile's barrier is at most one phase behind too.
+                    if (j >= 2 && !wait_or_abort(smem_u32(&ctrl->a_empty[(j - 2) % kAStages]), (uint32_t)((j - 2) / kAStages) & 1u,
+                                                 abort_flag, status, KVQ_DEV_MMA_TIMEOUT))
+                        break;
                     if (!wait_or_abort(smem_u32(&ctrl->a_empty[(j - 1) % kAStages]), (uint32_t)((j - 1) / kAStages) & 1u, abort_flag,
                                        status, KVQ_DEV_MMA_TIMEOUT))
                         break;

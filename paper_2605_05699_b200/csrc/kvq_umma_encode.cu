@@ -69,7 +69,7 @@ struct Cfg {
 struct Ctrl {
     uint64_t in_full[kInStages];
     uint64_t acc_full[kAccStages], acc_empty[kAccStages];
-    uint64_t b_ready;
+    uint64_t b_first, b_ready;
     uint32_t tmem_base;
     volatile uint32_t abort;
 };
@@ -181,7 +181,7 @@ __device__ __forceinline__ void build_b_rows(unsigned char *sB, const float *__r
                                              int c0, int c1, int lane)
 {
     constexpr int kSplit = Cfg<BF16>::kSplit;
-#pragma unroll 4
+#pragma unroll 8
     for (int c = c0; c < c1; ++c) {
         const float4 m = __ldg(reinterpret_cast<const float4 *>(e0 + (size_t)c * kD) + lane);
         const float f = __ldg(lam + c) * lift;
@@ -235,7 +235,8 @@ __global__ void __launch_bounds__(kThreads, 1)
             mbar_init(smem_u32(&ctrl->acc_full[s]), 1);
             mbar_init(smem_u32(&ctrl->acc_empty[s]), kEpiWarps / 2);
         }
-        mbar_init(smem_u32(&ctrl->b_ready), kEpiWarps / 2);
+        mbar_init(smem_u32(&ctrl->b_first), kEpiWarps);       // first B: all epilogue warps build it
+        mbar_init(smem_u32(&ctrl->b_ready), kEpiWarps / 2);   // later rebuilds: the set that owns the tile
         ctrl->abort = 0u;
         mbar_init_fence();
     }
@@ -296,7 +297,9 @@ __global__ void __launch_bounds__(kThreads, 1)
             TileCursor cur(tile_begin, tps);
             for (int j = 0; j < n_my; ++j, cur.advance(1)) {
                 const int s = j % kInStages, sc = j % kAccStages;
-                if (j == 0 || cur.first_of_segment()) {   // an epilogue set rebuilds B for this lambda row
+                if (j == 0) {   // all epilogue warps build the first B while the first x tiles are in flight
+                    if (!wait_or_abort(smem_u32(&ctrl->b_first), 0u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT)) break;
+                } else if (cur.first_of_segment()) {   // an epilogue set rebuilds B for this lambda row
                     if (!wait_or_abort(smem_u32(&ctrl->b_ready), builds & 1u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT)) break;
                     ++builds;
                 }
@@ -334,6 +337,17 @@ __global__ void __launch_bounds__(kThreads, 1)
         const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(h * 2 * kGroup);
         int64_t cached_seg = -1;
         float unlift = 1.0f;
+        if (n_my > 0) {   // B for the CTA's first lambda row: eight rows per warp, all sixteen warps
+            TileCursor first(tile_begin, tps);
+            const float *lam = prm.lambda + (prm.n_lambda == 1 ? 0 : first.seg) * kD;
+            const float lift = lift_of(lam, lane);
+            build_b_rows<BF16>(sB, prm.e0, lam, lift, (warp - 2) * 8, (warp - 2) * 8 + 8, lane);
+            fence_proxy_async();   // B is read by the tensor core through the async proxy
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctrl->b_first));
+            unlift = 1.0f / lift;
+            cached_seg = first.seg;
+        }
         TileCursor cur(tile_begin + set, tps);
         for (int j = set; j < n_my; j += 2, cur.advance(2)) {
             __syncwarp();
@@ -346,9 +360,9 @@ __global__ void __launch_bounds__(kThreads, 1)
             if (seg != cached_seg) {
                 const float *lam = prm.lambda + (prm.n_lambda == 1 ? 0 : seg) * kD;
                 const float lift = lift_of(lam, lane);
-                if (j == 0 || cur.first_of_segment()) {
-                    if (j > 0 && !wait_or_abort(smem_u32(&ctrl->acc_full[(j - 1) % kAccStages]), (uint32_t)((j - 1) / kAccStages) & 1u,
-                                                abort_flag, status, KVQ_DEV_MMA_TIMEOUT))
+                if (j > 0 && cur.first_of_segment()) {
+                    if (!wait_or_abort(smem_u32(&ctrl->acc_full[(j - 1) % kAccStages]), (uint32_t)((j - 1) / kAccStages) & 1u,
+                                       abort_flag, status, KVQ_DEV_MMA_TIMEOUT))
                         break;
                     build_b_rows<BF16>(sB, prm.e0, lam, lift, bw * 16, bw * 16 + 16, lane);
                     fence_proxy_async();   // B is read by the tensor core through the async proxy

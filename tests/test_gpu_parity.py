@@ -96,6 +96,16 @@ def test_encode_kernel_families_d128(enc_impl, dtype, N, n_lambda, rpl, kind):
     assert enc["mismatches"] <= max(2, int(1e-4 * N * 128))
 
 
+@pytest.mark.parametrize("rpl", [128, 200, 640])
+def test_many_lambda_rows_rebuild_the_gemm_operands_in_flight(rpl):
+    # every few tiles a new lambda row: the tensor-core kernels rebuild their B operand while other tiles are in flight
+    N = 60000
+    n_lambda = (N + rpl - 1) // rpl
+    for rep in range(2):
+        enc, dec = run_case(128, "f16", N, "k_outlier", 9500 + rpl + rep, n_lambda=n_lambda, rows_per_lambda=rpl,
+                            enc_impl="gemm", dec_impl="gemm")
+
+
 def test_lambda_scale_does_not_matter_to_the_gemm_encode():
     # lambda rows far from 1: the power-of-two lift keeps the split terms of W inside fp16's normal range
     for shift in (-12, 9):
