@@ -85,7 +85,7 @@ static kvq_status_t ensure_device(kvq_plan *p)
     }
     p->d_status = st;
     p->table_bytes = 256;
-    if (p->D == 128) {   // the GEMM decode kernel exists for D = 128
+    if (umma_encode_supported(p->D, false) || umma_decode_supported(p->D, false)) {   // tables of the tensor-core kernels
         const size_t bytes = sizeof(float) * (size_t)p->D * p->D;
         float *host = new (std::nothrow) float[(size_t)p->D * p->D];
         float *devp = nullptr;
@@ -268,7 +268,7 @@ static kvq_status_t encode_common(kvq_plan_t *plan, const void *x, kvq_dtype_t d
     kvq_status_t st = check_lambda(N, lambda, n_lambda, rows_per_lambda);
     if (st != KVQ_OK) return st;
     if (misaligned16(x) || misaligned16(packed) || misaligned16(scales)) return KVQ_ERR_ALIGNMENT;
-    const bool gemm_ok = plan->D == 128;
+    const bool gemm_ok = umma_encode_supported(plan->D, dtype == KVQ_BF16);
     if (plan->enc_impl == KVQ_IMPL_GEMM && !gemm_ok) return KVQ_ERR_UNSUPPORTED_DIM;
     if ((st = ensure_device(plan)) != KVQ_OK) return st;
     FftParams prm;
@@ -280,7 +280,7 @@ static kvq_status_t encode_common(kvq_plan_t *plan, const void *x, kvq_dtype_t d
     prm.out_add = out_add;
     // the tensor-core kernel pays a fixed set-up per launch (B operand build); small calls stay on the register FFT
     const bool use_gemm = gemm_ok && (plan->enc_impl == KVQ_IMPL_GEMM || (plan->enc_impl == KVQ_IMPL_AUTO && N >= kGemmEncodeMinRows));
-    cudaError_t e = use_gemm ? umma_encode_d128(dtype == KVQ_BF16, N, prm, plan->d_e0, static_cast<cudaStream_t>(cuda_stream))
+    cudaError_t e = use_gemm ? umma_encode(plan->D, dtype == KVQ_BF16, N, prm, plan->d_e0, static_cast<cudaStream_t>(cuda_stream))
                              : fft_encode(plan->D, dtype == KVQ_BF16, N, prm, static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
@@ -314,7 +314,7 @@ kvq_status_t kvq_decode(kvq_plan_t *plan, const uint8_t *packed, const void *sca
     kvq_status_t st = check_lambda(N, lambda, n_lambda, rows_per_lambda);
     if (st != KVQ_OK) return st;
     if (misaligned16(packed) || misaligned16(scales) || misaligned16(out)) return KVQ_ERR_ALIGNMENT;
-    const bool gemm_ok = plan->D == 128 && dtype == KVQ_F16;
+    const bool gemm_ok = umma_decode_supported(plan->D, dtype == KVQ_BF16);
     if (plan->dec_impl == KVQ_IMPL_GEMM && !gemm_ok) return KVQ_ERR_UNSUPPORTED_DIM;
     if ((st = ensure_device(plan)) != KVQ_OK) return st;
     if (gemm_ok && plan->dec_impl != KVQ_IMPL_FFT) {
@@ -328,7 +328,7 @@ kvq_status_t kvq_decode(kvq_plan_t *plan, const uint8_t *packed, const void *sca
         g.n_lambda = n_lambda;
         g.rows_per_lambda = rows_per_lambda < 1 ? 1 : rows_per_lambda;
         g.status = plan->d_status;
-        if (umma_decode_d128(N, g, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
+        if (umma_decode(plan->D, N, g, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
             (void)cudaGetLastError();
             return KVQ_ERR_CUDA;
         }

@@ -37,10 +37,13 @@ struct GemmParams {
     uint32_t *status;
 };
 
-cudaError_t umma_decode_d128(int64_t N, const GemmParams &prm, cudaStream_t stream);
-// tcgen05 DFT-as-GEMM encode (kvq_umma_encode.cu): takes the register-FFT argument block (sign words unused) and
-// the plan table e0 [D, D] fp32, e0[c][n] = M[c][n] s_n.
-cudaError_t umma_encode_d128(bool bf16, int64_t N, const FftParams &prm, const float *e0, cudaStream_t stream);
+// tcgen05 DFT-as-GEMM kernels (kvq_umma_decode.cu, kvq_umma_encode.cu): which (D, 16-bit type) pairs are built, and the
+// launchers.  Encode takes the register-FFT argument block (its sign words are unused) and the plan table e0 [D, D]
+// fp32, e0[c][n] = M[c][n] s_n; decode takes the table b0 = e0 transposed through GemmParams.
+bool umma_decode_supported(int D, bool bf16);
+bool umma_encode_supported(int D, bool bf16);
+cudaError_t umma_decode(int D, int64_t N, const GemmParams &prm, cudaStream_t stream);
+cudaError_t umma_encode(int D, bool bf16, int64_t N, const FftParams &prm, const float *e0, cudaStream_t stream);
 
 cudaError_t fft_encode(int D, bool bf16, int64_t N, const FftParams &prm, cudaStream_t stream);
 cudaError_t fft_decode(int D, bool bf16, int64_t N, const FftParams &prm, cudaStream_t stream);

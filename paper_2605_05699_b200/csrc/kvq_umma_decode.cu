@@ -1,32 +1,34 @@
-// Warp-specialised tcgen05 DFT-as-GEMM decode kernel of libkvq (sm_100a), D = 128, fp16 output.
+// Warp-specialised tcgen05 DFT-as-GEMM decode kernel of libkvq (sm_100a): D = 64, 96, 128, 160, fp16 output.
 //
 // The inverse path x^ = diag(s) M^T diag(1 / max(lambda, 1e-6)) (q (.) sigma) (Sec. 3.1 "unpack, irfft,
-// apply s"; Sec. 5.1 item 1) is a dense D x D contraction per vector.  A tile of 128 vectors is one
-// 128 x 128 x 128 GEMM on the 5th-generation tensor core, a quarter of the time the tile's bytes need
-// to cross HBM, so the kernel's job is to keep HBM busy: one persistent CTA per SM runs four roles that
-// hand tiles to one another through mbarriers and never wait for one another's latency.
+// apply s"; Sec. 5.1 item 1) is a dense D x D contraction per vector, for any even D (the mixed-radix
+// head dims need no special case here).  A tile of 128 vectors is one 128 x D x D GEMM on the
+// 5th-generation tensor core, a fraction of the time the tile's bytes need to cross HBM, so the kernel's
+// job is to keep HBM busy: one persistent CTA per SM runs four roles that hand tiles to one another
+// through mbarriers and never wait for one another's latency.
 //
-//   warp 0        producer   one TMA tensor load per tile: 128 packed rows (8 KB) into a ring of
-//                            shared-memory stages (64-byte swizzle, so that row-per-thread reads
-//                            are free of bank conflicts)
+//   warp 0        producer   one TMA tensor load per tile: 128 packed rows into a ring of shared-memory
+//                            stages, swizzled (or at a pitch) such that row-per-thread reads are free
+//                            of bank conflicts
 //   warps 2-9     dequant    two groups of four warps that take alternate tiles.  Thread t of a group
 //                            owns row t: nibbles -> fp16 codes -> times sigma * rho, two codes per
 //                            half2 instruction, stored straight into TENSOR MEMORY as the A operand
 //                            (tcgen05.st); the group scales come by plain loads, one tile ahead.
 //                            The group that meets the first tile of a new lambda row rebuilds B.
-//   warp 1        mma        one thread issues 8 K-steps of tcgen05.mma (A from tensor memory, B from
-//                            shared memory) into one of two accumulator stages and commits
+//   warp 1        mma        one thread issues D / 16 K-steps of tcgen05.mma (A from tensor memory, B
+//                            from shared memory) into one of two accumulator stages and commits
 //   warps 10-17   epilogue   two groups of four warps, alternate tiles.  Thread t reads accumulator
-//                            row t (tcgen05.ld), rounds to fp16, writes a 128-byte-swizzled staging
-//                            tile; one lane per warp issues two TMA tensor stores (32 rows x 128 B
-//                            each).  The output tensor map is three-dimensional (column, row within
-//                            lambda segment, segment), so the hardware clips a tile that ends with
-//                            its segment or with the tensor: no per-row tail code.
+//                            row t (tcgen05.ld), rounds to fp16, writes a swizzled staging tile; one
+//                            lane per warp issues the TMA tensor stores (32 rows x 128 B boxes, plus a
+//                            64-byte one when D / 32 is odd).  The output tensor maps are
+//                            three-dimensional (column, row within lambda segment, segment), so the
+//                            hardware clips a tile that ends with its segment or with the tensor: no
+//                            per-row tail code.
 //
-//   A [128 vectors, K = 128]  fp16 in tensor memory: lane = vector, 64 columns of two codes each
-//   B [N = 128 outputs, K]    fp16 in shared memory, K-major, 128-byte swizzle:
-//                             W'[n, c] = s_n M[c, n] / max(lambda_c, 1e-6) / rho, rho a power of two
-//   D [128, 128]              fp32 accumulator in tensor memory, two stages
+//   A [128 vectors, K = D]   fp16 in tensor memory: lane = vector, D / 2 columns of two codes each
+//   B [N = D outputs, K]     fp16 in shared memory, K-major, 128-byte swizzle, K blocks of 64:
+//                            W'[n, c] = s_n M[c, n] / max(lambda_c, 1e-6) / rho, rho a power of two
+//   D [128, D]               fp32 accumulator in tensor memory, two stages
 //
 // The K order inside a word of 8 codes is (0,4,1,5,2,6,3,7): that is how the half2 nibble trick
 // delivers them, and B is built in the same order, so no instruction is spent on reordering.
@@ -35,128 +37,54 @@
 // vector before the output rounding.  Every wait on an mbarrier is bounded: on a time-out the role
 // records the reason in the status word, raises the CTA's abort flag and leaves its loop; the CTA
 // then frees its tensor memory and returns.
-#include <cuda.h>
-
-#include "kvq_device.cuh"
 #include "kvq_internal.h"
+#include "kvq_umma.cuh"
 
 namespace kvq {
 
 namespace {
 
-constexpr int kD = 128;
-constexpr int kTile = 128;                 // vectors per tile = MMA M
-constexpr int kInStages = 6;               // packed tiles in flight
-constexpr int kAStages = 4;                // A operands in tensor memory
-constexpr int kAccStages = 2;              // accumulators in tensor memory
-constexpr int kThreads = 576;              // producer, mma, 2 x 4 dequant, 2 x 4 epilogue warps
-
-constexpr int kBBytes = 2 * kTile * 128;               // 32 KB: two K blocks of [128 rows x 128 B]
-constexpr int kInBytes = kTile * (kD / 2);             // 8 KB per packed tile
-constexpr int kOutWarpBytes = 2 * 32 * 128;            // 8 KB: two column halves of [32 rows x 128 B]
-constexpr int kOutBytes = 8 * kOutWarpBytes;           // one staging tile per epilogue warp
+constexpr int kTile = 128;       // vectors per tile = MMA M
+constexpr int kThreads = 576;    // producer, mma, 2 x 4 dequant, 2 x 4 epilogue warps
+constexpr int kInStages = 6;     // packed tiles in flight
+constexpr int kAccStages = 2;    // accumulators in tensor memory
 constexpr int kCtrlBytes = 256;
-constexpr int kSmemBytes = kBBytes + kInStages * kInBytes + kOutBytes + kCtrlBytes + 1024;
-
-constexpr uint32_t kAccCol0 = 0;                       // 2 x 128 accumulator columns
-constexpr uint32_t kACol0 = kAccStages * kD;           // then 4 x 64 columns of A
 constexpr uint32_t kTmemCols = 512;
 
-// instruction descriptor: D = f32, A = B = f16, both K-major, N = 128, M = 128
-constexpr uint32_t kIdesc = (1u << 4) | ((uint32_t)(kD >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
+template <int D>
+struct Cfg {
+    static_assert(D % 32 == 0 && D >= 64 && D <= 160, "head dim not built");
+    static constexpr int G = D / 32;                       // groups = 16-byte chunks of a packed row = 32-column accumulator chunks
+    static constexpr int kKSteps = D / 16;
+    static constexpr int kKBlocks = (D + 63) / 64;         // K blocks of 64 elements (the last one may be half used)
+    static constexpr int kBBlock = D * 128;                // bytes of one K block: D rows x 128 B
+    static constexpr int kBBytes = kKBlocks * kBBlock;
+    static constexpr int kInRow = D / 2;                   // packed bytes per row
+    static constexpr int kInBytes = kTile * kInRow;        // bytes one TMA load brings
+    static constexpr int kInPitch = (kInBytes + 1023) & ~1023;
+    // The packed tile is read row per thread, 16 bytes at a time.  Row pitches of 48 and 80 bytes spread eight
+    // consecutive rows over all banks by themselves; 32 and 64 bytes need the TMA swizzle of that width.
+    static constexpr int kInSwizzleBits = D == 64 ? 1 : D == 128 ? 2 : 0;
+    static constexpr int kOutWarpBytes = 32 * 2 * D;       // staging of one epilogue warp: G / 2 boxes of 4 KB (+ one of 2 KB)
+    static constexpr int kOutBytes = 8 * kOutWarpBytes;
+    static constexpr int kSmemBytes = kBBytes + kInStages * kInPitch + kOutBytes + kCtrlBytes + 1024;
+    // tensor memory: two accumulators of D columns, then the A stages of D / 2 columns
+    static constexpr uint32_t kAccStride = D <= 128 ? 128 : 256;
+    static constexpr int kAStages = D <= 128 ? 4 : 2;
+    __host__ __device__ static constexpr uint32_t acc_col(int s) { return (uint32_t)s * kAccStride; }
+    __host__ __device__ static constexpr uint32_t a_col(int s) { return D <= 128 ? 256u + 64u * (uint32_t)s : 160u + 256u * (uint32_t)s; }
+    static constexpr uint32_t kIdesc = umma_idesc_m128(D, false);
+};
 
 struct Ctrl {
     uint64_t in_full[kInStages], in_empty[kInStages];
-    uint64_t a_full[kAStages], a_empty[kAStages];
+    uint64_t a_full[4], a_empty[4];
     uint64_t acc_full[kAccStages], acc_empty[kAccStages];
     uint64_t b_first;
     uint32_t tmem_base;
     volatile uint32_t abort;
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
-
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr)
-{
-    // start address >> 4 | LBO 0 | SBO 1024 B (8 rows x 128 B) | version 1 | 128-byte swizzle
-    return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(1024u >> 4) << 32) | (1ull << 46) | (2ull << 61);
-}
-
-__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t cols)
-{
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(cols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols)
-{
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-// D[tmem] (+)= A[tmem] * B[smem]
-__device__ __forceinline__ void umma_f16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
-        "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-
-__device__ __forceinline__ void umma_commit(uint32_t bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr)
-        : "memory");
-}
-
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16])
-{
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
-        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr),
-        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
-        "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
-        : "memory");
-}
-
-__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-
-// TMA tensor load, two coordinates, completion on an mbarrier (no multicast)
-__device__ __forceinline__ void tma_load_2d(uint32_t dst_smem, const CUtensorMap *tm, int c0, int c1, uint32_t bar)
-{
-    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
-                     dst_smem),
-                 "l"(reinterpret_cast<uint64_t>(tm)), "r"(c0), "r"(c1), "r"(bar)
-                 : "memory");
-}
-
-// TMA tensor store, three coordinates; joins the thread's current bulk group
-__device__ __forceinline__ void tma_store_3d(const CUtensorMap *tm, int c0, int c1, int c2, uint32_t src_smem)
-{
-    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%1, %2, %3}], [%4];" ::"l"(
-                     reinterpret_cast<uint64_t>(tm)),
-                 "r"(c0), "r"(c1), "r"(c2), "r"(src_smem)
-                 : "memory");
-}
-
 
 __device__ __forceinline__ uint32_t lop3_and_or(uint32_t a, uint32_t b, uint32_t c)
 {
@@ -165,63 +93,84 @@ __device__ __forceinline__ uint32_t lop3_and_or(uint32_t a, uint32_t b, uint32_t
     return d;
 }
 
-// byte offset of 16-byte chunk j (0..15 along K) of row r in a [2 K blocks][128 rows][128 B] swizzled operand
-__device__ __forceinline__ uint32_t sw128_chunk(int r, int j)
-{
-    return (uint32_t)((j >> 3) * (kTile * 128) + r * 128 + (((j & 7) ^ (r & 7)) << 4));
-}
-
-// 1 / max(lambda, 1e-6) for the four channels 4 lane .. 4 lane + 3 of lambda row `lam`, divided by rho, the
-// power of two that brings the row's largest reciprocal into [1, 2).  Every lane of the warp gets rho.
-__device__ __forceinline__ float4 recip_lambda4(const float *__restrict__ lam, int lane, float &rho)
-{
-    const float4 l = __ldg(reinterpret_cast<const float4 *>(lam) + lane);
-    float4 r = make_float4(__frcp_rn(fmaxf(l.x, 1e-6f)), __frcp_rn(fmaxf(l.y, 1e-6f)), __frcp_rn(fmaxf(l.z, 1e-6f)),
-                           __frcp_rn(fmaxf(l.w, 1e-6f)));
-    float mx = fmaxf(fmaxf(r.x, r.y), fmaxf(r.z, r.w));
+// 1 / max(lambda, 1e-6) for the channels this lane covers (4 i .. 4 i + 3, i = lane and, for D > 128, lane + 32),
+// divided by rho, the power of two that brings the row's largest reciprocal into [1, 2).  Every lane gets rho.
+template <int D>
+struct RecipLambda {
+    static constexpr int kPasses = (D / 4 + 31) / 32;
+    float4 r[kPasses];
+    float rho;
+    __device__ __forceinline__ RecipLambda(const float *__restrict__ lam, int lane)
+    {
+        float mx = 0.0f;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
-    rho = __uint_as_float(__float_as_uint(mx) & 0x7F800000u);   // 2^floor(log2 max): exact to divide by
-    r.x /= rho, r.y /= rho, r.z /= rho, r.w /= rho;
-    return r;
-}
+        for (int p = 0; p < kPasses; ++p) {
+            const int i = lane + 32 * p;
+            r[p] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            if (i < D / 4) {
+                const float4 l = __ldg(reinterpret_cast<const float4 *>(lam) + i);
+                r[p] = make_float4(__frcp_rn(fmaxf(l.x, 1e-6f)), __frcp_rn(fmaxf(l.y, 1e-6f)), __frcp_rn(fmaxf(l.z, 1e-6f)),
+                                   __frcp_rn(fmaxf(l.w, 1e-6f)));
+            }
+            mx = fmaxf(mx, fmaxf(fmaxf(r[p].x, r[p].y), fmaxf(r[p].z, r[p].w)));
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+        rho = __uint_as_float(__float_as_uint(mx) & 0x7F800000u);   // 2^floor(log2 max): exact to divide by
+#pragma unroll
+        for (int p = 0; p < kPasses; ++p) r[p].x /= rho, r[p].y /= rho, r[p].z /= rho, r[p].w /= rho;
+    }
+};
 
-// Rows [n0, n1) of the B operand, by one warp: lane l reads the four table entries b0[n][4l .. 4l+3]
-// (one coalesced 512-byte row per step), scales them, trades two values with its neighbour so that each
-// lane holds two K-ordered pairs, and writes 8 bytes of the swizzled row.
-__device__ __forceinline__ void build_b_rows(unsigned char *sB, const float *__restrict__ b0, float4 rl, int n0, int n1, int lane)
+// Rows [n0, n1) of the B operand, by one warp: a lane reads four table entries b0[n][4 i .. 4 i + 3] (coalesced
+// rows), scales them, trades two values with its neighbour so that each lane holds two K-ordered pairs, and
+// writes 8 bytes of the swizzled row.
+template <int D>
+__device__ __forceinline__ void build_b_rows(unsigned char *sB, const float *__restrict__ b0, const RecipLambda<D> &rl, int n0, int n1,
+                                             int lane)
 {
     const bool odd = lane & 1;
-    const int w = lane >> 1;   // word of 8 codes = 16-byte chunk of the K-major row
-#pragma unroll 8
+#pragma unroll 4
     for (int n = n0; n < n1; ++n) {
-        const float4 m = __ldg(reinterpret_cast<const float4 *>(b0 + (size_t)n * kD) + lane);
-        auto sat = [](float v) { return fminf(fmaxf(v, -65504.0f), 65504.0f); };
-        const float vx = sat(m.x * rl.x), vy = sat(m.y * rl.y), vz = sat(m.z * rl.z), vw = sat(m.w * rl.w);
-        // even lane holds codes 8w .. 8w+3, odd lane 8w+4 .. 8w+7; K order of the word is (0,4,1,5,2,6,3,7)
-        const float r0 = __shfl_xor_sync(0xFFFFFFFFu, odd ? vx : vz, 1);
-        const float r1 = __shfl_xor_sync(0xFFFFFFFFu, odd ? vy : vw, 1);
-        uint2 o;
-        o.x = odd ? narrow2<false>(r0, vz) : narrow2<false>(vx, r0);   // odd: (2, 6)   even: (0, 4)
-        o.y = odd ? narrow2<false>(r1, vw) : narrow2<false>(vy, r1);   // odd: (3, 7)   even: (1, 5)
-        *reinterpret_cast<uint2 *>(sB + sw128_chunk(n, w) + (odd ? 8 : 0)) = o;
+#pragma unroll
+        for (int p = 0; p < RecipLambda<D>::kPasses; ++p) {
+            const int i = lane + 32 * p;
+            const bool live = i < D / 4;
+            float4 m = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            if (live) m = __ldg(reinterpret_cast<const float4 *>(b0 + (size_t)n * D) + i);
+            auto sat = [](float v) { return fminf(fmaxf(v, -65504.0f), 65504.0f); };
+            const float vx = sat(m.x * rl.r[p].x), vy = sat(m.y * rl.r[p].y), vz = sat(m.z * rl.r[p].z), vw = sat(m.w * rl.r[p].w);
+            // even lane holds codes 8w .. 8w+3, odd lane 8w+4 .. 8w+7; K order of the word is (0,4,1,5,2,6,3,7)
+            const float r0 = __shfl_xor_sync(0xFFFFFFFFu, odd ? vx : vz, 1);
+            const float r1 = __shfl_xor_sync(0xFFFFFFFFu, odd ? vy : vw, 1);
+            uint2 o;
+            o.x = odd ? narrow2<false>(r0, vz) : narrow2<false>(vx, r0);   // odd: (2, 6)   even: (0, 4)
+            o.y = odd ? narrow2<false>(r1, vw) : narrow2<false>(vy, r1);   // odd: (3, 7)   even: (1, 5)
+            const int w = i >> 1;   // word of 8 codes = 16-byte chunk w of the K-major row: K block w / 8, chunk w % 8
+            if (live)
+                *reinterpret_cast<uint2 *>(sB + (w >> 3) * Cfg<D>::kBBlock + n * 128 + (((w & 7) ^ (n & 7)) << 4) + (odd ? 8 : 0)) = o;
+        }
     }
 }
 
-// Bounded wait that also gives up when another role of the CTA has raised the abort flag.
-__device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *status,
-                                              uint32_t reason)
+// The D / 32 fp16 group scales of one row, as packed 16-bit pairs.
+template <int G>
+__device__ __forceinline__ void load_row_scales(const uint16_t *__restrict__ sp, uint32_t (&sb)[(G + 1) / 2])
 {
-    for (uint32_t it = 0; it < (1u << 22); ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (it > 32) {
-            if (*abort_flag) return false;
-            __nanosleep(32);
-        }
+    if constexpr (G == 8) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4 *>(sp));
+        sb[0] = v.x, sb[1] = v.y, sb[2] = v.z, sb[3] = v.w;
+    } else if constexpr (G == 4) {
+        const uint2 v = __ldg(reinterpret_cast<const uint2 *>(sp));
+        sb[0] = v.x, sb[1] = v.y;
+    } else if constexpr (G == 2) {
+        sb[0] = __ldg(reinterpret_cast<const uint32_t *>(sp));
+    } else {   // rows of 6 or 10 bytes are only 2-byte aligned
+#pragma unroll
+        for (int j = 0; j < (G + 1) / 2; ++j) sb[j] = 0;
+#pragma unroll
+        for (int j = 0; j < G; ++j) sb[j / 2] |= (uint32_t)__ldg(sp + j) << (16 * (j & 1));
     }
-    *abort_flag = 1u;
-    atomicOr(status, reason);
-    return false;
 }
 
 }  // namespace
@@ -230,19 +179,27 @@ struct UmmaDecodeParams {
     GemmParams g;
     int64_t rpl;        // rows per lambda segment (N when there is one lambda row)
     int64_t n_seg;      // segments
-    int64_t n_full;     // segments of exactly rpl rows, covered by the main output map; a shorter last one uses the tail map
+    int64_t n_full;     // segments of exactly rpl rows, covered by the main output maps; a shorter last one uses the tail maps
 };
 
+struct UmmaDecodeMaps {
+    CUtensorMap packed;            // [N, D / 2] bytes, box 128 rows
+    CUtensorMap wide, wide_tail;   // output, boxes of 64 columns x 32 rows (128-byte swizzle)
+    CUtensorMap slim, slim_tail;   // output, boxes of 32 columns x 32 rows (64-byte swizzle), used when D / 32 is odd
+};
+
+template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
-    kvq_decode_umma_d128_kernel(const __grid_constant__ UmmaDecodeParams prm, const __grid_constant__ CUtensorMap tm_packed,
-                                const __grid_constant__ CUtensorMap tm_out, const __grid_constant__ CUtensorMap tm_out_tail)
+    kvq_decode_umma_kernel(const __grid_constant__ UmmaDecodeParams prm, const __grid_constant__ UmmaDecodeMaps maps)
 {
+    using C = Cfg<D>;
+    constexpr int G = C::G;
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     unsigned char *sB = smem;
-    unsigned char *sIn = sB + kBBytes;
-    unsigned char *sOut = sIn + kInStages * kInBytes;
-    Ctrl *ctrl = reinterpret_cast<Ctrl *>(sOut + kOutBytes);
+    unsigned char *sIn = sB + C::kBBytes;
+    unsigned char *sOut = sIn + kInStages * C::kInPitch;
+    Ctrl *ctrl = reinterpret_cast<Ctrl *>(sOut + C::kOutBytes);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -251,7 +208,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             mbar_init(smem_u32(&ctrl->in_full[s]), 1);
             mbar_init(smem_u32(&ctrl->in_empty[s]), 4);
         }
-        for (int s = 0; s < kAStages; ++s) {
+        for (int s = 0; s < C::kAStages; ++s) {
             mbar_init(smem_u32(&ctrl->a_full[s]), 4);
             mbar_init(smem_u32(&ctrl->a_empty[s]), 1);
         }
@@ -275,7 +232,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     const int64_t tile_end = tile_begin + per_cta < n_tiles ? tile_begin + per_cta : n_tiles;
     const int n_my = tile_end > tile_begin ? (int)(tile_end - tile_begin) : 0;
     const int64_t seg_first = n_my > 0 ? tile_begin / tps : 0;
-    auto lambda_row = [&](int64_t seg) -> const float * { return prm.g.lambda + (prm.g.n_lambda == 1 ? 0 : seg) * kD; };
+    auto lambda_row = [&](int64_t seg) -> const float * { return prm.g.lambda + (prm.g.n_lambda == 1 ? 0 : seg) * D; };
 
     fence_proxy_async();
     tc_fence_before();
@@ -285,12 +242,11 @@ __global__ void __launch_bounds__(kThreads, 1)
     volatile uint32_t *abort_flag = &ctrl->abort;
     uint32_t *status = prm.g.status;
 
-    // ---- B for the first tile's lambda row: the sixteen dequant and epilogue warps build eight rows each while the
+    // ---- B for the first tile's lambda row: the sixteen dequant and epilogue warps build D / 16 rows each while the
     // ---- producer's first loads are in flight; the mma warp waits for all of them
     if (n_my > 0 && warp >= 2) {
-        float rho;
-        const float4 rl = recip_lambda4(lambda_row(seg_first), lane, rho);
-        build_b_rows(sB, prm.g.b0, rl, (warp - 2) * 8, (warp - 2) * 8 + 8, lane);
+        const RecipLambda<D> rl(lambda_row(seg_first), lane);
+        build_b_rows<D>(sB, prm.g.b0, rl, (warp - 2) * (D / 16), (warp - 1) * (D / 16), lane);
         fence_proxy_async();   // B is read by the tensor core through the async proxy
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&ctrl->b_first));
@@ -309,8 +265,8 @@ __global__ void __launch_bounds__(kThreads, 1)
                 if (!ok) break;
                 const int64_t row0 = cur.seg * rpl + cur.row_in_segment();
                 const uint32_t bar = smem_u32(&ctrl->in_full[s]);
-                mbar_arrive_expect_tx(bar, kInBytes);
-                tma_load_2d(smem_u32(sIn + s * kInBytes), &tm_packed, 0, (int)row0, bar);
+                mbar_arrive_expect_tx(bar, C::kInBytes);
+                tma_load_2d(smem_u32(sIn + s * C::kInPitch), &maps.packed, 0, (int)row0, bar);
                 issued = j + 1;
             }
             if (!ok) {
@@ -322,22 +278,25 @@ __global__ void __launch_bounds__(kThreads, 1)
     } else if (warp == 1) {
         // =========================== mma issuer ===========================
         if (lane == 0) {
-            const uint32_t b_addr = smem_u32(sB);
+            const uint64_t b_desc = smem_desc_sw128(smem_u32(sB));
+            const uint32_t b_lo = (uint32_t)b_desc, b_hi = (uint32_t)(b_desc >> 32);
             int n_mma = n_my;
             if (n_my > 0 && !wait_or_abort(smem_u32(&ctrl->b_first), 0u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT)) n_mma = 0;
             for (int j = 0; j < n_mma; ++j) {
-                const int sa = j % kAStages, sc = j % kAccStages;
-                if (!wait_or_abort(smem_u32(&ctrl->a_full[sa]), (uint32_t)(j / kAStages) & 1u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT)) break;
+                const int sa = j % C::kAStages, sc = j % kAccStages;
+                if (!wait_or_abort(smem_u32(&ctrl->a_full[sa]), (uint32_t)(j / C::kAStages) & 1u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT)) break;
                 if (!wait_or_abort(smem_u32(&ctrl->acc_empty[sc]), ((uint32_t)(j / kAccStages) & 1u) ^ 1u, abort_flag, status,
                                    KVQ_DEV_SLOT_TIMEOUT))
                     break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + kAccCol0 + (uint32_t)sc * kD;
-                const uint32_t a_tmem = tmem_base + kACol0 + (uint32_t)sa * (kD / 2);
+                const uint32_t d_tmem = tmem_base + C::acc_col(sc);
+                const uint32_t a_tmem = tmem_base + C::a_col(sa);
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const uint32_t koff = (uint32_t)((ks >> 2) * (kTile * 128) + (ks & 3) * 32);
-                    umma_f16_ts(d_tmem, a_tmem + (uint32_t)ks * 8u, smem_desc_sw128(b_addr + koff), kIdesc, ks > 0 ? 1u : 0u);
+                for (int ks = 0; ks < C::kKSteps; ++ks) {
+                    const uint32_t koff = (uint32_t)(ks >> 2) * (C::kBBlock >> 4) + (uint32_t)(ks & 3) * 2u;   // (bytes >> 4) of K-step ks
+                    const uint64_t bd = ((uint64_t)b_hi << 32) | (uint64_t)(b_lo + koff);
+                    if (ks > 0) umma_f16_ts<true>(d_tmem, a_tmem + (uint32_t)ks * 8u, bd, C::kIdesc);
+                    else umma_f16_ts<false>(d_tmem, a_tmem, bd, C::kIdesc);
                 }
                 umma_commit(smem_u32(&ctrl->acc_full[sc]));
                 umma_commit(smem_u32(&ctrl->a_empty[sa]));
@@ -348,71 +307,75 @@ __global__ void __launch_bounds__(kThreads, 1)
         const int grp = (warp - 2) >> 2;        // this group takes tiles grp, grp + 2, ...
         const int q = warp & 3;                 // tensor-memory lane quarter this warp may touch
         const int r = q * 32 + lane;            // tile row and tensor-memory lane of this thread
-        const uint2 *scales = static_cast<const uint2 *>(prm.g.scales);   // 4 fp16 scales per row
-        const uint32_t swz = (uint32_t)((r >> 1) & 3);
+        const uint16_t *scales = static_cast<const uint16_t *>(prm.g.scales);   // D / 32 fp16 scales per row
+        const uint32_t swz = C::kInSwizzleBits == 2 ? (uint32_t)((r >> 1) & 3) : C::kInSwizzleBits == 1 ? (uint32_t)((r >> 2) & 1) : 0u;
         int64_t cached_seg = n_my > 0 ? seg_first : -1;   // B holds this row's table (built above)
-        float rho;
-        (void)recip_lambda4(lambda_row(seg_first), lane, rho);
+        float rho = RecipLambda<D>(lambda_row(seg_first), lane).rho;
 
         TileCursor cur(tile_begin + grp, tps), ahead(tile_begin + grp, tps);   // this tile; the tile whose scales are fetched
-        auto load_scales = [&](int j) -> uint2 {
-            if (j >= n_my) return make_uint2(0u, 0u);
-            const int64_t row = ahead.seg * rpl + ahead.row_in_segment() + r;
-            return row < N ? __ldg(scales + row) : make_uint2(0u, 0u);
+        uint32_t sc_next[(G + 1) / 2];
+        auto fetch_scales = [&](int j) {
+#pragma unroll
+            for (int i = 0; i < (G + 1) / 2; ++i) sc_next[i] = 0u;
+            if (j < n_my) {
+                const int64_t row = ahead.seg * rpl + ahead.row_in_segment() + r;
+                if (row < N) load_row_scales<G>(scales + row * G, sc_next);
+            }
         };
 
-        uint2 sc_next = load_scales(grp);
+        fetch_scales(grp);
         for (int j = grp; j < n_my; j += 2, cur.advance(2)) {
-            const uint2 sc = sc_next;
+            uint32_t sc[(G + 1) / 2];
+#pragma unroll
+            for (int i = 0; i < (G + 1) / 2; ++i) sc[i] = sc_next[i];
             ahead.advance(2);
-            sc_next = load_scales(j + 2);
+            fetch_scales(j + 2);
             const int64_t seg = cur.seg;
 
             // ---- a new lambda row: this group needs its rho; the group that meets the row's first tile rebuilds B
             if (seg != cached_seg) {
-                const float4 rl = recip_lambda4(lambda_row(seg), lane, rho);
+                const RecipLambda<D> rl(lambda_row(seg), lane);
+                rho = rl.rho;
                 if (cur.first_of_segment()) {
                     // Every MMA issued so far has read B: the commit of the previous tile (the other group's) covers them
                     // all.  A parity wait can only tell a phase from its neighbours, and the other group may lag by more
                     // than one of its tiles, so first wait for this group's own last tile (its barrier is at most one
                     // phase behind, this group waited on it before writing that tile): MMAs complete in order, so after it
                     // the previous tile's barrier is at most one phase behind too.
-                    if (j >= 2 && !wait_or_abort(smem_u32(&ctrl->a_empty[(j - 2) % kAStages]), (uint32_t)((j - 2) / kAStages) & 1u,
+                    if (j >= 2 && !wait_or_abort(smem_u32(&ctrl->a_empty[(j - 2) % C::kAStages]), (uint32_t)((j - 2) / C::kAStages) & 1u,
                                                  abort_flag, status, KVQ_DEV_MMA_TIMEOUT))
                         break;
-                    if (!wait_or_abort(smem_u32(&ctrl->a_empty[(j - 1) % kAStages]), (uint32_t)((j - 1) / kAStages) & 1u, abort_flag,
+                    if (!wait_or_abort(smem_u32(&ctrl->a_empty[(j - 1) % C::kAStages]), (uint32_t)((j - 1) / C::kAStages) & 1u, abort_flag,
                                        status, KVQ_DEV_MMA_TIMEOUT))
                         break;
-                    build_b_rows(sB, prm.g.b0, rl, q * 32, q * 32 + 32, lane);
+                    build_b_rows<D>(sB, prm.g.b0, rl, q * (D / 4), (q + 1) * (D / 4), lane);
                     fence_proxy_async();   // B is read by the tensor core through the async proxy
                 }
                 cached_seg = seg;
             }
 
             // ---- this tile's packed rows have landed; the A stage is free again
-            const int s = j % kInStages, sa = j % kAStages;
+            const int s = j % kInStages, sa = j % C::kAStages;
             if (!wait_or_abort(smem_u32(&ctrl->in_full[s]), (uint32_t)(j / kInStages) & 1u, abort_flag, status, KVQ_DEV_LOAD_TIMEOUT)) break;
-            uint4 pk[4];
+            uint4 pk[G];
             {
-                const unsigned char *row = sIn + s * kInBytes + r * (kD / 2);
+                const unsigned char *row = sIn + s * C::kInPitch + r * C::kInRow;
 #pragma unroll
-                for (int c = 0; c < 4; ++c) pk[c] = *reinterpret_cast<const uint4 *>(row + (((uint32_t)c ^ swz) << 4));
+                for (int c = 0; c < G; ++c) pk[c] = *reinterpret_cast<const uint4 *>(row + (((uint32_t)c ^ swz) << 4));
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctrl->in_empty[s]));   // the values are in registers
-            if (!wait_or_abort(smem_u32(&ctrl->a_empty[sa]), ((uint32_t)(j / kAStages) & 1u) ^ 1u, abort_flag, status, KVQ_DEV_MMA_TIMEOUT))
+            if (!wait_or_abort(smem_u32(&ctrl->a_empty[sa]), ((uint32_t)(j / C::kAStages) & 1u) ^ 1u, abort_flag, status, KVQ_DEV_MMA_TIMEOUT))
                 break;
             tc_fence_after();
 
             // ---- nibbles -> fp16 codes -> times sigma * rho, two codes per instruction
-            const uint32_t a_row = tmem_base + ((uint32_t)(q * 32) << 16) + kACol0 + (uint32_t)sa * (kD / 2);
-            const __half2 sa2 = *reinterpret_cast<const __half2 *>(&sc.x), sb2 = *reinterpret_cast<const __half2 *>(&sc.y);
-            const float2 fa = __half22float2(sa2), fb = __half22float2(sb2);
-            const float sg[4] = {fa.x * rho, fa.y * rho, fb.x * rho, fb.y * rho};
+            const uint32_t a_row = tmem_base + ((uint32_t)(q * 32) << 16) + C::a_col(sa);
             const __half2 h1032 = __float2half2_rn(1032.0f);
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {   // chunk c = group c: 32 codes, 16 tensor-memory columns
-                const __half2 s2 = __float2half2_rn(sg[c]);
+            for (int c = 0; c < G; ++c) {   // chunk c = group c: 32 codes, 16 tensor-memory columns
+                const float sig = __half2float(__ushort_as_half((unsigned short)((sc[c >> 1] >> (16 * (c & 1))) & 0xFFFFu)));
+                const __half2 s2 = __float2half2_rn(sig * rho);
                 const uint32_t words[4] = {pk[c].x, pk[c].y, pk[c].z, pk[c].w};
                 uint32_t a[16];
 #pragma unroll
@@ -436,8 +399,8 @@ __global__ void __launch_bounds__(kThreads, 1)
         // =========================== epilogue: accumulator -> fp16 -> TMA store ===========================
         const int grp = (warp - 10) >> 2;
         const int q = warp & 3;
-        unsigned char *stg = sOut + (warp - 10) * kOutWarpBytes;   // this warp's staging tile: two [32 rows x 128 B] halves
-        const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16) + kAccCol0;
+        unsigned char *stg = sOut + (warp - 10) * C::kOutWarpBytes;   // this warp's staging tile
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
         TileCursor cur(tile_begin + grp, tps);
         for (int j = grp; j < n_my; j += 2, cur.advance(2)) {
             const int sc = j % kAccStages;
@@ -446,11 +409,13 @@ __global__ void __launch_bounds__(kThreads, 1)
             if (lane == 0) bulk_wait_read_all();   // this warp's previous stores have read the staging tile
             __syncwarp();
 #pragma unroll
-            for (int cc = 0; cc < 4; ++cc) {   // 32 accumulator columns = 64 bytes of the output row
+            for (int cc = 0; cc < G; ++cc) {   // 32 accumulator columns = 64 bytes of the output row
                 uint32_t v[32];
-                tmem_ld32(lane_addr + (uint32_t)sc * kD + (uint32_t)cc * 32u, v);
+                tmem_ld32(lane_addr + C::acc_col(sc) + (uint32_t)cc * 32u, v);
                 tmem_ld_wait();
-                unsigned char *half_base = stg + (cc >> 1) * (32 * 128) + lane * 128;   // column half = one store box
+                constexpr int kWideBoxes = G / 2;
+                const bool wide = (cc >> 1) < kWideBoxes;   // inside a 64-column box, or the last 32-column one
+                unsigned char *box = stg + (cc >> 1) * (32 * 128);
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     uint4 o;
@@ -458,8 +423,12 @@ __global__ void __launch_bounds__(kThreads, 1)
                     o.y = narrow2<false>(__uint_as_float(v[8 * k + 2]), __uint_as_float(v[8 * k + 3]));
                     o.z = narrow2<false>(__uint_as_float(v[8 * k + 4]), __uint_as_float(v[8 * k + 5]));
                     o.w = narrow2<false>(__uint_as_float(v[8 * k + 6]), __uint_as_float(v[8 * k + 7]));
-                    const int chunk = (cc & 1) * 4 + k;   // 16-byte chunk of the 128-byte half row
-                    *reinterpret_cast<uint4 *>(half_base + ((chunk ^ (lane & 7)) << 4)) = o;
+                    if (wide) {   // [32 rows][128 B], 128-byte swizzle
+                        const int chunk = (cc & 1) * 4 + k;
+                        *reinterpret_cast<uint4 *>(box + lane * 128 + ((chunk ^ (lane & 7)) << 4)) = o;
+                    } else {      // [32 rows][64 B], 64-byte swizzle
+                        *reinterpret_cast<uint4 *>(box + lane * 64 + ((k ^ ((lane >> 1) & 3)) << 4)) = o;
+                    }
                 }
             }
             tc_fence_before();
@@ -470,10 +439,14 @@ __global__ void __launch_bounds__(kThreads, 1)
                 const int64_t seg = cur.seg;
                 const int row_in_seg = (int)cur.row_in_segment() + q * 32;
                 const bool tail = seg >= prm.n_full;
-                const CUtensorMap *tm = tail ? &tm_out_tail : &tm_out;
                 const int segc = tail ? 0 : (int)seg;
-                tma_store_3d(tm, 0, row_in_seg, segc, smem_u32(stg));
-                tma_store_3d(tm, 64, row_in_seg, segc, smem_u32(stg + 32 * 128));
+                const CUtensorMap *tw = tail ? &maps.wide_tail : &maps.wide;
+#pragma unroll
+                for (int b = 0; b < G / 2; ++b) tma_store_3d(tw, 64 * b, row_in_seg, segc, smem_u32(stg + b * (32 * 128)));
+                if constexpr (G & 1) {
+                    const CUtensorMap *ts = tail ? &maps.slim_tail : &maps.slim;
+                    tma_store_3d(ts, 64 * (G / 2), row_in_seg, segc, smem_u32(stg + (G / 2) * (32 * 128)));
+                }
                 bulk_commit();
             }
         }
@@ -493,41 +466,19 @@ __global__ void __launch_bounds__(kThreads, 1)
 // ------------------------------------------------------------------------------------------------
 namespace {
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
-                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_tiled_fn()
+template <int D>
+cudaError_t launch(int64_t N, const GemmParams &g, cudaStream_t stream)
 {
-    static EncodeTiledFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-        else
-            (void)cudaGetLastError();
-    }
-    return fn;
-}
-
-}  // namespace
-
-cudaError_t umma_decode_d128(int64_t N, const GemmParams &g, cudaStream_t stream)
-{
+    using C = Cfg<D>;
     static int sms = 0;
     if (sms == 0) {
-        cudaError_t e = cudaFuncSetAttribute(kvq_decode_umma_d128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(kvq_decode_umma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
         if (e != cudaSuccess) return e;
         int dev = 0;
         if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
         if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
     }
-    EncodeTiledFn enc = encode_tiled_fn();
-    if (!enc) return cudaErrorNotSupported;
+    if (!tensor_map_encode_fn()) return cudaErrorNotSupported;
     if (N >= (int64_t)1 << 31) return cudaErrorInvalidValue;   // tensor-map coordinates are 32-bit
 
     UmmaDecodeParams prm;
@@ -536,42 +487,52 @@ cudaError_t umma_decode_d128(int64_t N, const GemmParams &g, cudaStream_t stream
     prm.n_seg = (N + prm.rpl - 1) / prm.rpl;
     prm.n_full = N / prm.rpl;
 
-    CUtensorMap tm_packed, tm_out, tm_tail;
+    UmmaDecodeMaps maps;
     {
-        const cuuint64_t dims[2] = {(cuuint64_t)(kD / 2), (cuuint64_t)N};
-        const cuuint64_t strides[1] = {(cuuint64_t)(kD / 2)};
-        const cuuint32_t box[2] = {(cuuint32_t)(kD / 2), (cuuint32_t)kTile};
-        const cuuint32_t es[2] = {1, 1};
-        if (enc(&tm_packed, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(g.packed), dims, strides, box, es,
-                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-            return cudaErrorInvalidValue;
+        const cuuint64_t dims[2] = {(cuuint64_t)C::kInRow, (cuuint64_t)N};
+        const cuuint64_t strides[1] = {(cuuint64_t)C::kInRow};
+        const cuuint32_t box[2] = {(cuuint32_t)C::kInRow, (cuuint32_t)kTile};
+        const CUtensorMapSwizzle sw = C::kInSwizzleBits == 2 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                      : C::kInSwizzleBits == 1 ? CU_TENSOR_MAP_SWIZZLE_32B
+                                                               : CU_TENSOR_MAP_SWIZZLE_NONE;
+        if (!make_tensor_map(&maps.packed, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, g.packed, dims, strides, box, sw)) return cudaErrorInvalidValue;
     }
-    auto out_map = [&](CUtensorMap *tm, void *base, int64_t rows, int64_t segs) -> bool {
-        const cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)rows, (cuuint64_t)segs};
-        const cuuint64_t strides[2] = {(cuuint64_t)(2 * kD), (cuuint64_t)(2 * kD) * (cuuint64_t)rows};
-        const cuuint32_t box[3] = {64, 32, 1};
-        const cuuint32_t es[3] = {1, 1, 1};
-        return enc(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    auto out_map = [&](CUtensorMap *tm, void *base, int64_t rows, int64_t segs, bool wide) -> bool {
+        const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)rows, (cuuint64_t)segs};
+        const cuuint64_t strides[2] = {(cuuint64_t)(2 * D), (cuuint64_t)(2 * D) * (cuuint64_t)rows};
+        const cuuint32_t box[3] = {wide ? 64u : 32u, 32u, 1u};
+        return make_tensor_map(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, base, dims, strides, box,
+                               wide ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B);
     };
     const int64_t tail_rows = N - prm.n_full * prm.rpl;
-    if (prm.n_full > 0) {
-        if (!out_map(&tm_out, g.out, prm.rpl, prm.n_full)) return cudaErrorInvalidValue;
-    }
-    if (tail_rows > 0) {
-        unsigned char *base = static_cast<unsigned char *>(g.out) + (size_t)prm.n_full * prm.rpl * (2 * kD);
-        if (!out_map(&tm_tail, base, tail_rows, 1)) return cudaErrorInvalidValue;
-    } else {
-        tm_tail = tm_out;
-    }
-    if (prm.n_full == 0) tm_out = tm_tail;
+    unsigned char *tail_base = static_cast<unsigned char *>(g.out) + (size_t)prm.n_full * prm.rpl * (2 * D);
+    if (prm.n_full > 0 && (!out_map(&maps.wide, g.out, prm.rpl, prm.n_full, true) || !out_map(&maps.slim, g.out, prm.rpl, prm.n_full, false)))
+        return cudaErrorInvalidValue;
+    if (tail_rows > 0 && (!out_map(&maps.wide_tail, tail_base, tail_rows, 1, true) || !out_map(&maps.slim_tail, tail_base, tail_rows, 1, false)))
+        return cudaErrorInvalidValue;
+    if (tail_rows == 0) maps.wide_tail = maps.wide, maps.slim_tail = maps.slim;
+    if (prm.n_full == 0) maps.wide = maps.wide_tail, maps.slim = maps.slim_tail;
 
     const int64_t tiles = prm.n_seg * ((prm.rpl + kTile - 1) / kTile);
     const int grid = (int)(tiles < sms ? tiles : sms);
-    kvq_decode_umma_d128_kernel<<<grid, kThreads, kSmemBytes, stream>>>(prm, tm_packed, tm_out, tm_tail);
+    kvq_decode_umma_kernel<D><<<grid, kThreads, C::kSmemBytes, stream>>>(prm, maps);
     count_launch();
     return cudaGetLastError();
+}
+
+}  // namespace
+
+bool umma_decode_supported(int D, bool bf16) { return !bf16 && (D == 64 || D == 96 || D == 128 || D == 160); }
+
+cudaError_t umma_decode(int D, int64_t N, const GemmParams &g, cudaStream_t stream)
+{
+    switch (D) {
+        case 64: return launch<64>(N, g, stream);
+        case 96: return launch<96>(N, g, stream);
+        case 128: return launch<128>(N, g, stream);
+        case 160: return launch<160>(N, g, stream);
+    }
+    return cudaErrorInvalidValue;
 }
 
 }  // namespace kvq

@@ -140,7 +140,7 @@ def test_gemm_encode_serves_large_appends():
 
 
 def test_gemm_kernels_are_refused_where_they_are_not_built():
-    for D, dtype in [(256, torch.float16), (128, torch.bfloat16), (96, torch.float16)]:
+    for D, dtype in [(256, torch.float16), (128, torch.bfloat16), (96, torch.bfloat16)]:
         plan = kb.Plan(D, G, 1)
         kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_AUTO, kb.KVQ_IMPL_GEMM)
         pk, sc = plan.empty_packed(8), plan.empty_scales(8)
@@ -149,10 +149,10 @@ def test_gemm_kernels_are_refused_where_they_are_not_built():
             kb.kvq_decode(plan.handle, pk, sc, torch.ones(D, device="cuda"), out)
         assert e.value.status == kb.KVQ_ERR_UNSUPPORTED_DIM
         plan.close()
-    for D in (96, 256):
+    for D, dtype in [(256, torch.float16), (256, torch.bfloat16), (160, torch.bfloat16)]:
         plan = kb.Plan(D, G, 1)
         kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_GEMM, kb.KVQ_IMPL_AUTO)
-        x = torch.zeros(8, D, dtype=torch.float16, device="cuda")
+        x = torch.zeros(8, D, dtype=dtype, device="cuda")
         with pytest.raises(kb.KvqError) as e:
             kb.kvq_encode(plan.handle, x, torch.ones(D, device="cuda"), plan.empty_packed(8), plan.empty_scales(8))
         assert e.value.status == kb.KVQ_ERR_UNSUPPORTED_DIM
@@ -182,7 +182,17 @@ def test_lambda_scale_does_not_matter_to_the_gemm_decode():
 @pytest.mark.parametrize("dtype", ["f16", "bf16"])
 @pytest.mark.parametrize("D", [64, 96, 128, 160, 256])
 def test_all_dims_ragged_with_straddling_lambda_rows(D, dtype):
-    run_case(D, dtype, 1000, "k_outlier", 2000 + D, n_lambda=4, rows_per_lambda=333)
+    run_case(D, dtype, 1000, "k_outlier", 2000 + D, n_lambda=4, rows_per_lambda=333, enc_impl="fft", dec_impl="fft")
+
+
+# the tensor-core kernels, wherever they are built: encode fp16 D <= 160 and bf16 D <= 128, decode fp16 D <= 160
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("D", [64, 96, 128, 160])
+@pytest.mark.parametrize("N,n_lambda,rpl", [(1000, 4, 333), (20000, 1, 0), (129, 1, 0)])
+def test_gemm_kernels_all_dims(D, dtype, N, n_lambda, rpl):
+    enc_impl = "fft" if (D == 160 and dtype == "bf16") else "gemm"
+    dec_impl = "gemm" if dtype == "f16" else "fft"
+    run_case(D, dtype, N, "k_outlier", 2100 + D + N, n_lambda=n_lambda, rows_per_lambda=rpl, enc_impl=enc_impl, dec_impl=dec_impl)
 
 
 @pytest.mark.parametrize("N", [1, 31, 32, 33, 4100])
@@ -202,9 +212,11 @@ def test_empty_input_is_a_noop():
 
 # ---- config 4: mixed-radix head dims, 65536 vectors each ------------------------------------
 
+@pytest.mark.parametrize("impl", ["fft", "gemm"])
 @pytest.mark.parametrize("D", [96, 160])
-def test_config4_mixed_radix(D):
-    run_case(D, "f16", 65536, "lognormal", 4000 + D)
+def test_config4_mixed_radix(D, impl):
+    # the register FFT takes the radix-3 / radix-5 path; the tensor-core kernels contract with the D x D matrix directly
+    run_case(D, "f16", 65536, "lognormal", 4000 + D, enc_impl=impl, dec_impl=impl)
 
 
 # ---- config 2: Qwen2.5-1.5B-shaped cache: prefill, appends, full-prefix decode -------------
