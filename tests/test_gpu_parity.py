@@ -140,7 +140,7 @@ def test_gemm_encode_serves_large_appends():
 
 
 def test_gemm_kernels_are_refused_where_they_are_not_built():
-    for D, dtype in [(256, torch.float16), (128, torch.bfloat16), (96, torch.bfloat16)]:
+    for D, dtype in [(64, torch.bfloat16), (128, torch.bfloat16), (96, torch.bfloat16)]:
         plan = kb.Plan(D, G, 1)
         kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_AUTO, kb.KVQ_IMPL_GEMM)
         pk, sc = plan.empty_packed(8), plan.empty_scales(8)
@@ -175,6 +175,17 @@ def test_lambda_scale_does_not_matter_to_the_gemm_decode():
         out = gpu_decode(plan, pk, sc, lam.cuda(), "f16")
         parity.check_decode(bits(out), ob, o64, ko.F16, "gemm decode, lambda x 2^%d" % shift)
         plan.close()
+
+
+# ---- D = 256 decode on the tensor cores: CTA pairs, one term for fp16 output, split operands for bf16 output
+
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("N,n_lambda,rpl,kind", [(4096, 1, 0, "c1"), (1000, 4, 333, "k_outlier"), (1, 1, 0, "gaussian"),
+                                                 (129, 1, 0, "gaussian"), (40000, 9, 4500, "k_outlier"), (30000, 150, 200, "c1")])
+def test_gemm_decode_d256(dtype, N, n_lambda, rpl, kind):
+    enc, dec = run_case(256, dtype, N, kind, 9700 + N, n_lambda=n_lambda, rows_per_lambda=rpl, enc_impl="fft", dec_impl="gemm")
+    if dtype == "bf16":
+        assert dec["rows_needing_tie_rule"] < 0.02
 
 
 # ---- every head dim and dtype, ragged N (several tiles plus a tail), lambda rows that straddle tiles
