@@ -434,11 +434,12 @@ cudaError_t launch(int64_t N, const FftParams &f, const float *e0, cudaStream_t 
 
 }  // namespace
 
-bool umma_encode_supported(int D, bool bf16) { return D == 64 || D == 96 || D == 128 || (D == 160 && !bf16); }
+bool umma_encode_supported(int D, bool bf16) { return D == 64 || D == 96 || D == 128 || D == 256 || (D == 160 && !bf16); }
 
 cudaError_t umma_encode(int D, bool bf16, int64_t N, const FftParams &f, const float *e0, cudaStream_t stream)
 {
     if (!tensor_map_encode_fn()) return cudaErrorNotSupported;
+    if (D == 256) return umma_encode_d256(bf16, N, f, e0, stream);   // its own kernel: CTA pairs, x through a ring of K blocks
     switch (D) {
         case 64: return bf16 ? launch<64, true>(N, f, e0, stream) : launch<64, false>(N, f, e0, stream);
         case 96: return bf16 ? launch<96, true>(N, f, e0, stream) : launch<96, false>(N, f, e0, stream);

@@ -1,0 +1,428 @@
+// Warp-specialised tcgen05 DFT-as-GEMM encode kernel of libkvq (sm_100a) for D = 256, fp16 or bf16 input.
+//
+// Same contraction and the same split of W into 16-bit terms as kvq_umma_encode.cu (v = lambda (.) M (s (.) x),
+// Sec. 3.1 Eq. 1-2, Sec. 5.1 item 1; W 2^k = W1 + W2 for fp16 input, W1 + W2 + W3 for bf16), with the two changes
+// that D = 256 forces:
+//
+//   * the split B operand (2 or 3 x 128 KB) does not fit one CTA's shared memory, so CTAs work in pairs on the
+//     same tiles and each computes one half of the channels (four groups): B is [128 channels, K = 256] per
+//     term and CTA.  The two CTAs of a pair share nothing and never wait for each other; the x tile is read
+//     twice (the second read hits L2).
+//   * what shared memory is left holds less than one x tile next to a three-term B, so x moves through a ring
+//     of K blocks (64 columns x 128 rows, 16 KB): the mma thread issues the K steps of a block for every term
+//     as soon as the block has landed and releases it with a commit of its own.
+//
+// Roles as in kvq_umma_encode.cu: producer (TMA), one mma thread, two epilogue sets of eight warps on
+// alternate tiles (thread = (row, two groups)); four accumulator stages of 128 columns; every wait is bounded.
+#include "kvq_internal.h"
+#include "kvq_umma.cuh"
+
+namespace kvq {
+
+namespace {
+
+constexpr int kTile = 128;                 // vectors per tile = MMA M
+constexpr int kGroup = 32;
+constexpr int kThreads = 576;              // producer, mma, 16 epilogue warps
+constexpr int kEpiWarps = 16;
+constexpr int kBlockBytes = kTile * 128;   // one K block of the x tile: 128 rows x 128 B
+constexpr int kCtrlBytes = 256;
+constexpr int kSmemLimit = 232448;         // 227 KB of dynamic shared memory per CTA
+constexpr uint32_t kTmemCols = 512;
+
+constexpr float kMagicRound = 12582912.0f + 8.0f;   // 1.5 * 2^23 + 8: (v + magic) has q + 8 in its low bits
+constexpr uint32_t kMagicBits = 0x4B400000u;
+constexpr uint32_t kMagicSum = kMagicBits * 0x11111111u;   // sum_i kMagicBits * 16^i  (mod 2^32)
+
+constexpr int kD = 256;
+constexpr int kG = kD / kGroup;            // 8 scales per row
+constexpr int kHalfN = 128;                // channels per CTA = MMA N
+constexpr int kKBlocks = kD / 64;          // 4 K blocks per tile
+constexpr int kBBlock = kHalfN * 128;      // one K block of one split term: 128 rows x 128 B
+constexpr int kBTerm = kKBlocks * kBBlock; // 64 KB
+constexpr int kAccStages = 4;
+constexpr int kMaxRing = 6;
+
+template <bool BF16>
+struct Cfg {
+    static constexpr int kSplit = BF16 ? 3 : 2;
+    static constexpr int kBBytes = kSplit * kBTerm;
+    static constexpr int kRoom = (kSmemLimit - 1024 - kCtrlBytes - kBBytes) / kBlockBytes;
+    static constexpr int kRing = kRoom < kMaxRing ? kRoom : kMaxRing;   // K blocks of x in flight: 6 (fp16), 2 (bf16)
+    static_assert(kRing >= 2, "no room for the x ring");
+    static constexpr int kSmemBytes = kBBytes + kRing * kBlockBytes + kCtrlBytes + 1024;
+    static constexpr uint32_t kIdesc = umma_idesc_m128(kHalfN, BF16);
+};
+
+struct Ctrl {
+    uint64_t in_full[kMaxRing], in_empty[kMaxRing];
+    uint64_t acc_full[4], acc_empty[4];
+    uint64_t b_first, b_ready;
+    uint32_t tmem_base;
+    volatile uint32_t abort;
+};
+static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
+
+// 2^k for a lambda row: the power of two that brings max_c lambda_c sqrt(2 / D) into [2^13, 2^14), so that
+// the first split term of W 2^k stays below fp16's maximum and the later ones above its subnormals.
+// Every lane of the warp gets the same value.
+template <int D>
+__device__ __forceinline__ float lift_of(const float *__restrict__ lam, int lane)
+{
+    float mx = 0.0f;
+#pragma unroll
+    for (int p = 0; p < (D / 4 + 31) / 32; ++p) {
+        const int i = lane + 32 * p;
+        if (i < D / 4) {
+            const float4 l = __ldg(reinterpret_cast<const float4 *>(lam) + i);
+            mx = fmaxf(mx, fmaxf(fmaxf(fabsf(l.x), fabsf(l.y)), fmaxf(fabsf(l.z), fabsf(l.w))));
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+    constexpr float kRowScale = (float)ct_sqrt(2.0 / (double)D);        // largest entry of M
+    mx = fminf(fmaxf(mx * kRowScale, 1e-30f), 1e30f);
+    const int e = (int)((__float_as_uint(mx) >> 23) & 0xFFu) - 127;      // floor(log2 mx)
+    return __uint_as_float((uint32_t)(127 + 13 - e) << 23);
+}
+
+// Rows [c0, c1) of every split term of this CTA's half of the B operand (channel 128 half + c), by one warp: a lane
+// reads four table entries per pass (coalesced rows), scales them by lambda_c 2^k, peels off 16-bit terms and
+// writes 8 bytes of each term's swizzled row.
+template <bool BF16>
+__device__ __forceinline__ void build_b_rows(unsigned char *sB, const float *__restrict__ e0, const float *__restrict__ lam, float lift,
+                                             int half, int c0, int c1, int lane)
+{
+    using C = Cfg<BF16>;
+#pragma unroll 2
+    for (int c = c0; c < c1; ++c) {
+        const int cg = half * kHalfN + c;
+        const float f = __ldg(lam + cg) * lift;
+#pragma unroll
+        for (int p = 0; p < 2; ++p) {
+            const int i = lane + 32 * p;
+            const float4 m = __ldg(reinterpret_cast<const float4 *>(e0 + (size_t)cg * kD) + i);
+            float w[4] = {m.x * f, m.y * f, m.z * f, m.w * f};
+            const int ch = i >> 1;   // 16-byte chunk of the K-major row: K block ch / 8, chunk ch % 8
+            const uint32_t off = (uint32_t)((ch >> 3) * kBBlock + c * 128 + (((ch & 7) ^ (c & 7)) << 4) + ((i & 1) ? 8 : 0));
+#pragma unroll
+            for (int t = 0; t < C::kSplit; ++t) {
+                const uint32_t lo = narrow2<BF16>(w[0], w[1]), hi = narrow2<BF16>(w[2], w[3]);
+                *reinterpret_cast<uint2 *>(sB + t * kBTerm + off) = make_uint2(lo, hi);
+                if (t + 1 < C::kSplit) {   // what the 16-bit term left behind (exact in fp32)
+                    const float2 a = widen2<BF16>(lo), b = widen2<BF16>(hi);
+                    w[0] -= a.x, w[1] -= a.y, w[2] -= b.x, w[3] -= b.y;
+                }
+            }
+        }
+    }
+}
+
+}  // namespace
+
+struct UmmaEncode256Params {
+    const float *lambda;   // [n_lambda, D] fp32
+    const float *e0;       // plan table [D, D] fp32: e0[c][n] = M[c][n] s_n
+    unsigned char *packed; // [*, D/2] bytes out
+    uint16_t *scales;      // [*, D/32] fp16 out
+    int64_t N;
+    int64_t n_lambda;
+    int64_t rpl;           // rows per lambda segment (N when there is one lambda row)
+    int64_t n_seg;
+    int64_t out_mul, out_add;   // output row of input row r is r * out_mul + out_add
+    uint32_t *status;
+};
+
+template <bool BF16>
+__global__ void __launch_bounds__(kThreads, 1)
+    kvq_encode_umma_d256_kernel(const __grid_constant__ UmmaEncode256Params prm, const __grid_constant__ CUtensorMap tm_x)
+{
+    using C = Cfg<BF16>;
+    constexpr int kRing = C::kRing;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    unsigned char *sB = smem;                                   // kSplit terms
+    unsigned char *sIn = sB + C::kBBytes;                       // ring of K blocks of x
+    Ctrl *ctrl = reinterpret_cast<Ctrl *>(sIn + kRing * kBlockBytes);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int half = blockIdx.x & 1;            // which 128 channels this CTA computes
+    const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kRing; ++s) {
+            mbar_init(smem_u32(&ctrl->in_full[s]), 1);
+            mbar_init(smem_u32(&ctrl->in_empty[s]), 1);
+        }
+        for (int s = 0; s < kAccStages; ++s) {
+            mbar_init(smem_u32(&ctrl->acc_full[s]), 1);
+            mbar_init(smem_u32(&ctrl->acc_empty[s]), kEpiWarps / 2);
+        }
+        mbar_init(smem_u32(&ctrl->b_first), kEpiWarps);       // first B: all epilogue warps build it
+        mbar_init(smem_u32(&ctrl->b_ready), kEpiWarps / 2);   // later rebuilds: the set that owns the tile
+        ctrl->abort = 0u;
+        mbar_init_fence();
+    }
+    if (warp == 0) tmem_alloc(smem_u32(&ctrl->tmem_base), kTmemCols);
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctrl->tmem_base;
+    volatile uint32_t *abort_flag = &ctrl->abort;
+    uint32_t *status = prm.status;
+
+    // ---- tiles: lambda segments of rpl rows, cut into tiles of 128 rows; a contiguous range per CTA pair
+    const int64_t N = prm.N, rpl = prm.rpl;
+    const int64_t tps = (rpl + kTile - 1) / kTile;                 // tiles per segment
+    const int64_t n_tiles = prm.n_seg * tps;
+    const int64_t per_pair = (n_tiles + n_pairs - 1) / n_pairs;
+    const int64_t tile_begin = (int64_t)pair * per_pair;
+    const int64_t tile_end = tile_begin + per_pair < n_tiles ? tile_begin + per_pair : n_tiles;
+    const int n_my = tile_end > tile_begin ? (int)(tile_end - tile_begin) : 0;
+
+    if (warp == 0) {
+        // =========================== producer ===========================
+        if (lane == 0) {
+            int issued = 0;
+            bool ok = true;
+            TileCursor cur(tile_begin, tps);
+            for (int j = 0; j < n_my && ok; ++j, cur.advance(1)) {
+                const int64_t row0 = cur.seg * rpl + cur.row_in_segment();
+#pragma unroll
+                for (int kb = 0; kb < kKBlocks; ++kb) {
+                    const int u = kKBlocks * j + kb, s = u % kRing;
+                    ok = wait_or_abort(smem_u32(&ctrl->in_empty[s]), ((uint32_t)(u / kRing) & 1u) ^ 1u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT);
+                    if (!ok) break;
+                    const uint32_t bar = smem_u32(&ctrl->in_full[s]);
+                    mbar_arrive_expect_tx(bar, kBlockBytes);
+                    tma_load_2d(smem_u32(sIn + s * kBlockBytes), &tm_x, 64 * kb, (int)row0, bar);
+                    issued = u + 1;
+                }
+            }
+            if (!ok) {
+                // give this thread's own copies in flight a bounded chance to land before the CTA goes away
+                for (int u = issued > kRing ? issued - kRing : 0; u < issued; ++u)
+                    (void)mbar_wait_bounded(smem_u32(&ctrl->in_full[u % kRing]), (uint32_t)(u / kRing) & 1u, 1u << 16);
+            }
+        }
+    } else if (warp == 1) {
+        // =========================== mma issuer ===========================
+        if (lane == 0) {
+            // Descriptors differ only in their 14-bit start-address field (bytes >> 4): one base per operand, one add per MMA.
+            const uint64_t b_desc = smem_desc_sw128(smem_u32(sB));
+            const uint64_t a_desc = smem_desc_sw128(smem_u32(sIn));
+            const uint32_t b_lo = (uint32_t)b_desc, b_hi = (uint32_t)(b_desc >> 32);
+            const uint32_t a_lo = (uint32_t)a_desc, a_hi = (uint32_t)(a_desc >> 32);
+            uint32_t builds = 0;
+            bool ok = true;
+            TileCursor cur(tile_begin, tps);
+            for (int j = 0; j < n_my && ok; ++j, cur.advance(1)) {
+                const int sc = j % kAccStages;
+                if (j == 0) {   // all epilogue warps build the first B while the first x blocks are in flight
+                    if (!wait_or_abort(smem_u32(&ctrl->b_first), 0u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT)) break;
+                } else if (cur.first_of_segment()) {   // an epilogue set rebuilds B for this lambda row
+                    if (!wait_or_abort(smem_u32(&ctrl->b_ready), builds & 1u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT)) break;
+                    ++builds;
+                }
+                if (!wait_or_abort(smem_u32(&ctrl->acc_empty[sc]), ((uint32_t)(j / kAccStages) & 1u) ^ 1u, abort_flag, status,
+                                   KVQ_DEV_SLOT_TIMEOUT))
+                    break;
+                const uint32_t d_tmem = tmem_base + (uint32_t)sc * kHalfN;
+#pragma unroll
+                for (int kb = 0; kb < kKBlocks; ++kb) {
+                    const int u = kKBlocks * j + kb, s = u % kRing;
+                    if (!wait_or_abort(smem_u32(&ctrl->in_full[s]), (uint32_t)(u / kRing) & 1u, abort_flag, status, KVQ_DEV_LOAD_TIMEOUT)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t a_lo_s = a_lo + (uint32_t)s * (kBlockBytes >> 4);
+#pragma unroll
+                    for (int t = 0; t < C::kSplit; ++t) {
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks) {   // the four K steps of this block
+                            const uint64_t ad = ((uint64_t)a_hi << 32) | (uint64_t)(a_lo_s + (uint32_t)ks * 2u);
+                            const uint64_t bd = ((uint64_t)b_hi << 32) |
+                                                (uint64_t)(b_lo + (uint32_t)t * (kBTerm >> 4) + (uint32_t)kb * (kBBlock >> 4) + (uint32_t)ks * 2u);
+                            if (kb > 0 || t > 0 || ks > 0) umma_f16_ss<true>(d_tmem, ad, bd, C::kIdesc);
+                            else umma_f16_ss<false>(d_tmem, ad, bd, C::kIdesc);
+                        }
+                    }
+                    umma_commit(smem_u32(&ctrl->in_empty[s]));   // the tensor core has read this block of x
+                }
+                if (ok) umma_commit(smem_u32(&ctrl->acc_full[sc]));
+            }
+        }
+    } else {
+        // =========================== epilogue: accumulator -> scales, codes, nibbles ===========================
+        // Two sets of eight warps take alternate tiles, so that one set's waits (barrier, tensor-memory load)
+        // hide behind the other set's arithmetic.  Thread = (row, half row).
+        const int set = (warp - 2) >> 3;        // this set takes tiles set, set + 2, ...
+        const int q = warp & 3;                 // tensor-memory lane quarter this warp may touch
+        const int h = ((warp - 2) >> 2) & 1;    // half of the row
+        const int r = q * 32 + lane;            // tile row of this thread
+        const int bw = (warp - 2) & 7;          // position within the set: 16 rows of B per warp when the set rebuilds B
+        const int g0 = 2 * h;                   // this thread's groups within the CTA's four: g0, g0 + 1
+        const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16);
+        int64_t cached_seg = -1;
+        float unlift = 1.0f;
+        if (n_my > 0) {   // B for the CTA's first lambda row: D / 16 rows per warp, all sixteen warps
+            TileCursor first(tile_begin, tps);
+            const float *lam = prm.lambda + (prm.n_lambda == 1 ? 0 : first.seg) * kD;
+            const float lift = lift_of<kD>(lam, lane);
+            build_b_rows<BF16>(sB, prm.e0, lam, lift, half, (warp - 2) * 8, (warp - 1) * 8, lane);
+            fence_proxy_async();   // B is read by the tensor core through the async proxy
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctrl->b_first));
+            unlift = 1.0f / lift;
+            cached_seg = first.seg;
+        }
+        TileCursor cur(tile_begin + set, tps);
+        for (int j = set; j < n_my; j += 2, cur.advance(2)) {
+            __syncwarp();
+            const int64_t seg = cur.seg;
+            const int64_t off = cur.row_in_segment();
+
+            // ---- a new lambda row.  Every set needs its lift; the set that owns the row's first tile rebuilds B,
+            // ---- once every MMA that read the old B is complete (the previous tile's accumulator is full), and
+            // ---- tells the mma warp.
+            if (seg != cached_seg) {
+                const float *lam = prm.lambda + (prm.n_lambda == 1 ? 0 : seg) * kD;
+                const float lift = lift_of<kD>(lam, lane);
+                if (j > 0 && cur.first_of_segment()) {
+                    if (!wait_or_abort(smem_u32(&ctrl->acc_full[(j - 1) % kAccStages]), (uint32_t)((j - 1) / kAccStages) & 1u,
+                                       abort_flag, status, KVQ_DEV_MMA_TIMEOUT))
+                        break;
+                    build_b_rows<BF16>(sB, prm.e0, lam, lift, half, bw * 16, (bw + 1) * 16, lane);
+                    fence_proxy_async();   // B is read by the tensor core through the async proxy
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&ctrl->b_ready));
+                }
+                unlift = 1.0f / lift;
+                cached_seg = seg;
+            }
+
+            const int sc = j % kAccStages;
+            if (!wait_or_abort(smem_u32(&ctrl->acc_full[sc]), (uint32_t)(j / kAccStages) & 1u, abort_flag, status, KVQ_DEV_MMA_TIMEOUT)) break;
+            tc_fence_after();
+
+            // ---- rows of the tile that exist: the segment (and with it the tensor) may end inside the tile
+            int64_t seg_rows = N - seg * rpl;
+            if (seg_rows > rpl) seg_rows = rpl;
+            const bool live = off + r < seg_rows;
+            const int64_t orow = (seg * rpl + off + r) * prm.out_mul + prm.out_add;
+#pragma unroll
+            for (int gi = 0; gi < 2; ++gi) {
+                const int g = g0 + gi;       // warp-uniform; group within this CTA's half
+                {
+                    uint32_t vb[32];
+                    tmem_ld32(t_addr + (uint32_t)sc * kHalfN + (uint32_t)(g * kGroup), vb);
+                    tmem_ld_wait();
+                    if (gi == 1) {   // this thread's last group is in registers: hand the accumulator back
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&ctrl->acc_empty[sc]));
+                    }
+                    // ---- scale: sigma = fp16(absmax / 7); codes are taken against the stored value
+                    float amax = 0.0f;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) amax = fmaxf(amax, fabsf(__uint_as_float(vb[i])));
+                    amax *= unlift;
+                    const float sig = fminf(__fdiv_rn(amax, 7.0f), 65504.0f);
+                    const __half hs = __float2half_rn(sig);
+                    const float sg = __half2float(hs);
+                    const float rs1 = sg > 0.0f ? __frcp_rn(sg) : 0.0f;
+                    const bool clamp = !(amax * rs1 < 7.25f);   // saturated or subnormal scale: codes could leave [-7, 7]
+                    const float rs = rs1 * unlift;              // applies to the lifted accumulator values
+
+                    // ---- round, bias to unsigned nibbles, pack 8 codes per word
+                    uint32_t words[4];
+#pragma unroll
+                    for (int w = 0; w < 4; ++w) {
+                        uint32_t acc = 0;
+                        if (!clamp) {
+#pragma unroll
+                            for (int e = 0; e < 8; ++e)
+                                acc += __float_as_uint(fmaf(__uint_as_float(vb[8 * w + e]), rs, kMagicRound)) << (4 * e);
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 8; ++e)
+                                acc += __float_as_uint(fminf(fmaxf(__uint_as_float(vb[8 * w + e]) * rs, -7.0f), 7.0f) + kMagicRound) << (4 * e);
+                        }
+                        words[w] = (acc - kMagicSum) ^ 0x88888888u;
+                    }
+                    if (live) {
+                        const int gg = 4 * half + g;   // group within the row
+                        *reinterpret_cast<uint4 *>(prm.packed + orow * (kD / 2) + gg * 16) = make_uint4(words[0], words[1], words[2], words[3]);
+                        prm.scales[orow * kG + gg] = __half_as_ushort(hs);
+                    }
+                }
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        if (*abort_flag) __nanosleep(20000);   // let tensor-core work that was already issued drain
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------------
+namespace {
+
+template <bool BF16>
+cudaError_t launch(int64_t N, const FftParams &f, const float *e0, cudaStream_t stream)
+{
+    using C = Cfg<BF16>;
+    static int sms = 0;
+    if (sms == 0) {
+        cudaError_t e = cudaFuncSetAttribute(kvq_encode_umma_d256_kernel<BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+        if (e != cudaSuccess) return e;
+        int dev = 0;
+        if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+        if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+    }
+    if (N >= (int64_t)1 << 31) return cudaErrorInvalidValue;   // tensor-map coordinates are 32-bit
+
+    UmmaEncode256Params prm;
+    prm.lambda = f.lambda;
+    prm.e0 = e0;
+    prm.packed = static_cast<unsigned char *>(f.packed);
+    prm.scales = static_cast<uint16_t *>(f.scales);
+    prm.N = N;
+    prm.n_lambda = f.n_lambda;
+    prm.rpl = f.n_lambda == 1 ? N : f.rows_per_lambda;
+    prm.n_seg = (N + prm.rpl - 1) / prm.rpl;
+    prm.out_mul = f.out_mul;
+    prm.out_add = f.out_add;
+    prm.status = f.status;
+
+    CUtensorMap tm_x;
+    const cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)N};
+    const cuuint64_t strides[1] = {(cuuint64_t)(2 * kD)};
+    const cuuint32_t box[2] = {64, (cuuint32_t)kTile};
+    if (!make_tensor_map(&tm_x, BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, f.in, dims, strides, box,
+                         CU_TENSOR_MAP_SWIZZLE_128B))
+        return cudaErrorInvalidValue;
+
+    const int64_t tiles = prm.n_seg * ((prm.rpl + kTile - 1) / kTile);
+    const int64_t pairs = tiles < sms / 2 ? tiles : sms / 2;
+    kvq_encode_umma_d256_kernel<BF16><<<(int)(2 * pairs), kThreads, C::kSmemBytes, stream>>>(prm, tm_x);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t umma_encode_d256(bool bf16, int64_t N, const FftParams &f, const float *e0, cudaStream_t stream)
+{
+    if (!tensor_map_encode_fn()) return cudaErrorNotSupported;
+    return bf16 ? launch<true>(N, f, e0, stream) : launch<false>(N, f, e0, stream);
+}
+
+}  // namespace kvq
