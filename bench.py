@@ -37,7 +37,7 @@ D = 128
 GROUP = 32
 BYTES_PER_VEC = 2 * D + D // 2 + 2 * (D // GROUP)   # 328: fp16 row + packed row + fp16 scales
 FALLBACK_HBM_GBS = 6650.0
-METRIC = "kvq_hot_path_algorithmic_GBps"
+METRIC = "hot-path algorithmic GB/s (encode + append + full-prefix decode; encode ns/vec and prefix-decode GB/s in detail)"
 UNIT = "GB/s"
 
 
@@ -56,6 +56,23 @@ def workload_shape():
     shp = wl.LLAMA3_70B
     streams = 2 * shp.kv_heads * shp.batch          # K and V streams of one layer: 64
     return shp, streams, shp.prefix                 # T = 32768 rows per stream
+
+
+def slot_seed(rank: int, slot: int, n_slots: int) -> int:
+    """Seed of layer slot `slot` on rank `rank`: ranks own disjoint layers (weak scaling, no exchange between them)."""
+    return 5000 + 10 * (rank * n_slots + slot)
+
+
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """The job's time is the slowest rank's: MAX all-reduce of a device-measured time (NCCL on GPUs, gloo in the CPU test)."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
 
 
 class ClockSampler:
@@ -135,7 +152,7 @@ def run_ours(args):
     lam = wl.make_lambda(2, D, 71 + rank, device=dev)             # one lambda row for K, one for V
     slots = []
     for s in range(n_slots):
-        seed = 5000 + 10 * (rank * n_slots + s)
+        seed = slot_seed(rank, s, n_slots)
         xk = wl.make_vectors(N // 2, D, shp.dtype, "k_outlier", seed, device=dev)
         xv = wl.make_vectors(N // 2, D, shp.dtype, "gaussian", seed + 1, device=dev)
         x = torch.cat([xk, xv], 0)
@@ -189,11 +206,7 @@ def run_ours(args):
     barrier()
     launches = kb.kvq_launch_count() - launches0
     clocks = sampler.stop() if rank == 0 else None
-    ms_total = t0.elapsed_time(t1)
-    if world > 1:
-        tt = torch.tensor([ms_total], device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms_total = float(tt.item())
+    ms_total = max_over_ranks(t0.elapsed_time(t1), world, dev)
     assert kb.kvq_plan_device_status(h) == 0, "a device-side wait timed out"
 
     enc_ms = [e[0].elapsed_time(e[1]) for e in evs]
@@ -225,11 +238,7 @@ def run_ours(args):
             e2e_step()
         b.record()
         barrier()
-        ms_e2e = a.elapsed_time(b)
-        if world > 1:
-            tt = torch.tensor([ms_e2e], device=dev)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            ms_e2e = float(tt.item())
+        ms_e2e = max_over_ranks(a.elapsed_time(b), world, dev)
         step_bytes = (2 * N + S) * BYTES_PER_VEC
         e2e = {"value": world * e2e_steps * step_bytes / (ms_e2e * 1e-3) / 1e9, "unit": UNIT,
                "h2d_bytes_per_step": hx.numel() * 2 + hnew.numel() * 2, "d2h_bytes_per_step": hout.numel() * 2,
@@ -241,6 +250,7 @@ def run_ours(args):
             dist.destroy_process_group()
         return
 
+    d256 = measure_d256(kb, wl, dev)
     step_bytes = (2 * N + S) * BYTES_PER_VEC
     value = world * args.steps * step_bytes / (ms_total * 1e-3) / 1e9
     peak, peak_src = measured_peak()
@@ -260,7 +270,7 @@ def run_ours(args):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32", "data": "synthetic",
+        "dtype": "f16 operands, f32 accumulate", "data": "synthetic",
         "config": {"workload": "llama-3-70b-shaped KV cache (config 5): one layer per step = encode 2x1,048,576 "
                                "vectors + append 64 + full-prefix decode 2,097,152 vectors, D=128 fp16 g=32",
                    "vectors_per_step": 2 * N + S, "bytes_per_vector": BYTES_PER_VEC, "io_dtype": "f16",
@@ -273,7 +283,8 @@ def run_ours(args):
             "append_us": 1e3 * sum(app_ms) / len(app_ms),
             "encode_ms_min": min(enc_ms), "decode_ms_min": min(dec_ms),
             "model_sweep_decode_ms_80_layers": 80 * dec_avg,
-            "paper_context": "paper: 24.6 ns/vec encode at D=128 on an Apple M1 GPU (fp32 in, Sec. 7.1)",
+            "paper_context": "paper: 24.6 ns/vec encode at D=128, ~50 ns/vec at D=256 on an Apple M1 GPU (fp32 in, Sec. 7.1)",
+            "d256_bf16_gemma_shaped": d256,
         },
         "roofline": roofline,
         "cpu_baseline": cpu,
@@ -286,9 +297,47 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-# DRAM bytes per full launch from ncu (dram__bytes_read.sum + dram__bytes_write.sum), filled in from the
-# committed profile summaries under profiles/; None until a capture exists.
-TRAFFIC = {"decode": None, "encode": None}
+def measure_d256(kb, wl, dev, iters=10):
+    """Outside the timed region: the Gemma-3-1B-shaped cache (config 3: 26 layers x K,V x 4096 tokens, D=256 bf16) in one
+    encode and one decode launch over all layers (52 lambda rows), device-timed, two buffer sets in rotation."""
+    import torch
+
+    Dh, T, L = 256, 4096, 52
+    Nv = L * T
+    bpv = 2 * Dh + Dh // 2 + 2 * (Dh // GROUP)
+    plan = kb.Plan(Dh, GROUP, 33)
+    lam = wl.make_lambda(L, Dh, 34, device=dev)
+    sets = []
+    for i in range(2):
+        x = wl.make_vectors(Nv, Dh, "bf16", "c1", 35 + i, device=dev)
+        sets.append((x, plan.empty_packed(Nv, dev), plan.empty_scales(Nv, dev), torch.empty_like(x)))
+    enc, dec = [], []
+    for i in range(iters + 2):
+        x, pk, sc, out = sets[i % 2]
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        e[0].record()
+        kb.kvq_encode(plan.handle, x, lam, pk, sc, T)
+        e[1].record()
+        kb.kvq_decode(plan.handle, pk, sc, lam, out, T)
+        e[2].record()
+        torch.cuda.synchronize()
+        if i >= 2:
+            enc.append(e[0].elapsed_time(e[1]))
+            dec.append(e[1].elapsed_time(e[2]))
+    assert kb.kvq_plan_device_status(plan.handle) == 0
+    plan.close()
+    em, dm = statistics.median(enc), statistics.median(dec)
+    peak, _ = measured_peak()
+    return {"vectors": Nv, "bytes_per_vector": bpv, "encode_ns_per_vec": em * 1e6 / Nv, "encode_GBps": Nv * bpv / (em * 1e-3) / 1e9,
+            "decode_ns_per_vec": dm * 1e6 / Nv, "prefix_decode_GBps": Nv * bpv / (dm * 1e-3) / 1e9,
+            "prefix_decode_frac_of_hbm_peak": Nv * bpv / (dm * 1e-3) / 1e9 / peak,
+            "note": "working set 140 MB per launch, about the size of L2: not a roofline number"}
+
+
+# DRAM bytes per full launch (2,097,152 vectors, the bench's launch size) from ncu: dram__bytes_read.sum +
+# dram__bytes_write.sum, one-pass capture; see profiles/dram_traffic_d128_n2097152.md.  Reads match the algorithmic
+# bytes; writes are short of them by what is still in the 126 MB L2 when the kernel ends.
+TRAFFIC = {"decode": 151436288 + 478505472, "encode": 537912832 + 128682752}
 
 
 # --------------------------------------------------------------------------------------------

@@ -52,11 +52,14 @@ typedef enum {
 typedef enum { KVQ_F16 = 0, KVQ_BF16 = 1 } kvq_dtype_t;
 
 /* Which kernel family serves a call.  AUTO picks the fastest one that meets the
- * tolerances for the plan's D and the call's dtype. */
+ * tolerances for the plan's D and the call's dtype: the tensor-core kernel where one is
+ * built (for kvq_encode / kvq_append only on calls of at least 4096 rows), else the FFT. */
 typedef enum {
     KVQ_IMPL_AUTO = 0,
     KVQ_IMPL_FFT = 1, /* fp32 register FFT, one thread per vector: every D and dtype */
-    KVQ_IMPL_GEMM = 2 /* tcgen05 DFT-as-GEMM (encode: D = 128; decode: D = 128, fp16); KVQ_ERR_UNSUPPORTED_DIM elsewhere */
+    KVQ_IMPL_GEMM = 2 /* tcgen05 DFT-as-GEMM.  encode / append: fp16 for D = 64, 96, 128, 160, 256, bf16 for
+                         D = 64, 96, 128, 256; decode: fp16 for the same D, bf16 for D = 256.  Elsewhere the
+                         compute calls return KVQ_ERR_UNSUPPORTED_DIM. */
 } kvq_impl_t;
 
 /*
