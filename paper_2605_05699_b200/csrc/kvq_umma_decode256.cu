@@ -51,9 +51,10 @@ struct Ctrl {
     uint64_t in_full[kInStages], in_empty[kInStages];
     uint64_t a_full[kAStages], a_empty[2][kAStages];   // a_empty[g][s]: a unit of dequant group g has been read from stage s
     uint64_t acc_full[kAccStages], acc_empty[kAccStages];
-    uint64_t b_first, b_free;
+    uint64_t b_first;
     uint32_t tmem_base;
     volatile uint32_t abort;
+    volatile uint32_t b_epoch;   // lambda rows whose last MMA is complete, counted from the CTA's first one
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
 
@@ -169,8 +170,8 @@ __global__ void __launch_bounds__(kThreads, 1)
             mbar_init(smem_u32(&ctrl->acc_empty[s]), 4);
         }
         mbar_init(smem_u32(&ctrl->b_first), 16);
-        mbar_init(smem_u32(&ctrl->b_free), 1);
         ctrl->abort = 0u;
+        ctrl->b_epoch = 0u;
         mbar_init_fence();
     }
     if (warp == 0) tmem_alloc(smem_u32(&ctrl->tmem_base), kTmemCols);
@@ -236,8 +237,17 @@ __global__ void __launch_bounds__(kThreads, 1)
             TileCursor cur(tile_begin, tps);
             for (int j = 0; j < n_mma && ok; ++j, cur.advance(1)) {
                 const int sc = j % kAccStages;
-                // a new lambda row: tell the dequant group that rebuilds B when every MMA issued so far has read the old one
-                if (j > 0 && cur.first_of_segment()) umma_commit(smem_u32(&ctrl->b_free));
+                // A new lambda row: a dequant group will overwrite B once every MMA issued so far has read the old one.  This
+                // thread waits for the previous tile's accumulator barrier itself (it is at most one phase behind: the stage
+                // was free when that tile was issued) and publishes a count; a counter, unlike a parity, cannot be misread
+                // by a group that skipped a rebuild.  The tensor core drains once per lambda row.
+                if (j > 0 && cur.first_of_segment()) {
+                    if (!wait_or_abort(smem_u32(&ctrl->acc_full[(j - 1) % kAccStages]), (uint32_t)((j - 1) / kAccStages) & 1u, abort_flag,
+                                       status, KVQ_DEV_MMA_TIMEOUT))
+                        break;
+                    ctrl->b_epoch = (uint32_t)(cur.seg - seg_first);
+                    __threadfence_block();
+                }
                 if (!wait_or_abort(smem_u32(&ctrl->acc_empty[sc]), ((uint32_t)(j / kAccStages) & 1u) ^ 1u, abort_flag, status,
                                    KVQ_DEV_SLOT_TIMEOUT))
                     break;
@@ -299,11 +309,26 @@ __global__ void __launch_bounds__(kThreads, 1)
                 const RecipLambda rl(lambda_row(seg), lane);
                 rho = rl.rho;
                 if (cur.first_of_segment()) {
-                    // every MMA issued so far must have read B: the mma thread commits b_free once per new lambda row, after
-                    // the last tile of the old one (a barrier of its own: the A-stage barriers cycle once per K half and a
-                    // parity wait on them could not tell "not yet" from "already two phases on")
-                    if (!wait_or_abort(smem_u32(&ctrl->b_free), (uint32_t)(seg - seg_first - 1) & 1u, abort_flag, status, KVQ_DEV_MMA_TIMEOUT))
-                        break;
+                    // every MMA issued so far must have read B: the mma thread says so by raising b_epoch to this row's index
+                    {
+                        const uint32_t need = (uint32_t)(seg - seg_first);
+                        bool freed = false;
+                        for (uint32_t it = 0; it < (1u << 22); ++it) {
+                            if (ctrl->b_epoch >= need) {
+                                freed = true;
+                                break;
+                            }
+                            if (*abort_flag) break;
+                            __nanosleep(64);
+                        }
+                        if (!freed) {
+                            if (!*abort_flag) {
+                                *abort_flag = 1u;
+                                atomicOr(status, KVQ_DEV_MMA_TIMEOUT);
+                            }
+                            break;
+                        }
+                    }
                     build_b_rows<C::kBTerms>(sB, prm.g.b0, rl, half, q * 32, q * 32 + 32, lane);
                     fence_proxy_async();   // B is read by the tensor core through the async proxy
                 }

@@ -181,7 +181,8 @@ def test_lambda_scale_does_not_matter_to_the_gemm_decode():
 
 @pytest.mark.parametrize("dtype", ["f16", "bf16"])
 @pytest.mark.parametrize("N,n_lambda,rpl,kind", [(4096, 1, 0, "c1"), (1000, 4, 333, "k_outlier"), (1, 1, 0, "gaussian"),
-                                                 (129, 1, 0, "gaussian"), (40000, 9, 4500, "k_outlier"), (30000, 150, 200, "c1")])
+                                                 (129, 1, 0, "gaussian"), (40000, 9, 4500, "k_outlier"), (30000, 150, 200, "c1"),
+                                                 (30000, 235, 128, "c1"), (40000, 105, 384, "k_outlier")])
 def test_gemm_kernels_d256(dtype, N, n_lambda, rpl, kind):
     enc, dec = run_case(256, dtype, N, kind, 9700 + N, n_lambda=n_lambda, rows_per_lambda=rpl, enc_impl="gemm", dec_impl="gemm")
     assert enc["mismatches"] <= max(2, int(1e-4 * N * 256))
