@@ -328,7 +328,7 @@ kvq_status_t kvq_decode(kvq_plan_t *plan, const uint8_t *packed, const void *sca
         g.n_lambda = n_lambda;
         g.rows_per_lambda = rows_per_lambda < 1 ? 1 : rows_per_lambda;
         g.status = plan->d_status;
-        if (umma_decode(plan->D, dtype == KVQ_BF16, N, g, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
+        if (umma_decode(plan->D, dtype == KVQ_BF16, N, g, plan->sign_xor, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
             (void)cudaGetLastError();
             return KVQ_ERR_CUDA;
         }

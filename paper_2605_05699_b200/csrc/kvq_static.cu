@@ -131,7 +131,7 @@ extern "C" kvq_status_t kvq_decode_static(kvq_plan_t *plan, const uint8_t *packe
     g.n_lambda = n_lambda;
     g.rows_per_lambda = rows_per_lambda < 1 ? 1 : rows_per_lambda;
     g.status = status;
-    if (umma_decode(128, false, N, g, stream) != cudaSuccess) {
+    if (umma_decode(128, false, N, g, plan->sign_xor, stream) != cudaSuccess) {
         (void)cudaGetLastError();
         return KVQ_ERR_CUDA;
     }

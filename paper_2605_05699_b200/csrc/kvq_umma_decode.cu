@@ -524,9 +524,9 @@ cudaError_t launch(int64_t N, const GemmParams &g, cudaStream_t stream)
 
 bool umma_decode_supported(int D, bool bf16) { return D == 256 || (!bf16 && (D == 64 || D == 96 || D == 128 || D == 160)); }
 
-cudaError_t umma_decode(int D, bool bf16, int64_t N, const GemmParams &g, cudaStream_t stream)
+cudaError_t umma_decode(int D, bool bf16, int64_t N, const GemmParams &g, const uint32_t *sign_xor, cudaStream_t stream)
 {
-    if (D == 256) return umma_decode_d256(bf16, N, g, stream);   // its own kernel: CTA pairs, split operands for bf16
+    if (D == 256) return umma_decode_d256(bf16, N, g, sign_xor, stream);   // its own kernel: radix-2 split, split operands for bf16
     if (bf16) return cudaErrorInvalidValue;
     switch (D) {
         case 64: return launch<64>(N, g, stream);

@@ -3,20 +3,35 @@
 // Same contraction as kvq_umma_decode.cu, x^ = diag(s) M^T diag(1 / max(lambda, 1e-6)) (q (.) sigma) (Sec. 3.1,
 // Sec. 5.1 item 1), with two changes that D = 256 forces:
 //
-//   * the B operand (256 x 256) does not fit one CTA's shared memory next to the staging buffers once it
-//     is split for precision, so CTAs work in pairs on the same tiles and each computes one half of the
-//     output columns: B is [128 outputs, K = 256] per CTA.  The two CTAs of a pair share nothing and never
-//     wait for each other; the packed tile is read twice (the second read hits L2).
-//   * bf16 output has a rounding step 8x coarser than fp16, and a result that is off by 1e-4 of the
-//     vector's rms already lands on the other side of enough rounding boundaries to miss the 1e-3
-//     tolerance.  So for bf16 both operands are carried in two fp16 terms: a = q sigma rho has 15
-//     significant bits and splits exactly into a_hi + a_lo (one half2 FMA), W' = W_hi + W_lo, and
-//     x^ = a_hi W_hi + a_lo W_hi + a_hi W_lo accumulates in fp32 (the a_lo W_lo term is below 1e-7).
-//     fp16 output needs one term.
+//   * One radix-2 step of the transform is taken out of the GEMM.  Every row of M is cos or sin of 2 pi k n / D,
+//     so moving n by D / 2 multiplies the row by (-1)^k, and in the packing of Eq. 2 the parity of k is the parity
+//     of the channel c.  With E_n the sum over the even channels and O_n the sum over the odd ones (n < 128),
+//         x^_n = s_n (E_n + O_n),      x^_{n+128} = s_{n+128} (E_n - O_n) = (s_n s_{n+128}) s_n (E_n - O_n).
+//     E and O are two 128 x 128 x 128 GEMMs instead of one 128 x 256 x 256: half the tensor-core work, and a B
+//     operand (64 KB per fp16 term) that fits one CTA's shared memory even when it is split for precision.  The
+//     half2 nibble trick already delivers the codes in pairs (c, c + 4) of equal parity, so routing them to the
+//     two A operands costs nothing; the +- and the signs are a few instructions per output in the epilogue.
+//   * bf16 output has a rounding step 8x coarser than fp16, and a result that is off by 1e-4 of the vector's rms
+//     already lands on the other side of enough rounding boundaries to miss the 1e-3 tolerance.  So for bf16 both
+//     operands are carried in two fp16 terms: a = q sigma rho has 15 significant bits and splits exactly into
+//     a_hi + a_lo (one half2 FMA), W' = W_hi + W_lo, and a_hi W_hi + a_lo W_hi + a_hi W_lo accumulates in fp32
+//     (the a_lo W_lo term is below 1e-7).  fp16 output needs one term.
 //
-// The A operand lives in tensor memory by K halves (128 codes: 64 columns, twice that with a_lo), two
-// stages; the accumulator (128 columns) has two stages.  Roles as in kvq_umma_decode.cu: producer (TMA),
-// two dequant groups, one mma thread, two epilogue groups; every wait is bounded.
+//   warp 0        producer   one TMA tensor load per tile: 128 packed rows x 128 B, 128-byte swizzle, 4 stages (2 for bf16)
+//   warps 2-9     dequant    two groups of four warps, thread = row, both on every tile: group 0 turns the even
+//                            channels of the row's packed words into the A operand of the E GEMM, group 1 the
+//                            odd ones into that of the O GEMM (tensor memory; two stages each for fp16 output,
+//                            one with a_lo beside a_hi for bf16).  Each group also owns the B operand of its
+//                            GEMM and rebuilds it when the lambda row changes, behind its own barriers.
+//   warp 1        mma        per tile: E GEMM into accumulator columns 0-127, O GEMM into 128-255 (8 K-steps per
+//                            term each, A from tensor memory, B from shared memory)
+//   warps 10-17   epilogue   all eight warps on every tile (the accumulator has one stage): thread = (row, 64 of the
+//                            128 column pairs); E + O and E - O, sign, 16-bit rounding, 64-byte-swizzled staging,
+//                            TMA tensor stores of 32 x 32 boxes; the accumulator is released as soon as the last
+//                            values are in registers
+//
+// Every wait is bounded: on a time-out the role records the reason in the status word, raises the CTA's abort
+// flag and leaves its loop; the CTA then frees its tensor memory and returns.
 #include "kvq_internal.h"
 #include "kvq_umma.cuh"
 
@@ -27,34 +42,36 @@ namespace {
 constexpr int kD = 256;
 constexpr int kG = kD / 32;
 constexpr int kTile = 128;       // vectors per tile = MMA M
-constexpr int kHalfN = 128;      // output columns per CTA = MMA N
-constexpr int kThreads = 576;    // producer, mma, 2 x 4 dequant, 2 x 4 epilogue warps
-constexpr int kInStages = 4;     // packed tiles in flight (16 KB each); even, so that a stage always serves the same dequant group
-constexpr int kAStages = 2;      // K halves of A in tensor memory
-constexpr int kAccStages = 2;
+constexpr int kHalf = 128;       // outputs n < 128 per GEMM = MMA N; also K of each GEMM (channels of one parity)
+constexpr int kThreads = 576;    // producer, mma, 2 x 4 dequant, 8 epilogue warps
+constexpr int kMaxInStages = 4;
 constexpr int kInBytes = kTile * (kD / 2);             // 16 KB
-constexpr int kBBlock = kHalfN * 128;                  // one K block of 64: 128 rows x 128 B
-constexpr int kBTerm = 4 * kBBlock;                    // 64 KB: K = 256
-constexpr int kOutWarpBytes = 32 * 128;                // one 64-column box per epilogue warp
-constexpr int kCtrlBytes = 256;
+constexpr int kBBlock = kHalf * 128;                   // one K block of 64: 128 rows x 128 B
+constexpr int kBPart = 2 * kBBlock;                    // 32 KB: one parity of one term, K = 128
+constexpr int kOutWarpBytes = 2 * 2 * 32 * 64;         // per epilogue warp: two chunks x two [32 rows][64 B] boxes
+constexpr int kCtrlBytes = 512;
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kACol0 = 256;                       // accumulators at 0 and 128; A stages of 128 columns behind them
-constexpr uint32_t kIdesc = umma_idesc_m128(kHalfN, false);
+constexpr uint32_t kACol0 = 256;                       // accumulator E at 0, O at 128; A of parity p at 256 + 128 p (hi, then lo)
+constexpr uint32_t kIdesc = umma_idesc_m128(kHalf, false);
 
 template <bool BF16OUT>
 struct Cfg {
-    static constexpr int kBTerms = BF16OUT ? 2 : 1;    // W_hi (, W_lo)
-    static constexpr int kSmemBytes = kBTerms * kBTerm + kInStages * kInBytes + 8 * kOutWarpBytes + kCtrlBytes + 1024;
+    static constexpr int kTerms = BF16OUT ? 2 : 1;     // fp16 terms per operand
+    static constexpr int kAStages = BF16OUT ? 1 : 2;   // per parity: 128 columns hold a_hi | a_lo, or two stages of a_hi
+    static constexpr int kBBytes = kTerms * 2 * kBPart;
+    static constexpr int kInStages = BF16OUT ? 2 : 4;  // packed tiles in flight (16 KB each): what the split B leaves room for
+    static constexpr int kSmemBytes = kBBytes + kInStages * kInBytes + 8 * kOutWarpBytes + kCtrlBytes + 1024;
 };
 
 struct Ctrl {
-    uint64_t in_full[kInStages], in_empty[kInStages];
-    uint64_t a_full[kAStages], a_empty[2][kAStages];   // a_empty[g][s]: a unit of dequant group g has been read from stage s
-    uint64_t acc_full[kAccStages], acc_empty[kAccStages];
+    uint64_t in_full[kMaxInStages], in_empty[kMaxInStages];
+    uint64_t a_full[2][2], a_empty[2][2];   // [parity][stage]
+    uint64_t acc_full, acc_empty;
     uint64_t b_first;
     uint32_t tmem_base;
     volatile uint32_t abort;
-    volatile uint32_t b_epoch;   // lambda rows whose last MMA is complete, counted from the CTA's first one
+    uint32_t pad[2];
+    uint4 flip[16];   // sign-bit masks of s_n s_{n+128} for the output pairs (n, n + 1), n = 0, 2, .. 126
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
 
@@ -63,6 +80,14 @@ __device__ __forceinline__ uint32_t lop3_and_or(uint32_t a, uint32_t b, uint32_t
     uint32_t d;
     asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));   // (a & b) | c
     return d;
+}
+
+// 8 consecutive columns of this thread's tensor-memory lane
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&r)[8])
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"r"(taddr), "r"(r[0]), "r"(r[1]),
+                 "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+                 : "memory");
 }
 
 // 1 / max(lambda, 1e-6) for the channels 4 i .. 4 i + 3, i = lane and lane + 32, divided by rho, the power of two
@@ -88,36 +113,39 @@ struct RecipLambda {
     }
 };
 
-// Rows [n0, n1) of this CTA's half of the B operand (output column 128 half + n), by one warp.  A lane reads four
-// table entries per pass, scales them, trades two values with its neighbour so that each lane holds two K-ordered
-// pairs (the K order of a word of 8 codes is (0,4,1,5,2,6,3,7)), peels off fp16 terms and writes 8 bytes of each
-// term's swizzled row.
+// Rows [n0, n1) (outputs n < 128) of the B operand of parity p (0: E GEMM, even channels; 1: O GEMM), by one warp.
+// The table row b0[n][c] = s_n M[c][n] is used as it is: the accumulators then hold s_n E_n and s_n O_n.  Lanes 2w and 2w + 1 hold
+// channels 8w .. 8w + 7; the K order inside a word is the one the nibble trick produces, pairs (c, c + 4): the even
+// lane assembles the pair (8w + p, 8w + p + 4), the odd lane (8w + p + 2, 8w + p + 6), each from one value of its
+// own and one of its neighbour's.  Terms: fp16(W'), then what that left behind.
 template <int TERMS>
-__device__ __forceinline__ void build_b_rows(unsigned char *sB, const float *__restrict__ b0, const RecipLambda &rl, int half, int n0,
-                                             int n1, int lane)
+__device__ __forceinline__ void build_b_rows(unsigned char *sB, const float *__restrict__ b0, const RecipLambda &rl, int p, int n0, int n1, int lane)
 {
     const bool odd = lane & 1;
-#pragma unroll 2
+#pragma unroll 4
     for (int n = n0; n < n1; ++n) {
 #pragma unroll
-        for (int p = 0; p < 2; ++p) {
-            const int i = lane + 32 * p;
-            const float4 m = __ldg(reinterpret_cast<const float4 *>(b0 + (size_t)(half * kHalfN + n) * kD) + i);
+        for (int ps = 0; ps < 2; ++ps) {
+            const int i = lane + 32 * ps;
+            const float4 m = __ldg(reinterpret_cast<const float4 *>(b0 + (size_t)n * kD) + i);
             auto sat = [](float v) { return fminf(fmaxf(v, -65504.0f), 65504.0f); };
-            const float vx = sat(m.x * rl.r[p].x), vy = sat(m.y * rl.r[p].y), vz = sat(m.z * rl.r[p].z), vw = sat(m.w * rl.r[p].w);
-            const float r0 = __shfl_xor_sync(0xFFFFFFFFu, odd ? vx : vz, 1);
-            const float r1 = __shfl_xor_sync(0xFFFFFFFFu, odd ? vy : vw, 1);
-            float w[4];   // two K-ordered pairs: odd lane (2, 6), (3, 7); even lane (0, 4), (1, 5)
-            w[0] = odd ? r0 : vx, w[1] = odd ? vz : r0, w[2] = odd ? r1 : vy, w[3] = odd ? vw : r1;
-            const int ch = i >> 1;   // 16-byte chunk of the K-major row: K block ch / 8, chunk ch % 8
-            const uint32_t off = (uint32_t)((ch >> 3) * kBBlock + n * 128 + (((ch & 7) ^ (n & 7)) << 4) + (odd ? 8 : 0));
+            // this lane's two channels of parity p: 4 i + p and 4 i + p + 2
+            const float v0 = sat((p ? m.y : m.x) * (p ? rl.r[ps].y : rl.r[ps].x));
+            const float v2 = sat((p ? m.w : m.z) * (p ? rl.r[ps].w : rl.r[ps].z));
+            // even lane (channels 8w ..): keeps v0 = 8w + p, needs the odd lane's v0 = 8w + p + 4
+            // odd lane (channels 8w + 4 ..): keeps v2 = 8w + p + 6, needs the even lane's v2 = 8w + p + 2
+            const float got = __shfl_xor_sync(0xFFFFFFFFu, odd ? v0 : v2, 1);
+            float w0 = odd ? got : v0, w1 = odd ? v2 : got;
+            const int wd = i >> 1;   // word of 8 codes: columns 2 wd (even lane) and 2 wd + 1 (odd lane) of the K-major row
+            const int ch = wd >> 1;  // 16-byte chunk: K block ch / 8, chunk ch % 8
+            const uint32_t off = (uint32_t)(p * kBPart + (ch >> 3) * kBBlock + n * 128 + (((ch & 7) ^ (n & 7)) << 4) + ((wd & 1) ? 8 : 0) + (odd ? 4 : 0));
 #pragma unroll
             for (int t = 0; t < TERMS; ++t) {
-                const uint32_t lo = narrow2<false>(w[0], w[1]), hi = narrow2<false>(w[2], w[3]);
-                *reinterpret_cast<uint2 *>(sB + t * kBTerm + off) = make_uint2(lo, hi);
+                const uint32_t h = narrow2<false>(w0, w1);
+                *reinterpret_cast<uint32_t *>(sB + t * (2 * kBPart) + off) = h;
                 if (t + 1 < TERMS) {   // what the fp16 term left behind (exact in fp32)
-                    const float2 a = widen2<false>(lo), b = widen2<false>(hi);
-                    w[0] -= a.x, w[1] -= a.y, w[2] -= b.x, w[3] -= b.y;
+                    const float2 a = widen2<false>(h);
+                    w0 -= a.x, w1 -= a.y;
                 }
             }
         }
@@ -131,11 +159,12 @@ struct UmmaDecode256Params {
     int64_t rpl;        // rows per lambda segment (N when there is one lambda row)
     int64_t n_seg;      // segments
     int64_t n_full;     // segments of exactly rpl rows, covered by the main output map; a shorter last one uses the tail map
+    uint32_t sign_xor[128];   // word m: bit 15 set if s_{2m} = -1, bit 31 set if s_{2m+1} = -1
 };
 
 struct UmmaDecode256Maps {
     CUtensorMap packed;       // [N, 128] bytes, box 128 rows, 128-byte swizzle
-    CUtensorMap out, tail;    // output, boxes of 64 columns x 32 rows (128-byte swizzle)
+    CUtensorMap out, tail;    // output, boxes of 32 columns x 32 rows (64-byte swizzle)
 };
 
 template <bool BF16OUT>
@@ -143,46 +172,45 @@ __global__ void __launch_bounds__(kThreads, 1)
     kvq_decode_umma_d256_kernel(const __grid_constant__ UmmaDecode256Params prm, const __grid_constant__ UmmaDecode256Maps maps)
 {
     using C = Cfg<BF16OUT>;
-    constexpr int kATerms = BF16OUT ? 2 : 1;
+    constexpr int kTerms = C::kTerms, kInStages = C::kInStages;
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    unsigned char *sB = smem;
-    unsigned char *sIn = sB + C::kBTerms * kBTerm;
+    unsigned char *sB = smem;                           // [term][parity][2 K blocks][128 rows][128 B]
+    unsigned char *sIn = sB + C::kBBytes;
     unsigned char *sOut = sIn + kInStages * kInBytes;
     Ctrl *ctrl = reinterpret_cast<Ctrl *>(sOut + 8 * kOutWarpBytes);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int half = blockIdx.x & 1;            // which 128 output columns this CTA computes
-    const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kInStages; ++s) {
             mbar_init(smem_u32(&ctrl->in_full[s]), 1);
-            mbar_init(smem_u32(&ctrl->in_empty[s]), 4);
+            mbar_init(smem_u32(&ctrl->in_empty[s]), 8);   // both dequant groups read every tile
         }
-        for (int s = 0; s < kAStages; ++s) {
-            mbar_init(smem_u32(&ctrl->a_full[s]), 4);
-            mbar_init(smem_u32(&ctrl->a_empty[0][s]), 1);
-            mbar_init(smem_u32(&ctrl->a_empty[1][s]), 1);
-        }
-        for (int s = 0; s < kAccStages; ++s) {
-            mbar_init(smem_u32(&ctrl->acc_full[s]), 1);
-            mbar_init(smem_u32(&ctrl->acc_empty[s]), 4);
-        }
+        for (int p = 0; p < 2; ++p)
+            for (int st = 0; st < 2; ++st) {
+                mbar_init(smem_u32(&ctrl->a_full[p][st]), 4);
+                mbar_init(smem_u32(&ctrl->a_empty[p][st]), 1);
+            }
+        mbar_init(smem_u32(&ctrl->acc_full), 1);
+        mbar_init(smem_u32(&ctrl->acc_empty), 8);
         mbar_init(smem_u32(&ctrl->b_first), 16);
         ctrl->abort = 0u;
-        ctrl->b_epoch = 0u;
         mbar_init_fence();
+    }
+    if (threadIdx.x >= 32 && threadIdx.x < 96) {   // sign of s_n s_{n+128}: the xor of the two sign bits
+        const int m = threadIdx.x - 32;
+        reinterpret_cast<uint32_t *>(ctrl->flip)[m] = prm.sign_xor[m] ^ prm.sign_xor[m + 64];
     }
     if (warp == 0) tmem_alloc(smem_u32(&ctrl->tmem_base), kTmemCols);
 
-    // ---- tiles: lambda segments of rpl rows, cut into tiles of 128 rows; a contiguous range of tiles per CTA pair
+    // ---- tiles: lambda segments of rpl rows, cut into tiles of 128 rows; a contiguous range of tiles per CTA
     const int64_t N = prm.g.N, rpl = prm.rpl;
     const int64_t tps = (rpl + kTile - 1) / kTile;
     const int64_t n_tiles = prm.n_seg * tps;
-    const int64_t per_pair = (n_tiles + n_pairs - 1) / n_pairs;
-    const int64_t tile_begin = (int64_t)pair * per_pair;
-    const int64_t tile_end = tile_begin + per_pair < n_tiles ? tile_begin + per_pair : n_tiles;
+    const int64_t per_cta = (n_tiles + gridDim.x - 1) / gridDim.x;
+    const int64_t tile_begin = (int64_t)blockIdx.x * per_cta;
+    const int64_t tile_end = tile_begin + per_cta < n_tiles ? tile_begin + per_cta : n_tiles;
     const int n_my = tile_end > tile_begin ? (int)(tile_end - tile_begin) : 0;
     const int64_t seg_first = n_my > 0 ? tile_begin / tps : 0;
     auto lambda_row = [&](int64_t seg) -> const float * { return prm.g.lambda + (prm.g.n_lambda == 1 ? 0 : seg) * kD; };
@@ -195,10 +223,12 @@ __global__ void __launch_bounds__(kThreads, 1)
     volatile uint32_t *abort_flag = &ctrl->abort;
     uint32_t *status = prm.g.status;
 
-    // ---- B for the first tile's lambda row: the sixteen dequant and epilogue warps build eight rows each
+    // ---- B for the first tile's lambda row: of the sixteen dequant and epilogue warps, eight build the E operand
+    // ---- and eight the O operand, sixteen rows each
     if (n_my > 0 && warp >= 2) {
         const RecipLambda rl(lambda_row(seg_first), lane);
-        build_b_rows<C::kBTerms>(sB, prm.g.b0, rl, half, (warp - 2) * 8, (warp - 1) * 8, lane);
+        const int bp = ((warp - 2) >> 2) & 1, bw = ((warp - 2) & 3) + 4 * ((warp - 2) >> 3);   // parity, position among its eight
+        build_b_rows<kTerms>(sB, prm.g.b0, rl, bp, bw * 16, bw * 16 + 16, lane);
         fence_proxy_async();   // B is read by the tensor core through the async proxy
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&ctrl->b_first));
@@ -234,104 +264,71 @@ __global__ void __launch_bounds__(kThreads, 1)
             int n_mma = n_my;
             if (n_my > 0 && !wait_or_abort(smem_u32(&ctrl->b_first), 0u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT)) n_mma = 0;
             bool ok = true;
-            TileCursor cur(tile_begin, tps);
-            for (int j = 0; j < n_mma && ok; ++j, cur.advance(1)) {
-                const int sc = j % kAccStages;
-                // A new lambda row: a dequant group will overwrite B once every MMA issued so far has read the old one.  This
-                // thread waits for the previous tile's accumulator barrier itself (it is at most one phase behind: the stage
-                // was free when that tile was issued) and publishes a count; a counter, unlike a parity, cannot be misread
-                // by a group that skipped a rebuild.  The tensor core drains once per lambda row.
-                if (j > 0 && cur.first_of_segment()) {
-                    if (!wait_or_abort(smem_u32(&ctrl->acc_full[(j - 1) % kAccStages]), (uint32_t)((j - 1) / kAccStages) & 1u, abort_flag,
-                                       status, KVQ_DEV_MMA_TIMEOUT))
-                        break;
-                    ctrl->b_epoch = (uint32_t)(cur.seg - seg_first);
-                    __threadfence_block();
-                }
-                if (!wait_or_abort(smem_u32(&ctrl->acc_empty[sc]), ((uint32_t)(j / kAccStages) & 1u) ^ 1u, abort_flag, status,
-                                   KVQ_DEV_SLOT_TIMEOUT))
-                    break;
-                const uint32_t d_tmem = tmem_base + (uint32_t)sc * kHalfN;
+            for (int j = 0; j < n_mma && ok; ++j) {
+                // the epilogue has taken the previous tile's E and O out of tensor memory
+                if (!wait_or_abort(smem_u32(&ctrl->acc_empty), ((uint32_t)j & 1u) ^ 1u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT)) break;
+                const int sa = j % C::kAStages;
 #pragma unroll
-                for (int kh = 0; kh < 2; ++kh) {   // K halves arrive one after the other
-                    const int u = 2 * j + kh, sa = u % kAStages;
-                    if (!wait_or_abort(smem_u32(&ctrl->a_full[sa]), (uint32_t)(u / kAStages) & 1u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT)) {
+                for (int p = 0; p < 2; ++p) {   // E GEMM, then O GEMM
+                    if (!wait_or_abort(smem_u32(&ctrl->a_full[p][sa]), (uint32_t)(j / C::kAStages) & 1u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT)) {
                         ok = false;
                         break;
                     }
                     tc_fence_after();
-                    const uint32_t a_tmem = tmem_base + kACol0 + (uint32_t)sa * 128u;
+                    const uint32_t d_tmem = tmem_base + (uint32_t)p * kHalf;
+                    const uint32_t a_tmem = tmem_base + kACol0 + (uint32_t)p * 128u + (uint32_t)sa * 64u;
                     // terms: a_hi W_hi (, a_lo W_hi, a_hi W_lo)
 #pragma unroll
                     for (int t = 0; t < (BF16OUT ? 3 : 1); ++t) {
                         const uint32_t a_base = a_tmem + (t == 1 ? 64u : 0u);
-                        const uint32_t b_term = (t == 2 ? (uint32_t)(kBTerm >> 4) : 0u);
+                        const uint32_t b_part = (uint32_t)((t == 2 ? 2 * kBPart : 0) + p * kBPart) >> 4;
 #pragma unroll
                         for (int ks = 0; ks < 8; ++ks) {
-                            // (bytes >> 4) of K-step 8 kh + ks: K block 2 kh + ks / 4
-                            const uint32_t koff = (uint32_t)(2 * kh + (ks >> 2)) * (kBBlock >> 4) + (uint32_t)(ks & 3) * 2u;
-                            const uint64_t bd = ((uint64_t)b_hi << 32) | (uint64_t)(b_lo + b_term + koff);
-                            if (kh > 0 || t > 0 || ks > 0) umma_f16_ts<true>(d_tmem, a_base + (uint32_t)ks * 8u, bd, kIdesc);
+                            const uint32_t koff = (uint32_t)(ks >> 2) * (kBBlock >> 4) + (uint32_t)(ks & 3) * 2u;   // (bytes >> 4) of K-step ks
+                            const uint64_t bd = ((uint64_t)b_hi << 32) | (uint64_t)(b_lo + b_part + koff);
+                            if (t > 0 || ks > 0) umma_f16_ts<true>(d_tmem, a_base + (uint32_t)ks * 8u, bd, kIdesc);
                             else umma_f16_ts<false>(d_tmem, a_base, bd, kIdesc);
                         }
                     }
-                    umma_commit(smem_u32(&ctrl->a_empty[j & 1][sa]));   // tile j belongs to dequant group j & 1
+                    umma_commit(smem_u32(&ctrl->a_empty[p][sa]));
                 }
-                if (ok) umma_commit(smem_u32(&ctrl->acc_full[sc]));
+                if (ok) umma_commit(smem_u32(&ctrl->acc_full));
             }
         }
     } else if (warp < 10) {
-        // =========================== dequant: packed codes -> A in tensor memory ===========================
-        const int grp = (warp - 2) >> 2;        // this group takes tiles grp, grp + 2, ...
+        // =========================== dequant: packed codes -> A operands in tensor memory ===========================
+        const int p = (warp - 2) >> 2;          // this group's parity: 0 = even channels (E GEMM), 1 = odd channels (O GEMM)
         const int q = warp & 3;                 // tensor-memory lane quarter this warp may touch
         const int r = q * 32 + lane;            // tile row and tensor-memory lane of this thread
         const uint4 *scales = static_cast<const uint4 *>(prm.g.scales);   // 8 fp16 scales per row
         int64_t cached_seg = n_my > 0 ? seg_first : -1;   // B holds this row's table (built above)
         float rho = RecipLambda(lambda_row(seg_first), lane).rho;
 
-        TileCursor cur(tile_begin + grp, tps), ahead(tile_begin + grp, tps);
+        TileCursor cur(tile_begin, tps), ahead(tile_begin, tps);
         auto fetch_scales = [&](int j) -> uint4 {
             if (j >= n_my) return make_uint4(0u, 0u, 0u, 0u);
             const int64_t row = ahead.seg * rpl + ahead.row_in_segment() + r;
             return row < N ? __ldg(scales + row) : make_uint4(0u, 0u, 0u, 0u);
         };
-        uint4 sc_next = fetch_scales(grp);
-        bool ok = true;
-        for (int j = grp; j < n_my && ok; j += 2, cur.advance(2)) {
+        uint4 sc_next = fetch_scales(0);
+        for (int j = 0; j < n_my; ++j, cur.advance(1)) {
             const uint4 sc4 = sc_next;
             const uint32_t sc[4] = {sc4.x, sc4.y, sc4.z, sc4.w};
-            ahead.advance(2);
-            sc_next = fetch_scales(j + 2);
+            ahead.advance(1);
+            sc_next = fetch_scales(j + 1);
             const int64_t seg = cur.seg;
+            const int sa = j % C::kAStages;
 
-            // ---- a new lambda row: this group needs its rho; the group that meets the row's first tile rebuilds B
+            // ---- a new lambda row: new rho, and this group rebuilds the B operand of its own GEMM once every MMA of that
+            // ---- GEMM issued so far is complete: the previous tile's, on this group's own barriers (it sees every phase)
             if (seg != cached_seg) {
                 const RecipLambda rl(lambda_row(seg), lane);
                 rho = rl.rho;
-                if (cur.first_of_segment()) {
-                    // every MMA issued so far must have read B: the mma thread says so by raising b_epoch to this row's index
-                    {
-                        const uint32_t need = (uint32_t)(seg - seg_first);
-                        bool freed = false;
-                        for (uint32_t it = 0; it < (1u << 22); ++it) {
-                            if (ctrl->b_epoch >= need) {
-                                freed = true;
-                                break;
-                            }
-                            if (*abort_flag) break;
-                            __nanosleep(64);
-                        }
-                        if (!freed) {
-                            if (!*abort_flag) {
-                                *abort_flag = 1u;
-                                atomicOr(status, KVQ_DEV_MMA_TIMEOUT);
-                            }
-                            break;
-                        }
-                    }
-                    build_b_rows<C::kBTerms>(sB, prm.g.b0, rl, half, q * 32, q * 32 + 32, lane);
-                    fence_proxy_async();   // B is read by the tensor core through the async proxy
-                }
+                if (!wait_or_abort(smem_u32(&ctrl->a_empty[p][(j - 1) % C::kAStages]), (uint32_t)((j - 1) / C::kAStages) & 1u, abort_flag,
+                                   status, KVQ_DEV_MMA_TIMEOUT))
+                    break;
+                build_b_rows<kTerms>(sB, prm.g.b0, rl, p, q * 32, q * 32 + 32, lane);
+                fence_proxy_async();   // B is read by the tensor core through the async proxy
                 cached_seg = seg;
             }
 
@@ -347,61 +344,51 @@ __global__ void __launch_bounds__(kThreads, 1)
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctrl->in_empty[s]));   // the values are in registers
 
+            // ---- the operand stage is free again (the MMAs of the tile that used it last are complete)
+            if (!wait_or_abort(smem_u32(&ctrl->a_empty[p][sa]), ((uint32_t)(j / C::kAStages) & 1u) ^ 1u, abort_flag, status, KVQ_DEV_MMA_TIMEOUT))
+                break;
+            tc_fence_after();
+            const uint32_t a_row = tmem_base + ((uint32_t)(q * 32) << 16) + kACol0 + (uint32_t)p * 128u + (uint32_t)sa * 64u;
             const __half2 h1032 = __float2half2_rn(1032.0f);
 #pragma unroll
-            for (int kh = 0; kh < 2; ++kh) {   // K half kh: groups 4 kh .. 4 kh + 3
-                const int u = 2 * j + kh, sa = u % kAStages;
-                // The stage was last used by unit u - 2, a K half of the other group's tile j - 1.  Each (group, stage)
-                // pair has a barrier of its own, so that this group sees its phases one by one: a parity wait cannot
-                // tell a phase from the one two before it.
-                if (j >= 1 && !wait_or_abort(smem_u32(&ctrl->a_empty[(j - 1) & 1][sa]), (uint32_t)((u - 2) / 4) & 1u, abort_flag, status,
-                                             KVQ_DEV_MMA_TIMEOUT)) {
-                    ok = false;
-                    break;
-                }
-                tc_fence_after();
-                const uint32_t a_row = tmem_base + ((uint32_t)(q * 32) << 16) + kACol0 + (uint32_t)sa * 128u;
+            for (int c = 0; c < kG; ++c) {   // group c: 16 codes of this parity, 8 tensor-memory columns
+                const float sig = __half2float(__ushort_as_half((unsigned short)((sc[c >> 1] >> (16 * (c & 1))) & 0xFFFFu)));
+                const __half2 s2 = __float2half2_rn(sig * rho);
+                const uint32_t words[4] = {pk[c].x, pk[c].y, pk[c].z, pk[c].w};
+                uint32_t a_hi[8], a_lo[8];
 #pragma unroll
-                for (int cc = 0; cc < 4; ++cc) {
-                    const int c = 4 * kh + cc;   // group: 32 codes, 16 tensor-memory columns
-                    const float sig = __half2float(__ushort_as_half((unsigned short)((sc[c >> 1] >> (16 * (c & 1))) & 0xFFFFu)));
-                    const __half2 s2 = __float2half2_rn(sig * rho);
-                    const uint32_t words[4] = {pk[c].x, pk[c].y, pk[c].z, pk[c].w};
-                    uint32_t a_hi[16], a_lo[16];
+                for (int i = 0; i < 4; ++i) {
+                    const uint32_t w = (words[i] ^ 0x88888888u) >> (4 * p);   // nibbles hold q + 8; parity p starts at nibble p
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const uint32_t w = words[i] ^ 0x88888888u;   // nibbles now hold q + 8
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const uint32_t m = lop3_and_or(w >> (4 * e), 0x000F000Fu, 0x64006400u);   // {1024 + n_e, 1024 + n_{e+4}}
-                            const __half2 qq = __hsub2(*reinterpret_cast<const __half2 *>(&m), h1032);   // exact codes
-                            const __half2 hi = __hmul2(qq, s2);                                          // one rounding
-                            a_hi[4 * i + e] = *reinterpret_cast<const uint32_t *>(&hi);
-                            if constexpr (kATerms == 2) {
-                                const __half2 lo = __hfma2(qq, s2, __hneg2(hi));   // q s - hi: exact, the product has 15 bits
-                                a_lo[4 * i + e] = *reinterpret_cast<const uint32_t *>(&lo);
-                            }
+                    for (int t = 0; t < 2; ++t) {
+                        // nibbles 2t + p and 2t + p + 4 of the word: channels 8w + 2t + p and + 4, both of parity p
+                        const uint32_t m = lop3_and_or(w >> (8 * t), 0x000F000Fu, 0x64006400u);   // {1024 + n, 1024 + n'}
+                        const __half2 qq = __hsub2(*reinterpret_cast<const __half2 *>(&m), h1032);       // exact codes
+                        const __half2 hi = __hmul2(qq, s2);                                               // one rounding
+                        a_hi[2 * i + t] = *reinterpret_cast<const uint32_t *>(&hi);
+                        if constexpr (kTerms == 2) {
+                            const __half2 lo = __hfma2(qq, s2, __hneg2(hi));   // q s - hi: exact, the product has 15 bits
+                            a_lo[2 * i + t] = *reinterpret_cast<const uint32_t *>(&lo);
                         }
                     }
-                    tmem_st16(a_row + 16u * (uint32_t)cc, a_hi);
-                    if constexpr (kATerms == 2) tmem_st16(a_row + 64u + 16u * (uint32_t)cc, a_lo);
                 }
-                tmem_st_wait();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&ctrl->a_full[sa]));
+                tmem_st8(a_row + 8u * (uint32_t)c, a_hi);
+                if constexpr (kTerms == 2) tmem_st8(a_row + 64u + 8u * (uint32_t)c, a_lo);
             }
+            tmem_st_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctrl->a_full[p][sa]));
         }
     } else {
-        // =========================== epilogue: accumulator -> 16-bit -> TMA store ===========================
-        const int grp = (warp - 10) >> 2;
+        // =========================== epilogue: E, O -> x^ -> TMA store ===========================
         const int q = warp & 3;
-        unsigned char *stg = sOut + (warp - 10) * kOutWarpBytes;   // one [32 rows][128 B] box
+        const int ch = (warp - 10) >> 2;                            // this warp's half of the column pairs: n in [64 ch, 64 ch + 64)
+        unsigned char *stg_base = sOut + (warp - 10) * kOutWarpBytes;   // per chunk: two [32 rows][64 B] boxes
         const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
-        TileCursor cur(tile_begin + grp, tps);
-        for (int j = grp; j < n_my; j += 2, cur.advance(2)) {
-            const int sc = j % kAccStages;
-            if (!wait_or_abort(smem_u32(&ctrl->acc_full[sc]), (uint32_t)(j / kAccStages) & 1u, abort_flag, status, KVQ_DEV_MMA_TIMEOUT)) break;
+        TileCursor cur(tile_begin, tps);
+        for (int j = 0; j < n_my; ++j, cur.advance(1)) {
+            if (!wait_or_abort(smem_u32(&ctrl->acc_full), (uint32_t)j & 1u, abort_flag, status, KVQ_DEV_MMA_TIMEOUT)) break;
             tc_fence_after();
             const int64_t seg = cur.seg;
             const int row_in_seg = (int)cur.row_in_segment() + q * 32;
@@ -409,31 +396,42 @@ __global__ void __launch_bounds__(kThreads, 1)
             const CUtensorMap *tm = tail ? &maps.tail : &maps.out;
             const int segc = tail ? 0 : (int)seg;
 #pragma unroll
-            for (int b = 0; b < 2; ++b) {   // two boxes of 64 columns through the same staging tile
-                if (lane == 0) bulk_wait_read_all();   // the previous store has read the staging tile
+            for (int cc = 0; cc < 2; ++cc) {   // 32 column pairs at a time: outputs n0 .. n0 + 31 and 128 + n0 ..
+                const int n0 = 64 * ch + 32 * cc;
+                unsigned char *stg = stg_base + cc * (2 * 32 * 64);
+                uint32_t e[32], o[32];
+                tmem_ld32(lane_addr + (uint32_t)n0, e);
+                tmem_ld32(lane_addr + (uint32_t)(kHalf + n0), o);
+                tmem_ld_wait();
+                if (cc == 1) {   // the last values are in registers: hand the accumulator back
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&ctrl->acc_empty));
+                }
+                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");   // the stores of this chunk's boxes one tile ago have read them
                 __syncwarp();
 #pragma unroll
-                for (int cc = 0; cc < 2; ++cc) {
-                    uint32_t v[32];
-                    tmem_ld32(lane_addr + (uint32_t)sc * kHalfN + (uint32_t)(2 * b + cc) * 32u, v);
-                    tmem_ld_wait();
+                for (int k = 0; k < 4; ++k) {   // 16-byte chunk k of each box row: 8 outputs
+                    const uint4 fl = ctrl->flip[(n0 >> 3) + k];   // warp-uniform address: a broadcast
+                    const uint32_t f[4] = {fl.x, fl.y, fl.z, fl.w};
+                    uint32_t lo[4], hi[4];
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        uint4 o;
-                        o.x = narrow2<BF16OUT>(__uint_as_float(v[8 * k]), __uint_as_float(v[8 * k + 1]));
-                        o.y = narrow2<BF16OUT>(__uint_as_float(v[8 * k + 2]), __uint_as_float(v[8 * k + 3]));
-                        o.z = narrow2<BF16OUT>(__uint_as_float(v[8 * k + 4]), __uint_as_float(v[8 * k + 5]));
-                        o.w = narrow2<BF16OUT>(__uint_as_float(v[8 * k + 6]), __uint_as_float(v[8 * k + 7]));
-                        const int chunk = cc * 4 + k;
-                        *reinterpret_cast<uint4 *>(stg + lane * 128 + ((chunk ^ (lane & 7)) << 4)) = o;
+                    for (int v = 0; v < 4; ++v) {
+                        const int i = 8 * k + 2 * v;
+                        const float e0 = __uint_as_float(e[i]), e1 = __uint_as_float(e[i + 1]);
+                        const float o0 = __uint_as_float(o[i]), o1 = __uint_as_float(o[i + 1]);
+                        lo[v] = narrow2<BF16OUT>(e0 + o0, e1 + o1);          // s_n is already in E and O
+                        hi[v] = narrow2<BF16OUT>(e0 - o0, e1 - o1) ^ f[v];   // times s_n s_{n+128}
                     }
+                    const uint32_t off = (uint32_t)(lane * 64 + ((k ^ ((lane >> 1) & 3)) << 4));   // 64-byte swizzle
+                    *reinterpret_cast<uint4 *>(stg + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                    *reinterpret_cast<uint4 *>(stg + 32 * 64 + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
                 }
-                if (b == 1) tc_fence_before();
                 fence_proxy_async();
                 __syncwarp();
                 if (lane == 0) {
-                    if (b == 1) mbar_arrive(smem_u32(&ctrl->acc_empty[sc]));
-                    tma_store_3d(tm, half * kHalfN + 64 * b, row_in_seg, segc, smem_u32(stg));
+                    tma_store_3d(tm, n0, row_in_seg, segc, smem_u32(stg));
+                    tma_store_3d(tm, kHalf + n0, row_in_seg, segc, smem_u32(stg + 32 * 64));
                     bulk_commit();
                 }
             }
@@ -455,7 +453,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 namespace {
 
 template <bool BF16OUT>
-cudaError_t launch(int64_t N, const GemmParams &g, cudaStream_t stream)
+cudaError_t launch(int64_t N, const GemmParams &g, const uint32_t *sign_xor, cudaStream_t stream)
 {
     using C = Cfg<BF16OUT>;
     static int sms = 0;
@@ -474,6 +472,7 @@ cudaError_t launch(int64_t N, const GemmParams &g, cudaStream_t stream)
     prm.rpl = g.n_lambda == 1 ? N : g.rows_per_lambda;
     prm.n_seg = (N + prm.rpl - 1) / prm.rpl;
     prm.n_full = N / prm.rpl;
+    for (int i = 0; i < 128; ++i) prm.sign_xor[i] = sign_xor[i];
 
     UmmaDecode256Maps maps;
     {
@@ -486,9 +485,9 @@ cudaError_t launch(int64_t N, const GemmParams &g, cudaStream_t stream)
     auto out_map = [&](CUtensorMap *tm, void *base, int64_t rows, int64_t segs) -> bool {
         const cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)rows, (cuuint64_t)segs};
         const cuuint64_t strides[2] = {(cuuint64_t)(2 * kD), (cuuint64_t)(2 * kD) * (cuuint64_t)rows};
-        const cuuint32_t box[3] = {64u, 32u, 1u};
+        const cuuint32_t box[3] = {32u, 32u, 1u};
         return make_tensor_map(tm, BF16OUT ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, base, dims, strides, box,
-                               CU_TENSOR_MAP_SWIZZLE_128B);
+                               CU_TENSOR_MAP_SWIZZLE_64B);
     };
     const int64_t tail_rows = N - prm.n_full * prm.rpl;
     unsigned char *tail_base = static_cast<unsigned char *>(g.out) + (size_t)prm.n_full * prm.rpl * (2 * kD);
@@ -498,17 +497,17 @@ cudaError_t launch(int64_t N, const GemmParams &g, cudaStream_t stream)
     if (prm.n_full == 0) maps.out = maps.tail;
 
     const int64_t tiles = prm.n_seg * ((prm.rpl + kTile - 1) / kTile);
-    const int64_t pairs = tiles < sms / 2 ? tiles : sms / 2;
-    kvq_decode_umma_d256_kernel<BF16OUT><<<(int)(2 * pairs), kThreads, C::kSmemBytes, stream>>>(prm, maps);
+    const int grid = (int)(tiles < sms ? tiles : sms);
+    kvq_decode_umma_d256_kernel<BF16OUT><<<grid, kThreads, C::kSmemBytes, stream>>>(prm, maps);
     count_launch();
     return cudaGetLastError();
 }
 
 }  // namespace
 
-cudaError_t umma_decode_d256(bool bf16, int64_t N, const GemmParams &g, cudaStream_t stream)
+cudaError_t umma_decode_d256(bool bf16, int64_t N, const GemmParams &g, const uint32_t *sign_xor, cudaStream_t stream)
 {
-    return bf16 ? launch<true>(N, g, stream) : launch<false>(N, g, stream);
+    return bf16 ? launch<true>(N, g, sign_xor, stream) : launch<false>(N, g, sign_xor, stream);
 }
 
 }  // namespace kvq
