@@ -259,6 +259,40 @@ int kvqo_srft_inverse(int D, const int8_t *sg, const double *z, double *x, int64
 }
 
 /* ------------------------------------------------------------------ */
+/* static lambda calibration (Sec. 7.1: "lambda_d = 1 / per-channel   */
+/* max of the SRFT output", taken once over a set of calibration      */
+/* vectors).  a_c = max_n |z_{n,c}|, lambda_c = 1 / a_c; a channel    */
+/* that is zero on every vector gets lambda_c = 1 (reading: any value */
+/* serves, the channel carries nothing).  Inputs are half-precision   */
+/* bit patterns widened exactly; the maxima are also returned.        */
+/* ------------------------------------------------------------------ */
+int kvqo_calibrate_lambda(int D, const int8_t *sg, const uint16_t *x, int dtype, int64_t N, double *lambda, double *amax)
+{
+    if (D < 2 || (D & 1) || N < 0) return 1;
+    trig_t t;
+    if (trig_init(&t, D)) return 2;
+    for (int c = 0; c < D; ++c) amax[c] = 0.0;
+    double *xv = (double *)malloc(sizeof(double) * (size_t)D * 2);
+    if (!xv) {
+        trig_free(&t);
+        return 2;
+    }
+    double *zv = xv + D;
+    for (int64_t r = 0; r < N; ++r) {
+        for (int n = 0; n < D; ++n) xv[n] = widen(x[r * D + n], dtype);
+        srft_forward_one(&t, sg, xv, zv);
+        for (int c = 0; c < D; ++c) {
+            double a = fabs(zv[c]);
+            if (a > amax[c]) amax[c] = a;
+        }
+    }
+    for (int c = 0; c < D; ++c) lambda[c] = amax[c] > 0.0 ? 1.0 / amax[c] : 1.0;
+    free(xv);
+    trig_free(&t);
+    return 0;
+}
+
+/* ------------------------------------------------------------------ */
 /* nibble layout (Sec. 3.2: byte = (q[2i+1] << 4) | (q[2i] & 0xF))     */
 /* ------------------------------------------------------------------ */
 

@@ -59,6 +59,8 @@ def _load():
         lib.kvqo_srft_forward.argtypes = [i32, p, p, p, i64]
         lib.kvqo_srft_inverse.restype = i32
         lib.kvqo_srft_inverse.argtypes = [i32, p, p, p, i64]
+        lib.kvqo_calibrate_lambda.restype = i32
+        lib.kvqo_calibrate_lambda.argtypes = [i32, p, p, i32, i64, p, p]
         lib.kvqo_pack_nibbles.restype = None
         lib.kvqo_pack_nibbles.argtypes = [p, i64, p]
         lib.kvqo_unpack_nibbles.restype = None
@@ -168,6 +170,20 @@ def srft_inverse(z, sg) -> np.ndarray:
     if rc:
         raise ValueError("kvqo_srft_inverse: rc=%d" % rc)
     return x
+
+
+def calibrate_lambda(x_raw, dtype: int, sg):
+    """Static lambda calibration (Sec. 7.1): lambda_c = 1 / max_n |SRFT(x_n)_c| over the rows of ``x_raw``
+    (half-precision bit patterns).  Returns (lambda [D] float64, amax [D] float64)."""
+    x = _raw16(x_raw)
+    D = x.shape[-1]
+    sg = np.ascontiguousarray(sg, dtype=np.int8)
+    lam = np.empty(D, dtype=np.float64)
+    amax = np.empty(D, dtype=np.float64)
+    rc = _load().kvqo_calibrate_lambda(D, _ptr(sg), _ptr(x), dtype, x.size // D, _ptr(lam), _ptr(amax))
+    if rc:
+        raise ValueError("kvqo_calibrate_lambda: rc=%d" % rc)
+    return lam, amax
 
 
 # ---- nibbles --------------------------------------------------------------

@@ -13,6 +13,7 @@ import pytest
 import torch
 
 from oracle import kvq_oracle as ko
+from paper_2605_05699_b200 import workloads as wl
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 DIMS = [2, 4, 8, 12, 64, 96, 128, 160, 256]
@@ -457,3 +458,44 @@ def test_layout_sizes_reproduce_the_papers_compression_arithmetic():
     assert abs((4 * D + packed_bytes + 4) - p["bytes_per_vec_fp32in_int4_d128"]) <= 1
     assert 5 * D * math.log2(D) == p["nominal_flops_d128"]
     assert math.log2(64 / 2) == p["fft_passes_d64"] and math.log2(128 / 2) == p["fft_passes_d128"]
+
+
+# ---- static lambda calibration (Sec. 7.1) -------------------------------------------------------
+
+@pytest.mark.parametrize("D", [64, 96, 128])
+def test_calibration_closed_form_on_vectors_with_known_spectra(D):
+    # rows that are inverse transforms of a_c e_c have exactly one non-zero channel each: lambda_c = 1 / max a_c
+    rng = np.random.default_rng(5)
+    sg = ko.signs(D, 9)
+    amps = rng.uniform(0.25, 4.0, size=(3, D))
+    amps *= rng.choice([-1.0, 1.0], size=amps.shape)
+    z = np.zeros((3 * D, D))
+    for rep in range(3):
+        z[rep * D + np.arange(D), np.arange(D)] = amps[rep]
+    x = ko.srft_inverse(z, sg)
+    # feed fp64-exact values through the fp16 entry point: keep only what fp16 holds, then compare with the same data
+    xb = ko.f64_to_f16(x)
+    lam, amax = ko.calibrate_lambda(xb, ko.F16, sg)
+    zz = ko.srft_forward(ko.f16_to_f64(xb), sg)
+    assert np.allclose(amax, np.abs(zz).max(axis=0), rtol=0, atol=0)          # the definition, on the rounded inputs
+    assert np.allclose(amax, np.abs(amps).max(axis=0), rtol=2e-3)             # the construction, up to fp16 input rounding
+    assert np.allclose(lam * amax, 1.0, rtol=1e-15)
+
+
+def test_calibration_makes_every_channel_peak_at_one_and_is_row_order_invariant():
+    D = 128
+    sg = ko.signs(D, 3)
+    x = wl.make_vectors(700, D, "f16", "k_outlier", 77)
+    xb = wl.raw_bits(x)
+    lam, amax = ko.calibrate_lambda(xb, ko.F16, sg)
+    v = ko.srft_forward(ko.f16_to_f64(xb), sg) * lam
+    assert np.allclose(np.abs(v).max(axis=0), 1.0, rtol=1e-14) and np.abs(v).max() <= 1.0 + 1e-14
+    perm = np.random.default_rng(1).permutation(len(xb))
+    lam2, _ = ko.calibrate_lambda(xb[perm], ko.F16, sg)
+    assert np.array_equal(lam, lam2)
+    # scaling the data by a power of two scales lambda by its inverse exactly
+    lam4, _ = ko.calibrate_lambda(wl.raw_bits(x * 4), ko.F16, sg)
+    assert np.array_equal(lam4 * 4, lam)
+    # a channel that never carries anything gets lambda = 1
+    lam0, amax0 = ko.calibrate_lambda(np.zeros((5, D), dtype=np.uint16), ko.F16, sg)
+    assert np.all(lam0 == 1.0) and np.all(amax0 == 0.0)
