@@ -137,6 +137,19 @@ kvq_status_t kvq_append(kvq_plan_t *plan, const void *x_new /* [S, D] */, kvq_dt
                         void *cuda_stream);
 
 /*
+ * kvq_calibrate_lambda -- static calibration of the per-channel rescale (Sec. 7.1: lambda_d = 1 / per-channel
+ * maximum of the SRFT output, taken in one pass over calibration vectors).
+ *   x           device, [N, D] row-major, fp16 or bf16 per `dtype`; 16-byte aligned: the calibration vectors.
+ *   lambda_out  device out, fp32 [D]; 16-byte aligned: lambda_c = 1 / max_n |(M (s (.) x_n))_c|, and 1 for a channel that
+ *               is zero on every vector (also for N == 0).  Used as the accumulator during the call.
+ * Runs the forward tensor-core kernel with lambda = 1 and an epilogue that reduces |z| over rows, then a D-thread
+ * kernel that takes reciprocals: two launches on the stream, no allocation beyond the plan's first use.  Built where
+ * the tensor-core encode kernel is (KVQ_ERR_UNSUPPORTED_DIM for D = 160 with bf16).
+ */
+kvq_status_t kvq_calibrate_lambda(kvq_plan_t *plan, const void *x, kvq_dtype_t dtype, int64_t N, float *lambda_out,
+                                  void *cuda_stream);
+
+/*
  * kvq_decode_static -- kvq_decode for callers that may not allocate device memory.  (The paper has
  * no counterpart: this entry point exists for how the library is embedded, not for the method.)
  *

@@ -37,7 +37,7 @@ KVQ_IMPL_GEMM = 2
 # every symbol include/kvq.h declares
 EXPORTS = (
     "kvq_plan_create", "kvq_plan_destroy", "kvq_plan_get_signs", "kvq_plan_describe", "kvq_plan_set_impl",
-    "kvq_plan_device_status", "kvq_encode", "kvq_decode", "kvq_append", "kvq_decode_static", "kvq_status_string",
+    "kvq_plan_device_status", "kvq_encode", "kvq_decode", "kvq_append", "kvq_decode_static", "kvq_calibrate_lambda", "kvq_status_string",
     "kvq_launch_count",
 )
 
@@ -79,6 +79,8 @@ def lib() -> ctypes.CDLL:
         L.kvq_append.argtypes = [vp, vp, i32, i64, vp, i64, i64, vp, vp, i64, i64, vp]
         L.kvq_decode_static.restype = i32
         L.kvq_decode_static.argtypes = [vp, vp, vp, i64, vp, i64, i64, vp, i32, vp, vp]
+        L.kvq_calibrate_lambda.restype = i32
+        L.kvq_calibrate_lambda.argtypes = [vp, vp, i32, i64, vp, vp]
         L.kvq_status_string.restype = ctypes.c_char_p
         L.kvq_status_string.argtypes = [i32]
         L.kvq_launch_count.restype = u64
@@ -213,6 +215,14 @@ def kvq_decode_static(plan: int, packed: torch.Tensor, scales: torch.Tensor, lam
                                        n_lambda, rows_per_lambda, _dev(out, "out"), _dtype_code(out), sw,
                                        _stream(stream)),
                "kvq_decode_static")
+
+
+def kvq_calibrate_lambda(plan: int, x: torch.Tensor, lambda_out: torch.Tensor, stream=None) -> None:
+    D = x.shape[-1]
+    N = x.numel() // D
+    with torch.cuda.device(x.device):
+        _check(lib().kvq_calibrate_lambda(plan, _dev(x, "x"), _dtype_code(x), N, _dev(lambda_out, "lambda_out"), _stream(stream)),
+               "kvq_calibrate_lambda")
 
 
 class Plan:

@@ -347,6 +347,46 @@ kvq_status_t kvq_decode(kvq_plan_t *plan, const uint8_t *packed, const void *sca
     return KVQ_OK;
 }
 
+// lambda_c = 1 / amax_c (1 where the channel carried nothing), in place over the bit patterns the reducing epilogue left
+static __global__ void kvq_calibrate_finish_kernel(float *lambda, int D)
+{
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c < D) {
+        const float a = lambda[c];
+        lambda[c] = a > 0.0f ? 1.0f / a : 1.0f;
+    }
+}
+
+kvq_status_t kvq_calibrate_lambda(kvq_plan_t *plan, const void *x, kvq_dtype_t dtype, int64_t N, float *lambda_out, void *cuda_stream)
+{
+    if (!plan || N < 0 || !lambda_out) return KVQ_ERR_INVALID_ARG;
+    if (dtype != KVQ_F16 && dtype != KVQ_BF16) return KVQ_ERR_INVALID_ARG;
+    if (N > 0 && !x) return KVQ_ERR_INVALID_ARG;
+    if (misaligned16(x) || misaligned16(lambda_out)) return KVQ_ERR_ALIGNMENT;
+    if (!umma_encode_supported(plan->D, dtype == KVQ_BF16)) return KVQ_ERR_UNSUPPORTED_DIM;
+    kvq_status_t st = ensure_device(plan);
+    if (st != KVQ_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemsetAsync(lambda_out, 0, sizeof(float) * (size_t)plan->D, stream) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return KVQ_ERR_CUDA;
+    }
+    if (N > 0) {
+        FftParams prm;
+        fill_params(plan, prm, N, nullptr, 1, 1);
+        prm.in = x;
+        if (umma_calibrate(plan->D, dtype == KVQ_BF16, N, prm, plan->d_e0, reinterpret_cast<uint32_t *>(lambda_out), stream) !=
+            cudaSuccess) {
+            (void)cudaGetLastError();
+            return KVQ_ERR_CUDA;
+        }
+    }
+    kvq_calibrate_finish_kernel<<<(plan->D + 127) / 128, 128, 0, stream>>>(lambda_out, plan->D);
+    count_launch();
+    if (cudaGetLastError() != cudaSuccess) return KVQ_ERR_CUDA;
+    return KVQ_OK;
+}
+
 const char *kvq_status_string(kvq_status_t status)
 {
     switch (status) {

@@ -44,6 +44,8 @@ bool umma_decode_supported(int D, bool bf16);
 bool umma_encode_supported(int D, bool bf16);
 cudaError_t umma_decode(int D, bool bf16, int64_t N, const GemmParams &prm, const uint32_t *sign_xor /* host, 128 words */,
                         cudaStream_t stream);
+cudaError_t umma_calibrate(int D, bool bf16, int64_t N, const FftParams &prm, const float *e0, uint32_t *amax_bits, cudaStream_t stream);
+cudaError_t umma_calibrate_d256(bool bf16, int64_t N, const FftParams &prm, const float *e0, uint32_t *amax_bits, cudaStream_t stream);
 cudaError_t umma_encode_d256(bool bf16, int64_t N, const FftParams &prm, const float *e0, cudaStream_t stream);   // kvq_umma_encode256.cu
 cudaError_t umma_decode_d256(bool bf16, int64_t N, const GemmParams &prm, const uint32_t *sign_xor, cudaStream_t stream);   // kvq_umma_decode256.cu
 cudaError_t umma_encode(int D, bool bf16, int64_t N, const FftParams &prm, const float *e0, cudaStream_t stream);

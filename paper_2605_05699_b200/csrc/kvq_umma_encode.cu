@@ -87,11 +87,11 @@ static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
 template <int D>
 __device__ __forceinline__ float lift_of(const float *__restrict__ lam, int lane)
 {
-    float mx = 0.0f;
+    float mx = lam ? 0.0f : 1.0f;   // no lambda row (calibration): lambda = 1
 #pragma unroll
     for (int p = 0; p < (D / 4 + 31) / 32; ++p) {
         const int i = lane + 32 * p;
-        if (i < D / 4) {
+        if (lam && i < D / 4) {
             const float4 l = __ldg(reinterpret_cast<const float4 *>(lam) + i);
             mx = fmaxf(mx, fmaxf(fmaxf(fabsf(l.x), fabsf(l.y)), fmaxf(fabsf(l.z), fabsf(l.w))));
         }
@@ -114,7 +114,7 @@ __device__ __forceinline__ void build_b_rows(unsigned char *sB, const float *__r
     using C = Cfg<D, BF16>;
 #pragma unroll 4
     for (int c = c0; c < c1; ++c) {
-        const float f = __ldg(lam + c) * lift;
+        const float f = lam ? __ldg(lam + c) * lift : lift;
 #pragma unroll
         for (int p = 0; p < (D / 4 + 31) / 32; ++p) {
             const int i = lane + 32 * p;
@@ -150,9 +150,10 @@ struct UmmaEncodeParams {
     int64_t n_seg;
     int64_t out_mul, out_add;   // output row of input row r is r * out_mul + out_add
     uint32_t *status;
+    uint32_t *amax_bits;        // calibration only: [D] running column maxima as fp32 bit patterns (start at zero)
 };
 
-template <int D, bool BF16>
+template <int D, bool BF16, bool CALIB>
 __global__ void __launch_bounds__(kThreads, 1)
     kvq_encode_umma_kernel(const __grid_constant__ UmmaEncodeParams prm, const __grid_constant__ CUtensorMap tm_x)
 {
@@ -285,7 +286,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         float unlift = 1.0f;
         if (n_my > 0) {   // B for the CTA's first lambda row: D / 16 rows per warp, all sixteen warps
             TileCursor first(tile_begin, tps);
-            const float *lam = prm.lambda + (prm.n_lambda == 1 ? 0 : first.seg) * D;
+            const float *lam = CALIB ? nullptr : prm.lambda + (prm.n_lambda == 1 ? 0 : first.seg) * D;
             const float lift = lift_of<D>(lam, lane);
             build_b_rows<D, BF16>(sB, prm.e0, lam, lift, (warp - 2) * (D / 16), (warp - 1) * (D / 16), lane);
             fence_proxy_async();   // B is read by the tensor core through the async proxy
@@ -294,6 +295,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             unlift = 1.0f / lift;
             cached_seg = first.seg;
         }
+        float colmax[C::kGroupsPerPart] = {};   // calibration: lane i keeps the running maximum of column i of each of this thread's groups
         TileCursor cur(tile_begin + set, tps);
         for (int j = set; j < n_my; j += 2, cur.advance(2)) {
             __syncwarp();
@@ -304,7 +306,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             // ---- once every MMA that read the old B is complete (the previous tile's accumulator is full), and
             // ---- tells the mma warp.
             if (seg != cached_seg) {
-                const float *lam = prm.lambda + (prm.n_lambda == 1 ? 0 : seg) * D;
+                const float *lam = CALIB ? nullptr : prm.lambda + (prm.n_lambda == 1 ? 0 : seg) * D;
                 const float lift = lift_of<D>(lam, lane);
                 if (j > 0 && cur.first_of_segment()) {
                     if (!wait_or_abort(smem_u32(&ctrl->acc_full[(j - 1) % kAccStages]), (uint32_t)((j - 1) / kAccStages) & 1u,
@@ -339,6 +341,15 @@ __global__ void __launch_bounds__(kThreads, 1)
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(smem_u32(&ctrl->acc_empty[sc]));
+                    }
+                    if constexpr (CALIB) {
+                        // column maxima over the warp's 32 rows (rows past the end were filled with zeros by the TMA load)
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            const uint32_t m = __reduce_max_sync(0xFFFFFFFFu, vb[i] & 0x7FFFFFFFu);   // |v| orders like its bits
+                            if (lane == i) colmax[gi] = fmaxf(colmax[gi], __uint_as_float(m));
+                        }
+                        continue;
                     }
                     // ---- scale: sigma = fp16(absmax / 7); codes are taken against the stored value
                     float amax = 0.0f;
@@ -375,6 +386,11 @@ __global__ void __launch_bounds__(kThreads, 1)
                 }
             }
         }
+        if constexpr (CALIB) {   // this warp's maxima of its 32 rows of every tile -> the global column maxima
+#pragma unroll
+            for (int gi = 0; gi < C::kGroupsPerPart; ++gi)
+                if (g0 + gi < g1) atomicMax(prm.amax_bits + (g0 + gi) * kGroup + lane, __float_as_uint(colmax[gi] * unlift));
+        }
     }
 
     tc_fence_before();
@@ -390,13 +406,13 @@ __global__ void __launch_bounds__(kThreads, 1)
 // ------------------------------------------------------------------------------------------------
 namespace {
 
-template <int D, bool BF16>
-cudaError_t launch(int64_t N, const FftParams &f, const float *e0, cudaStream_t stream)
+template <int D, bool BF16, bool CALIB = false>
+cudaError_t launch(int64_t N, const FftParams &f, const float *e0, cudaStream_t stream, uint32_t *amax_bits = nullptr)
 {
     using C = Cfg<D, BF16>;
     static int sms = 0;
     if (sms == 0) {
-        cudaError_t e = cudaFuncSetAttribute(kvq_encode_umma_kernel<D, BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(kvq_encode_umma_kernel<D, BF16, CALIB>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
         if (e != cudaSuccess) return e;
         int dev = 0;
         if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
@@ -416,6 +432,7 @@ cudaError_t launch(int64_t N, const FftParams &f, const float *e0, cudaStream_t 
     prm.out_mul = f.out_mul;
     prm.out_add = f.out_add;
     prm.status = f.status;
+    prm.amax_bits = amax_bits;
 
     CUtensorMap tm_x;
     const cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)N};
@@ -427,7 +444,7 @@ cudaError_t launch(int64_t N, const FftParams &f, const float *e0, cudaStream_t 
 
     const int64_t tiles = prm.n_seg * ((prm.rpl + kTile - 1) / kTile);
     const int grid = (int)(tiles < sms ? tiles : sms);
-    kvq_encode_umma_kernel<D, BF16><<<grid, kThreads, C::kSmemBytes, stream>>>(prm, tm_x);
+    kvq_encode_umma_kernel<D, BF16, CALIB><<<grid, kThreads, C::kSmemBytes, stream>>>(prm, tm_x);
     count_launch();
     return cudaGetLastError();
 }
@@ -445,6 +462,21 @@ cudaError_t umma_encode(int D, bool bf16, int64_t N, const FftParams &f, const f
         case 96: return bf16 ? launch<96, true>(N, f, e0, stream) : launch<96, false>(N, f, e0, stream);
         case 128: return bf16 ? launch<128, true>(N, f, e0, stream) : launch<128, false>(N, f, e0, stream);
         case 160: return bf16 ? cudaErrorInvalidValue : launch<160, false>(N, f, e0, stream);
+    }
+    return cudaErrorInvalidValue;
+}
+
+// Column maxima of |M (s (.) x)| over the N rows of x, accumulated into amax_bits [D] (fp32 bit patterns, zeroed by the
+// caller on the same stream): the forward GEMM with lambda = 1 and a reducing epilogue.
+cudaError_t umma_calibrate(int D, bool bf16, int64_t N, const FftParams &f, const float *e0, uint32_t *amax_bits, cudaStream_t stream)
+{
+    if (!tensor_map_encode_fn()) return cudaErrorNotSupported;
+    if (D == 256) return umma_calibrate_d256(bf16, N, f, e0, amax_bits, stream);
+    switch (D) {
+        case 64: return bf16 ? launch<64, true, true>(N, f, e0, stream, amax_bits) : launch<64, false, true>(N, f, e0, stream, amax_bits);
+        case 96: return bf16 ? launch<96, true, true>(N, f, e0, stream, amax_bits) : launch<96, false, true>(N, f, e0, stream, amax_bits);
+        case 128: return bf16 ? launch<128, true, true>(N, f, e0, stream, amax_bits) : launch<128, false, true>(N, f, e0, stream, amax_bits);
+        case 160: return bf16 ? cudaErrorInvalidValue : launch<160, false, true>(N, f, e0, stream, amax_bits);
     }
     return cudaErrorInvalidValue;
 }

@@ -69,11 +69,11 @@ static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
 template <int D>
 __device__ __forceinline__ float lift_of(const float *__restrict__ lam, int lane)
 {
-    float mx = 0.0f;
+    float mx = lam ? 0.0f : 1.0f;   // no lambda row (calibration): lambda = 1
 #pragma unroll
     for (int p = 0; p < (D / 4 + 31) / 32; ++p) {
         const int i = lane + 32 * p;
-        if (i < D / 4) {
+        if (lam && i < D / 4) {
             const float4 l = __ldg(reinterpret_cast<const float4 *>(lam) + i);
             mx = fmaxf(mx, fmaxf(fmaxf(fabsf(l.x), fabsf(l.y)), fmaxf(fabsf(l.z), fabsf(l.w))));
         }
@@ -97,7 +97,7 @@ __device__ __forceinline__ void build_b_rows(unsigned char *sB, const float *__r
 #pragma unroll 2
     for (int c = c0; c < c1; ++c) {
         const int cg = half * kHalfN + c;
-        const float f = __ldg(lam + cg) * lift;
+        const float f = lam ? __ldg(lam + cg) * lift : lift;
 #pragma unroll
         for (int p = 0; p < 2; ++p) {
             const int i = lane + 32 * p;
@@ -131,9 +131,10 @@ struct UmmaEncode256Params {
     int64_t n_seg;
     int64_t out_mul, out_add;   // output row of input row r is r * out_mul + out_add
     uint32_t *status;
+    uint32_t *amax_bits;        // calibration only: [D] running column maxima as fp32 bit patterns (start at zero)
 };
 
-template <bool BF16>
+template <bool BF16, bool CALIB>
 __global__ void __launch_bounds__(kThreads, 1)
     kvq_encode_umma_d256_kernel(const __grid_constant__ UmmaEncode256Params prm, const __grid_constant__ CUtensorMap tm_x)
 {
@@ -269,7 +270,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         float unlift = 1.0f;
         if (n_my > 0) {   // B for the CTA's first lambda row: D / 16 rows per warp, all sixteen warps
             TileCursor first(tile_begin, tps);
-            const float *lam = prm.lambda + (prm.n_lambda == 1 ? 0 : first.seg) * kD;
+            const float *lam = CALIB ? nullptr : prm.lambda + (prm.n_lambda == 1 ? 0 : first.seg) * kD;
             const float lift = lift_of<kD>(lam, lane);
             build_b_rows<BF16>(sB, prm.e0, lam, lift, half, (warp - 2) * 8, (warp - 1) * 8, lane);
             fence_proxy_async();   // B is read by the tensor core through the async proxy
@@ -278,6 +279,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             unlift = 1.0f / lift;
             cached_seg = first.seg;
         }
+        float colmax[2] = {};   // calibration: lane i keeps the running maximum of column i of each of this thread's groups
         TileCursor cur(tile_begin + set, tps);
         for (int j = set; j < n_my; j += 2, cur.advance(2)) {
             __syncwarp();
@@ -288,7 +290,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             // ---- once every MMA that read the old B is complete (the previous tile's accumulator is full), and
             // ---- tells the mma warp.
             if (seg != cached_seg) {
-                const float *lam = prm.lambda + (prm.n_lambda == 1 ? 0 : seg) * kD;
+                const float *lam = CALIB ? nullptr : prm.lambda + (prm.n_lambda == 1 ? 0 : seg) * kD;
                 const float lift = lift_of<kD>(lam, lane);
                 if (j > 0 && cur.first_of_segment()) {
                     if (!wait_or_abort(smem_u32(&ctrl->acc_full[(j - 1) % kAccStages]), (uint32_t)((j - 1) / kAccStages) & 1u,
@@ -323,6 +325,15 @@ __global__ void __launch_bounds__(kThreads, 1)
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(smem_u32(&ctrl->acc_empty[sc]));
+                    }
+                    if constexpr (CALIB) {
+                        // column maxima over the warp's 32 rows (rows past the end were filled with zeros by the TMA load)
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            const uint32_t m = __reduce_max_sync(0xFFFFFFFFu, vb[i] & 0x7FFFFFFFu);   // |v| orders like its bits
+                            if (lane == i) colmax[gi] = fmaxf(colmax[gi], __uint_as_float(m));
+                        }
+                        continue;
                     }
                     // ---- scale: sigma = fp16(absmax / 7); codes are taken against the stored value
                     float amax = 0.0f;
@@ -360,6 +371,11 @@ __global__ void __launch_bounds__(kThreads, 1)
                 }
             }
         }
+        if constexpr (CALIB) {   // this warp's maxima of its 32 rows of every tile -> the global column maxima
+#pragma unroll
+            for (int gi = 0; gi < 2; ++gi)
+                atomicMax(prm.amax_bits + (4 * half + g0 + gi) * kGroup + lane, __float_as_uint(colmax[gi] * unlift));
+        }
     }
 
     tc_fence_before();
@@ -375,13 +391,13 @@ __global__ void __launch_bounds__(kThreads, 1)
 // ------------------------------------------------------------------------------------------------
 namespace {
 
-template <bool BF16>
-cudaError_t launch(int64_t N, const FftParams &f, const float *e0, cudaStream_t stream)
+template <bool BF16, bool CALIB = false>
+cudaError_t launch(int64_t N, const FftParams &f, const float *e0, cudaStream_t stream, uint32_t *amax_bits = nullptr)
 {
     using C = Cfg<BF16>;
     static int sms = 0;
     if (sms == 0) {
-        cudaError_t e = cudaFuncSetAttribute(kvq_encode_umma_d256_kernel<BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(kvq_encode_umma_d256_kernel<BF16, CALIB>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
         if (e != cudaSuccess) return e;
         int dev = 0;
         if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
@@ -401,6 +417,7 @@ cudaError_t launch(int64_t N, const FftParams &f, const float *e0, cudaStream_t 
     prm.out_mul = f.out_mul;
     prm.out_add = f.out_add;
     prm.status = f.status;
+    prm.amax_bits = amax_bits;
 
     CUtensorMap tm_x;
     const cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)N};
@@ -412,7 +429,7 @@ cudaError_t launch(int64_t N, const FftParams &f, const float *e0, cudaStream_t 
 
     const int64_t tiles = prm.n_seg * ((prm.rpl + kTile - 1) / kTile);
     const int64_t pairs = tiles < sms / 2 ? tiles : sms / 2;
-    kvq_encode_umma_d256_kernel<BF16><<<(int)(2 * pairs), kThreads, C::kSmemBytes, stream>>>(prm, tm_x);
+    kvq_encode_umma_d256_kernel<BF16, CALIB><<<(int)(2 * pairs), kThreads, C::kSmemBytes, stream>>>(prm, tm_x);
     count_launch();
     return cudaGetLastError();
 }
@@ -423,6 +440,12 @@ cudaError_t umma_encode_d256(bool bf16, int64_t N, const FftParams &f, const flo
 {
     if (!tensor_map_encode_fn()) return cudaErrorNotSupported;
     return bf16 ? launch<true>(N, f, e0, stream) : launch<false>(N, f, e0, stream);
+}
+
+cudaError_t umma_calibrate_d256(bool bf16, int64_t N, const FftParams &f, const float *e0, uint32_t *amax_bits, cudaStream_t stream)
+{
+    if (!tensor_map_encode_fn()) return cudaErrorNotSupported;
+    return bf16 ? launch<true, true>(N, f, e0, stream, amax_bits) : launch<false, true>(N, f, e0, stream, amax_bits);
 }
 
 }  // namespace kvq

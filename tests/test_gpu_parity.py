@@ -190,6 +190,50 @@ def test_gemm_kernels_d256(dtype, N, n_lambda, rpl, kind):
         assert dec["rows_needing_tie_rule"] < 0.02
 
 
+# ---- static lambda calibration (Sec. 7.1): lambda_c = 1 / max over the calibration vectors of |SRFT(x)_c|
+
+@pytest.mark.parametrize("D,dtype", [(64, "f16"), (96, "f16"), (128, "f16"), (128, "bf16"), (160, "f16"), (256, "f16"), (256, "bf16")])
+@pytest.mark.parametrize("N", [1, 700, 40000])
+def test_calibrate_lambda_matches_the_oracle(D, dtype, N):
+    plan = kb.Plan(D, G, 50 + D)
+    sg = plan.signs()
+    x = wl.make_vectors(N, D, dtype, "k_outlier", 60 + D + N)
+    lam_o, amax_o = ko.calibrate_lambda(bits(x), DT[dtype], sg)
+    lam = torch.full((D,), -1.0, dtype=torch.float32, device="cuda")
+    kb.kvq_calibrate_lambda(plan.handle, x.cuda(), lam)
+    torch.cuda.synchronize()
+    assert kb.kvq_plan_device_status(plan.handle) == 0
+    got = lam.cpu().numpy().astype(np.float64)
+    assert np.all(np.isfinite(got)) and np.all(got > 0)
+    # fp32 accumulation of exact products against fp64.  The error of a coefficient is relative to the vector's norm (the
+    # transform is orthonormal), not to the coefficient, which may be a small remainder of cancelling terms.
+    xnorm = float(np.linalg.norm(x.double().numpy(), axis=1).max())
+    assert np.abs(1.0 / got - amax_o).max() <= 2e-6 * xnorm
+    if N >= 700:   # with many vectors every channel's maximum is of the order of the norms, and lambda itself agrees
+        assert np.abs(got / lam_o - 1.0).max() <= 1e-4
+    # used as lambda, every rescaled channel stays within [-1, 1]: no group scale exceeds fp16(1 / 7) by more than rounding
+    packed, scales = gpu_encode(plan, x.cuda(), lam)
+    assert float(scales.float().max()) <= (1.0 / 7.0) * (1.0 + 2e-3)
+    plan.close()
+
+
+def test_calibrate_lambda_edge_cases():
+    plan = kb.Plan(128, G, 3)
+    lam = torch.full((128,), -1.0, dtype=torch.float32, device="cuda")
+    kb.kvq_calibrate_lambda(plan.handle, torch.empty(0, 128, dtype=torch.float16, device="cuda"), lam)
+    torch.cuda.synchronize()
+    assert bool((lam == 1.0).all())                       # no vectors: lambda = 1
+    kb.kvq_calibrate_lambda(plan.handle, torch.zeros(300, 128, dtype=torch.float16, device="cuda"), lam)
+    torch.cuda.synchronize()
+    assert bool((lam == 1.0).all())                       # channels that carry nothing: lambda = 1
+    plan.close()
+    p160 = kb.Plan(160, G, 3)
+    with pytest.raises(kb.KvqError) as e:
+        kb.kvq_calibrate_lambda(p160.handle, torch.zeros(8, 160, dtype=torch.bfloat16, device="cuda"), torch.empty(160, device="cuda"))
+    assert e.value.status == kb.KVQ_ERR_UNSUPPORTED_DIM
+    p160.close()
+
+
 # ---- every head dim and dtype, ragged N (several tiles plus a tail), lambda rows that straddle tiles
 
 @pytest.mark.parametrize("dtype", ["f16", "bf16"])
