@@ -137,6 +137,22 @@ kvq_status_t kvq_append(kvq_plan_t *plan, const void *x_new /* [S, D] */, kvq_dt
                         void *cuda_stream);
 
 /*
+ * kvq_flush_block -- the residual-window flush with the dequantized-prefix cache (Sec. 7.2: new tokens wait in a short
+ * fp16 window; when it is full the block is quantized, and the already dequantized prefix is kept, so that a decode step
+ * costs O(new rows) instead of O(prefix)).  Quantizes `rows` new vectors of each of S streams into rows
+ * [pos0, pos0 + rows) of the int4 caches (exactly what `rows` kvq_append calls would store) and writes the dequantized
+ * values of those rows (exactly what kvq_decode of the caches would give there) into the same rows of dq_cache.
+ *   x_block       device, [S, rows, D] row-major, fp16 or bf16 per `dtype`; 16-byte aligned.
+ *   lambda, n_lambda, streams_per_lambda, packed_cache [S, T_max, D/2], scales_cache [S, T_max, D/group]: as in kvq_append.
+ *   dq_cache      device out, [S, T_max, D] of the same 16-bit type; 16-byte aligned.  Only rows [pos0, pos0 + rows) are written.
+ * Requires 0 <= pos0 and pos0 + rows <= T_max.  S == 0 or rows == 0 is a no-op.  Two launches on the stream.  The
+ * window itself (holding the not yet flushed tokens in fp16) is the caller's buffer: this call is its flush.
+ */
+kvq_status_t kvq_flush_block(kvq_plan_t *plan, const void *x_block, kvq_dtype_t dtype, int64_t S, int64_t rows,
+                             const float *lambda, int64_t n_lambda, int64_t streams_per_lambda, uint8_t *packed_cache,
+                             void *scales_cache, void *dq_cache, int64_t T_max, int64_t pos0, void *cuda_stream);
+
+/*
  * kvq_calibrate_lambda -- static calibration of the per-channel rescale (Sec. 7.1: lambda_d = 1 / per-channel
  * maximum of the SRFT output, taken in one pass over calibration vectors).
  *   x           device, [N, D] row-major, fp16 or bf16 per `dtype`; 16-byte aligned: the calibration vectors.

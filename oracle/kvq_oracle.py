@@ -280,3 +280,25 @@ def append(x_new_raw, dtype: int, sg, lam, group: int, packed_cache, scales_cach
                              _ptr(packed_cache), _ptr(scales_cache), T_max, pos)
     if rc:
         raise ValueError("kvqo_append: rc=%d" % rc)
+
+
+def flush_block(x_block_raw, dtype: int, sg, lam, group: int, packed_cache, scales_cache, dq_cache, pos0: int,
+                streams_per_lambda: int = 0):
+    """Residual-window flush with a dequantized-prefix cache (Sec. 7.2), written as its definition: the block's rows
+    are appended one token at a time, then the rows just stored are decoded into the same rows of ``dq_cache``
+    ([S, T_max, D] raw 16-bit).  Nothing else in the three caches is written."""
+    x = _raw16(x_block_raw)
+    S, rows, D = x.shape
+    if dq_cache.dtype != np.uint16 or not dq_cache.flags.c_contiguous:
+        raise TypeError("dq_cache must be contiguous uint16 bits")
+    T_max = packed_cache.shape[1]
+    if pos0 < 0 or pos0 + rows > T_max:
+        raise ValueError("block does not fit the cache")
+    lam2, nl = _lam(lam, D)
+    spl = streams_per_lambda if streams_per_lambda >= 1 else 1
+    for t in range(rows):
+        append(np.ascontiguousarray(x[:, t]), dtype, sg, lam, group, packed_cache, scales_cache, pos0 + t, streams_per_lambda)
+    for s in range(S):
+        row = lam2[s // spl if nl > 1 else 0]
+        dq_cache[s, pos0:pos0 + rows] = decode(packed_cache[s, pos0:pos0 + rows], scales_cache[s, pos0:pos0 + rows], sg, row,
+                                               group, dtype)

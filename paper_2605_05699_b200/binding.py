@@ -37,7 +37,7 @@ KVQ_IMPL_GEMM = 2
 # every symbol include/kvq.h declares
 EXPORTS = (
     "kvq_plan_create", "kvq_plan_destroy", "kvq_plan_get_signs", "kvq_plan_describe", "kvq_plan_set_impl",
-    "kvq_plan_device_status", "kvq_encode", "kvq_decode", "kvq_append", "kvq_decode_static", "kvq_calibrate_lambda", "kvq_status_string",
+    "kvq_plan_device_status", "kvq_encode", "kvq_decode", "kvq_append", "kvq_decode_static", "kvq_calibrate_lambda", "kvq_flush_block", "kvq_status_string",
     "kvq_launch_count",
 )
 
@@ -79,6 +79,8 @@ def lib() -> ctypes.CDLL:
         L.kvq_append.argtypes = [vp, vp, i32, i64, vp, i64, i64, vp, vp, i64, i64, vp]
         L.kvq_decode_static.restype = i32
         L.kvq_decode_static.argtypes = [vp, vp, vp, i64, vp, i64, i64, vp, i32, vp, vp]
+        L.kvq_flush_block.restype = i32
+        L.kvq_flush_block.argtypes = [vp, vp, i32, i64, i64, vp, i64, i64, vp, vp, vp, i64, i64, vp]
         L.kvq_calibrate_lambda.restype = i32
         L.kvq_calibrate_lambda.argtypes = [vp, vp, i32, i64, vp, vp]
         L.kvq_status_string.restype = ctypes.c_char_p
@@ -215,6 +217,18 @@ def kvq_decode_static(plan: int, packed: torch.Tensor, scales: torch.Tensor, lam
                                        n_lambda, rows_per_lambda, _dev(out, "out"), _dtype_code(out), sw,
                                        _stream(stream)),
                "kvq_decode_static")
+
+
+def kvq_flush_block(plan: int, x_block: torch.Tensor, lam: torch.Tensor, packed_cache: torch.Tensor, scales_cache: torch.Tensor,
+                    dq_cache: torch.Tensor, pos0: int, streams_per_lambda: int = 0, stream=None) -> None:
+    S, rows, D = x_block.shape
+    T_max = packed_cache.shape[-2]
+    n_lambda = lam.numel() // D
+    with torch.cuda.device(x_block.device):
+        _check(lib().kvq_flush_block(plan, _dev(x_block, "x_block"), _dtype_code(x_block), S, rows, _dev(lam, "lambda"), n_lambda,
+                                     streams_per_lambda, _dev(packed_cache, "packed_cache"), _dev(scales_cache, "scales_cache"),
+                                     _dev(dq_cache, "dq_cache"), T_max, pos0, _stream(stream)),
+               "kvq_flush_block")
 
 
 def kvq_calibrate_lambda(plan: int, x: torch.Tensor, lambda_out: torch.Tensor, stream=None) -> None:

@@ -161,8 +161,8 @@ static void fill_params(const kvq_plan *p, FftParams &prm, int64_t N, const floa
     prm.lambda = lambda;
     prm.n_lambda = n_lambda;
     prm.rows_per_lambda = rows_per_lambda < 1 ? 1 : rows_per_lambda;
-    prm.out_mul = 1;
-    prm.out_add = 0;
+    prm.out_map = RowMap{1, 1, 0};
+    prm.in_map = RowMap{1, 1, 0};
     prm.status = p->d_status;
     std::memcpy(prm.sign_xor, p->sign_xor, sizeof(prm.sign_xor));
 }
@@ -259,7 +259,7 @@ kvq_status_t kvq_plan_device_status(kvq_plan_t *plan, uint32_t *word)
 
 static kvq_status_t encode_common(kvq_plan_t *plan, const void *x, kvq_dtype_t dtype, int64_t N, const float *lambda,
                                   int64_t n_lambda, int64_t rows_per_lambda, uint8_t *packed, void *scales,
-                                  int64_t out_mul, int64_t out_add, void *cuda_stream)
+                                  const RowMap &out_map, void *cuda_stream)
 {
     if (!plan || N < 0) return KVQ_ERR_INVALID_ARG;
     if (dtype != KVQ_F16 && dtype != KVQ_BF16) return KVQ_ERR_INVALID_ARG;
@@ -276,8 +276,7 @@ static kvq_status_t encode_common(kvq_plan_t *plan, const void *x, kvq_dtype_t d
     prm.in = x;
     prm.packed = packed;
     prm.scales = scales;
-    prm.out_mul = out_mul;
-    prm.out_add = out_add;
+    prm.out_map = out_map;
     // the tensor-core kernel pays a fixed set-up per launch (B operand build); small calls stay on the register FFT
     const bool use_gemm = gemm_ok && (plan->enc_impl == KVQ_IMPL_GEMM || (plan->enc_impl == KVQ_IMPL_AUTO && N >= kGemmEncodeMinRows));
     cudaError_t e = use_gemm ? umma_encode(plan->D, dtype == KVQ_BF16, N, prm, plan->d_e0, static_cast<cudaStream_t>(cuda_stream))
@@ -292,7 +291,7 @@ static kvq_status_t encode_common(kvq_plan_t *plan, const void *x, kvq_dtype_t d
 kvq_status_t kvq_encode(kvq_plan_t *plan, const void *x, kvq_dtype_t dtype, int64_t N, const float *lambda,
                         int64_t n_lambda, int64_t rows_per_lambda, uint8_t *packed, void *scales, void *cuda_stream)
 {
-    return encode_common(plan, x, dtype, N, lambda, n_lambda, rows_per_lambda, packed, scales, 1, 0, cuda_stream);
+    return encode_common(plan, x, dtype, N, lambda, n_lambda, rows_per_lambda, packed, scales, RowMap{1, 1, 0}, cuda_stream);
 }
 
 kvq_status_t kvq_append(kvq_plan_t *plan, const void *x_new, kvq_dtype_t dtype, int64_t S, const float *lambda,
@@ -301,7 +300,7 @@ kvq_status_t kvq_append(kvq_plan_t *plan, const void *x_new, kvq_dtype_t dtype, 
 {
     if (T_max < 1 || pos < 0 || pos >= T_max) return KVQ_ERR_INVALID_ARG;
     return encode_common(plan, x_new, dtype, S, lambda, n_lambda, streams_per_lambda, packed_cache, scales_cache,
-                         T_max, pos, cuda_stream);
+                         RowMap{1, T_max, pos}, cuda_stream);
 }
 
 kvq_status_t kvq_decode(kvq_plan_t *plan, const uint8_t *packed, const void *scales, int64_t N, const float *lambda,
@@ -341,6 +340,38 @@ kvq_status_t kvq_decode(kvq_plan_t *plan, const uint8_t *packed, const void *sca
     prm.out = out;
     cudaError_t e = fft_decode(plan->D, dtype == KVQ_BF16, N, prm, static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        return KVQ_ERR_CUDA;
+    }
+    return KVQ_OK;
+}
+
+kvq_status_t kvq_flush_block(kvq_plan_t *plan, const void *x_block, kvq_dtype_t dtype, int64_t S, int64_t rows, const float *lambda,
+                             int64_t n_lambda, int64_t streams_per_lambda, uint8_t *packed_cache, void *scales_cache, void *dq_cache,
+                             int64_t T_max, int64_t pos0, void *cuda_stream)
+{
+    if (!plan || S < 0 || rows < 0) return KVQ_ERR_INVALID_ARG;
+    if (T_max < 1 || pos0 < 0 || rows > T_max || pos0 > T_max - rows) return KVQ_ERR_INVALID_ARG;
+    if (dtype != KVQ_F16 && dtype != KVQ_BF16) return KVQ_ERR_INVALID_ARG;
+    if (S == 0 || rows == 0) return KVQ_OK;
+    if (!dq_cache) return KVQ_ERR_INVALID_ARG;
+    if (misaligned16(dq_cache)) return KVQ_ERR_ALIGNMENT;
+    if (S > INT64_MAX / rows) return KVQ_ERR_INVALID_ARG;
+    const int64_t N = S * rows;
+    // lambda row of block row r: stream (r / rows) / streams_per_lambda
+    const int64_t rpl = (streams_per_lambda < 1 ? 1 : streams_per_lambda) * rows;
+    const RowMap map{rows, T_max, pos0};
+    kvq_status_t st = encode_common(plan, x_block, dtype, N, lambda, n_lambda, rpl, packed_cache, scales_cache, map, cuda_stream);
+    if (st != KVQ_OK) return st;
+    // the same rows back out of the int4 cache into the dequantized-prefix cache: what a later full-prefix decode would give
+    FftParams prm;
+    fill_params(plan, prm, N, lambda, n_lambda, rpl);
+    prm.packed = packed_cache;
+    prm.scales = scales_cache;
+    prm.out = dq_cache;
+    prm.in_map = map;
+    prm.out_map = map;
+    if (fft_decode(plan->D, dtype == KVQ_BF16, N, prm, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
         (void)cudaGetLastError();
         return KVQ_ERR_CUDA;
     }

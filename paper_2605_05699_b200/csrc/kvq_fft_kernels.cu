@@ -372,7 +372,7 @@ __global__ void __launch_bounds__(WARPS * 32) kvq_encode_fft_kernel(const __grid
                 __syncwarp();
             }
             if (active && lr == cur) {
-                const int64_t orow = r * prm.out_mul + prm.out_add;
+                const int64_t orow = prm.out_map(r);
                 encode_row<D, GRP, P, BF16>(
                     reinterpret_cast<const uint4 *>(in_base + (stage * 32 + lane) * S::IN_STRIDE), prm.sign_xor,
                     reinterpret_cast<const float4 *>(lam_cache), reinterpret_cast<uint4 *>(out_row), stash,
@@ -421,7 +421,7 @@ __global__ void __launch_bounds__(WARPS * 32) kvq_decode_fft_kernel(const __grid
         const uint32_t bar = stage ? bar1 : bar0;
         if (r < N) {
             mbar_arrive_expect_tx(bar, D / 2);
-            bulk_load(smem_u32(in_base + (stage * 32 + lane) * S::IN_STRIDE), packed + r * (D / 2), D / 2, bar);
+            bulk_load(smem_u32(in_base + (stage * 32 + lane) * S::IN_STRIDE), packed + prm.in_map(r) * (D / 2), D / 2, bar);
         } else {
             mbar_arrive(bar);
         }
@@ -432,7 +432,7 @@ __global__ void __launch_bounds__(WARPS * 32) kvq_decode_fft_kernel(const __grid
 #pragma unroll
         for (int j = 0; j < (G + 1) / 2; ++j) sb[j] = 0;
         if (r < N) {
-            const uint16_t *sp = scales + r * G;
+            const uint16_t *sp = scales + prm.in_map(r) * G;
             if constexpr ((G * 2) % 16 == 0) {
 #pragma unroll
                 for (int j = 0; j < G / 8; ++j) {
@@ -504,7 +504,7 @@ __global__ void __launch_bounds__(WARPS * 32) kvq_decode_fft_kernel(const __grid
                     reinterpret_cast<const uint4 *>(in_base + (stage * 32 + lane) * S::IN_STRIDE), sig, prm.sign_xor,
                     reinterpret_cast<const float4 *>(lam_cache), reinterpret_cast<uint4 *>(out_row), stash, lane);
                 fence_proxy_async();
-                bulk_store(static_cast<unsigned char *>(prm.out) + r * (2 * D), smem_u32(out_row), 2 * D);
+                bulk_store(static_cast<unsigned char *>(prm.out) + prm.out_map(r) * (2 * D), smem_u32(out_row), 2 * D);
                 bulk_commit();
             }
             todo &= ~mine;

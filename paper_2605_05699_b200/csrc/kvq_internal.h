@@ -10,6 +10,17 @@
 
 namespace kvq {
 
+// Where row r of a contiguous block of rows lives in a cache laid out [stream][T][...]: every `rps` consecutive rows of
+// the block belong to one stream and go to rows base .. base + rps - 1 of it; `stride` = rows per stream of the cache.
+// The identity is {1, 1, 0}; kvq_append is {1, T_max, pos}.
+struct RowMap {
+    int64_t rps, stride, base;
+    __host__ __device__ __forceinline__ int64_t operator()(int64_t r) const
+    {
+        return rps == 1 ? r * stride + base : (r / rps) * stride + base + (r % rps);
+    }
+};
+
 // Arguments of the register-FFT kernels.  Passed by value as a __grid_constant__
 // parameter, so the sign words are read straight from the constant bank.
 struct FftParams {
@@ -20,7 +31,8 @@ struct FftParams {
     void *out;             // decode: x^ [N, D] half precision
     int64_t N;
     int64_t n_lambda, rows_per_lambda;
-    int64_t out_mul, out_add;   // encode: output row of input row r is r * out_mul + out_add
+    RowMap out_map;             // row of packed / scales (encode) or of out (decode) that row r goes to
+    RowMap in_map;              // decode: row of packed / scales that row r comes from
     uint32_t *status;           // per-plan device status word
     uint32_t sign_xor[128];     // word m: bit 15 set if s_{2m} = -1, bit 31 set if s_{2m+1} = -1
 };

@@ -148,7 +148,7 @@ struct UmmaEncodeParams {
     int64_t n_lambda;
     int64_t rpl;           // rows per lambda segment (N when there is one lambda row)
     int64_t n_seg;
-    int64_t out_mul, out_add;   // output row of input row r is r * out_mul + out_add
+    RowMap out_map;        // output row of input row r
     uint32_t *status;
     uint32_t *amax_bits;        // calibration only: [D] running column maxima as fp32 bit patterns (start at zero)
 };
@@ -329,7 +329,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             int64_t seg_rows = N - seg * rpl;
             if (seg_rows > rpl) seg_rows = rpl;
             const bool live = off + r < seg_rows;
-            const int64_t orow = (seg * rpl + off + r) * prm.out_mul + prm.out_add;
+            const int64_t orow = prm.out_map(seg * rpl + off + r);
 #pragma unroll
             for (int gi = 0; gi < C::kGroupsPerPart; ++gi) {
                 const int g = g0 + gi;       // warp-uniform
@@ -429,8 +429,7 @@ cudaError_t launch(int64_t N, const FftParams &f, const float *e0, cudaStream_t 
     prm.n_lambda = f.n_lambda;
     prm.rpl = f.n_lambda == 1 ? N : f.rows_per_lambda;
     prm.n_seg = (N + prm.rpl - 1) / prm.rpl;
-    prm.out_mul = f.out_mul;
-    prm.out_add = f.out_add;
+    prm.out_map = f.out_map;
     prm.status = f.status;
     prm.amax_bits = amax_bits;
 

@@ -339,6 +339,66 @@ def test_append_touches_only_row_pos():
     plan.close()
 
 
+@pytest.mark.parametrize("D,dtype,S,T_max,spl,blocks", [
+    (128, "f16", 112, 300, 2, (256, 1, 16, 27)),       # a prefill block, then window flushes of 1, 16 and a ragged 27
+    (128, "f16", 3, 9000, 1, (8192, 64)),              # blocks long enough for the tensor-core encode
+    (256, "bf16", 26, 80, 1, (33, 32, 15)),
+    (96, "f16", 7, 40, 7, (5, 35)),
+])
+def test_flush_block_fills_the_int4_and_the_dequantized_caches(D, dtype, S, T_max, spl, blocks):
+    odt = ko.F16 if dtype == "f16" else ko.BF16
+    tdt = torch.float16 if dtype == "f16" else torch.bfloat16
+    plan = kb.Plan(D, G, 31)
+    sg = plan.signs()
+    n_lambda = (S + spl - 1) // spl
+    lam = wl.make_lambda(n_lambda, D, 61)
+    x_all = wl.make_vectors(S * T_max, D, dtype, "k_outlier", 62).view(S, T_max, D)
+    packed = torch.full((S, T_max, D // 2), 0xAB, dtype=torch.uint8, device="cuda")
+    scales = torch.full((S, T_max, D // G), 1.25, dtype=torch.float16, device="cuda")
+    dq = torch.full((S, T_max, D), 3.0, dtype=tdt, device="cuda")
+    lamd = lam.cuda()
+    pos = 0
+    for rows in blocks:
+        kb.kvq_flush_block(plan.handle, x_all[:, pos:pos + rows].contiguous().cuda(), lamd, packed, scales, dq, pos, spl)
+        pos += rows
+    torch.cuda.synchronize()
+    assert kb.kvq_plan_device_status(plan.handle) == 0
+    # rows past the flushed prefix are untouched
+    assert bool((packed[:, pos:] == 0xAB).all()) and bool((scales[:, pos:] == 1.25).all()) and bool((dq[:, pos:] == 3.0).all())
+    # the int4 cache equals one encode of the whole prefix (oracle), the dequantized cache its full-prefix decode
+    xp = x_all[:, :pos].reshape(-1, D)
+    ora = ko.encode(bits(xp), odt, sg, lam.numpy(), G, spl * pos, want_v=True)
+    pk = packed[:, :pos].reshape(-1, D // 2).cpu().numpy()
+    sb = bits(scales[:, :pos].reshape(-1, D // G))
+    parity.check_encode(pk, sb, ora, G, "flush int4 cache")
+    ob, o64 = ko.decode(pk, sb, sg, lam.numpy(), G, odt, spl * pos, want_f64=True)
+    parity.check_decode(bits(dq[:, :pos].reshape(-1, D)), ob, o64, odt, "flush dequantized cache")
+    # and the product's own full-prefix decode of the int4 cache gives the same rows (the incremental path's claim)
+    full = gpu_decode(plan, packed[:, :pos].reshape(-1, D // 2).contiguous(), scales[:, :pos].reshape(-1, D // G).contiguous(),
+                      lamd, dtype, spl * pos)
+    parity.check_decode(bits(full), ob, o64, odt, "full-prefix decode of the flushed cache")
+    plan.close()
+
+
+def test_flush_block_rejects_blocks_outside_the_cache():
+    D, S, T = 128, 4, 16
+    plan = kb.Plan(D, G, 1)
+    x = wl.make_vectors(S * 8, D, "f16", "gaussian", 1).view(S, 8, D).cuda()
+    lam = wl.make_lambda(1, D, 2).cuda()
+    packed = torch.zeros(S, T, D // 2, dtype=torch.uint8, device="cuda")
+    scales = torch.zeros(S, T, D // G, dtype=torch.float16, device="cuda")
+    dq = torch.zeros(S, T, D, dtype=torch.float16, device="cuda")
+    with pytest.raises(kb.KvqError):
+        kb.kvq_flush_block(plan.handle, x, lam, packed, scales, dq, 9, 0)
+    with pytest.raises(kb.KvqError):
+        kb.kvq_flush_block(plan.handle, x, lam, packed, scales, dq, -1, 0)
+    kb.kvq_flush_block(plan.handle, x, lam, packed, scales, dq, 8, 0)     # the last block that fits
+    kb.kvq_flush_block(plan.handle, x[:, :0], lam, packed, scales, dq, 16, 0)   # an empty block is a no-op
+    torch.cuda.synchronize()
+    assert kb.kvq_plan_device_status(plan.handle) == 0
+    plan.close()
+
+
 # ---- config 3: Gemma-3-1B-shaped, D = 256 bf16, prefix sweep ---------------------------------
 
 @pytest.mark.parametrize("prefix", [256, 1024])

@@ -428,6 +428,37 @@ def test_append_writes_row_pos_of_every_stream_and_nothing_else():
     assert (pc[:, mask] == 0xAB).all() and (sc[:, mask] == 0x1234).all()
 
 
+def test_flushing_blocks_that_cover_the_prefix_equals_the_full_prefix_decode():
+    # Sec. 7.2: the incremental path (flush a block, keep its dequantized rows) must leave exactly what encoding the
+    # whole prefix at once and decoding all of it would give, whatever the block boundaries are
+    D, g, S, T = 64, 32, 5, 23
+    r = rng(41)
+    s = ko.signs(D, 8)
+    lam = r.uniform(0.5, 2, (3, D)).astype(np.float32)
+    x16 = (r.standard_normal((S, T, D)) * 3).astype(np.float16)
+    pc = np.full((S, T, D // 2), 0xCD, dtype=np.uint8)
+    sc = np.full((S, T, D // g), 0x4321, dtype=np.uint16)
+    dq = np.full((S, T, D), 0x7777, dtype=np.uint16)
+    pos = 0
+    for rows in (1, 7, 2, 8):                      # 18 of the 23 rows, ragged blocks
+        ko.flush_block(x16[:, pos:pos + rows], ko.F16, s, lam, g, pc, sc, dq, pos, streams_per_lambda=2)
+        pos += rows
+    assert (pc[:, pos:] == 0xCD).all() and (sc[:, pos:] == 0x4321).all() and (dq[:, pos:] == 0x7777).all()
+    whole = ko.encode(x16[:, :pos].reshape(-1, D), ko.F16, s, lam, g, rows_per_lambda=2 * pos)
+    assert np.array_equal(pc[:, :pos].reshape(-1, D // 2), whole["packed"])
+    assert np.array_equal(sc[:, :pos].reshape(-1, D // g), whole["scales"])
+    full = ko.decode(whole["packed"], whole["scales"], s, lam, g, ko.F16, rows_per_lambda=2 * pos)
+    assert np.array_equal(dq[:, :pos].reshape(-1, D), full)
+    # a second flush over rows already written replaces them and only them
+    before = dq.copy()
+    ko.flush_block(x16[:, 20:22], ko.F16, s, lam, g, pc, sc, dq, 3, streams_per_lambda=2)
+    changed = np.zeros(T, bool)
+    changed[3:5] = True
+    assert np.array_equal(dq[:, ~changed], before[:, ~changed]) and not np.array_equal(dq[:, changed], before[:, changed])
+    with pytest.raises(ValueError):
+        ko.flush_block(x16[:, :4], ko.F16, s, lam, g, pc, sc, dq, T - 3, streams_per_lambda=2)
+
+
 # --------------------------------------------------------------------------
 # numbers the paper prints about the layout
 # --------------------------------------------------------------------------
