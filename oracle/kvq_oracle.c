@@ -28,6 +28,10 @@
  * algorithm.  Vectors are independent; an OpenMP loop over vectors is the only
  * parallelism.
  *
+ *   base variants (Sec. 3.2 steps 3-4; Sec. 4.1 "Quantization"): the same path with b = 8 (scale = absmax / 127,
+ *     codes in [-127, 127], one two's-complement byte per value) and / or one scale per vector (g = D, "per-token").
+ *     The *_b entry points take the bit width b in {4, 8}; the entry points without it are b = 4.
+ *
  * Readings where the paper is silent (each is listed in the design notes):
  *   - DFT sign convention e^{-2 pi i k n / D}; the imaginary part is packed as
  *     the transform returns it (the usual "rfft" convention).
@@ -315,6 +319,19 @@ void kvqo_unpack_nibbles(const uint8_t *bytes, int64_t n, int8_t *q)
 /* quantizer                                                           */
 /* ------------------------------------------------------------------ */
 
+/* codes of one vector to / from their stored bytes: nibble pairs for b = 4, one two's-complement byte per value for b = 8 */
+static void store_codes(const int8_t *q, int D, int bits, uint8_t *dst)
+{
+    if (bits == 4) kvqo_pack_nibbles(q, D, dst);
+    else memcpy(dst, q, (size_t)D);
+}
+
+static void load_codes(const uint8_t *src, int D, int bits, int8_t *q)
+{
+    if (bits == 4) kvqo_unpack_nibbles(src, D, q);
+    else memcpy(q, src, (size_t)D);
+}
+
 static int64_t lambda_row(int64_t r, int64_t n_lambda, int64_t rows_per_lambda)
 {
     return n_lambda == 1 ? 0 : r / rows_per_lambda;
@@ -330,22 +347,23 @@ static int check_common(int D, int g, int64_t N, int64_t n_lambda, int64_t rows_
 }
 
 /* steps 4-7 for one vector whose packed transform z is given */
-static void quantize_one(int D, int g, const double *z, const float *lam, int8_t *q, uint16_t *scales,
+static void quantize_one(int D, int g, int bits, const double *z, const float *lam, int8_t *q, uint16_t *scales,
                          double *v_out)
 {
+    const double qmax = (double)((1 << (bits - 1)) - 1);   /* 2^{b-1} - 1: 7 or 127 */
     double v[D];
     for (int c = 0; c < D; ++c) v[c] = (double)lam[c] * z[c];
     for (int j = 0; j < D / g; ++j) {
         double a = 0.0;
         for (int c = j * g; c < (j + 1) * g; ++c)
             if (fabs(v[c]) > a) a = fabs(v[c]);
-        uint16_t sb = kvqo_f64_to_f16_sat(a / 7.0);
+        uint16_t sb = kvqo_f64_to_f16_sat(a / qmax);
         double sigma = kvqo_f16_to_f64(sb);
         scales[j] = sb;
         for (int c = j * g; c < (j + 1) * g; ++c) {
             double t = sigma > 0.0 ? rint(v[c] / sigma) : 0.0;   /* rint: half to even */
-            if (t > 7.0) t = 7.0;
-            if (t < -7.0) t = -7.0;
+            if (t > qmax) t = qmax;
+            if (t < -qmax) t = -qmax;
             q[c] = (int8_t)t;
         }
     }
@@ -354,11 +372,12 @@ static void quantize_one(int D, int g, const double *z, const float *lam, int8_t
 
 /* Forward path on fp64 input rows.  codes (nullable) receives the unpacked
  * int4 codes [N,D]; v_out (nullable) the rescaled transform lambda (.) z. */
-int kvqo_encode_f64(int D, int g, const int8_t *sg, const double *x, int64_t N, const float *lam,
-                    int64_t n_lambda, int64_t rows_per_lambda, uint8_t *packed, uint16_t *scales,
-                    int8_t *codes, double *v_out)
+int kvqo_encode_f64_b(int D, int g, int bits, const int8_t *sg, const double *x, int64_t N, const float *lam,
+                      int64_t n_lambda, int64_t rows_per_lambda, uint8_t *packed, uint16_t *scales,
+                      int8_t *codes, double *v_out)
 {
-    if (check_common(D, g, N, n_lambda, rows_per_lambda)) return 1;
+    if (check_common(D, g, N, n_lambda, rows_per_lambda) || (bits != 4 && bits != 8)) return 1;
+    const int row_bytes = D * bits / 8;
     trig_t t;
     if (trig_init(&t, D)) return 2;
     const int G = D / g;
@@ -367,21 +386,29 @@ int kvqo_encode_f64(int D, int g, const int8_t *sg, const double *x, int64_t N, 
         double z[D];
         int8_t q[D];
         srft_forward_one(&t, sg, x + r * D, z);
-        quantize_one(D, g, z, lam + lambda_row(r, n_lambda, rows_per_lambda) * D, q, scales + r * G,
+        quantize_one(D, g, bits, z, lam + lambda_row(r, n_lambda, rows_per_lambda) * D, q, scales + r * G,
                      v_out ? v_out + r * D : NULL);
-        kvqo_pack_nibbles(q, D, packed + r * (D / 2));
+        store_codes(q, D, bits, packed + r * row_bytes);
         if (codes) memcpy(codes + r * D, q, (size_t)D);
     }
     trig_free(&t);
     return 0;
 }
 
-/* Forward path on fp16 / bf16 rows: widen exactly, then as above. */
-int kvqo_encode(int D, int g, const int8_t *sg, const uint16_t *x, int dtype, int64_t N,
-                const float *lam, int64_t n_lambda, int64_t rows_per_lambda, uint8_t *packed,
-                uint16_t *scales, int8_t *codes, double *v_out)
+int kvqo_encode_f64(int D, int g, const int8_t *sg, const double *x, int64_t N, const float *lam,
+                    int64_t n_lambda, int64_t rows_per_lambda, uint8_t *packed, uint16_t *scales,
+                    int8_t *codes, double *v_out)
 {
-    if (check_common(D, g, N, n_lambda, rows_per_lambda)) return 1;
+    return kvqo_encode_f64_b(D, g, 4, sg, x, N, lam, n_lambda, rows_per_lambda, packed, scales, codes, v_out);
+}
+
+/* Forward path on fp16 / bf16 rows: widen exactly, then as above. */
+int kvqo_encode_b(int D, int g, int bits, const int8_t *sg, const uint16_t *x, int dtype, int64_t N,
+                  const float *lam, int64_t n_lambda, int64_t rows_per_lambda, uint8_t *packed,
+                  uint16_t *scales, int8_t *codes, double *v_out)
+{
+    if (check_common(D, g, N, n_lambda, rows_per_lambda) || (bits != 4 && bits != 8)) return 1;
+    const int row_bytes = D * bits / 8;
     trig_t t;
     if (trig_init(&t, D)) return 2;
     const int G = D / g;
@@ -391,22 +418,30 @@ int kvqo_encode(int D, int g, const int8_t *sg, const uint16_t *x, int dtype, in
         int8_t q[D];
         for (int n = 0; n < D; ++n) xr[n] = widen(x[r * D + n], dtype);
         srft_forward_one(&t, sg, xr, z);
-        quantize_one(D, g, z, lam + lambda_row(r, n_lambda, rows_per_lambda) * D, q, scales + r * G,
+        quantize_one(D, g, bits, z, lam + lambda_row(r, n_lambda, rows_per_lambda) * D, q, scales + r * G,
                      v_out ? v_out + r * D : NULL);
-        kvqo_pack_nibbles(q, D, packed + r * (D / 2));
+        store_codes(q, D, bits, packed + r * row_bytes);
         if (codes) memcpy(codes + r * D, q, (size_t)D);
     }
     trig_free(&t);
     return 0;
 }
 
+int kvqo_encode(int D, int g, const int8_t *sg, const uint16_t *x, int dtype, int64_t N,
+                const float *lam, int64_t n_lambda, int64_t rows_per_lambda, uint8_t *packed,
+                uint16_t *scales, int8_t *codes, double *v_out)
+{
+    return kvqo_encode_b(D, g, 4, sg, x, dtype, N, lam, n_lambda, rows_per_lambda, packed, scales, codes, v_out);
+}
+
 /* Inverse path.  out (nullable) gets x^ rounded to dtype; out_f64 (nullable) the
  * unrounded fp64 reconstruction. */
-int kvqo_decode(int D, int g, const int8_t *sg, const uint8_t *packed, const uint16_t *scales,
-                int64_t N, const float *lam, int64_t n_lambda, int64_t rows_per_lambda, uint16_t *out,
-                int dtype, double *out_f64)
+int kvqo_decode_b(int D, int g, int bits, const int8_t *sg, const uint8_t *packed, const uint16_t *scales,
+                  int64_t N, const float *lam, int64_t n_lambda, int64_t rows_per_lambda, uint16_t *out,
+                  int dtype, double *out_f64)
 {
-    if (check_common(D, g, N, n_lambda, rows_per_lambda)) return 1;
+    if (check_common(D, g, N, n_lambda, rows_per_lambda) || (bits != 4 && bits != 8)) return 1;
+    const int row_bytes = D * bits / 8;
     trig_t t;
     if (trig_init(&t, D)) return 2;
     const int G = D / g;
@@ -415,7 +450,7 @@ int kvqo_decode(int D, int g, const int8_t *sg, const uint8_t *packed, const uin
         int8_t q[D];
         double z[D], xr[D];
         const float *l = lam + lambda_row(r, n_lambda, rows_per_lambda) * D;
-        kvqo_unpack_nibbles(packed + r * (D / 2), D, q);
+        load_codes(packed + r * row_bytes, D, bits, q);
         for (int c = 0; c < D; ++c) {
             double sigma = kvqo_f16_to_f64(scales[r * G + c / g]);
             double lc = (double)l[c] > 1e-6 ? (double)l[c] : 1e-6;    /* clamp at 1e-6 */
@@ -429,6 +464,13 @@ int kvqo_decode(int D, int g, const int8_t *sg, const uint8_t *packed, const uin
     }
     trig_free(&t);
     return 0;
+}
+
+int kvqo_decode(int D, int g, const int8_t *sg, const uint8_t *packed, const uint16_t *scales,
+                int64_t N, const float *lam, int64_t n_lambda, int64_t rows_per_lambda, uint16_t *out,
+                int dtype, double *out_f64)
+{
+    return kvqo_decode_b(D, g, 4, sg, packed, scales, N, lam, n_lambda, rows_per_lambda, out, dtype, out_f64);
 }
 
 /* Decode-step append: quantize S new vectors (one per stream) and write them to

@@ -71,6 +71,12 @@ def _load():
         lib.kvqo_encode.argtypes = [i32, i32, p, p, i32, i64, p, i64, i64, p, p, p, p]
         lib.kvqo_decode.restype = i32
         lib.kvqo_decode.argtypes = [i32, i32, p, p, p, i64, p, i64, i64, p, i32, p]
+        lib.kvqo_encode_f64_b.restype = i32
+        lib.kvqo_encode_f64_b.argtypes = [i32, i32, i32, p, p, i64, p, i64, i64, p, p, p, p]
+        lib.kvqo_encode_b.restype = i32
+        lib.kvqo_encode_b.argtypes = [i32, i32, i32, p, p, i32, i64, p, i64, i64, p, p, p, p]
+        lib.kvqo_decode_b.restype = i32
+        lib.kvqo_decode_b.argtypes = [i32, i32, i32, p, p, p, i64, p, i64, i64, p, i32, p]
         lib.kvqo_append.restype = i32
         lib.kvqo_append.argtypes = [i32, i32, p, p, i32, i64, p, i64, i64, p, p, i64, i64]
         lib.kvqo_num_threads.restype = i32
@@ -204,19 +210,20 @@ def unpack_nibbles(b) -> np.ndarray:
 
 # ---- quantizer ------------------------------------------------------------
 
-def encode_f64(x, sg, lam, group: int, rows_per_lambda: int = 0, want_v: bool = False):
-    """Forward path on fp64 rows.  Returns dict(packed, scales, codes[, v])."""
+def encode_f64(x, sg, lam, group: int, rows_per_lambda: int = 0, want_v: bool = False, bits: int = 4):
+    """Forward path on fp64 rows.  Returns dict(packed, scales, codes[, v]).  ``packed`` is [N, D/2] nibble pairs for
+    bits = 4 and [N, D] two's-complement bytes for bits = 8."""
     x = np.ascontiguousarray(x, dtype=np.float64)
     D = x.shape[-1]
     N = x.size // D
     sg = np.ascontiguousarray(sg, dtype=np.int8)
     lam, nl = _lam(lam, D)
-    packed = np.empty((N, D // 2), dtype=np.uint8)
+    packed = np.empty((N, D * bits // 8), dtype=np.uint8)
     scales = np.empty((N, D // group), dtype=np.uint16)
     codes = np.empty((N, D), dtype=np.int8)
     v = np.empty((N, D), dtype=np.float64) if want_v else None
-    rc = _load().kvqo_encode_f64(D, group, _ptr(sg), _ptr(x), N, _ptr(lam), nl, rows_per_lambda,
-                                 _ptr(packed), _ptr(scales), _ptr(codes), _ptr(v))
+    rc = _load().kvqo_encode_f64_b(D, group, bits, _ptr(sg), _ptr(x), N, _ptr(lam), nl, rows_per_lambda,
+                                   _ptr(packed), _ptr(scales), _ptr(codes), _ptr(v))
     if rc:
         raise ValueError("kvqo_encode_f64: rc=%d" % rc)
     out = {"packed": packed, "scales": scales, "codes": codes}
@@ -225,19 +232,19 @@ def encode_f64(x, sg, lam, group: int, rows_per_lambda: int = 0, want_v: bool = 
     return out
 
 
-def encode(x_raw, dtype: int, sg, lam, group: int, rows_per_lambda: int = 0, want_v: bool = False):
+def encode(x_raw, dtype: int, sg, lam, group: int, rows_per_lambda: int = 0, want_v: bool = False, bits: int = 4):
     """Forward path on fp16 / bf16 rows given as raw bits.  Returns dict(packed, scales, codes[, v])."""
     x = _raw16(x_raw)
     D = x.shape[-1]
     N = x.size // D
     sg = np.ascontiguousarray(sg, dtype=np.int8)
     lam, nl = _lam(lam, D)
-    packed = np.empty((N, D // 2), dtype=np.uint8)
+    packed = np.empty((N, D * bits // 8), dtype=np.uint8)
     scales = np.empty((N, D // group), dtype=np.uint16)
     codes = np.empty((N, D), dtype=np.int8)
     v = np.empty((N, D), dtype=np.float64) if want_v else None
-    rc = _load().kvqo_encode(D, group, _ptr(sg), _ptr(x), dtype, N, _ptr(lam), nl, rows_per_lambda,
-                             _ptr(packed), _ptr(scales), _ptr(codes), _ptr(v))
+    rc = _load().kvqo_encode_b(D, group, bits, _ptr(sg), _ptr(x), dtype, N, _ptr(lam), nl, rows_per_lambda,
+                               _ptr(packed), _ptr(scales), _ptr(codes), _ptr(v))
     if rc:
         raise ValueError("kvqo_encode: rc=%d" % rc)
     out = {"packed": packed, "scales": scales, "codes": codes}
@@ -246,18 +253,19 @@ def encode(x_raw, dtype: int, sg, lam, group: int, rows_per_lambda: int = 0, wan
     return out
 
 
-def decode(packed, scales, sg, lam, group: int, dtype: int, rows_per_lambda: int = 0, want_f64: bool = False):
+def decode(packed, scales, sg, lam, group: int, dtype: int, rows_per_lambda: int = 0, want_f64: bool = False,
+           bits: int = 4):
     """Inverse path.  Returns raw bits of the rounded output, or (bits, fp64) if want_f64."""
-    packed = np.ascontiguousarray(packed, dtype=np.uint8)
-    D = packed.shape[-1] * 2
-    N = packed.size // (D // 2)
+    packed = np.ascontiguousarray(packed).view(np.uint8)
+    D = packed.shape[-1] * 8 // bits
+    N = packed.size // packed.shape[-1]
     scales = _raw16(scales)
     sg = np.ascontiguousarray(sg, dtype=np.int8)
     lam, nl = _lam(lam, D)
     out = np.empty((N, D), dtype=np.uint16)
     o64 = np.empty((N, D), dtype=np.float64) if want_f64 else None
-    rc = _load().kvqo_decode(D, group, _ptr(sg), _ptr(packed), _ptr(scales), N, _ptr(lam), nl,
-                             rows_per_lambda, _ptr(out), dtype, _ptr(o64))
+    rc = _load().kvqo_decode_b(D, group, bits, _ptr(sg), _ptr(packed), _ptr(scales), N, _ptr(lam), nl,
+                               rows_per_lambda, _ptr(out), dtype, _ptr(o64))
     if rc:
         raise ValueError("kvqo_decode: rc=%d" % rc)
     return (out, o64) if want_f64 else out

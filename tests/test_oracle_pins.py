@@ -428,6 +428,87 @@ def test_append_writes_row_pos_of_every_stream_and_nothing_else():
     assert (pc[:, mask] == 0xAB).all() and (sc[:, mask] == 0x1234).all()
 
 
+# --------------------------------------------------------------------------
+# base variants: one scale per vector (g = D) and 8-bit codes (Sec. 3.2 steps 3-4, Sec. 4.1)
+# --------------------------------------------------------------------------
+
+@pytest.mark.parametrize("bits", [4, 8])
+def test_two_spike_spectrum_tells_the_group_span_and_the_code_range(bits):
+    # z = a e_5 + (a / 10) e_40: the spikes sit in different groups of 32.  With one scale per group both codes are
+    # +-Q; with one scale per vector the small spike is rint(Q / 10): 1 for Q = 7, 13 for Q = 127.
+    D, Q = 128, (1 << (bits - 1)) - 1
+    s = ko.signs(D, 3)
+    a = 3.0
+    z = np.zeros((1, D))
+    z[0, 5], z[0, 40] = a, -a / 10
+    x = ko.srft_inverse(z, s)
+    lam = np.ones(D, np.float32)
+    e32 = ko.encode_f64(x, s, lam, 32, bits=bits)
+    eD = ko.encode_f64(x, s, lam, D, bits=bits)
+    assert e32["scales"].shape == (1, 4) and eD["scales"].shape == (1, 1)
+    want32 = np.zeros(D, np.int8)
+    want32[5], want32[40] = Q, -Q
+    wantD = want32.copy()
+    wantD[40] = -int(np.rint(Q / 10))
+    assert np.array_equal(e32["codes"][0], want32) and np.array_equal(eD["codes"][0], wantD)
+    assert eD["scales"][0, 0] == np.float16(a / Q).view(np.uint16)
+    assert np.array_equal(e32["scales"][0], np.array([a / Q, a / 10 / Q, 0, 0], np.float16).view(np.uint16))
+    # bytes: nibble pairs for 4 bits, the codes themselves for 8
+    if bits == 8:
+        assert eD["packed"].shape == (1, D) and np.array_equal(eD["packed"].view(np.int8), eD["codes"])
+    else:
+        assert eD["packed"].shape == (1, D // 2) and np.array_equal(ko.unpack_nibbles(eD["packed"]), eD["codes"])
+    # decode: the spikes come back as code x stored scale
+    _, xr = ko.decode(eD["packed"], eD["scales"], s, lam, D, ko.F16, want_f64=True, bits=bits)
+    sig = float(np.float16(a / Q))
+    zr = ko.srft_forward(xr, s)[0]
+    want = np.zeros(D)
+    want[5], want[40] = Q * sig, wantD[40] * sig
+    assert np.allclose(zr, want, atol=1e-12)
+
+
+@pytest.mark.parametrize("bits,g", [(4, 128), (8, 128), (8, 32)])
+def test_uniform_quantizer_properties_of_the_base_variants(bits, g):
+    D, N, Q = 128, 400, (1 << (bits - 1)) - 1
+    r = rng(50 + bits + g)
+    s = ko.signs(D, 9)
+    lam = r.uniform(0.5, 2, D).astype(np.float32)
+    x = r.standard_normal((N, D))
+    e = ko.encode_f64(x, s, lam, g, want_v=True, bits=bits)
+    v, q = e["v"], e["codes"].astype(np.float64)
+    sig = ko.f16_to_f64(e["scales"]).repeat(g, axis=1)
+    amax = np.abs(v).reshape(N, D // g, g).max(axis=2).repeat(g, axis=1)
+    # the stored scale is absmax / Q up to its fp16 rounding; the largest coordinate of a group gets code +-Q
+    assert np.all(np.abs(sig * Q - amax) <= amax * 2.0 ** -11)
+    assert np.all(np.abs(q).reshape(N, D // g, g).max(axis=2) == Q) and np.abs(q).max() == Q
+    # rounding to the nearest code: half a step, plus the clamp where fp16 rounded the scale down
+    assert np.all(np.abs(v - q * sig) <= sig / 2 + np.maximum(amax - Q * sig, 0) + 1e-15)
+    if bits == 8:   # fine steps: the error is uniform on a step, variance step^2 / 12 (textbook)
+        ratio = ((v - q * sig) ** 2).mean() / (sig ** 2 / 12).mean()
+        assert 0.9 < ratio < 1.1
+    # the inverse undoes lambda and the transform exactly: what is lost is the rounding alone
+    _, xr = ko.decode(e["packed"], e["scales"], s, lam, g, ko.F16, want_f64=True, bits=bits)
+    zr = ko.srft_forward(xr, s) * lam
+    assert np.allclose(zr, q * sig, atol=1e-9)
+
+
+def test_a_group_of_the_whole_vector_equals_groups_of_32_that_share_their_maximum():
+    # special case that reduces to the pinned g = 32 path: when every group of 32 has the same abs-max, one scale per
+    # vector and one per group are the same quantizer
+    D = 128
+    r = rng(77)
+    s = ko.signs(D, 2)
+    z = r.uniform(-1, 1, (50, D))
+    z[:, [3, 35, 70, 127]] = 1.5
+    x = ko.srft_inverse(z, s)
+    lam = np.ones(D, np.float32)
+    for bits in (4, 8):
+        a = ko.encode_f64(x, s, lam, 32, bits=bits)
+        b = ko.encode_f64(x, s, lam, D, bits=bits)
+        assert np.array_equal(a["codes"], b["codes"]) and np.array_equal(a["packed"], b["packed"])
+        assert np.array_equal(a["scales"], b["scales"].repeat(4, axis=1))
+
+
 def test_flushing_blocks_that_cover_the_prefix_equals_the_full_prefix_decode():
     # Sec. 7.2: the incremental path (flush a block, keep its dequantized rows) must leave exactly what encoding the
     # whole prefix at once and decoding all of it would give, whatever the block boundaries are
