@@ -251,6 +251,7 @@ def run_ours(args):
         return
 
     d256 = measure_d256(kb, wl, dev)
+    incr = measure_incremental(kb, wl, dev, dec_avg_ms=sum(dec_ms) / len(dec_ms))
     step_bytes = (2 * N + S) * BYTES_PER_VEC
     value = world * args.steps * step_bytes / (ms_total * 1e-3) / 1e9
     peak, peak_src = measured_peak()
@@ -285,6 +286,7 @@ def run_ours(args):
             "model_sweep_decode_ms_80_layers": 80 * dec_avg,
             "paper_context": "paper: 24.6 ns/vec encode at D=128, ~50 ns/vec at D=256 on an Apple M1 GPU (fp32 in, Sec. 7.1)",
             "d256_bf16_gemma_shaped": d256,
+            "incremental_decode": incr,
         },
         "roofline": roofline,
         "cpu_baseline": cpu,
@@ -334,10 +336,41 @@ def measure_d256(kb, wl, dev, iters=10):
             "note": "working set 140 MB per launch, about the size of L2: not a roofline number"}
 
 
+def measure_incremental(kb, wl, dev, dec_avg_ms, iters=20, window=16):
+    """Outside the timed region: the window flush of Sec. 7.2 on the bench's cache shape (64 streams x 32,768 tokens,
+    D=128 fp16): 16 new tokens per stream go into the int4 cache and the dequantized-prefix cache in one kvq_flush_block
+    call, against re-decoding the whole prefix (the timed step's decode) once per generated token."""
+    import torch
+
+    shp, S, T = workload_shape()
+    plan = kb.Plan(D, GROUP, 44)
+    lam = wl.make_lambda(2, D, 45, device=dev)
+    packed = torch.zeros(S, T, D // 2, dtype=torch.uint8, device=dev)
+    scales = torch.zeros(S, T, D // GROUP, dtype=torch.float16, device=dev)
+    dq = torch.zeros(S, T, D, dtype=torch.float16, device=dev)
+    blocks = [wl.make_vectors(S * window, D, shp.dtype, "gaussian", 46 + i, device=dev).view(S, window, D) for i in range(4)]
+    ms = []
+    for i in range(iters + 3):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        pos0 = (i * 4099 * window) % (T - window)
+        e0.record()
+        kb.kvq_flush_block(plan.handle, blocks[i % 4], lam, packed, scales, dq, pos0, S // 2)
+        e1.record()
+        torch.cuda.synchronize()
+        if i >= 3:
+            ms.append(e0.elapsed_time(e1))
+    assert kb.kvq_plan_device_status(plan.handle) == 0
+    plan.close()
+    flush_us = 1e3 * statistics.median(ms)
+    return {"window_tokens": window, "streams": S, "flush_us": flush_us, "flush_us_per_generated_token": flush_us / window,
+            "full_prefix_decode_us_per_generated_token": 1e3 * dec_avg_ms,
+            "note": "one layer; the flush is two launches of %d vectors (launch-bound), independent of the prefix length" % (S * window)}
+
+
 # DRAM bytes per full launch (2,097,152 vectors, the bench's launch size) from ncu: dram__bytes_read.sum +
 # dram__bytes_write.sum, one-pass capture; see profiles/dram_traffic_d128_n2097152.md.  Reads match the algorithmic
 # bytes; writes are short of them by what is still in the 126 MB L2 when the kernel ends.
-TRAFFIC = {"decode": 151436288 + 478505472, "encode": 537912832 + 128682752}
+TRAFFIC = {"decode": 151400960 + 478458624, "encode": 537686272 + 128796672}
 
 
 # --------------------------------------------------------------------------------------------

@@ -67,13 +67,25 @@ typedef enum {
  * random sign vector drawn at initialization") and fixes the radix plan of the length-D/2
  * complex FFT (Sec. 3.2 step 2; mixed radix 3 / 5 for D = 96 / 160).
  *   D      head dimension; supported: 64, 96, 128, 160, 256.
- *   group  coordinates per scale; supported: 32 (must divide D).
+ *   group  coordinates per scale; supported: 32, or D (one scale per vector).
  *   seed   sign n is -1 when the top bit of the n-th SplitMix64 output for this seed is set.
  *   out    host pointer receiving the plan.
  * Touches no GPU: device tables are created on the first compute call, on the device that is
  * current then.  Errors: INVALID_ARG (null out), UNSUPPORTED_DIM, NOMEM.
  */
 kvq_status_t kvq_plan_create(int D, int group, uint64_t seed, kvq_plan_t **out);
+
+/*
+ * kvq_plan_create_ex -- kvq_plan_create with the quantizer's base variants (Sec. 3.2 steps 3-4; Sec. 4.1 "Quantization":
+ * uniform symmetric codes with one scale per head-dim vector):
+ *   group  32, or D for one scale per vector ("per-token"): scales are then [N, 1] fp16.
+ *   bits   4 (codes in [-7, 7], two per byte as in kvq_encode) or 8 (scale = absmax / 127, codes in [-127, 127], one
+ *          two's-complement byte per value: `packed` rows are D bytes).
+ * Everything else is as for kvq_plan_create, which is (group, bits = 4).  Wherever a comment of this header says
+ * "[*, D/2] bytes" a plan with bits = 8 takes [*, D] bytes.  The tensor-core kernels serve group = 32, bits = 4 only:
+ * other plans run on the register-FFT kernels (KVQ_IMPL_GEMM is refused with UNSUPPORTED_DIM, kvq_decode_static too).
+ */
+kvq_status_t kvq_plan_create_ex(int D, int group, int bits, uint64_t seed, kvq_plan_t **out);
 
 /* Frees the plan and its device tables.  NULL is a no-op.  The caller must make sure no call
  * using the plan is still running on the GPU. */

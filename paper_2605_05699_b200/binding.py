@@ -36,7 +36,7 @@ KVQ_IMPL_GEMM = 2
 
 # every symbol include/kvq.h declares
 EXPORTS = (
-    "kvq_plan_create", "kvq_plan_destroy", "kvq_plan_get_signs", "kvq_plan_describe", "kvq_plan_set_impl",
+    "kvq_plan_create", "kvq_plan_create_ex", "kvq_plan_destroy", "kvq_plan_get_signs", "kvq_plan_describe", "kvq_plan_set_impl",
     "kvq_plan_device_status", "kvq_encode", "kvq_decode", "kvq_append", "kvq_decode_static", "kvq_calibrate_lambda", "kvq_flush_block", "kvq_status_string",
     "kvq_launch_count",
 )
@@ -61,6 +61,8 @@ def lib() -> ctypes.CDLL:
         i32, i64, u64, vp = ctypes.c_int, ctypes.c_int64, ctypes.c_uint64, ctypes.c_void_p
         L.kvq_plan_create.restype = i32
         L.kvq_plan_create.argtypes = [i32, i32, u64, ctypes.POINTER(vp)]
+        L.kvq_plan_create_ex.restype = i32
+        L.kvq_plan_create_ex.argtypes = [i32, i32, i32, u64, ctypes.POINTER(vp)]
         L.kvq_plan_destroy.restype = i32
         L.kvq_plan_destroy.argtypes = [vp]
         L.kvq_plan_get_signs.restype = i32
@@ -131,6 +133,12 @@ def _stream(stream) -> int:
 def kvq_plan_create(D: int, group: int, seed: int) -> int:
     h = ctypes.c_void_p()
     _check(lib().kvq_plan_create(D, group, ctypes.c_uint64(seed & (2**64 - 1)), ctypes.byref(h)), "kvq_plan_create")
+    return h.value
+
+
+def kvq_plan_create_ex(D: int, group: int, bits: int, seed: int) -> int:
+    h = ctypes.c_void_p()
+    _check(lib().kvq_plan_create_ex(D, group, bits, ctypes.c_uint64(seed & (2**64 - 1)), ctypes.byref(h)), "kvq_plan_create_ex")
     return h.value
 
 
@@ -240,11 +248,12 @@ def kvq_calibrate_lambda(plan: int, x: torch.Tensor, lambda_out: torch.Tensor, s
 
 
 class Plan:
-    """Owns a ``kvq_plan_t`` handle: ``Plan(D, group, seed).handle`` goes to the kvq_* calls."""
+    """Owns a ``kvq_plan_t`` handle: ``Plan(D, group, seed).handle`` goes to the kvq_* calls.  ``bits=8`` or
+    ``group=D`` select the base variants (kvq_plan_create_ex)."""
 
-    def __init__(self, D: int, group: int = 32, seed: int = 0):
-        self.D, self.group, self.seed = D, group, seed
-        self.handle = kvq_plan_create(D, group, seed)
+    def __init__(self, D: int, group: int = 32, seed: int = 0, bits: int = 4):
+        self.D, self.group, self.seed, self.bits = D, group, seed, bits
+        self.handle = kvq_plan_create(D, group, seed) if bits == 4 and group == 32 else kvq_plan_create_ex(D, group, bits, seed)
 
     def signs(self):
         return kvq_plan_get_signs(self.handle, self.D)
@@ -262,7 +271,7 @@ class Plan:
 
     # allocation helpers for callers that do not bring their own buffers
     def empty_packed(self, N: int, device="cuda") -> torch.Tensor:
-        return torch.empty(N, self.D // 2, dtype=torch.uint8, device=device)
+        return torch.empty(N, self.D * self.bits // 8, dtype=torch.uint8, device=device)
 
     def empty_scales(self, N: int, device="cuda") -> torch.Tensor:
         return torch.empty(N, self.D // self.group, dtype=torch.float16, device=device)

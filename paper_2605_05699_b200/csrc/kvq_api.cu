@@ -171,13 +171,19 @@ extern "C" {
 
 kvq_status_t kvq_plan_create(int D, int group, uint64_t seed, kvq_plan_t **out)
 {
+    return kvq_plan_create_ex(D, group, 4, seed, out);
+}
+
+kvq_status_t kvq_plan_create_ex(int D, int group, int bits, uint64_t seed, kvq_plan_t **out)
+{
     if (!out) return KVQ_ERR_INVALID_ARG;
     *out = nullptr;
-    if (!dim_supported(D) || group != 32 || D % group) return KVQ_ERR_UNSUPPORTED_DIM;
+    if (!dim_supported(D) || (group != 32 && group != D) || (bits != 4 && bits != 8)) return KVQ_ERR_UNSUPPORTED_DIM;
     kvq_plan *p = new (std::nothrow) kvq_plan();
     if (!p) return KVQ_ERR_NOMEM;
     p->D = D;
     p->group = group;
+    p->bits = bits;
     p->seed = seed;
     p->enc_impl = p->dec_impl = KVQ_IMPL_AUTO;
     p->device = -1;
@@ -257,6 +263,9 @@ kvq_status_t kvq_plan_device_status(kvq_plan_t *plan, uint32_t *word)
     return *word ? KVQ_ERR_TIMEOUT : KVQ_OK;
 }
 
+// the tensor-core kernels exist for the fused layout only: groups of 32, 4-bit codes
+static bool gemm_layout(const kvq_plan *p) { return p->group == 32 && p->bits == 4; }
+
 static kvq_status_t encode_common(kvq_plan_t *plan, const void *x, kvq_dtype_t dtype, int64_t N, const float *lambda,
                                   int64_t n_lambda, int64_t rows_per_lambda, uint8_t *packed, void *scales,
                                   const RowMap &out_map, void *cuda_stream)
@@ -268,7 +277,7 @@ static kvq_status_t encode_common(kvq_plan_t *plan, const void *x, kvq_dtype_t d
     kvq_status_t st = check_lambda(N, lambda, n_lambda, rows_per_lambda);
     if (st != KVQ_OK) return st;
     if (misaligned16(x) || misaligned16(packed) || misaligned16(scales)) return KVQ_ERR_ALIGNMENT;
-    const bool gemm_ok = umma_encode_supported(plan->D, dtype == KVQ_BF16);
+    const bool gemm_ok = gemm_layout(plan) && umma_encode_supported(plan->D, dtype == KVQ_BF16);
     if (plan->enc_impl == KVQ_IMPL_GEMM && !gemm_ok) return KVQ_ERR_UNSUPPORTED_DIM;
     if ((st = ensure_device(plan)) != KVQ_OK) return st;
     FftParams prm;
@@ -280,7 +289,7 @@ static kvq_status_t encode_common(kvq_plan_t *plan, const void *x, kvq_dtype_t d
     // the tensor-core kernel pays a fixed set-up per launch (B operand build); small calls stay on the register FFT
     const bool use_gemm = gemm_ok && (plan->enc_impl == KVQ_IMPL_GEMM || (plan->enc_impl == KVQ_IMPL_AUTO && N >= kGemmEncodeMinRows));
     cudaError_t e = use_gemm ? umma_encode(plan->D, dtype == KVQ_BF16, N, prm, plan->d_e0, static_cast<cudaStream_t>(cuda_stream))
-                             : fft_encode(plan->D, dtype == KVQ_BF16, N, prm, static_cast<cudaStream_t>(cuda_stream));
+                             : fft_encode(plan->D, plan->group, plan->bits, dtype == KVQ_BF16, N, prm, static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
         return KVQ_ERR_CUDA;
@@ -313,7 +322,7 @@ kvq_status_t kvq_decode(kvq_plan_t *plan, const uint8_t *packed, const void *sca
     kvq_status_t st = check_lambda(N, lambda, n_lambda, rows_per_lambda);
     if (st != KVQ_OK) return st;
     if (misaligned16(packed) || misaligned16(scales) || misaligned16(out)) return KVQ_ERR_ALIGNMENT;
-    const bool gemm_ok = umma_decode_supported(plan->D, dtype == KVQ_BF16);
+    const bool gemm_ok = gemm_layout(plan) && umma_decode_supported(plan->D, dtype == KVQ_BF16);
     if (plan->dec_impl == KVQ_IMPL_GEMM && !gemm_ok) return KVQ_ERR_UNSUPPORTED_DIM;
     if ((st = ensure_device(plan)) != KVQ_OK) return st;
     if (gemm_ok && plan->dec_impl != KVQ_IMPL_FFT) {
@@ -338,7 +347,7 @@ kvq_status_t kvq_decode(kvq_plan_t *plan, const uint8_t *packed, const void *sca
     prm.packed = const_cast<uint8_t *>(packed);
     prm.scales = const_cast<void *>(scales);
     prm.out = out;
-    cudaError_t e = fft_decode(plan->D, dtype == KVQ_BF16, N, prm, static_cast<cudaStream_t>(cuda_stream));
+    cudaError_t e = fft_decode(plan->D, plan->group, plan->bits, dtype == KVQ_BF16, N, prm, static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
         return KVQ_ERR_CUDA;
@@ -371,7 +380,7 @@ kvq_status_t kvq_flush_block(kvq_plan_t *plan, const void *x_block, kvq_dtype_t 
     prm.out = dq_cache;
     prm.in_map = map;
     prm.out_map = map;
-    if (fft_decode(plan->D, dtype == KVQ_BF16, N, prm, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
+    if (fft_decode(plan->D, plan->group, plan->bits, dtype == KVQ_BF16, N, prm, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
         (void)cudaGetLastError();
         return KVQ_ERR_CUDA;
     }

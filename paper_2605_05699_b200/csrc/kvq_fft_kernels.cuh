@@ -1,5 +1,7 @@
 // fp32 register-FFT kernels of libkvq: kvq_encode / kvq_append / kvq_decode for every
-// supported head dimension and both half-precision types.
+// supported head dimension, both half-precision types, groups of 32 or of the whole vector,
+// and 4- or 8-bit codes.  Kernel templates; each (group, bits) variant is instantiated in a
+// translation unit of its own (kvq_fft_*.cu) through KVQ_FFT_DEFINE_VARIANT.
 //
 // Mapping.  One thread owns one vector for its whole life: the length-D/2 complex
 // FFT, the Hermitian glue, the lambda rescale, the per-group abs-max, the rounding
@@ -21,6 +23,7 @@
 // the mirrored decimation in time on the inverse).  The first pass parks D/2
 // floats in a per-warp shared-memory stash while the second runs, which halves
 // the live registers of a thread.
+#pragma once
 #include "kvq_fft.cuh"
 #include "kvq_internal.h"
 
@@ -29,14 +32,16 @@ namespace kvq {
 constexpr float kMagicRound = 12582912.0f + 8.0f;   // 1.5 * 2^23 + 8: (v + magic) has q + 8 in its low bits
 constexpr uint32_t kMagicBits = 0x4B400000u;
 constexpr uint32_t kMagicSum = kMagicBits * 0x11111111u;   // sum_i kMagicBits * 16^i  (mod 2^32)
+constexpr float kMagicRound8 = 12582912.0f + 128.0f;       // 8-bit codes: q + 128 in the low byte
+constexpr uint32_t kMagicSum8 = kMagicBits * 0x01010101u;  // sum_i kMagicBits * 256^i (mod 2^32)
 
 // ------------------------------------------------------------------------------------------
 // shared-memory geometry (per warp)
 // ------------------------------------------------------------------------------------------
-template <int D, int P>
+template <int D, int P, int BITS>
 struct EncSmem {
     static constexpr int IN_STRIDE = 2 * D + 16;
-    static constexpr int OUT_STRIDE = D / 2 + 16;
+    static constexpr int OUT_STRIDE = D * BITS / 8 + 16;
     static constexpr int IN_BYTES = 2 * 32 * IN_STRIDE;
     static constexpr int OUT_BYTES = 32 * OUT_STRIDE;
     static constexpr int STASH_BYTES = (P == 2) ? D * 64 : 0;
@@ -44,9 +49,9 @@ struct EncSmem {
     static constexpr int WARP_BYTES = IN_BYTES + OUT_BYTES + STASH_BYTES + LAM_BYTES;
 };
 
-template <int D, int P>
+template <int D, int P, int BITS>
 struct DecSmem {
-    static constexpr int IN_STRIDE = D / 2 + 16;
+    static constexpr int IN_STRIDE = D * BITS / 8 + 16;
     static constexpr int OUT_STRIDE = 2 * D + 16;
     static constexpr int IN_BYTES = 2 * 32 * IN_STRIDE;
     static constexpr int OUT_BYTES = 32 * OUT_STRIDE;
@@ -61,16 +66,18 @@ constexpr int kBarBytes = 128;   // room for 2 mbarriers per warp, up to 8 warps
 // forward path of one row (Sec. 3.2 steps 1-4, fused lambda and group scales of Sec. 7.1)
 //   row      this lane's D half-precision inputs in shared memory
 //   lam      lambda row in shared memory (warp-shared)
-//   out      this lane's D/2 output bytes in shared memory
+//   out      this lane's D BITS / 8 output bytes in shared memory
 //   stash    warp stash, float4 [D/8][32] (P == 2 only)
 //   scl      this row's D/GRP fp16 scales in global memory
+// BITS = 8 (Sec. 3.2 step 4): codes in [-127, 127], one two's-complement byte per value.
 // ------------------------------------------------------------------------------------------
-template <int D, int GRP, int P, bool BF16>
+template <int D, int GRP, int BITS, int P, bool BF16>
 __device__ __forceinline__ void encode_row(const uint4 *__restrict__ row, const uint32_t *__restrict__ sign_xor,
                                            const float4 *__restrict__ lam, uint4 *__restrict__ out,
                                            float4 *__restrict__ stash, uint16_t *__restrict__ scl, int lane)
 {
     constexpr int H = D / 2, L = H / P, G = D / GRP, SLOTS = D / P;
+    constexpr float Q = (float)((1 << (BITS - 1)) - 1);   // largest code: 7 or 127
     float amax[G];
 #pragma unroll
     for (int j = 0; j < G; ++j) amax[j] = 0.0f;
@@ -135,18 +142,18 @@ __device__ __forceinline__ void encode_row(const uint4 *__restrict__ row, const 
         }
     });
 
-    // ---- scales: sigma = fp16(absmax / 7); codes are taken against the stored value
+    // ---- scales: sigma = fp16(absmax / Q); codes are taken against the stored value
     float rs[G];
     bool clamp[G];
     uint32_t sbits[G];
 #pragma unroll
     for (int j = 0; j < G; ++j) {
-        float sig = fminf(__fdiv_rn(amax[j], 7.0f), 65504.0f);
+        float sig = fminf(__fdiv_rn(amax[j], Q), 65504.0f);
         __half hs = __float2half_rn(sig);
         sbits[j] = (uint32_t)__half_as_ushort(hs);
         float sg = __half2float(hs);
         rs[j] = sg > 0.0f ? __frcp_rn(sg) : 0.0f;
-        clamp[j] = !(amax[j] * rs[j] < 7.25f);   // saturated or subnormal scale: codes could leave [-7, 7]
+        clamp[j] = !(amax[j] * rs[j] < Q + 0.25f);   // saturated or subnormal scale: codes could leave [-Q, Q]
     }
     // ---- scales out (coalesced across the warp: consecutive rows are consecutive in memory)
     if constexpr ((G * 2) % 16 == 0) {
@@ -172,12 +179,12 @@ __device__ __forceinline__ void encode_row(const uint4 *__restrict__ row, const 
         for (int j = 0; j < G; ++j) scl[j] = (uint16_t)sbits[j];
     }
 
-    // ---- round, bias to unsigned nibbles, pack 8 codes per word, 4 words per 16-byte store
+    // ---- round, bias to unsigned codes, pack: 32 codes per step are one 16-byte store of nibbles or two of bytes
     static_for<D / 32>([&](auto ii) {
         constexpr int I = decltype(ii)::value;
-        uint32_t words[4];
+        uint32_t words[BITS];
         static_for<4>([&](auto ww) {
-            constexpr int wi = 4 * I + decltype(ww)::value;   // word index: codes 8 wi .. 8 wi + 7
+            constexpr int wi = 4 * I + decltype(ww)::value;   // octet index: codes 8 wi .. 8 wi + 7
             constexpr int j = (8 * wi) / GRP;
             float t[8];
             if constexpr (P == 1) {
@@ -188,41 +195,63 @@ __device__ __forceinline__ void encode_row(const uint4 *__restrict__ row, const 
                 t[0] = s4.x, t[2] = s4.y, t[4] = s4.z, t[6] = s4.w;
                 t[1] = v[4 * wi], t[3] = v[4 * wi + 1], t[5] = v[4 * wi + 2], t[7] = v[4 * wi + 3];
             }
-            uint32_t acc = 0;
-            if (!clamp[j]) {
+            if constexpr (BITS == 4) {
+                uint32_t acc = 0;
+                if (!clamp[j]) {
 #pragma unroll
-                for (int e = 0; e < 8; ++e) acc += __float_as_uint(fmaf(t[e], rs[j], kMagicRound)) << (4 * e);
+                    for (int e = 0; e < 8; ++e) acc += __float_as_uint(fmaf(t[e], rs[j], kMagicRound)) << (4 * e);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e)
+                        acc += __float_as_uint(fminf(fmaxf(t[e] * rs[j], -Q), Q) + kMagicRound) << (4 * e);
+                }
+                words[decltype(ww)::value] = (acc - kMagicSum) ^ 0x88888888u;
             } else {
+                uint32_t acc[2] = {0u, 0u};
+                if (!clamp[j]) {
 #pragma unroll
-                for (int e = 0; e < 8; ++e)
-                    acc += __float_as_uint(fminf(fmaxf(t[e] * rs[j], -7.0f), 7.0f) + kMagicRound) << (4 * e);
+                    for (int e = 0; e < 8; ++e) acc[e >> 2] += __float_as_uint(fmaf(t[e], rs[j], kMagicRound8)) << (8 * (e & 3));
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e)
+                        acc[e >> 2] += __float_as_uint(fminf(fmaxf(t[e] * rs[j], -Q), Q) + kMagicRound8) << (8 * (e & 3));
+                }
+                words[2 * decltype(ww)::value] = (acc[0] - kMagicSum8) ^ 0x80808080u;
+                words[2 * decltype(ww)::value + 1] = (acc[1] - kMagicSum8) ^ 0x80808080u;
             }
-            words[decltype(ww)::value] = (acc - kMagicSum) ^ 0x88888888u;
         });
-        out[I] = make_uint4(words[0], words[1], words[2], words[3]);
+        if constexpr (BITS == 4) {
+            out[I] = make_uint4(words[0], words[1], words[2], words[3]);
+        } else {
+            out[2 * I] = make_uint4(words[0], words[1], words[2], words[3]);
+            out[2 * I + 1] = make_uint4(words[4], words[5], words[6], words[7]);
+        }
     });
 }
 
 // ------------------------------------------------------------------------------------------
 // inverse path of one row (Sec. 3.1: "unpack, irfft, apply s"; 1 / max(lambda, 1e-6) of Sec. 5.1)
-//   row      this lane's D/2 packed bytes in shared memory
+//   row      this lane's D BITS / 8 code bytes in shared memory
 //   sig      this row's D/GRP scales, already widened
 //   rl       1 / max(lambda, 1e-6) in shared memory (warp-shared)
 //   out      this lane's D half-precision outputs in shared memory
 //   stash    warp stash, float4 [D/8][32] (P == 2 only)
 // ------------------------------------------------------------------------------------------
-template <int D, int GRP, int P, bool BF16>
+template <int D, int GRP, int BITS, int P, bool BF16>
 __device__ __forceinline__ void decode_row(const uint4 *__restrict__ row, const float *__restrict__ sig,
                                            const uint32_t *__restrict__ sign_xor, const float4 *__restrict__ rl,
                                            uint4 *__restrict__ out, float4 *__restrict__ stash, int lane)
 {
     constexpr int H = D / 2, L = H / P, SLOTS = D / P;
-    uint32_t pk[D / 8];
-    static_for<D / 32>([&](auto ii) {
+    constexpr int CPW = 32 / BITS;                                       // codes per 32-bit word
+    constexpr uint32_t kBias = BITS == 4 ? 0x88888888u : 0x80808080u;    // two's complement -> q + 8 / q + 128
+    constexpr float kUnbias = BITS == 4 ? 8388616.0f : 8388736.0f;       // 2^23 + 8 / 2^23 + 128
+    uint32_t pk[D / CPW];
+    static_for<D / CPW / 4>([&](auto ii) {
         constexpr int I = decltype(ii)::value;
         uint4 a = row[I];
-        pk[4 * I] = a.x ^ 0x88888888u, pk[4 * I + 1] = a.y ^ 0x88888888u;
-        pk[4 * I + 2] = a.z ^ 0x88888888u, pk[4 * I + 3] = a.w ^ 0x88888888u;
+        pk[4 * I] = a.x ^ kBias, pk[4 * I + 1] = a.y ^ kBias;
+        pk[4 * I + 2] = a.z ^ kBias, pk[4 * I + 3] = a.w ^ kBias;
     });
 
     static_for<P>([&](auto pp) {
@@ -236,8 +265,8 @@ __device__ __forceinline__ void decode_row(const uint4 *__restrict__ row, const 
             static_for<4>([&](auto tt) {
                 constexpr int c = 4 * I + decltype(tt)::value;
                 if constexpr (c % P == p) {
-                    uint32_t n = (pk[c / 8] >> (4 * (c % 8))) & 0xFu;          // q + 8
-                    float f = __uint_as_float(0x4B000000u | n) - 8388616.0f;   // q, exactly
+                    uint32_t n = (pk[c / CPW] >> (BITS * (c % CPW))) & ((1u << BITS) - 1u);   // q + 8 or q + 128
+                    float f = __uint_as_float(0x4B000000u | n) - kUnbias;                     // q, exactly
                     z[c / P] = f * (sig[c / GRP] * r[c % 4]);
                 }
             });
@@ -302,10 +331,11 @@ __device__ __forceinline__ void fill_lambda(float *cache, const float *__restric
     }
 }
 
-template <int D, int GRP, int P, bool BF16, int WARPS>
+template <int D, int GRP, int BITS, int P, bool BF16, int WARPS>
 __global__ void __launch_bounds__(WARPS * 32) kvq_encode_fft_kernel(const __grid_constant__ FftParams prm)
 {
-    using S = EncSmem<D, P>;
+    using S = EncSmem<D, P, BITS>;
+    constexpr int kRowBytes = D * BITS / 8;
     extern __shared__ __align__(128) unsigned char smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     unsigned char *wb = smem + kBarBytes + (size_t)warp * S::WARP_BYTES;
@@ -373,12 +403,12 @@ __global__ void __launch_bounds__(WARPS * 32) kvq_encode_fft_kernel(const __grid
             }
             if (active && lr == cur) {
                 const int64_t orow = prm.out_map(r);
-                encode_row<D, GRP, P, BF16>(
+                encode_row<D, GRP, BITS, P, BF16>(
                     reinterpret_cast<const uint4 *>(in_base + (stage * 32 + lane) * S::IN_STRIDE), prm.sign_xor,
                     reinterpret_cast<const float4 *>(lam_cache), reinterpret_cast<uint4 *>(out_row), stash,
                     static_cast<uint16_t *>(prm.scales) + orow * (D / GRP), lane);
                 fence_proxy_async();
-                bulk_store(static_cast<unsigned char *>(prm.packed) + orow * (D / 2), smem_u32(out_row), D / 2);
+                bulk_store(static_cast<unsigned char *>(prm.packed) + orow * kRowBytes, smem_u32(out_row), kRowBytes);
                 bulk_commit();
             }
             todo &= ~mine;
@@ -387,11 +417,12 @@ __global__ void __launch_bounds__(WARPS * 32) kvq_encode_fft_kernel(const __grid
     bulk_wait_all();
 }
 
-template <int D, int GRP, int P, bool BF16, int WARPS>
+template <int D, int GRP, int BITS, int P, bool BF16, int WARPS>
 __global__ void __launch_bounds__(WARPS * 32) kvq_decode_fft_kernel(const __grid_constant__ FftParams prm)
 {
-    using S = DecSmem<D, P>;
+    using S = DecSmem<D, P, BITS>;
     constexpr int G = D / GRP;
+    constexpr int kRowBytes = D * BITS / 8;
     extern __shared__ __align__(128) unsigned char smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     unsigned char *wb = smem + kBarBytes + (size_t)warp * S::WARP_BYTES;
@@ -420,8 +451,8 @@ __global__ void __launch_bounds__(WARPS * 32) kvq_decode_fft_kernel(const __grid
         const int64_t r = t * 32 + lane;
         const uint32_t bar = stage ? bar1 : bar0;
         if (r < N) {
-            mbar_arrive_expect_tx(bar, D / 2);
-            bulk_load(smem_u32(in_base + (stage * 32 + lane) * S::IN_STRIDE), packed + prm.in_map(r) * (D / 2), D / 2, bar);
+            mbar_arrive_expect_tx(bar, kRowBytes);
+            bulk_load(smem_u32(in_base + (stage * 32 + lane) * S::IN_STRIDE), packed + prm.in_map(r) * kRowBytes, kRowBytes, bar);
         } else {
             mbar_arrive(bar);
         }
@@ -500,7 +531,7 @@ __global__ void __launch_bounds__(WARPS * 32) kvq_decode_fft_kernel(const __grid
                 __syncwarp();
             }
             if (active && lr == cur) {
-                decode_row<D, GRP, P, BF16>(
+                decode_row<D, GRP, BITS, P, BF16>(
                     reinterpret_cast<const uint4 *>(in_base + (stage * 32 + lane) * S::IN_STRIDE), sig, prm.sign_xor,
                     reinterpret_cast<const float4 *>(lam_cache), reinterpret_cast<uint4 *>(out_row), stash, lane);
                 fence_proxy_async();
@@ -518,13 +549,15 @@ __global__ void __launch_bounds__(WARPS * 32) kvq_decode_fft_kernel(const __grid
 // ------------------------------------------------------------------------------------------
 template <typename Kern>
 static cudaError_t launch_persistent(Kern kern, int warps, size_t smem, int64_t N, const FftParams &prm,
-                                     cudaStream_t stream, int *cached_blocks_per_sm, int *cached_sms)
+                                     cudaStream_t stream, DeviceSlots *slots)
 {
+    int dev = 0;
+    cudaError_t e = current_device_slot(&dev);
+    if (e != cudaSuccess) return e;
+    int *cached_blocks_per_sm = &slots->blocks_per_sm[dev], *cached_sms = &slots->sms[dev];
     if (*cached_blocks_per_sm == 0) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        int dev = 0, nb = 0, sms = 0;
-        if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+        if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+        int nb = 0, sms = 0;
         if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
         if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, kern, warps * 32, smem)) != cudaSuccess) return e;
         if (nb < 1) return cudaErrorLaunchOutOfResources;
@@ -540,48 +573,57 @@ static cudaError_t launch_persistent(Kern kern, int warps, size_t smem, int64_t 
     return cudaGetLastError();
 }
 
-template <int D, int P, bool BF16, int WARPS>
+// GRP == 0 stands for one group over the whole vector (GRP = D).
+template <int D, int GRP, int BITS, int P, bool BF16, int WARPS>
 static cudaError_t launch_encode(int64_t N, const FftParams &prm, cudaStream_t stream)
 {
-    static int nb = 0, sms = 0;
-    constexpr size_t smem = kBarBytes + (size_t)WARPS * EncSmem<D, P>::WARP_BYTES;
-    return launch_persistent(kvq_encode_fft_kernel<D, 32, P, BF16, WARPS>, WARPS, smem, N, prm, stream, &nb, &sms);
+    static DeviceSlots slots;
+    constexpr int kGrp = GRP ? GRP : D;
+    constexpr size_t smem = kBarBytes + (size_t)WARPS * EncSmem<D, P, BITS>::WARP_BYTES;
+    static_assert(smem <= 232448, "encode kernel: shared memory over the per-CTA limit");
+    return launch_persistent(kvq_encode_fft_kernel<D, kGrp, BITS, P, BF16, WARPS>, WARPS, smem, N, prm, stream, &slots);
 }
 
-template <int D, int P, bool BF16, int WARPS>
+template <int D, int GRP, int BITS, int P, bool BF16, int WARPS>
 static cudaError_t launch_decode(int64_t N, const FftParams &prm, cudaStream_t stream)
 {
-    static int nb = 0, sms = 0;
-    constexpr size_t smem = kBarBytes + (size_t)WARPS * DecSmem<D, P>::WARP_BYTES;
-    return launch_persistent(kvq_decode_fft_kernel<D, 32, P, BF16, WARPS>, WARPS, smem, N, prm, stream, &nb, &sms);
+    static DeviceSlots slots;
+    constexpr int kGrp = GRP ? GRP : D;
+    constexpr size_t smem = kBarBytes + (size_t)WARPS * DecSmem<D, P, BITS>::WARP_BYTES;
+    static_assert(smem <= 232448, "decode kernel: shared memory over the per-CTA limit");
+    return launch_persistent(kvq_decode_fft_kernel<D, kGrp, BITS, P, BF16, WARPS>, WARPS, smem, N, prm, stream, &slots);
 }
 
-#define KVQ_DISPATCH(FN, DD, PP, WW)                                                    \
-    case DD:                                                                            \
-        return bf16 ? FN<DD, PP, true, WW>(N, prm, stream) : FN<DD, PP, false, WW>(N, prm, stream);
+// Defines kvq::ENC and kvq::DEC, the per-D dispatchers of one (GRP, BITS) variant.  Four warps per CTA, three for
+// the D = 256 encode with byte codes (its staging rows would not fit otherwise).
+#define KVQ_FFT_CASE(FN, GRP, BITS, DD, PP, WW)                                                               \
+    case DD:                                                                                                  \
+        return bf16 ? FN<DD, GRP, BITS, PP, true, WW>(N, prm, stream) : FN<DD, GRP, BITS, PP, false, WW>(N, prm, stream);
 
-cudaError_t fft_encode(int D, bool bf16, int64_t N, const FftParams &prm, cudaStream_t stream)
-{
-    switch (D) {
-        KVQ_DISPATCH(launch_encode, 64, 1, 4)
-        KVQ_DISPATCH(launch_encode, 96, 1, 4)
-        KVQ_DISPATCH(launch_encode, 128, 1, 4)
-        KVQ_DISPATCH(launch_encode, 160, 2, 4)
-        KVQ_DISPATCH(launch_encode, 256, 2, 4)
+#define KVQ_FFT_DEFINE_VARIANT(ENC, DEC, GRP, BITS)                                                           \
+    namespace kvq {                                                                                           \
+    cudaError_t ENC(int D, bool bf16, int64_t N, const FftParams &prm, cudaStream_t stream)                   \
+    {                                                                                                         \
+        switch (D) {                                                                                          \
+            KVQ_FFT_CASE(launch_encode, GRP, BITS, 64, 1, 4)                                                  \
+            KVQ_FFT_CASE(launch_encode, GRP, BITS, 96, 1, 4)                                                  \
+            KVQ_FFT_CASE(launch_encode, GRP, BITS, 128, 1, 4)                                                 \
+            KVQ_FFT_CASE(launch_encode, GRP, BITS, 160, 2, 4)                                                 \
+            KVQ_FFT_CASE(launch_encode, GRP, BITS, 256, 2, (BITS == 8 ? 3 : 4))                               \
+        }                                                                                                     \
+        return cudaErrorInvalidValue;                                                                         \
+    }                                                                                                         \
+    cudaError_t DEC(int D, bool bf16, int64_t N, const FftParams &prm, cudaStream_t stream)                   \
+    {                                                                                                         \
+        switch (D) {                                                                                          \
+            KVQ_FFT_CASE(launch_decode, GRP, BITS, 64, 1, 4)                                                  \
+            KVQ_FFT_CASE(launch_decode, GRP, BITS, 96, 1, 4)                                                  \
+            KVQ_FFT_CASE(launch_decode, GRP, BITS, 128, 1, 4)                                                 \
+            KVQ_FFT_CASE(launch_decode, GRP, BITS, 160, 2, 4)                                                 \
+            KVQ_FFT_CASE(launch_decode, GRP, BITS, 256, 2, 4)                                                 \
+        }                                                                                                     \
+        return cudaErrorInvalidValue;                                                                         \
+    }                                                                                                         \
     }
-    return cudaErrorInvalidValue;
-}
-
-cudaError_t fft_decode(int D, bool bf16, int64_t N, const FftParams &prm, cudaStream_t stream)
-{
-    switch (D) {
-        KVQ_DISPATCH(launch_decode, 64, 1, 4)
-        KVQ_DISPATCH(launch_decode, 96, 1, 4)
-        KVQ_DISPATCH(launch_decode, 128, 1, 4)
-        KVQ_DISPATCH(launch_decode, 160, 2, 4)
-        KVQ_DISPATCH(launch_decode, 256, 2, 4)
-    }
-    return cudaErrorInvalidValue;
-}
 
 }  // namespace kvq

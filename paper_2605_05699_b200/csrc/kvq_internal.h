@@ -26,7 +26,7 @@ struct RowMap {
 struct FftParams {
     const void *in;        // encode: x [N, D] half precision
     const float *lambda;   // [n_lambda, D] fp32
-    void *packed;          // [*, D/2] bytes (encode: out, decode: in)
+    void *packed;          // [*, D bits / 8] bytes (encode: out, decode: in)
     void *scales;          // [*, D/group] fp16 (encode: out, decode: in)
     void *out;             // decode: x^ [N, D] half precision
     int64_t N;
@@ -62,8 +62,24 @@ cudaError_t umma_encode_d256(bool bf16, int64_t N, const FftParams &prm, const f
 cudaError_t umma_decode_d256(bool bf16, int64_t N, const GemmParams &prm, const uint32_t *sign_xor, cudaStream_t stream);   // kvq_umma_decode256.cu
 cudaError_t umma_encode(int D, bool bf16, int64_t N, const FftParams &prm, const float *e0, cudaStream_t stream);
 
-cudaError_t fft_encode(int D, bool bf16, int64_t N, const FftParams &prm, cudaStream_t stream);
-cudaError_t fft_decode(int D, bool bf16, int64_t N, const FftParams &prm, cudaStream_t stream);
+// group: 32 or D (one scale per vector); bits: 4 or 8
+cudaError_t fft_encode(int D, int group, int bits, bool bf16, int64_t N, const FftParams &prm, cudaStream_t stream);
+cudaError_t fft_decode(int D, int group, int bits, bool bf16, int64_t N, const FftParams &prm, cudaStream_t stream);
+
+
+// A kernel's opt-in shared-memory size is a per-device function attribute, and SM counts differ between devices: the
+// launchers keep what they looked up in one slot per device ordinal.  Racing first calls write the same values.
+constexpr int kMaxDevices = 64;
+struct DeviceSlots {
+    int sms[kMaxDevices] = {};
+    int blocks_per_sm[kMaxDevices] = {};
+};
+inline cudaError_t current_device_slot(int *dev)
+{
+    cudaError_t e = cudaGetDevice(dev);
+    if (e != cudaSuccess) return e;
+    return (*dev < 0 || *dev >= kMaxDevices) ? cudaErrorInvalidDevice : cudaSuccess;
+}
 
 void count_launch();
 
@@ -72,6 +88,7 @@ void count_launch();
 // The plan behind the opaque kvq_plan_t handle.
 struct kvq_plan {
     int D, group;
+    int bits;              // 4 (nibble pairs) or 8 (one byte per code)
     uint64_t seed;
     int8_t signs[256];
     uint32_t sign_xor[128];

@@ -56,8 +56,7 @@ struct DeviceSlot {
     uint64_t table_seed = 0;
 };
 
-constexpr int kMaxDevices = 64;
-DeviceSlot g_slots[kMaxDevices];
+DeviceSlot g_slots[kvq::kMaxDevices];
 std::mutex g_mu;
 
 bool misaligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
@@ -72,7 +71,8 @@ extern "C" kvq_status_t kvq_decode_static(kvq_plan_t *plan, const uint8_t *packe
     if (!plan || N < 0) return KVQ_ERR_INVALID_ARG;
     if (dtype != KVQ_F16 && dtype != KVQ_BF16) return KVQ_ERR_INVALID_ARG;
     if (plan->D > kStaticMaxD) return KVQ_ERR_SCRATCH_LIMIT;                 // the table would not fit the block
-    if (plan->D != 128 || dtype != KVQ_F16) return KVQ_ERR_UNSUPPORTED_DIM;  // the kernel behind it: D = 128, fp16
+    if (plan->D != 128 || dtype != KVQ_F16 || plan->group != 32 || plan->bits != 4)
+        return KVQ_ERR_UNSUPPORTED_DIM;   // the kernel behind it: D = 128, fp16, groups of 32, 4-bit codes
     if (N == 0) return KVQ_OK;
     if (!packed || !scales || !out || !lambda || n_lambda < 1) return KVQ_ERR_INVALID_ARG;
     if (n_lambda > 1) {
@@ -88,7 +88,7 @@ extern "C" kvq_status_t kvq_decode_static(kvq_plan_t *plan, const uint8_t *packe
         (void)cudaGetLastError();
         return KVQ_ERR_CUDA;
     }
-    if (dev < 0 || dev >= kMaxDevices) return KVQ_ERR_INVALID_ARG;
+    if (dev < 0 || dev >= kvq::kMaxDevices) return KVQ_ERR_INVALID_ARG;
 
     std::lock_guard<std::mutex> lk(g_mu);
     DeviceSlot &slot = g_slots[dev];

@@ -470,13 +470,16 @@ template <int D>
 cudaError_t launch(int64_t N, const GemmParams &g, cudaStream_t stream)
 {
     using C = Cfg<D>;
-    static int sms = 0;
+    static DeviceSlots slots;
+    int dev = 0;
+    cudaError_t e = current_device_slot(&dev);
+    if (e != cudaSuccess) return e;
+    int &sms = slots.sms[dev];
     if (sms == 0) {
-        cudaError_t e = cudaFuncSetAttribute(kvq_decode_umma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
-        if (e != cudaSuccess) return e;
-        int dev = 0;
-        if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
-        if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+        int n = 0;
+        if ((e = cudaFuncSetAttribute(kvq_decode_umma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes)) != cudaSuccess) return e;
+        if ((e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+        sms = n;
     }
     if (!tensor_map_encode_fn()) return cudaErrorNotSupported;
     if (N >= (int64_t)1 << 31) return cudaErrorInvalidValue;   // tensor-map coordinates are 32-bit

@@ -456,13 +456,16 @@ template <bool BF16OUT>
 cudaError_t launch(int64_t N, const GemmParams &g, const uint32_t *sign_xor, cudaStream_t stream)
 {
     using C = Cfg<BF16OUT>;
-    static int sms = 0;
+    static DeviceSlots slots;
+    int dev = 0;
+    cudaError_t e = current_device_slot(&dev);
+    if (e != cudaSuccess) return e;
+    int &sms = slots.sms[dev];
     if (sms == 0) {
-        cudaError_t e = cudaFuncSetAttribute(kvq_decode_umma_d256_kernel<BF16OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
-        if (e != cudaSuccess) return e;
-        int dev = 0;
-        if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
-        if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+        int n = 0;
+        if ((e = cudaFuncSetAttribute(kvq_decode_umma_d256_kernel<BF16OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes)) != cudaSuccess) return e;
+        if ((e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+        sms = n;
     }
     if (!tensor_map_encode_fn()) return cudaErrorNotSupported;
     if (N >= (int64_t)1 << 31) return cudaErrorInvalidValue;   // tensor-map coordinates are 32-bit

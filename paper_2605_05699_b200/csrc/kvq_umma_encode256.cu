@@ -395,13 +395,16 @@ template <bool BF16, bool CALIB = false>
 cudaError_t launch(int64_t N, const FftParams &f, const float *e0, cudaStream_t stream, uint32_t *amax_bits = nullptr)
 {
     using C = Cfg<BF16>;
-    static int sms = 0;
+    static DeviceSlots slots;
+    int dev = 0;
+    cudaError_t e = current_device_slot(&dev);
+    if (e != cudaSuccess) return e;
+    int &sms = slots.sms[dev];
     if (sms == 0) {
-        cudaError_t e = cudaFuncSetAttribute(kvq_encode_umma_d256_kernel<BF16, CALIB>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
-        if (e != cudaSuccess) return e;
-        int dev = 0;
-        if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
-        if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+        int n = 0;
+        if ((e = cudaFuncSetAttribute(kvq_encode_umma_d256_kernel<BF16, CALIB>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes)) != cudaSuccess) return e;
+        if ((e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+        sms = n;
     }
     if (N >= (int64_t)1 << 31) return cudaErrorInvalidValue;   // tensor-map coordinates are 32-bit
 

@@ -27,21 +27,29 @@ def f16_bits_to_f64(b):
     return np.ascontiguousarray(b).view(np.uint16).view(np.float16).astype(np.float64)
 
 
-def check_encode(gpu_packed, gpu_scales_bits, ora, group, label=""):
-    """gpu_packed [N,D/2] uint8, gpu_scales_bits [N,G] uint16, ora = oracle.encode(..., want_v=True)."""
-    gpu_packed = np.ascontiguousarray(gpu_packed)
+def check_encode(gpu_packed, gpu_scales_bits, ora, group, label="", bits=4):
+    """gpu_packed [N, D bits/8] uint8, gpu_scales_bits [N,G] uint16, ora = oracle.encode(..., want_v=True, bits=bits).
+    The rules are those of the 4-bit codes with 7 read as 2^(bits-1) - 1; 8-bit codes are one byte each."""
+    gpu_packed = np.ascontiguousarray(gpu_packed).view(np.uint8)
     gpu_scales_bits = np.ascontiguousarray(gpu_scales_bits).view(np.uint16)
-    N, Dh = gpu_packed.shape
-    D = 2 * Dh
+    Q = (1 << (bits - 1)) - 1
+    N = gpu_packed.shape[0]
+    D = gpu_packed.shape[1] * 8 // bits
     G = D // group
-    q_gpu = ko.unpack_nibbles(gpu_packed)
-    # pack/unpack bit-exactness
-    assert np.array_equal(ko.pack_nibbles(q_gpu), gpu_packed), label + ": repacking the GPU codes changes bytes"
-    assert q_gpu.min(initial=0) >= -7 and q_gpu.max(initial=0) <= 7, label + ": code outside [-7, 7]"
     q_or = ora["codes"]
+    if bits == 4:
+        q_gpu = ko.unpack_nibbles(gpu_packed)
+        # pack/unpack bit-exactness
+        assert np.array_equal(ko.pack_nibbles(q_gpu), gpu_packed), label + ": repacking the GPU codes changes bytes"
+    else:
+        q_gpu = gpu_packed.view(np.int8)
+    assert q_gpu.min(initial=0) >= -Q and q_gpu.max(initial=0) <= Q, label + ": code outside [-%d, %d]" % (Q, Q)
     same = q_gpu == q_or
     byte_same = gpu_packed == ora["packed"]
-    assert np.array_equal(byte_same, same[:, 0::2] & same[:, 1::2]), label + ": byte layout disagrees with codes"
+    if bits == 4:
+        assert np.array_equal(byte_same, same[:, 0::2] & same[:, 1::2]), label + ": byte layout disagrees with codes"
+    else:
+        assert np.array_equal(byte_same, same), label + ": byte layout disagrees with codes"
 
     # scales
     bg = gpu_scales_bits.astype(np.int64)
@@ -68,7 +76,7 @@ def check_encode(gpu_packed, gpu_scales_bits, ora, group, label=""):
         with np.errstate(divide="ignore", invalid="ignore"):
             t_g, t_o = v / s_g, v / s_o
         at_tie = (np.abs(t_g - boundary) <= TIE_TOL) | (np.abs(t_o - boundary) <= TIE_TOL)
-        own = (s_g != s_o) & (np.clip(np.rint(t_g), -7, 7) == qg)
+        own = (s_g != s_o) & (np.clip(np.rint(t_g), -Q, Q) == qg)
         bad = ~(at_tie | own)
         assert not bad.any(), label + ": %d mismatched codes are not at a rounding tie (e.g. t=%r)" % (
             bad.sum(), t_o[bad][:4])

@@ -399,6 +399,75 @@ def test_flush_block_rejects_blocks_outside_the_cache():
     plan.close()
 
 
+# ---- base variants: one scale per vector and / or 8-bit codes (register-FFT kernels) -------------------
+
+@pytest.mark.parametrize("D,dtype,per_vector,nbits", [
+    (64, "f16", True, 4), (64, "f16", True, 8), (64, "bf16", False, 8),
+    (96, "f16", True, 4), (96, "bf16", True, 8),
+    (128, "f16", True, 4), (128, "f16", False, 8), (128, "bf16", True, 8),
+    (160, "f16", True, 8), (160, "bf16", False, 8),
+    (256, "bf16", True, 4), (256, "f16", True, 8), (256, "bf16", False, 8),
+])
+def test_base_variants_per_vector_scale_and_byte_codes(D, dtype, per_vector, nbits):
+    N, n_lambda, rpl = 5003, 3, 1700          # ragged, lambda rows straddle the warps' tiles
+    group = D if per_vector else G
+    odt = ko.F16 if dtype == "f16" else ko.BF16
+    plan = kb.Plan(D, group, 90 + D, bits=nbits)
+    sg = plan.signs()
+    lam = wl.make_lambda(n_lambda, D, 91)
+    x = wl.make_vectors(N, D, dtype, "k_outlier", 92 + nbits)
+    xd, lamd = x.cuda(), lam.cuda()
+    packed, scales = plan.empty_packed(N), plan.empty_scales(N)
+    assert packed.shape == (N, D * nbits // 8) and scales.shape == (N, D // group)
+    kb.kvq_encode(plan.handle, xd, lamd, packed, scales, rpl)
+    out = torch.empty(N, D, dtype=xd.dtype, device="cuda")
+    kb.kvq_decode(plan.handle, packed, scales, lamd, out, rpl)
+    torch.cuda.synchronize()
+    assert kb.kvq_plan_device_status(plan.handle) == 0
+    ora = ko.encode(bits(x), odt, sg, lam.numpy(), group, rpl, want_v=True, bits=nbits)
+    pk, sb = packed.cpu().numpy(), bits(scales)
+    parity.check_encode(pk, sb, ora, group, "variant encode", bits=nbits)
+    ob, o64 = ko.decode(pk, sb, sg, lam.numpy(), group, odt, rpl, want_f64=True, bits=nbits)
+    parity.check_decode(bits(out), ob, o64, odt, "variant decode")
+    plan.close()
+
+
+def test_base_variants_append_and_flush_and_refusals():
+    D, S, T = 128, 24, 40
+    plan = kb.Plan(D, D, 7, bits=8)
+    sg = plan.signs()
+    lam = wl.make_lambda(S, D, 8)
+    x = wl.make_vectors(S * T, D, "f16", "gaussian", 9).view(S, T, D)
+    packed = torch.full((S, T, D), 0x55, dtype=torch.uint8, device="cuda")
+    scales = torch.full((S, T, 1), 2.0, dtype=torch.float16, device="cuda")
+    dq = torch.full((S, T, D), 3.0, dtype=torch.float16, device="cuda")
+    lamd = lam.cuda()
+    kb.kvq_flush_block(plan.handle, x[:, :32].contiguous().cuda(), lamd, packed, scales, dq, 0, 1)
+    for t in range(32, 37):
+        kb.kvq_append(plan.handle, x[:, t].contiguous().cuda(), lamd, packed, scales, t, 1)
+    torch.cuda.synchronize()
+    assert kb.kvq_plan_device_status(plan.handle) == 0
+    assert bool((packed[:, 37:] == 0x55).all()) and bool((scales[:, 37:] == 2.0).all()) and bool((dq[:, 32:] == 3.0).all())
+    ora = ko.encode(bits(x[:, :37].reshape(-1, D)), ko.F16, sg, lam.numpy(), D, 37, want_v=True, bits=8)
+    pk, sb = packed[:, :37].reshape(-1, D).cpu().numpy(), bits(scales[:, :37].reshape(-1, 1))
+    parity.check_encode(pk, sb, ora, D, "variant cache", bits=8)
+    pk32, sb32 = packed[:, :32].reshape(-1, D).cpu().numpy(), bits(scales[:, :32].reshape(-1, 1))
+    ob, o64 = ko.decode(pk32, sb32, sg, lam.numpy(), D, ko.F16, 32, want_f64=True, bits=8)
+    parity.check_decode(bits(dq[:, :32].reshape(-1, D)), ob, o64, ko.F16, "variant dequantized cache")
+    # the tensor-core kernels and the no-allocation decode serve the fused layout only
+    kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_GEMM, kb.KVQ_IMPL_GEMM)
+    o = torch.empty(S * T, D, dtype=torch.float16, device="cuda")
+    with pytest.raises(kb.KvqError):
+        kb.kvq_decode(plan.handle, packed.view(-1, D), scales.view(-1, 1), lamd, o, T)
+    with pytest.raises(kb.KvqError):
+        kb.kvq_encode(plan.handle, x.reshape(-1, D).cuda(), lamd, packed.view(-1, D), scales.view(-1, 1), T)
+    plan.close()
+    with pytest.raises(kb.KvqError):
+        kb.Plan(128, 64, 1)           # groups other than 32 or D
+    with pytest.raises(kb.KvqError):
+        kb.Plan(128, 32, 1, bits=6)
+
+
 # ---- config 3: Gemma-3-1B-shaped, D = 256 bf16, prefix sweep ---------------------------------
 
 @pytest.mark.parametrize("prefix", [256, 1024])

@@ -54,6 +54,14 @@ def test_unsupported_dims_and_groups_are_rejected():
         assert L.kvq_plan_create(D, g, 1, ctypes.byref(h)) == kb.KVQ_ERR_UNSUPPORTED_DIM
         assert h.value is None
     assert L.kvq_plan_create(128, 32, 1, None) == kb.KVQ_ERR_INVALID_ARG
+    # base variants: one scale per vector (group = D) and 8-bit codes are plans too; nothing else is
+    for D, g, b in [(128, 128, 4), (96, 96, 8), (256, 32, 8), (64, 64, 8)]:
+        p = kb.Plan(D, g, 1, bits=b)
+        assert p.empty_packed(3, "cpu").shape == (3, D * b // 8) and p.empty_scales(3, "cpu").shape == (3, D // g)
+        p.close()
+    for D, g, b in [(128, 32, 5), (128, 32, 16), (128, 32, 0), (128, 64, 8), (96, 128, 4)]:
+        assert L.kvq_plan_create_ex(D, g, b, 1, ctypes.byref(h)) == kb.KVQ_ERR_UNSUPPORTED_DIM
+        assert h.value is None
 
 
 def test_bad_arguments_are_rejected_on_the_host():
