@@ -32,6 +32,10 @@
  *     codes in [-127, 127], one two's-complement byte per value) and / or one scale per vector (g = D, "per-token").
  *     The *_b entry points take the bit width b in {4, 8}; the entry points without it are b = 4.
  *
+ *   learned rotation at inference (Sec. 5.1 item 2): an orthogonal R in R^{DxD} sits between the transform and
+ *     lambda: v = lambda (.) (R z) on the way in, z^ = R^T (v^ / max(lambda, 1e-6)) on the way out.  The *_br entry
+ *     points take R row-major in fp64 (NULL = no rotation); training R is not part of this.
+ *
  * Readings where the paper is silent (each is listed in the design notes):
  *   - DFT sign convention e^{-2 pi i k n / D}; the imaginary part is packed as
  *     the transform returns it (the usual "rfft" convention).
@@ -319,6 +323,16 @@ void kvqo_unpack_nibbles(const uint8_t *bytes, int64_t n, int8_t *q)
 /* quantizer                                                           */
 /* ------------------------------------------------------------------ */
 
+/* y = R z (transpose == 0) or y = R^T z (transpose != 0); R row-major [D, D].  Plain sums in index order. */
+static void rotate_one(int D, const double *R, int transpose, const double *z, double *y)
+{
+    for (int i = 0; i < D; ++i) {
+        double s = 0.0;
+        for (int j = 0; j < D; ++j) s += (transpose ? R[(size_t)j * D + i] : R[(size_t)i * D + j]) * z[j];
+        y[i] = s;
+    }
+}
+
 /* codes of one vector to / from their stored bytes: nibble pairs for b = 4, one two's-complement byte per value for b = 8 */
 static void store_codes(const int8_t *q, int D, int bits, uint8_t *dst)
 {
@@ -372,9 +386,9 @@ static void quantize_one(int D, int g, int bits, const double *z, const float *l
 
 /* Forward path on fp64 input rows.  codes (nullable) receives the unpacked
  * int4 codes [N,D]; v_out (nullable) the rescaled transform lambda (.) z. */
-int kvqo_encode_f64_b(int D, int g, int bits, const int8_t *sg, const double *x, int64_t N, const float *lam,
-                      int64_t n_lambda, int64_t rows_per_lambda, uint8_t *packed, uint16_t *scales,
-                      int8_t *codes, double *v_out)
+int kvqo_encode_f64_br(int D, int g, int bits, const double *rot, const int8_t *sg, const double *x, int64_t N,
+                       const float *lam, int64_t n_lambda, int64_t rows_per_lambda, uint8_t *packed, uint16_t *scales,
+                       int8_t *codes, double *v_out)
 {
     if (check_common(D, g, N, n_lambda, rows_per_lambda) || (bits != 4 && bits != 8)) return 1;
     const int row_bytes = D * bits / 8;
@@ -383,9 +397,13 @@ int kvqo_encode_f64_b(int D, int g, int bits, const int8_t *sg, const double *x,
     const int G = D / g;
 #pragma omp parallel for schedule(static)
     for (int64_t r = 0; r < N; ++r) {
-        double z[D];
+        double z[D], y[D];
         int8_t q[D];
         srft_forward_one(&t, sg, x + r * D, z);
+        if (rot) {
+            rotate_one(D, rot, 0, z, y);
+            memcpy(z, y, sizeof(double) * (size_t)D);
+        }
         quantize_one(D, g, bits, z, lam + lambda_row(r, n_lambda, rows_per_lambda) * D, q, scales + r * G,
                      v_out ? v_out + r * D : NULL);
         store_codes(q, D, bits, packed + r * row_bytes);
@@ -393,6 +411,13 @@ int kvqo_encode_f64_b(int D, int g, int bits, const int8_t *sg, const double *x,
     }
     trig_free(&t);
     return 0;
+}
+
+int kvqo_encode_f64_b(int D, int g, int bits, const int8_t *sg, const double *x, int64_t N, const float *lam,
+                      int64_t n_lambda, int64_t rows_per_lambda, uint8_t *packed, uint16_t *scales,
+                      int8_t *codes, double *v_out)
+{
+    return kvqo_encode_f64_br(D, g, bits, NULL, sg, x, N, lam, n_lambda, rows_per_lambda, packed, scales, codes, v_out);
 }
 
 int kvqo_encode_f64(int D, int g, const int8_t *sg, const double *x, int64_t N, const float *lam,
@@ -403,9 +428,9 @@ int kvqo_encode_f64(int D, int g, const int8_t *sg, const double *x, int64_t N, 
 }
 
 /* Forward path on fp16 / bf16 rows: widen exactly, then as above. */
-int kvqo_encode_b(int D, int g, int bits, const int8_t *sg, const uint16_t *x, int dtype, int64_t N,
-                  const float *lam, int64_t n_lambda, int64_t rows_per_lambda, uint8_t *packed,
-                  uint16_t *scales, int8_t *codes, double *v_out)
+int kvqo_encode_br(int D, int g, int bits, const double *rot, const int8_t *sg, const uint16_t *x, int dtype, int64_t N,
+                   const float *lam, int64_t n_lambda, int64_t rows_per_lambda, uint8_t *packed,
+                   uint16_t *scales, int8_t *codes, double *v_out)
 {
     if (check_common(D, g, N, n_lambda, rows_per_lambda) || (bits != 4 && bits != 8)) return 1;
     const int row_bytes = D * bits / 8;
@@ -418,6 +443,10 @@ int kvqo_encode_b(int D, int g, int bits, const int8_t *sg, const uint16_t *x, i
         int8_t q[D];
         for (int n = 0; n < D; ++n) xr[n] = widen(x[r * D + n], dtype);
         srft_forward_one(&t, sg, xr, z);
+        if (rot) {
+            rotate_one(D, rot, 0, z, xr);
+            memcpy(z, xr, sizeof(double) * (size_t)D);
+        }
         quantize_one(D, g, bits, z, lam + lambda_row(r, n_lambda, rows_per_lambda) * D, q, scales + r * G,
                      v_out ? v_out + r * D : NULL);
         store_codes(q, D, bits, packed + r * row_bytes);
@@ -425,6 +454,13 @@ int kvqo_encode_b(int D, int g, int bits, const int8_t *sg, const uint16_t *x, i
     }
     trig_free(&t);
     return 0;
+}
+
+int kvqo_encode_b(int D, int g, int bits, const int8_t *sg, const uint16_t *x, int dtype, int64_t N,
+                  const float *lam, int64_t n_lambda, int64_t rows_per_lambda, uint8_t *packed,
+                  uint16_t *scales, int8_t *codes, double *v_out)
+{
+    return kvqo_encode_br(D, g, bits, NULL, sg, x, dtype, N, lam, n_lambda, rows_per_lambda, packed, scales, codes, v_out);
 }
 
 int kvqo_encode(int D, int g, const int8_t *sg, const uint16_t *x, int dtype, int64_t N,
@@ -436,9 +472,9 @@ int kvqo_encode(int D, int g, const int8_t *sg, const uint16_t *x, int dtype, in
 
 /* Inverse path.  out (nullable) gets x^ rounded to dtype; out_f64 (nullable) the
  * unrounded fp64 reconstruction. */
-int kvqo_decode_b(int D, int g, int bits, const int8_t *sg, const uint8_t *packed, const uint16_t *scales,
-                  int64_t N, const float *lam, int64_t n_lambda, int64_t rows_per_lambda, uint16_t *out,
-                  int dtype, double *out_f64)
+int kvqo_decode_br(int D, int g, int bits, const double *rot, const int8_t *sg, const uint8_t *packed,
+                   const uint16_t *scales, int64_t N, const float *lam, int64_t n_lambda, int64_t rows_per_lambda,
+                   uint16_t *out, int dtype, double *out_f64)
 {
     if (check_common(D, g, N, n_lambda, rows_per_lambda) || (bits != 4 && bits != 8)) return 1;
     const int row_bytes = D * bits / 8;
@@ -456,6 +492,10 @@ int kvqo_decode_b(int D, int g, int bits, const int8_t *sg, const uint8_t *packe
             double lc = (double)l[c] > 1e-6 ? (double)l[c] : 1e-6;    /* clamp at 1e-6 */
             z[c] = (double)q[c] * sigma / lc;
         }
+        if (rot) {
+            rotate_one(D, rot, 1, z, xr);
+            memcpy(z, xr, sizeof(double) * (size_t)D);
+        }
         srft_inverse_one(&t, sg, z, xr);
         for (int n = 0; n < D; ++n) {
             if (out) out[r * D + n] = narrow(xr[n], dtype);
@@ -464,6 +504,13 @@ int kvqo_decode_b(int D, int g, int bits, const int8_t *sg, const uint8_t *packe
     }
     trig_free(&t);
     return 0;
+}
+
+int kvqo_decode_b(int D, int g, int bits, const int8_t *sg, const uint8_t *packed, const uint16_t *scales,
+                  int64_t N, const float *lam, int64_t n_lambda, int64_t rows_per_lambda, uint16_t *out,
+                  int dtype, double *out_f64)
+{
+    return kvqo_decode_br(D, g, bits, NULL, sg, packed, scales, N, lam, n_lambda, rows_per_lambda, out, dtype, out_f64);
 }
 
 int kvqo_decode(int D, int g, const int8_t *sg, const uint8_t *packed, const uint16_t *scales,

@@ -71,12 +71,12 @@ def _load():
         lib.kvqo_encode.argtypes = [i32, i32, p, p, i32, i64, p, i64, i64, p, p, p, p]
         lib.kvqo_decode.restype = i32
         lib.kvqo_decode.argtypes = [i32, i32, p, p, p, i64, p, i64, i64, p, i32, p]
-        lib.kvqo_encode_f64_b.restype = i32
-        lib.kvqo_encode_f64_b.argtypes = [i32, i32, i32, p, p, i64, p, i64, i64, p, p, p, p]
-        lib.kvqo_encode_b.restype = i32
-        lib.kvqo_encode_b.argtypes = [i32, i32, i32, p, p, i32, i64, p, i64, i64, p, p, p, p]
-        lib.kvqo_decode_b.restype = i32
-        lib.kvqo_decode_b.argtypes = [i32, i32, i32, p, p, p, i64, p, i64, i64, p, i32, p]
+        lib.kvqo_encode_f64_br.restype = i32
+        lib.kvqo_encode_f64_br.argtypes = [i32, i32, i32, p, p, p, i64, p, i64, i64, p, p, p, p]
+        lib.kvqo_encode_br.restype = i32
+        lib.kvqo_encode_br.argtypes = [i32, i32, i32, p, p, p, i32, i64, p, i64, i64, p, p, p, p]
+        lib.kvqo_decode_br.restype = i32
+        lib.kvqo_decode_br.argtypes = [i32, i32, i32, p, p, p, p, i64, p, i64, i64, p, i32, p]
         lib.kvqo_append.restype = i32
         lib.kvqo_append.argtypes = [i32, i32, p, p, i32, i64, p, i64, i64, p, p, i64, i64]
         lib.kvqo_num_threads.restype = i32
@@ -96,6 +96,16 @@ def _raw16(x) -> np.ndarray:
     if x.dtype != np.uint16:
         raise TypeError("half-precision data must be float16 or raw uint16 bits")
     return x
+
+
+def _rot(rot, D):
+    """None, or the rotation as a contiguous fp64 [D, D] array (row-major)."""
+    if rot is None:
+        return None
+    rot = np.ascontiguousarray(rot, dtype=np.float64)
+    if rot.shape != (D, D):
+        raise ValueError("rotation must be [D, D]")
+    return rot
 
 
 def _lam(lam, D):
@@ -210,7 +220,7 @@ def unpack_nibbles(b) -> np.ndarray:
 
 # ---- quantizer ------------------------------------------------------------
 
-def encode_f64(x, sg, lam, group: int, rows_per_lambda: int = 0, want_v: bool = False, bits: int = 4):
+def encode_f64(x, sg, lam, group: int, rows_per_lambda: int = 0, want_v: bool = False, bits: int = 4, rot=None):
     """Forward path on fp64 rows.  Returns dict(packed, scales, codes[, v]).  ``packed`` is [N, D/2] nibble pairs for
     bits = 4 and [N, D] two's-complement bytes for bits = 8."""
     x = np.ascontiguousarray(x, dtype=np.float64)
@@ -222,8 +232,9 @@ def encode_f64(x, sg, lam, group: int, rows_per_lambda: int = 0, want_v: bool = 
     scales = np.empty((N, D // group), dtype=np.uint16)
     codes = np.empty((N, D), dtype=np.int8)
     v = np.empty((N, D), dtype=np.float64) if want_v else None
-    rc = _load().kvqo_encode_f64_b(D, group, bits, _ptr(sg), _ptr(x), N, _ptr(lam), nl, rows_per_lambda,
-                                   _ptr(packed), _ptr(scales), _ptr(codes), _ptr(v))
+    rot = _rot(rot, D)
+    rc = _load().kvqo_encode_f64_br(D, group, bits, _ptr(rot), _ptr(sg), _ptr(x), N, _ptr(lam), nl, rows_per_lambda,
+                                    _ptr(packed), _ptr(scales), _ptr(codes), _ptr(v))
     if rc:
         raise ValueError("kvqo_encode_f64: rc=%d" % rc)
     out = {"packed": packed, "scales": scales, "codes": codes}
@@ -232,7 +243,8 @@ def encode_f64(x, sg, lam, group: int, rows_per_lambda: int = 0, want_v: bool = 
     return out
 
 
-def encode(x_raw, dtype: int, sg, lam, group: int, rows_per_lambda: int = 0, want_v: bool = False, bits: int = 4):
+def encode(x_raw, dtype: int, sg, lam, group: int, rows_per_lambda: int = 0, want_v: bool = False, bits: int = 4,
+           rot=None):
     """Forward path on fp16 / bf16 rows given as raw bits.  Returns dict(packed, scales, codes[, v])."""
     x = _raw16(x_raw)
     D = x.shape[-1]
@@ -243,8 +255,9 @@ def encode(x_raw, dtype: int, sg, lam, group: int, rows_per_lambda: int = 0, wan
     scales = np.empty((N, D // group), dtype=np.uint16)
     codes = np.empty((N, D), dtype=np.int8)
     v = np.empty((N, D), dtype=np.float64) if want_v else None
-    rc = _load().kvqo_encode_b(D, group, bits, _ptr(sg), _ptr(x), dtype, N, _ptr(lam), nl, rows_per_lambda,
-                               _ptr(packed), _ptr(scales), _ptr(codes), _ptr(v))
+    rot = _rot(rot, D)
+    rc = _load().kvqo_encode_br(D, group, bits, _ptr(rot), _ptr(sg), _ptr(x), dtype, N, _ptr(lam), nl, rows_per_lambda,
+                                _ptr(packed), _ptr(scales), _ptr(codes), _ptr(v))
     if rc:
         raise ValueError("kvqo_encode: rc=%d" % rc)
     out = {"packed": packed, "scales": scales, "codes": codes}
@@ -254,7 +267,7 @@ def encode(x_raw, dtype: int, sg, lam, group: int, rows_per_lambda: int = 0, wan
 
 
 def decode(packed, scales, sg, lam, group: int, dtype: int, rows_per_lambda: int = 0, want_f64: bool = False,
-           bits: int = 4):
+           bits: int = 4, rot=None):
     """Inverse path.  Returns raw bits of the rounded output, or (bits, fp64) if want_f64."""
     packed = np.ascontiguousarray(packed).view(np.uint8)
     D = packed.shape[-1] * 8 // bits
@@ -264,8 +277,9 @@ def decode(packed, scales, sg, lam, group: int, dtype: int, rows_per_lambda: int
     lam, nl = _lam(lam, D)
     out = np.empty((N, D), dtype=np.uint16)
     o64 = np.empty((N, D), dtype=np.float64) if want_f64 else None
-    rc = _load().kvqo_decode_b(D, group, bits, _ptr(sg), _ptr(packed), _ptr(scales), N, _ptr(lam), nl,
-                               rows_per_lambda, _ptr(out), dtype, _ptr(o64))
+    rot = _rot(rot, D)
+    rc = _load().kvqo_decode_br(D, group, bits, _ptr(rot), _ptr(sg), _ptr(packed), _ptr(scales), N, _ptr(lam), nl,
+                                rows_per_lambda, _ptr(out), dtype, _ptr(o64))
     if rc:
         raise ValueError("kvqo_decode: rc=%d" % rc)
     return (out, o64) if want_f64 else out

@@ -11,7 +11,7 @@
 //
 // For the larger D the complex FFT is split once more by output parity into
 // P = 2 sequential passes of length L = H/2 (decimation in frequency), which
-// halves the number of live registers; see kvq_fft_kernels.cu.
+// halves the number of live registers; see kvq_fft_kernels.cuh.
 #pragma once
 
 #include "kvq_device.cuh"

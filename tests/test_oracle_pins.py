@@ -509,6 +509,81 @@ def test_a_group_of_the_whole_vector_equals_groups_of_32_that_share_their_maximu
         assert np.array_equal(a["scales"], b["scales"].repeat(4, axis=1))
 
 
+# --------------------------------------------------------------------------
+# learned rotation at inference (Sec. 5.1 item 2): v = lambda (.) (R z), z^ = R^T (v^ / lambda)
+# --------------------------------------------------------------------------
+
+def _random_orthogonal(D, seed):
+    q, r = np.linalg.qr(rng(seed).standard_normal((D, D)))
+    return q * np.sign(np.diag(r))
+
+
+def test_identity_rotation_changes_nothing():
+    D = 96
+    s = ko.signs(D, 4)
+    x = rng(60).standard_normal((40, D)).astype(np.float16)
+    lam = rng(61).uniform(0.5, 2, D).astype(np.float32)
+    a = ko.encode(x, ko.F16, s, lam, 32, want_v=True)
+    b = ko.encode(x, ko.F16, s, lam, 32, want_v=True, rot=np.eye(D))
+    assert all(np.array_equal(a[k], b[k]) for k in ("packed", "scales", "codes", "v"))
+    assert np.array_equal(ko.decode(a["packed"], a["scales"], s, lam, 32, ko.F16),
+                          ko.decode(a["packed"], a["scales"], s, lam, 32, ko.F16, rot=np.eye(D)))
+
+
+def test_the_rotation_that_undoes_the_transform_leaves_the_plain_quantizer():
+    # R = T^T for the transform matrix T (z = T x): then R z = x, and the path is the quantizer applied to lambda (.) x
+    # itself; on the way out R^T = T meets the inverse transform T^T, so the output is q sigma / lambda.  A rotation
+    # applied transposed, or on the wrong side of lambda, fails this.
+    D = 64
+    s = ko.signs(D, 12)
+    R = ko.srft_forward(np.eye(D), s)          # row i = T e_i, i.e. R = T^T
+    assert np.allclose(R @ R.T, np.eye(D), atol=1e-13)
+    r = rng(62)
+    q_true = r.integers(-7, 8, (30, D)).astype(np.float64)
+    q_true[:, [0, 40]] = 7                     # every group of 32 peaks at 7: sigma = step exactly
+    step = 0.25
+    lam = np.where(np.arange(D) % 2 == 0, 2.0, 0.5).astype(np.float32)
+    x = q_true * step / lam                    # lambda (.) x = q step, exactly (powers of two)
+    e = ko.encode_f64(x, s, lam, 32, want_v=True, rot=R)
+    assert np.allclose(e["v"], q_true * step, atol=1e-13)
+    assert np.array_equal(e["codes"], q_true.astype(np.int8))
+    assert np.all(e["scales"] == np.float16(step).view(np.uint16))
+    _, xr = ko.decode(e["packed"], e["scales"], s, lam, 32, ko.F16, want_f64=True, rot=R)
+    assert np.allclose(xr, x, atol=1e-13)
+    # without the rotation the same input gives something else
+    assert not np.array_equal(ko.encode_f64(x, s, lam, 32)["codes"], e["codes"])
+
+
+def test_a_permutation_rotation_permutes_the_codes_of_a_per_vector_quantizer():
+    D = 128
+    s = ko.signs(D, 5)
+    x = rng(63).standard_normal((25, D))
+    perm = rng(64).permutation(D)
+    P = np.zeros((D, D))
+    P[np.arange(D), perm] = 1.0               # (P z)_i = z_perm[i]
+    one = np.ones(D, np.float32)
+    for nbits in (4, 8):
+        a = ko.encode_f64(x, s, one, D, bits=nbits)
+        b = ko.encode_f64(x, s, one, D, bits=nbits, rot=P)
+        assert np.array_equal(b["codes"], a["codes"][:, perm]) and np.array_equal(a["scales"], b["scales"])
+
+
+def test_an_orthogonal_rotation_keeps_norms_and_is_undone_by_its_transpose():
+    D = 160
+    s = ko.signs(D, 6)
+    R = _random_orthogonal(D, 65)
+    x = rng(66).standard_normal((20, D))
+    one = np.ones(D, np.float32)
+    e = ko.encode_f64(x, s, one, 32, want_v=True, rot=R)
+    assert np.allclose(np.linalg.norm(e["v"], axis=1), np.linalg.norm(x, axis=1), rtol=1e-12)
+    assert np.allclose(e["v"], ko.srft_forward(x, s) @ R.T, atol=1e-12)
+    _, xr = ko.decode(e["packed"], e["scales"], s, one, 32, ko.F16, want_f64=True, rot=R)
+    vq = e["codes"] * ko.f16_to_f64(e["scales"]).repeat(32, axis=1)
+    # end to end the path is orthogonal: the reconstruction error is the rounding error, rotated
+    assert np.allclose(np.linalg.norm(xr - x, axis=1), np.linalg.norm(vq - e["v"], axis=1), rtol=1e-9)
+    assert np.allclose(ko.srft_forward(xr, s) @ R.T, vq, atol=1e-12)
+
+
 def test_flushing_blocks_that_cover_the_prefix_equals_the_full_prefix_decode():
     # Sec. 7.2: the incremental path (flush a block, keep its dequantized rows) must leave exactly what encoding the
     # whole prefix at once and decoding all of it would give, whatever the block boundaries are
