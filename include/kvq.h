@@ -87,6 +87,22 @@ kvq_status_t kvq_plan_create(int D, int group, uint64_t seed, kvq_plan_t **out);
  */
 kvq_status_t kvq_plan_create_ex(int D, int group, int bits, uint64_t seed, kvq_plan_t **out);
 
+/*
+ * kvq_plan_set_rotation -- learned rotation at inference (Sec. 5.1 item 2): an orthogonal R in R^{D x D} between the
+ * transform and lambda, v = lambda (.) (R z) on the way in and z^ = R^T (v^ / max(lambda, 1e-6)) on the way out.
+ *   R_host   HOST pointer, [D, D] row-major fp32, copied by the call; NULL removes the rotation.  The library does not
+ *            check that R is orthogonal: the inverse path applies R^T.  Training R is the caller's business.
+ * The rotation is folded into the D x D tables of the tensor-core kernels, so it costs nothing per vector, and it
+ * exists only where those kernels do: group = 32, bits = 4; kvq_encode / kvq_append / kvq_calibrate_lambda for the
+ * (D, dtype) pairs KVQ_IMPL_GEMM lists for encode, kvq_decode for those it lists for decode (D = 256 then runs a
+ * dense 256 x 256 kernel).  On a rotated plan every call takes the tensor-core path whatever its size;
+ * KVQ_IMPL_FFT, kvq_flush_block, kvq_decode_static and unsupported (D, dtype) pairs return UNSUPPORTED_DIM.
+ * If the plan's device tables already exist they are rewritten after a device synchronisation: call it with the
+ * plan's device current and no call using the plan in flight on another thread.
+ * Errors: INVALID_ARG (null plan, non-finite entry, wrong device), UNSUPPORTED_DIM, NOMEM, CUDA.
+ */
+kvq_status_t kvq_plan_set_rotation(kvq_plan_t *plan, const float *R_host /* [D, D] or NULL */);
+
 /* Frees the plan and its device tables.  NULL is a no-op.  The caller must make sure no call
  * using the plan is still running on the GPU. */
 kvq_status_t kvq_plan_destroy(kvq_plan_t *plan);

@@ -36,7 +36,7 @@ KVQ_IMPL_GEMM = 2
 
 # every symbol include/kvq.h declares
 EXPORTS = (
-    "kvq_plan_create", "kvq_plan_create_ex", "kvq_plan_destroy", "kvq_plan_get_signs", "kvq_plan_describe", "kvq_plan_set_impl",
+    "kvq_plan_create", "kvq_plan_create_ex", "kvq_plan_set_rotation", "kvq_plan_destroy", "kvq_plan_get_signs", "kvq_plan_describe", "kvq_plan_set_impl",
     "kvq_plan_device_status", "kvq_encode", "kvq_decode", "kvq_append", "kvq_decode_static", "kvq_calibrate_lambda", "kvq_flush_block", "kvq_status_string",
     "kvq_launch_count",
 )
@@ -61,6 +61,8 @@ def lib() -> ctypes.CDLL:
         i32, i64, u64, vp = ctypes.c_int, ctypes.c_int64, ctypes.c_uint64, ctypes.c_void_p
         L.kvq_plan_create.restype = i32
         L.kvq_plan_create.argtypes = [i32, i32, u64, ctypes.POINTER(vp)]
+        L.kvq_plan_set_rotation.restype = i32
+        L.kvq_plan_set_rotation.argtypes = [vp, vp]
         L.kvq_plan_create_ex.restype = i32
         L.kvq_plan_create_ex.argtypes = [i32, i32, i32, u64, ctypes.POINTER(vp)]
         L.kvq_plan_destroy.restype = i32
@@ -140,6 +142,24 @@ def kvq_plan_create_ex(D: int, group: int, bits: int, seed: int) -> int:
     h = ctypes.c_void_p()
     _check(lib().kvq_plan_create_ex(D, group, bits, ctypes.c_uint64(seed & (2**64 - 1)), ctypes.byref(h)), "kvq_plan_create_ex")
     return h.value
+
+
+def kvq_plan_set_rotation(plan: int, R, D: int) -> None:
+    """R: host fp32 [D, D] (torch CPU tensor or numpy array) for a plan of head dimension D, or None to remove the
+    rotation."""
+    if R is None:
+        _check(lib().kvq_plan_set_rotation(plan, None), "kvq_plan_set_rotation")
+        return
+    if isinstance(R, torch.Tensor):
+        if R.is_cuda:
+            raise ValueError("the rotation is a host matrix")
+        R = R.detach().to(torch.float32).contiguous().numpy()
+    import numpy as np
+
+    R = np.ascontiguousarray(R, dtype=np.float32)
+    if R.shape != (D, D):
+        raise ValueError("the rotation must be [D, D]")
+    _check(lib().kvq_plan_set_rotation(plan, R.ctypes.data_as(ctypes.c_void_p)), "kvq_plan_set_rotation")
 
 
 def kvq_plan_destroy(plan: int) -> None:
@@ -257,6 +277,9 @@ class Plan:
 
     def signs(self):
         return kvq_plan_get_signs(self.handle, self.D)
+
+    def set_rotation(self, R) -> None:
+        kvq_plan_set_rotation(self.handle, R, self.D)
 
     def close(self):
         if getattr(self, "handle", None):

@@ -4,6 +4,7 @@
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <vector>
 
 #include "../../include/kvq.h"
 #include "kvq_internal.h"
@@ -46,19 +47,51 @@ static int radix_plan(int n, int *out)
 //   D^-1/2                       (c = 0),        (-1)^n D^-1/2               (c = D/2),
 //   sqrt(2/D) cos(2 pi c n / D)  (0 < c < D/2),  -sqrt(2/D) sin(2 pi k n / D) (c = D/2 + k, 0 < k < D/2).
 // M is orthogonal, so the inverse transform is x^_n = s_n sum_c M[c][n] z^_c.
-static void build_b0(const kvq_plan *p, float *b0)
+// With a rotation R (Sec. 5.1 item 2: v = lambda (.) R z, z^ = R^T (v^ / lambda)) the table becomes
+// b0'[n][c'] = sum_c b0[n][c] R[c'][c]: the forward table is its transpose either way.  Sums in fp64.
+// Returns the largest |entry|.
+static double build_b0(const kvq_plan *p, float *b0)
 {
     const int D = p->D, H = D / 2;
     const double pi = 3.14159265358979323846;
-    for (int n = 0; n < D; ++n)
+    std::vector<double> row((size_t)D);
+    double tmax = 0.0;
+    for (int n = 0; n < D; ++n) {
         for (int c = 0; c < D; ++c) {
             double m;
             if (c == 0) m = 1.0 / std::sqrt((double)D);
             else if (c == H) m = ((n & 1) ? -1.0 : 1.0) / std::sqrt((double)D);
             else if (c < H) m = std::sqrt(2.0 / D) * std::cos(2.0 * pi * (double)((long)c * n % D) / D);
             else m = -std::sqrt(2.0 / D) * std::sin(2.0 * pi * (double)((long)(c - H) * n % D) / D);
-            b0[(size_t)n * D + c] = (float)(p->signs[n] * m);
+            row[(size_t)c] = p->signs[n] * m;
         }
+        for (int c = 0; c < D; ++c) {
+            double v = row[(size_t)c];
+            if (p->rot) {
+                v = 0.0;
+                for (int k = 0; k < D; ++k) v += row[(size_t)k] * p->rot[(size_t)c * D + k];
+            }
+            b0[(size_t)n * D + c] = (float)v;
+            tmax = std::fmax(tmax, std::fabs(v));
+        }
+    }
+    return tmax;
+}
+
+// Host copies of both tables: b0 [n][c] for the decode kernels, its transpose e0 [c][n] for the encode kernels.
+static bool make_tables(kvq_plan *p, std::vector<float> &b0, std::vector<float> &e0)
+{
+    const size_t D = (size_t)p->D;
+    try {
+        b0.resize(D * D);
+        e0.resize(D * D);
+    } catch (...) {
+        return false;
+    }
+    p->table_max = (float)build_b0(p, b0.data());
+    for (size_t n = 0; n < D; ++n)
+        for (size_t c = 0; c < D; ++c) e0[c * D + n] = b0[n * D + c];
+    return true;
 }
 
 using namespace kvq;
@@ -87,58 +120,33 @@ static kvq_status_t ensure_device(kvq_plan *p)
     p->table_bytes = 256;
     if (umma_encode_supported(p->D, false) || umma_decode_supported(p->D, false)) {   // tables of the tensor-core kernels
         const size_t bytes = sizeof(float) * (size_t)p->D * p->D;
-        float *host = new (std::nothrow) float[(size_t)p->D * p->D];
-        float *devp = nullptr;
-        if (!host || cudaMalloc(&devp, bytes) != cudaSuccess) {
+        std::vector<float> b0, e0;
+        float *db = nullptr, *de = nullptr;
+        bool ok = make_tables(p, b0, e0) && cudaMalloc(&db, bytes) == cudaSuccess && cudaMalloc(&de, bytes) == cudaSuccess;
+        kvq_status_t why = KVQ_ERR_NOMEM;
+        if (ok) {
+            ok = cudaMemcpy(db, b0.data(), bytes, cudaMemcpyHostToDevice) == cudaSuccess &&
+                 cudaMemcpy(de, e0.data(), bytes, cudaMemcpyHostToDevice) == cudaSuccess;
+            why = KVQ_ERR_CUDA;
+        }
+        if (!ok) {
             (void)cudaGetLastError();
-            delete[] host;
+            if (db) cudaFree(db);
+            if (de) cudaFree(de);
             cudaFree(st);
             p->d_status = nullptr;
-            return KVQ_ERR_NOMEM;
+            return why;
         }
-        build_b0(p, host);
-        cudaError_t e = cudaMemcpy(devp, host, bytes, cudaMemcpyHostToDevice);
-        delete[] host;
-        if (e != cudaSuccess) {
-            (void)cudaGetLastError();
-            cudaFree(devp);
-            cudaFree(st);
-            p->d_status = nullptr;
-            return KVQ_ERR_CUDA;
-        }
-        p->d_b0 = devp;
-        p->table_bytes += bytes;
-        // the forward table is the transpose: e0[c][n] = b0[n][c]
-        float *hostT = new (std::nothrow) float[(size_t)p->D * p->D];
-        float *devT = nullptr;
-        bool okT = hostT && cudaMalloc(&devT, bytes) == cudaSuccess;
-        if (okT) {
-            float *tmp = new (std::nothrow) float[(size_t)p->D * p->D];
-            okT = tmp != nullptr;
-            if (okT) {
-                build_b0(p, tmp);
-                for (int n = 0; n < p->D; ++n)
-                    for (int c = 0; c < p->D; ++c) hostT[(size_t)c * p->D + n] = tmp[(size_t)n * p->D + c];
-                okT = cudaMemcpy(devT, hostT, bytes, cudaMemcpyHostToDevice) == cudaSuccess;
-            }
-            delete[] tmp;
-        }
-        delete[] hostT;
-        if (!okT) {
-            (void)cudaGetLastError();
-            if (devT) cudaFree(devT);
-            cudaFree(devp);
-            cudaFree(st);
-            p->d_b0 = nullptr;
-            p->d_status = nullptr;
-            return KVQ_ERR_NOMEM;
-        }
-        p->d_e0 = devT;
-        p->table_bytes += bytes;
+        p->d_b0 = db;
+        p->d_e0 = de;
+        p->table_bytes += 2 * bytes;
     }
     p->device = dev;
     return KVQ_OK;
 }
+
+// the tensor-core kernels exist for the fused layout only: groups of 32, 4-bit codes
+static bool gemm_layout(const kvq_plan *p) { return p->group == 32 && p->bits == 4; }
 
 static bool misaligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
 
@@ -164,6 +172,7 @@ static void fill_params(const kvq_plan *p, FftParams &prm, int64_t N, const floa
     prm.out_map = RowMap{1, 1, 0};
     prm.in_map = RowMap{1, 1, 0};
     prm.status = p->d_status;
+    prm.table_max = p->table_max;
     std::memcpy(prm.sign_xor, p->sign_xor, sizeof(prm.sign_xor));
 }
 
@@ -191,6 +200,8 @@ kvq_status_t kvq_plan_create_ex(int D, int group, int bits, uint64_t seed, kvq_p
     p->d_b0 = nullptr;
     p->d_e0 = nullptr;
     p->table_bytes = 0;
+    p->rot = nullptr;
+    p->table_max = (float)std::sqrt(2.0 / D);
     std::memset(p->signs, 0, sizeof(p->signs));
     std::memset(p->sign_xor, 0, sizeof(p->sign_xor));
     for (int n = 0; n < D; ++n) {
@@ -214,7 +225,50 @@ kvq_status_t kvq_plan_destroy(kvq_plan_t *plan)
     if (plan->d_e0) {
         if (cudaFree(plan->d_e0) != cudaSuccess) (void)cudaGetLastError();
     }
+    delete[] plan->rot;
     delete plan;
+    return KVQ_OK;
+}
+
+kvq_status_t kvq_plan_set_rotation(kvq_plan_t *plan, const float *R_host)
+{
+    if (!plan) return KVQ_ERR_INVALID_ARG;
+    // the rotation lives in the tensor-core kernels' tables: the plan must be one they serve
+    if (R_host && (!gemm_layout(plan) || !umma_encode_supported(plan->D, false))) return KVQ_ERR_UNSUPPORTED_DIM;
+    std::lock_guard<std::mutex> lk(plan->mu);
+    const size_t n = (size_t)plan->D * plan->D;
+    double *rot = nullptr;
+    if (R_host) {
+        rot = new (std::nothrow) double[n];
+        if (!rot) return KVQ_ERR_NOMEM;
+        for (size_t i = 0; i < n; ++i) {
+            if (!std::isfinite(R_host[i])) {
+                delete[] rot;
+                return KVQ_ERR_INVALID_ARG;
+            }
+            rot[i] = (double)R_host[i];
+        }
+    }
+    delete[] plan->rot;
+    plan->rot = rot;
+    if (plan->device < 0 || !plan->d_b0) {   // tables are built on first use
+        if (!rot) plan->table_max = (float)std::sqrt(2.0 / plan->D);
+        return KVQ_OK;
+    }
+    // tables exist: rewrite them in place, on the plan's device, after everything queued there has finished
+    int cur = -1;
+    if (cudaGetDevice(&cur) != cudaSuccess || cur != plan->device) {
+        (void)cudaGetLastError();
+        return KVQ_ERR_INVALID_ARG;
+    }
+    std::vector<float> b0, e0;
+    if (!make_tables(plan, b0, e0)) return KVQ_ERR_NOMEM;
+    const size_t bytes = sizeof(float) * n;
+    if (cudaDeviceSynchronize() != cudaSuccess || cudaMemcpy(plan->d_b0, b0.data(), bytes, cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemcpy(plan->d_e0, e0.data(), bytes, cudaMemcpyHostToDevice) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return KVQ_ERR_CUDA;
+    }
     return KVQ_OK;
 }
 
@@ -263,9 +317,6 @@ kvq_status_t kvq_plan_device_status(kvq_plan_t *plan, uint32_t *word)
     return *word ? KVQ_ERR_TIMEOUT : KVQ_OK;
 }
 
-// the tensor-core kernels exist for the fused layout only: groups of 32, 4-bit codes
-static bool gemm_layout(const kvq_plan *p) { return p->group == 32 && p->bits == 4; }
-
 static kvq_status_t encode_common(kvq_plan_t *plan, const void *x, kvq_dtype_t dtype, int64_t N, const float *lambda,
                                   int64_t n_lambda, int64_t rows_per_lambda, uint8_t *packed, void *scales,
                                   const RowMap &out_map, void *cuda_stream)
@@ -279,6 +330,7 @@ static kvq_status_t encode_common(kvq_plan_t *plan, const void *x, kvq_dtype_t d
     if (misaligned16(x) || misaligned16(packed) || misaligned16(scales)) return KVQ_ERR_ALIGNMENT;
     const bool gemm_ok = gemm_layout(plan) && umma_encode_supported(plan->D, dtype == KVQ_BF16);
     if (plan->enc_impl == KVQ_IMPL_GEMM && !gemm_ok) return KVQ_ERR_UNSUPPORTED_DIM;
+    if (plan->rot && (!gemm_ok || plan->enc_impl == KVQ_IMPL_FFT)) return KVQ_ERR_UNSUPPORTED_DIM;   // the rotation is in the GEMM tables
     if ((st = ensure_device(plan)) != KVQ_OK) return st;
     FftParams prm;
     fill_params(plan, prm, N, lambda, n_lambda, rows_per_lambda);
@@ -287,7 +339,7 @@ static kvq_status_t encode_common(kvq_plan_t *plan, const void *x, kvq_dtype_t d
     prm.scales = scales;
     prm.out_map = out_map;
     // the tensor-core kernel pays a fixed set-up per launch (B operand build); small calls stay on the register FFT
-    const bool use_gemm = gemm_ok && (plan->enc_impl == KVQ_IMPL_GEMM || (plan->enc_impl == KVQ_IMPL_AUTO && N >= kGemmEncodeMinRows));
+    const bool use_gemm = gemm_ok && (plan->rot || plan->enc_impl == KVQ_IMPL_GEMM || (plan->enc_impl == KVQ_IMPL_AUTO && N >= kGemmEncodeMinRows));
     cudaError_t e = use_gemm ? umma_encode(plan->D, dtype == KVQ_BF16, N, prm, plan->d_e0, static_cast<cudaStream_t>(cuda_stream))
                              : fft_encode(plan->D, plan->group, plan->bits, dtype == KVQ_BF16, N, prm, static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) {
@@ -324,6 +376,7 @@ kvq_status_t kvq_decode(kvq_plan_t *plan, const uint8_t *packed, const void *sca
     if (misaligned16(packed) || misaligned16(scales) || misaligned16(out)) return KVQ_ERR_ALIGNMENT;
     const bool gemm_ok = gemm_layout(plan) && umma_decode_supported(plan->D, dtype == KVQ_BF16);
     if (plan->dec_impl == KVQ_IMPL_GEMM && !gemm_ok) return KVQ_ERR_UNSUPPORTED_DIM;
+    if (plan->rot && (!gemm_ok || plan->dec_impl == KVQ_IMPL_FFT)) return KVQ_ERR_UNSUPPORTED_DIM;   // the rotation is in the GEMM tables
     if ((st = ensure_device(plan)) != KVQ_OK) return st;
     if (gemm_ok && plan->dec_impl != KVQ_IMPL_FFT) {
         GemmParams g;
@@ -336,7 +389,11 @@ kvq_status_t kvq_decode(kvq_plan_t *plan, const uint8_t *packed, const void *sca
         g.n_lambda = n_lambda;
         g.rows_per_lambda = rows_per_lambda < 1 ? 1 : rows_per_lambda;
         g.status = plan->d_status;
-        if (umma_decode(plan->D, dtype == KVQ_BF16, N, g, plan->sign_xor, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
+        // D = 256: the radix-2 kernel needs the transform's even / odd structure, which a rotation destroys
+        const cudaError_t e = plan->rot && plan->D == 256
+                                  ? umma_decode_d256_dense(dtype == KVQ_BF16, N, g, static_cast<cudaStream_t>(cuda_stream))
+                                  : umma_decode(plan->D, dtype == KVQ_BF16, N, g, plan->sign_xor, static_cast<cudaStream_t>(cuda_stream));
+        if (e != cudaSuccess) {
             (void)cudaGetLastError();
             return KVQ_ERR_CUDA;
         }
@@ -364,6 +421,7 @@ kvq_status_t kvq_flush_block(kvq_plan_t *plan, const void *x_block, kvq_dtype_t 
     if (dtype != KVQ_F16 && dtype != KVQ_BF16) return KVQ_ERR_INVALID_ARG;
     if (S == 0 || rows == 0) return KVQ_OK;
     if (!dq_cache) return KVQ_ERR_INVALID_ARG;
+    if (plan->rot) return KVQ_ERR_UNSUPPORTED_DIM;   // its decode half runs on the register FFT, which has no rotation
     if (misaligned16(dq_cache)) return KVQ_ERR_ALIGNMENT;
     if (S > INT64_MAX / rows) return KVQ_ERR_INVALID_ARG;
     const int64_t N = S * rows;

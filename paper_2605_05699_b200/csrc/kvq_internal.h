@@ -34,6 +34,7 @@ struct FftParams {
     RowMap out_map;             // row of packed / scales (encode) or of out (decode) that row r goes to
     RowMap in_map;              // decode: row of packed / scales that row r comes from
     uint32_t *status;           // per-plan device status word
+    float table_max;            // tensor-core encode: largest |entry| of the plan's forward table (sqrt(2/D) without a rotation)
     uint32_t sign_xor[128];     // word m: bit 15 set if s_{2m} = -1, bit 31 set if s_{2m+1} = -1
 };
 
@@ -60,6 +61,7 @@ cudaError_t umma_calibrate(int D, bool bf16, int64_t N, const FftParams &prm, co
 cudaError_t umma_calibrate_d256(bool bf16, int64_t N, const FftParams &prm, const float *e0, uint32_t *amax_bits, cudaStream_t stream);
 cudaError_t umma_encode_d256(bool bf16, int64_t N, const FftParams &prm, const float *e0, cudaStream_t stream);   // kvq_umma_encode256.cu
 cudaError_t umma_decode_d256(bool bf16, int64_t N, const GemmParams &prm, const uint32_t *sign_xor, cudaStream_t stream);   // kvq_umma_decode256.cu
+cudaError_t umma_decode_d256_dense(bool bf16, int64_t N, const GemmParams &prm, cudaStream_t stream);   // kvq_umma_decode256_dense.cu: any table
 cudaError_t umma_encode(int D, bool bf16, int64_t N, const FftParams &prm, const float *e0, cudaStream_t stream);
 
 // group: 32 or D (one scale per vector); bits: 4 or 8
@@ -100,4 +102,6 @@ struct kvq_plan {
     float *d_b0;           // [D, D] fp32 inverse-transform matrix with the signs folded in (GEMM decode), or null
     float *d_e0;           // [D, D] fp32 forward-transform matrix with the signs folded in (GEMM encode), or null
     size_t table_bytes;
+    double *rot;           // host, [D, D] row-major: the rotation between the transform and lambda, or null
+    float table_max;       // largest |entry| of the forward table
 };

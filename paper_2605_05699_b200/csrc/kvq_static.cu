@@ -71,8 +71,8 @@ extern "C" kvq_status_t kvq_decode_static(kvq_plan_t *plan, const uint8_t *packe
     if (!plan || N < 0) return KVQ_ERR_INVALID_ARG;
     if (dtype != KVQ_F16 && dtype != KVQ_BF16) return KVQ_ERR_INVALID_ARG;
     if (plan->D > kStaticMaxD) return KVQ_ERR_SCRATCH_LIMIT;                 // the table would not fit the block
-    if (plan->D != 128 || dtype != KVQ_F16 || plan->group != 32 || plan->bits != 4)
-        return KVQ_ERR_UNSUPPORTED_DIM;   // the kernel behind it: D = 128, fp16, groups of 32, 4-bit codes
+    if (plan->D != 128 || dtype != KVQ_F16 || plan->group != 32 || plan->bits != 4 || plan->rot)
+        return KVQ_ERR_UNSUPPORTED_DIM;   // the kernel behind it: D = 128, fp16, groups of 32, 4-bit codes, no rotation
     if (N == 0) return KVQ_OK;
     if (!packed || !scales || !out || !lambda || n_lambda < 1) return KVQ_ERR_INVALID_ARG;
     if (n_lambda > 1) {

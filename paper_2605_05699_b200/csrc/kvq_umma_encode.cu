@@ -81,11 +81,11 @@ struct Ctrl {
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
 
-// 2^k for a lambda row: the power of two that brings max_c lambda_c sqrt(2 / D) into [2^13, 2^14), so that
+// 2^k for a lambda row: the power of two that brings max_c lambda_c max|table entry| (sqrt(2 / D) without a rotation) into [2^13, 2^14), so that
 // the first split term of W 2^k stays below fp16's maximum and the later ones above its subnormals.
 // Every lane of the warp gets the same value.
 template <int D>
-__device__ __forceinline__ float lift_of(const float *__restrict__ lam, int lane)
+__device__ __forceinline__ float lift_of(const float *__restrict__ lam, float table_max, int lane)
 {
     float mx = lam ? 0.0f : 1.0f;   // no lambda row (calibration): lambda = 1
 #pragma unroll
@@ -98,8 +98,7 @@ __device__ __forceinline__ float lift_of(const float *__restrict__ lam, int lane
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
-    constexpr float kRowScale = (float)ct_sqrt(2.0 / (double)D);        // largest entry of M
-    mx = fminf(fmaxf(mx * kRowScale, 1e-30f), 1e30f);
+    mx = fminf(fmaxf(mx * table_max, 1e-30f), 1e30f);   // table_max: largest |entry| of the table
     const int e = (int)((__float_as_uint(mx) >> 23) & 0xFFu) - 127;      // floor(log2 mx)
     return __uint_as_float((uint32_t)(127 + 13 - e) << 23);
 }
@@ -149,6 +148,7 @@ struct UmmaEncodeParams {
     int64_t rpl;           // rows per lambda segment (N when there is one lambda row)
     int64_t n_seg;
     RowMap out_map;        // output row of input row r
+    float table_max;       // largest |entry| of e0
     uint32_t *status;
     uint32_t *amax_bits;        // calibration only: [D] running column maxima as fp32 bit patterns (start at zero)
 };
@@ -287,7 +287,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         if (n_my > 0) {   // B for the CTA's first lambda row: D / 16 rows per warp, all sixteen warps
             TileCursor first(tile_begin, tps);
             const float *lam = CALIB ? nullptr : prm.lambda + (prm.n_lambda == 1 ? 0 : first.seg) * D;
-            const float lift = lift_of<D>(lam, lane);
+            const float lift = lift_of<D>(lam, prm.table_max, lane);
             build_b_rows<D, BF16>(sB, prm.e0, lam, lift, (warp - 2) * (D / 16), (warp - 1) * (D / 16), lane);
             fence_proxy_async();   // B is read by the tensor core through the async proxy
             __syncwarp();
@@ -307,7 +307,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             // ---- tells the mma warp.
             if (seg != cached_seg) {
                 const float *lam = CALIB ? nullptr : prm.lambda + (prm.n_lambda == 1 ? 0 : seg) * D;
-                const float lift = lift_of<D>(lam, lane);
+                const float lift = lift_of<D>(lam, prm.table_max, lane);
                 if (j > 0 && cur.first_of_segment()) {
                     if (!wait_or_abort(smem_u32(&ctrl->acc_full[(j - 1) % kAccStages]), (uint32_t)((j - 1) / kAccStages) & 1u,
                                        abort_flag, status, KVQ_DEV_MMA_TIMEOUT))
@@ -433,6 +433,7 @@ cudaError_t launch(int64_t N, const FftParams &f, const float *e0, cudaStream_t 
     prm.rpl = f.n_lambda == 1 ? N : f.rows_per_lambda;
     prm.n_seg = (N + prm.rpl - 1) / prm.rpl;
     prm.out_map = f.out_map;
+    prm.table_max = f.table_max;
     prm.status = f.status;
     prm.amax_bits = amax_bits;
 

@@ -99,6 +99,20 @@ def make_lambda(n_rows: int, D: int, seed: int, device="cpu") -> torch.Tensor:
     return 0.5 + 1.5 * torch.rand(n_rows, D, generator=g, device=device, dtype=torch.float32)
 
 
+def make_rotation(D: int, seed: int, near_identity: float = 0.0) -> torch.Tensor:
+    """A seeded orthogonal matrix, host fp32 ``[D, D]``: the stand-in for a learned rotation (no trained one exists
+    here).  ``near_identity`` = 0 gives a Haar-like draw (QR of a Gaussian matrix, column signs fixed); a value t > 0
+    gives exp(t (U - U^T)) for Gaussian U, the near-identity shape a short training run starts from and stays close to."""
+    g = _gen(seed, "cpu")
+    u = torch.randn(D, D, generator=g, dtype=torch.float64)
+    if near_identity > 0.0:
+        q = torch.linalg.matrix_exp(near_identity * (u - u.T))
+    else:
+        q, r = torch.linalg.qr(u)
+        q = q * torch.sign(torch.diagonal(r))
+    return q.to(torch.float32).contiguous()
+
+
 def raw_bits(x: torch.Tensor):
     """Host uint16 bit patterns of a half-precision tensor (what the oracle consumes)."""
     return x.detach().cpu().contiguous().view(torch.int16).numpy().view("uint16")

@@ -468,6 +468,88 @@ def test_base_variants_append_and_flush_and_refusals():
         kb.Plan(128, 32, 1, bits=6)
 
 
+# ---- rotation between the transform and lambda, folded into the tensor-core kernels' tables ---------------
+
+@pytest.mark.parametrize("D,dtype,near", [
+    (64, "f16", 0.0), (96, "f16", 0.02), (128, "f16", 0.0), (128, "f16", 0.02), (160, "f16", 0.0),
+    (256, "f16", 0.0), (256, "bf16", 0.0), (256, "bf16", 0.02),
+])
+def test_rotated_plan_matches_the_oracle(D, dtype, near):
+    N, n_lambda, rpl = 3000, 3, 1100           # ragged; lambda rows end inside tiles
+    odt = ko.F16 if dtype == "f16" else ko.BF16
+    plan = kb.Plan(D, G, 300 + D)
+    sg = plan.signs()
+    R = wl.make_rotation(D, 301, near)
+    plan.set_rotation(R)
+    Rd = R.numpy().astype(np.float64)
+    lam = wl.make_lambda(n_lambda, D, 302)
+    x = wl.make_vectors(N, D, dtype, "k_outlier", 303)
+    packed, scales = gpu_encode(plan, x.cuda(), lam.cuda(), rpl)
+    ora = ko.encode(bits(x), odt, sg, lam.numpy(), G, rpl, want_v=True, rot=Rd)
+    pk, sb = packed.cpu().numpy(), bits(scales)
+    parity.check_encode(pk, sb, ora, G, "rotated encode")
+    out = gpu_decode(plan, packed, scales, lam.cuda(), dtype, rpl)
+    ob, o64 = ko.decode(pk, sb, sg, lam.numpy(), G, odt, rpl, want_f64=True, rot=Rd)
+    parity.check_decode(bits(out), ob, o64, odt, "rotated decode")
+    # the rotation matters: without it the oracle gives other codes
+    assert (ko.encode(bits(x[:64]), odt, sg, lam.numpy()[:1], G)["codes"] != ora["codes"][:64]).mean() > 0.2
+    plan.close()
+
+
+def test_rotation_can_be_set_and_removed_on_a_plan_in_use():
+    D, N = 128, 2048
+    plan = kb.Plan(D, G, 5)
+    sg = plan.signs()
+    lam = wl.make_lambda(1, D, 6)
+    x = wl.make_vectors(N, D, "f16", "gaussian", 7)
+    xd, lamd = x.cuda(), lam.cuda()
+    base = [t.clone() for t in gpu_encode(plan, xd, lamd)]            # first use: the device tables now exist
+    R = wl.make_rotation(D, 8)
+    plan.set_rotation(R)                                               # rewrites them in place
+    packed, scales = gpu_encode(plan, xd, lamd)                        # small call: still the tensor-core path
+    ora = ko.encode(bits(x), ko.F16, sg, lam.numpy(), G, want_v=True, rot=R.numpy().astype(np.float64))
+    parity.check_encode(packed.cpu().numpy(), bits(scales), ora, G, "rotation set after first use")
+    # append on a rotated plan
+    pc = torch.zeros(N, 4, D // 2, dtype=torch.uint8, device="cuda")
+    sc = torch.zeros(N, 4, D // G, dtype=torch.float16, device="cuda")
+    kb.kvq_append(plan.handle, xd, lamd, pc, sc, 2, 0)
+    torch.cuda.synchronize()
+    parity.check_encode(pc[:, 2].contiguous().cpu().numpy(), bits(sc[:, 2].contiguous()), ora, G, "rotated append")
+    assert bool((pc[:, [0, 1, 3]] == 0).all())
+    # calibration sees the rotated coordinates
+    lam_cal = torch.empty(D, dtype=torch.float32, device="cuda")
+    kb.kvq_calibrate_lambda(plan.handle, xd, lam_cal)
+    torch.cuda.synchronize()
+    v1 = ko.encode(bits(x), ko.F16, sg, np.ones(D, np.float32), G, want_v=True, rot=R.numpy().astype(np.float64))["v"]
+    amax = np.abs(v1).max(axis=0)
+    assert np.abs(1.0 / lam_cal.cpu().numpy().astype(np.float64) - amax).max() <= 2e-6 * np.linalg.norm(v1, axis=1).max()
+    # what a rotated plan refuses
+    dq = torch.zeros(N, 4, D, dtype=torch.float16, device="cuda")
+    with pytest.raises(kb.KvqError):
+        kb.kvq_flush_block(plan.handle, xd.view(N, 1, D), lamd, pc, sc, dq, 0, 0)
+    kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_FFT, kb.KVQ_IMPL_FFT)
+    with pytest.raises(kb.KvqError):
+        gpu_encode(plan, xd, lamd)
+    with pytest.raises(kb.KvqError):
+        kb.kvq_decode(plan.handle, packed, scales, lamd, torch.empty(N, D, dtype=torch.float16, device="cuda"), 0)
+    kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_AUTO, kb.KVQ_IMPL_AUTO)
+    # and removed again: the plan is what it was
+    plan.set_rotation(None)
+    again = gpu_encode(plan, xd, lamd)
+    assert torch.equal(again[0], base[0]) and torch.equal(again[1], base[1])
+    plan.close()
+    # plans the tensor-core kernels do not serve take no rotation
+    for p in (kb.Plan(128, 128, 1), kb.Plan(128, 32, 1, bits=8)):
+        with pytest.raises(kb.KvqError):
+            p.set_rotation(R)
+        p.close()
+    p = kb.Plan(160, G, 1)
+    p.set_rotation(wl.make_rotation(160, 9))
+    with pytest.raises(kb.KvqError):       # bf16 at D = 160 has no tensor-core kernel, and a rotated plan has no other
+        gpu_encode(p, wl.make_vectors(64, 160, "bf16", "gaussian", 1).cuda(), wl.make_lambda(1, 160, 2).cuda())
+    p.close()
+
+
 # ---- config 3: Gemma-3-1B-shaped, D = 256 bf16, prefix sweep ---------------------------------
 
 @pytest.mark.parametrize("prefix", [256, 1024])

@@ -6,10 +6,12 @@ import re
 
 import numpy as np
 import pytest
+import torch
 
 from oracle import kvq_oracle as ko
 from paper_2605_05699_b200 import binding as kb
 from paper_2605_05699_b200 import build as kbuild
+from paper_2605_05699_b200 import workloads as wl
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
@@ -62,6 +64,29 @@ def test_unsupported_dims_and_groups_are_rejected():
     for D, g, b in [(128, 32, 5), (128, 32, 16), (128, 32, 0), (128, 64, 8), (96, 128, 4)]:
         assert L.kvq_plan_create_ex(D, g, b, 1, ctypes.byref(h)) == kb.KVQ_ERR_UNSUPPORTED_DIM
         assert h.value is None
+
+
+def test_rotation_is_validated_on_the_host():
+    p = kb.Plan(128, 32, 1)
+    R = wl.make_rotation(128, 3)
+    assert torch.allclose(R @ R.T, torch.eye(128), atol=1e-5)
+    p.set_rotation(R)            # before any GPU use: kept on the host until the tables are built
+    p.set_rotation(None)
+    bad = R.clone()
+    bad[5, 7] = float("nan")
+    with pytest.raises(kb.KvqError) as e:
+        p.set_rotation(bad)
+    assert e.value.status == kb.KVQ_ERR_INVALID_ARG
+    with pytest.raises(ValueError):
+        p.set_rotation(R[:64, :64])
+    p.close()
+    for q in (kb.Plan(128, 128, 1), kb.Plan(128, 32, 1, bits=8)):
+        with pytest.raises(kb.KvqError) as e:
+            q.set_rotation(R)
+        assert e.value.status == kb.KVQ_ERR_UNSUPPORTED_DIM
+        q.close()
+    near = wl.make_rotation(64, 4, near_identity=0.02)
+    assert torch.allclose(near @ near.T, torch.eye(64), atol=1e-5) and float((near - torch.eye(64)).abs().max()) < 0.5
 
 
 def test_bad_arguments_are_rejected_on_the_host():
