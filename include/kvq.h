@@ -51,15 +51,17 @@ typedef enum {
 
 typedef enum { KVQ_F16 = 0, KVQ_BF16 = 1 } kvq_dtype_t;
 
-/* Which kernel family serves a call.  AUTO picks the fastest one that meets the
- * tolerances for the plan's D and the call's dtype: the tensor-core kernel where one is
- * built (for kvq_encode / kvq_append only on calls of at least 4096 rows), else the FFT. */
+/* Which kernel family serves a call.  AUTO picks by size and shape: the matrix-vector kernel for calls of up to
+ * 2048 rows (1024 for D > 128; such calls are latency-bound), beyond that the tensor-core kernel where one is built for the plan's D and
+ * layout and the call's dtype (for kvq_encode / kvq_append from 4096 rows on), else the register FFT. */
 typedef enum {
     KVQ_IMPL_AUTO = 0,
-    KVQ_IMPL_FFT = 1, /* fp32 register FFT, one thread per vector: every D and dtype */
-    KVQ_IMPL_GEMM = 2 /* tcgen05 DFT-as-GEMM.  encode / append: fp16 for D = 64, 96, 128, 160, 256, bf16 for
-                         D = 64, 96, 128, 256; decode: fp16 for the same D, bf16 for D = 256.  Elsewhere the
-                         compute calls return KVQ_ERR_UNSUPPORTED_DIM. */
+    KVQ_IMPL_FFT = 1,   /* fp32 register FFT, one thread per vector: every D, dtype and layout; no rotation */
+    KVQ_IMPL_GEMM = 2,  /* tcgen05 DFT-as-GEMM, group = 32 and bits = 4 only.  encode / append: fp16 for D = 64, 96, 128,
+                           160, 256, bf16 for D = 64, 96, 128, 256; decode: fp16 for the same D, bf16 for D = 256.
+                           Elsewhere the compute calls return KVQ_ERR_UNSUPPORTED_DIM. */
+    KVQ_IMPL_MATVEC = 3 /* fp32 matrix-vector product with the plan's D x D table, a CTA per 8 vectors: every D, dtype
+                           and layout, rotated plans included; meant for small calls, correct (and slow) at any size */
 } kvq_impl_t;
 
 /*
@@ -83,7 +85,8 @@ kvq_status_t kvq_plan_create(int D, int group, uint64_t seed, kvq_plan_t **out);
  *          two's-complement byte per value: `packed` rows are D bytes).
  * Everything else is as for kvq_plan_create, which is (group, bits = 4).  Wherever a comment of this header says
  * "[*, D/2] bytes" a plan with bits = 8 takes [*, D] bytes.  The tensor-core kernels serve group = 32, bits = 4 only:
- * other plans run on the register-FFT kernels (KVQ_IMPL_GEMM is refused with UNSUPPORTED_DIM, kvq_decode_static too).
+ * other plans run on the register-FFT and matrix-vector kernels (KVQ_IMPL_GEMM is refused with UNSUPPORTED_DIM,
+ * kvq_decode_static too).
  */
 kvq_status_t kvq_plan_create_ex(int D, int group, int bits, uint64_t seed, kvq_plan_t **out);
 
@@ -92,14 +95,15 @@ kvq_status_t kvq_plan_create_ex(int D, int group, int bits, uint64_t seed, kvq_p
  * transform and lambda, v = lambda (.) (R z) on the way in and z^ = R^T (v^ / max(lambda, 1e-6)) on the way out.
  *   R_host   HOST pointer, [D, D] row-major fp32, copied by the call; NULL removes the rotation.  The library does not
  *            check that R is orthogonal: the inverse path applies R^T.  Training R is the caller's business.
- * The rotation is folded into the D x D tables of the tensor-core kernels, so it costs nothing per vector, and it
- * exists only where those kernels do: group = 32, bits = 4; kvq_encode / kvq_append / kvq_calibrate_lambda for the
- * (D, dtype) pairs KVQ_IMPL_GEMM lists for encode, kvq_decode for those it lists for decode (D = 256 then runs a
- * dense 256 x 256 kernel).  On a rotated plan every call takes the tensor-core path whatever its size;
- * KVQ_IMPL_FFT, kvq_flush_block, kvq_decode_static and unsupported (D, dtype) pairs return UNSUPPORTED_DIM.
+ * The rotation is folded into the plan's D x D tables, so it costs nothing per vector in the kernels that contract
+ * with those tables: the tensor-core kernels (KVQ_IMPL_GEMM; D = 256 decode then runs a dense 256 x 256 kernel) and
+ * the matrix-vector kernels (KVQ_IMPL_MATVEC).  A rotated plan never takes the register FFT: AUTO uses the
+ * tensor-core kernel where KVQ_IMPL_GEMM lists one for the call and the matrix-vector kernel everywhere else (every
+ * layout and dtype works, large calls outside the GEMM list are slow); KVQ_IMPL_FFT and kvq_decode_static return
+ * UNSUPPORTED_DIM.
  * If the plan's device tables already exist they are rewritten after a device synchronisation: call it with the
  * plan's device current and no call using the plan in flight on another thread.
- * Errors: INVALID_ARG (null plan, non-finite entry, wrong device), UNSUPPORTED_DIM, NOMEM, CUDA.
+ * Errors: INVALID_ARG (null plan, non-finite entry, wrong device), NOMEM, CUDA.
  */
 kvq_status_t kvq_plan_set_rotation(kvq_plan_t *plan, const float *R_host /* [D, D] or NULL */);
 
@@ -173,7 +177,8 @@ kvq_status_t kvq_append(kvq_plan_t *plan, const void *x_new /* [S, D] */, kvq_dt
  *   x_block       device, [S, rows, D] row-major, fp16 or bf16 per `dtype`; 16-byte aligned.
  *   lambda, n_lambda, streams_per_lambda, packed_cache [S, T_max, D/2], scales_cache [S, T_max, D/group]: as in kvq_append.
  *   dq_cache      device out, [S, T_max, D] of the same 16-bit type; 16-byte aligned.  Only rows [pos0, pos0 + rows) are written.
- * Requires 0 <= pos0 and pos0 + rows <= T_max.  S == 0 or rows == 0 is a no-op.  Two launches on the stream.  The
+ * Requires 0 <= pos0 and pos0 + rows <= T_max.  S == 0 or rows == 0 is a no-op.  Two launches on the stream (the
+ * matrix-vector kernels when S * rows <= 2048 (1024 for D > 128) or the plan is rotated).  The
  * window itself (holding the not yet flushed tokens in fp16) is the caller's buffer: this call is its flush.
  */
 kvq_status_t kvq_flush_block(kvq_plan_t *plan, const void *x_block, kvq_dtype_t dtype, int64_t S, int64_t rows,

@@ -33,6 +33,7 @@ KVQ_BF16 = 1
 KVQ_IMPL_AUTO = 0
 KVQ_IMPL_FFT = 1
 KVQ_IMPL_GEMM = 2
+KVQ_IMPL_MATVEC = 3
 
 # every symbol include/kvq.h declares
 EXPORTS = (

@@ -25,6 +25,8 @@ static inline uint64_t splitmix64_at(uint64_t seed, uint64_t n)
 
 // AUTO sends kvq_encode / kvq_append calls of at least this many rows to the tensor-core kernel.
 constexpr int64_t kGemmEncodeMinRows = 4096;
+// calls up to this size are latency-bound: matrix-vector kernel (measured cross-over with the other two families)
+static int64_t matvec_max_rows(int D) { return D <= 128 ? 2048 : 1024; }
 
 static bool dim_supported(int D) { return D == 64 || D == 96 || D == 128 || D == 160 || D == 256; }
 
@@ -233,8 +235,6 @@ kvq_status_t kvq_plan_destroy(kvq_plan_t *plan)
 kvq_status_t kvq_plan_set_rotation(kvq_plan_t *plan, const float *R_host)
 {
     if (!plan) return KVQ_ERR_INVALID_ARG;
-    // the rotation lives in the tensor-core kernels' tables: the plan must be one they serve
-    if (R_host && (!gemm_layout(plan) || !umma_encode_supported(plan->D, false))) return KVQ_ERR_UNSUPPORTED_DIM;
     std::lock_guard<std::mutex> lk(plan->mu);
     const size_t n = (size_t)plan->D * plan->D;
     double *rot = nullptr;
@@ -294,7 +294,7 @@ kvq_status_t kvq_plan_describe(const kvq_plan_t *plan, int *radices, int *n_radi
 kvq_status_t kvq_plan_set_impl(kvq_plan_t *plan, kvq_impl_t encode_impl, kvq_impl_t decode_impl)
 {
     if (!plan) return KVQ_ERR_INVALID_ARG;
-    if ((int)encode_impl < 0 || (int)encode_impl > 2 || (int)decode_impl < 0 || (int)decode_impl > 2)
+    if ((int)encode_impl < 0 || (int)encode_impl > 3 || (int)decode_impl < 0 || (int)decode_impl > 3)
         return KVQ_ERR_INVALID_ARG;
     plan->enc_impl = encode_impl;
     plan->dec_impl = decode_impl;
@@ -328,9 +328,10 @@ static kvq_status_t encode_common(kvq_plan_t *plan, const void *x, kvq_dtype_t d
     kvq_status_t st = check_lambda(N, lambda, n_lambda, rows_per_lambda);
     if (st != KVQ_OK) return st;
     if (misaligned16(x) || misaligned16(packed) || misaligned16(scales)) return KVQ_ERR_ALIGNMENT;
-    const bool gemm_ok = gemm_layout(plan) && umma_encode_supported(plan->D, dtype == KVQ_BF16);
+    const bool bf16 = dtype == KVQ_BF16;
+    const bool gemm_ok = gemm_layout(plan) && umma_encode_supported(plan->D, bf16);
     if (plan->enc_impl == KVQ_IMPL_GEMM && !gemm_ok) return KVQ_ERR_UNSUPPORTED_DIM;
-    if (plan->rot && (!gemm_ok || plan->enc_impl == KVQ_IMPL_FFT)) return KVQ_ERR_UNSUPPORTED_DIM;   // the rotation is in the GEMM tables
+    if (plan->rot && plan->enc_impl == KVQ_IMPL_FFT) return KVQ_ERR_UNSUPPORTED_DIM;   // the rotation lives in the D x D tables
     if ((st = ensure_device(plan)) != KVQ_OK) return st;
     FftParams prm;
     fill_params(plan, prm, N, lambda, n_lambda, rows_per_lambda);
@@ -338,10 +339,20 @@ static kvq_status_t encode_common(kvq_plan_t *plan, const void *x, kvq_dtype_t d
     prm.packed = packed;
     prm.scales = scales;
     prm.out_map = out_map;
-    // the tensor-core kernel pays a fixed set-up per launch (B operand build); small calls stay on the register FFT
-    const bool use_gemm = gemm_ok && (plan->rot || plan->enc_impl == KVQ_IMPL_GEMM || (plan->enc_impl == KVQ_IMPL_AUTO && N >= kGemmEncodeMinRows));
-    cudaError_t e = use_gemm ? umma_encode(plan->D, dtype == KVQ_BF16, N, prm, plan->d_e0, static_cast<cudaStream_t>(cuda_stream))
-                             : fft_encode(plan->D, plan->group, plan->bits, dtype == KVQ_BF16, N, prm, static_cast<cudaStream_t>(cuda_stream));
+    // AUTO: the matrix-vector kernel for small calls (latency), the tensor-core kernel from kGemmEncodeMinRows rows on
+    // (it pays a fixed operand build per launch), the register FFT in between and where no tensor-core kernel is built.
+    // A rotated plan has no FFT path: matrix-vector wherever the tensor-core kernel does not apply.
+    kvq_impl_t impl = plan->enc_impl;
+    if (impl == KVQ_IMPL_AUTO) {
+        if (N <= matvec_max_rows(plan->D)) impl = KVQ_IMPL_MATVEC;
+        else if (gemm_ok && (plan->rot || N >= kGemmEncodeMinRows)) impl = KVQ_IMPL_GEMM;
+        else impl = plan->rot ? KVQ_IMPL_MATVEC : KVQ_IMPL_FFT;
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e;
+    if (impl == KVQ_IMPL_GEMM) e = umma_encode(plan->D, bf16, N, prm, plan->d_e0, stream);
+    else if (impl == KVQ_IMPL_MATVEC) e = matvec_encode(plan->D, plan->group, plan->bits, bf16, N, prm, plan->d_b0, stream);
+    else e = fft_encode(plan->D, plan->group, plan->bits, bf16, N, prm, stream);
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
         return KVQ_ERR_CUDA;
@@ -374,11 +385,19 @@ kvq_status_t kvq_decode(kvq_plan_t *plan, const uint8_t *packed, const void *sca
     kvq_status_t st = check_lambda(N, lambda, n_lambda, rows_per_lambda);
     if (st != KVQ_OK) return st;
     if (misaligned16(packed) || misaligned16(scales) || misaligned16(out)) return KVQ_ERR_ALIGNMENT;
-    const bool gemm_ok = gemm_layout(plan) && umma_decode_supported(plan->D, dtype == KVQ_BF16);
+    const bool bf16 = dtype == KVQ_BF16;
+    const bool gemm_ok = gemm_layout(plan) && umma_decode_supported(plan->D, bf16);
     if (plan->dec_impl == KVQ_IMPL_GEMM && !gemm_ok) return KVQ_ERR_UNSUPPORTED_DIM;
-    if (plan->rot && (!gemm_ok || plan->dec_impl == KVQ_IMPL_FFT)) return KVQ_ERR_UNSUPPORTED_DIM;   // the rotation is in the GEMM tables
+    if (plan->rot && plan->dec_impl == KVQ_IMPL_FFT) return KVQ_ERR_UNSUPPORTED_DIM;   // the rotation lives in the D x D tables
     if ((st = ensure_device(plan)) != KVQ_OK) return st;
-    if (gemm_ok && plan->dec_impl != KVQ_IMPL_FFT) {
+    kvq_impl_t impl = plan->dec_impl;
+    if (impl == KVQ_IMPL_AUTO) {
+        if (N <= matvec_max_rows(plan->D)) impl = KVQ_IMPL_MATVEC;
+        else if (gemm_ok) impl = KVQ_IMPL_GEMM;
+        else impl = plan->rot ? KVQ_IMPL_MATVEC : KVQ_IMPL_FFT;
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (impl == KVQ_IMPL_GEMM) {
         GemmParams g;
         g.packed = packed;
         g.scales = scales;
@@ -390,9 +409,8 @@ kvq_status_t kvq_decode(kvq_plan_t *plan, const uint8_t *packed, const void *sca
         g.rows_per_lambda = rows_per_lambda < 1 ? 1 : rows_per_lambda;
         g.status = plan->d_status;
         // D = 256: the radix-2 kernel needs the transform's even / odd structure, which a rotation destroys
-        const cudaError_t e = plan->rot && plan->D == 256
-                                  ? umma_decode_d256_dense(dtype == KVQ_BF16, N, g, static_cast<cudaStream_t>(cuda_stream))
-                                  : umma_decode(plan->D, dtype == KVQ_BF16, N, g, plan->sign_xor, static_cast<cudaStream_t>(cuda_stream));
+        const cudaError_t e = plan->rot && plan->D == 256 ? umma_decode_d256_dense(bf16, N, g, stream)
+                                                          : umma_decode(plan->D, bf16, N, g, plan->sign_xor, stream);
         if (e != cudaSuccess) {
             (void)cudaGetLastError();
             return KVQ_ERR_CUDA;
@@ -404,7 +422,8 @@ kvq_status_t kvq_decode(kvq_plan_t *plan, const uint8_t *packed, const void *sca
     prm.packed = const_cast<uint8_t *>(packed);
     prm.scales = const_cast<void *>(scales);
     prm.out = out;
-    cudaError_t e = fft_decode(plan->D, plan->group, plan->bits, dtype == KVQ_BF16, N, prm, static_cast<cudaStream_t>(cuda_stream));
+    const cudaError_t e = impl == KVQ_IMPL_MATVEC ? matvec_decode(plan->D, plan->group, plan->bits, bf16, N, prm, plan->d_e0, stream)
+                                                  : fft_decode(plan->D, plan->group, plan->bits, bf16, N, prm, stream);
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
         return KVQ_ERR_CUDA;
@@ -421,7 +440,6 @@ kvq_status_t kvq_flush_block(kvq_plan_t *plan, const void *x_block, kvq_dtype_t 
     if (dtype != KVQ_F16 && dtype != KVQ_BF16) return KVQ_ERR_INVALID_ARG;
     if (S == 0 || rows == 0) return KVQ_OK;
     if (!dq_cache) return KVQ_ERR_INVALID_ARG;
-    if (plan->rot) return KVQ_ERR_UNSUPPORTED_DIM;   // its decode half runs on the register FFT, which has no rotation
     if (misaligned16(dq_cache)) return KVQ_ERR_ALIGNMENT;
     if (S > INT64_MAX / rows) return KVQ_ERR_INVALID_ARG;
     const int64_t N = S * rows;
@@ -438,7 +456,13 @@ kvq_status_t kvq_flush_block(kvq_plan_t *plan, const void *x_block, kvq_dtype_t 
     prm.out = dq_cache;
     prm.in_map = map;
     prm.out_map = map;
-    if (fft_decode(plan->D, plan->group, plan->bits, dtype == KVQ_BF16, N, prm, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
+    // small blocks (the window flush) and rotated plans: matrix-vector kernel; large plain blocks: register FFT
+    if (plan->rot && plan->dec_impl == KVQ_IMPL_FFT) return KVQ_ERR_UNSUPPORTED_DIM;
+    const bool mv = plan->rot || plan->dec_impl == KVQ_IMPL_MATVEC || (plan->dec_impl != KVQ_IMPL_FFT && N <= matvec_max_rows(plan->D));
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const cudaError_t e = mv ? matvec_decode(plan->D, plan->group, plan->bits, dtype == KVQ_BF16, N, prm, plan->d_e0, stream)
+                             : fft_decode(plan->D, plan->group, plan->bits, dtype == KVQ_BF16, N, prm, stream);
+    if (e != cudaSuccess) {
         (void)cudaGetLastError();
         return KVQ_ERR_CUDA;
     }

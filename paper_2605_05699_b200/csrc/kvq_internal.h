@@ -64,6 +64,9 @@ cudaError_t umma_decode_d256(bool bf16, int64_t N, const GemmParams &prm, const 
 cudaError_t umma_decode_d256_dense(bool bf16, int64_t N, const GemmParams &prm, cudaStream_t stream);   // kvq_umma_decode256_dense.cu: any table
 cudaError_t umma_encode(int D, bool bf16, int64_t N, const FftParams &prm, const float *e0, cudaStream_t stream);
 
+// fp32 matrix-vector kernels for small calls (kvq_matvec.cu): every layout, dtype and D; b0 / e0 are the plan's tables
+cudaError_t matvec_encode(int D, int group, int bits, bool bf16, int64_t N, const FftParams &prm, const float *b0, cudaStream_t stream);
+cudaError_t matvec_decode(int D, int group, int bits, bool bf16, int64_t N, const FftParams &prm, const float *e0, cudaStream_t stream);
 // group: 32 or D (one scale per vector); bits: 4 or 8
 cudaError_t fft_encode(int D, int group, int bits, bool bf16, int64_t N, const FftParams &prm, cudaStream_t stream);
 cudaError_t fft_decode(int D, int group, int bits, bool bf16, int64_t N, const FftParams &prm, cudaStream_t stream);

@@ -36,7 +36,7 @@ def gpu_decode(plan, packed, scales, lam, dtype, rows_per_lambda=0):
     return out
 
 
-IMPL = {"auto": kb.KVQ_IMPL_AUTO, "fft": kb.KVQ_IMPL_FFT, "gemm": kb.KVQ_IMPL_GEMM}
+IMPL = {"auto": kb.KVQ_IMPL_AUTO, "fft": kb.KVQ_IMPL_FFT, "gemm": kb.KVQ_IMPL_GEMM, "matvec": kb.KVQ_IMPL_MATVEC}
 
 
 def run_case(D, dtype, N, kind, seed, n_lambda=1, rows_per_lambda=0, plan_seed=None, enc_impl="auto", dec_impl="auto"):
@@ -399,6 +399,33 @@ def test_flush_block_rejects_blocks_outside_the_cache():
     plan.close()
 
 
+# ---- the matrix-vector kernels of the small calls, forced at sizes that span many CTAs and a ragged last one ------
+
+@pytest.mark.parametrize("D,dtype", [(64, "f16"), (64, "bf16"), (96, "f16"), (96, "bf16"), (128, "f16"), (128, "bf16"),
+                                     (160, "f16"), (160, "bf16"), (256, "f16"), (256, "bf16")])
+def test_matvec_kernels_all_dims(D, dtype):
+    run_case(D, dtype, 2051, "k_outlier", 7000 + D, n_lambda=5, rows_per_lambda=411, enc_impl="matvec", dec_impl="matvec")
+    run_case(D, dtype, 5, "gaussian", 7100 + D, enc_impl="matvec", dec_impl="matvec")
+
+
+def test_small_calls_take_the_matvec_kernels_and_agree_with_the_fft():
+    # AUTO below 2048 rows is the matrix-vector kernel; its codes agree with the register FFT except at rounding ties
+    D, N = 128, 1500
+    plan = kb.Plan(D, G, 11)
+    x = wl.make_vectors(N, D, "f16", "k_outlier", 12).cuda()
+    lam = wl.make_lambda(1, D, 13).cuda()
+    n0 = kb.kvq_launch_count()
+    pa, sa = gpu_encode(plan, x, lam)
+    kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_MATVEC, kb.KVQ_IMPL_MATVEC)
+    pm, sm_ = gpu_encode(plan, x, lam)
+    assert torch.equal(pa, pm) and torch.equal(sa, sm_)
+    kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_FFT, kb.KVQ_IMPL_FFT)
+    pf, sf = gpu_encode(plan, x, lam)
+    assert kb.kvq_launch_count() - n0 == 3
+    assert float((pa == pf).float().mean()) > 0.999 and float((sa == sf).float().mean()) > 0.99
+    plan.close()
+
+
 # ---- base variants: one scale per vector and / or 8-bit codes (register-FFT kernels) -------------------
 
 @pytest.mark.parametrize("D,dtype,per_vector,nbits", [
@@ -408,11 +435,13 @@ def test_flush_block_rejects_blocks_outside_the_cache():
     (160, "f16", True, 8), (160, "bf16", False, 8),
     (256, "bf16", True, 4), (256, "f16", True, 8), (256, "bf16", False, 8),
 ])
-def test_base_variants_per_vector_scale_and_byte_codes(D, dtype, per_vector, nbits):
+@pytest.mark.parametrize("impl", ["fft", "matvec"])
+def test_base_variants_per_vector_scale_and_byte_codes(D, dtype, per_vector, nbits, impl):
     N, n_lambda, rpl = 5003, 3, 1700          # ragged, lambda rows straddle the warps' tiles
     group = D if per_vector else G
     odt = ko.F16 if dtype == "f16" else ko.BF16
     plan = kb.Plan(D, group, 90 + D, bits=nbits)
+    kb.kvq_plan_set_impl(plan.handle, IMPL[impl], IMPL[impl])
     sg = plan.signs()
     lam = wl.make_lambda(n_lambda, D, 91)
     x = wl.make_vectors(N, D, dtype, "k_outlier", 92 + nbits)
@@ -523,10 +552,15 @@ def test_rotation_can_be_set_and_removed_on_a_plan_in_use():
     v1 = ko.encode(bits(x), ko.F16, sg, np.ones(D, np.float32), G, want_v=True, rot=R.numpy().astype(np.float64))["v"]
     amax = np.abs(v1).max(axis=0)
     assert np.abs(1.0 / lam_cal.cpu().numpy().astype(np.float64) - amax).max() <= 2e-6 * np.linalg.norm(v1, axis=1).max()
-    # what a rotated plan refuses
+    # the window flush of a rotated plan (matrix-vector kernels)
     dq = torch.zeros(N, 4, D, dtype=torch.float16, device="cuda")
-    with pytest.raises(kb.KvqError):
-        kb.kvq_flush_block(plan.handle, xd.view(N, 1, D), lamd, pc, sc, dq, 0, 0)
+    kb.kvq_flush_block(plan.handle, xd.view(N, 1, D), lamd, pc, sc, dq, 1, 0)
+    torch.cuda.synchronize()
+    pk1, sb1 = pc[:, 1].contiguous().cpu().numpy(), bits(sc[:, 1].contiguous())
+    parity.check_encode(pk1, sb1, ora, G, "rotated flush")
+    ob, o64 = ko.decode(pk1, sb1, sg, lam.numpy(), G, ko.F16, want_f64=True, rot=R.numpy().astype(np.float64))
+    parity.check_decode(bits(dq[:, 1].contiguous()), ob, o64, ko.F16, "rotated flush, dequantized rows")
+    # what a rotated plan refuses: the register FFT
     kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_FFT, kb.KVQ_IMPL_FFT)
     with pytest.raises(kb.KvqError):
         gpu_encode(plan, xd, lamd)
@@ -538,16 +572,22 @@ def test_rotation_can_be_set_and_removed_on_a_plan_in_use():
     again = gpu_encode(plan, xd, lamd)
     assert torch.equal(again[0], base[0]) and torch.equal(again[1], base[1])
     plan.close()
-    # plans the tensor-core kernels do not serve take no rotation
-    for p in (kb.Plan(128, 128, 1), kb.Plan(128, 32, 1, bits=8)):
-        with pytest.raises(kb.KvqError):
-            p.set_rotation(R)
+    # layouts and dtypes without a tensor-core kernel: a rotated plan runs them on the matrix-vector kernels
+    for Dv, dtv, grp, nb in [(128, "f16", 128, 4), (128, "f16", 32, 8), (160, "bf16", 32, 4)]:
+        p = kb.Plan(Dv, grp, 1, bits=nb)
+        Rv = wl.make_rotation(Dv, 9)
+        p.set_rotation(Rv)
+        xv = wl.make_vectors(5000, Dv, dtv, "gaussian", 1)
+        lv = wl.make_lambda(1, Dv, 2)
+        odt = ko.F16 if dtv == "f16" else ko.BF16
+        pkv, scv = gpu_encode(p, xv.cuda(), lv.cuda())
+        orv = ko.encode(bits(xv), odt, p.signs(), lv.numpy(), grp, want_v=True, bits=nb, rot=Rv.numpy().astype(np.float64))
+        parity.check_encode(pkv.cpu().numpy(), bits(scv), orv, grp, "rotated, no tensor-core kernel", bits=nb)
+        outv = gpu_decode(p, pkv, scv, lv.cuda(), dtv)
+        obv, o64v = ko.decode(pkv.cpu().numpy(), bits(scv), p.signs(), lv.numpy(), grp, odt, want_f64=True, bits=nb,
+                              rot=Rv.numpy().astype(np.float64))
+        parity.check_decode(bits(outv), obv, o64v, odt, "rotated, no tensor-core kernel")
         p.close()
-    p = kb.Plan(160, G, 1)
-    p.set_rotation(wl.make_rotation(160, 9))
-    with pytest.raises(kb.KvqError):       # bf16 at D = 160 has no tensor-core kernel, and a rotated plan has no other
-        gpu_encode(p, wl.make_vectors(64, 160, "bf16", "gaussian", 1).cuda(), wl.make_lambda(1, 160, 2).cuda())
-    p.close()
 
 
 # ---- config 3: Gemma-3-1B-shaped, D = 256 bf16, prefix sweep ---------------------------------

@@ -80,10 +80,8 @@ def test_rotation_is_validated_on_the_host():
     with pytest.raises(ValueError):
         p.set_rotation(R[:64, :64])
     p.close()
-    for q in (kb.Plan(128, 128, 1), kb.Plan(128, 32, 1, bits=8)):
-        with pytest.raises(kb.KvqError) as e:
-            q.set_rotation(R)
-        assert e.value.status == kb.KVQ_ERR_UNSUPPORTED_DIM
+    for q in (kb.Plan(128, 128, 1), kb.Plan(128, 32, 1, bits=8)):    # every layout takes a rotation
+        q.set_rotation(R)
         q.close()
     near = wl.make_rotation(64, 4, near_identity=0.02)
     assert torch.allclose(near @ near.T, torch.eye(64), atol=1e-5) and float((near - torch.eye(64)).abs().max()) < 0.5
