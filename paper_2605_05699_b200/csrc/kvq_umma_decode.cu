@@ -126,32 +126,63 @@ struct RecipLambda {
 // rows), scales them, trades two values with its neighbour so that each lane holds two K-ordered pairs, and
 // writes 8 bytes of the swizzled row.
 template <int D>
+__device__ __forceinline__ void build_b_quad(unsigned char *sB, float4 m, const RecipLambda<D> &rl, int n, int p, int lane)
+{
+    const bool odd = lane & 1;
+    const int i = lane + 32 * p;
+    const bool live = i < D / 4;
+    auto sat = [](float v) { return fminf(fmaxf(v, -65504.0f), 65504.0f); };
+    const float vx = sat(m.x * rl.r[p].x), vy = sat(m.y * rl.r[p].y), vz = sat(m.z * rl.r[p].z), vw = sat(m.w * rl.r[p].w);
+    // even lane holds codes 8w .. 8w+3, odd lane 8w+4 .. 8w+7; K order of the word is (0,4,1,5,2,6,3,7)
+    const float r0 = __shfl_xor_sync(0xFFFFFFFFu, odd ? vx : vz, 1);
+    const float r1 = __shfl_xor_sync(0xFFFFFFFFu, odd ? vy : vw, 1);
+    uint2 o;
+    o.x = odd ? narrow2<false>(r0, vz) : narrow2<false>(vx, r0);   // odd: (2, 6)   even: (0, 4)
+    o.y = odd ? narrow2<false>(r1, vw) : narrow2<false>(vy, r1);   // odd: (3, 7)   even: (1, 5)
+    const int w = i >> 1;   // word of 8 codes = 16-byte chunk w of the K-major row: K block w / 8, chunk w % 8
+    if (live) *reinterpret_cast<uint2 *>(sB + (w >> 3) * Cfg<D>::kBBlock + n * 128 + (((w & 7) ^ (n & 7)) << 4) + (odd ? 8 : 0)) = o;
+}
+
+template <int D>
 __device__ __forceinline__ void build_b_rows(unsigned char *sB, const float *__restrict__ b0, const RecipLambda<D> &rl, int n0, int n1,
                                              int lane)
 {
-    const bool odd = lane & 1;
 #pragma unroll 4
     for (int n = n0; n < n1; ++n) {
 #pragma unroll
         for (int p = 0; p < RecipLambda<D>::kPasses; ++p) {
             const int i = lane + 32 * p;
-            const bool live = i < D / 4;
             float4 m = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-            if (live) m = __ldg(reinterpret_cast<const float4 *>(b0 + (size_t)n * D) + i);
-            auto sat = [](float v) { return fminf(fmaxf(v, -65504.0f), 65504.0f); };
-            const float vx = sat(m.x * rl.r[p].x), vy = sat(m.y * rl.r[p].y), vz = sat(m.z * rl.r[p].z), vw = sat(m.w * rl.r[p].w);
-            // even lane holds codes 8w .. 8w+3, odd lane 8w+4 .. 8w+7; K order of the word is (0,4,1,5,2,6,3,7)
-            const float r0 = __shfl_xor_sync(0xFFFFFFFFu, odd ? vx : vz, 1);
-            const float r1 = __shfl_xor_sync(0xFFFFFFFFu, odd ? vy : vw, 1);
-            uint2 o;
-            o.x = odd ? narrow2<false>(r0, vz) : narrow2<false>(vx, r0);   // odd: (2, 6)   even: (0, 4)
-            o.y = odd ? narrow2<false>(r1, vw) : narrow2<false>(vy, r1);   // odd: (3, 7)   even: (1, 5)
-            const int w = i >> 1;   // word of 8 codes = 16-byte chunk w of the K-major row: K block w / 8, chunk w % 8
-            if (live)
-                *reinterpret_cast<uint2 *>(sB + (w >> 3) * Cfg<D>::kBBlock + n * 128 + (((w & 7) ^ (n & 7)) << 4) + (odd ? 8 : 0)) = o;
+            if (i < D / 4) m = __ldg(reinterpret_cast<const float4 *>(b0 + (size_t)n * D) + i);
+            build_b_quad<D>(sB, m, rl, n, p, lane);
         }
     }
 }
+
+// The first build of a CTA: its D / 16 table rows per warp are requested at kernel entry, all at once, and turned
+// into B rows here, once lambda has arrived too: one round trip to L2 instead of one per batch of rows.
+template <int D>
+struct FirstRows {
+    static constexpr int kRows = D / 16, kPasses = RecipLambda<D>::kPasses;
+    float4 m[kRows][kPasses];
+    __device__ __forceinline__ void load(const float *__restrict__ b0, int n0, int lane)
+    {
+#pragma unroll
+        for (int k = 0; k < kRows; ++k)
+#pragma unroll
+            for (int p = 0; p < kPasses; ++p) {
+                const int i = lane + 32 * p;
+                m[k][p] = i < D / 4 ? __ldg(reinterpret_cast<const float4 *>(b0 + (size_t)(n0 + k) * D) + i) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            }
+    }
+    __device__ __forceinline__ void build(unsigned char *sB, const RecipLambda<D> &rl, int n0, int lane) const
+    {
+#pragma unroll
+        for (int k = 0; k < kRows; ++k)
+#pragma unroll
+            for (int p = 0; p < kPasses; ++p) build_b_quad<D>(sB, m[k][p], rl, n0 + k, p, lane);
+    }
+};
 
 // The D / 32 fp16 group scales of one row, as packed 16-bit pairs.
 template <int G>
@@ -234,23 +265,30 @@ __global__ void __launch_bounds__(kThreads, 1)
     const int64_t seg_first = n_my > 0 ? tile_begin / tps : 0;
     auto lambda_row = [&](int64_t seg) -> const float * { return prm.g.lambda + (prm.g.n_lambda == 1 ? 0 : seg) * D; };
 
-    fence_proxy_async();
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = ctrl->tmem_base;
-    volatile uint32_t *abort_flag = &ctrl->abort;
-    uint32_t *status = prm.g.status;
-
     // ---- B for the first tile's lambda row: the sixteen dequant and epilogue warps build D / 16 rows each while the
-    // ---- producer's first loads are in flight; the mma warp waits for all of them
+    // ---- producer's first loads are in flight; the mma warp waits for all of them.  Table rows and lambda are
+    // ---- requested before the set-up barrier, so that their latency runs under it.
     if (n_my > 0 && warp >= 2) {
+        FirstRows<D> rows;
+        rows.load(prm.g.b0, (warp - 2) * (D / 16), lane);
         const RecipLambda<D> rl(lambda_row(seg_first), lane);
-        build_b_rows<D>(sB, prm.g.b0, rl, (warp - 2) * (D / 16), (warp - 1) * (D / 16), lane);
+        fence_proxy_async();
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+        rows.build(sB, rl, (warp - 2) * (D / 16), lane);
         fence_proxy_async();   // B is read by the tensor core through the async proxy
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&ctrl->b_first));
+    } else {
+        fence_proxy_async();
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
     }
+    const uint32_t tmem_base = ctrl->tmem_base;
+    volatile uint32_t *abort_flag = &ctrl->abort;
+    uint32_t *status = prm.g.status;
 
     if (warp == 0) {
         // =========================== producer ===========================

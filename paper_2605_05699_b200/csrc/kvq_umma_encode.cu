@@ -106,35 +106,71 @@ __device__ __forceinline__ float lift_of(const float *__restrict__ lam, float ta
 // Rows [c0, c1) of every split term of the B operand, by one warp: a lane reads four table entries
 // e0[c][4 i .. 4 i + 3] (coalesced rows), scales them by lambda_c 2^k, peels off 16-bit terms and writes
 // 8 bytes of each term's swizzled row.
+// One quad of row c of every split term: the four table entries m scaled by f = lambda_c 2^k, 16-bit terms peeled
+// off one after the other, 8 bytes of each term's swizzled row written.
+template <int D, bool BF16>
+__device__ __forceinline__ void build_b_quad(unsigned char *sB, float4 m, float f, int c, int i)
+{
+    using C = Cfg<D, BF16>;
+    float w[4] = {m.x * f, m.y * f, m.z * f, m.w * f};
+    const int ch = i >> 1;   // 16-byte chunk of the K-major row: K block ch / 8, chunk ch % 8
+    const uint32_t off = (uint32_t)((ch >> 3) * C::kBBlock + c * 128 + (((ch & 7) ^ (c & 7)) << 4) + ((i & 1) ? 8 : 0));
+#pragma unroll
+    for (int t = 0; t < C::kSplit; ++t) {
+        const uint32_t lo = narrow2<BF16>(w[0], w[1]), hi = narrow2<BF16>(w[2], w[3]);
+        *reinterpret_cast<uint2 *>(sB + t * C::kBTerm + off) = make_uint2(lo, hi);
+        if (t + 1 < C::kSplit) {   // what the 16-bit term left behind (exact in fp32)
+            const float2 a = widen2<BF16>(lo), b = widen2<BF16>(hi);
+            w[0] -= a.x, w[1] -= a.y, w[2] -= b.x, w[3] -= b.y;
+        }
+    }
+}
+
 template <int D, bool BF16>
 __device__ __forceinline__ void build_b_rows(unsigned char *sB, const float *__restrict__ e0, const float *__restrict__ lam, float lift,
                                              int c0, int c1, int lane)
 {
-    using C = Cfg<D, BF16>;
 #pragma unroll 4
     for (int c = c0; c < c1; ++c) {
         const float f = lam ? __ldg(lam + c) * lift : lift;
 #pragma unroll
         for (int p = 0; p < (D / 4 + 31) / 32; ++p) {
             const int i = lane + 32 * p;
-            if (i < D / 4) {
-                const float4 m = __ldg(reinterpret_cast<const float4 *>(e0 + (size_t)c * D) + i);
-                float w[4] = {m.x * f, m.y * f, m.z * f, m.w * f};
-                const int ch = i >> 1;   // 16-byte chunk of the K-major row: K block ch / 8, chunk ch % 8
-                const uint32_t off = (uint32_t)((ch >> 3) * C::kBBlock + c * 128 + (((ch & 7) ^ (c & 7)) << 4) + ((i & 1) ? 8 : 0));
-#pragma unroll
-                for (int t = 0; t < C::kSplit; ++t) {
-                    const uint32_t lo = narrow2<BF16>(w[0], w[1]), hi = narrow2<BF16>(w[2], w[3]);
-                    *reinterpret_cast<uint2 *>(sB + t * C::kBTerm + off) = make_uint2(lo, hi);
-                    if (t + 1 < C::kSplit) {   // what the 16-bit term left behind (exact in fp32)
-                        const float2 a = widen2<BF16>(lo), b = widen2<BF16>(hi);
-                        w[0] -= a.x, w[1] -= a.y, w[2] -= b.x, w[3] -= b.y;
-                    }
-                }
-            }
+            if (i < D / 4) build_b_quad<D, BF16>(sB, __ldg(reinterpret_cast<const float4 *>(e0 + (size_t)c * D) + i), f, c, i);
         }
     }
 }
+
+// The first build of a CTA: a warp's D / 16 table rows and their lambda entries are requested at kernel entry, all at
+// once, and turned into B rows once the lift is known: one round trip to L2 instead of one per batch of rows.
+template <int D, bool BF16>
+struct FirstRows {
+    static constexpr int kRows = D / 16, kPasses = (D / 4 + 31) / 32;
+    float4 m[kRows][kPasses];
+    float lam_c[kRows];
+    __device__ __forceinline__ void load(const float *__restrict__ e0, const float *__restrict__ lam, int c0, int lane)
+    {
+#pragma unroll
+        for (int k = 0; k < kRows; ++k) {
+#pragma unroll
+            for (int p = 0; p < kPasses; ++p) {
+                const int i = lane + 32 * p;
+                m[k][p] = i < D / 4 ? __ldg(reinterpret_cast<const float4 *>(e0 + (size_t)(c0 + k) * D) + i) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            }
+            lam_c[k] = lam ? __ldg(lam + c0 + k) : 1.0f;
+        }
+    }
+    __device__ __forceinline__ void build(unsigned char *sB, float lift, int c0, int lane) const
+    {
+#pragma unroll
+        for (int k = 0; k < kRows; ++k)
+#pragma unroll
+            for (int p = 0; p < kPasses; ++p) {
+                const int i = lane + 32 * p;
+                if (i < D / 4) build_b_quad<D, BF16>(sB, m[k][p], lam_c[k] * lift, c0 + k, i);
+            }
+    }
+};
 
 }  // namespace
 
@@ -179,13 +215,6 @@ __global__ void __launch_bounds__(kThreads, 1)
         mbar_init_fence();
     }
     if (warp == 0) tmem_alloc(smem_u32(&ctrl->tmem_base), kTmemCols);
-    fence_proxy_async();
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = ctrl->tmem_base;
-    volatile uint32_t *abort_flag = &ctrl->abort;
-    uint32_t *status = prm.status;
 
     // ---- tiles: lambda segments of rpl rows, cut into tiles of 128 rows; a contiguous range per CTA
     const int64_t N = prm.N, rpl = prm.rpl;
@@ -195,6 +224,34 @@ __global__ void __launch_bounds__(kThreads, 1)
     const int64_t tile_begin = (int64_t)blockIdx.x * per_cta;
     const int64_t tile_end = tile_begin + per_cta < n_tiles ? tile_begin + per_cta : n_tiles;
     const int n_my = tile_end > tile_begin ? (int)(tile_end - tile_begin) : 0;
+
+    // ---- B for the CTA's first lambda row: D / 16 rows per epilogue warp.  Table rows and lambda are requested before
+    // ---- the set-up barrier, so that their latency runs under it and under the first x loads.
+    float first_lift = 1.0f;
+    int64_t first_seg = -1;
+    if (n_my > 0 && warp >= 2) {
+        first_seg = tile_begin / tps;
+        const float *lam = CALIB ? nullptr : prm.lambda + (prm.n_lambda == 1 ? 0 : first_seg) * D;
+        FirstRows<D, BF16> rows;
+        rows.load(prm.e0, lam, (warp - 2) * (D / 16), lane);
+        first_lift = lift_of<D>(lam, prm.table_max, lane);
+        fence_proxy_async();
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+        rows.build(sB, first_lift, (warp - 2) * (D / 16), lane);
+        fence_proxy_async();   // B is read by the tensor core through the async proxy
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&ctrl->b_first));
+    } else {
+        fence_proxy_async();
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+    }
+    const uint32_t tmem_base = ctrl->tmem_base;
+    volatile uint32_t *abort_flag = &ctrl->abort;
+    uint32_t *status = prm.status;
 
     if (warp == 0) {
         // =========================== producer ===========================
@@ -282,19 +339,8 @@ __global__ void __launch_bounds__(kThreads, 1)
         const int g0 = h * C::kGroupsPerPart;                                        // this thread's groups: g0 .. g1 - 1
         const int g1 = h == 0 ? C::kGroupsPerPart : G;
         const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16);
-        int64_t cached_seg = -1;
-        float unlift = 1.0f;
-        if (n_my > 0) {   // B for the CTA's first lambda row: D / 16 rows per warp, all sixteen warps
-            TileCursor first(tile_begin, tps);
-            const float *lam = CALIB ? nullptr : prm.lambda + (prm.n_lambda == 1 ? 0 : first.seg) * D;
-            const float lift = lift_of<D>(lam, prm.table_max, lane);
-            build_b_rows<D, BF16>(sB, prm.e0, lam, lift, (warp - 2) * (D / 16), (warp - 1) * (D / 16), lane);
-            fence_proxy_async();   // B is read by the tensor core through the async proxy
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&ctrl->b_first));
-            unlift = 1.0f / lift;
-            cached_seg = first.seg;
-        }
+        int64_t cached_seg = first_seg;           // B holds this row's table (built above)
+        float unlift = 1.0f / first_lift;
         float colmax[C::kGroupsPerPart] = {};   // calibration: lane i keeps the running maximum of column i of each of this thread's groups
         TileCursor cur(tile_begin + set, tps);
         for (int j = set; j < n_my; j += 2, cur.advance(2)) {
