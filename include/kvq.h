@@ -58,7 +58,7 @@ typedef enum {
     KVQ_IMPL_AUTO = 0,
     KVQ_IMPL_FFT = 1,   /* fp32 register FFT, one thread per vector: every D, dtype and layout; no rotation */
     KVQ_IMPL_GEMM = 2,  /* tcgen05 DFT-as-GEMM, group = 32 and bits = 4 only.  encode / append: fp16 for D = 64, 96, 128,
-                           160, 256, bf16 for D = 64, 96, 128, 256; decode: fp16 for the same D, bf16 for D = 256.
+                           160, 256, bf16 for D = 64, 96, 128, 256; decode: the same.
                            Elsewhere the compute calls return KVQ_ERR_UNSUPPORTED_DIM. */
     KVQ_IMPL_MATVEC = 3 /* fp32 matrix-vector product with the plan's D x D table, a CTA per 8 vectors: every D, dtype
                            and layout, rotated plans included; meant for small calls, correct (and slow) at any size */

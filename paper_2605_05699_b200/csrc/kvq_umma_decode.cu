@@ -51,14 +51,21 @@ constexpr int kAccStages = 2;    // accumulators in tensor memory
 constexpr int kCtrlBytes = 256;
 constexpr uint32_t kTmemCols = 512;
 
-template <int D>
+// BF16OUT: bfloat16 output rounds 8x coarser than fp16, and a result that is off by 1e-4 of the vector's rms already
+// lands on the other side of enough rounding boundaries to miss the 1e-3 tolerance.  Both operands are then carried
+// in two fp16 terms: a = q sigma rho has 15 significant bits and splits exactly into a_hi + a_lo (one half2 FMA),
+// W' = W_hi + W_lo, and x^ = a_hi W_hi + a_lo W_hi + a_hi W_lo accumulates in fp32 (a_lo W_lo is below 1e-7).
+template <int D, bool BF16OUT>
 struct Cfg {
     static_assert(D % 32 == 0 && D >= 64 && D <= 160, "head dim not built");
+    static_assert(!BF16OUT || D <= 128, "two-term operands: tensor memory holds them for D <= 128 only");
+    static constexpr int kTerms = BF16OUT ? 2 : 1;         // W_hi (, W_lo); a_hi (, a_lo)
     static constexpr int G = D / 32;                       // groups = 16-byte chunks of a packed row = 32-column accumulator chunks
     static constexpr int kKSteps = D / 16;
     static constexpr int kKBlocks = (D + 63) / 64;         // K blocks of 64 elements (the last one may be half used)
     static constexpr int kBBlock = D * 128;                // bytes of one K block: D rows x 128 B
-    static constexpr int kBBytes = kKBlocks * kBBlock;
+    static constexpr int kBTerm = kKBlocks * kBBlock;
+    static constexpr int kBBytes = kTerms * kBTerm;
     static constexpr int kInRow = D / 2;                   // packed bytes per row
     static constexpr int kInBytes = kTile * kInRow;        // bytes one TMA load brings
     static constexpr int kInPitch = (kInBytes + 1023) & ~1023;
@@ -68,11 +75,16 @@ struct Cfg {
     static constexpr int kOutWarpBytes = 32 * 2 * D;       // staging of one epilogue warp: G / 2 boxes of 4 KB (+ one of 2 KB)
     static constexpr int kOutBytes = 8 * kOutWarpBytes;
     static constexpr int kSmemBytes = kBBytes + kInStages * kInPitch + kOutBytes + kCtrlBytes + 1024;
-    // tensor memory: two accumulators of D columns, then the A stages of D / 2 columns
+    // tensor memory: two accumulators of D columns, then the A stages of D / 2 columns per term (a_lo 64 columns
+    // behind a_hi)
     static constexpr uint32_t kAccStride = D <= 128 ? 128 : 256;
-    static constexpr int kAStages = D <= 128 ? 4 : 2;
+    static constexpr int kAStages = BF16OUT ? 2 : D <= 128 ? 4 : 2;
+    static constexpr uint32_t kALo = 64;
     __host__ __device__ static constexpr uint32_t acc_col(int s) { return (uint32_t)s * kAccStride; }
-    __host__ __device__ static constexpr uint32_t a_col(int s) { return D <= 128 ? 256u + 64u * (uint32_t)s : 160u + 256u * (uint32_t)s; }
+    __host__ __device__ static constexpr uint32_t a_col(int s)
+    {
+        return D <= 128 ? 256u + 64u * (uint32_t)kTerms * (uint32_t)s : 160u + 256u * (uint32_t)s;
+    }
     static constexpr uint32_t kIdesc = umma_idesc_m128(D, false);
 };
 
@@ -125,25 +137,34 @@ struct RecipLambda {
 // Rows [n0, n1) of the B operand, by one warp: a lane reads four table entries b0[n][4 i .. 4 i + 3] (coalesced
 // rows), scales them, trades two values with its neighbour so that each lane holds two K-ordered pairs, and
 // writes 8 bytes of the swizzled row.
-template <int D>
+template <int D, bool BF16OUT>
 __device__ __forceinline__ void build_b_quad(unsigned char *sB, float4 m, const RecipLambda<D> &rl, int n, int p, int lane)
 {
+    using C = Cfg<D, BF16OUT>;
     const bool odd = lane & 1;
     const int i = lane + 32 * p;
     const bool live = i < D / 4;
     auto sat = [](float v) { return fminf(fmaxf(v, -65504.0f), 65504.0f); };
-    const float vx = sat(m.x * rl.r[p].x), vy = sat(m.y * rl.r[p].y), vz = sat(m.z * rl.r[p].z), vw = sat(m.w * rl.r[p].w);
-    // even lane holds codes 8w .. 8w+3, odd lane 8w+4 .. 8w+7; K order of the word is (0,4,1,5,2,6,3,7)
-    const float r0 = __shfl_xor_sync(0xFFFFFFFFu, odd ? vx : vz, 1);
-    const float r1 = __shfl_xor_sync(0xFFFFFFFFu, odd ? vy : vw, 1);
-    uint2 o;
-    o.x = odd ? narrow2<false>(r0, vz) : narrow2<false>(vx, r0);   // odd: (2, 6)   even: (0, 4)
-    o.y = odd ? narrow2<false>(r1, vw) : narrow2<false>(vy, r1);   // odd: (3, 7)   even: (1, 5)
+    float vx = sat(m.x * rl.r[p].x), vy = sat(m.y * rl.r[p].y), vz = sat(m.z * rl.r[p].z), vw = sat(m.w * rl.r[p].w);
     const int w = i >> 1;   // word of 8 codes = 16-byte chunk w of the K-major row: K block w / 8, chunk w % 8
-    if (live) *reinterpret_cast<uint2 *>(sB + (w >> 3) * Cfg<D>::kBBlock + n * 128 + (((w & 7) ^ (n & 7)) << 4) + (odd ? 8 : 0)) = o;
+    unsigned char *dst = sB + (w >> 3) * C::kBBlock + n * 128 + (((w & 7) ^ (n & 7)) << 4) + (odd ? 8 : 0);
+#pragma unroll
+    for (int t = 0; t < C::kTerms; ++t) {
+        // even lane holds codes 8w .. 8w+3, odd lane 8w+4 .. 8w+7; K order of the word is (0,4,1,5,2,6,3,7)
+        const float r0 = __shfl_xor_sync(0xFFFFFFFFu, odd ? vx : vz, 1);
+        const float r1 = __shfl_xor_sync(0xFFFFFFFFu, odd ? vy : vw, 1);
+        uint2 o;
+        o.x = odd ? narrow2<false>(r0, vz) : narrow2<false>(vx, r0);   // odd: (2, 6)   even: (0, 4)
+        o.y = odd ? narrow2<false>(r1, vw) : narrow2<false>(vy, r1);   // odd: (3, 7)   even: (1, 5)
+        if (live) *reinterpret_cast<uint2 *>(dst + t * C::kBTerm) = o;
+        if (t + 1 < C::kTerms) {   // what the fp16 term left behind (exact in fp32)
+            vx -= __half2float(__float2half_rn(vx)), vy -= __half2float(__float2half_rn(vy));
+            vz -= __half2float(__float2half_rn(vz)), vw -= __half2float(__float2half_rn(vw));
+        }
+    }
 }
 
-template <int D>
+template <int D, bool BF16OUT>
 __device__ __forceinline__ void build_b_rows(unsigned char *sB, const float *__restrict__ b0, const RecipLambda<D> &rl, int n0, int n1,
                                              int lane)
 {
@@ -154,14 +175,14 @@ __device__ __forceinline__ void build_b_rows(unsigned char *sB, const float *__r
             const int i = lane + 32 * p;
             float4 m = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
             if (i < D / 4) m = __ldg(reinterpret_cast<const float4 *>(b0 + (size_t)n * D) + i);
-            build_b_quad<D>(sB, m, rl, n, p, lane);
+            build_b_quad<D, BF16OUT>(sB, m, rl, n, p, lane);
         }
     }
 }
 
 // The first build of a CTA: its D / 16 table rows per warp are requested at kernel entry, all at once, and turned
 // into B rows here, once lambda has arrived too: one round trip to L2 instead of one per batch of rows.
-template <int D>
+template <int D, bool BF16OUT>
 struct FirstRows {
     static constexpr int kRows = D / 16, kPasses = RecipLambda<D>::kPasses;
     float4 m[kRows][kPasses];
@@ -180,7 +201,7 @@ struct FirstRows {
 #pragma unroll
         for (int k = 0; k < kRows; ++k)
 #pragma unroll
-            for (int p = 0; p < kPasses; ++p) build_b_quad<D>(sB, m[k][p], rl, n0 + k, p, lane);
+            for (int p = 0; p < kPasses; ++p) build_b_quad<D, BF16OUT>(sB, m[k][p], rl, n0 + k, p, lane);
     }
 };
 
@@ -219,11 +240,11 @@ struct UmmaDecodeMaps {
     CUtensorMap slim, slim_tail;   // output, boxes of 32 columns x 32 rows (64-byte swizzle), used when D / 32 is odd
 };
 
-template <int D>
+template <int D, bool BF16OUT>
 __global__ void __launch_bounds__(kThreads, 1)
     kvq_decode_umma_kernel(const __grid_constant__ UmmaDecodeParams prm, const __grid_constant__ UmmaDecodeMaps maps)
 {
-    using C = Cfg<D>;
+    using C = Cfg<D, BF16OUT>;
     constexpr int G = C::G;
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -269,7 +290,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     // ---- producer's first loads are in flight; the mma warp waits for all of them.  Table rows and lambda are
     // ---- requested before the set-up barrier, so that their latency runs under it.
     if (n_my > 0 && warp >= 2) {
-        FirstRows<D> rows;
+        FirstRows<D, BF16OUT> rows;
         rows.load(prm.g.b0, (warp - 2) * (D / 16), lane);
         const RecipLambda<D> rl(lambda_row(seg_first), lane);
         fence_proxy_async();
@@ -329,12 +350,18 @@ __global__ void __launch_bounds__(kThreads, 1)
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + C::acc_col(sc);
                 const uint32_t a_tmem = tmem_base + C::a_col(sa);
+                // bf16 output: a_hi W_hi + a_lo W_hi + a_hi W_lo
 #pragma unroll
-                for (int ks = 0; ks < C::kKSteps; ++ks) {
-                    const uint32_t koff = (uint32_t)(ks >> 2) * (C::kBBlock >> 4) + (uint32_t)(ks & 3) * 2u;   // (bytes >> 4) of K-step ks
-                    const uint64_t bd = ((uint64_t)b_hi << 32) | (uint64_t)(b_lo + koff);
-                    if (ks > 0) umma_f16_ts<true>(d_tmem, a_tmem + (uint32_t)ks * 8u, bd, C::kIdesc);
-                    else umma_f16_ts<false>(d_tmem, a_tmem, bd, C::kIdesc);
+                for (int set = 0; set < (BF16OUT ? 3 : 1); ++set) {
+                    const uint32_t a_set = a_tmem + (set == 1 ? C::kALo : 0u);
+                    const uint32_t b_set = b_lo + (set == 2 ? (uint32_t)(C::kBTerm >> 4) : 0u);
+#pragma unroll
+                    for (int ks = 0; ks < C::kKSteps; ++ks) {
+                        const uint32_t koff = (uint32_t)(ks >> 2) * (C::kBBlock >> 4) + (uint32_t)(ks & 3) * 2u;   // (bytes >> 4) of K-step ks
+                        const uint64_t bd = ((uint64_t)b_hi << 32) | (uint64_t)(b_set + koff);
+                        if (set > 0 || ks > 0) umma_f16_ts<true>(d_tmem, a_set + (uint32_t)ks * 8u, bd, C::kIdesc);
+                        else umma_f16_ts<false>(d_tmem, a_set, bd, C::kIdesc);
+                    }
                 }
                 umma_commit(smem_u32(&ctrl->acc_full[sc]));
                 umma_commit(smem_u32(&ctrl->a_empty[sa]));
@@ -386,7 +413,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                     if (!wait_or_abort(smem_u32(&ctrl->a_empty[(j - 1) % C::kAStages]), (uint32_t)((j - 1) / C::kAStages) & 1u, abort_flag,
                                        status, KVQ_DEV_MMA_TIMEOUT))
                         break;
-                    build_b_rows<D>(sB, prm.g.b0, rl, q * (D / 4), (q + 1) * (D / 4), lane);
+                    build_b_rows<D, BF16OUT>(sB, prm.g.b0, rl, q * (D / 4), (q + 1) * (D / 4), lane);
                     fence_proxy_async();   // B is read by the tensor core through the async proxy
                 }
                 cached_seg = seg;
@@ -415,18 +442,24 @@ __global__ void __launch_bounds__(kThreads, 1)
                 const float sig = __half2float(__ushort_as_half((unsigned short)((sc[c >> 1] >> (16 * (c & 1))) & 0xFFFFu)));
                 const __half2 s2 = __float2half2_rn(sig * rho);
                 const uint32_t words[4] = {pk[c].x, pk[c].y, pk[c].z, pk[c].w};
-                uint32_t a[16];
+                uint32_t a[16], al[BF16OUT ? 16 : 1];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const uint32_t u = words[i] ^ 0x88888888u;   // nibbles now hold q + 8
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         const uint32_t m = lop3_and_or(u >> (4 * e), 0x000F000Fu, 0x64006400u);   // {1024 + n_e, 1024 + n_{e+4}}
-                        const __half2 h = __hmul2(__hsub2(*reinterpret_cast<const __half2 *>(&m), h1032), s2);   // exact q, one rounding
+                        const __half2 q2 = __hsub2(*reinterpret_cast<const __half2 *>(&m), h1032);     // exact q
+                        const __half2 h = __hmul2(q2, s2);                                                 // one rounding
                         a[4 * i + e] = *reinterpret_cast<const uint32_t *>(&h);
+                        if constexpr (BF16OUT) {   // what the rounding left behind: q s2 - h, exact in fp16
+                            const __half2 l = __hfma2(q2, s2, __hneg2(h));
+                            al[4 * i + e] = *reinterpret_cast<const uint32_t *>(&l);
+                        }
                     }
                 }
                 tmem_st16(a_row + 16u * (uint32_t)c, a);
+                if constexpr (BF16OUT) tmem_st16(a_row + C::kALo + 16u * (uint32_t)c, al);
             }
             tmem_st_wait();
             tc_fence_before();
@@ -457,10 +490,10 @@ __global__ void __launch_bounds__(kThreads, 1)
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     uint4 o;
-                    o.x = narrow2<false>(__uint_as_float(v[8 * k]), __uint_as_float(v[8 * k + 1]));
-                    o.y = narrow2<false>(__uint_as_float(v[8 * k + 2]), __uint_as_float(v[8 * k + 3]));
-                    o.z = narrow2<false>(__uint_as_float(v[8 * k + 4]), __uint_as_float(v[8 * k + 5]));
-                    o.w = narrow2<false>(__uint_as_float(v[8 * k + 6]), __uint_as_float(v[8 * k + 7]));
+                    o.x = narrow2<BF16OUT>(__uint_as_float(v[8 * k]), __uint_as_float(v[8 * k + 1]));
+                    o.y = narrow2<BF16OUT>(__uint_as_float(v[8 * k + 2]), __uint_as_float(v[8 * k + 3]));
+                    o.z = narrow2<BF16OUT>(__uint_as_float(v[8 * k + 4]), __uint_as_float(v[8 * k + 5]));
+                    o.w = narrow2<BF16OUT>(__uint_as_float(v[8 * k + 6]), __uint_as_float(v[8 * k + 7]));
                     if (wide) {   // [32 rows][128 B], 128-byte swizzle
                         const int chunk = (cc & 1) * 4 + k;
                         *reinterpret_cast<uint4 *>(box + lane * 128 + ((chunk ^ (lane & 7)) << 4)) = o;
@@ -504,10 +537,10 @@ __global__ void __launch_bounds__(kThreads, 1)
 // ------------------------------------------------------------------------------------------------
 namespace {
 
-template <int D>
+template <int D, bool BF16OUT>
 cudaError_t launch(int64_t N, const GemmParams &g, cudaStream_t stream)
 {
-    using C = Cfg<D>;
+    using C = Cfg<D, BF16OUT>;
     static DeviceSlots slots;
     int dev = 0;
     cudaError_t e = current_device_slot(&dev);
@@ -515,7 +548,7 @@ cudaError_t launch(int64_t N, const GemmParams &g, cudaStream_t stream)
     int &sms = slots.sms[dev];
     if (sms == 0) {
         int n = 0;
-        if ((e = cudaFuncSetAttribute(kvq_decode_umma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes)) != cudaSuccess) return e;
+        if ((e = cudaFuncSetAttribute(kvq_decode_umma_kernel<D, BF16OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes)) != cudaSuccess) return e;
         if ((e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
         sms = n;
     }
@@ -542,7 +575,7 @@ cudaError_t launch(int64_t N, const GemmParams &g, cudaStream_t stream)
         const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)rows, (cuuint64_t)segs};
         const cuuint64_t strides[2] = {(cuuint64_t)(2 * D), (cuuint64_t)(2 * D) * (cuuint64_t)rows};
         const cuuint32_t box[3] = {wide ? 64u : 32u, 32u, 1u};
-        return make_tensor_map(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, base, dims, strides, box,
+        return make_tensor_map(tm, BF16OUT ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, base, dims, strides, box,
                                wide ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B);
     };
     const int64_t tail_rows = N - prm.n_full * prm.rpl;
@@ -556,24 +589,23 @@ cudaError_t launch(int64_t N, const GemmParams &g, cudaStream_t stream)
 
     const int64_t tiles = prm.n_seg * ((prm.rpl + kTile - 1) / kTile);
     const int grid = (int)(tiles < sms ? tiles : sms);
-    kvq_decode_umma_kernel<D><<<grid, kThreads, C::kSmemBytes, stream>>>(prm, maps);
+    kvq_decode_umma_kernel<D, BF16OUT><<<grid, kThreads, C::kSmemBytes, stream>>>(prm, maps);
     count_launch();
     return cudaGetLastError();
 }
 
 }  // namespace
 
-bool umma_decode_supported(int D, bool bf16) { return D == 256 || (!bf16 && (D == 64 || D == 96 || D == 128 || D == 160)); }
+bool umma_decode_supported(int D, bool bf16) { return D == 256 || D == 64 || D == 96 || D == 128 || (!bf16 && D == 160); }
 
 cudaError_t umma_decode(int D, bool bf16, int64_t N, const GemmParams &g, const uint32_t *sign_xor, cudaStream_t stream)
 {
     if (D == 256) return umma_decode_d256(bf16, N, g, sign_xor, stream);   // its own kernel: radix-2 split, split operands for bf16
-    if (bf16) return cudaErrorInvalidValue;
     switch (D) {
-        case 64: return launch<64>(N, g, stream);
-        case 96: return launch<96>(N, g, stream);
-        case 128: return launch<128>(N, g, stream);
-        case 160: return launch<160>(N, g, stream);
+        case 64: return bf16 ? launch<64, true>(N, g, stream) : launch<64, false>(N, g, stream);
+        case 96: return bf16 ? launch<96, true>(N, g, stream) : launch<96, false>(N, g, stream);
+        case 128: return bf16 ? launch<128, true>(N, g, stream) : launch<128, false>(N, g, stream);
+        case 160: return bf16 ? cudaErrorInvalidValue : launch<160, false>(N, g, stream);
     }
     return cudaErrorInvalidValue;
 }
