@@ -1,14 +1,14 @@
 // Warp-specialised tcgen05 DFT-as-GEMM encode kernel of libkvq (sm_100a) for D = 256, fp16 or bf16 input.
 //
 // Same contraction and the same split of W into 16-bit terms as kvq_umma_encode.cu (v = lambda (.) M (s (.) x),
-// Sec. 3.1 Eq. 1-2, Sec. 5.1 item 1; W 2^k = W1 + W2 for fp16 input, W1 + W2 + W3 for bf16), with the two changes
+// Sec. 3.1 Eq. 1-2, Sec. 5.1 item 1; W 2^k = W1 + W2, a third term for bf16 in the calibration pass), with the two changes
 // that D = 256 forces:
 //
 //   * the split B operand (2 or 3 x 128 KB) does not fit one CTA's shared memory, so CTAs work in pairs on the
 //     same tiles and each computes one half of the channels (four groups): B is [128 channels, K = 256] per
 //     term and CTA.  The two CTAs of a pair share nothing and never wait for each other; the x tile is read
 //     twice (the second read hits L2).
-//   * what shared memory is left holds less than one x tile next to a three-term B, so x moves through a ring
+//   * what shared memory is left holds little more than one x tile next to B, so x moves through a ring
 //     of K blocks (64 columns x 128 rows, 16 KB): the mma thread issues the K steps of a block for every term
 //     as soon as the block has landed and releases it with a commit of its own.
 //
@@ -43,12 +43,13 @@ constexpr int kBTerm = kKBlocks * kBBlock; // 64 KB
 constexpr int kAccStages = 4;
 constexpr int kMaxRing = 6;
 
-template <bool BF16>
+// CALIB: the calibration pass keeps a third bf16 term (it runs once; its result is compared at 1e-6 of the vector norm)
+template <bool BF16, bool CALIB = false>
 struct Cfg {
-    static constexpr int kSplit = BF16 ? 3 : 2;
+    static constexpr int kSplit = (BF16 && CALIB) ? 3 : 2;
     static constexpr int kBBytes = kSplit * kBTerm;
     static constexpr int kRoom = (kSmemLimit - 1024 - kCtrlBytes - kBBytes) / kBlockBytes;
-    static constexpr int kRing = kRoom < kMaxRing ? kRoom : kMaxRing;   // K blocks of x in flight: 6 (fp16), 2 (bf16)
+    static constexpr int kRing = kRoom < kMaxRing ? kRoom : kMaxRing;   // K blocks of x in flight: 6 (2 next to a three-term B)
     static_assert(kRing >= 2, "no room for the x ring");
     static constexpr int kSmemBytes = kBBytes + kRing * kBlockBytes + kCtrlBytes + 1024;
     static constexpr uint32_t kIdesc = umma_idesc_m128(kHalfN, BF16);
@@ -88,11 +89,11 @@ __device__ __forceinline__ float lift_of(const float *__restrict__ lam, float ta
 // Rows [c0, c1) of every split term of this CTA's half of the B operand (channel 128 half + c), by one warp: a lane
 // reads four table entries per pass (coalesced rows), scales them by lambda_c 2^k, peels off 16-bit terms and
 // writes 8 bytes of each term's swizzled row.
-template <bool BF16>
+template <bool BF16, bool CALIB>
 __device__ __forceinline__ void build_b_rows(unsigned char *sB, const float *__restrict__ e0, const float *__restrict__ lam, float lift,
                                              int half, int c0, int c1, int lane)
 {
-    using C = Cfg<BF16>;
+    using C = Cfg<BF16, CALIB>;
 #pragma unroll 2
     for (int c = c0; c < c1; ++c) {
         const int cg = half * kHalfN + c;
@@ -138,7 +139,7 @@ template <bool BF16, bool CALIB>
 __global__ void __launch_bounds__(kThreads, 1)
     kvq_encode_umma_d256_kernel(const __grid_constant__ UmmaEncode256Params prm, const __grid_constant__ CUtensorMap tm_x)
 {
-    using C = Cfg<BF16>;
+    using C = Cfg<BF16, CALIB>;
     constexpr int kRing = C::kRing;
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -272,7 +273,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             TileCursor first(tile_begin, tps);
             const float *lam = CALIB ? nullptr : prm.lambda + (prm.n_lambda == 1 ? 0 : first.seg) * kD;
             const float lift = lift_of<kD>(lam, prm.table_max, lane);
-            build_b_rows<BF16>(sB, prm.e0, lam, lift, half, (warp - 2) * 8, (warp - 1) * 8, lane);
+            build_b_rows<BF16, CALIB>(sB, prm.e0, lam, lift, half, (warp - 2) * 8, (warp - 1) * 8, lane);
             fence_proxy_async();   // B is read by the tensor core through the async proxy
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctrl->b_first));
@@ -296,7 +297,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                     if (!wait_or_abort(smem_u32(&ctrl->acc_full[(j - 1) % kAccStages]), (uint32_t)((j - 1) / kAccStages) & 1u,
                                        abort_flag, status, KVQ_DEV_MMA_TIMEOUT))
                         break;
-                    build_b_rows<BF16>(sB, prm.e0, lam, lift, half, bw * 16, (bw + 1) * 16, lane);
+                    build_b_rows<BF16, CALIB>(sB, prm.e0, lam, lift, half, bw * 16, (bw + 1) * 16, lane);
                     fence_proxy_async();   // B is read by the tensor core through the async proxy
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&ctrl->b_ready));
@@ -394,7 +395,7 @@ namespace {
 template <bool BF16, bool CALIB = false>
 cudaError_t launch(int64_t N, const FftParams &f, const float *e0, cudaStream_t stream, uint32_t *amax_bits = nullptr)
 {
-    using C = Cfg<BF16>;
+    using C = Cfg<BF16, CALIB>;
     static DeviceSlots slots;
     int dev = 0;
     cudaError_t e = current_device_slot(&dev);

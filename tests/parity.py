@@ -3,7 +3,8 @@
 Tolerances (the benchmark spec's, with the readings the design notes list):
   * nibble pack / unpack: bit-exact (GPU bytes unpack to the GPU's own codes and repack to the same bytes;
     where codes agree the bytes agree).
-  * int4 codes: identical on >= 99.99 % of entries; every mismatch is off by exactly one and lies at a
+  * int4 codes: identical on >= 99.99 % of the entries of a tensor (a caller that splits one tensor into small
+    subsamples passes a looser per-subsample bound and applies 99.99 % to the whole); every mismatch is off by exactly one and lies at a
     rounding tie: with t = v_oracle / sigma in fp64, |t - boundary| <= 1e-3 for sigma = the GPU's or the
     oracle's stored scale; or, when the two stored scales differ (by one fp16 ulp at most), the GPU code is
     the correctly rounded code for the GPU's own stored scale.
@@ -27,7 +28,7 @@ def f16_bits_to_f64(b):
     return np.ascontiguousarray(b).view(np.uint16).view(np.float16).astype(np.float64)
 
 
-def check_encode(gpu_packed, gpu_scales_bits, ora, group, label="", bits=4):
+def check_encode(gpu_packed, gpu_scales_bits, ora, group, label="", bits=4, min_agree=CODE_AGREEMENT):
     """gpu_packed [N, D bits/8] uint8, gpu_scales_bits [N,G] uint16, ora = oracle.encode(..., want_v=True, bits=bits).
     The rules are those of the 4-bit codes with 7 read as 2^(bits-1) - 1; 8-bit codes are one byte each."""
     gpu_packed = np.ascontiguousarray(gpu_packed).view(np.uint8)
@@ -64,7 +65,7 @@ def check_encode(gpu_packed, gpu_scales_bits, ora, group, label="", bits=4):
 
     # codes
     agree = float(same.mean()) if same.size else 1.0
-    assert agree >= CODE_AGREEMENT, label + ": only %.6f of the codes agree" % agree
+    assert agree >= min_agree, label + ": only %.6f of the codes agree" % agree
     rr, cc = np.nonzero(~same)
     if rr.size:
         v = ora["v"][rr, cc]
@@ -80,7 +81,7 @@ def check_encode(gpu_packed, gpu_scales_bits, ora, group, label="", bits=4):
         bad = ~(at_tie | own)
         assert not bad.any(), label + ": %d mismatched codes are not at a rounding tie (e.g. t=%r)" % (
             bad.sum(), t_o[bad][:4])
-    return {"agree": agree, "mismatches": int(rr.size), "scale_flips": scale_flip_frac,
+    return {"agree": agree, "mismatches": int(rr.size), "codes": int(same.size), "scale_flips": scale_flip_frac,
             "scale_rel_l2": float(rel.max(initial=0))}
 
 
