@@ -122,7 +122,7 @@ template <int TERMS>
 __device__ __forceinline__ void build_b_rows(unsigned char *sB, const float *__restrict__ b0, const RecipLambda &rl, int p, int n0, int n1, int lane)
 {
     const bool odd = lane & 1;
-#pragma unroll 4
+#pragma unroll 8   // 16 row quads in flight per lane: the build is a chain of L2 round trips, not arithmetic
     for (int n = n0; n < n1; ++n) {
 #pragma unroll
         for (int ps = 0; ps < 2; ++ps) {
