@@ -125,10 +125,38 @@ def _dev(t: torch.Tensor, what: str) -> int:
     return t.data_ptr()
 
 
-def _stream(stream) -> int:
+_raw_stream = getattr(torch._C, "_cuda_getCurrentRawStream", None)
+
+
+def _stream(stream, device: torch.device = None) -> int:
     if stream is None:
-        return torch.cuda.current_stream().cuda_stream
+        if _raw_stream is not None and device is not None and device.index is not None:
+            return _raw_stream(device.index)   # the handle itself: no Stream object per call
+        return torch.cuda.current_stream(device).cuda_stream
     return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+class _on_device:
+    """Makes ``device`` current for the call (a plan's tables live on the device of its first use) and restores the
+    previous one; costs one query when it already is current, which is the usual case."""
+    __slots__ = ("idx", "prev")
+
+    def __init__(self, device: torch.device):
+        self.idx = device.index
+        self.prev = -1
+
+    def __enter__(self):
+        if self.idx is not None:
+            cur = torch.cuda.current_device()
+            if cur != self.idx:
+                self.prev = cur
+                torch.cuda.set_device(self.idx)
+        return self
+
+    def __exit__(self, *exc):
+        if self.prev >= 0:
+            torch.cuda.set_device(self.prev)
+        return False
 
 
 # ---- C entry points, same names ---------------------------------------------------------
@@ -200,9 +228,9 @@ def kvq_encode(plan: int, x: torch.Tensor, lam: torch.Tensor, packed: torch.Tens
     D = x.shape[-1]
     N = x.numel() // D
     n_lambda = lam.numel() // D
-    with torch.cuda.device(x.device):
+    with _on_device(x.device):
         _check(lib().kvq_encode(plan, _dev(x, "x"), _dtype_code(x), N, _dev(lam, "lambda"), n_lambda,
-                                rows_per_lambda, _dev(packed, "packed"), _dev(scales, "scales"), _stream(stream)),
+                                rows_per_lambda, _dev(packed, "packed"), _dev(scales, "scales"), _stream(stream, x.device)),
                "kvq_encode")
 
 
@@ -211,9 +239,9 @@ def kvq_decode(plan: int, packed: torch.Tensor, scales: torch.Tensor, lam: torch
     D = out.shape[-1]
     N = out.numel() // D
     n_lambda = lam.numel() // D
-    with torch.cuda.device(out.device):
+    with _on_device(out.device):
         _check(lib().kvq_decode(plan, _dev(packed, "packed"), _dev(scales, "scales"), N, _dev(lam, "lambda"),
-                                n_lambda, rows_per_lambda, _dev(out, "out"), _dtype_code(out), _stream(stream)),
+                                n_lambda, rows_per_lambda, _dev(out, "out"), _dtype_code(out), _stream(stream, out.device)),
                "kvq_decode")
 
 
@@ -223,10 +251,10 @@ def kvq_append(plan: int, x_new: torch.Tensor, lam: torch.Tensor, packed_cache: 
     S = x_new.numel() // D
     T_max = packed_cache.shape[-2]
     n_lambda = lam.numel() // D
-    with torch.cuda.device(x_new.device):
+    with _on_device(x_new.device):
         _check(lib().kvq_append(plan, _dev(x_new, "x_new"), _dtype_code(x_new), S, _dev(lam, "lambda"), n_lambda,
                                 streams_per_lambda, _dev(packed_cache, "packed_cache"),
-                                _dev(scales_cache, "scales_cache"), T_max, pos, _stream(stream)),
+                                _dev(scales_cache, "scales_cache"), T_max, pos, _stream(stream, x_new.device)),
                "kvq_append")
 
 
@@ -241,10 +269,10 @@ def kvq_decode_static(plan: int, packed: torch.Tensor, scales: torch.Tensor, lam
     N = out.numel() // D
     n_lambda = lam.numel() // D
     sw = None if status_word is None else _dev(status_word, "status_word")
-    with torch.cuda.device(out.device):
+    with _on_device(out.device):
         _check(lib().kvq_decode_static(plan, _dev(packed, "packed"), _dev(scales, "scales"), N, _dev(lam, "lambda"),
                                        n_lambda, rows_per_lambda, _dev(out, "out"), _dtype_code(out), sw,
-                                       _stream(stream)),
+                                       _stream(stream, out.device)),
                "kvq_decode_static")
 
 
@@ -253,18 +281,18 @@ def kvq_flush_block(plan: int, x_block: torch.Tensor, lam: torch.Tensor, packed_
     S, rows, D = x_block.shape
     T_max = packed_cache.shape[-2]
     n_lambda = lam.numel() // D
-    with torch.cuda.device(x_block.device):
+    with _on_device(x_block.device):
         _check(lib().kvq_flush_block(plan, _dev(x_block, "x_block"), _dtype_code(x_block), S, rows, _dev(lam, "lambda"), n_lambda,
                                      streams_per_lambda, _dev(packed_cache, "packed_cache"), _dev(scales_cache, "scales_cache"),
-                                     _dev(dq_cache, "dq_cache"), T_max, pos0, _stream(stream)),
+                                     _dev(dq_cache, "dq_cache"), T_max, pos0, _stream(stream, x_block.device)),
                "kvq_flush_block")
 
 
 def kvq_calibrate_lambda(plan: int, x: torch.Tensor, lambda_out: torch.Tensor, stream=None) -> None:
     D = x.shape[-1]
     N = x.numel() // D
-    with torch.cuda.device(x.device):
-        _check(lib().kvq_calibrate_lambda(plan, _dev(x, "x"), _dtype_code(x), N, _dev(lambda_out, "lambda_out"), _stream(stream)),
+    with _on_device(x.device):
+        _check(lib().kvq_calibrate_lambda(plan, _dev(x, "x"), _dtype_code(x), N, _dev(lambda_out, "lambda_out"), _stream(stream, x.device)),
                "kvq_calibrate_lambda")
 
 
