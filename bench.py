@@ -3,11 +3,11 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
-Workload: BASELINE config 5, the Llama-3-70B-shaped cache (80 layers x 8 KV heads x D=128 fp16,
+Workload: the Llama-3-70B-shaped cache (80 layers x 8 KV heads x D=128 fp16,
 batch 4, prefix 32768).  One STEP is one pass of the whole hot path over one layer of that cache:
 
     kvq_encode   K and V of the layer: 2 x 1,048,576 vectors (bulk prefill encode, one launch, tensor-core kernel)
-    kvq_append   one new vector per (K/V, head, batch) stream: 64 vectors written at the last row (register-FFT kernel)
+    kvq_append   one new vector per (K/V, head, batch) stream: 64 vectors written at the last row (matrix-vector kernel)
     kvq_decode   full-prefix read of the layer: 2,097,152 vectors back to fp16 (one launch, tensor-core kernel)
 
 Successive steps rotate over distinct layer slots, so every buffer a kernel touches (0.15 - 0.54 GB)

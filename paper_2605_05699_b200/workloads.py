@@ -42,7 +42,7 @@ class CacheShape:
         return self.streams * self.prefix
 
 
-# BASELINE configs 2, 3 and 5 (model shapes from Sec. 4.1 and Table 3).
+# Model-shaped configurations (shapes from Sec. 4.1 and Table 3).
 QWEN25_1P5B = CacheShape("qwen2.5-1.5b-shaped", 28, 2, 128, 1, 1024, "f16")
 GEMMA3_1B = CacheShape("gemma-3-1b-shaped", 26, 1, 256, 1, 4096, "bf16")
 LLAMA3_70B = CacheShape("llama-3-70b-shaped", 80, 8, 128, 4, 32768, "f16")

@@ -1,6 +1,6 @@
 """Parity rules between the CUDA path and the fp64 oracle, written once.
 
-Tolerances (the benchmark spec's, with the readings the design notes list):
+Tolerances (the project's stated ones, with the readings the design notes list):
   * nibble pack / unpack: bit-exact (GPU bytes unpack to the GPU's own codes and repack to the same bytes;
     where codes agree the bytes agree).
   * int4 codes: identical on >= 99.99 % of the entries of a tensor (a caller that splits one tensor into small
