@@ -147,8 +147,8 @@ static kvq_status_t ensure_device(kvq_plan *p)
     return KVQ_OK;
 }
 
-// the tensor-core kernels exist for the fused layout only: groups of 32, 4-bit codes
-static bool gemm_layout(const kvq_plan *p) { return p->group == 32 && p->bits == 4; }
+// the tensor-core kernels exist for 4-bit codes: groups of 32 (the fused layout) or one scale per vector
+static bool gemm_layout(const kvq_plan *p) { return p->bits == 4 && (p->group == 32 || p->group == p->D); }
 
 static bool misaligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
 
@@ -329,7 +329,8 @@ static kvq_status_t encode_common(kvq_plan_t *plan, const void *x, kvq_dtype_t d
     if (st != KVQ_OK) return st;
     if (misaligned16(x) || misaligned16(packed) || misaligned16(scales)) return KVQ_ERR_ALIGNMENT;
     const bool bf16 = dtype == KVQ_BF16;
-    const bool gemm_ok = gemm_layout(plan) && umma_encode_supported(plan->D, bf16);
+    const bool per_vector = plan->group == plan->D;
+    const bool gemm_ok = gemm_layout(plan) && (per_vector ? umma_encode_per_vector_supported(plan->D, bf16) : umma_encode_supported(plan->D, bf16));
     if (plan->enc_impl == KVQ_IMPL_GEMM && !gemm_ok) return KVQ_ERR_UNSUPPORTED_DIM;
     if (plan->rot && plan->enc_impl == KVQ_IMPL_FFT) return KVQ_ERR_UNSUPPORTED_DIM;   // the rotation lives in the D x D tables
     if ((st = ensure_device(plan)) != KVQ_OK) return st;
@@ -350,7 +351,7 @@ static kvq_status_t encode_common(kvq_plan_t *plan, const void *x, kvq_dtype_t d
     }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     cudaError_t e;
-    if (impl == KVQ_IMPL_GEMM) e = umma_encode(plan->D, bf16, N, prm, plan->d_e0, stream);
+    if (impl == KVQ_IMPL_GEMM) e = umma_encode(plan->D, bf16, per_vector, N, prm, plan->d_e0, stream);
     else if (impl == KVQ_IMPL_MATVEC) e = matvec_encode(plan->D, plan->group, plan->bits, bf16, N, prm, plan->d_b0, stream);
     else e = fft_encode(plan->D, plan->group, plan->bits, bf16, N, prm, stream);
     if (e != cudaSuccess) {
@@ -407,6 +408,7 @@ kvq_status_t kvq_decode(kvq_plan_t *plan, const uint8_t *packed, const void *sca
         g.N = N;
         g.n_lambda = n_lambda;
         g.rows_per_lambda = rows_per_lambda < 1 ? 1 : rows_per_lambda;
+        g.per_vector = plan->group == plan->D;
         g.status = plan->d_status;
         // D = 256: the radix-2 kernel needs the transform's even / odd structure, which a rotation destroys
         const cudaError_t e = plan->rot && plan->D == 256 ? umma_decode_d256_dense(bf16, N, g, stream)

@@ -31,6 +31,7 @@ struct FftParams {
     void *out;             // decode: x^ [N, D] half precision
     int64_t N;
     int64_t n_lambda, rows_per_lambda;
+    int per_vector;        // one scale per vector (group = D) instead of one per 32 channels
     RowMap out_map;             // row of packed / scales (encode) or of out (decode) that row r goes to
     RowMap in_map;              // decode: row of packed / scales that row r comes from
     uint32_t *status;           // per-plan device status word
@@ -41,12 +42,13 @@ struct FftParams {
 // Arguments of the tcgen05 DFT-as-GEMM decode kernel (kvq_umma_decode.cu).
 struct GemmParams {
     const void *packed;    // [N, D/2] bytes
-    const void *scales;    // [N, D/group] fp16
+    const void *scales;    // [N, D/32] fp16, or [N, 1] when per_vector
     const float *lambda;   // [n_lambda, D] fp32
     void *out;             // [N, D] fp16
     const float *b0;       // plan table [D, D] fp32: b0[n][c] = s_n M[c][n], M the real orthogonal DFT matrix of Eq. 1-2
     int64_t N;
     int64_t n_lambda, rows_per_lambda;
+    int per_vector;        // one scale per vector (group = D) instead of one per 32 channels
     uint32_t *status;
 };
 
@@ -62,7 +64,8 @@ cudaError_t umma_calibrate_d256(bool bf16, int64_t N, const FftParams &prm, cons
 cudaError_t umma_encode_d256(bool bf16, int64_t N, const FftParams &prm, const float *e0, cudaStream_t stream);   // kvq_umma_encode256.cu
 cudaError_t umma_decode_d256(bool bf16, int64_t N, const GemmParams &prm, const uint32_t *sign_xor, cudaStream_t stream);   // kvq_umma_decode256.cu
 cudaError_t umma_decode_d256_dense(bool bf16, int64_t N, const GemmParams &prm, cudaStream_t stream);   // kvq_umma_decode256_dense.cu: any table
-cudaError_t umma_encode(int D, bool bf16, int64_t N, const FftParams &prm, const float *e0, cudaStream_t stream);
+bool umma_encode_per_vector_supported(int D, bool bf16);
+cudaError_t umma_encode(int D, bool bf16, bool per_vector, int64_t N, const FftParams &prm, const float *e0, cudaStream_t stream);
 
 // fp32 matrix-vector kernels for small calls (kvq_matvec.cu): every layout, dtype and D; b0 / e0 are the plan's tables
 cudaError_t matvec_encode(int D, int group, int bits, bool bf16, int64_t N, const FftParams &prm, const float *b0, cudaStream_t stream);

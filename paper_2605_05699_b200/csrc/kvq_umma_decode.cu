@@ -384,7 +384,15 @@ __global__ void __launch_bounds__(kThreads, 1)
             for (int i = 0; i < (G + 1) / 2; ++i) sc_next[i] = 0u;
             if (j < n_my) {
                 const int64_t row = ahead.seg * rpl + ahead.row_in_segment() + r;
-                if (row < N) load_row_scales<G>(scales + row * G, sc_next);
+                if (row < N) {
+                    if (prm.g.per_vector) {   // one scale per vector: the same value in every group's slot
+                        const uint32_t s1 = (uint32_t)__ldg(scales + row);
+#pragma unroll
+                        for (int i = 0; i < (G + 1) / 2; ++i) sc_next[i] = s1 | (s1 << 16);
+                    } else {
+                        load_row_scales<G>(scales + row * G, sc_next);
+                    }
+                }
             }
         };
 

@@ -308,7 +308,13 @@ __global__ void __launch_bounds__(kThreads, 1)
         auto fetch_scales = [&](int j) -> uint4 {
             if (j >= n_my) return make_uint4(0u, 0u, 0u, 0u);
             const int64_t row = ahead.seg * rpl + ahead.row_in_segment() + r;
-            return row < N ? __ldg(scales + row) : make_uint4(0u, 0u, 0u, 0u);
+            if (row >= N) return make_uint4(0u, 0u, 0u, 0u);
+            if (prm.g.per_vector) {   // one scale per vector: the same value in every group's slot
+                const uint32_t s1 = (uint32_t)__ldg(reinterpret_cast<const uint16_t *>(prm.g.scales) + row);
+                const uint32_t s2 = s1 | (s1 << 16);
+                return make_uint4(s2, s2, s2, s2);
+            }
+            return __ldg(scales + row);
         };
         uint4 sc_next = fetch_scales(0);
         for (int j = 0; j < n_my; ++j, cur.advance(1)) {

@@ -47,7 +47,7 @@ constexpr int kGroup = 32;
 constexpr int kThreads = 576;              // producer, mma, 16 epilogue warps
 constexpr int kEpiWarps = 16;
 constexpr int kBlockBytes = kTile * 128;   // one K block of the x tile: 128 rows x 128 B
-constexpr int kCtrlBytes = 256;
+constexpr int kCtrlBytes = 4608;            // barriers and flags, then the row maxima the two half-row threads trade
 constexpr int kSmemLimit = 232448;         // 227 KB of dynamic shared memory per CTA
 constexpr uint32_t kTmemCols = 512;
 
@@ -81,8 +81,11 @@ struct Ctrl {
     uint64_t in_full[4];
     uint64_t acc_full[4], acc_empty[4];
     uint64_t b_first, b_ready;
+    uint64_t pair[2][4];        // one scale per vector: the two warps that share 32 rows of a set meet here, once per tile
     uint32_t tmem_base;
     volatile uint32_t abort;
+    uint32_t pad[2];
+    float rowmax[2][2][2][kTile];   // [tile parity within the set][set][half row][row]
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
 
@@ -194,7 +197,8 @@ struct UmmaEncodeParams {
     uint32_t *amax_bits;        // calibration only: [D] running column maxima as fp32 bit patterns (start at zero)
 };
 
-template <int D, bool BF16, bool CALIB>
+// PERVEC: one scale per vector (group = D; Sec. 3.2 step 3, Sec. 4.1) instead of one per 32 channels.
+template <int D, bool BF16, bool CALIB, bool PERVEC>
 __global__ void __launch_bounds__(kThreads, 1)
     kvq_encode_umma_kernel(const __grid_constant__ UmmaEncodeParams prm, const __grid_constant__ CUtensorMap tm_x)
 {
@@ -216,6 +220,8 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
         mbar_init(smem_u32(&ctrl->b_first), kEpiWarps);       // first B: all epilogue warps build it
         mbar_init(smem_u32(&ctrl->b_ready), kEpiWarps / 2);   // later rebuilds: the set that owns the tile
+        for (int s = 0; s < 2; ++s)
+            for (int qq = 0; qq < 4; ++qq) mbar_init(smem_u32(&ctrl->pair[s][qq]), 2);
         ctrl->abort = 0u;
         mbar_init_fence();
     }
@@ -381,6 +387,38 @@ __global__ void __launch_bounds__(kThreads, 1)
             if (seg_rows > rpl) seg_rows = rpl;
             const bool live = off + r < seg_rows;
             const int64_t orow = prm.out_map(seg * rpl + off + r);
+            // ---- one scale per vector: the row's maximum first (this thread's half, then the other half's through
+            // ---- shared memory), then a second pass over the accumulator for the codes
+            float row_rs = 0.0f;
+            bool row_clamp = false;
+            if constexpr (PERVEC) {
+                float m = 0.0f;
+#pragma unroll
+                for (int gi = 0; gi < C::kGroupsPerPart; ++gi) {
+                    const int g = g0 + gi;
+                    if (g < g1) {
+                        uint32_t vb[32];
+                        tmem_ld32(t_addr + (uint32_t)sc * C::kAccStride + (uint32_t)(g * kGroup), vb);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) m = fmaxf(m, fabsf(__uint_as_float(vb[i])));
+                    }
+                }
+                const int it = (j - set) >> 1;   // this set's tile count: parity of the pair barrier and of the buffer
+                ctrl->rowmax[it & 1][set][h][r] = m;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctrl->pair[set][q]));
+                if (!wait_or_abort(smem_u32(&ctrl->pair[set][q]), (uint32_t)it & 1u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT)) break;
+                m = fmaxf(m, ctrl->rowmax[it & 1][set][h ^ 1][r]);
+                const float amax = m * unlift;
+                const float sig = fminf(__fdiv_rn(amax, 7.0f), 65504.0f);
+                const __half hs = __float2half_rn(sig);
+                const float sg = __half2float(hs);
+                const float rs1 = sg > 0.0f ? __frcp_rn(sg) : 0.0f;
+                row_clamp = !(amax * rs1 < 7.25f);
+                row_rs = rs1 * unlift;
+                if (live && h == 0) prm.scales[orow] = __half_as_ushort(hs);
+            }
 #pragma unroll
             for (int gi = 0; gi < C::kGroupsPerPart; ++gi) {
                 const int g = g0 + gi;       // warp-uniform
@@ -403,16 +441,21 @@ __global__ void __launch_bounds__(kThreads, 1)
                         continue;
                     }
                     // ---- scale: sigma = fp16(absmax / 7); codes are taken against the stored value
-                    float amax = 0.0f;
+                    float rs = row_rs;
+                    bool clamp = row_clamp;
+                    __half hs = __float2half_rn(0.0f);
+                    if constexpr (!PERVEC) {
+                        float amax = 0.0f;
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) amax = fmaxf(amax, fabsf(__uint_as_float(vb[i])));
-                    amax *= unlift;
-                    const float sig = fminf(__fdiv_rn(amax, 7.0f), 65504.0f);
-                    const __half hs = __float2half_rn(sig);
-                    const float sg = __half2float(hs);
-                    const float rs1 = sg > 0.0f ? __frcp_rn(sg) : 0.0f;
-                    const bool clamp = !(amax * rs1 < 7.25f);   // saturated or subnormal scale: codes could leave [-7, 7]
-                    const float rs = rs1 * unlift;              // applies to the lifted accumulator values
+                        for (int i = 0; i < 32; ++i) amax = fmaxf(amax, fabsf(__uint_as_float(vb[i])));
+                        amax *= unlift;
+                        const float sig = fminf(__fdiv_rn(amax, 7.0f), 65504.0f);
+                        hs = __float2half_rn(sig);
+                        const float sg = __half2float(hs);
+                        const float rs1 = sg > 0.0f ? __frcp_rn(sg) : 0.0f;
+                        clamp = !(amax * rs1 < 7.25f);   // saturated or subnormal scale: codes could leave [-7, 7]
+                        rs = rs1 * unlift;               // applies to the lifted accumulator values
+                    }
 
                     // ---- round, bias to unsigned nibbles, pack 8 codes per word
                     uint32_t words[4];
@@ -432,7 +475,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                     }
                     if (live) {
                         *reinterpret_cast<uint4 *>(prm.packed + orow * (D / 2) + g * 16) = make_uint4(words[0], words[1], words[2], words[3]);
-                        prm.scales[orow * G + g] = __half_as_ushort(hs);
+                        if constexpr (!PERVEC) prm.scales[orow * G + g] = __half_as_ushort(hs);
                     }
                 }
             }
@@ -457,7 +500,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 // ------------------------------------------------------------------------------------------------
 namespace {
 
-template <int D, bool BF16, bool CALIB = false>
+template <int D, bool BF16, bool CALIB = false, bool PERVEC = false>
 cudaError_t launch(int64_t N, const FftParams &f, const float *e0, cudaStream_t stream, uint32_t *amax_bits = nullptr)
 {
     using C = Cfg<D, BF16, CALIB>;
@@ -468,7 +511,7 @@ cudaError_t launch(int64_t N, const FftParams &f, const float *e0, cudaStream_t 
     int &sms = slots.sms[dev];
     if (sms == 0) {
         int n = 0;
-        if ((e = cudaFuncSetAttribute(kvq_encode_umma_kernel<D, BF16, CALIB>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes)) != cudaSuccess) return e;
+        if ((e = cudaFuncSetAttribute(kvq_encode_umma_kernel<D, BF16, CALIB, PERVEC>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes)) != cudaSuccess) return e;
         if ((e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
         sms = n;
     }
@@ -498,7 +541,7 @@ cudaError_t launch(int64_t N, const FftParams &f, const float *e0, cudaStream_t 
 
     const int64_t tiles = prm.n_seg * ((prm.rpl + kTile - 1) / kTile);
     const int grid = (int)(tiles < sms ? tiles : sms);
-    kvq_encode_umma_kernel<D, BF16, CALIB><<<grid, kThreads, C::kSmemBytes, stream>>>(prm, tm_x);
+    kvq_encode_umma_kernel<D, BF16, CALIB, PERVEC><<<grid, kThreads, C::kSmemBytes, stream>>>(prm, tm_x);
     count_launch();
     return cudaGetLastError();
 }
@@ -507,9 +550,21 @@ cudaError_t launch(int64_t N, const FftParams &f, const float *e0, cudaStream_t 
 
 bool umma_encode_supported(int D, bool bf16) { return D == 64 || D == 96 || D == 128 || D == 256 || (D == 160 && !bf16); }
 
-cudaError_t umma_encode(int D, bool bf16, int64_t N, const FftParams &f, const float *e0, cudaStream_t stream)
+// one scale per vector: the row maximum is traded inside a CTA, which the D = 256 kernel (a row split over two CTAs) cannot do
+bool umma_encode_per_vector_supported(int D, bool bf16) { return D != 256 && umma_encode_supported(D, bf16); }
+
+cudaError_t umma_encode(int D, bool bf16, bool per_vector, int64_t N, const FftParams &f, const float *e0, cudaStream_t stream)
 {
     if (!tensor_map_encode_fn()) return cudaErrorNotSupported;
+    if (per_vector) {
+        switch (D) {
+            case 64: return bf16 ? launch<64, true, false, true>(N, f, e0, stream) : launch<64, false, false, true>(N, f, e0, stream);
+            case 96: return bf16 ? launch<96, true, false, true>(N, f, e0, stream) : launch<96, false, false, true>(N, f, e0, stream);
+            case 128: return bf16 ? launch<128, true, false, true>(N, f, e0, stream) : launch<128, false, false, true>(N, f, e0, stream);
+            case 160: return bf16 ? cudaErrorInvalidValue : launch<160, false, false, true>(N, f, e0, stream);
+        }
+        return cudaErrorInvalidValue;
+    }
     if (D == 256) return umma_encode_d256(bf16, N, f, e0, stream);   // its own kernel: CTA pairs, x through a ring of K blocks
     switch (D) {
         case 64: return bf16 ? launch<64, true>(N, f, e0, stream) : launch<64, false>(N, f, e0, stream);
