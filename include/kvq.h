@@ -53,7 +53,7 @@ typedef enum { KVQ_F16 = 0, KVQ_BF16 = 1 } kvq_dtype_t;
 
 /* Which kernel family serves a call.  AUTO picks by size and shape: the matrix-vector kernel for calls of up to
  * 2048 rows (1024 for D > 128; such calls are latency-bound), beyond that the tensor-core kernel where one is built for the plan's D and
- * layout and the call's dtype (for kvq_encode / kvq_append from 4096 rows on), else the register FFT. */
+ * layout and the call's dtype, else the register FFT. */
 typedef enum {
     KVQ_IMPL_AUTO = 0,
     KVQ_IMPL_FFT = 1,   /* fp32 register FFT, one thread per vector: every D, dtype and layout; no rotation */

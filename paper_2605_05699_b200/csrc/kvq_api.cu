@@ -24,7 +24,6 @@ static inline uint64_t splitmix64_at(uint64_t seed, uint64_t n)
 }
 
 // AUTO sends kvq_encode / kvq_append calls of at least this many rows to the tensor-core kernel.
-constexpr int64_t kGemmEncodeMinRows = 4096;
 // calls up to this size are latency-bound: matrix-vector kernel (measured cross-over with the other two families)
 static int64_t matvec_max_rows(int D) { return D <= 128 ? 2048 : 1024; }
 
@@ -340,13 +339,13 @@ static kvq_status_t encode_common(kvq_plan_t *plan, const void *x, kvq_dtype_t d
     prm.packed = packed;
     prm.scales = scales;
     prm.out_map = out_map;
-    // AUTO: the matrix-vector kernel for small calls (latency), the tensor-core kernel from kGemmEncodeMinRows rows on
-    // (it pays a fixed operand build per launch), the register FFT in between and where no tensor-core kernel is built.
-    // A rotated plan has no FFT path: matrix-vector wherever the tensor-core kernel does not apply.
+    // AUTO: the matrix-vector kernel for small calls (latency), beyond that the tensor-core kernel (measured faster than
+    // the register FFT at every size above the matrix-vector limit), the register FFT where no tensor-core kernel is
+    // built.  A rotated plan has no FFT path: matrix-vector wherever the tensor-core kernel does not apply.
     kvq_impl_t impl = plan->enc_impl;
     if (impl == KVQ_IMPL_AUTO) {
         if (N <= matvec_max_rows(plan->D)) impl = KVQ_IMPL_MATVEC;
-        else if (gemm_ok && (plan->rot || N >= kGemmEncodeMinRows)) impl = KVQ_IMPL_GEMM;
+        else if (gemm_ok) impl = KVQ_IMPL_GEMM;
         else impl = plan->rot ? KVQ_IMPL_MATVEC : KVQ_IMPL_FFT;
     }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
