@@ -26,6 +26,7 @@ KVQ_ERR_CUDA = 4
 KVQ_ERR_TIMEOUT = 5
 KVQ_ERR_NOMEM = 6
 KVQ_ERR_SCRATCH_LIMIT = 7
+KVQ_ERR_RANGE = 8
 
 KVQ_F16 = 0
 KVQ_BF16 = 1
@@ -218,7 +219,7 @@ def kvq_plan_set_impl(plan: int, encode_impl: int, decode_impl: int) -> None:
 def kvq_plan_device_status(plan: int) -> int:
     w = ctypes.c_uint32()
     st = lib().kvq_plan_device_status(plan, ctypes.byref(w))
-    if st not in (KVQ_OK, KVQ_ERR_TIMEOUT):
+    if st not in (KVQ_OK, KVQ_ERR_TIMEOUT, KVQ_ERR_RANGE):
         raise KvqError(st, "kvq_plan_device_status")
     return int(w.value)
 

@@ -313,7 +313,8 @@ kvq_status_t kvq_plan_device_status(kvq_plan_t *plan, uint32_t *word)
         (void)cudaGetLastError();
         return KVQ_ERR_CUDA;
     }
-    return *word ? KVQ_ERR_TIMEOUT : KVQ_OK;
+    if (*word & 7u) return KVQ_ERR_TIMEOUT;
+    return *word ? KVQ_ERR_RANGE : KVQ_OK;
 }
 
 static kvq_status_t encode_common(kvq_plan_t *plan, const void *x, kvq_dtype_t dtype, int64_t N, const float *lambda,
@@ -521,6 +522,7 @@ const char *kvq_status_string(kvq_status_t status)
         case KVQ_ERR_TIMEOUT: return "KVQ_ERR_TIMEOUT";
         case KVQ_ERR_NOMEM: return "KVQ_ERR_NOMEM";
         case KVQ_ERR_SCRATCH_LIMIT: return "KVQ_ERR_SCRATCH_LIMIT";
+        case KVQ_ERR_RANGE: return "KVQ_ERR_RANGE";
     }
     return "KVQ_ERR_UNKNOWN";
 }

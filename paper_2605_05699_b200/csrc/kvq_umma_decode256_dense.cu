@@ -373,7 +373,10 @@ __global__ void __launch_bounds__(kThreads, 1)
                 for (int cc = 0; cc < 4; ++cc) {
                     const int c = 4 * kh + cc;   // group: 32 codes, 16 tensor-memory columns
                     const float sig = __half2float(__ushort_as_half((unsigned short)((sc[c >> 1] >> (16 * (c & 1))) & 0xFFFFu)));
-                    const __half2 s2 = __float2half2_rn(sig * rho);
+                    const float sr = sig * rho;
+                const __half2 s2 = __float2half2_rn(sr);
+                // the A operand q sigma rho is fp16: it overflows beyond 7 sr = 65504 and loses bits once sr is subnormal
+                if (sr != 0.0f && (sr > 9357.0f || sr < 6.1035156e-5f)) atomicOr(status, KVQ_DEV_RANGE);
                     const uint32_t words[4] = {pk[c].x, pk[c].y, pk[c].z, pk[c].w};
                     uint32_t a_hi[16], a_lo[16];
 #pragma unroll

@@ -91,7 +91,7 @@ def rel_l2_rows(a, b):
     return np.where(den > 0, num / np.where(den > 0, den, 1.0), num)
 
 
-def check_decode(gpu_bits, ora_bits, ora_f64, dtype, label=""):
+def check_decode(gpu_bits, ora_bits, ora_f64, dtype, label="", max_tie_rows=0.05):
     """gpu_bits / ora_bits: raw uint16 bits of the half-precision outputs [N, D]; ora_f64: the oracle's
     reconstruction before its rounding to the output dtype.
 
@@ -101,7 +101,8 @@ def check_decode(gpu_bits, ora_bits, ora_f64, dtype, label=""):
     such flip on a dominant channel is already 4e-3 of the vector norm.  A vector that fails the plain
     comparison is therefore compared again without the elements where the two outputs are neighbours in
     the format and the exact value lies within 1e-3 of the vector's rms from their midpoint; it must
-    then pass, and such vectors must be rare.
+    then pass, and such vectors must be rare (``max_tie_rows``; a test made of vectors whose outputs sit in the format's
+    subnormal range, where one ulp is a large part of the value, raises it).
     """
     gb = np.ascontiguousarray(gpu_bits).view(np.uint16)
     g = ko.widen(gb, dtype)
@@ -124,7 +125,7 @@ def check_decode(gpu_bits, ora_bits, ora_f64, dtype, label=""):
         assert rel.max() <= REL_L2, label + ": reconstruction relative L2 %.3g (plain %.3g)" % (rel.max(), plain.max())
         worst = max(worst, float(rel.max()))
     frac = float(need.mean()) if need.size else 0.0
-    assert frac < 0.05, label + ": %.3g of the vectors pass only with the output-tie rule" % frac
+    assert frac < max_tie_rows, label + ": %.3g of the vectors pass only with the output-tie rule" % frac
     return {"rel_l2_max": worst, "rel_l2_plain_max": float(plain.max(initial=0)),
             "rel_l2_plain_mean": float(plain.mean()) if plain.size else 0.0, "rows_needing_tie_rule": frac,
             "bit_equal": float((gb == ora_bits).mean()) if g.size else 1.0}

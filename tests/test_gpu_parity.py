@@ -36,6 +36,15 @@ def gpu_decode(plan, packed, scales, lam, dtype, rows_per_lambda=0):
     return out
 
 
+def gpu_decode_raw(plan, packed, scales, lam, dtype, rows_per_lambda=0):
+    """gpu_decode without the finiteness assumption of the callers that follow it with check_decode on every row."""
+    out = torch.empty(packed.shape[0], plan.D, dtype=wl.torch_dtype(dtype), device="cuda")
+    kb.kvq_decode(plan.handle, packed, scales, lam, out, rows_per_lambda)
+    torch.cuda.synchronize()
+    assert kb.kvq_plan_device_status(plan.handle) & 7 == 0     # no bounded wait ran out; bit 3 (number range) is the caller's to judge
+    return out
+
+
 IMPL = {"auto": kb.KVQ_IMPL_AUTO, "fft": kb.KVQ_IMPL_FFT, "gemm": kb.KVQ_IMPL_GEMM, "matvec": kb.KVQ_IMPL_MATVEC}
 
 
@@ -621,6 +630,74 @@ def test_rotation_can_be_set_and_removed_on_a_plan_in_use():
                               rot=Rv.numpy().astype(np.float64))
         parity.check_decode(bits(outv), obv, o64v, odt, "rotated, no tensor-core kernel")
         p.close()
+
+
+# ---- degenerate inputs: zero vectors, zero / subnormal / saturated scales, single spikes, pure tones ------------------
+
+def _degenerate_rows(D, dtype):
+    tdt = torch.float16 if dtype == "f16" else torch.bfloat16
+    n = torch.arange(D, dtype=torch.float64)
+    rows = [torch.zeros(D, dtype=torch.float64)]                                   # scale 0, codes 0
+    rows.append(torch.ones(D, dtype=torch.float64))                                # DC only
+    rows.append(torch.where(n % 2 == 0, 1.0, -1.0).to(torch.float64))              # Nyquist only
+    rows.append(torch.cos(2 * np.pi * 5 * n / D))                                  # one bin
+    for pos, val in ((0, 1.0), (D - 1, -3.0), (D // 2, 2.0 ** -14), (7, 6.0e-8 if dtype == "f16" else 1e-30)):
+        e = torch.zeros(D, dtype=torch.float64)
+        e[pos] = val
+        rows.append(e)                                                            # spikes: flat spectrum, down to subnormal scales
+    g = torch.Generator().manual_seed(5)
+    noise = torch.randn(D, generator=g, dtype=torch.float64)
+    rows.append(noise * 1e-6)                                                      # fp16 scale in its subnormal range: codes are clamped
+    rows.append(noise * 2e-8)                                                      # scale rounds to zero or to the smallest subnormal
+    rows.append(noise * (1.5e4 if dtype == "f16" else 1e20))                       # abs-max / 7 beyond fp16: the scale saturates at 65504
+    rows.append(noise * (6.0e4 / float(noise.abs().max())) if dtype == "f16" else noise * 1e30)
+    rows.append(noise)
+    x = torch.stack(rows).to(tdt)
+    return x.repeat(23, 1)                                                         # 299 rows: three tiles, the last one ragged
+
+
+@pytest.mark.parametrize("impl", ["fft", "gemm", "matvec"])
+@pytest.mark.parametrize("D,dtype", [(128, "f16"), (128, "bf16"), (64, "f16"), (256, "bf16")])
+def test_degenerate_inputs(D, dtype, impl):
+    odt = ko.F16 if dtype == "f16" else ko.BF16
+    x = _degenerate_rows(D, dtype)
+    for lam in (torch.ones(1, D), wl.make_lambda(1, D, 18), 16.0 * wl.make_lambda(1, D, 19)):   # x16: saturated scales in fp16 too
+        plan = kb.Plan(D, G, 17)                                                  # a plan each: the status word is sticky
+        kb.kvq_plan_set_impl(plan.handle, IMPL[impl], IMPL[impl])
+        sg = plan.signs()
+        packed, scales = gpu_encode(plan, x.cuda(), lam.cuda())
+        assert bool(torch.isfinite(scales).all())
+        ora = ko.encode(bits(x), odt, sg, lam.numpy(), G, want_v=True)
+        pk, sb = packed.cpu().numpy(), bits(scales)
+        parity.check_encode(pk, sb, ora, G, "degenerate encode (%s)" % impl, min_agree=0.999)
+        assert not pk[0::13].any() and not sb[0::13].any()                         # the zero vector: zero scales, zero codes
+        # decode what the oracle stored, so that both sides start from the same bytes; rows whose reconstruction leaves
+        # the output format's range are compared on the oracle's finite rows only
+        ob, o64 = ko.decode(ora["packed"], ora["scales"], sg, lam.numpy(), G, odt, want_f64=True)
+        out = gpu_decode_raw(plan, torch.from_numpy(ora["packed"]).cuda(),
+                             torch.from_numpy(ora["scales"].view(np.int16)).view(torch.float16).cuda(), lam.cuda(), dtype)
+        # the tensor-core decode carries q sigma rho as an fp16 operand (rho: the power of two at or below the largest
+        # 1 / lambda): outside fp16's normal range it says so in the status word (bit 3) instead of giving the row;
+        # the other families are fp32 there
+        fp16_operands = impl == "gemm"
+        lim = 65504.0 if dtype == "f16" else 3.0e38
+        ok = np.abs(o64).max(axis=1) < 0.25 * lim
+        if fp16_operands:
+            rho = 2.0 ** np.floor(np.log2(1.0 / float(lam.min())))
+            sr = ko.f16_to_f64(ora["scales"]) * rho
+            in_range = ((sr == 0) | ((sr >= 2.0 ** -14) & (sr <= 9357.0))).all(axis=1)
+            assert 0.5 * len(ok) <= in_range.sum() < len(ok)
+            ok &= in_range
+        assert ok.sum() >= 0.5 * len(ok)
+        # several of these rows reconstruct to values in the output format's subnormal range, where neighbouring
+        # roundings are a large part of the value: the tie rule decides them, and they are not rare here by construction
+        parity.check_decode(bits(out)[ok], ob[ok], o64[ok], odt, "degenerate decode (%s)" % impl, max_tie_rows=0.5)
+        word = kb.kvq_plan_device_status(plan.handle)
+        if fp16_operands:
+            assert word == 8    # the rows outside the operand range were met and reported
+        else:
+            assert word == 0
+        plan.close()
 
 
 # ---- config 3: Gemma-3-1B-shaped, D = 256 bf16, prefix sweep ---------------------------------
