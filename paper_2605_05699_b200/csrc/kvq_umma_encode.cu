@@ -550,12 +550,13 @@ cudaError_t launch(int64_t N, const FftParams &f, const float *e0, cudaStream_t 
 
 bool umma_encode_supported(int D, bool bf16) { return D == 64 || D == 96 || D == 128 || D == 256 || (D == 160 && !bf16); }
 
-// one scale per vector: the row maximum is traded inside a CTA, which the D = 256 kernel (a row split over two CTAs) cannot do
-bool umma_encode_per_vector_supported(int D, bool bf16) { return D != 256 && umma_encode_supported(D, bf16); }
+// one scale per vector: the row maximum is traded inside a CTA, or across the cluster pair of the D = 256 kernel
+bool umma_encode_per_vector_supported(int D, bool bf16) { return umma_encode_supported(D, bf16); }
 
 cudaError_t umma_encode(int D, bool bf16, bool per_vector, int64_t N, const FftParams &f, const float *e0, cudaStream_t stream)
 {
     if (!tensor_map_encode_fn()) return cudaErrorNotSupported;
+    if (D == 256) return umma_encode_d256(bf16, per_vector, N, f, e0, stream);   // its own kernel: CTA pairs, x through a ring of K blocks
     if (per_vector) {
         switch (D) {
             case 64: return bf16 ? launch<64, true, false, true>(N, f, e0, stream) : launch<64, false, false, true>(N, f, e0, stream);
@@ -565,7 +566,6 @@ cudaError_t umma_encode(int D, bool bf16, bool per_vector, int64_t N, const FftP
         }
         return cudaErrorInvalidValue;
     }
-    if (D == 256) return umma_encode_d256(bf16, N, f, e0, stream);   // its own kernel: CTA pairs, x through a ring of K blocks
     switch (D) {
         case 64: return bf16 ? launch<64, true>(N, f, e0, stream) : launch<64, false>(N, f, e0, stream);
         case 96: return bf16 ? launch<96, true>(N, f, e0, stream) : launch<96, false>(N, f, e0, stream);

@@ -44,14 +44,17 @@ constexpr int kAccStages = 4;
 constexpr int kMaxRing = 6;
 
 // CALIB: the calibration pass keeps a third bf16 term (it runs once; its result is compared at 1e-6 of the vector norm)
-template <bool BF16, bool CALIB = false>
+// PERVEC: one scale per vector.  A row's 256 channels sit in two CTAs, so the pair runs as a thread-block cluster and
+// the four half-row maxima of a row (two warps in each CTA) meet in both CTAs' shared memory.
+template <bool BF16, bool CALIB = false, bool PERVEC = false>
 struct Cfg {
     static constexpr int kSplit = (BF16 && CALIB) ? 3 : 2;
     static constexpr int kBBytes = kSplit * kBTerm;
-    static constexpr int kRoom = (kSmemLimit - 1024 - kCtrlBytes - kBBytes) / kBlockBytes;
+    static constexpr int kMaxBytes = PERVEC ? 2 * 2 * 4 * kTile * (int)sizeof(float) : 0;   // [tile parity][set][party][row]
+    static constexpr int kRoom = (kSmemLimit - 1024 - kCtrlBytes - kMaxBytes - kBBytes) / kBlockBytes;
     static constexpr int kRing = kRoom < kMaxRing ? kRoom : kMaxRing;   // K blocks of x in flight: 6 (2 next to a three-term B)
     static_assert(kRing >= 2, "no room for the x ring");
-    static constexpr int kSmemBytes = kBBytes + kRing * kBlockBytes + kCtrlBytes + 1024;
+    static constexpr int kSmemBytes = kBBytes + kRing * kBlockBytes + kCtrlBytes + kMaxBytes + 1024;
     static constexpr uint32_t kIdesc = umma_idesc_m128(kHalfN, BF16);
 };
 
@@ -59,10 +62,58 @@ struct Ctrl {
     uint64_t in_full[kMaxRing], in_empty[kMaxRing];
     uint64_t acc_full[4], acc_empty[4];
     uint64_t b_first, b_ready;
+    uint64_t quad[2][4];        // one scale per vector: the four warps (two per CTA of the pair) that share 32 rows of a set
     uint32_t tmem_base;
     volatile uint32_t abort;
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
+
+// ---- thread-block cluster of two CTAs: the partner's shared memory and barriers (one scale per vector only)
+__device__ __forceinline__ uint32_t cluster_map(uint32_t smem_addr, uint32_t cta_rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(cta_rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_st_f32(uint32_t cluster_addr, float v)
+{
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(cluster_addr), "f"(v) : "memory");
+}
+__device__ __forceinline__ void cluster_mbar_arrive(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// wait_or_abort with cluster-scope acquire: the values the partner CTA stored before its arrive are visible afterwards
+__device__ __forceinline__ bool wait_cluster_or_abort(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *status,
+                                                      uint32_t reason)
+{
+    for (uint32_t it = 0; it < (1u << 22); ++it) {
+        if (mbar_try_wait_cluster(bar, parity)) return true;
+        if (it > 32) {
+            if (*abort_flag) return false;
+            __nanosleep(32);
+        }
+    }
+    *abort_flag = 1u;
+    atomicOr(status, reason);
+    return false;
+}
 
 // 2^k for a lambda row: the power of two that brings max_c lambda_c max|table entry| (sqrt(2 / D) without a rotation) into [2^13, 2^14), so that
 // the first split term of W 2^k stays below fp16's maximum and the later ones above its subnormals.
@@ -135,17 +186,17 @@ struct UmmaEncode256Params {
     uint32_t *amax_bits;        // calibration only: [D] running column maxima as fp32 bit patterns (start at zero)
 };
 
-template <bool BF16, bool CALIB>
-__global__ void __launch_bounds__(kThreads, 1)
-    kvq_encode_umma_d256_kernel(const __grid_constant__ UmmaEncode256Params prm, const __grid_constant__ CUtensorMap tm_x)
+template <bool BF16, bool CALIB, bool PERVEC>
+__device__ __forceinline__ void encode_d256_body(const UmmaEncode256Params &prm, const CUtensorMap &tm_x)
 {
-    using C = Cfg<BF16, CALIB>;
+    using C = Cfg<BF16, CALIB, PERVEC>;
     constexpr int kRing = C::kRing;
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     unsigned char *sB = smem;                                   // kSplit terms
     unsigned char *sIn = sB + C::kBBytes;                       // ring of K blocks of x
     Ctrl *ctrl = reinterpret_cast<Ctrl *>(sIn + kRing * kBlockBytes);
+    float *rowmax = reinterpret_cast<float *>(reinterpret_cast<unsigned char *>(ctrl) + kCtrlBytes);   // PERVEC: [parity][set][party][row]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int half = blockIdx.x & 1;            // which 128 channels this CTA computes
@@ -162,6 +213,8 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
         mbar_init(smem_u32(&ctrl->b_first), kEpiWarps);       // first B: all epilogue warps build it
         mbar_init(smem_u32(&ctrl->b_ready), kEpiWarps / 2);   // later rebuilds: the set that owns the tile
+        for (int s = 0; s < 2; ++s)
+            for (int qq = 0; qq < 4; ++qq) mbar_init(smem_u32(&ctrl->quad[s][qq]), 4);
         ctrl->abort = 0u;
         mbar_init_fence();
     }
@@ -170,6 +223,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    if constexpr (PERVEC) cluster_sync_all();   // the partner's barriers exist before anyone arrives on them
     const uint32_t tmem_base = ctrl->tmem_base;
     volatile uint32_t *abort_flag = &ctrl->abort;
     uint32_t *status = prm.status;
@@ -315,6 +369,43 @@ __global__ void __launch_bounds__(kThreads, 1)
             if (seg_rows > rpl) seg_rows = rpl;
             const bool live = off + r < seg_rows;
             const int64_t orow = prm.out_map(seg * rpl + off + r);
+            // ---- one scale per vector: this thread's maximum over its 64 channels goes to both CTAs of the pair; the four
+            // ---- parties of a row (two half-row threads in each CTA) meet on a four-arrival barrier in each CTA, once per
+            // ---- tile; buffers alternate with the tile parity, so a party cannot overwrite what another still reads
+            float row_rs = 0.0f;
+            bool row_clamp = false;
+            if constexpr (PERVEC) {
+                float m = 0.0f;
+#pragma unroll
+                for (int gi = 0; gi < 2; ++gi) {
+                    uint32_t vb[32];
+                    tmem_ld32(t_addr + (uint32_t)sc * kHalfN + (uint32_t)((g0 + gi) * kGroup), vb);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) m = fmaxf(m, fabsf(__uint_as_float(vb[i])));
+                }
+                const int it = (j - set) >> 1;                       // this set's tile count
+                float *slot = rowmax + (((it & 1) * 2 + set) * 4) * kTile;   // [party][row] of this buffer
+                const int party = 2 * half + h;
+                slot[party * kTile + r] = m;
+                cluster_st_f32(cluster_map(smem_u32(slot + party * kTile + r), (uint32_t)(half ^ 1)), m);
+                asm volatile("fence.acq_rel.cluster;" ::: "memory");   // every lane's stores before lane 0's arrives
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(smem_u32(&ctrl->quad[set][q]));
+                    cluster_mbar_arrive(cluster_map(smem_u32(&ctrl->quad[set][q]), (uint32_t)(half ^ 1)));
+                }
+                if (!wait_cluster_or_abort(smem_u32(&ctrl->quad[set][q]), (uint32_t)it & 1u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT)) break;
+                m = fmaxf(fmaxf(slot[r], slot[kTile + r]), fmaxf(slot[2 * kTile + r], slot[3 * kTile + r]));
+                const float amax = m * unlift;
+                const float sig = fminf(__fdiv_rn(amax, 7.0f), 65504.0f);
+                const __half hs = __float2half_rn(sig);
+                const float sg = __half2float(hs);
+                const float rs1 = sg > 0.0f ? __frcp_rn(sg) : 0.0f;
+                row_clamp = !(amax * rs1 < 7.25f);
+                row_rs = rs1 * unlift;
+                if (live && party == 0) prm.scales[orow] = __half_as_ushort(hs);
+            }
 #pragma unroll
             for (int gi = 0; gi < 2; ++gi) {
                 const int g = g0 + gi;       // warp-uniform; group within this CTA's half
@@ -337,16 +428,21 @@ __global__ void __launch_bounds__(kThreads, 1)
                         continue;
                     }
                     // ---- scale: sigma = fp16(absmax / 7); codes are taken against the stored value
-                    float amax = 0.0f;
+                    float rs = row_rs;
+                    bool clamp = row_clamp;
+                    __half hs = __float2half_rn(0.0f);
+                    if constexpr (!PERVEC) {
+                        float amax = 0.0f;
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) amax = fmaxf(amax, fabsf(__uint_as_float(vb[i])));
-                    amax *= unlift;
-                    const float sig = fminf(__fdiv_rn(amax, 7.0f), 65504.0f);
-                    const __half hs = __float2half_rn(sig);
-                    const float sg = __half2float(hs);
-                    const float rs1 = sg > 0.0f ? __frcp_rn(sg) : 0.0f;
-                    const bool clamp = !(amax * rs1 < 7.25f);   // saturated or subnormal scale: codes could leave [-7, 7]
-                    const float rs = rs1 * unlift;              // applies to the lifted accumulator values
+                        for (int i = 0; i < 32; ++i) amax = fmaxf(amax, fabsf(__uint_as_float(vb[i])));
+                        amax *= unlift;
+                        const float sig = fminf(__fdiv_rn(amax, 7.0f), 65504.0f);
+                        hs = __float2half_rn(sig);
+                        const float sg = __half2float(hs);
+                        const float rs1 = sg > 0.0f ? __frcp_rn(sg) : 0.0f;
+                        clamp = !(amax * rs1 < 7.25f);   // saturated or subnormal scale: codes could leave [-7, 7]
+                        rs = rs1 * unlift;               // applies to the lifted accumulator values
+                    }
 
                     // ---- round, bias to unsigned nibbles, pack 8 codes per word
                     uint32_t words[4];
@@ -367,7 +463,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                     if (live) {
                         const int gg = 4 * half + g;   // group within the row
                         *reinterpret_cast<uint4 *>(prm.packed + orow * (kD / 2) + gg * 16) = make_uint4(words[0], words[1], words[2], words[3]);
-                        prm.scales[orow * kG + gg] = __half_as_ushort(hs);
+                        if constexpr (!PERVEC) prm.scales[orow * kG + gg] = __half_as_ushort(hs);
                     }
                 }
             }
@@ -385,6 +481,22 @@ __global__ void __launch_bounds__(kThreads, 1)
         if (*abort_flag) __nanosleep(20000);   // let tensor-core work that was already issued drain
         tmem_dealloc(tmem_base, kTmemCols);
     }
+    if constexpr (PERVEC) cluster_sync_all();   // neither CTA leaves while the other may still store into its shared memory
+}
+
+template <bool BF16, bool CALIB>
+__global__ void __launch_bounds__(kThreads, 1)
+    kvq_encode_umma_d256_kernel(const __grid_constant__ UmmaEncode256Params prm, const __grid_constant__ CUtensorMap tm_x)
+{
+    encode_d256_body<BF16, CALIB, false>(prm, tm_x);
+}
+
+// one scale per vector: the same body with the CTA pair as a cluster (launched with a cluster dimension of 2)
+template <bool BF16>
+__global__ void __launch_bounds__(kThreads, 1)
+    kvq_encode_umma_d256_pv_kernel(const __grid_constant__ UmmaEncode256Params prm, const __grid_constant__ CUtensorMap tm_x)
+{
+    encode_d256_body<BF16, false, true>(prm, tm_x);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -392,10 +504,14 @@ __global__ void __launch_bounds__(kThreads, 1)
 // ------------------------------------------------------------------------------------------------
 namespace {
 
-template <bool BF16, bool CALIB = false>
+template <bool BF16, bool CALIB = false, bool PERVEC = false>
 cudaError_t launch(int64_t N, const FftParams &f, const float *e0, cudaStream_t stream, uint32_t *amax_bits = nullptr)
 {
-    using C = Cfg<BF16, CALIB>;
+    using C = Cfg<BF16, CALIB, PERVEC>;
+    auto kern = [] {
+        if constexpr (PERVEC) return kvq_encode_umma_d256_pv_kernel<BF16>;
+        else return kvq_encode_umma_d256_kernel<BF16, CALIB>;
+    }();
     static DeviceSlots slots;
     int dev = 0;
     cudaError_t e = current_device_slot(&dev);
@@ -403,7 +519,7 @@ cudaError_t launch(int64_t N, const FftParams &f, const float *e0, cudaStream_t 
     int &sms = slots.sms[dev];
     if (sms == 0) {
         int n = 0;
-        if ((e = cudaFuncSetAttribute(kvq_encode_umma_d256_kernel<BF16, CALIB>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes)) != cudaSuccess) return e;
+        if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes)) != cudaSuccess) return e;
         if ((e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
         sms = n;
     }
@@ -432,17 +548,45 @@ cudaError_t launch(int64_t N, const FftParams &f, const float *e0, cudaStream_t 
         return cudaErrorInvalidValue;
 
     const int64_t tiles = prm.n_seg * ((prm.rpl + kTile - 1) / kTile);
-    const int64_t pairs = tiles < sms / 2 ? tiles : sms / 2;
-    kvq_encode_umma_d256_kernel<BF16, CALIB><<<(int)(2 * pairs), kThreads, C::kSmemBytes, stream>>>(prm, tm_x);
+    int64_t pairs = tiles < sms / 2 ? tiles : sms / 2;
+    if constexpr (PERVEC) {
+        // the pair is a cluster of two CTAs: as many pairs as the device holds at once (SMs of a cluster share a GPC)
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)sms, 1, 1);
+        cfg.blockDim = dim3(kThreads, 1, 1);
+        cfg.dynamicSmemBytes = C::kSmemBytes;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int &fit = slots.blocks_per_sm[dev];   // clusters resident at once, looked up once per device
+        if (fit == 0) {
+            int n = 0;
+            if ((e = cudaOccupancyMaxActiveClusters(&n, kern, &cfg)) != cudaSuccess) return e;
+            if (n < 1) return cudaErrorLaunchOutOfResources;
+            fit = n;
+        }
+        if (pairs > fit) pairs = fit;
+        cfg.gridDim = dim3((unsigned)(2 * pairs), 1, 1);
+        e = cudaLaunchKernelEx(&cfg, kern, prm, tm_x);
+        count_launch();
+        return e != cudaSuccess ? e : cudaGetLastError();
+    }
+    kern<<<(int)(2 * pairs), kThreads, C::kSmemBytes, stream>>>(prm, tm_x);
     count_launch();
     return cudaGetLastError();
 }
 
 }  // namespace
 
-cudaError_t umma_encode_d256(bool bf16, int64_t N, const FftParams &f, const float *e0, cudaStream_t stream)
+cudaError_t umma_encode_d256(bool bf16, bool per_vector, int64_t N, const FftParams &f, const float *e0, cudaStream_t stream)
 {
     if (!tensor_map_encode_fn()) return cudaErrorNotSupported;
+    if (per_vector) return bf16 ? launch<true, false, true>(N, f, e0, stream) : launch<false, false, true>(N, f, e0, stream);
     return bf16 ? launch<true>(N, f, e0, stream) : launch<false>(N, f, e0, stream);
 }
 

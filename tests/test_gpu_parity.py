@@ -480,15 +480,14 @@ def test_base_variants_per_vector_scale_and_byte_codes(D, dtype, per_vector, nbi
 @pytest.mark.parametrize("D,dtype,N,n_lambda,rpl", [
     (128, "f16", 20000, 1, 0), (128, "f16", 40000, 200, 200), (128, "bf16", 20000, 3, 7000), (64, "f16", 9000, 1, 0),
     (64, "bf16", 9000, 2, 4500), (96, "f16", 9000, 1, 0), (96, "bf16", 5000, 1, 0), (160, "f16", 9000, 4, 2300),
-    (256, "f16", 9000, 1, 0), (256, "bf16", 9000, 3, 3100),
+    (256, "f16", 9000, 1, 0), (256, "bf16", 9000, 3, 3100), (256, "bf16", 60000, 300, 200), (256, "f16", 129, 1, 0),
 ])
 def test_one_scale_per_vector_on_the_tensor_cores(D, dtype, N, n_lambda, rpl):
-    # group = D, 4-bit codes: the tensor-core encode trades the row maximum between its two half-row threads (D <= 160;
-    # D = 256 encodes on the register FFT), the tensor-core decode reads one scale per row (every D)
+    # group = D, 4-bit codes: the tensor-core encode trades the row maximum between its two half-row threads (D <= 160)
+    # or between the four of a cluster pair (D = 256), the tensor-core decode reads one scale per row
     odt = ko.F16 if dtype == "f16" else ko.BF16
     plan = kb.Plan(D, D, 60 + D)
-    enc_impl = kb.KVQ_IMPL_FFT if D == 256 else kb.KVQ_IMPL_GEMM
-    kb.kvq_plan_set_impl(plan.handle, enc_impl, kb.KVQ_IMPL_GEMM)
+    kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_GEMM, kb.KVQ_IMPL_GEMM)
     sg = plan.signs()
     lam = wl.make_lambda(n_lambda, D, 61)
     x = wl.make_vectors(N, D, dtype, "k_outlier", 62 + N)
