@@ -47,8 +47,8 @@ typedef enum {
     KVQ_ERR_TIMEOUT = 5,         /* a bounded device-side wait ran out (see kvq_plan_device_status) */
     KVQ_ERR_NOMEM = 6,
     KVQ_ERR_SCRATCH_LIMIT = 7,   /* the plan needs more fixed scratch than kvq_decode_static holds */
-    KVQ_ERR_RANGE = 8            /* a tensor-core decode met a stored scale outside its operand range (see
-                                    kvq_plan_device_status) */
+    KVQ_ERR_RANGE = 8            /* the dense D = 256 decode of a rotated plan met a stored scale outside its
+                                    operand range (see kvq_plan_device_status) */
 } kvq_status_t;
 
 typedef enum { KVQ_F16 = 0, KVQ_BF16 = 1 } kvq_dtype_t;
@@ -129,14 +129,13 @@ kvq_status_t kvq_plan_set_impl(kvq_plan_t *plan, kvq_impl_t encode_impl, kvq_imp
 /* Synchronizes the current device and returns the plan's device status word through *word
  * (host): 0 when no kernel using this plan ever gave up a bounded wait or left its number
  * range.  Bits 0-2: a bounded wait ran out (load, tensor-core commit, pipeline slot): returns
- * KVQ_ERR_TIMEOUT.  Bit 3: a tensor-core kvq_decode met a non-zero stored scale sigma with
- * sigma rho outside [2^-14, 9357], rho the power of two at or below the lambda row's largest
- * 1 / max(lambda, 1e-6).  That kernel carries q sigma / lambda as an fp16 operand: above the
- * range it overflows (an fp16 output could not hold the result either), below it the operand is
- * subnormal and the row loses relative precision (vectors of magnitude below about 1e-3 / rho).
- * Zero scales are exact.  Decode such data with KVQ_IMPL_FFT or KVQ_IMPL_MATVEC (fp32
- * throughout).  Returns KVQ_ERR_RANGE if that is the only bit set.  The word is sticky for the
- * plan's lifetime. */
+ * KVQ_ERR_TIMEOUT.  Bit 3: the dense D = 256 tensor-core decode of a ROTATED plan met a non-zero
+ * stored scale sigma with sigma rho outside [2^-14, 9357], rho the power of two at or below the
+ * lambda row's largest 1 / max(lambda, 1e-6).  The tensor-core decode kernels carry
+ * q sigma / lambda as an fp16 operand; all but that one rescale such rows (very small or very
+ * large vectors) by a power of two and are exact for them, that one reports them here and the
+ * rows concerned are wrong: decode such data with KVQ_IMPL_MATVEC.  Returns KVQ_ERR_RANGE if
+ * that is the only bit set.  The word is sticky for the plan's lifetime. */
 kvq_status_t kvq_plan_device_status(kvq_plan_t *plan, uint32_t *word);
 
 /*

@@ -48,7 +48,8 @@ constexpr int kTile = 128;       // vectors per tile = MMA M
 constexpr int kThreads = 576;    // producer, mma, 2 x 4 dequant, 2 x 4 epilogue warps
 constexpr int kInStages = 6;     // packed tiles in flight
 constexpr int kAccStages = 2;    // accumulators in tensor memory
-constexpr int kCtrlBytes = 256;
+constexpr int kCtrlBytes = 4608;   // barriers and flags, then eight tiles' worth of per-row output scales
+constexpr int kRowScaleSlots = 8;  // a dequant group is never more than seven tiles ahead of the epilogue that reads its slot
 constexpr uint32_t kTmemCols = 512;
 
 // BF16OUT: bfloat16 output rounds 8x coarser than fp16, and a result that is off by 1e-4 of the vector's rms already
@@ -95,6 +96,7 @@ struct Ctrl {
     uint64_t b_first;
     uint32_t tmem_base;
     volatile uint32_t abort;
+    float row_scale[kRowScaleSlots][kTile];   // what the epilogue multiplies a row by (1 unless its scales left fp16's comfort zone)
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
 
@@ -442,16 +444,36 @@ __global__ void __launch_bounds__(kThreads, 1)
                 break;
             tc_fence_after();
 
+            // ---- the A operand q sigma rho is fp16.  A row whose scales would take it out of fp16's normal range (a very
+            // ---- small or very large vector) is carried times a power of two instead, which the epilogue takes out again
+            // ---- in fp32; every other row has the factor 1 and costs the epilogue nothing.
+            float pw = 1.0f;
+            {
+                uint32_t smax = 0u, smin = 0xFFFFu;
+#pragma unroll
+                for (int c = 0; c < G; ++c) {
+                    const uint32_t s = (sc[c >> 1] >> (16 * (c & 1))) & 0x7FFFu;   // fp16 bits of a non-negative number order like integers
+                    smax = max(smax, s);
+                    if (s != 0u) smin = min(smin, s);
+                }
+                const float tmax = __half2float(__ushort_as_half((unsigned short)smax)) * rho;
+                const float tmin = __half2float(__ushort_as_half((unsigned short)(smin == 0xFFFFu ? 0u : smin))) * rho;
+                float inv = 1.0f;
+                if (tmax > 9000.0f || (tmin != 0.0f && tmin < 6.1035156e-5f)) {
+                    // 2^floor(log2 tmax) -> 2^7: the largest operand lands in [896, 1792), sums of 128 of them stay inside fp16
+                    const int e = (int)((__float_as_uint(fminf(fmaxf(tmax, 1e-30f), 1e30f)) >> 23) & 0xFFu) - 127;
+                    pw = __uint_as_float((uint32_t)(127 + 7 - e) << 23);
+                    inv = __uint_as_float((uint32_t)(127 - 7 + e) << 23);
+                }
+                ctrl->row_scale[j & (kRowScaleSlots - 1)][r] = inv;
+            }
             // ---- nibbles -> fp16 codes -> times sigma * rho, two codes per instruction
             const uint32_t a_row = tmem_base + ((uint32_t)(q * 32) << 16) + C::a_col(sa);
             const __half2 h1032 = __float2half2_rn(1032.0f);
 #pragma unroll
             for (int c = 0; c < G; ++c) {   // chunk c = group c: 32 codes, 16 tensor-memory columns
                 const float sig = __half2float(__ushort_as_half((unsigned short)((sc[c >> 1] >> (16 * (c & 1))) & 0xFFFFu)));
-                const float sr = sig * rho;
-                const __half2 s2 = __float2half2_rn(sr);
-                // the A operand q sigma rho is fp16: it overflows beyond 7 sr = 65504 and loses bits once sr is subnormal
-                if (sr != 0.0f && (sr > 9357.0f || sr < 6.1035156e-5f)) atomicOr(status, KVQ_DEV_RANGE);
+                const __half2 s2 = __float2half2_rn(sig * rho * pw);
                 const uint32_t words[4] = {pk[c].x, pk[c].y, pk[c].z, pk[c].w};
                 uint32_t a[16], al[BF16OUT ? 16 : 1];
 #pragma unroll
@@ -474,6 +496,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             }
             tmem_st_wait();
             tc_fence_before();
+            __threadfence_block();   // the row scales, for the epilogue that follows this tile's accumulator
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctrl->a_full[sa]));
         }
@@ -490,11 +513,17 @@ __global__ void __launch_bounds__(kThreads, 1)
             tc_fence_after();
             if (lane == 0) bulk_wait_read_all();   // this warp's previous stores have read the staging tile
             __syncwarp();
+            const float row_inv = ctrl->row_scale[j & (kRowScaleSlots - 1)][q * 32 + lane];
+            const bool rescale = __any_sync(0xFFFFFFFFu, row_inv != 1.0f);   // rare: a row outside the operand's comfort zone
 #pragma unroll
             for (int cc = 0; cc < G; ++cc) {   // 32 accumulator columns = 64 bytes of the output row
                 uint32_t v[32];
                 tmem_ld32(lane_addr + C::acc_col(sc) + (uint32_t)cc * 32u, v);
                 tmem_ld_wait();
+                if (rescale) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * row_inv);
+                }
                 constexpr int kWideBoxes = G / 2;
                 const bool wide = (cc >> 1) < kWideBoxes;   // inside a 64-column box, or the last 32-column one
                 unsigned char *box = stg + (cc >> 1) * (32 * 128);

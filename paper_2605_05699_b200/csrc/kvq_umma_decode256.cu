@@ -60,7 +60,11 @@ struct Cfg {
     static constexpr int kAStages = BF16OUT ? 1 : 2;   // per parity: 128 columns hold a_hi | a_lo, or two stages of a_hi
     static constexpr int kBBytes = kTerms * 2 * kBPart;
     static constexpr int kInStages = BF16OUT ? 2 : 4;  // packed tiles in flight (16 KB each): what the split B leaves room for
-    static constexpr int kSmemBytes = kBBytes + kInStages * kInBytes + 8 * kOutWarpBytes + kCtrlBytes + 1024;
+    // per-row output scales of the tiles between a dequant group and the epilogue: as many slots as a group can run ahead
+    static constexpr int kScaleSlots = 2 * kAStages;
+    static constexpr int kScaleBytes = kScaleSlots * kTile * (int)sizeof(float);
+    static constexpr int kSmemBytes = kBBytes + kInStages * kInBytes + 8 * kOutWarpBytes + kCtrlBytes + kScaleBytes + 1024;
+    static_assert(kSmemBytes <= 232448, "shared memory over the per-CTA limit");
 };
 
 struct Ctrl {
@@ -179,6 +183,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     unsigned char *sIn = sB + C::kBBytes;
     unsigned char *sOut = sIn + kInStages * kInBytes;
     Ctrl *ctrl = reinterpret_cast<Ctrl *>(sOut + 8 * kOutWarpBytes);
+    float *row_scale = reinterpret_cast<float *>(reinterpret_cast<unsigned char *>(ctrl) + kCtrlBytes);   // [slot][row]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -354,15 +359,36 @@ __global__ void __launch_bounds__(kThreads, 1)
             if (!wait_or_abort(smem_u32(&ctrl->a_empty[p][sa]), ((uint32_t)(j / C::kAStages) & 1u) ^ 1u, abort_flag, status, KVQ_DEV_MMA_TIMEOUT))
                 break;
             tc_fence_after();
+            // ---- the A operand q sigma rho is fp16.  A row whose scales would take it out of fp16's normal range (a very
+            // ---- small or very large vector) is carried times a power of two instead, which the epilogue takes out again
+            // ---- in fp32; every other row has the factor 1 and costs the epilogue nothing.  Both parity groups see the
+            // ---- same scales and take the same factor; group 0 posts it.
+            float pw = 1.0f;
+            {
+                uint32_t smax = 0u, smin = 0xFFFFu;
+#pragma unroll
+                for (int c = 0; c < kG; ++c) {
+                    const uint32_t s = (sc[c >> 1] >> (16 * (c & 1))) & 0x7FFFu;   // fp16 bits of a non-negative number order like integers
+                    smax = max(smax, s);
+                    if (s != 0u) smin = min(smin, s);
+                }
+                const float tmax = __half2float(__ushort_as_half((unsigned short)smax)) * rho;
+                const float tmin = __half2float(__ushort_as_half((unsigned short)(smin == 0xFFFFu ? 0u : smin))) * rho;
+                float inv = 1.0f;
+                if (tmax > 9000.0f || (tmin != 0.0f && tmin < 6.1035156e-5f)) {
+                    // 2^floor(log2 tmax) -> 2^7: the largest operand lands in [896, 1792), sums of 128 of them stay inside fp16
+                    const int e = (int)((__float_as_uint(fminf(fmaxf(tmax, 1e-30f), 1e30f)) >> 23) & 0xFFu) - 127;
+                    pw = __uint_as_float((uint32_t)(127 + 7 - e) << 23);
+                    inv = __uint_as_float((uint32_t)(127 - 7 + e) << 23);
+                }
+                if (p == 0) row_scale[(j % C::kScaleSlots) * kTile + r] = inv;
+            }
             const uint32_t a_row = tmem_base + ((uint32_t)(q * 32) << 16) + kACol0 + (uint32_t)p * 128u + (uint32_t)sa * 64u;
             const __half2 h1032 = __float2half2_rn(1032.0f);
 #pragma unroll
             for (int c = 0; c < kG; ++c) {   // group c: 16 codes of this parity, 8 tensor-memory columns
                 const float sig = __half2float(__ushort_as_half((unsigned short)((sc[c >> 1] >> (16 * (c & 1))) & 0xFFFFu)));
-                const float sr = sig * rho;
-                const __half2 s2 = __float2half2_rn(sr);
-                // the A operand q sigma rho is fp16: it overflows beyond 7 sr = 65504 and loses bits once sr is subnormal
-                if (sr != 0.0f && (sr > 9357.0f || sr < 6.1035156e-5f)) atomicOr(status, KVQ_DEV_RANGE);
+                const __half2 s2 = __float2half2_rn(sig * rho * pw);
                 const uint32_t words[4] = {pk[c].x, pk[c].y, pk[c].z, pk[c].w};
                 uint32_t a_hi[8], a_lo[8];
 #pragma unroll
@@ -386,6 +412,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             }
             tmem_st_wait();
             tc_fence_before();
+            __threadfence_block();   // the row scales, for the epilogue that follows this tile's accumulator
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctrl->a_full[p][sa]));
         }
@@ -404,6 +431,8 @@ __global__ void __launch_bounds__(kThreads, 1)
             const bool tail = seg >= prm.n_full;
             const CUtensorMap *tm = tail ? &maps.tail : &maps.out;
             const int segc = tail ? 0 : (int)seg;
+            const float row_inv = row_scale[(j % C::kScaleSlots) * kTile + q * 32 + lane];
+            const bool rescale = __any_sync(0xFFFFFFFFu, row_inv != 1.0f);   // rare: a row outside the operand's comfort zone
 #pragma unroll
             for (int cc = 0; cc < 2; ++cc) {   // 32 column pairs at a time: outputs n0 .. n0 + 31 and 128 + n0 ..
                 const int n0 = 64 * ch + 32 * cc;
@@ -412,6 +441,13 @@ __global__ void __launch_bounds__(kThreads, 1)
                 tmem_ld32(lane_addr + (uint32_t)n0, e);
                 tmem_ld32(lane_addr + (uint32_t)(kHalf + n0), o);
                 tmem_ld_wait();
+                if (rescale) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        e[i] = __float_as_uint(__uint_as_float(e[i]) * row_inv);
+                        o[i] = __float_as_uint(__uint_as_float(o[i]) * row_inv);
+                    }
+                }
                 if (cc == 1) {   // the last values are in registers: hand the accumulator back
                     tc_fence_before();
                     __syncwarp();
