@@ -59,8 +59,9 @@ typedef enum { KVQ_F16 = 0, KVQ_BF16 = 1 } kvq_dtype_t;
 typedef enum {
     KVQ_IMPL_AUTO = 0,
     KVQ_IMPL_FFT = 1,   /* fp32 register FFT, one thread per vector: every D, dtype and layout; no rotation */
-    KVQ_IMPL_GEMM = 2,  /* tcgen05 DFT-as-GEMM, bits = 4 only.  encode / append: fp16 for D = 64, 96, 128, 160, 256,
-                           bf16 for D = 64, 96, 128, 256; decode: the same (D, dtype) pairs; either group size.
+    KVQ_IMPL_GEMM = 2,  /* tcgen05 DFT-as-GEMM.  bits = 4: encode / append: fp16 for D = 64, 96, 128, 160, 256, bf16 for
+                           D = 64, 96, 128, 256; decode: the same (D, dtype) pairs; either group size.  bits = 8:
+                           D <= 160 only, decode for the same pairs, encode for fp16 input only.
                            Elsewhere the compute calls return KVQ_ERR_UNSUPPORTED_DIM. */
     KVQ_IMPL_MATVEC = 3 /* fp32 matrix-vector product with the plan's D x D table, a CTA per 8 vectors: every D, dtype
                            and layout, rotated plans included; meant for small calls, correct (and slow) at any size */
@@ -86,8 +87,8 @@ kvq_status_t kvq_plan_create(int D, int group, uint64_t seed, kvq_plan_t **out);
  *   bits   4 (codes in [-7, 7], two per byte as in kvq_encode) or 8 (scale = absmax / 127, codes in [-127, 127], one
  *          two's-complement byte per value: `packed` rows are D bytes).
  * Everything else is as for kvq_plan_create, which is (group, bits = 4).  Wherever a comment of this header says
- * "[*, D/2] bytes" a plan with bits = 8 takes [*, D] bytes.  The tensor-core kernels serve bits = 4 (either group
- * size): other plans run on the register-FFT and matrix-vector kernels
+ * "[*, D/2] bytes" a plan with bits = 8 takes [*, D] bytes.  The tensor-core kernels serve either group size, and
+ * bits = 8 up to D = 160 (see KVQ_IMPL_GEMM); elsewhere such plans run on the register-FFT and matrix-vector kernels
  * (KVQ_IMPL_GEMM is refused with UNSUPPORTED_DIM); kvq_decode_static serves group = 32, bits = 4 only.
  */
 kvq_status_t kvq_plan_create_ex(int D, int group, int bits, uint64_t seed, kvq_plan_t **out);

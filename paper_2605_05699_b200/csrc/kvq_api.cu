@@ -146,8 +146,16 @@ static kvq_status_t ensure_device(kvq_plan *p)
     return KVQ_OK;
 }
 
-// the tensor-core kernels exist for 4-bit codes: groups of 32 (the fused layout) or one scale per vector
-static bool gemm_layout(const kvq_plan *p) { return p->bits == 4 && (p->group == 32 || p->group == p->D); }
+// the tensor-core kernels take groups of 32 (the fused layout) or one scale per vector; byte codes up to D = 160
+static bool gemm_encode_ok(const kvq_plan *p, bool bf16)
+{
+    if (p->bits == 8) return umma_encode_bits8_supported(p->D, bf16);
+    return p->group == p->D ? umma_encode_per_vector_supported(p->D, bf16) : umma_encode_supported(p->D, bf16);
+}
+static bool gemm_decode_ok(const kvq_plan *p, bool bf16)
+{
+    return p->bits == 8 ? umma_decode_bits8_supported(p->D, bf16) : umma_decode_supported(p->D, bf16);
+}
 
 static bool misaligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
 
@@ -174,6 +182,7 @@ static void fill_params(const kvq_plan *p, FftParams &prm, int64_t N, const floa
     prm.in_map = RowMap{1, 1, 0};
     prm.status = p->d_status;
     prm.table_max = p->table_max;
+    prm.bits = p->bits;
     std::memcpy(prm.sign_xor, p->sign_xor, sizeof(prm.sign_xor));
 }
 
@@ -330,7 +339,7 @@ static kvq_status_t encode_common(kvq_plan_t *plan, const void *x, kvq_dtype_t d
     if (misaligned16(x) || misaligned16(packed) || misaligned16(scales)) return KVQ_ERR_ALIGNMENT;
     const bool bf16 = dtype == KVQ_BF16;
     const bool per_vector = plan->group == plan->D;
-    const bool gemm_ok = gemm_layout(plan) && (per_vector ? umma_encode_per_vector_supported(plan->D, bf16) : umma_encode_supported(plan->D, bf16));
+    const bool gemm_ok = gemm_encode_ok(plan, bf16);
     if (plan->enc_impl == KVQ_IMPL_GEMM && !gemm_ok) return KVQ_ERR_UNSUPPORTED_DIM;
     if (plan->rot && plan->enc_impl == KVQ_IMPL_FFT) return KVQ_ERR_UNSUPPORTED_DIM;   // the rotation lives in the D x D tables
     if ((st = ensure_device(plan)) != KVQ_OK) return st;
@@ -387,7 +396,7 @@ kvq_status_t kvq_decode(kvq_plan_t *plan, const uint8_t *packed, const void *sca
     if (st != KVQ_OK) return st;
     if (misaligned16(packed) || misaligned16(scales) || misaligned16(out)) return KVQ_ERR_ALIGNMENT;
     const bool bf16 = dtype == KVQ_BF16;
-    const bool gemm_ok = gemm_layout(plan) && umma_decode_supported(plan->D, bf16);
+    const bool gemm_ok = gemm_decode_ok(plan, bf16);
     if (plan->dec_impl == KVQ_IMPL_GEMM && !gemm_ok) return KVQ_ERR_UNSUPPORTED_DIM;
     if (plan->rot && plan->dec_impl == KVQ_IMPL_FFT) return KVQ_ERR_UNSUPPORTED_DIM;   // the rotation lives in the D x D tables
     if ((st = ensure_device(plan)) != KVQ_OK) return st;
@@ -412,7 +421,7 @@ kvq_status_t kvq_decode(kvq_plan_t *plan, const uint8_t *packed, const void *sca
         g.status = plan->d_status;
         // D = 256: the radix-2 kernel needs the transform's even / odd structure, which a rotation destroys
         const cudaError_t e = plan->rot && plan->D == 256 ? umma_decode_d256_dense(bf16, N, g, stream)
-                                                          : umma_decode(plan->D, bf16, N, g, plan->sign_xor, stream);
+                                                          : umma_decode(plan->D, bf16, plan->bits, N, g, plan->sign_xor, stream);
         if (e != cudaSuccess) {
             (void)cudaGetLastError();
             return KVQ_ERR_CUDA;

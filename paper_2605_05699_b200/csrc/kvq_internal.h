@@ -36,6 +36,7 @@ struct FftParams {
     RowMap in_map;              // decode: row of packed / scales that row r comes from
     uint32_t *status;           // per-plan device status word
     float table_max;            // tensor-core encode: largest |entry| of the plan's forward table (sqrt(2/D) without a rotation)
+    int bits;                   // tensor-core encode: 4 or 8 (the register-FFT launchers take it as an argument)
     uint32_t sign_xor[128];     // word m: bit 15 set if s_{2m} = -1, bit 31 set if s_{2m+1} = -1
 };
 
@@ -57,7 +58,8 @@ struct GemmParams {
 // fp32, e0[c][n] = M[c][n] s_n; decode takes the table b0 = e0 transposed through GemmParams.
 bool umma_decode_supported(int D, bool bf16);
 bool umma_encode_supported(int D, bool bf16);
-cudaError_t umma_decode(int D, bool bf16, int64_t N, const GemmParams &prm, const uint32_t *sign_xor /* host, 128 words */,
+bool umma_decode_bits8_supported(int D, bool bf16);
+cudaError_t umma_decode(int D, bool bf16, int bits, int64_t N, const GemmParams &prm, const uint32_t *sign_xor /* host, 128 words */,
                         cudaStream_t stream);
 cudaError_t umma_calibrate(int D, bool bf16, int64_t N, const FftParams &prm, const float *e0, uint32_t *amax_bits, cudaStream_t stream);
 cudaError_t umma_calibrate_d256(bool bf16, int64_t N, const FftParams &prm, const float *e0, uint32_t *amax_bits, cudaStream_t stream);
@@ -65,6 +67,7 @@ cudaError_t umma_encode_d256(bool bf16, bool per_vector, int64_t N, const FftPar
 cudaError_t umma_decode_d256(bool bf16, int64_t N, const GemmParams &prm, const uint32_t *sign_xor, cudaStream_t stream);   // kvq_umma_decode256.cu
 cudaError_t umma_decode_d256_dense(bool bf16, int64_t N, const GemmParams &prm, cudaStream_t stream);   // kvq_umma_decode256_dense.cu: any table
 bool umma_encode_per_vector_supported(int D, bool bf16);
+bool umma_encode_bits8_supported(int D, bool bf16);
 cudaError_t umma_encode(int D, bool bf16, bool per_vector, int64_t N, const FftParams &prm, const float *e0, cudaStream_t stream);
 
 // fp32 matrix-vector kernels for small calls (kvq_matvec.cu): every layout, dtype and D; b0 / e0 are the plan's tables

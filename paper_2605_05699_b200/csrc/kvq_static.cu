@@ -132,7 +132,7 @@ extern "C" kvq_status_t kvq_decode_static(kvq_plan_t *plan, const uint8_t *packe
     g.rows_per_lambda = rows_per_lambda < 1 ? 1 : rows_per_lambda;
     g.per_vector = 0;
     g.status = status;
-    if (umma_decode(128, false, N, g, plan->sign_xor, stream) != cudaSuccess) {
+    if (umma_decode(128, false, 4, N, g, plan->sign_xor, stream) != cudaSuccess) {
         (void)cudaGetLastError();
         return KVQ_ERR_CUDA;
     }

@@ -46,7 +46,7 @@ namespace {
 
 constexpr int kTile = 128;       // vectors per tile = MMA M
 constexpr int kThreads = 576;    // producer, mma, 2 x 4 dequant, 2 x 4 epilogue warps
-constexpr int kInStages = 6;     // packed tiles in flight
+constexpr int kMaxInStages = 6;  // packed tiles in flight, at most
 constexpr int kAccStages = 2;    // accumulators in tensor memory
 constexpr int kCtrlBytes = 4608;   // barriers and flags, then eight tiles' worth of per-row output scales
 constexpr int kRowScaleSlots = 8;  // a dequant group is never more than seven tiles ahead of the epilogue that reads its slot
@@ -56,10 +56,13 @@ constexpr uint32_t kTmemCols = 512;
 // lands on the other side of enough rounding boundaries to miss the 1e-3 tolerance.  Both operands are then carried
 // in two fp16 terms: a = q sigma rho has 15 significant bits and splits exactly into a_hi + a_lo (one half2 FMA),
 // W' = W_hi + W_lo, and x^ = a_hi W_hi + a_lo W_hi + a_hi W_lo accumulates in fp32 (a_lo W_lo is below 1e-7).
-template <int D, bool BF16OUT>
+// BITS: 4 (nibble pairs) or 8 (one two's-complement byte per code; scale = absmax / 127).  The byte path dequantises
+// pairs of neighbouring codes, so its K order is the natural one and the B operand is built to match.
+template <int D, bool BF16OUT, int BITS = 4>
 struct Cfg {
     static_assert(D % 32 == 0 && D >= 64 && D <= 160, "head dim not built");
     static_assert(!BF16OUT || D <= 128, "two-term operands: tensor memory holds them for D <= 128 only");
+    static_assert(BITS == 4 || BITS == 8, "code width not built");
     static constexpr int kTerms = BF16OUT ? 2 : 1;         // W_hi (, W_lo); a_hi (, a_lo)
     static constexpr int G = D / 32;                       // groups = 16-byte chunks of a packed row = 32-column accumulator chunks
     static constexpr int kKSteps = D / 16;
@@ -67,14 +70,18 @@ struct Cfg {
     static constexpr int kBBlock = D * 128;                // bytes of one K block: D rows x 128 B
     static constexpr int kBTerm = kKBlocks * kBBlock;
     static constexpr int kBBytes = kTerms * kBTerm;
-    static constexpr int kInRow = D / 2;                   // packed bytes per row
+    static constexpr int kInRow = D * BITS / 8;            // code bytes per row
     static constexpr int kInBytes = kTile * kInRow;        // bytes one TMA load brings
     static constexpr int kInPitch = (kInBytes + 1023) & ~1023;
     // The packed tile is read row per thread, 16 bytes at a time.  Row pitches of 48 and 80 bytes spread eight
-    // consecutive rows over all banks by themselves; 32 and 64 bytes need the TMA swizzle of that width.
-    static constexpr int kInSwizzleBits = D == 64 ? 1 : D == 128 ? 2 : 0;
+    // consecutive rows over all banks by themselves (96 and 160 bytes over half of them); 32, 64 and 128 bytes need
+    // the TMA swizzle of that width.
+    static constexpr int kInSwizzleBits = kInRow == 32 ? 1 : kInRow == 64 ? 2 : kInRow == 128 ? 3 : 0;
     static constexpr int kOutWarpBytes = 32 * 2 * D;       // staging of one epilogue warp: G / 2 boxes of 4 KB (+ one of 2 KB)
     static constexpr int kOutBytes = 8 * kOutWarpBytes;
+    static constexpr int kRoom = (232448 - 1024 - kCtrlBytes - kBBytes - kOutBytes) / kInPitch;
+    static constexpr int kInStages = kRoom < kMaxInStages ? kRoom : kMaxInStages;
+    static_assert(kInStages >= 3, "too few packed tiles in flight");
     static constexpr int kSmemBytes = kBBytes + kInStages * kInPitch + kOutBytes + kCtrlBytes + 1024;
     // tensor memory: two accumulators of D columns, then the A stages of D / 2 columns per term (a_lo 64 columns
     // behind a_hi)
@@ -90,7 +97,7 @@ struct Cfg {
 };
 
 struct Ctrl {
-    uint64_t in_full[kInStages], in_empty[kInStages];
+    uint64_t in_full[kMaxInStages], in_empty[kMaxInStages];
     uint64_t a_full[4], a_empty[4];
     uint64_t acc_full[kAccStages], acc_empty[kAccStages];
     uint64_t b_first;
@@ -139,10 +146,10 @@ struct RecipLambda {
 // Rows [n0, n1) of the B operand, by one warp: a lane reads four table entries b0[n][4 i .. 4 i + 3] (coalesced
 // rows), scales them, trades two values with its neighbour so that each lane holds two K-ordered pairs, and
 // writes 8 bytes of the swizzled row.
-template <int D, bool BF16OUT>
+template <int D, bool BF16OUT, int BITS>
 __device__ __forceinline__ void build_b_quad(unsigned char *sB, float4 m, const RecipLambda<D> &rl, int n, int p, int lane)
 {
-    using C = Cfg<D, BF16OUT>;
+    using C = Cfg<D, BF16OUT, BITS>;
     const bool odd = lane & 1;
     const int i = lane + 32 * p;
     const bool live = i < D / 4;
@@ -152,12 +159,17 @@ __device__ __forceinline__ void build_b_quad(unsigned char *sB, float4 m, const 
     unsigned char *dst = sB + (w >> 3) * C::kBBlock + n * 128 + (((w & 7) ^ (n & 7)) << 4) + (odd ? 8 : 0);
 #pragma unroll
     for (int t = 0; t < C::kTerms; ++t) {
-        // even lane holds codes 8w .. 8w+3, odd lane 8w+4 .. 8w+7; K order of the word is (0,4,1,5,2,6,3,7)
-        const float r0 = __shfl_xor_sync(0xFFFFFFFFu, odd ? vx : vz, 1);
-        const float r1 = __shfl_xor_sync(0xFFFFFFFFu, odd ? vy : vw, 1);
         uint2 o;
-        o.x = odd ? narrow2<false>(r0, vz) : narrow2<false>(vx, r0);   // odd: (2, 6)   even: (0, 4)
-        o.y = odd ? narrow2<false>(r1, vw) : narrow2<false>(vy, r1);   // odd: (3, 7)   even: (1, 5)
+        if constexpr (BITS == 4) {
+            // even lane holds codes 8w .. 8w+3, odd lane 8w+4 .. 8w+7; K order of the word is (0,4,1,5,2,6,3,7)
+            const float r0 = __shfl_xor_sync(0xFFFFFFFFu, odd ? vx : vz, 1);
+            const float r1 = __shfl_xor_sync(0xFFFFFFFFu, odd ? vy : vw, 1);
+            o.x = odd ? narrow2<false>(r0, vz) : narrow2<false>(vx, r0);   // odd: (2, 6)   even: (0, 4)
+            o.y = odd ? narrow2<false>(r1, vw) : narrow2<false>(vy, r1);   // odd: (3, 7)   even: (1, 5)
+        } else {   // byte codes: natural K order, this lane's four channels side by side
+            o.x = narrow2<false>(vx, vy);
+            o.y = narrow2<false>(vz, vw);
+        }
         if (live) *reinterpret_cast<uint2 *>(dst + t * C::kBTerm) = o;
         if (t + 1 < C::kTerms) {   // what the fp16 term left behind (exact in fp32)
             vx -= __half2float(__float2half_rn(vx)), vy -= __half2float(__float2half_rn(vy));
@@ -166,7 +178,7 @@ __device__ __forceinline__ void build_b_quad(unsigned char *sB, float4 m, const 
     }
 }
 
-template <int D, bool BF16OUT>
+template <int D, bool BF16OUT, int BITS>
 __device__ __forceinline__ void build_b_rows(unsigned char *sB, const float *__restrict__ b0, const RecipLambda<D> &rl, int n0, int n1,
                                              int lane)
 {
@@ -177,14 +189,14 @@ __device__ __forceinline__ void build_b_rows(unsigned char *sB, const float *__r
             const int i = lane + 32 * p;
             float4 m = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
             if (i < D / 4) m = __ldg(reinterpret_cast<const float4 *>(b0 + (size_t)n * D) + i);
-            build_b_quad<D, BF16OUT>(sB, m, rl, n, p, lane);
+            build_b_quad<D, BF16OUT, BITS>(sB, m, rl, n, p, lane);
         }
     }
 }
 
 // The first build of a CTA: its D / 16 table rows per warp are requested at kernel entry, all at once, and turned
 // into B rows here, once lambda has arrived too: one round trip to L2 instead of one per batch of rows.
-template <int D, bool BF16OUT>
+template <int D, bool BF16OUT, int BITS>
 struct FirstRows {
     static constexpr int kRows = D / 16, kPasses = RecipLambda<D>::kPasses;
     float4 m[kRows][kPasses];
@@ -203,7 +215,7 @@ struct FirstRows {
 #pragma unroll
         for (int k = 0; k < kRows; ++k)
 #pragma unroll
-            for (int p = 0; p < kPasses; ++p) build_b_quad<D, BF16OUT>(sB, m[k][p], rl, n0 + k, p, lane);
+            for (int p = 0; p < kPasses; ++p) build_b_quad<D, BF16OUT, BITS>(sB, m[k][p], rl, n0 + k, p, lane);
     }
 };
 
@@ -242,12 +254,12 @@ struct UmmaDecodeMaps {
     CUtensorMap slim, slim_tail;   // output, boxes of 32 columns x 32 rows (64-byte swizzle), used when D / 32 is odd
 };
 
-template <int D, bool BF16OUT>
+template <int D, bool BF16OUT, int BITS>
 __global__ void __launch_bounds__(kThreads, 1)
     kvq_decode_umma_kernel(const __grid_constant__ UmmaDecodeParams prm, const __grid_constant__ UmmaDecodeMaps maps)
 {
-    using C = Cfg<D, BF16OUT>;
-    constexpr int G = C::G;
+    using C = Cfg<D, BF16OUT, BITS>;
+    constexpr int G = C::G, kInStages = C::kInStages;
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     unsigned char *sB = smem;
@@ -292,7 +304,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     // ---- producer's first loads are in flight; the mma warp waits for all of them.  Table rows and lambda are
     // ---- requested before the set-up barrier, so that their latency runs under it.
     if (n_my > 0 && warp >= 2) {
-        FirstRows<D, BF16OUT> rows;
+        FirstRows<D, BF16OUT, BITS> rows;
         rows.load(prm.g.b0, (warp - 2) * (D / 16), lane);
         const RecipLambda<D> rl(lambda_row(seg_first), lane);
         fence_proxy_async();
@@ -375,7 +387,10 @@ __global__ void __launch_bounds__(kThreads, 1)
         const int q = warp & 3;                 // tensor-memory lane quarter this warp may touch
         const int r = q * 32 + lane;            // tile row and tensor-memory lane of this thread
         const uint16_t *scales = static_cast<const uint16_t *>(prm.g.scales);   // D / 32 fp16 scales per row
-        const uint32_t swz = C::kInSwizzleBits == 2 ? (uint32_t)((r >> 1) & 3) : C::kInSwizzleBits == 1 ? (uint32_t)((r >> 2) & 1) : 0u;
+        const uint32_t swz = C::kInSwizzleBits == 3   ? (uint32_t)(r & 7)
+                             : C::kInSwizzleBits == 2 ? (uint32_t)((r >> 1) & 3)
+                             : C::kInSwizzleBits == 1 ? (uint32_t)((r >> 2) & 1)
+                                                      : 0u;
         int64_t cached_seg = n_my > 0 ? seg_first : -1;   // B holds this row's table (built above)
         float rho = RecipLambda<D>(lambda_row(seg_first), lane).rho;
 
@@ -423,7 +438,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                     if (!wait_or_abort(smem_u32(&ctrl->a_empty[(j - 1) % C::kAStages]), (uint32_t)((j - 1) / C::kAStages) & 1u, abort_flag,
                                        status, KVQ_DEV_MMA_TIMEOUT))
                         break;
-                    build_b_rows<D, BF16OUT>(sB, prm.g.b0, rl, q * (D / 4), (q + 1) * (D / 4), lane);
+                    build_b_rows<D, BF16OUT, BITS>(sB, prm.g.b0, rl, q * (D / 4), (q + 1) * (D / 4), lane);
                     fence_proxy_async();   // B is read by the tensor core through the async proxy
                 }
                 cached_seg = seg;
@@ -432,14 +447,14 @@ __global__ void __launch_bounds__(kThreads, 1)
             // ---- this tile's packed rows have landed; the A stage is free again
             const int s = j % kInStages, sa = j % C::kAStages;
             if (!wait_or_abort(smem_u32(&ctrl->in_full[s]), (uint32_t)(j / kInStages) & 1u, abort_flag, status, KVQ_DEV_LOAD_TIMEOUT)) break;
-            uint4 pk[G];
-            {
-                const unsigned char *row = sIn + s * C::kInPitch + r * C::kInRow;
+            const unsigned char *row = sIn + s * C::kInPitch + r * C::kInRow;
+            uint4 pk[BITS == 4 ? G : 1];
+            if constexpr (BITS == 4) {
 #pragma unroll
                 for (int c = 0; c < G; ++c) pk[c] = *reinterpret_cast<const uint4 *>(row + (((uint32_t)c ^ swz) << 4));
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctrl->in_empty[s]));   // the values are in registers
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&ctrl->in_empty[s]));   // the values are in registers
             if (!wait_or_abort(smem_u32(&ctrl->a_empty[sa]), ((uint32_t)(j / C::kAStages) & 1u) ^ 1u, abort_flag, status, KVQ_DEV_MMA_TIMEOUT))
                 break;
             tc_fence_after();
@@ -459,8 +474,9 @@ __global__ void __launch_bounds__(kThreads, 1)
                 const float tmax = __half2float(__ushort_as_half((unsigned short)smax)) * rho;
                 const float tmin = __half2float(__ushort_as_half((unsigned short)(smin == 0xFFFFu ? 0u : smin))) * rho;
                 float inv = 1.0f;
-                if (tmax > 9000.0f || (tmin != 0.0f && tmin < 6.1035156e-5f)) {
-                    // 2^floor(log2 tmax) -> 2^7: the largest operand lands in [896, 1792), sums of 128 of them stay inside fp16
+                constexpr float kMaxT = BITS == 4 ? 9000.0f : 500.0f;   // largest code (7 or 127) times this stays inside fp16
+                if (tmax > kMaxT || (tmin != 0.0f && tmin < 6.1035156e-5f)) {
+                    // 2^floor(log2 tmax) -> 2^7: the largest operand lands in [896, 1792) (byte codes: below 32512)
                     const int e = (int)((__float_as_uint(fminf(fmaxf(tmax, 1e-30f), 1e30f)) >> 23) & 0xFFu) - 127;
                     pw = __uint_as_float((uint32_t)(127 + 7 - e) << 23);
                     inv = __uint_as_float((uint32_t)(127 - 7 + e) << 23);
@@ -474,25 +490,48 @@ __global__ void __launch_bounds__(kThreads, 1)
             for (int c = 0; c < G; ++c) {   // chunk c = group c: 32 codes, 16 tensor-memory columns
                 const float sig = __half2float(__ushort_as_half((unsigned short)((sc[c >> 1] >> (16 * (c & 1))) & 0xFFFFu)));
                 const __half2 s2 = __float2half2_rn(sig * rho * pw);
-                const uint32_t words[4] = {pk[c].x, pk[c].y, pk[c].z, pk[c].w};
                 uint32_t a[16], al[BF16OUT ? 16 : 1];
+                auto put = [&](int k, __half2 q2) {   // K-pair k of the group: one rounding, and what it left behind
+                    const __half2 h = __hmul2(q2, s2);
+                    a[k] = *reinterpret_cast<const uint32_t *>(&h);
+                    if constexpr (BF16OUT) {   // q s2 - h, exact in fp16
+                        const __half2 l = __hfma2(q2, s2, __hneg2(h));
+                        al[k] = *reinterpret_cast<const uint32_t *>(&l);
+                    }
+                };
+                if constexpr (BITS == 4) {
+                    const uint32_t words[4] = {pk[c].x, pk[c].y, pk[c].z, pk[c].w};
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const uint32_t u = words[i] ^ 0x88888888u;   // nibbles now hold q + 8
+                    for (int i = 0; i < 4; ++i) {
+                        const uint32_t u = words[i] ^ 0x88888888u;   // nibbles now hold q + 8
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const uint32_t m = lop3_and_or(u >> (4 * e), 0x000F000Fu, 0x64006400u);   // {1024 + n_e, 1024 + n_{e+4}}
-                        const __half2 q2 = __hsub2(*reinterpret_cast<const __half2 *>(&m), h1032);     // exact q
-                        const __half2 h = __hmul2(q2, s2);                                                 // one rounding
-                        a[4 * i + e] = *reinterpret_cast<const uint32_t *>(&h);
-                        if constexpr (BF16OUT) {   // what the rounding left behind: q s2 - h, exact in fp16
-                            const __half2 l = __hfma2(q2, s2, __hneg2(h));
-                            al[4 * i + e] = *reinterpret_cast<const uint32_t *>(&l);
+                        for (int e = 0; e < 4; ++e) {
+                            const uint32_t m = lop3_and_or(u >> (4 * e), 0x000F000Fu, 0x64006400u);   // {1024 + n_e, 1024 + n_{e+4}}
+                            put(4 * i + e, __hsub2(*reinterpret_cast<const __half2 *>(&m), h1032));    // exact q
+                        }
+                    }
+                } else {   // 32 byte codes: two 16-byte chunks of the row, pairs of neighbours
+                    const __half2 h1152 = __float2half2_rn(1152.0f);
+#pragma unroll
+                    for (int hc = 0; hc < 2; ++hc) {
+                        const uint4 pc = *reinterpret_cast<const uint4 *>(row + (((uint32_t)(2 * c + hc) ^ swz) << 4));
+                        const uint32_t words[4] = {pc.x, pc.y, pc.z, pc.w};
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const uint32_t u = words[i] ^ 0x80808080u;                 // bytes now hold q + 128
+                            const uint32_t m01 = __byte_perm(u, 0x64646464u, 0x4140);   // {1024 + b0, 1024 + b1} as fp16 bit patterns
+                            const uint32_t m23 = __byte_perm(u, 0x64646464u, 0x4342);
+                            put(8 * hc + 2 * i, __hsub2(*reinterpret_cast<const __half2 *>(&m01), h1152));       // exact q
+                            put(8 * hc + 2 * i + 1, __hsub2(*reinterpret_cast<const __half2 *>(&m23), h1152));
                         }
                     }
                 }
                 tmem_st16(a_row + 16u * (uint32_t)c, a);
                 if constexpr (BF16OUT) tmem_st16(a_row + C::kALo + 16u * (uint32_t)c, al);
+            }
+            if constexpr (BITS == 8) {   // the packed rows were read group by group: only now is their stage free
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctrl->in_empty[s]));
             }
             tmem_st_wait();
             tc_fence_before();
@@ -577,10 +616,10 @@ __global__ void __launch_bounds__(kThreads, 1)
 // ------------------------------------------------------------------------------------------------
 namespace {
 
-template <int D, bool BF16OUT>
+template <int D, bool BF16OUT, int BITS = 4>
 cudaError_t launch(int64_t N, const GemmParams &g, cudaStream_t stream)
 {
-    using C = Cfg<D, BF16OUT>;
+    using C = Cfg<D, BF16OUT, BITS>;
     static DeviceSlots slots;
     int dev = 0;
     cudaError_t e = current_device_slot(&dev);
@@ -588,7 +627,7 @@ cudaError_t launch(int64_t N, const GemmParams &g, cudaStream_t stream)
     int &sms = slots.sms[dev];
     if (sms == 0) {
         int n = 0;
-        if ((e = cudaFuncSetAttribute(kvq_decode_umma_kernel<D, BF16OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes)) != cudaSuccess) return e;
+        if ((e = cudaFuncSetAttribute(kvq_decode_umma_kernel<D, BF16OUT, BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes)) != cudaSuccess) return e;
         if ((e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
         sms = n;
     }
@@ -606,7 +645,8 @@ cudaError_t launch(int64_t N, const GemmParams &g, cudaStream_t stream)
         const cuuint64_t dims[2] = {(cuuint64_t)C::kInRow, (cuuint64_t)N};
         const cuuint64_t strides[1] = {(cuuint64_t)C::kInRow};
         const cuuint32_t box[2] = {(cuuint32_t)C::kInRow, (cuuint32_t)kTile};
-        const CUtensorMapSwizzle sw = C::kInSwizzleBits == 2 ? CU_TENSOR_MAP_SWIZZLE_64B
+        const CUtensorMapSwizzle sw = C::kInSwizzleBits == 3   ? CU_TENSOR_MAP_SWIZZLE_128B
+                                      : C::kInSwizzleBits == 2 ? CU_TENSOR_MAP_SWIZZLE_64B
                                       : C::kInSwizzleBits == 1 ? CU_TENSOR_MAP_SWIZZLE_32B
                                                                : CU_TENSOR_MAP_SWIZZLE_NONE;
         if (!make_tensor_map(&maps.packed, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, g.packed, dims, strides, box, sw)) return cudaErrorInvalidValue;
@@ -629,7 +669,7 @@ cudaError_t launch(int64_t N, const GemmParams &g, cudaStream_t stream)
 
     const int64_t tiles = prm.n_seg * ((prm.rpl + kTile - 1) / kTile);
     const int grid = (int)(tiles < sms ? tiles : sms);
-    kvq_decode_umma_kernel<D, BF16OUT><<<grid, kThreads, C::kSmemBytes, stream>>>(prm, maps);
+    kvq_decode_umma_kernel<D, BF16OUT, BITS><<<grid, kThreads, C::kSmemBytes, stream>>>(prm, maps);
     count_launch();
     return cudaGetLastError();
 }
@@ -638,8 +678,20 @@ cudaError_t launch(int64_t N, const GemmParams &g, cudaStream_t stream)
 
 bool umma_decode_supported(int D, bool bf16) { return D == 256 || D == 64 || D == 96 || D == 128 || (!bf16 && D == 160); }
 
-cudaError_t umma_decode(int D, bool bf16, int64_t N, const GemmParams &g, const uint32_t *sign_xor, cudaStream_t stream)
+// byte codes: the D <= 160 kernel only
+bool umma_decode_bits8_supported(int D, bool bf16) { return D != 256 && umma_decode_supported(D, bf16); }
+
+cudaError_t umma_decode(int D, bool bf16, int bits, int64_t N, const GemmParams &g, const uint32_t *sign_xor, cudaStream_t stream)
 {
+    if (bits == 8) {
+        switch (D) {
+            case 64: return bf16 ? launch<64, true, 8>(N, g, stream) : launch<64, false, 8>(N, g, stream);
+            case 96: return bf16 ? launch<96, true, 8>(N, g, stream) : launch<96, false, 8>(N, g, stream);
+            case 128: return bf16 ? launch<128, true, 8>(N, g, stream) : launch<128, false, 8>(N, g, stream);
+            case 160: return bf16 ? cudaErrorInvalidValue : launch<160, false, 8>(N, g, stream);
+        }
+        return cudaErrorInvalidValue;
+    }
     if (D == 256) return umma_decode_d256(bf16, N, g, sign_xor, stream);   // its own kernel: radix-2 split, split operands for bf16
     switch (D) {
         case 64: return bf16 ? launch<64, true>(N, g, stream) : launch<64, false>(N, g, stream);

@@ -54,6 +54,8 @@ constexpr uint32_t kTmemCols = 512;
 constexpr float kMagicRound = 12582912.0f + 8.0f;   // 1.5 * 2^23 + 8: (v + magic) has q + 8 in its low bits
 constexpr uint32_t kMagicBits = 0x4B400000u;
 constexpr uint32_t kMagicSum = kMagicBits * 0x11111111u;   // sum_i kMagicBits * 16^i  (mod 2^32)
+constexpr float kMagicRound8 = 12582912.0f + 128.0f;       // byte codes: q + 128 in the low byte
+constexpr uint32_t kMagicSum8 = kMagicBits * 0x01010101u;  // sum_i kMagicBits * 256^i (mod 2^32)
 
 // CALIB: the calibration pass keeps a third bf16 term (it runs once; its result is compared at 1e-6 of the vector norm)
 template <int D, bool BF16, bool CALIB = false>
@@ -193,6 +195,7 @@ struct UmmaEncodeParams {
     int64_t n_seg;
     RowMap out_map;        // output row of input row r
     float table_max;       // largest |entry| of e0
+    int bits;              // 4: nibble pairs; 8: one two's-complement byte per code, scale = absmax / 127
     uint32_t *status;
     uint32_t *amax_bits;        // calibration only: [D] running column maxima as fp32 bit patterns (start at zero)
 };
@@ -387,6 +390,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             if (seg_rows > rpl) seg_rows = rpl;
             const bool live = off + r < seg_rows;
             const int64_t orow = prm.out_map(seg * rpl + off + r);
+            const float Q = prm.bits == 4 ? 7.0f : 127.0f;   // largest code (warp-uniform)
             // ---- one scale per vector: the row's maximum first (this thread's half, then the other half's through
             // ---- shared memory), then a second pass over the accumulator for the codes
             float row_rs = 0.0f;
@@ -411,11 +415,11 @@ __global__ void __launch_bounds__(kThreads, 1)
                 if (!wait_or_abort(smem_u32(&ctrl->pair[set][q]), (uint32_t)it & 1u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT)) break;
                 m = fmaxf(m, ctrl->rowmax[it & 1][set][h ^ 1][r]);
                 const float amax = m * unlift;
-                const float sig = fminf(__fdiv_rn(amax, 7.0f), 65504.0f);
+                const float sig = fminf(__fdiv_rn(amax, Q), 65504.0f);
                 const __half hs = __float2half_rn(sig);
                 const float sg = __half2float(hs);
                 const float rs1 = sg > 0.0f ? __frcp_rn(sg) : 0.0f;
-                row_clamp = !(amax * rs1 < 7.25f);
+                row_clamp = !(amax * rs1 < Q + 0.25f);
                 row_rs = rs1 * unlift;
                 if (live && h == 0) prm.scales[orow] = __half_as_ushort(hs);
             }
@@ -449,32 +453,55 @@ __global__ void __launch_bounds__(kThreads, 1)
 #pragma unroll
                         for (int i = 0; i < 32; ++i) amax = fmaxf(amax, fabsf(__uint_as_float(vb[i])));
                         amax *= unlift;
-                        const float sig = fminf(__fdiv_rn(amax, 7.0f), 65504.0f);
+                        const float sig = fminf(__fdiv_rn(amax, Q), 65504.0f);
                         hs = __float2half_rn(sig);
                         const float sg = __half2float(hs);
                         const float rs1 = sg > 0.0f ? __frcp_rn(sg) : 0.0f;
-                        clamp = !(amax * rs1 < 7.25f);   // saturated or subnormal scale: codes could leave [-7, 7]
+                        clamp = !(amax * rs1 < Q + 0.25f);   // saturated or subnormal scale: codes could leave [-Q, Q]
                         rs = rs1 * unlift;               // applies to the lifted accumulator values
                     }
 
-                    // ---- round, bias to unsigned nibbles, pack 8 codes per word
-                    uint32_t words[4];
+                    // ---- round, bias to unsigned codes, pack: 8 nibbles or 4 bytes per word
+                    if (prm.bits == 4) {
+                        uint32_t words[4];
 #pragma unroll
-                    for (int w = 0; w < 4; ++w) {
-                        uint32_t acc = 0;
-                        if (!clamp) {
+                        for (int w = 0; w < 4; ++w) {
+                            uint32_t acc = 0;
+                            if (!clamp) {
 #pragma unroll
-                            for (int e = 0; e < 8; ++e)
-                                acc += __float_as_uint(fmaf(__uint_as_float(vb[8 * w + e]), rs, kMagicRound)) << (4 * e);
-                        } else {
+                                for (int e = 0; e < 8; ++e)
+                                    acc += __float_as_uint(fmaf(__uint_as_float(vb[8 * w + e]), rs, kMagicRound)) << (4 * e);
+                            } else {
 #pragma unroll
-                            for (int e = 0; e < 8; ++e)
-                                acc += __float_as_uint(fminf(fmaxf(__uint_as_float(vb[8 * w + e]) * rs, -7.0f), 7.0f) + kMagicRound) << (4 * e);
+                                for (int e = 0; e < 8; ++e)
+                                    acc += __float_as_uint(fminf(fmaxf(__uint_as_float(vb[8 * w + e]) * rs, -7.0f), 7.0f) + kMagicRound) << (4 * e);
+                            }
+                            words[w] = (acc - kMagicSum) ^ 0x88888888u;
                         }
-                        words[w] = (acc - kMagicSum) ^ 0x88888888u;
+                        if (live) *reinterpret_cast<uint4 *>(prm.packed + orow * (D / 2) + g * 16) = make_uint4(words[0], words[1], words[2], words[3]);
+                    } else {
+                        uint32_t words[8];
+#pragma unroll
+                        for (int w = 0; w < 8; ++w) {
+                            uint32_t acc = 0;
+                            if (!clamp) {
+#pragma unroll
+                                for (int e = 0; e < 4; ++e)
+                                    acc += __float_as_uint(fmaf(__uint_as_float(vb[4 * w + e]), rs, kMagicRound8)) << (8 * e);
+                            } else {
+#pragma unroll
+                                for (int e = 0; e < 4; ++e)
+                                    acc += __float_as_uint(fminf(fmaxf(__uint_as_float(vb[4 * w + e]) * rs, -127.0f), 127.0f) + kMagicRound8) << (8 * e);
+                            }
+                            words[w] = (acc - kMagicSum8) ^ 0x80808080u;
+                        }
+                        if (live) {
+                            uint4 *dst = reinterpret_cast<uint4 *>(prm.packed + orow * D + g * 32);
+                            dst[0] = make_uint4(words[0], words[1], words[2], words[3]);
+                            dst[1] = make_uint4(words[4], words[5], words[6], words[7]);
+                        }
                     }
                     if (live) {
-                        *reinterpret_cast<uint4 *>(prm.packed + orow * (D / 2) + g * 16) = make_uint4(words[0], words[1], words[2], words[3]);
                         if constexpr (!PERVEC) prm.scales[orow * G + g] = __half_as_ushort(hs);
                     }
                 }
@@ -528,6 +555,7 @@ cudaError_t launch(int64_t N, const FftParams &f, const float *e0, cudaStream_t 
     prm.n_seg = (N + prm.rpl - 1) / prm.rpl;
     prm.out_map = f.out_map;
     prm.table_max = f.table_max;
+    prm.bits = f.bits;
     prm.status = f.status;
     prm.amax_bits = amax_bits;
 
@@ -552,6 +580,10 @@ bool umma_encode_supported(int D, bool bf16) { return D == 64 || D == 96 || D ==
 
 // one scale per vector: the row maximum is traded inside a CTA, or across the cluster pair of the D = 256 kernel
 bool umma_encode_per_vector_supported(int D, bool bf16) { return umma_encode_supported(D, bf16); }
+
+// byte codes: the D <= 160 kernel, fp16 input only (the code step is 18 times finer than with 4 bits: two bf16 terms of W
+// would leave 2e-4 of the codes on the wrong side of a rounding)
+bool umma_encode_bits8_supported(int D, bool bf16) { return !bf16 && D != 256 && umma_encode_supported(D, bf16); }
 
 cudaError_t umma_encode(int D, bool bf16, bool per_vector, int64_t N, const FftParams &f, const float *e0, cudaStream_t stream)
 {

@@ -451,13 +451,16 @@ def test_small_calls_take_the_matvec_kernels_and_agree_with_the_fft():
     (160, "f16", True, 8), (160, "bf16", False, 8),
     (256, "bf16", True, 4), (256, "f16", True, 8), (256, "bf16", False, 8),
 ])
-@pytest.mark.parametrize("impl", ["fft", "matvec"])
+@pytest.mark.parametrize("impl", ["fft", "matvec", "gemm"])
 def test_base_variants_per_vector_scale_and_byte_codes(D, dtype, per_vector, nbits, impl):
+    if impl == "gemm" and ((D == 256 and nbits == 8) or (D == 160 and dtype == "bf16")):
+        pytest.skip("no tensor-core kernel for this layout: covered by the refusal test")
+    enc_impl = "fft" if (impl == "gemm" and nbits == 8 and dtype == "bf16") else impl   # byte codes from bf16: no tensor-core encode
     N, n_lambda, rpl = 5003, 3, 1700          # ragged, lambda rows straddle the warps' tiles
     group = D if per_vector else G
     odt = ko.F16 if dtype == "f16" else ko.BF16
     plan = kb.Plan(D, group, 90 + D, bits=nbits)
-    kb.kvq_plan_set_impl(plan.handle, IMPL[impl], IMPL[impl])
+    kb.kvq_plan_set_impl(plan.handle, IMPL[enc_impl], IMPL[impl])
     sg = plan.signs()
     lam = wl.make_lambda(n_lambda, D, 91)
     x = wl.make_vectors(N, D, dtype, "k_outlier", 92 + nbits)
@@ -503,11 +506,11 @@ def test_one_scale_per_vector_on_the_tensor_cores(D, dtype, N, n_lambda, rpl):
 
 
 def test_base_variants_append_and_flush_and_refusals():
-    D, S, T = 128, 24, 40
+    D, S, T = 256, 24, 40
     plan = kb.Plan(D, D, 7, bits=8)
     sg = plan.signs()
     lam = wl.make_lambda(S, D, 8)
-    x = wl.make_vectors(S * T, D, "f16", "gaussian", 9).view(S, T, D)
+    x = wl.make_vectors(S * T, D, "f16", "gaussian", 9).view(S, T, D)   # byte codes at D = 256: register FFT and matrix-vector only
     packed = torch.full((S, T, D), 0x55, dtype=torch.uint8, device="cuda")
     scales = torch.full((S, T, 1), 2.0, dtype=torch.float16, device="cuda")
     dq = torch.full((S, T, D), 3.0, dtype=torch.float16, device="cuda")
@@ -524,7 +527,7 @@ def test_base_variants_append_and_flush_and_refusals():
     pk32, sb32 = packed[:, :32].reshape(-1, D).cpu().numpy(), bits(scales[:, :32].reshape(-1, 1))
     ob, o64 = ko.decode(pk32, sb32, sg, lam.numpy(), D, ko.F16, 32, want_f64=True, bits=8)
     parity.check_decode(bits(dq[:, :32].reshape(-1, D)), ob, o64, ko.F16, "variant dequantized cache")
-    # the tensor-core kernels and the no-allocation decode serve the fused layout only
+    # the tensor-core kernels do not serve byte codes at D = 256
     kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_GEMM, kb.KVQ_IMPL_GEMM)
     o = torch.empty(S * T, D, dtype=torch.float16, device="cuda")
     with pytest.raises(kb.KvqError):
