@@ -57,12 +57,13 @@ constexpr uint32_t kMagicSum = kMagicBits * 0x11111111u;   // sum_i kMagicBits *
 constexpr float kMagicRound8 = 12582912.0f + 128.0f;       // byte codes: q + 128 in the low byte
 constexpr uint32_t kMagicSum8 = kMagicBits * 0x01010101u;  // sum_i kMagicBits * 256^i (mod 2^32)
 
-// CALIB: the calibration pass keeps a third bf16 term (it runs once; its result is compared at 1e-6 of the vector norm)
-template <int D, bool BF16, bool CALIB = false>
+// THREE: a third bf16 term of W.  The calibration pass takes it (it runs once; its result is compared at 1e-6 of the
+// vector norm), and so do byte codes, whose step is 18 times finer than that of 4-bit codes.
+template <int D, bool BF16, bool THREE = false>
 struct Cfg {
     static_assert(D % 32 == 0 && D >= 64 && D <= 160, "head dim not built");
     static constexpr int G = D / kGroup;
-    static constexpr int kSplit = (BF16 && CALIB) ? 3 : 2;
+    static constexpr int kSplit = (BF16 && THREE) ? 3 : 2;
     static constexpr int kKSteps = D / 16;
     static constexpr int kKBlocks = (D + 63) / 64;              // K blocks of 64 elements (the last one may be half used)
     static constexpr int kXBytes = kKBlocks * kBlockBytes;      // one x tile
@@ -118,10 +119,10 @@ __device__ __forceinline__ float lift_of(const float *__restrict__ lam, float ta
 // 8 bytes of each term's swizzled row.
 // One quad of row c of every split term: the four table entries m scaled by f = lambda_c 2^k, 16-bit terms peeled
 // off one after the other, 8 bytes of each term's swizzled row written.
-template <int D, bool BF16, bool CALIB>
+template <int D, bool BF16, bool THREE>
 __device__ __forceinline__ void build_b_quad(unsigned char *sB, float4 m, float f, int c, int i)
 {
-    using C = Cfg<D, BF16, CALIB>;
+    using C = Cfg<D, BF16, THREE>;
     float w[4] = {m.x * f, m.y * f, m.z * f, m.w * f};
     const int ch = i >> 1;   // 16-byte chunk of the K-major row: K block ch / 8, chunk ch % 8
     const uint32_t off = (uint32_t)((ch >> 3) * C::kBBlock + c * 128 + (((ch & 7) ^ (c & 7)) << 4) + ((i & 1) ? 8 : 0));
@@ -136,7 +137,7 @@ __device__ __forceinline__ void build_b_quad(unsigned char *sB, float4 m, float 
     }
 }
 
-template <int D, bool BF16, bool CALIB>
+template <int D, bool BF16, bool THREE>
 __device__ __forceinline__ void build_b_rows(unsigned char *sB, const float *__restrict__ e0, const float *__restrict__ lam, float lift,
                                              int c0, int c1, int lane)
 {
@@ -146,14 +147,14 @@ __device__ __forceinline__ void build_b_rows(unsigned char *sB, const float *__r
 #pragma unroll
         for (int p = 0; p < (D / 4 + 31) / 32; ++p) {
             const int i = lane + 32 * p;
-            if (i < D / 4) build_b_quad<D, BF16, CALIB>(sB, __ldg(reinterpret_cast<const float4 *>(e0 + (size_t)c * D) + i), f, c, i);
+            if (i < D / 4) build_b_quad<D, BF16, THREE>(sB, __ldg(reinterpret_cast<const float4 *>(e0 + (size_t)c * D) + i), f, c, i);
         }
     }
 }
 
 // The first build of a CTA: a warp's D / 16 table rows and their lambda entries are requested at kernel entry, all at
 // once, and turned into B rows once the lift is known: one round trip to L2 instead of one per batch of rows.
-template <int D, bool BF16, bool CALIB>
+template <int D, bool BF16, bool THREE>
 struct FirstRows {
     static constexpr int kRows = D / 16, kPasses = (D / 4 + 31) / 32;
     float4 m[kRows][kPasses];
@@ -177,7 +178,7 @@ struct FirstRows {
 #pragma unroll
             for (int p = 0; p < kPasses; ++p) {
                 const int i = lane + 32 * p;
-                if (i < D / 4) build_b_quad<D, BF16, CALIB>(sB, m[k][p], lam_c[k] * lift, c0 + k, i);
+                if (i < D / 4) build_b_quad<D, BF16, THREE>(sB, m[k][p], lam_c[k] * lift, c0 + k, i);
             }
     }
 };
@@ -201,11 +202,12 @@ struct UmmaEncodeParams {
 };
 
 // PERVEC: one scale per vector (group = D; Sec. 3.2 step 3, Sec. 4.1) instead of one per 32 channels.
-template <int D, bool BF16, bool CALIB, bool PERVEC>
+// WIDE: byte codes from bf16 input (three terms of W).
+template <int D, bool BF16, bool CALIB, bool PERVEC, bool WIDE>
 __global__ void __launch_bounds__(kThreads, 1)
     kvq_encode_umma_kernel(const __grid_constant__ UmmaEncodeParams prm, const __grid_constant__ CUtensorMap tm_x)
 {
-    using C = Cfg<D, BF16, CALIB>;
+    using C = Cfg<D, BF16, CALIB || WIDE>;
     constexpr int G = C::G, kInStages = C::kInStages, kAccStages = C::kAccStages;
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -246,7 +248,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     if (n_my > 0 && warp >= 2) {
         first_seg = tile_begin / tps;
         const float *lam = CALIB ? nullptr : prm.lambda + (prm.n_lambda == 1 ? 0 : first_seg) * D;
-        FirstRows<D, BF16, CALIB> rows;
+        FirstRows<D, BF16, CALIB || WIDE> rows;
         rows.load(prm.e0, lam, (warp - 2) * (D / 16), lane);
         first_lift = lift_of<D>(lam, prm.table_max, lane);
         fence_proxy_async();
@@ -372,7 +374,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                     if (!wait_or_abort(smem_u32(&ctrl->acc_full[(j - 1) % kAccStages]), (uint32_t)((j - 1) / kAccStages) & 1u,
                                        abort_flag, status, KVQ_DEV_MMA_TIMEOUT))
                         break;
-                    build_b_rows<D, BF16, CALIB>(sB, prm.e0, lam, lift, bw * (D / 8), (bw + 1) * (D / 8), lane);
+                    build_b_rows<D, BF16, CALIB || WIDE>(sB, prm.e0, lam, lift, bw * (D / 8), (bw + 1) * (D / 8), lane);
                     fence_proxy_async();   // B is read by the tensor core through the async proxy
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&ctrl->b_ready));
@@ -527,10 +529,10 @@ __global__ void __launch_bounds__(kThreads, 1)
 // ------------------------------------------------------------------------------------------------
 namespace {
 
-template <int D, bool BF16, bool CALIB = false, bool PERVEC = false>
+template <int D, bool BF16, bool CALIB = false, bool PERVEC = false, bool WIDE = false>
 cudaError_t launch(int64_t N, const FftParams &f, const float *e0, cudaStream_t stream, uint32_t *amax_bits = nullptr)
 {
-    using C = Cfg<D, BF16, CALIB>;
+    using C = Cfg<D, BF16, CALIB || WIDE>;
     static DeviceSlots slots;
     int dev = 0;
     cudaError_t e = current_device_slot(&dev);
@@ -538,7 +540,7 @@ cudaError_t launch(int64_t N, const FftParams &f, const float *e0, cudaStream_t 
     int &sms = slots.sms[dev];
     if (sms == 0) {
         int n = 0;
-        if ((e = cudaFuncSetAttribute(kvq_encode_umma_kernel<D, BF16, CALIB, PERVEC>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes)) != cudaSuccess) return e;
+        if ((e = cudaFuncSetAttribute(kvq_encode_umma_kernel<D, BF16, CALIB, PERVEC, WIDE>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes)) != cudaSuccess) return e;
         if ((e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
         sms = n;
     }
@@ -569,7 +571,7 @@ cudaError_t launch(int64_t N, const FftParams &f, const float *e0, cudaStream_t 
 
     const int64_t tiles = prm.n_seg * ((prm.rpl + kTile - 1) / kTile);
     const int grid = (int)(tiles < sms ? tiles : sms);
-    kvq_encode_umma_kernel<D, BF16, CALIB, PERVEC><<<grid, kThreads, C::kSmemBytes, stream>>>(prm, tm_x);
+    kvq_encode_umma_kernel<D, BF16, CALIB, PERVEC, WIDE><<<grid, kThreads, C::kSmemBytes, stream>>>(prm, tm_x);
     count_launch();
     return cudaGetLastError();
 }
@@ -581,14 +583,22 @@ bool umma_encode_supported(int D, bool bf16) { return D == 64 || D == 96 || D ==
 // one scale per vector: the row maximum is traded inside a CTA, or across the cluster pair of the D = 256 kernel
 bool umma_encode_per_vector_supported(int D, bool bf16) { return umma_encode_supported(D, bf16); }
 
-// byte codes: the D <= 160 kernel, fp16 input only (the code step is 18 times finer than with 4 bits: two bf16 terms of W
-// would leave 2e-4 of the codes on the wrong side of a rounding)
-bool umma_encode_bits8_supported(int D, bool bf16) { return !bf16 && D != 256 && umma_encode_supported(D, bf16); }
+// byte codes: the D <= 160 kernel (the code step is 18 times finer than with 4 bits: two bf16 terms of W would leave 2e-4
+// of the codes on the wrong side of a rounding, so bf16 input takes the three-term instantiation)
+bool umma_encode_bits8_supported(int D, bool bf16) { return D != 256 && umma_encode_supported(D, bf16); }
 
 cudaError_t umma_encode(int D, bool bf16, bool per_vector, int64_t N, const FftParams &f, const float *e0, cudaStream_t stream)
 {
     if (!tensor_map_encode_fn()) return cudaErrorNotSupported;
     if (D == 256) return umma_encode_d256(bf16, per_vector, N, f, e0, stream);   // its own kernel: CTA pairs, x through a ring of K blocks
+    if (bf16 && f.bits == 8) {   // three bf16 terms
+        switch (D) {
+            case 64: return per_vector ? launch<64, true, false, true, true>(N, f, e0, stream) : launch<64, true, false, false, true>(N, f, e0, stream);
+            case 96: return per_vector ? launch<96, true, false, true, true>(N, f, e0, stream) : launch<96, true, false, false, true>(N, f, e0, stream);
+            case 128: return per_vector ? launch<128, true, false, true, true>(N, f, e0, stream) : launch<128, true, false, false, true>(N, f, e0, stream);
+        }
+        return cudaErrorInvalidValue;
+    }
     if (per_vector) {
         switch (D) {
             case 64: return bf16 ? launch<64, true, false, true>(N, f, e0, stream) : launch<64, false, false, true>(N, f, e0, stream);

@@ -455,7 +455,7 @@ def test_small_calls_take_the_matvec_kernels_and_agree_with_the_fft():
 def test_base_variants_per_vector_scale_and_byte_codes(D, dtype, per_vector, nbits, impl):
     if impl == "gemm" and ((D == 256 and nbits == 8) or (D == 160 and dtype == "bf16")):
         pytest.skip("no tensor-core kernel for this layout: covered by the refusal test")
-    enc_impl = "fft" if (impl == "gemm" and nbits == 8 and dtype == "bf16") else impl   # byte codes from bf16: no tensor-core encode
+    enc_impl = impl
     N, n_lambda, rpl = 5003, 3, 1700          # ragged, lambda rows straddle the warps' tiles
     group = D if per_vector else G
     odt = ko.F16 if dtype == "f16" else ko.BF16
