@@ -736,6 +736,39 @@ def test_config3_gemma_shaped_prefix_4096_sampled():
     _full_size_sampled(256, "bf16", 2 * wl.GEMMA3_1B.layers * 4096, "c1", 6100, 2 * wl.GEMMA3_1B.layers, 4096)
 
 
+# ---- beyond 2^32 bytes: row offsets must be 64-bit in every kernel family -------------------------------------------
+
+@pytest.mark.parametrize("impl", ["gemm", "fft", "matvec"])
+def test_row_offsets_beyond_four_gigabytes(impl):
+    # 17,000,001 vectors of D = 128 fp16: x and x^ are 4.35 GB each, so the last rows sit past byte 2^32 of their buffers
+    # (and past row 2^24); sampled rows at both ends and in between go to the oracle
+    D, N = 128, 17_000_001
+    n_lambda, rpl = 3, 6_000_000
+    plan = kb.Plan(D, G, 23)
+    kb.kvq_plan_set_impl(plan.handle, IMPL[impl], IMPL[impl])
+    sg = plan.signs()
+    lam = wl.make_lambda(n_lambda, D, 24)
+    x = wl.make_vectors(1 << 20, D, "f16", "k_outlier", 25, device="cuda").repeat(17, 1)[:N].contiguous()   # 16 + 1 copies
+    x[-4096:] = wl.make_vectors(4096, D, "f16", "gaussian", 26, device="cuda")                                # a distinct tail
+    assert x.numel() * 2 > 1 << 32
+    lamd = lam.cuda()
+    packed, scales = gpu_encode(plan, x, lamd, rpl)
+    out = gpu_decode(plan, packed, scales, lamd, "f16", rpl)
+    g = torch.Generator().manual_seed(3)
+    idx = torch.unique(torch.cat([torch.arange(0, 512), torch.arange(N - 1024, N), torch.randint(0, N, (2048,), generator=g),
+                                  torch.arange(2 * rpl - 300, 2 * rpl + 300)]))
+    idx_d = idx.cuda()
+    xs, pk, sc, od = x[idx_d].cpu(), packed[idx_d].cpu().numpy(), bits(scales[idx_d]), bits(out[idx_d])
+    lrow = (idx // rpl).numpy()
+    for l in np.unique(lrow):
+        m = lrow == l
+        ora = ko.encode(bits(xs)[m], ko.F16, sg, lam.numpy()[l], G, want_v=True)
+        parity.check_encode(pk[m], sc[m], ora, G, "rows past 4 GB, encode, lambda row %d" % l, min_agree=0.9995)
+        ob, o64 = ko.decode(pk[m], sc[m], sg, lam.numpy()[l], G, ko.F16, want_f64=True)
+        parity.check_decode(od[m], ob, o64, ko.F16, "rows past 4 GB, decode, lambda row %d" % l)
+    plan.close()
+
+
 # ---- config 5: Llama-3-70B-shaped: one layer's K (1,048,576 vectors) per launch, sampled rows -
 
 def _full_size_sampled(D, dtype, N, kind, seed, n_lambda, rows_per_lambda, n_random=4096, dec_impl="auto", enc_impl="auto"):

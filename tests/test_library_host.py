@@ -66,6 +66,20 @@ def test_unsupported_dims_and_groups_are_rejected():
         assert h.value is None
 
 
+def test_the_header_is_plain_c():
+    # the boundary is a C ABI: the header must compile as C, on its own
+    import subprocess
+    import tempfile
+
+    hdr = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "include", "kvq.h")
+    with tempfile.TemporaryDirectory() as d:
+        src = os.path.join(d, "use.c")
+        with open(src, "w") as f:
+            f.write('#include "%s"\nint main(void) { kvq_plan_t *p = 0; return (int)kvq_plan_destroy(p) + (int)KVQ_IMPL_MATVEC * 0; }\n' % hdr)
+        r = subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-fsyntax-only", src], capture_output=True, text=True)
+        assert r.returncode == 0, r.stderr
+
+
 def test_rotation_is_validated_on_the_host():
     p = kb.Plan(128, 32, 1)
     R = wl.make_rotation(128, 3)
