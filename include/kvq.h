@@ -61,7 +61,8 @@ typedef enum {
     KVQ_IMPL_FFT = 1,   /* fp32 register FFT, one thread per vector: every D, dtype and layout; no rotation */
     KVQ_IMPL_GEMM = 2,  /* tcgen05 DFT-as-GEMM.  bits = 4: encode / append: fp16 for D = 64, 96, 128, 160, 256, bf16 for
                            D = 64, 96, 128, 256; decode: the same (D, dtype) pairs; either group size.  bits = 8:
-                           D <= 160 only, the same (D, dtype) pairs.
+                           D <= 160 only, the same (D, dtype) pairs.  At most 2^31 - 1 rows per call (AUTO falls back
+                           to the register FFT beyond).
                            Elsewhere the compute calls return KVQ_ERR_UNSUPPORTED_DIM. */
     KVQ_IMPL_MATVEC = 3 /* fp32 matrix-vector product with the plan's D x D table, a CTA per 8 vectors: every D, dtype
                            and layout, rotated plans included; meant for small calls, correct (and slow) at any size */

@@ -339,7 +339,8 @@ static kvq_status_t encode_common(kvq_plan_t *plan, const void *x, kvq_dtype_t d
     if (misaligned16(x) || misaligned16(packed) || misaligned16(scales)) return KVQ_ERR_ALIGNMENT;
     const bool bf16 = dtype == KVQ_BF16;
     const bool per_vector = plan->group == plan->D;
-    const bool gemm_ok = gemm_encode_ok(plan, bf16);
+    // tensor-map coordinates are 32-bit: the tensor-core kernels take up to 2^31 - 1 rows per call
+    const bool gemm_ok = gemm_encode_ok(plan, bf16) && N < ((int64_t)1 << 31);
     if (plan->enc_impl == KVQ_IMPL_GEMM && !gemm_ok) return KVQ_ERR_UNSUPPORTED_DIM;
     if (plan->rot && plan->enc_impl == KVQ_IMPL_FFT) return KVQ_ERR_UNSUPPORTED_DIM;   // the rotation lives in the D x D tables
     if ((st = ensure_device(plan)) != KVQ_OK) return st;
@@ -396,7 +397,7 @@ kvq_status_t kvq_decode(kvq_plan_t *plan, const uint8_t *packed, const void *sca
     if (st != KVQ_OK) return st;
     if (misaligned16(packed) || misaligned16(scales) || misaligned16(out)) return KVQ_ERR_ALIGNMENT;
     const bool bf16 = dtype == KVQ_BF16;
-    const bool gemm_ok = gemm_decode_ok(plan, bf16);
+    const bool gemm_ok = gemm_decode_ok(plan, bf16) && N < ((int64_t)1 << 31);
     if (plan->dec_impl == KVQ_IMPL_GEMM && !gemm_ok) return KVQ_ERR_UNSUPPORTED_DIM;
     if (plan->rot && plan->dec_impl == KVQ_IMPL_FFT) return KVQ_ERR_UNSUPPORTED_DIM;   // the rotation lives in the D x D tables
     if ((st = ensure_device(plan)) != KVQ_OK) return st;
