@@ -213,4 +213,21 @@ __device__ __forceinline__ uint32_t narrow2(float lo, float hi)
     }
 }
 
+// ---------------------------------------------------------------------------
+// round-to-nearest-even codes by the magic-number trick (Sec. 3.2 step 4): v / sigma + 1.5 * 2^23 (+ bias) has the
+// biased code in its low mantissa bits, so eight nibbles (four bytes) are gathered with shifts and one subtraction
+// ---------------------------------------------------------------------------
+constexpr float kMagicRound = 12582912.0f + 8.0f;          // 1.5 * 2^23 + 8: (v + magic) has q + 8 in its low bits
+constexpr uint32_t kMagicBits = 0x4B400000u;
+constexpr uint32_t kMagicSum = kMagicBits * 0x11111111u;   // sum_i kMagicBits * 16^i  (mod 2^32)
+constexpr float kMagicRound8 = 12582912.0f + 128.0f;       // byte codes: q + 128 in the low byte
+constexpr uint32_t kMagicSum8 = kMagicBits * 0x01010101u;  // sum_i kMagicBits * 256^i (mod 2^32)
+
+__device__ __forceinline__ uint32_t lop3_and_or(uint32_t a, uint32_t b, uint32_t c)
+{
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));   // (a & b) | c
+    return d;
+}
+
 }  // namespace kvq

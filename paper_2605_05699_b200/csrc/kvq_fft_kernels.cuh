@@ -29,11 +29,6 @@
 
 namespace kvq {
 
-constexpr float kMagicRound = 12582912.0f + 8.0f;   // 1.5 * 2^23 + 8: (v + magic) has q + 8 in its low bits
-constexpr uint32_t kMagicBits = 0x4B400000u;
-constexpr uint32_t kMagicSum = kMagicBits * 0x11111111u;   // sum_i kMagicBits * 16^i  (mod 2^32)
-constexpr float kMagicRound8 = 12582912.0f + 128.0f;       // 8-bit codes: q + 128 in the low byte
-constexpr uint32_t kMagicSum8 = kMagicBits * 0x01010101u;  // sum_i kMagicBits * 256^i (mod 2^32)
 
 // ------------------------------------------------------------------------------------------
 // shared-memory geometry (per warp)

@@ -113,6 +113,30 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap *tm, int c0, int 
                  : "memory");
 }
 
+// The A operand of the decode kernels, q sigma rho, is fp16.  A row whose G stored scales (packed 16-bit pairs in sc)
+// would take it out of fp16's normal range -- sigma rho above max_t (the largest code times it must fit) or a non-zero
+// sigma rho below 2^-14 -- is carried times a power of two instead: the function returns that factor (1 for every other
+// row) and its inverse through inv, which the epilogue applies to the row's accumulators in fp32.  The factor takes
+// 2^floor(log2(largest sigma rho)) to 2^7, so the largest operand lands in [7 * 128, 7 * 256) (byte codes: below 32512).
+template <int G>
+__device__ __forceinline__ float operand_rescue(const uint32_t (&sc)[(G + 1) / 2], float rho, float max_t, float &inv)
+{
+    uint32_t smax = 0u, smin = 0xFFFFu;
+#pragma unroll
+    for (int c = 0; c < G; ++c) {
+        const uint32_t s = (sc[c >> 1] >> (16 * (c & 1))) & 0x7FFFu;   // fp16 bits of a non-negative number order like integers
+        smax = max(smax, s);
+        if (s != 0u) smin = min(smin, s);
+    }
+    const float tmax = __half2float(__ushort_as_half((unsigned short)smax)) * rho;
+    const float tmin = __half2float(__ushort_as_half((unsigned short)(smin == 0xFFFFu ? 0u : smin))) * rho;
+    inv = 1.0f;
+    if (!(tmax > max_t || (tmin != 0.0f && tmin < 6.1035156e-5f))) return 1.0f;
+    const int e = (int)((__float_as_uint(fminf(fmaxf(tmax, 1e-30f), 1e30f)) >> 23) & 0xFFu) - 127;
+    inv = __uint_as_float((uint32_t)(127 - 7 + e) << 23);
+    return __uint_as_float((uint32_t)(127 + 7 - e) << 23);
+}
+
 // Bounded wait that also gives up when another role of the CTA has raised the abort flag.  On a
 // time-out it raises the flag itself and records `reason` in the status word.
 __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *status,

@@ -107,13 +107,6 @@ struct Ctrl {
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
 
-__device__ __forceinline__ uint32_t lop3_and_or(uint32_t a, uint32_t b, uint32_t c)
-{
-    uint32_t d;
-    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));   // (a & b) | c
-    return d;
-}
-
 // 1 / max(lambda, 1e-6) for the channels this lane covers (4 i .. 4 i + 3, i = lane and, for D > 128, lane + 32),
 // divided by rho, the power of two that brings the row's largest reciprocal into [1, 2).  Every lane gets rho.
 template <int D>
@@ -462,27 +455,9 @@ __global__ void __launch_bounds__(kThreads, 1)
             // ---- the A operand q sigma rho is fp16.  A row whose scales would take it out of fp16's normal range (a very
             // ---- small or very large vector) is carried times a power of two instead, which the epilogue takes out again
             // ---- in fp32; every other row has the factor 1 and costs the epilogue nothing.
-            float pw = 1.0f;
-            {
-                uint32_t smax = 0u, smin = 0xFFFFu;
-#pragma unroll
-                for (int c = 0; c < G; ++c) {
-                    const uint32_t s = (sc[c >> 1] >> (16 * (c & 1))) & 0x7FFFu;   // fp16 bits of a non-negative number order like integers
-                    smax = max(smax, s);
-                    if (s != 0u) smin = min(smin, s);
-                }
-                const float tmax = __half2float(__ushort_as_half((unsigned short)smax)) * rho;
-                const float tmin = __half2float(__ushort_as_half((unsigned short)(smin == 0xFFFFu ? 0u : smin))) * rho;
-                float inv = 1.0f;
-                constexpr float kMaxT = BITS == 4 ? 9000.0f : 500.0f;   // largest code (7 or 127) times this stays inside fp16
-                if (tmax > kMaxT || (tmin != 0.0f && tmin < 6.1035156e-5f)) {
-                    // 2^floor(log2 tmax) -> 2^7: the largest operand lands in [896, 1792) (byte codes: below 32512)
-                    const int e = (int)((__float_as_uint(fminf(fmaxf(tmax, 1e-30f), 1e30f)) >> 23) & 0xFFu) - 127;
-                    pw = __uint_as_float((uint32_t)(127 + 7 - e) << 23);
-                    inv = __uint_as_float((uint32_t)(127 - 7 + e) << 23);
-                }
-                ctrl->row_scale[j & (kRowScaleSlots - 1)][r] = inv;
-            }
+            float inv;
+            const float pw = operand_rescue<G>(sc, rho, BITS == 4 ? 9000.0f : 500.0f, inv);   // 7 (127) times this stays inside fp16
+            ctrl->row_scale[j & (kRowScaleSlots - 1)][r] = inv;
             // ---- nibbles -> fp16 codes -> times sigma * rho, two codes per instruction
             const uint32_t a_row = tmem_base + ((uint32_t)(q * 32) << 16) + C::a_col(sa);
             const __half2 h1032 = __float2half2_rn(1032.0f);

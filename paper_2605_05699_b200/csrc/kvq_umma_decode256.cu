@@ -79,13 +79,6 @@ struct Ctrl {
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
 
-__device__ __forceinline__ uint32_t lop3_and_or(uint32_t a, uint32_t b, uint32_t c)
-{
-    uint32_t d;
-    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));   // (a & b) | c
-    return d;
-}
-
 // 8 consecutive columns of this thread's tensor-memory lane
 __device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&r)[8])
 {
@@ -363,26 +356,9 @@ __global__ void __launch_bounds__(kThreads, 1)
             // ---- small or very large vector) is carried times a power of two instead, which the epilogue takes out again
             // ---- in fp32; every other row has the factor 1 and costs the epilogue nothing.  Both parity groups see the
             // ---- same scales and take the same factor; group 0 posts it.
-            float pw = 1.0f;
-            {
-                uint32_t smax = 0u, smin = 0xFFFFu;
-#pragma unroll
-                for (int c = 0; c < kG; ++c) {
-                    const uint32_t s = (sc[c >> 1] >> (16 * (c & 1))) & 0x7FFFu;   // fp16 bits of a non-negative number order like integers
-                    smax = max(smax, s);
-                    if (s != 0u) smin = min(smin, s);
-                }
-                const float tmax = __half2float(__ushort_as_half((unsigned short)smax)) * rho;
-                const float tmin = __half2float(__ushort_as_half((unsigned short)(smin == 0xFFFFu ? 0u : smin))) * rho;
-                float inv = 1.0f;
-                if (tmax > 9000.0f || (tmin != 0.0f && tmin < 6.1035156e-5f)) {
-                    // 2^floor(log2 tmax) -> 2^7: the largest operand lands in [896, 1792), sums of 128 of them stay inside fp16
-                    const int e = (int)((__float_as_uint(fminf(fmaxf(tmax, 1e-30f), 1e30f)) >> 23) & 0xFFu) - 127;
-                    pw = __uint_as_float((uint32_t)(127 + 7 - e) << 23);
-                    inv = __uint_as_float((uint32_t)(127 - 7 + e) << 23);
-                }
-                if (p == 0) row_scale[(j % C::kScaleSlots) * kTile + r] = inv;
-            }
+            float inv;
+            const float pw = operand_rescue<kG>(sc, rho, 9000.0f, inv);
+            if (p == 0) row_scale[(j % C::kScaleSlots) * kTile + r] = inv;
             const uint32_t a_row = tmem_base + ((uint32_t)(q * 32) << 16) + kACol0 + (uint32_t)p * 128u + (uint32_t)sa * 64u;
             const __half2 h1032 = __float2half2_rn(1032.0f);
 #pragma unroll

@@ -60,13 +60,6 @@ struct Ctrl {
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
 
-__device__ __forceinline__ uint32_t lop3_and_or(uint32_t a, uint32_t b, uint32_t c)
-{
-    uint32_t d;
-    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));   // (a & b) | c
-    return d;
-}
-
 // 1 / max(lambda, 1e-6) for the channels 4 i .. 4 i + 3, i = lane and lane + 32, divided by rho, the power of two
 // that brings the row's largest reciprocal into [1, 2).  Every lane gets rho.
 struct RecipLambda {

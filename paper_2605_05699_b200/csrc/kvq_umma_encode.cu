@@ -51,11 +51,6 @@ constexpr int kCtrlBytes = 4608;            // barriers and flags, then the row 
 constexpr int kSmemLimit = 232448;         // 227 KB of dynamic shared memory per CTA
 constexpr uint32_t kTmemCols = 512;
 
-constexpr float kMagicRound = 12582912.0f + 8.0f;   // 1.5 * 2^23 + 8: (v + magic) has q + 8 in its low bits
-constexpr uint32_t kMagicBits = 0x4B400000u;
-constexpr uint32_t kMagicSum = kMagicBits * 0x11111111u;   // sum_i kMagicBits * 16^i  (mod 2^32)
-constexpr float kMagicRound8 = 12582912.0f + 128.0f;       // byte codes: q + 128 in the low byte
-constexpr uint32_t kMagicSum8 = kMagicBits * 0x01010101u;  // sum_i kMagicBits * 256^i (mod 2^32)
 
 // THREE: a third bf16 term of W.  The calibration pass takes it (it runs once; its result is compared at 1e-6 of the
 // vector norm), and so do byte codes, whose step is 18 times finer than that of 4-bit codes.

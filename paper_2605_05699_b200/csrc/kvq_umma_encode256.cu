@@ -30,9 +30,6 @@ constexpr int kCtrlBytes = 256;
 constexpr int kSmemLimit = 232448;         // 227 KB of dynamic shared memory per CTA
 constexpr uint32_t kTmemCols = 512;
 
-constexpr float kMagicRound = 12582912.0f + 8.0f;   // 1.5 * 2^23 + 8: (v + magic) has q + 8 in its low bits
-constexpr uint32_t kMagicBits = 0x4B400000u;
-constexpr uint32_t kMagicSum = kMagicBits * 0x11111111u;   // sum_i kMagicBits * 16^i  (mod 2^32)
 
 constexpr int kD = 256;
 constexpr int kG = kD / kGroup;            // 8 scales per row
