@@ -47,8 +47,8 @@ typedef enum {
     KVQ_ERR_TIMEOUT = 5,         /* a bounded device-side wait ran out (see kvq_plan_device_status) */
     KVQ_ERR_NOMEM = 6,
     KVQ_ERR_SCRATCH_LIMIT = 7,   /* the plan needs more fixed scratch than kvq_decode_static holds */
-    KVQ_ERR_RANGE = 8            /* the dense D = 256 decode of a rotated plan met a stored scale outside its
-                                    operand range (see kvq_plan_device_status) */
+    KVQ_ERR_RANGE = 8            /* a tensor-core decode met a lambda row or a stored scale outside its operand
+                                    range (see kvq_plan_device_status) */
 } kvq_status_t;
 
 typedef enum { KVQ_F16 = 0, KVQ_BF16 = 1 } kvq_dtype_t;
@@ -131,13 +131,17 @@ kvq_status_t kvq_plan_set_impl(kvq_plan_t *plan, kvq_impl_t encode_impl, kvq_imp
 /* Synchronizes the current device and returns the plan's device status word through *word
  * (host): 0 when no kernel using this plan ever gave up a bounded wait or left its number
  * range.  Bits 0-2: a bounded wait ran out (load, tensor-core commit, pipeline slot): returns
- * KVQ_ERR_TIMEOUT.  Bit 3: the dense D = 256 tensor-core decode of a ROTATED plan met a non-zero
- * stored scale sigma with sigma rho outside [2^-14, 9357], rho the power of two at or below the
- * lambda row's largest 1 / max(lambda, 1e-6).  The tensor-core decode kernels carry
- * q sigma / lambda as an fp16 operand; all but that one rescale such rows (very small or very
- * large vectors) by a power of two and are exact for them, that one reports them here and the
- * rows concerned are wrong: decode such data with KVQ_IMPL_MATVEC.  Returns KVQ_ERR_RANGE if
- * that is the only bit set.  The word is sticky for the plan's lifetime. */
+ * KVQ_ERR_TIMEOUT.  Bit 3: a tensor-core kvq_decode met data outside its operand range; the rows
+ * concerned are wrong, decode them with KVQ_IMPL_MATVEC or KVQ_IMPL_FFT (fp32 throughout).
+ * Those kernels carry q sigma / lambda and the table entries divided by lambda as fp16 operands:
+ *   - a lambda row whose reciprocals 1 / max(lambda, 1e-6) span more than a factor of 2^8
+ *     (entries at or below the 1e-6 clamp next to ordinary ones, for instance) loses bits on the
+ *     channels with the small reciprocals: every tensor-core decode kernel reports it;
+ *   - a non-zero stored scale sigma with sigma rho outside [2^-14, 9357] (rho: the power of two at
+ *     or below the row's largest reciprocal; very small or very large vectors): all kernels but
+ *     one rescale such rows by a power of two and are exact for them; the dense D = 256 kernel
+ *     of ROTATED plans reports them instead.
+ * Returns KVQ_ERR_RANGE if bit 3 is the only bit set.  The word is sticky for the plan's lifetime. */
 kvq_status_t kvq_plan_device_status(kvq_plan_t *plan, uint32_t *word);
 
 /*

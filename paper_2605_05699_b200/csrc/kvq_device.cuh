@@ -17,7 +17,7 @@ enum : uint32_t {
     KVQ_DEV_LOAD_TIMEOUT = 1u,   // a bounded wait for a bulk load ran out
     KVQ_DEV_MMA_TIMEOUT = 2u,    // a bounded wait for a tensor-core commit ran out
     KVQ_DEV_SLOT_TIMEOUT = 4u,   // a bounded wait for a free pipeline slot ran out
-    KVQ_DEV_RANGE = 8u,          // the dense D = 256 decode met a stored scale that takes q sigma / lambda out of fp16's normal range
+    KVQ_DEV_RANGE = 8u,          // a tensor-core decode met a lambda row or a stored scale outside its fp16 operands' range
 };
 
 // ---------------------------------------------------------------------------

@@ -114,9 +114,10 @@ struct RecipLambda {
     static constexpr int kPasses = (D / 4 + 31) / 32;
     float4 r[kPasses];
     float rho;
+    bool wide;   // the reciprocals span more than 2^8: B, which carries them in fp16 next to each other, loses bits on the small ones
     __device__ __forceinline__ RecipLambda(const float *__restrict__ lam, int lane)
     {
-        float mx = 0.0f;
+        float mx = 0.0f, mn = 3.0e38f;
 #pragma unroll
         for (int p = 0; p < kPasses; ++p) {
             const int i = lane + 32 * p;
@@ -127,10 +128,15 @@ struct RecipLambda {
                                    __frcp_rn(fmaxf(l.w, 1e-6f)));
             }
             mx = fmaxf(mx, fmaxf(fmaxf(r[p].x, r[p].y), fmaxf(r[p].z, r[p].w)));
+            if (i < D / 4) mn = fminf(mn, fminf(fminf(r[p].x, r[p].y), fminf(r[p].z, r[p].w)));
         }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+        for (int o = 16; o > 0; o >>= 1) {
+            mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+            mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, o));
+        }
         rho = __uint_as_float(__float_as_uint(mx) & 0x7F800000u);   // 2^floor(log2 max): exact to divide by
+        wide = mn < rho * 0.00390625f;
 #pragma unroll
         for (int p = 0; p < kPasses; ++p) r[p].x /= rho, r[p].y /= rho, r[p].z /= rho, r[p].w /= rho;
     }
@@ -300,6 +306,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         FirstRows<D, BF16OUT, BITS> rows;
         rows.load(prm.g.b0, (warp - 2) * (D / 16), lane);
         const RecipLambda<D> rl(lambda_row(seg_first), lane);
+        if (rl.wide && warp == 2 && lane == 0) atomicOr(prm.g.status, KVQ_DEV_RANGE);
         fence_proxy_async();
         tc_fence_before();
         __syncthreads();
@@ -431,6 +438,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                     if (!wait_or_abort(smem_u32(&ctrl->a_empty[(j - 1) % C::kAStages]), (uint32_t)((j - 1) / C::kAStages) & 1u, abort_flag,
                                        status, KVQ_DEV_MMA_TIMEOUT))
                         break;
+                    if (rl.wide && q == 0 && lane == 0) atomicOr(status, KVQ_DEV_RANGE);
                     build_b_rows<D, BF16OUT, BITS>(sB, prm.g.b0, rl, q * (D / 4), (q + 1) * (D / 4), lane);
                     fence_proxy_async();   // B is read by the tensor core through the async proxy
                 }

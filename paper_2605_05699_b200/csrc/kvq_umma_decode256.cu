@@ -92,19 +92,25 @@ __device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&r)[8])
 struct RecipLambda {
     float4 r[2];
     float rho;
+    bool wide;   // the reciprocals span more than 2^8: B, which carries them in fp16 next to each other, loses bits on the small ones
     __device__ __forceinline__ RecipLambda(const float *__restrict__ lam, int lane)
     {
-        float mx = 0.0f;
+        float mx = 0.0f, mn = 3.0e38f;
 #pragma unroll
         for (int p = 0; p < 2; ++p) {
             const float4 l = __ldg(reinterpret_cast<const float4 *>(lam) + lane + 32 * p);
             r[p] = make_float4(__frcp_rn(fmaxf(l.x, 1e-6f)), __frcp_rn(fmaxf(l.y, 1e-6f)), __frcp_rn(fmaxf(l.z, 1e-6f)),
                                __frcp_rn(fmaxf(l.w, 1e-6f)));
             mx = fmaxf(mx, fmaxf(fmaxf(r[p].x, r[p].y), fmaxf(r[p].z, r[p].w)));
+            mn = fminf(mn, fminf(fminf(r[p].x, r[p].y), fminf(r[p].z, r[p].w)));
         }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+        for (int o = 16; o > 0; o >>= 1) {
+            mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+            mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, o));
+        }
         rho = __uint_as_float(__float_as_uint(mx) & 0x7F800000u);   // 2^floor(log2 max): exact to divide by
+        wide = mn < rho * 0.00390625f;
 #pragma unroll
         for (int p = 0; p < 2; ++p) r[p].x /= rho, r[p].y /= rho, r[p].z /= rho, r[p].w /= rho;
     }
@@ -225,6 +231,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     // ---- and eight the O operand, sixteen rows each
     if (n_my > 0 && warp >= 2) {
         const RecipLambda rl(lambda_row(seg_first), lane);
+        if (rl.wide && warp == 2 && lane == 0) atomicOr(prm.g.status, KVQ_DEV_RANGE);
         const int bp = ((warp - 2) >> 2) & 1, bw = ((warp - 2) & 3) + 4 * ((warp - 2) >> 3);   // parity, position among its eight
         build_b_rows<kTerms>(sB, prm.g.b0, rl, bp, bw * 16, bw * 16 + 16, lane);
         fence_proxy_async();   // B is read by the tensor core through the async proxy
@@ -327,6 +334,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             // ---- GEMM issued so far is complete: the previous tile's, on this group's own barriers (it sees every phase)
             if (seg != cached_seg) {
                 const RecipLambda rl(lambda_row(seg), lane);
+                if (rl.wide && q == 0 && lane == 0) atomicOr(status, KVQ_DEV_RANGE);
                 rho = rl.rho;
                 if (!wait_or_abort(smem_u32(&ctrl->a_empty[p][(j - 1) % C::kAStages]), (uint32_t)((j - 1) / C::kAStages) & 1u, abort_flag,
                                    status, KVQ_DEV_MMA_TIMEOUT))

@@ -65,19 +65,25 @@ static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
 struct RecipLambda {
     float4 r[2];
     float rho;
+    bool wide;   // the reciprocals span more than 2^8: B, which carries them in fp16 next to each other, loses bits on the small ones
     __device__ __forceinline__ RecipLambda(const float *__restrict__ lam, int lane)
     {
-        float mx = 0.0f;
+        float mx = 0.0f, mn = 3.0e38f;
 #pragma unroll
         for (int p = 0; p < 2; ++p) {
             const float4 l = __ldg(reinterpret_cast<const float4 *>(lam) + lane + 32 * p);
             r[p] = make_float4(__frcp_rn(fmaxf(l.x, 1e-6f)), __frcp_rn(fmaxf(l.y, 1e-6f)), __frcp_rn(fmaxf(l.z, 1e-6f)),
                                __frcp_rn(fmaxf(l.w, 1e-6f)));
             mx = fmaxf(mx, fmaxf(fmaxf(r[p].x, r[p].y), fmaxf(r[p].z, r[p].w)));
+            mn = fminf(mn, fminf(fminf(r[p].x, r[p].y), fminf(r[p].z, r[p].w)));
         }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+        for (int o = 16; o > 0; o >>= 1) {
+            mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+            mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, o));
+        }
         rho = __uint_as_float(__float_as_uint(mx) & 0x7F800000u);   // 2^floor(log2 max): exact to divide by
+        wide = mn < rho * 0.00390625f;
 #pragma unroll
         for (int p = 0; p < 2; ++p) r[p].x /= rho, r[p].y /= rho, r[p].z /= rho, r[p].w /= rho;
     }
@@ -193,6 +199,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     // ---- B for the first tile's lambda row: the sixteen dequant and epilogue warps build eight rows each
     if (n_my > 0 && warp >= 2) {
         const RecipLambda rl(lambda_row(seg_first), lane);
+        if (rl.wide && warp == 2 && lane == 0) atomicOr(prm.g.status, KVQ_DEV_RANGE);
         build_b_rows<C::kBTerms>(sB, prm.g.b0, rl, half, (warp - 2) * 8, (warp - 1) * 8, lane);
         fence_proxy_async();   // B is read by the tensor core through the async proxy
         __syncwarp();
@@ -308,6 +315,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             // ---- a new lambda row: this group needs its rho; the group that meets the row's first tile rebuilds B
             if (seg != cached_seg) {
                 const RecipLambda rl(lambda_row(seg), lane);
+                if (rl.wide && q == 0 && lane == 0) atomicOr(status, KVQ_DEV_RANGE);
                 rho = rl.rho;
                 if (cur.first_of_segment()) {
                     // every MMA issued so far must have read B: the mma thread says so by raising b_epoch to this row's index

@@ -690,6 +690,45 @@ def test_degenerate_inputs(D, dtype, impl):
         plan.close()
 
 
+@pytest.mark.parametrize("impl", ["fft", "gemm", "matvec"])
+@pytest.mark.parametrize("D,dtype", [(128, "f16"), (256, "bf16"), (96, "f16")])
+@pytest.mark.parametrize("wild", [False, True])
+def test_degenerate_lambda(D, dtype, impl, wild):
+    # mild: lambda entries spread over a factor of 100 inside a row, and a row a thousand times smaller than the other.
+    # wild: entries that are zero, negative, below the 1e-6 clamp of the inverse path, or very large: the forward path
+    # multiplies by them as they are, the inverse divides by max(lambda, 1e-6) (Sec. 5.1 item 1).  The tensor-core decode
+    # carries 1 / lambda inside an fp16 operand next to the other channels' and says so (status bit 3) when a row's
+    # reciprocals span more than 2^8; the other families are fp32 and exact.
+    odt = ko.F16 if dtype == "f16" else ko.BF16
+    N = 3000
+    lam = wl.make_lambda(2, D, 40)
+    lam[0] = lam[0] * torch.logspace(-1, 1, D)[torch.randperm(D, generator=torch.Generator().manual_seed(1))]
+    lam[1, :] = 1e-3 * lam[1, :]
+    if wild:
+        lam[0, 3], lam[0, 17], lam[0, 40], lam[0, D - 1], lam[0, 64] = 0.0, -1.5, 1e-8, 3e3, 1e-6
+        lam[1, 5] = 2.0e-7
+    x = wl.make_vectors(N, D, dtype, "k_outlier", 41)
+    plan = kb.Plan(D, G, 42)
+    kb.kvq_plan_set_impl(plan.handle, IMPL[impl], IMPL[impl])
+    sg = plan.signs()
+    packed, scales = gpu_encode(plan, x.cuda(), lam.cuda(), 1500)
+    ora = ko.encode(bits(x), odt, sg, lam.numpy(), G, 1500, want_v=True)
+    parity.check_encode(packed.cpu().numpy(), bits(scales), ora, G, "odd lambda encode (%s)" % impl)
+    ob, o64 = ko.decode(ora["packed"], ora["scales"], sg, lam.numpy(), G, odt, 1500, want_f64=True)
+    out = gpu_decode_raw(plan, torch.from_numpy(ora["packed"]).cuda(),
+                         torch.from_numpy(ora["scales"].view(np.int16)).view(torch.float16).cuda(), lam.cuda(), dtype, 1500)
+    word = kb.kvq_plan_device_status(plan.handle)
+    if wild and impl == "gemm":
+        assert word == 8                             # reported, not decoded: KVQ_IMPL_MATVEC / KVQ_IMPL_FFT are the exact paths
+    else:
+        assert word == 0
+        lim = 65504.0 if dtype == "f16" else 3.0e38
+        ok = np.abs(o64).max(axis=1) < 0.25 * lim    # dividing by 1e-6 takes some rows out of fp16's range: both sides then say inf
+        assert ok.sum() >= 0.3 * N
+        parity.check_decode(bits(out)[ok], ob[ok], o64[ok], odt, "odd lambda decode (%s)" % impl)
+    plan.close()
+
+
 def test_rotated_d256_decode_reports_scales_outside_its_operand_range():
     # the dense 256 x 256 kernel of rotated plans has no room for the per-row rescue: it flags such rows (status bit 3)
     # and leaves them to the matrix-vector kernel, which is fp32 throughout
