@@ -144,6 +144,10 @@ kvq_status_t kvq_plan_set_impl(kvq_plan_t *plan, kvq_impl_t encode_impl, kvq_imp
  * Returns KVQ_ERR_RANGE if bit 3 is the only bit set.  The word is sticky for the plan's lifetime. */
 kvq_status_t kvq_plan_device_status(kvq_plan_t *plan, uint32_t *word);
 
+/* Synchronizes the current device and clears the plan's device status word (after the caller has dealt with what it
+ * reported).  Call it with the plan's device current and no call using the plan in flight. */
+kvq_status_t kvq_plan_clear_device_status(kvq_plan_t *plan);
+
 /*
  * kvq_encode -- forward path (Sec. 3.2 steps 1-4 with the fused lambda and per-group scales of
  * Sec. 7.1) on N vectors.

@@ -38,7 +38,7 @@ KVQ_IMPL_MATVEC = 3
 
 # every symbol include/kvq.h declares
 EXPORTS = (
-    "kvq_plan_create", "kvq_plan_create_ex", "kvq_plan_set_rotation", "kvq_plan_destroy", "kvq_plan_get_signs", "kvq_plan_describe", "kvq_plan_set_impl",
+    "kvq_plan_create", "kvq_plan_create_ex", "kvq_plan_set_rotation", "kvq_plan_clear_device_status", "kvq_plan_destroy", "kvq_plan_get_signs", "kvq_plan_describe", "kvq_plan_set_impl",
     "kvq_plan_device_status", "kvq_encode", "kvq_decode", "kvq_append", "kvq_decode_static", "kvq_calibrate_lambda", "kvq_flush_block", "kvq_status_string",
     "kvq_launch_count",
 )
@@ -63,6 +63,8 @@ def lib() -> ctypes.CDLL:
         i32, i64, u64, vp = ctypes.c_int, ctypes.c_int64, ctypes.c_uint64, ctypes.c_void_p
         L.kvq_plan_create.restype = i32
         L.kvq_plan_create.argtypes = [i32, i32, u64, ctypes.POINTER(vp)]
+        L.kvq_plan_clear_device_status.restype = i32
+        L.kvq_plan_clear_device_status.argtypes = [vp]
         L.kvq_plan_set_rotation.restype = i32
         L.kvq_plan_set_rotation.argtypes = [vp, vp]
         L.kvq_plan_create_ex.restype = i32
@@ -222,6 +224,10 @@ def kvq_plan_device_status(plan: int) -> int:
     if st not in (KVQ_OK, KVQ_ERR_TIMEOUT, KVQ_ERR_RANGE):
         raise KvqError(st, "kvq_plan_device_status")
     return int(w.value)
+
+
+def kvq_plan_clear_device_status(plan: int) -> None:
+    _check(lib().kvq_plan_clear_device_status(plan), "kvq_plan_clear_device_status")
 
 
 def kvq_encode(plan: int, x: torch.Tensor, lam: torch.Tensor, packed: torch.Tensor, scales: torch.Tensor,

@@ -326,6 +326,17 @@ kvq_status_t kvq_plan_device_status(kvq_plan_t *plan, uint32_t *word)
     return *word ? KVQ_ERR_RANGE : KVQ_OK;
 }
 
+kvq_status_t kvq_plan_clear_device_status(kvq_plan_t *plan)
+{
+    if (!plan) return KVQ_ERR_INVALID_ARG;
+    if (!plan->d_status) return KVQ_OK;   // never used on a device
+    if (cudaDeviceSynchronize() != cudaSuccess || cudaMemset(plan->d_status, 0, sizeof(uint32_t)) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return KVQ_ERR_CUDA;
+    }
+    return KVQ_OK;
+}
+
 static kvq_status_t encode_common(kvq_plan_t *plan, const void *x, kvq_dtype_t dtype, int64_t N, const float *lambda,
                                   int64_t n_lambda, int64_t rows_per_lambda, uint8_t *packed, void *scales,
                                   const RowMap &out_map, void *cuda_stream)

@@ -720,6 +720,8 @@ def test_degenerate_lambda(D, dtype, impl, wild):
     word = kb.kvq_plan_device_status(plan.handle)
     if wild and impl == "gemm":
         assert word == 8                             # reported, not decoded: KVQ_IMPL_MATVEC / KVQ_IMPL_FFT are the exact paths
+        kb.kvq_plan_clear_device_status(plan.handle)
+        assert kb.kvq_plan_device_status(plan.handle) == 0
     else:
         assert word == 0
         lim = 65504.0 if dtype == "f16" else 3.0e38
