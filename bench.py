@@ -419,7 +419,7 @@ def measure_incremental(kb, wl, dev, dec_avg_ms, iters=20, window=16):
     flush_us = 1e3 * statistics.median(ms)
     return {"window_tokens": window, "streams": S, "flush_us": flush_us, "flush_us_per_generated_token": flush_us / window,
             "full_prefix_decode_us_per_generated_token": 1e3 * dec_avg_ms,
-            "note": "one layer; the flush is two launches of %d vectors (launch-bound), independent of the prefix length" % (S * window)}
+            "note": "one layer; the flush is one launch over %d vectors (launch-bound), independent of the prefix length" % (S * window)}
 
 
 # DRAM bytes per full launch (2,097,152 vectors, the bench's launch size) from ncu: dram__bytes_read.sum +

@@ -196,8 +196,10 @@ kvq_status_t kvq_append(kvq_plan_t *plan, const void *x_new /* [S, D] */, kvq_dt
  *   x_block       device, [S, rows, D] row-major, fp16 or bf16 per `dtype`; 16-byte aligned.
  *   lambda, n_lambda, streams_per_lambda, packed_cache [S, T_max, D/2], scales_cache [S, T_max, D/group]: as in kvq_append.
  *   dq_cache      device out, [S, T_max, D] of the same 16-bit type; 16-byte aligned.  Only rows [pos0, pos0 + rows) are written.
- * Requires 0 <= pos0 and pos0 + rows <= T_max.  S == 0 or rows == 0 is a no-op.  Two launches on the stream (the
- * matrix-vector kernels when S * rows <= 2048 (1024 for D > 128) or the plan is rotated).  The
+ * Requires 0 <= pos0 and pos0 + rows <= T_max.  S == 0 or rows == 0 is a no-op.  One launch on the stream when
+ * S * rows <= 2048 (1024 for D > 128): the matrix-vector kernel quantizes a vector, dequantizes it from the values it
+ * stored and transforms it back in the same CTA.  Larger blocks take two launches (the encode as kvq_encode picks it,
+ * then a decode of the stored rows).  The
  * window itself (holding the not yet flushed tokens in fp16) is the caller's buffer: this call is its flush.
  */
 kvq_status_t kvq_flush_block(kvq_plan_t *plan, const void *x_block, kvq_dtype_t dtype, int64_t S, int64_t rows,

@@ -337,9 +337,18 @@ kvq_status_t kvq_plan_clear_device_status(kvq_plan_t *plan)
     return KVQ_OK;
 }
 
+// The decode half of a block flush: small blocks (the window flush) and rotated plans take the matrix-vector kernel,
+// large plain blocks the register FFT.
+static bool flush_decode_is_matvec(const kvq_plan_t *plan, int64_t N)
+{
+    return plan->rot || plan->dec_impl == KVQ_IMPL_MATVEC || (plan->dec_impl != KVQ_IMPL_FFT && N <= matvec_max_rows(plan->D));
+}
+
+// dq / fused: the window flush.  Where the call takes the matrix-vector kernel and the plan's decode side would take it
+// too, the dequantized rows go to dq (rows out_map(r)) in the same launch and *fused is set.
 static kvq_status_t encode_common(kvq_plan_t *plan, const void *x, kvq_dtype_t dtype, int64_t N, const float *lambda,
                                   int64_t n_lambda, int64_t rows_per_lambda, uint8_t *packed, void *scales,
-                                  const RowMap &out_map, void *cuda_stream)
+                                  const RowMap &out_map, void *cuda_stream, void *dq = nullptr, bool *fused = nullptr)
 {
     if (!plan || N < 0) return KVQ_ERR_INVALID_ARG;
     if (dtype != KVQ_F16 && dtype != KVQ_BF16) return KVQ_ERR_INVALID_ARG;
@@ -373,7 +382,11 @@ static kvq_status_t encode_common(kvq_plan_t *plan, const void *x, kvq_dtype_t d
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     cudaError_t e;
     if (impl == KVQ_IMPL_GEMM) e = umma_encode(plan->D, bf16, per_vector, N, prm, plan->d_e0, stream);
-    else if (impl == KVQ_IMPL_MATVEC) e = matvec_encode(plan->D, plan->group, plan->bits, bf16, N, prm, plan->d_b0, stream);
+    else if (impl == KVQ_IMPL_MATVEC && dq && fused && flush_decode_is_matvec(plan, N)) {
+        prm.out = dq;
+        e = matvec_flush(plan->D, plan->group, plan->bits, bf16, N, prm, plan->d_b0, plan->d_e0, stream);
+        *fused = e == cudaSuccess;
+    } else if (impl == KVQ_IMPL_MATVEC) e = matvec_encode(plan->D, plan->group, plan->bits, bf16, N, prm, plan->d_b0, stream);
     else e = fft_encode(plan->D, plan->group, plan->bits, bf16, N, prm, stream);
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
@@ -469,8 +482,11 @@ kvq_status_t kvq_flush_block(kvq_plan_t *plan, const void *x_block, kvq_dtype_t 
     // lambda row of block row r: stream (r / rows) / streams_per_lambda
     const int64_t rpl = (streams_per_lambda < 1 ? 1 : streams_per_lambda) * rows;
     const RowMap map{rows, T_max, pos0};
-    kvq_status_t st = encode_common(plan, x_block, dtype, N, lambda, n_lambda, rpl, packed_cache, scales_cache, map, cuda_stream);
-    if (st != KVQ_OK) return st;
+    if (plan->rot && plan->dec_impl == KVQ_IMPL_FFT) return KVQ_ERR_UNSUPPORTED_DIM;
+    bool fused = false;
+    kvq_status_t st = encode_common(plan, x_block, dtype, N, lambda, n_lambda, rpl, packed_cache, scales_cache, map, cuda_stream,
+                                    dq_cache, &fused);
+    if (st != KVQ_OK || fused) return st;
     // the same rows back out of the int4 cache into the dequantized-prefix cache: what a later full-prefix decode would give
     FftParams prm;
     fill_params(plan, prm, N, lambda, n_lambda, rpl);
@@ -479,9 +495,7 @@ kvq_status_t kvq_flush_block(kvq_plan_t *plan, const void *x_block, kvq_dtype_t 
     prm.out = dq_cache;
     prm.in_map = map;
     prm.out_map = map;
-    // small blocks (the window flush) and rotated plans: matrix-vector kernel; large plain blocks: register FFT
-    if (plan->rot && plan->dec_impl == KVQ_IMPL_FFT) return KVQ_ERR_UNSUPPORTED_DIM;
-    const bool mv = plan->rot || plan->dec_impl == KVQ_IMPL_MATVEC || (plan->dec_impl != KVQ_IMPL_FFT && N <= matvec_max_rows(plan->D));
+    const bool mv = flush_decode_is_matvec(plan, N);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const cudaError_t e = mv ? matvec_decode(plan->D, plan->group, plan->bits, dtype == KVQ_BF16, N, prm, plan->d_e0, stream)
                              : fft_decode(plan->D, plan->group, plan->bits, dtype == KVQ_BF16, N, prm, stream);

@@ -73,6 +73,8 @@ cudaError_t umma_encode(int D, bool bf16, bool per_vector, int64_t N, const FftP
 // fp32 matrix-vector kernels for small calls (kvq_matvec.cu): every layout, dtype and D; b0 / e0 are the plan's tables
 cudaError_t matvec_encode(int D, int group, int bits, bool bf16, int64_t N, const FftParams &prm, const float *b0, cudaStream_t stream);
 cudaError_t matvec_decode(int D, int group, int bits, bool bf16, int64_t N, const FftParams &prm, const float *e0, cudaStream_t stream);
+cudaError_t matvec_flush(int D, int group, int bits, bool bf16, int64_t N, const FftParams &prm, const float *b0, const float *e0,
+                         cudaStream_t stream);   // encode + decode of the same rows in one launch
 // group: 32 or D (one scale per vector); bits: 4 or 8
 cudaError_t fft_encode(int D, int group, int bits, bool bf16, int64_t N, const FftParams &prm, cudaStream_t stream);
 cudaError_t fft_decode(int D, int group, int bits, bool bf16, int64_t N, const FftParams &prm, cudaStream_t stream);

@@ -33,6 +33,7 @@ struct MatvecParams {
     void *scales;          // [*, D / group] fp16
     void *out;             // decode: [*, D] half precision
     const float *table;    // encode: b0[n][c] (column c of the forward transform along a row); decode: e0[c][n]
+    const float *table2;   // fused window flush: e0[c][n], for the way back
     int64_t N, n_lambda, rows_per_lambda;
     RowMap out_map, in_map;
     int group, bits;
@@ -131,7 +132,11 @@ __device__ __forceinline__ void matvec(const float *__restrict__ table, float4 (
 // ------------------------------------------------------------------------------------------------
 // encode: x -> codes and scales  (Sec. 3.2 steps 1-4, lambda and group scales of Sec. 7.1)
 // ------------------------------------------------------------------------------------------------
-template <int D, bool BF16>
+// FLUSH: the window flush in one launch (Sec. 7.2).  After the codes of a vector are stored, the warp that finished it puts
+// q sigma / max(lambda, 1e-6) -- what kvq_decode would rebuild from the stored bytes -- back into shared memory, and the
+// CTA runs the matrix-vector product once more with the inverse table: rows out_map(r) of prm.out get the dequantized
+// vectors.
+template <int D, bool BF16, bool FLUSH>
 __global__ void __launch_bounds__(kWarps * 32) kvq_encode_matvec_kernel(const __grid_constant__ MatvecParams prm)
 {
     using Gm = Geo<D>;
@@ -168,8 +173,9 @@ __global__ void __launch_bounds__(kWarps * 32) kvq_encode_matvec_kernel(const __
     matvec<D>(prm.table, t, xs, red, warp, lane, z);
 
     // ---- warp w finishes vector w
-    if (r >= prm.N) return;
-    const int64_t orow = prm.out_map(r);
+    const bool live = r < prm.N;
+    if (!FLUSH && !live) return;
+    const int64_t orow = live ? prm.out_map(r) : 0;
     const bool per_vector = prm.group == D;
     const float Q = prm.bits == 4 ? 7.0f : 127.0f;
     float amax[P];
@@ -210,20 +216,45 @@ __global__ void __launch_bounds__(kWarps * 32) kvq_encode_matvec_kernel(const __
         const float rs = sg > 0.0f ? __frcp_rn(sg) : 0.0f;
         const bool clamp = !(amax[p] * rs < Q + 0.25f);   // saturated or subnormal scale: codes could leave [-Q, Q]
         if (i >= D / 4) continue;
-        if (per_vector ? (lane == 0 && p == 0) : ((i & 7) == 0))
+        if (live && (per_vector ? (lane == 0 && p == 0) : ((i & 7) == 0)))
             scl[orow * (D / prm.group) + (per_vector ? 0 : i >> 3)] = __half_as_ushort(hs);
         uint32_t code[4];
+        float qf[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             const float t = clamp ? fminf(fmaxf(z[p][e] * rs, -Q), Q) + 12582912.0f : fmaf(z[p][e], rs, 12582912.0f);
             code[e] = __float_as_uint(t);   // low bits: q in two's complement (1.5 * 2^23 + q)
+            qf[e] = t - 12582912.0f;        // q itself, exactly
         }
-        if (prm.bits == 4) {
-            const uint32_t w = (code[0] & 0xFu) | ((code[1] & 0xFu) << 4) | ((code[2] & 0xFu) << 8) | ((code[3] & 0xFu) << 12);
-            *reinterpret_cast<uint16_t *>(pk + orow * (D / 2) + 2 * i) = (uint16_t)w;
-        } else {
-            const uint32_t w = (code[0] & 0xFFu) | ((code[1] & 0xFFu) << 8) | ((code[2] & 0xFFu) << 16) | (code[3] << 24);
-            *reinterpret_cast<uint32_t *>(pk + orow * D + 4 * i) = w;
+        if (live) {
+            if (prm.bits == 4) {
+                const uint32_t w = (code[0] & 0xFu) | ((code[1] & 0xFu) << 4) | ((code[2] & 0xFu) << 8) | ((code[3] & 0xFu) << 12);
+                *reinterpret_cast<uint16_t *>(pk + orow * (D / 2) + 2 * i) = (uint16_t)w;
+            } else {
+                const uint32_t w = (code[0] & 0xFFu) | ((code[1] & 0xFFu) << 8) | ((code[2] & 0xFFu) << 16) | (code[3] << 24);
+                *reinterpret_cast<uint32_t *>(pk + orow * D + 4 * i) = w;
+            }
+        }
+        if constexpr (FLUSH) {   // the way back starts from the stored values: q times the STORED scale over the clamped lambda
+            const float4 l = lam4[p];
+            const float4 o = make_float4(qf[0] * (sg * __frcp_rn(fmaxf(l.x, 1e-6f))), qf[1] * (sg * __frcp_rn(fmaxf(l.y, 1e-6f))),
+                                         qf[2] * (sg * __frcp_rn(fmaxf(l.z, 1e-6f))), qf[3] * (sg * __frcp_rn(fmaxf(l.w, 1e-6f))));
+            *reinterpret_cast<float4 *>(xs + warp * D + 4 * i) = live ? o : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        }
+    }
+    if constexpr (FLUSH) {
+        float4 t2[Gm::CH][P];
+        load_rows<D>(prm.table2, warp, lane, 0, t2);   // in flight across the barrier
+        __syncthreads();                               // every warp's vector is back in shared memory; red is free again
+        float y[P][4];
+        matvec<D>(prm.table2, t2, xs, red, warp, lane, y);
+        if (!live) return;
+        unsigned char *out = static_cast<unsigned char *>(prm.out) + orow * (2 * D);
+#pragma unroll
+        for (int p = 0; p < P; ++p) {
+            const int i = lane + 32 * p;
+            if (i < D / 4)
+                *reinterpret_cast<uint2 *>(out + 8 * i) = make_uint2(narrow2<BF16>(y[p][0], y[p][1]), narrow2<BF16>(y[p][2], y[p][3]));
         }
     }
 }
@@ -288,14 +319,15 @@ __global__ void __launch_bounds__(kWarps * 32) kvq_decode_matvec_kernel(const __
     }
 }
 
-template <int D, bool BF16, bool ENC>
+// MODE: 0 decode, 1 encode, 2 encode + decode of the same rows (window flush)
+template <int D, bool BF16, int MODE>
 cudaError_t launch(const MatvecParams &prm, cudaStream_t stream)
 {
     static DeviceSlots slots;
     int dev = 0;
     cudaError_t e = current_device_slot(&dev);
     if (e != cudaSuccess) return e;
-    auto kern = ENC ? kvq_encode_matvec_kernel<D, BF16> : kvq_decode_matvec_kernel<D, BF16>;
+    auto kern = MODE == 0 ? kvq_decode_matvec_kernel<D, BF16> : MODE == 1 ? kvq_encode_matvec_kernel<D, BF16, false> : kvq_encode_matvec_kernel<D, BF16, true>;
     if (slots.sms[dev] == 0) {
         if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<D>::kSmemBytes)) != cudaSuccess) return e;
         slots.sms[dev] = 1;
@@ -307,15 +339,15 @@ cudaError_t launch(const MatvecParams &prm, cudaStream_t stream)
     return cudaGetLastError();
 }
 
-template <bool ENC>
+template <int MODE>
 cudaError_t dispatch(int D, bool bf16, const MatvecParams &prm, cudaStream_t stream)
 {
     switch (D) {
-        case 64: return bf16 ? launch<64, true, ENC>(prm, stream) : launch<64, false, ENC>(prm, stream);
-        case 96: return bf16 ? launch<96, true, ENC>(prm, stream) : launch<96, false, ENC>(prm, stream);
-        case 128: return bf16 ? launch<128, true, ENC>(prm, stream) : launch<128, false, ENC>(prm, stream);
-        case 160: return bf16 ? launch<160, true, ENC>(prm, stream) : launch<160, false, ENC>(prm, stream);
-        case 256: return bf16 ? launch<256, true, ENC>(prm, stream) : launch<256, false, ENC>(prm, stream);
+        case 64: return bf16 ? launch<64, true, MODE>(prm, stream) : launch<64, false, MODE>(prm, stream);
+        case 96: return bf16 ? launch<96, true, MODE>(prm, stream) : launch<96, false, MODE>(prm, stream);
+        case 128: return bf16 ? launch<128, true, MODE>(prm, stream) : launch<128, false, MODE>(prm, stream);
+        case 160: return bf16 ? launch<160, true, MODE>(prm, stream) : launch<160, false, MODE>(prm, stream);
+        case 256: return bf16 ? launch<256, true, MODE>(prm, stream) : launch<256, false, MODE>(prm, stream);
     }
     return cudaErrorInvalidValue;
 }
@@ -325,6 +357,7 @@ MatvecParams from_fft(const FftParams &f, const float *table, int group, int bit
     MatvecParams p;
     p.in = f.in, p.lambda = f.lambda, p.packed = f.packed, p.scales = f.scales, p.out = f.out;
     p.table = table;
+    p.table2 = nullptr;
     p.N = f.N, p.n_lambda = f.n_lambda, p.rows_per_lambda = f.rows_per_lambda;
     p.out_map = f.out_map, p.in_map = f.in_map;
     p.group = group, p.bits = bits;
@@ -337,13 +370,24 @@ MatvecParams from_fft(const FftParams &f, const float *table, int group, int bit
 cudaError_t matvec_encode(int D, int group, int bits, bool bf16, int64_t N, const FftParams &f, const float *b0, cudaStream_t stream)
 {
     (void)N;
-    return dispatch<true>(D, bf16, from_fft(f, b0, group, bits), stream);
+    return dispatch<1>(D, bf16, from_fft(f, b0, group, bits), stream);
 }
 
 cudaError_t matvec_decode(int D, int group, int bits, bool bf16, int64_t N, const FftParams &f, const float *e0, cudaStream_t stream)
 {
     (void)N;
-    return dispatch<false>(D, bf16, from_fft(f, e0, group, bits), stream);
+    return dispatch<0>(D, bf16, from_fft(f, e0, group, bits), stream);
+}
+
+// The window flush in one launch: x rows -> codes and scales at rows out_map(r) of the caches, and the dequantized
+// vectors at the same rows of f.out.
+cudaError_t matvec_flush(int D, int group, int bits, bool bf16, int64_t N, const FftParams &f, const float *b0, const float *e0,
+                         cudaStream_t stream)
+{
+    (void)N;
+    MatvecParams p = from_fft(f, b0, group, bits);
+    p.table2 = e0;
+    return dispatch<2>(D, bf16, p, stream);
 }
 
 }  // namespace kvq

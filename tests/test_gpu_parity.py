@@ -396,6 +396,46 @@ def test_flush_block_fills_the_int4_and_the_dequantized_caches(D, dtype, S, T_ma
     plan.close()
 
 
+@pytest.mark.parametrize("D", [64, 96, 128, 160, 256])
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("group,nbits", [(G, 4), (0, 4), (G, 8)])
+def test_window_flush_in_one_launch_equals_decode_of_what_it_stored(D, dtype, group, nbits):
+    """A small flush runs as ONE matrix-vector launch that dequantizes in the encode's registers; the rows it leaves in the
+    dequantized cache must be, bit for bit, what the matrix-vector kvq_decode makes of the codes and scales it stored."""
+    g = group or D
+    tdt = torch.float16 if dtype == "f16" else torch.bfloat16
+    S, T_max, rows, pos0, spl = 13, 40, 11, 17, 3        # 143 vectors: 17 full CTAs of 8 and a ragged one
+    plan = kb.Plan(D, g, 77, nbits)
+    lamd = wl.make_lambda((S + spl - 1) // spl, D, 78).cuda()
+    x = wl.make_vectors(S * rows, D, dtype, "k_outlier", 79).view(S, rows, D).cuda()
+    packed = torch.full((S, T_max, D * nbits // 8), 0xAB, dtype=torch.uint8, device="cuda")
+    scales = torch.full((S, T_max, D // g), 1.25, dtype=torch.float16, device="cuda")
+    dq = torch.full((S, T_max, D), 3.0, dtype=tdt, device="cuda")
+    n0 = kb.kvq_launch_count()
+    kb.kvq_flush_block(plan.handle, x, lamd, packed, scales, dq, pos0, spl)
+    assert kb.kvq_launch_count() - n0 == 1
+    # the caches hold what the two-launch form (append-style encode, then decode) stores
+    p2, s2 = torch.full_like(packed, 0xAB), torch.full_like(scales, 1.25)
+    kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_MATVEC, kb.KVQ_IMPL_FFT)   # a decode side that is not matrix-vector: two launches
+    dq2 = torch.full_like(dq, 3.0)
+    n0 = kb.kvq_launch_count()
+    kb.kvq_flush_block(plan.handle, x, lamd, p2, s2, dq2, pos0, spl)
+    assert kb.kvq_launch_count() - n0 == 2
+    assert torch.equal(packed, p2) and torch.equal(scales, s2)
+    kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_MATVEC, kb.KVQ_IMPL_MATVEC)
+    blk_p = packed[:, pos0:pos0 + rows].reshape(S * rows, -1).contiguous()
+    blk_s = scales[:, pos0:pos0 + rows].reshape(S * rows, -1).contiguous()
+    out = torch.empty(S * rows, D, dtype=tdt, device="cuda")
+    kb.kvq_decode(plan.handle, blk_p, blk_s, lamd, out, spl * rows)
+    torch.cuda.synchronize()
+    assert kb.kvq_plan_device_status(plan.handle) == 0
+    assert torch.equal(dq[:, pos0:pos0 + rows].reshape(S * rows, D).view(torch.int16), out.view(torch.int16))
+    mask = torch.ones(T_max, dtype=torch.bool, device="cuda")
+    mask[pos0:pos0 + rows] = False
+    assert bool((dq[:, mask] == 3.0).all()) and bool((packed[:, mask] == 0xAB).all()) and bool((scales[:, mask] == 1.25).all())
+    plan.close()
+
+
 def test_flush_block_rejects_blocks_outside_the_cache():
     D, S, T = 128, 4, 16
     plan = kb.Plan(D, G, 1)
