@@ -279,9 +279,11 @@ def run_ours(args):
         return
 
     copy_gbs = measure_sustained_copy(slots, dev)
-    d256 = measure_d256(kb, wl, dev)
-    incr = measure_incremental(kb, wl, dev, dec_avg_ms=sum(dec_ms) / len(dec_ms))
-    sweep = measure_model_sweep(kb, wl, dev, shp.dtype, S, T)
+    d256 = incr = sweep = None
+    if not args.no_side:
+        d256 = measure_d256(kb, wl, dev)
+        incr = measure_incremental(kb, wl, dev, dec_avg_ms=sum(dec_ms) / len(dec_ms))
+        sweep = measure_model_sweep(kb, wl, dev, shp.dtype, S, T)
     step_bytes = (2 * N + S) * BYTES_PER_VEC
     value = world * args.steps * step_bytes / (ms_total * 1e-3) / 1e9
     peak, peak_src = measured_peak()
@@ -565,6 +567,8 @@ def main():
     ap.add_argument("--steps", type=int, default=2000)   # 0.6 s of back-to-back steps: long enough to sample the clocks under load
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-side", action="store_true",
+                    help="leave out the measurements beside the timed region (D=256, window flush, 80-layer sweep): for a launch list")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3

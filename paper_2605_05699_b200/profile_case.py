@@ -90,7 +90,7 @@ def sustain(a):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--op", choices=["encode", "decode", "append", "copy"], default="decode")
+    ap.add_argument("--op", choices=["encode", "decode", "append", "flush", "copy"], default="decode")
     ap.add_argument("--D", type=int, default=128)
     ap.add_argument("--dtype", choices=["f16", "bf16"], default="f16")
     ap.add_argument("--n", type=int, default=1 << 20)
@@ -100,7 +100,7 @@ def main():
     ap.add_argument("--sustain", type=float, default=0.0, help="seconds of back-to-back launches with nvidia-smi sampling")
     a = ap.parse_args()
     if a.sustain > 0:
-        if a.op == "append":
+        if a.op in ("append", "flush"):
             ap.error("--sustain takes encode, decode or copy")
         return sustain(a)
     if a.op == "copy":
@@ -126,14 +126,17 @@ def main():
             kb.kvq_encode(plan.handle, x, lam, packed, scales)
         elif a.op == "decode":
             kb.kvq_decode(plan.handle, packed, scales, lam, out)
-        else:
+        elif a.op == "append":
             kb.kvq_append(plan.handle, x[:4096], lam, packed.view(4096, -1, D // 2), scales.view(4096, -1, D // G), 1)
+        else:   # the window flush: 64 streams x 16 new tokens into caches of n / 64 rows per stream, one launch
+            kb.kvq_flush_block(plan.handle, x[:1024].view(64, 16, D), lam, packed.view(64, -1, D // 2), scales.view(64, -1, D // G),
+                               out.view(64, -1, D), 16)
         e1.record()
         torch.cuda.synchronize()
     ms = e0.elapsed_time(e1)
     assert kb.kvq_plan_device_status(plan.handle) == 0
     bpv = 2 * D + D // 2 + 2 * (D // G)
-    n_eff = 4096 if a.op == "append" else N
+    n_eff = 4096 if a.op == "append" else 1024 if a.op == "flush" else N
     print(json.dumps({"op": a.op, "D": D, "dtype": a.dtype, "n": n_eff, "impl": a.impl, "ms_last": ms,
                       "ns_per_vec": ms * 1e6 / n_eff, "algorithmic_GBps": n_eff * bpv / (ms * 1e-3) / 1e9}))
 
