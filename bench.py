@@ -477,11 +477,75 @@ def measure_incremental(kb, wl, dev, dec_avg_ms, iters=20, window=16):
     queued_us = 1e3 * e0.elapsed_time(e1) / iters
     assert kb.kvq_plan_device_status(plan.handle) == 0
     plan.close()
+    del packed, scales, dq
     flush_us = 1e3 * statistics.median(ms)
     return {"window_tokens": window, "streams": S, "flush_us": flush_us, "flush_us_queued": queued_us,
+            "append_dispatch": measure_append_dispatch(kb, wl, dev, shp.dtype, S),
             "flush_us_per_generated_token": flush_us / window,
             "full_prefix_decode_us_per_generated_token": 1e3 * dec_avg_ms,
             "note": "one layer; the flush is one launch over %d vectors (launch-bound), independent of the prefix length" % (S * window)}
+
+
+def measure_append_dispatch(kb, wl, dev, dtype, S, layers=80, T=1024, iters=20):
+    """Outside the timed region: what the per-step append of a whole model (80 layers x 64 streams) costs by how it is
+    dispatched -- one call per layer, the same 80 calls replayed as one CUDA graph (positions in device memory), and all
+    5120 streams in ONE call (layers are streams of one cache, lambda row per layer and K / V)."""
+    import torch
+
+    plan = kb.Plan(D, GROUP, 47)
+    lam = wl.make_lambda(2 * layers, D, 48, device=dev)
+    x = wl.make_vectors(layers * S, D, dtype, "gaussian", 49, device=dev).view(layers, S, D)
+    packed = torch.zeros(layers, S, T, D // 2, dtype=torch.uint8, device=dev)
+    scales = torch.zeros(layers, S, T, D // GROUP, dtype=torch.float16, device=dev)
+    pos = torch.zeros(1, dtype=torch.int64, device=dev)
+    h = plan.handle
+
+    def per_layer():
+        for l in range(layers):
+            kb.kvq_append_at(h, x[l], lam[2 * l:2 * l + 2], packed[l], scales[l], pos, S // 2)
+
+    def one_call():
+        kb.kvq_append_at(h, x.view(layers * S, D), lam, packed.view(layers * S, T, D // 2), scales.view(layers * S, T, D // GROUP),
+                         pos, S // 2)
+
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        per_layer()
+        one_call()
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        per_layer()
+        pos.add_(1)
+
+    def timed(fn):
+        out = []
+        for i in range(iters + 2):
+            pos.fill_(i % T)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            t0 = time.perf_counter()
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            wall = 1e6 * (time.perf_counter() - t0)
+            if i >= 2:
+                out.append((1e3 * e0.elapsed_time(e1), wall))
+        return statistics.median(o[0] for o in out), statistics.median(o[1] for o in out)
+
+    eager = timed(per_layer)
+    replay = timed(graph.replay)
+    single = timed(one_call)
+    assert kb.kvq_plan_device_status(h) == 0
+    plan.close()
+    return {"layers": layers, "streams_per_layer": S,
+            "call_per_layer_us": eager[0], "call_per_layer_host_wall_us": eager[1],
+            "cuda_graph_of_the_same_calls_us": replay[0], "cuda_graph_host_wall_us": replay[1],
+            "one_call_all_layers_us": single[0], "one_call_host_wall_us": single[1],
+            "note": "device time between events around the step / host wall time until the step has finished, medians; "
+                    "kvq_append_at reads the row from device memory, so the graph is replayed as is for every position"}
 
 
 # DRAM bytes per full launch (2,097,152 vectors, the bench's launch size) from ncu: dram__bytes_read.sum +

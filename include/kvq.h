@@ -141,7 +141,10 @@ kvq_status_t kvq_plan_set_impl(kvq_plan_t *plan, kvq_impl_t encode_impl, kvq_imp
  *     or below the row's largest reciprocal; very small or very large vectors): all kernels but
  *     one rescale such rows by a power of two and are exact for them; the dense D = 256 kernel
  *     of ROTATED plans reports them instead.
- * Returns KVQ_ERR_RANGE if bit 3 is the only bit set.  The word is sticky for the plan's lifetime. */
+ * Bit 4: kvq_append_at or kvq_flush_block_at found a position outside the cache in device memory and
+ * wrote nothing: returns KVQ_ERR_INVALID_ARG (unless bits 0-2 are set too).
+ * Returns KVQ_ERR_RANGE if bit 3 is the only bit set.  The word is sticky until
+ * kvq_plan_clear_device_status. */
 kvq_status_t kvq_plan_device_status(kvq_plan_t *plan, uint32_t *word);
 
 /* Synchronizes the current device and clears the plan's device status word (after the caller has dealt with what it
@@ -205,6 +208,27 @@ kvq_status_t kvq_append(kvq_plan_t *plan, const void *x_new /* [S, D] */, kvq_dt
 kvq_status_t kvq_flush_block(kvq_plan_t *plan, const void *x_block, kvq_dtype_t dtype, int64_t S, int64_t rows,
                              const float *lambda, int64_t n_lambda, int64_t streams_per_lambda, uint8_t *packed_cache,
                              void *scales_cache, void *dq_cache, int64_t T_max, int64_t pos0, void *cuda_stream);
+
+/*
+ * kvq_append_at, kvq_flush_block_at -- kvq_append and kvq_flush_block with the cache position held in DEVICE memory.
+ * (Sec. 7.2's decode loop is dominated by dispatch at these sizes; a loop that is recorded once as a CUDA graph and
+ * replayed needs every per-step value to come from memory, not from a launch argument.)
+ *   pos_device / pos0_device   device, one int64_t, 8-byte aligned: the row (first row) to write.  It is read when the
+ *                 kernel runs, so the same call -- or a CUDA graph that holds it -- serves successive positions once
+ *                 the caller updates that word on the same stream.  A value outside [0, T_max - 1] (append) or
+ *                 [0, T_max - rows] (flush) writes nothing and raises bit 4 of the plan's device status word.
+ * Everything else as in kvq_append / kvq_flush_block (same stored bytes, same dequantized rows).  Both always take the
+ * matrix-vector kernels, one launch whatever S and rows are (kvq_plan_set_impl is not consulted), make no other CUDA
+ * call once the plan has been used on the device, and so can be recorded into a CUDA graph after one call of any
+ * compute entry point on this plan and device outside the recording (that first call allocates the plan's tables).
+ */
+kvq_status_t kvq_append_at(kvq_plan_t *plan, const void *x_new /* [S, D] */, kvq_dtype_t dtype, int64_t S,
+                           const float *lambda, int64_t n_lambda, int64_t streams_per_lambda, uint8_t *packed_cache,
+                           void *scales_cache, int64_t T_max, const int64_t *pos_device, void *cuda_stream);
+kvq_status_t kvq_flush_block_at(kvq_plan_t *plan, const void *x_block, kvq_dtype_t dtype, int64_t S, int64_t rows,
+                                const float *lambda, int64_t n_lambda, int64_t streams_per_lambda, uint8_t *packed_cache,
+                                void *scales_cache, void *dq_cache, int64_t T_max, const int64_t *pos0_device,
+                                void *cuda_stream);
 
 /*
  * kvq_calibrate_lambda -- static calibration of the per-channel rescale (Sec. 7.1: lambda_d = 1 / per-channel

@@ -27,6 +27,7 @@ KVQ_ERR_TIMEOUT = 5
 KVQ_ERR_NOMEM = 6
 KVQ_ERR_SCRATCH_LIMIT = 7
 KVQ_ERR_RANGE = 8
+KVQ_DEV_POSITION = 16   # bit of the device status word: kvq_append_at / kvq_flush_block_at met a position outside the cache
 
 KVQ_F16 = 0
 KVQ_BF16 = 1
@@ -39,7 +40,8 @@ KVQ_IMPL_MATVEC = 3
 # every symbol include/kvq.h declares
 EXPORTS = (
     "kvq_plan_create", "kvq_plan_create_ex", "kvq_plan_set_rotation", "kvq_plan_clear_device_status", "kvq_plan_destroy", "kvq_plan_get_signs", "kvq_plan_describe", "kvq_plan_set_impl",
-    "kvq_plan_device_status", "kvq_encode", "kvq_decode", "kvq_append", "kvq_decode_static", "kvq_calibrate_lambda", "kvq_flush_block", "kvq_status_string",
+    "kvq_plan_device_status", "kvq_encode", "kvq_decode", "kvq_append", "kvq_decode_static", "kvq_calibrate_lambda", "kvq_flush_block", "kvq_append_at", "kvq_flush_block_at",
+    "kvq_status_string",
     "kvq_launch_count",
 )
 
@@ -89,6 +91,10 @@ def lib() -> ctypes.CDLL:
         L.kvq_decode_static.argtypes = [vp, vp, vp, i64, vp, i64, i64, vp, i32, vp, vp]
         L.kvq_flush_block.restype = i32
         L.kvq_flush_block.argtypes = [vp, vp, i32, i64, i64, vp, i64, i64, vp, vp, vp, i64, i64, vp]
+        L.kvq_append_at.restype = i32
+        L.kvq_append_at.argtypes = [vp, vp, i32, i64, vp, i64, i64, vp, vp, i64, vp, vp]
+        L.kvq_flush_block_at.restype = i32
+        L.kvq_flush_block_at.argtypes = [vp, vp, i32, i64, i64, vp, i64, i64, vp, vp, vp, i64, vp, vp]
         L.kvq_calibrate_lambda.restype = i32
         L.kvq_calibrate_lambda.argtypes = [vp, vp, i32, i64, vp, vp]
         L.kvq_status_string.restype = ctypes.c_char_p
@@ -221,7 +227,8 @@ def kvq_plan_set_impl(plan: int, encode_impl: int, decode_impl: int) -> None:
 def kvq_plan_device_status(plan: int) -> int:
     w = ctypes.c_uint32()
     st = lib().kvq_plan_device_status(plan, ctypes.byref(w))
-    if st not in (KVQ_OK, KVQ_ERR_TIMEOUT, KVQ_ERR_RANGE):
+    # the codes that describe the word (bit 4, a position outside the cache, reads KVQ_ERR_INVALID_ARG) are not failures of the call
+    if st not in (KVQ_OK, KVQ_ERR_TIMEOUT, KVQ_ERR_RANGE) and not (st == KVQ_ERR_INVALID_ARG and w.value & KVQ_DEV_POSITION):
         raise KvqError(st, "kvq_plan_device_status")
     return int(w.value)
 
@@ -293,6 +300,39 @@ def kvq_flush_block(plan: int, x_block: torch.Tensor, lam: torch.Tensor, packed_
                                      streams_per_lambda, _dev(packed_cache, "packed_cache"), _dev(scales_cache, "scales_cache"),
                                      _dev(dq_cache, "dq_cache"), T_max, pos0, _stream(stream, x_block.device)),
                "kvq_flush_block")
+
+
+def _pos_word(pos_device: torch.Tensor):
+    if pos_device.dtype != torch.int64 or pos_device.numel() != 1:
+        raise TypeError("the position word must be one int64 on the device")
+    return _dev(pos_device, "pos_device")
+
+
+def kvq_append_at(plan: int, x_new: torch.Tensor, lam: torch.Tensor, packed_cache: torch.Tensor, scales_cache: torch.Tensor,
+                  pos_device: torch.Tensor, streams_per_lambda: int = 0, stream=None) -> None:
+    """kvq_append with the row to write read from ``pos_device`` (one int64 on the device) when the kernel runs."""
+    D = x_new.shape[-1]
+    S = x_new.numel() // D
+    T_max = packed_cache.shape[-2]
+    n_lambda = lam.numel() // D
+    with _on_device(x_new.device):
+        _check(lib().kvq_append_at(plan, _dev(x_new, "x_new"), _dtype_code(x_new), S, _dev(lam, "lambda"), n_lambda,
+                                   streams_per_lambda, _dev(packed_cache, "packed_cache"), _dev(scales_cache, "scales_cache"),
+                                   T_max, _pos_word(pos_device), _stream(stream, x_new.device)),
+               "kvq_append_at")
+
+
+def kvq_flush_block_at(plan: int, x_block: torch.Tensor, lam: torch.Tensor, packed_cache: torch.Tensor, scales_cache: torch.Tensor,
+                       dq_cache: torch.Tensor, pos0_device: torch.Tensor, streams_per_lambda: int = 0, stream=None) -> None:
+    """kvq_flush_block with the first row to write read from ``pos0_device`` (one int64 on the device) when the kernel runs."""
+    S, rows, D = x_block.shape
+    T_max = packed_cache.shape[-2]
+    n_lambda = lam.numel() // D
+    with _on_device(x_block.device):
+        _check(lib().kvq_flush_block_at(plan, _dev(x_block, "x_block"), _dtype_code(x_block), S, rows, _dev(lam, "lambda"), n_lambda,
+                                        streams_per_lambda, _dev(packed_cache, "packed_cache"), _dev(scales_cache, "scales_cache"),
+                                        _dev(dq_cache, "dq_cache"), T_max, _pos_word(pos0_device), _stream(stream, x_block.device)),
+               "kvq_flush_block_at")
 
 
 def kvq_calibrate_lambda(plan: int, x: torch.Tensor, lambda_out: torch.Tensor, stream=None) -> None:

@@ -323,6 +323,7 @@ kvq_status_t kvq_plan_device_status(kvq_plan_t *plan, uint32_t *word)
         return KVQ_ERR_CUDA;
     }
     if (*word & 7u) return KVQ_ERR_TIMEOUT;
+    if (*word & 16u) return KVQ_ERR_INVALID_ARG;   // a position read on the device was outside the cache
     return *word ? KVQ_ERR_RANGE : KVQ_OK;
 }
 
@@ -348,7 +349,8 @@ static bool flush_decode_is_matvec(const kvq_plan_t *plan, int64_t N)
 // too, the dequantized rows go to dq (rows out_map(r)) in the same launch and *fused is set.
 static kvq_status_t encode_common(kvq_plan_t *plan, const void *x, kvq_dtype_t dtype, int64_t N, const float *lambda,
                                   int64_t n_lambda, int64_t rows_per_lambda, uint8_t *packed, void *scales,
-                                  const RowMap &out_map, void *cuda_stream, void *dq = nullptr, bool *fused = nullptr)
+                                  const RowMap &out_map, void *cuda_stream, void *dq = nullptr, bool *fused = nullptr,
+                                  const DevicePos *pos = nullptr)
 {
     if (!plan || N < 0) return KVQ_ERR_INVALID_ARG;
     if (dtype != KVQ_F16 && dtype != KVQ_BF16) return KVQ_ERR_INVALID_ARG;
@@ -361,8 +363,10 @@ static kvq_status_t encode_common(kvq_plan_t *plan, const void *x, kvq_dtype_t d
     const bool per_vector = plan->group == plan->D;
     // tensor-map coordinates are 32-bit: the tensor-core kernels take up to 2^31 - 1 rows per call
     const bool gemm_ok = gemm_encode_ok(plan, bf16) && N < ((int64_t)1 << 31);
-    if (plan->enc_impl == KVQ_IMPL_GEMM && !gemm_ok) return KVQ_ERR_UNSUPPORTED_DIM;
-    if (plan->rot && plan->enc_impl == KVQ_IMPL_FFT) return KVQ_ERR_UNSUPPORTED_DIM;   // the rotation lives in the D x D tables
+    if (!pos) {
+        if (plan->enc_impl == KVQ_IMPL_GEMM && !gemm_ok) return KVQ_ERR_UNSUPPORTED_DIM;
+        if (plan->rot && plan->enc_impl == KVQ_IMPL_FFT) return KVQ_ERR_UNSUPPORTED_DIM;   // the rotation lives in the D x D tables
+    }
     if ((st = ensure_device(plan)) != KVQ_OK) return st;
     FftParams prm;
     fill_params(plan, prm, N, lambda, n_lambda, rows_per_lambda);
@@ -373,7 +377,7 @@ static kvq_status_t encode_common(kvq_plan_t *plan, const void *x, kvq_dtype_t d
     // AUTO: the matrix-vector kernel for small calls (latency), beyond that the tensor-core kernel (measured faster than
     // the register FFT at every size above the matrix-vector limit), the register FFT where no tensor-core kernel is
     // built.  A rotated plan has no FFT path: matrix-vector wherever the tensor-core kernel does not apply.
-    kvq_impl_t impl = plan->enc_impl;
+    kvq_impl_t impl = pos ? KVQ_IMPL_MATVEC : plan->enc_impl;   // a position in device memory: the matrix-vector kernels read it
     if (impl == KVQ_IMPL_AUTO) {
         if (N <= matvec_max_rows(plan->D)) impl = KVQ_IMPL_MATVEC;
         else if (gemm_ok) impl = KVQ_IMPL_GEMM;
@@ -382,11 +386,11 @@ static kvq_status_t encode_common(kvq_plan_t *plan, const void *x, kvq_dtype_t d
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     cudaError_t e;
     if (impl == KVQ_IMPL_GEMM) e = umma_encode(plan->D, bf16, per_vector, N, prm, plan->d_e0, stream);
-    else if (impl == KVQ_IMPL_MATVEC && dq && fused && flush_decode_is_matvec(plan, N)) {
+    else if (impl == KVQ_IMPL_MATVEC && dq && fused && (pos || flush_decode_is_matvec(plan, N))) {
         prm.out = dq;
-        e = matvec_flush(plan->D, plan->group, plan->bits, bf16, N, prm, plan->d_b0, plan->d_e0, stream);
+        e = matvec_flush(plan->D, plan->group, plan->bits, bf16, N, prm, plan->d_b0, plan->d_e0, stream, pos);
         *fused = e == cudaSuccess;
-    } else if (impl == KVQ_IMPL_MATVEC) e = matvec_encode(plan->D, plan->group, plan->bits, bf16, N, prm, plan->d_b0, stream);
+    } else if (impl == KVQ_IMPL_MATVEC) e = matvec_encode(plan->D, plan->group, plan->bits, bf16, N, prm, plan->d_b0, stream, pos);
     else e = fft_encode(plan->D, plan->group, plan->bits, bf16, N, prm, stream);
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
@@ -467,26 +471,63 @@ kvq_status_t kvq_decode(kvq_plan_t *plan, const uint8_t *packed, const void *sca
     return KVQ_OK;
 }
 
+kvq_status_t kvq_append_at(kvq_plan_t *plan, const void *x_new, kvq_dtype_t dtype, int64_t S, const float *lambda,
+                           int64_t n_lambda, int64_t streams_per_lambda, uint8_t *packed_cache, void *scales_cache,
+                           int64_t T_max, const int64_t *pos_device, void *cuda_stream)
+{
+    if (T_max < 1) return KVQ_ERR_INVALID_ARG;
+    if (S == 0) return plan ? KVQ_OK : KVQ_ERR_INVALID_ARG;
+    if (!pos_device) return KVQ_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(pos_device) & 7u) return KVQ_ERR_ALIGNMENT;
+    const DevicePos pos{pos_device, T_max - 1};
+    return encode_common(plan, x_new, dtype, S, lambda, n_lambda, streams_per_lambda, packed_cache, scales_cache,
+                         RowMap{1, T_max, 0}, cuda_stream, nullptr, nullptr, &pos);
+}
+
+static kvq_status_t flush_common(kvq_plan_t *plan, const void *x_block, kvq_dtype_t dtype, int64_t S, int64_t rows,
+                                 const float *lambda, int64_t n_lambda, int64_t streams_per_lambda, uint8_t *packed_cache,
+                                 void *scales_cache, void *dq_cache, int64_t T_max, int64_t pos0, const int64_t *pos0_device,
+                                 bool at, void *cuda_stream);
+
 kvq_status_t kvq_flush_block(kvq_plan_t *plan, const void *x_block, kvq_dtype_t dtype, int64_t S, int64_t rows, const float *lambda,
                              int64_t n_lambda, int64_t streams_per_lambda, uint8_t *packed_cache, void *scales_cache, void *dq_cache,
                              int64_t T_max, int64_t pos0, void *cuda_stream)
+{
+    return flush_common(plan, x_block, dtype, S, rows, lambda, n_lambda, streams_per_lambda, packed_cache, scales_cache, dq_cache,
+                        T_max, pos0, nullptr, false, cuda_stream);
+}
+
+kvq_status_t kvq_flush_block_at(kvq_plan_t *plan, const void *x_block, kvq_dtype_t dtype, int64_t S, int64_t rows, const float *lambda,
+                                int64_t n_lambda, int64_t streams_per_lambda, uint8_t *packed_cache, void *scales_cache,
+                                void *dq_cache, int64_t T_max, const int64_t *pos0_device, void *cuda_stream)
+{
+    return flush_common(plan, x_block, dtype, S, rows, lambda, n_lambda, streams_per_lambda, packed_cache, scales_cache, dq_cache,
+                        T_max, 0, pos0_device, true, cuda_stream);
+}
+
+static kvq_status_t flush_common(kvq_plan_t *plan, const void *x_block, kvq_dtype_t dtype, int64_t S, int64_t rows,
+                                 const float *lambda, int64_t n_lambda, int64_t streams_per_lambda, uint8_t *packed_cache,
+                                 void *scales_cache, void *dq_cache, int64_t T_max, int64_t pos0, const int64_t *pos0_device,
+                                 bool at, void *cuda_stream)
 {
     if (!plan || S < 0 || rows < 0) return KVQ_ERR_INVALID_ARG;
     if (T_max < 1 || pos0 < 0 || rows > T_max || pos0 > T_max - rows) return KVQ_ERR_INVALID_ARG;
     if (dtype != KVQ_F16 && dtype != KVQ_BF16) return KVQ_ERR_INVALID_ARG;
     if (S == 0 || rows == 0) return KVQ_OK;
-    if (!dq_cache) return KVQ_ERR_INVALID_ARG;
-    if (misaligned16(dq_cache)) return KVQ_ERR_ALIGNMENT;
+    if (!dq_cache || (at && !pos0_device)) return KVQ_ERR_INVALID_ARG;
+    if (misaligned16(dq_cache) || (reinterpret_cast<uintptr_t>(pos0_device) & 7u)) return KVQ_ERR_ALIGNMENT;
     if (S > INT64_MAX / rows) return KVQ_ERR_INVALID_ARG;
     const int64_t N = S * rows;
     // lambda row of block row r: stream (r / rows) / streams_per_lambda
     const int64_t rpl = (streams_per_lambda < 1 ? 1 : streams_per_lambda) * rows;
     const RowMap map{rows, T_max, pos0};
-    if (plan->rot && plan->dec_impl == KVQ_IMPL_FFT) return KVQ_ERR_UNSUPPORTED_DIM;
+    if (!at && plan->rot && plan->dec_impl == KVQ_IMPL_FFT) return KVQ_ERR_UNSUPPORTED_DIM;
     bool fused = false;
+    const DevicePos pos{pos0_device, T_max - rows};
     kvq_status_t st = encode_common(plan, x_block, dtype, N, lambda, n_lambda, rpl, packed_cache, scales_cache, map, cuda_stream,
-                                    dq_cache, &fused);
+                                    dq_cache, &fused, at ? &pos : nullptr);
     if (st != KVQ_OK || fused) return st;
+    if (at) return KVQ_ERR_CUDA;   // the fused launch is the only form that reads the position on the device
     // the same rows back out of the int4 cache into the dequantized-prefix cache: what a later full-prefix decode would give
     FftParams prm;
     fill_params(plan, prm, N, lambda, n_lambda, rpl);

@@ -71,10 +71,17 @@ bool umma_encode_bits8_supported(int D, bool bf16);
 cudaError_t umma_encode(int D, bool bf16, bool per_vector, int64_t N, const FftParams &prm, const float *e0, cudaStream_t stream);
 
 // fp32 matrix-vector kernels for small calls (kvq_matvec.cu): every layout, dtype and D; b0 / e0 are the plan's tables
-cudaError_t matvec_encode(int D, int group, int bits, bool bf16, int64_t N, const FftParams &prm, const float *b0, cudaStream_t stream);
+// A cache position that lives in device memory (read when the kernel runs): the base row of the output row map; it must
+// lie in [0, limit], else the launch writes nothing and raises KVQ_DEV_POSITION in the plan's status word.
+struct DevicePos {
+    const int64_t *ptr;
+    int64_t limit;
+};
+cudaError_t matvec_encode(int D, int group, int bits, bool bf16, int64_t N, const FftParams &prm, const float *b0, cudaStream_t stream,
+                          const DevicePos *pos = nullptr);
 cudaError_t matvec_decode(int D, int group, int bits, bool bf16, int64_t N, const FftParams &prm, const float *e0, cudaStream_t stream);
 cudaError_t matvec_flush(int D, int group, int bits, bool bf16, int64_t N, const FftParams &prm, const float *b0, const float *e0,
-                         cudaStream_t stream);   // encode + decode of the same rows in one launch
+                         cudaStream_t stream, const DevicePos *pos = nullptr);   // encode + decode of the same rows in one launch
 // group: 32 or D (one scale per vector); bits: 4 or 8
 cudaError_t fft_encode(int D, int group, int bits, bool bf16, int64_t N, const FftParams &prm, cudaStream_t stream);
 cudaError_t fft_decode(int D, int group, int bits, bool bf16, int64_t N, const FftParams &prm, cudaStream_t stream);

@@ -37,7 +37,28 @@ struct MatvecParams {
     int64_t N, n_lambda, rows_per_lambda;
     RowMap out_map, in_map;
     int group, bits;
+    // Position on the device: when pos_dev is set, the base row of out_map is *pos_dev, read when the kernel runs, and must
+    // lie in [0, pos_limit]; otherwise the launch writes nothing and raises KVQ_DEV_POSITION in *status.
+    const int64_t *pos_dev;
+    int64_t pos_limit;
+    uint32_t *status;
 };
+
+// The row map of this launch's output rows: as passed, or based at the position found in device memory.  False (for the
+// whole grid alike) when that position is outside the cache.
+__device__ __forceinline__ bool resolve_out_map(const MatvecParams &prm, RowMap &map)
+{
+    map = prm.out_map;
+    if (prm.pos_dev) {
+        const int64_t p = __ldg(prm.pos_dev);
+        if (p < 0 || p > prm.pos_limit) {
+            if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(prm.status, KVQ_DEV_POSITION);
+            return false;
+        }
+        map.base = p;
+    }
+    return true;
+}
 
 template <int D>
 struct Geo {
@@ -150,6 +171,8 @@ __global__ void __launch_bounds__(kWarps * 32) kvq_encode_matvec_kernel(const __
     // ---- everything that does not depend on the vectors is requested first, so that one round trip covers it all
     float4 t[Gm::CH][P];
     load_rows<D>(prm.table, warp, lane, 0, t);
+    RowMap out_map;
+    if (!resolve_out_map(prm, out_map)) return;   // uniform over the grid: no barrier is left waiting
     float4 lam4[P];
 #pragma unroll
     for (int p = 0; p < P; ++p) {
@@ -175,7 +198,7 @@ __global__ void __launch_bounds__(kWarps * 32) kvq_encode_matvec_kernel(const __
     // ---- warp w finishes vector w
     const bool live = r < prm.N;
     if (!FLUSH && !live) return;
-    const int64_t orow = live ? prm.out_map(r) : 0;
+    const int64_t orow = live ? out_map(r) : 0;
     const bool per_vector = prm.group == D;
     const float Q = prm.bits == 4 ? 7.0f : 127.0f;
     float amax[P];
@@ -361,16 +384,20 @@ MatvecParams from_fft(const FftParams &f, const float *table, int group, int bit
     p.N = f.N, p.n_lambda = f.n_lambda, p.rows_per_lambda = f.rows_per_lambda;
     p.out_map = f.out_map, p.in_map = f.in_map;
     p.group = group, p.bits = bits;
+    p.pos_dev = nullptr, p.pos_limit = 0, p.status = f.status;
     return p;
 }
 
 }  // namespace
 
 // b0: the plan's [n][c] table; e0: its transpose
-cudaError_t matvec_encode(int D, int group, int bits, bool bf16, int64_t N, const FftParams &f, const float *b0, cudaStream_t stream)
+cudaError_t matvec_encode(int D, int group, int bits, bool bf16, int64_t N, const FftParams &f, const float *b0, cudaStream_t stream,
+                          const DevicePos *pos)
 {
     (void)N;
-    return dispatch<1>(D, bf16, from_fft(f, b0, group, bits), stream);
+    MatvecParams p = from_fft(f, b0, group, bits);
+    if (pos) p.pos_dev = pos->ptr, p.pos_limit = pos->limit;
+    return dispatch<1>(D, bf16, p, stream);
 }
 
 cudaError_t matvec_decode(int D, int group, int bits, bool bf16, int64_t N, const FftParams &f, const float *e0, cudaStream_t stream)
@@ -382,10 +409,11 @@ cudaError_t matvec_decode(int D, int group, int bits, bool bf16, int64_t N, cons
 // The window flush in one launch: x rows -> codes and scales at rows out_map(r) of the caches, and the dequantized
 // vectors at the same rows of f.out.
 cudaError_t matvec_flush(int D, int group, int bits, bool bf16, int64_t N, const FftParams &f, const float *b0, const float *e0,
-                         cudaStream_t stream)
+                         cudaStream_t stream, const DevicePos *pos)
 {
     (void)N;
     MatvecParams p = from_fft(f, b0, group, bits);
+    if (pos) p.pos_dev = pos->ptr, p.pos_limit = pos->limit;
     p.table2 = e0;
     return dispatch<2>(D, bf16, p, stream);
 }

@@ -436,6 +436,138 @@ def test_window_flush_in_one_launch_equals_decode_of_what_it_stored(D, dtype, gr
     plan.close()
 
 
+# ---- the cache position in device memory: kvq_append_at / kvq_flush_block_at, eager and replayed from a CUDA graph ----
+
+@pytest.mark.parametrize("D,dtype,group,nbits", [(128, "f16", G, 4), (256, "bf16", G, 4), (96, "f16", G, 4), (160, "bf16", G, 4),
+                                                 (64, "f16", 0, 4), (128, "bf16", G, 8)])
+def test_position_in_device_memory_gives_what_the_host_position_gives(D, dtype, group, nbits):
+    g = group or D
+    tdt = torch.float16 if dtype == "f16" else torch.bfloat16
+    S, T_max, rows, spl = 21, 48, 5, 4
+    plan = kb.Plan(D, g, 91, nbits)
+    lamd = wl.make_lambda((S + spl - 1) // spl, D, 92).cuda()
+    x_new = wl.make_vectors(S * 3, D, dtype, "k_outlier", 93).view(3, S, D).cuda()
+    x_blk = wl.make_vectors(S * rows * 2, D, dtype, "k_outlier", 94).view(2, S, rows, D).cuda()
+
+    def caches():
+        return (torch.full((S, T_max, D * nbits // 8), 0xAB, dtype=torch.uint8, device="cuda"),
+                torch.full((S, T_max, D // g), 1.25, dtype=torch.float16, device="cuda"),
+                torch.full((S, T_max, D), 3.0, dtype=tdt, device="cuda"))
+
+    pa, sa, da = caches()       # positions from the host
+    pb, sb, db = caches()       # the same positions from device memory
+    pos = torch.zeros(1, dtype=torch.int64, device="cuda")
+    steps = [("append", 0, 0), ("append", 1, T_max - 1), ("flush", 0, 7), ("append", 2, 12), ("flush", 1, T_max - rows)]
+    for kind, i, p in steps:
+        pos.fill_(p)
+        if kind == "append":
+            kb.kvq_append(plan.handle, x_new[i], lamd, pa, sa, p, spl)
+            kb.kvq_append_at(plan.handle, x_new[i], lamd, pb, sb, pos, spl)
+        else:
+            kb.kvq_flush_block(plan.handle, x_blk[i], lamd, pa, sa, da, p, spl)
+            kb.kvq_flush_block_at(plan.handle, x_blk[i], lamd, pb, sb, db, pos, spl)
+    torch.cuda.synchronize()
+    assert kb.kvq_plan_device_status(plan.handle) == 0
+    assert torch.equal(pa, pb) and torch.equal(sa, sb) and torch.equal(da.view(torch.int16), db.view(torch.int16))
+    assert not bool((pa[:, 7:7 + rows] == 0xAB).all())      # something was written at all
+
+    # a position outside the cache: nothing is written, the plan's status word says so, and clearing it restores service
+    for bad, call in ((T_max, "append"), (-1, "append"), (T_max - rows + 1, "flush"), (-3, "flush")):
+        pos.fill_(bad)
+        if call == "append":
+            kb.kvq_append_at(plan.handle, x_new[0], lamd, pb, sb, pos, spl)
+        else:
+            kb.kvq_flush_block_at(plan.handle, x_blk[0], lamd, pb, sb, db, pos, spl)
+        assert kb.kvq_plan_device_status(plan.handle) == kb.KVQ_DEV_POSITION
+        assert torch.equal(pa, pb) and torch.equal(sa, sb) and torch.equal(da.view(torch.int16), db.view(torch.int16))
+        kb.kvq_plan_clear_device_status(plan.handle)
+        assert kb.kvq_plan_device_status(plan.handle) == 0
+    plan.close()
+
+
+def test_append_at_beyond_the_small_call_limit_against_the_oracle():
+    """kvq_append_at always takes the matrix-vector kernel: 5120 streams (every layer, head and sequence of a large model in
+    one call) is past the size where kvq_append would change kernels."""
+    D, S, T_max, spl = 128, 5120, 6, 64
+    plan = kb.Plan(D, G, 95)
+    sg = plan.signs()
+    lam = wl.make_lambda(S // spl, D, 96)
+    x = wl.make_vectors(S, D, "f16", "k_outlier", 97)
+    packed = torch.full((S, T_max, D // 2), 0xAB, dtype=torch.uint8, device="cuda")
+    scales = torch.full((S, T_max, D // G), 1.25, dtype=torch.float16, device="cuda")
+    pos = torch.full((1,), 4, dtype=torch.int64, device="cuda")
+    n0 = kb.kvq_launch_count()
+    kb.kvq_append_at(plan.handle, x.cuda(), lam.cuda(), packed, scales, pos, spl)
+    assert kb.kvq_launch_count() - n0 == 1
+    torch.cuda.synchronize()
+    assert kb.kvq_plan_device_status(plan.handle) == 0
+    ora = ko.encode(bits(x), ko.F16, sg, lam.numpy(), G, spl, want_v=True)
+    parity.check_encode(packed[:, 4].contiguous().cpu().numpy(), bits(scales[:, 4].contiguous()), ora, G, "append_at, 5120 streams")
+    keep = [0, 1, 2, 3, 5]
+    assert bool((packed[:, keep] == 0xAB).all()) and bool((scales[:, keep] == 1.25).all())
+    plan.close()
+
+
+def test_decode_loop_replayed_from_a_cuda_graph():
+    """One decode step of the cache side -- advance the position word, append the new token of every stream, and flush the
+    window when it is full -- recorded once and replayed: the caches equal those of the same steps issued call by call."""
+    D, S, T_max, W, spl = 128, 16, 64, 4, 8
+    plan = kb.Plan(D, G, 98)
+    lamd = wl.make_lambda(S // spl, D, 99).cuda()
+    n_steps = 3 * W
+    xs = wl.make_vectors(n_steps * S, D, "f16", "k_outlier", 100).view(n_steps, S, D).cuda()
+
+    def caches():
+        return (torch.zeros(S, T_max, D // 2, dtype=torch.uint8, device="cuda"),
+                torch.zeros(S, T_max, D // G, dtype=torch.float16, device="cuda"),
+                torch.zeros(S, T_max, D, dtype=torch.float16, device="cuda"))
+
+    # reference: call by call with host positions
+    pa, sa, da = caches()
+    for t in range(n_steps):
+        kb.kvq_append(plan.handle, xs[t], lamd, pa, sa, t, spl)
+        if (t + 1) % W == 0:
+            blk = xs[t + 1 - W:t + 1].transpose(0, 1).contiguous()
+            kb.kvq_flush_block(plan.handle, blk, lamd, pa, sa, da, t + 1 - W, spl)
+    torch.cuda.synchronize()
+
+    # graphs: static inputs, the positions in device memory.  Two graphs, as a serving loop would hold: the every-step one
+    # and the one for steps that end a window.
+    pb, sb, db = caches()
+    x_static = torch.zeros(S, D, dtype=torch.float16, device="cuda")
+    blk_static = torch.zeros(S, W, D, dtype=torch.float16, device="cuda")
+    pos = torch.zeros(1, dtype=torch.int64, device="cuda")
+    pos0 = torch.zeros(1, dtype=torch.int64, device="cuda")
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):      # the plan's first use on the device and the kernels' first launches happen here
+        kb.kvq_append_at(plan.handle, x_static, lamd, pb, sb, pos, spl)
+        kb.kvq_flush_block_at(plan.handle, blk_static, lamd, pb, sb, db, pos0, spl)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    pb.zero_(), sb.zero_(), db.zero_()
+    g_step, g_flush = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g_step):
+        kb.kvq_append_at(plan.handle, x_static, lamd, pb, sb, pos, spl)
+        pos.add_(1)
+    with torch.cuda.graph(g_flush):
+        kb.kvq_flush_block_at(plan.handle, blk_static, lamd, pb, sb, db, pos0, spl)
+        pos0.add_(W)
+    pb.zero_(), sb.zero_(), db.zero_(), pos.zero_(), pos0.zero_()
+    for t in range(n_steps):
+        x_static.copy_(xs[t])
+        g_step.replay()
+        if (t + 1) % W == 0:
+            blk_static.copy_(xs[t + 1 - W:t + 1].transpose(0, 1))
+            g_flush.replay()
+    torch.cuda.synchronize()
+    assert kb.kvq_plan_device_status(plan.handle) == 0
+    assert int(pos.item()) == n_steps and int(pos0.item()) == n_steps
+    assert torch.equal(pa, pb) and torch.equal(sa, sb) and torch.equal(da.view(torch.int16), db.view(torch.int16))
+    assert bool((pb[:, :n_steps] != 0).any())
+    plan.close()
+
+
 def test_flush_block_rejects_blocks_outside_the_cache():
     D, S, T = 128, 4, 16
     plan = kb.Plan(D, G, 1)

@@ -130,6 +130,20 @@ def test_bad_arguments_are_rejected_on_the_host():
     assert app(p.handle, A, 0, 4, A, 1, 0, A, A, 16, -1, None) == kb.KVQ_ERR_INVALID_ARG
     assert app(p.handle, A, 0, 4, A, 1, 0, A, A, 0, 0, None) == kb.KVQ_ERR_INVALID_ARG
     assert app(p.handle, A, 0, 0, A, 1, 0, A, A, 16, 3, None) == kb.KVQ_OK
+    # the position-in-device-memory forms: the word itself is checked for presence and alignment, its value on the device
+    app_at = lambda *a: L.kvq_append_at(*a)
+    assert app_at(p.handle, A, 0, 4, A, 1, 0, A, A, 16, None, None) == kb.KVQ_ERR_INVALID_ARG
+    assert app_at(p.handle, A, 0, 4, A, 1, 0, A, A, 16, A + 4, None) == kb.KVQ_ERR_ALIGNMENT
+    assert app_at(p.handle, A, 0, 4, A, 1, 0, A, A, 0, A, None) == kb.KVQ_ERR_INVALID_ARG     # T_max
+    assert app_at(None, A, 0, 4, A, 1, 0, A, A, 16, A, None) == kb.KVQ_ERR_INVALID_ARG
+    assert app_at(p.handle, None, 0, 4, A, 1, 0, A, A, 16, A, None) == kb.KVQ_ERR_INVALID_ARG
+    assert app_at(p.handle, A, 0, 0, A, 1, 0, A, A, 16, A, None) == kb.KVQ_OK
+    fl_at = lambda *a: L.kvq_flush_block_at(*a)
+    assert fl_at(p.handle, A, 0, 4, 8, A, 1, 0, A, A, A, 16, None, None) == kb.KVQ_ERR_INVALID_ARG
+    assert fl_at(p.handle, A, 0, 4, 8, A, 1, 0, A, A, A, 16, A + 4, None) == kb.KVQ_ERR_ALIGNMENT
+    assert fl_at(p.handle, A, 0, 4, 17, A, 1, 0, A, A, A, 16, A, None) == kb.KVQ_ERR_INVALID_ARG  # more rows than the cache has
+    assert fl_at(p.handle, A, 0, 4, 8, A, 1, 0, A, A, None, 16, A, None) == kb.KVQ_ERR_INVALID_ARG
+    assert fl_at(p.handle, A, 0, 4, 0, A, 1, 0, A, A, A, 16, A, None) == kb.KVQ_OK
     assert L.kvq_plan_set_impl(p.handle, 9, 0) == kb.KVQ_ERR_INVALID_ARG
     assert L.kvq_plan_get_signs(p.handle, None) == kb.KVQ_ERR_INVALID_ARG
     assert kb.kvq_plan_device_status(p.handle) == 0
