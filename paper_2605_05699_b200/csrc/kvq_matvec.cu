@@ -67,6 +67,7 @@ struct Geo {
     // table rows a lane holds in flight per pass: the whole slice where registers allow (one L2 round trip per CTA)
     static constexpr int CH = P == 1 ? KW : (D == 160 ? 10 : 16);
     static_assert(D % (4 * kWarps) == 0 && KW % CH == 0, "slices must be whole quads and whole passes");
+    static constexpr bool kLoops = CH == KW;      // the slice stays in registers: a CTA may take several batches of vectors
     static constexpr int kSmemBytes = (kV * D + kWarps * kV * D) * (int)sizeof(float);
 };
 
@@ -157,22 +158,15 @@ __device__ __forceinline__ void matvec(const float *__restrict__ table, float4 (
 // q sigma / max(lambda, 1e-6) -- what kvq_decode would rebuild from the stored bytes -- back into shared memory, and the
 // CTA runs the matrix-vector product once more with the inverse table: rows out_map(r) of prm.out get the dequantized
 // vectors.
+// One batch of kV vectors.  t: the first pass of this warp's table rows, requested by the caller.
 template <int D, bool BF16, bool FLUSH>
-__global__ void __launch_bounds__(kWarps * 32) kvq_encode_matvec_kernel(const __grid_constant__ MatvecParams prm)
+__device__ __forceinline__ void encode_batch(const MatvecParams &prm, const RowMap &out_map, float4 (&t)[Geo<D>::CH][Geo<D>::P], float *xs,
+                                             float *red, int warp, int lane, int64_t batch)
 {
     using Gm = Geo<D>;
     constexpr int P = Gm::P;
-    extern __shared__ __align__(16) float sm[];
-    float *xs = sm, *red = sm + kV * D;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t v0 = (int64_t)blockIdx.x * kV;
+    const int64_t v0 = batch * kV;
     const int64_t r = v0 + warp;   // the vector this warp finishes
-
-    // ---- everything that does not depend on the vectors is requested first, so that one round trip covers it all
-    float4 t[Gm::CH][P];
-    load_rows<D>(prm.table, warp, lane, 0, t);
-    RowMap out_map;
-    if (!resolve_out_map(prm, out_map)) return;   // uniform over the grid: no barrier is left waiting
     float4 lam4[P];
 #pragma unroll
     for (int p = 0; p < P; ++p) {
@@ -197,7 +191,7 @@ __global__ void __launch_bounds__(kWarps * 32) kvq_encode_matvec_kernel(const __
 
     // ---- warp w finishes vector w
     const bool live = r < prm.N;
-    if (!FLUSH && !live) return;
+    if (!FLUSH && !live) return;   // only in a CTA's last batch, and no barrier follows
     const int64_t orow = live ? out_map(r) : 0;
     const bool per_vector = prm.group == D;
     const float Q = prm.bits == 4 ? 7.0f : 127.0f;
@@ -282,20 +276,43 @@ __global__ void __launch_bounds__(kWarps * 32) kvq_encode_matvec_kernel(const __
     }
 }
 
+// Where a warp's whole table slice fits its registers (D <= 128), a CTA takes batches blockIdx.x, blockIdx.x + gridDim.x,
+// ... and the launch is one resident wave: on calls of more batches than the device holds CTAs the table crosses L2 once
+// per CTA, not once per batch.  The barriers inside one batch also order the next batch's writes to xs and red after this
+// batch's reads.  For D > 128 a CTA takes one batch.
+template <int D, bool BF16, bool FLUSH>
+__global__ void __launch_bounds__(kWarps * 32) kvq_encode_matvec_kernel(const __grid_constant__ MatvecParams prm)
+{
+    using Gm = Geo<D>;
+    extern __shared__ __align__(16) float sm[];
+    float *xs = sm, *red = sm + kV * D;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    // ---- everything that does not depend on the vectors is requested first, so that one round trip covers it all
+    float4 t[Gm::CH][Gm::P];
+    load_rows<D>(prm.table, warp, lane, 0, t);
+    RowMap out_map;
+    if (!resolve_out_map(prm, out_map)) return;   // uniform over the grid: no barrier is left waiting
+    if constexpr (Gm::kLoops) {
+        const int64_t n_batches = (prm.N + kV - 1) / kV;
+#pragma unroll 1
+        for (int64_t batch = blockIdx.x; batch < n_batches; batch += gridDim.x)
+            encode_batch<D, BF16, FLUSH>(prm, out_map, t, xs, red, warp, lane, batch);
+    } else {
+        encode_batch<D, BF16, FLUSH>(prm, out_map, t, xs, red, warp, lane, blockIdx.x);
+    }
+}
+
 // ------------------------------------------------------------------------------------------------
 // decode: codes and scales -> x^  (Sec. 3.1 "unpack, irfft, apply s"; 1 / max(lambda, 1e-6) of Sec. 5.1)
 // ------------------------------------------------------------------------------------------------
 template <int D, bool BF16>
-__global__ void __launch_bounds__(kWarps * 32) kvq_decode_matvec_kernel(const __grid_constant__ MatvecParams prm)
+__device__ __forceinline__ void decode_batch(const MatvecParams &prm, float4 (&t)[Geo<D>::CH][Geo<D>::P], float *zs, float *red, int warp,
+                                             int lane, int64_t batch)
 {
     using Gm = Geo<D>;
     constexpr int P = Gm::P;
-    extern __shared__ __align__(16) float sm[];
-    float *zs = sm, *red = sm + kV * D;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t v0 = (int64_t)blockIdx.x * kV;
-    float4 t[Gm::CH][P];
-    load_rows<D>(prm.table, warp, lane, 0, t);   // in flight while the codes are fetched and dequantised
+    const int64_t v0 = batch * kV;
 
     // ---- the CTA's stored vectors, dequantised: q sigma / max(lambda, 1e-6), four coordinates per thread and pass
     const unsigned char *pk = static_cast<const unsigned char *>(prm.packed);
@@ -342,6 +359,24 @@ __global__ void __launch_bounds__(kWarps * 32) kvq_decode_matvec_kernel(const __
     }
 }
 
+template <int D, bool BF16>
+__global__ void __launch_bounds__(kWarps * 32) kvq_decode_matvec_kernel(const __grid_constant__ MatvecParams prm)
+{
+    using Gm = Geo<D>;
+    extern __shared__ __align__(16) float sm[];
+    float *zs = sm, *red = sm + kV * D;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    float4 t[Gm::CH][Gm::P];
+    load_rows<D>(prm.table, warp, lane, 0, t);   // in flight while the codes are fetched and dequantised
+    if constexpr (Gm::kLoops) {   // as in the encode kernel
+        const int64_t n_batches = (prm.N + kV - 1) / kV;
+#pragma unroll 1
+        for (int64_t batch = blockIdx.x; batch < n_batches; batch += gridDim.x) decode_batch<D, BF16>(prm, t, zs, red, warp, lane, batch);
+    } else {
+        decode_batch<D, BF16>(prm, t, zs, red, warp, lane, blockIdx.x);
+    }
+}
+
 // MODE: 0 decode, 1 encode, 2 encode + decode of the same rows (window flush)
 template <int D, bool BF16, int MODE>
 cudaError_t launch(const MatvecParams &prm, cudaStream_t stream)
@@ -351,13 +386,18 @@ cudaError_t launch(const MatvecParams &prm, cudaStream_t stream)
     cudaError_t e = current_device_slot(&dev);
     if (e != cudaSuccess) return e;
     auto kern = MODE == 0 ? kvq_decode_matvec_kernel<D, BF16> : MODE == 1 ? kvq_encode_matvec_kernel<D, BF16, false> : kvq_encode_matvec_kernel<D, BF16, true>;
-    if (slots.sms[dev] == 0) {
+    if (slots.sms[dev] == 0) {   // slots.sms: the CTAs of this kernel that the device holds at once
+        int sms = 0, per_sm = 0;
         if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<D>::kSmemBytes)) != cudaSuccess) return e;
-        slots.sms[dev] = 1;
+        if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+        if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kWarps * 32, Geo<D>::kSmemBytes)) != cudaSuccess) return e;
+        slots.sms[dev] = sms * (per_sm > 0 ? per_sm : 1);
     }
-    const int64_t ctas = (prm.N + kV - 1) / kV;
-    if (ctas > 0x7FFFFFFF) return cudaErrorInvalidValue;
-    kern<<<(int)ctas, kWarps * 32, Geo<D>::kSmemBytes, stream>>>(prm);
+    const int64_t batches = (prm.N + kV - 1) / kV;
+    if (batches > 0x7FFFFFFF) return cudaErrorInvalidValue;
+    // one resident wave of CTAs that loop over batches where the kernel does; else a CTA per batch
+    const int ctas = (int)(Geo<D>::kLoops && batches > slots.sms[dev] ? slots.sms[dev] : batches);
+    kern<<<ctas, kWarps * 32, Geo<D>::kSmemBytes, stream>>>(prm);
     count_launch();
     return cudaGetLastError();
 }
