@@ -508,6 +508,40 @@ def test_append_at_beyond_the_small_call_limit_against_the_oracle():
     plan.close()
 
 
+@pytest.mark.parametrize("D,dtype", [(64, "bf16"), (96, "f16"), (128, "f16"), (128, "bf16")])
+def test_matvec_kernels_past_one_resident_wave(D, dtype):
+    """More batches of 8 vectors than the device holds CTAs: a CTA of the D <= 128 kernels then takes several batches with its
+    table slice kept in registers.  Encode and decode against the oracle; the fused flush against the two-launch flush."""
+    run_case(D, dtype, 6007, "k_outlier", 7300 + D, n_lambda=3, rows_per_lambda=2100, enc_impl="matvec", dec_impl="matvec")
+    tdt = torch.float16 if dtype == "f16" else torch.bfloat16
+    S, T_max, rows, spl = 150, 40, 33, 50          # 4950 vectors: 619 batches
+    plan = kb.Plan(D, G, 7400 + D)
+    lamd = wl.make_lambda(S // spl, D, 7401).cuda()
+    x = wl.make_vectors(S * rows, D, dtype, "k_outlier", 7402).view(S, rows, D).cuda()
+    pos0 = torch.full((1,), 5, dtype=torch.int64, device="cuda")
+    pa = torch.zeros(S, T_max, D // 2, dtype=torch.uint8, device="cuda")
+    sa = torch.zeros(S, T_max, D // G, dtype=torch.float16, device="cuda")
+    da = torch.zeros(S, T_max, D, dtype=tdt, device="cuda")
+    pb, sb, db = torch.zeros_like(pa), torch.zeros_like(sa), torch.zeros_like(da)
+    n0 = kb.kvq_launch_count()
+    kb.kvq_flush_block_at(plan.handle, x, lamd, pa, sa, da, pos0, spl)              # one fused launch, looping CTAs
+    assert kb.kvq_launch_count() - n0 == 1
+    kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_MATVEC, kb.KVQ_IMPL_MATVEC)
+    kb.kvq_append(plan.handle, x[:, 0].contiguous(), lamd, pb, sb, 5, spl)           # the same rows by the unfused calls
+    for i in range(1, rows):
+        kb.kvq_append(plan.handle, x[:, i].contiguous(), lamd, pb, sb, 5 + i, spl)
+    blk_p = pb[:, 5:5 + rows].reshape(S * rows, -1).contiguous()
+    blk_s = sb[:, 5:5 + rows].reshape(S * rows, -1).contiguous()
+    out = torch.empty(S * rows, D, dtype=tdt, device="cuda")
+    kb.kvq_decode(plan.handle, blk_p, blk_s, lamd, out, spl * rows)
+    torch.cuda.synchronize()
+    assert kb.kvq_plan_device_status(plan.handle) == 0
+    assert torch.equal(pa, pb) and torch.equal(sa, sb)
+    assert torch.equal(da[:, 5:5 + rows].reshape(S * rows, D).view(torch.int16), out.view(torch.int16))
+    assert bool((da[:, :5] == 0).all()) and bool((da[:, 5 + rows:] == 0).all())
+    plan.close()
+
+
 def test_decode_loop_replayed_from_a_cuda_graph():
     """One decode step of the cache side -- advance the position word, append the new token of every stream, and flush the
     window when it is full -- recorded once and replayed: the caches equal those of the same steps issued call by call."""
