@@ -59,9 +59,9 @@ typedef enum { KVQ_F16 = 0, KVQ_BF16 = 1 } kvq_dtype_t;
 typedef enum {
     KVQ_IMPL_AUTO = 0,
     KVQ_IMPL_FFT = 1,   /* fp32 register FFT, one thread per vector: every D, dtype and layout; no rotation */
-    KVQ_IMPL_GEMM = 2,  /* tcgen05 DFT-as-GEMM.  bits = 4: encode / append: fp16 for D = 64, 96, 128, 160, 256, bf16 for
-                           D = 64, 96, 128, 256; decode: the same (D, dtype) pairs; either group size.  bits = 8:
-                           D <= 160 only, the same (D, dtype) pairs.  At most 2^31 - 1 rows per call (AUTO falls back
+    KVQ_IMPL_GEMM = 2,  /* tcgen05 DFT-as-GEMM.  bits = 4: encode / append: D = 64, 96, 128, 160, 256 in fp16 and bf16;
+                           decode: fp16 for the same D, bf16 for D = 64, 96, 128, 256; either group size.  bits = 8:
+                           D <= 160 in fp16, D <= 128 in bf16.  At most 2^31 - 1 rows per call (AUTO falls back
                            to the register FFT beyond).
                            Elsewhere the compute calls return KVQ_ERR_UNSUPPORTED_DIM. */
     KVQ_IMPL_MATVEC = 3 /* fp32 matrix-vector product with the plan's D x D table, a CTA per 8 vectors: every D, dtype

@@ -563,7 +563,7 @@ kvq_status_t kvq_calibrate_lambda(kvq_plan_t *plan, const void *x, kvq_dtype_t d
     if (dtype != KVQ_F16 && dtype != KVQ_BF16) return KVQ_ERR_INVALID_ARG;
     if (N > 0 && !x) return KVQ_ERR_INVALID_ARG;
     if (misaligned16(x) || misaligned16(lambda_out)) return KVQ_ERR_ALIGNMENT;
-    if (!umma_encode_supported(plan->D, dtype == KVQ_BF16)) return KVQ_ERR_UNSUPPORTED_DIM;
+    if (!umma_calibrate_supported(plan->D, dtype == KVQ_BF16)) return KVQ_ERR_UNSUPPORTED_DIM;
     kvq_status_t st = ensure_device(plan);
     if (st != KVQ_OK) return st;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);

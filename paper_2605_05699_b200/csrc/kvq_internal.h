@@ -58,6 +58,7 @@ struct GemmParams {
 // fp32, e0[c][n] = M[c][n] s_n; decode takes the table b0 = e0 transposed through GemmParams.
 bool umma_decode_supported(int D, bool bf16);
 bool umma_encode_supported(int D, bool bf16);
+bool umma_calibrate_supported(int D, bool bf16);
 bool umma_decode_bits8_supported(int D, bool bf16);
 cudaError_t umma_decode(int D, bool bf16, int bits, int64_t N, const GemmParams &prm, const uint32_t *sign_xor /* host, 128 words */,
                         cudaStream_t stream);

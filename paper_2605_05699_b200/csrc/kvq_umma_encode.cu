@@ -1,5 +1,5 @@
-// Warp-specialised tcgen05 DFT-as-GEMM encode kernel of libkvq (sm_100a): D = 64, 96, 128, 160; fp16 input for
-// all of them, bf16 input up to D = 128.
+// Warp-specialised tcgen05 DFT-as-GEMM encode kernel of libkvq (sm_100a): D = 64, 96, 128, 160; fp16 and bf16 input
+// (D = 160 with bf16: two x tiles in flight instead of four, and no three-term forms).
 //
 // The forward path v = lambda (.) M (s (.) x) (Sec. 3.1 Eq. 1-2, Sec. 5.1 item 1) is a dense D x D
 // contraction per vector, for any even D: v_c = sum_n W[c, n] x_n with W[c, n] = lambda_c M[c, n] s_n.  The
@@ -573,14 +573,21 @@ cudaError_t launch(int64_t N, const FftParams &f, const float *e0, cudaStream_t 
 
 }  // namespace
 
-bool umma_encode_supported(int D, bool bf16) { return D == 64 || D == 96 || D == 128 || D == 256 || (D == 160 && !bf16); }
+// D = 160 with bf16 input: two bf16 terms of W (120 KB) leave room for two x tiles in flight; the three-term forms
+// (calibration, byte codes) do not fit.
+bool umma_encode_supported(int D, bool bf16)
+{
+    (void)bf16;
+    return D == 64 || D == 96 || D == 128 || D == 160 || D == 256;
+}
+bool umma_calibrate_supported(int D, bool bf16) { return umma_encode_supported(D, bf16) && !(D == 160 && bf16); }
 
 // one scale per vector: the row maximum is traded inside a CTA, or across the cluster pair of the D = 256 kernel
 bool umma_encode_per_vector_supported(int D, bool bf16) { return umma_encode_supported(D, bf16); }
 
 // byte codes: the D <= 160 kernel (the code step is 18 times finer than with 4 bits: two bf16 terms of W would leave 2e-4
 // of the codes on the wrong side of a rounding, so bf16 input takes the three-term instantiation)
-bool umma_encode_bits8_supported(int D, bool bf16) { return D != 256 && umma_encode_supported(D, bf16); }
+bool umma_encode_bits8_supported(int D, bool bf16) { return D != 256 && !(D == 160 && bf16) && umma_encode_supported(D, bf16); }
 
 cudaError_t umma_encode(int D, bool bf16, bool per_vector, int64_t N, const FftParams &f, const float *e0, cudaStream_t stream)
 {
@@ -599,7 +606,7 @@ cudaError_t umma_encode(int D, bool bf16, bool per_vector, int64_t N, const FftP
             case 64: return bf16 ? launch<64, true, false, true>(N, f, e0, stream) : launch<64, false, false, true>(N, f, e0, stream);
             case 96: return bf16 ? launch<96, true, false, true>(N, f, e0, stream) : launch<96, false, false, true>(N, f, e0, stream);
             case 128: return bf16 ? launch<128, true, false, true>(N, f, e0, stream) : launch<128, false, false, true>(N, f, e0, stream);
-            case 160: return bf16 ? cudaErrorInvalidValue : launch<160, false, false, true>(N, f, e0, stream);
+            case 160: return bf16 ? launch<160, true, false, true>(N, f, e0, stream) : launch<160, false, false, true>(N, f, e0, stream);
         }
         return cudaErrorInvalidValue;
     }
@@ -607,7 +614,7 @@ cudaError_t umma_encode(int D, bool bf16, bool per_vector, int64_t N, const FftP
         case 64: return bf16 ? launch<64, true>(N, f, e0, stream) : launch<64, false>(N, f, e0, stream);
         case 96: return bf16 ? launch<96, true>(N, f, e0, stream) : launch<96, false>(N, f, e0, stream);
         case 128: return bf16 ? launch<128, true>(N, f, e0, stream) : launch<128, false>(N, f, e0, stream);
-        case 160: return bf16 ? cudaErrorInvalidValue : launch<160, false>(N, f, e0, stream);
+        case 160: return bf16 ? launch<160, true>(N, f, e0, stream) : launch<160, false>(N, f, e0, stream);
     }
     return cudaErrorInvalidValue;
 }

@@ -166,8 +166,8 @@ def test_gemm_kernels_are_refused_where_they_are_not_built():
             kb.kvq_decode(plan.handle, pk, sc, torch.ones(D, device="cuda"), out)
         assert e.value.status == kb.KVQ_ERR_UNSUPPORTED_DIM
         plan.close()
-    for D, dtype in [(160, torch.bfloat16)]:
-        plan = kb.Plan(D, G, 1)
+    for D, dtype, nbits in [(160, torch.bfloat16, 8), (256, torch.float16, 8)]:     # byte codes: three-term B does not fit
+        plan = kb.Plan(D, G, 1, nbits)
         kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_GEMM, kb.KVQ_IMPL_AUTO)
         x = torch.zeros(8, D, dtype=dtype, device="cuda")
         with pytest.raises(kb.KvqError) as e:
@@ -259,13 +259,13 @@ def test_all_dims_ragged_with_straddling_lambda_rows(D, dtype):
     run_case(D, dtype, 1000, "k_outlier", 2000 + D, n_lambda=4, rows_per_lambda=333, enc_impl="fft", dec_impl="fft")
 
 
-# the tensor-core kernels, wherever they are built: fp16 D <= 160 and bf16 D <= 128, both directions
+# the tensor-core kernels, wherever they are built: D <= 160 in both dtypes for the encode, fp16 D <= 160 and bf16 D <= 128 for the decode
 @pytest.mark.parametrize("dtype", ["f16", "bf16"])
 @pytest.mark.parametrize("D", [64, 96, 128, 160])
 @pytest.mark.parametrize("N,n_lambda,rpl", [(1000, 4, 333), (20000, 1, 0), (129, 1, 0)])
 def test_gemm_kernels_all_dims(D, dtype, N, n_lambda, rpl):
-    enc_impl = dec_impl = "fft" if (D == 160 and dtype == "bf16") else "gemm"
-    run_case(D, dtype, N, "k_outlier", 2100 + D + N, n_lambda=n_lambda, rows_per_lambda=rpl, enc_impl=enc_impl, dec_impl=dec_impl)
+    dec_impl = "fft" if (D == 160 and dtype == "bf16") else "gemm"
+    run_case(D, dtype, N, "k_outlier", 2100 + D + N, n_lambda=n_lambda, rows_per_lambda=rpl, enc_impl="gemm", dec_impl=dec_impl)
 
 
 @pytest.mark.parametrize("N", [1, 31, 32, 33, 4100])
@@ -689,14 +689,14 @@ def test_base_variants_per_vector_scale_and_byte_codes(D, dtype, per_vector, nbi
 @pytest.mark.parametrize("D,dtype,N,n_lambda,rpl", [
     (128, "f16", 20000, 1, 0), (128, "f16", 40000, 200, 200), (128, "bf16", 20000, 3, 7000), (64, "f16", 9000, 1, 0),
     (64, "bf16", 9000, 2, 4500), (96, "f16", 9000, 1, 0), (96, "bf16", 5000, 1, 0), (160, "f16", 9000, 4, 2300),
-    (256, "f16", 9000, 1, 0), (256, "bf16", 9000, 3, 3100), (256, "bf16", 60000, 300, 200), (256, "f16", 129, 1, 0),
+    (160, "bf16", 9000, 2, 4600), (256, "f16", 9000, 1, 0), (256, "bf16", 9000, 3, 3100), (256, "bf16", 60000, 300, 200), (256, "f16", 129, 1, 0),
 ])
 def test_one_scale_per_vector_on_the_tensor_cores(D, dtype, N, n_lambda, rpl):
     # group = D, 4-bit codes: the tensor-core encode trades the row maximum between its two half-row threads (D <= 160)
     # or between the four of a cluster pair (D = 256), the tensor-core decode reads one scale per row
     odt = ko.F16 if dtype == "f16" else ko.BF16
     plan = kb.Plan(D, D, 60 + D)
-    kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_GEMM, kb.KVQ_IMPL_GEMM)
+    kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_GEMM, kb.KVQ_IMPL_FFT if (D == 160 and dtype == "bf16") else kb.KVQ_IMPL_GEMM)
     sg = plan.signs()
     lam = wl.make_lambda(n_lambda, D, 61)
     x = wl.make_vectors(N, D, dtype, "k_outlier", 62 + N)
