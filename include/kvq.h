@@ -59,8 +59,8 @@ typedef enum { KVQ_F16 = 0, KVQ_BF16 = 1 } kvq_dtype_t;
 typedef enum {
     KVQ_IMPL_AUTO = 0,
     KVQ_IMPL_FFT = 1,   /* fp32 register FFT, one thread per vector: every D, dtype and layout; no rotation */
-    KVQ_IMPL_GEMM = 2,  /* tcgen05 DFT-as-GEMM.  bits = 4: encode / append: D = 64, 96, 128, 160, 256 in fp16 and bf16;
-                           decode: fp16 for the same D, bf16 for D = 64, 96, 128, 256; either group size.  bits = 8:
+    KVQ_IMPL_GEMM = 2,  /* tcgen05 DFT-as-GEMM.  bits = 4: encode / append and decode: D = 64, 96, 128, 160, 256 in fp16
+                           and bf16; either group size.  bits = 8:
                            D <= 160 in fp16, D <= 128 in bf16.  At most 2^31 - 1 rows per call (AUTO falls back
                            to the register FFT beyond).
                            Elsewhere the compute calls return KVQ_ERR_UNSUPPORTED_DIM. */

@@ -1,4 +1,4 @@
-// Warp-specialised tcgen05 DFT-as-GEMM decode kernel of libkvq (sm_100a): D = 64, 96, 128, 160, fp16 output.
+// Warp-specialised tcgen05 DFT-as-GEMM decode kernel of libkvq (sm_100a): D = 64, 96, 128, 160, fp16 or bf16 output.
 //
 // The inverse path x^ = diag(s) M^T diag(1 / max(lambda, 1e-6)) (q (.) sigma) (Sec. 3.1 "unpack, irfft,
 // apply s"; Sec. 5.1 item 1) is a dense D x D contraction per vector, for any even D (the mixed-radix
@@ -61,7 +61,7 @@ constexpr uint32_t kTmemCols = 512;
 template <int D, bool BF16OUT, int BITS = 4>
 struct Cfg {
     static_assert(D % 32 == 0 && D >= 64 && D <= 160, "head dim not built");
-    static_assert(!BF16OUT || D <= 128, "two-term operands: tensor memory holds them for D <= 128 only");
+    static_assert(!BF16OUT || BITS == 4 || D <= 128, "two-term operands with byte codes: shared memory holds them for D <= 128 only");
     static_assert(BITS == 4 || BITS == 8, "code width not built");
     static constexpr int kTerms = BF16OUT ? 2 : 1;         // W_hi (, W_lo); a_hi (, a_lo)
     static constexpr int G = D / 32;                       // groups = 16-byte chunks of a packed row = 32-column accumulator chunks
@@ -81,13 +81,18 @@ struct Cfg {
     static constexpr int kOutBytes = 8 * kOutWarpBytes;
     static constexpr int kRoom = (232448 - 1024 - kCtrlBytes - kBBytes - kOutBytes) / kInPitch;
     static constexpr int kInStages = kRoom < kMaxInStages ? kRoom : kMaxInStages;
-    static_assert(kInStages >= 3, "too few packed tiles in flight");
+    static_assert(kInStages >= (D == 160 && BF16OUT ? 2 : 3), "too few packed tiles in flight");
     static constexpr int kSmemBytes = kBBytes + kInStages * kInPitch + kOutBytes + kCtrlBytes + 1024;
-    // tensor memory: two accumulators of D columns, then the A stages of D / 2 columns per term (a_lo 64 columns
-    // behind a_hi)
+    // tensor memory, D <= 128: two accumulators of D columns, then the A stages of D / 2 columns per term (a_lo 64 columns
+    // behind a_hi).  D = 160: an accumulator and an A term of 80 columns in each half of the 512 columns; with two-term
+    // operands the two halves hold a_hi and a_lo of ONE stage (the tile is tensor-bound: 3 x 10 K-steps per tile).
     static constexpr uint32_t kAccStride = D <= 128 ? 128 : 256;
-    static constexpr int kAStages = BF16OUT ? 2 : D <= 128 ? 4 : 2;
-    static constexpr uint32_t kALo = 64;
+    static constexpr int kAStages = BF16OUT ? (D <= 128 ? 2 : 1) : D <= 128 ? 4 : 2;
+    // The "A full" / "A free" barriers form a ring of at least two, indexed by tile: the two dequant groups take alternate
+    // tiles, and a parity wait only tells a phase from its neighbours, so a barrier must not be shared by both groups.
+    // Tile j writes A stage j % kAStages once the MMAs of tile j - kAStages have completed (barrier (j - kAStages) % kABars).
+    static constexpr int kABars = kAStages < 2 ? 2 : kAStages;
+    static constexpr uint32_t kALo = D <= 128 ? 64 : 256;
     __host__ __device__ static constexpr uint32_t acc_col(int s) { return (uint32_t)s * kAccStride; }
     __host__ __device__ static constexpr uint32_t a_col(int s)
     {
@@ -273,7 +278,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             mbar_init(smem_u32(&ctrl->in_full[s]), 1);
             mbar_init(smem_u32(&ctrl->in_empty[s]), 4);
         }
-        for (int s = 0; s < C::kAStages; ++s) {
+        for (int s = 0; s < C::kABars; ++s) {
             mbar_init(smem_u32(&ctrl->a_full[s]), 4);
             mbar_init(smem_u32(&ctrl->a_empty[s]), 1);
         }
@@ -356,8 +361,8 @@ __global__ void __launch_bounds__(kThreads, 1)
             int n_mma = n_my;
             if (n_my > 0 && !wait_or_abort(smem_u32(&ctrl->b_first), 0u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT)) n_mma = 0;
             for (int j = 0; j < n_mma; ++j) {
-                const int sa = j % C::kAStages, sc = j % kAccStages;
-                if (!wait_or_abort(smem_u32(&ctrl->a_full[sa]), (uint32_t)(j / C::kAStages) & 1u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT)) break;
+                const int sa = j % C::kAStages, sb = j % C::kABars, sc = j % kAccStages;
+                if (!wait_or_abort(smem_u32(&ctrl->a_full[sb]), (uint32_t)(j / C::kABars) & 1u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT)) break;
                 if (!wait_or_abort(smem_u32(&ctrl->acc_empty[sc]), ((uint32_t)(j / kAccStages) & 1u) ^ 1u, abort_flag, status,
                                    KVQ_DEV_SLOT_TIMEOUT))
                     break;
@@ -378,7 +383,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                     }
                 }
                 umma_commit(smem_u32(&ctrl->acc_full[sc]));
-                umma_commit(smem_u32(&ctrl->a_empty[sa]));
+                umma_commit(smem_u32(&ctrl->a_empty[sb]));
             }
         }
     } else if (warp < 10) {
@@ -432,10 +437,10 @@ __global__ void __launch_bounds__(kThreads, 1)
                     // than one of its tiles, so first wait for this group's own last tile (its barrier is at most one
                     // phase behind, this group waited on it before writing that tile): MMAs complete in order, so after it
                     // the previous tile's barrier is at most one phase behind too.
-                    if (j >= 2 && !wait_or_abort(smem_u32(&ctrl->a_empty[(j - 2) % C::kAStages]), (uint32_t)((j - 2) / C::kAStages) & 1u,
+                    if (j >= 2 && !wait_or_abort(smem_u32(&ctrl->a_empty[(j - 2) % C::kABars]), (uint32_t)((j - 2) / C::kABars) & 1u,
                                                  abort_flag, status, KVQ_DEV_MMA_TIMEOUT))
                         break;
-                    if (!wait_or_abort(smem_u32(&ctrl->a_empty[(j - 1) % C::kAStages]), (uint32_t)((j - 1) / C::kAStages) & 1u, abort_flag,
+                    if (!wait_or_abort(smem_u32(&ctrl->a_empty[(j - 1) % C::kABars]), (uint32_t)((j - 1) / C::kABars) & 1u, abort_flag,
                                        status, KVQ_DEV_MMA_TIMEOUT))
                         break;
                     if (rl.wide && q == 0 && lane == 0) atomicOr(status, KVQ_DEV_RANGE);
@@ -446,7 +451,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             }
 
             // ---- this tile's packed rows have landed; the A stage is free again
-            const int s = j % kInStages, sa = j % C::kAStages;
+            const int s = j % kInStages, sa = j % C::kAStages, sb = j % C::kABars;
             if (!wait_or_abort(smem_u32(&ctrl->in_full[s]), (uint32_t)(j / kInStages) & 1u, abort_flag, status, KVQ_DEV_LOAD_TIMEOUT)) break;
             const unsigned char *row = sIn + s * C::kInPitch + r * C::kInRow;
             uint4 pk[BITS == 4 ? G : 1];
@@ -456,8 +461,12 @@ __global__ void __launch_bounds__(kThreads, 1)
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&ctrl->in_empty[s]));   // the values are in registers
             }
-            if (!wait_or_abort(smem_u32(&ctrl->a_empty[sa]), ((uint32_t)(j / C::kAStages) & 1u) ^ 1u, abort_flag, status, KVQ_DEV_MMA_TIMEOUT))
-                break;
+            if (j >= C::kAStages) {   // the MMAs that read this A stage last
+                const int jp = j - C::kAStages;
+                if (!wait_or_abort(smem_u32(&ctrl->a_empty[jp % C::kABars]), (uint32_t)(jp / C::kABars) & 1u, abort_flag, status,
+                                   KVQ_DEV_MMA_TIMEOUT))
+                    break;
+            }
             tc_fence_after();
 
             // ---- the A operand q sigma rho is fp16.  A row whose scales would take it out of fp16's normal range (a very
@@ -520,7 +529,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             tc_fence_before();
             __threadfence_block();   // the row scales, for the epilogue that follows this tile's accumulator
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&ctrl->a_full[sa]));
+            if (lane == 0) mbar_arrive(smem_u32(&ctrl->a_full[sb]));
         }
     } else {
         // =========================== epilogue: accumulator -> fp16 -> TMA store ===========================
@@ -659,10 +668,14 @@ cudaError_t launch(int64_t N, const GemmParams &g, cudaStream_t stream)
 
 }  // namespace
 
-bool umma_decode_supported(int D, bool bf16) { return D == 256 || D == 64 || D == 96 || D == 128 || (!bf16 && D == 160); }
+bool umma_decode_supported(int D, bool bf16)
+{
+    (void)bf16;
+    return D == 256 || D == 64 || D == 96 || D == 128 || D == 160;
+}
 
-// byte codes: the D <= 160 kernel only
-bool umma_decode_bits8_supported(int D, bool bf16) { return D != 256 && umma_decode_supported(D, bf16); }
+// byte codes: the D <= 160 kernel only (D <= 128 with bf16 output)
+bool umma_decode_bits8_supported(int D, bool bf16) { return D != 256 && !(D == 160 && bf16) && umma_decode_supported(D, bf16); }
 
 cudaError_t umma_decode(int D, bool bf16, int bits, int64_t N, const GemmParams &g, const uint32_t *sign_xor, cudaStream_t stream)
 {
@@ -680,7 +693,7 @@ cudaError_t umma_decode(int D, bool bf16, int bits, int64_t N, const GemmParams 
         case 64: return bf16 ? launch<64, true>(N, g, stream) : launch<64, false>(N, g, stream);
         case 96: return bf16 ? launch<96, true>(N, g, stream) : launch<96, false>(N, g, stream);
         case 128: return bf16 ? launch<128, true>(N, g, stream) : launch<128, false>(N, g, stream);
-        case 160: return bf16 ? cudaErrorInvalidValue : launch<160, false>(N, g, stream);
+        case 160: return bf16 ? launch<160, true>(N, g, stream) : launch<160, false>(N, g, stream);
     }
     return cudaErrorInvalidValue;
 }

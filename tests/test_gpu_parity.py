@@ -115,9 +115,9 @@ def test_many_lambda_rows_rebuild_the_gemm_operands_in_flight(rpl):
                             enc_impl="gemm", dec_impl="gemm")
 
 
-@pytest.mark.parametrize("D,rpl", [(128, 128), (128, 200), (64, 640), (96, 384)])
+@pytest.mark.parametrize("D,rpl", [(128, 128), (128, 200), (64, 640), (96, 384), (160, 128), (160, 333)])
 def test_bf16_output_on_the_tensor_cores_with_many_lambda_rows(D, rpl):
-    # two-term operands (a_hi + a_lo, W_hi + W_lo), two A stages, B rebuilt every few tiles
+    # two-term operands (a_hi + a_lo, W_hi + W_lo), two A stages (one at D = 160), B rebuilt every few tiles
     N = 40000
     run_case(D, "bf16", N, "k_outlier", 9700 + D + rpl, n_lambda=(N + rpl - 1) // rpl, rows_per_lambda=rpl,
              enc_impl="gemm", dec_impl="gemm")
@@ -157,8 +157,8 @@ def test_gemm_encode_serves_large_appends():
 
 
 def test_gemm_kernels_are_refused_where_they_are_not_built():
-    for D, dtype in [(160, torch.bfloat16)]:
-        plan = kb.Plan(D, G, 1)
+    for D, dtype, nbits in [(160, torch.bfloat16, 8), (256, torch.float16, 8)]:
+        plan = kb.Plan(D, G, 1, nbits)
         kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_AUTO, kb.KVQ_IMPL_GEMM)
         pk, sc = plan.empty_packed(8), plan.empty_scales(8)
         out = torch.empty(8, D, dtype=dtype, device="cuda")
@@ -259,13 +259,12 @@ def test_all_dims_ragged_with_straddling_lambda_rows(D, dtype):
     run_case(D, dtype, 1000, "k_outlier", 2000 + D, n_lambda=4, rows_per_lambda=333, enc_impl="fft", dec_impl="fft")
 
 
-# the tensor-core kernels, wherever they are built: D <= 160 in both dtypes for the encode, fp16 D <= 160 and bf16 D <= 128 for the decode
+# the tensor-core kernels of D <= 160, both dtypes, both directions
 @pytest.mark.parametrize("dtype", ["f16", "bf16"])
 @pytest.mark.parametrize("D", [64, 96, 128, 160])
 @pytest.mark.parametrize("N,n_lambda,rpl", [(1000, 4, 333), (20000, 1, 0), (129, 1, 0)])
 def test_gemm_kernels_all_dims(D, dtype, N, n_lambda, rpl):
-    dec_impl = "fft" if (D == 160 and dtype == "bf16") else "gemm"
-    run_case(D, dtype, N, "k_outlier", 2100 + D + N, n_lambda=n_lambda, rows_per_lambda=rpl, enc_impl="gemm", dec_impl=dec_impl)
+    run_case(D, dtype, N, "k_outlier", 2100 + D + N, n_lambda=n_lambda, rows_per_lambda=rpl, enc_impl="gemm", dec_impl="gemm")
 
 
 @pytest.mark.parametrize("N", [1, 31, 32, 33, 4100])
@@ -696,7 +695,7 @@ def test_one_scale_per_vector_on_the_tensor_cores(D, dtype, N, n_lambda, rpl):
     # or between the four of a cluster pair (D = 256), the tensor-core decode reads one scale per row
     odt = ko.F16 if dtype == "f16" else ko.BF16
     plan = kb.Plan(D, D, 60 + D)
-    kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_GEMM, kb.KVQ_IMPL_FFT if (D == 160 and dtype == "bf16") else kb.KVQ_IMPL_GEMM)
+    kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_GEMM, kb.KVQ_IMPL_GEMM)
     sg = plan.signs()
     lam = wl.make_lambda(n_lambda, D, 61)
     x = wl.make_vectors(N, D, dtype, "k_outlier", 62 + N)
@@ -865,7 +864,7 @@ def _degenerate_rows(D, dtype):
 
 
 @pytest.mark.parametrize("impl", ["fft", "gemm", "matvec"])
-@pytest.mark.parametrize("D,dtype", [(128, "f16"), (128, "bf16"), (64, "f16"), (256, "bf16")])
+@pytest.mark.parametrize("D,dtype", [(128, "f16"), (128, "bf16"), (64, "f16"), (256, "bf16"), (160, "bf16")])
 def test_degenerate_inputs(D, dtype, impl):
     odt = ko.F16 if dtype == "f16" else ko.BF16
     x = _degenerate_rows(D, dtype)
