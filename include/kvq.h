@@ -218,9 +218,10 @@ kvq_status_t kvq_flush_block(kvq_plan_t *plan, const void *x_block, kvq_dtype_t 
  *                 the caller updates that word on the same stream.  A value outside [0, T_max - 1] (append) or
  *                 [0, T_max - rows] (flush) writes nothing and raises bit 4 of the plan's device status word.
  * Everything else as in kvq_append / kvq_flush_block (same stored bytes, same dequantized rows).  Both always take the
- * matrix-vector kernels, one launch whatever S and rows are (kvq_plan_set_impl is not consulted), make no other CUDA
- * call once the plan has been used on the device, and so can be recorded into a CUDA graph after one call of any
- * compute entry point on this plan and device outside the recording (that first call allocates the plan's tables).
+ * matrix-vector kernels, one launch whatever S and rows are (kvq_plan_set_impl is not consulted).  The first call of an
+ * entry point for a given plan layout and dtype on a device allocates the plan's tables and sets the kernel's launch
+ * attributes; every later one makes no CUDA call but the launch, and so can be recorded into a CUDA graph: make one call
+ * of the same entry point with the same dtype outside the recording first.
  */
 kvq_status_t kvq_append_at(kvq_plan_t *plan, const void *x_new /* [S, D] */, kvq_dtype_t dtype, int64_t S,
                            const float *lambda, int64_t n_lambda, int64_t streams_per_lambda, uint8_t *packed_cache,
