@@ -450,7 +450,7 @@ kvq_status_t kvq_decode(kvq_plan_t *plan, const uint8_t *packed, const void *sca
         g.status = plan->d_status;
         // D = 256: the radix-2 kernel needs the transform's even / odd structure, which a rotation destroys
         const cudaError_t e = plan->rot && plan->D == 256 ? umma_decode_d256_dense(bf16, N, g, stream)
-                                                          : umma_decode(plan->D, bf16, plan->bits, N, g, plan->sign_xor, stream);
+                                                          : umma_decode(plan->D, bf16, plan->bits, N, g, plan->sign_xor, stream, !plan->rot);
         if (e != cudaSuccess) {
             (void)cudaGetLastError();
             return KVQ_ERR_CUDA;

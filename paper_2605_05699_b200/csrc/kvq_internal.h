@@ -61,7 +61,7 @@ bool umma_encode_supported(int D, bool bf16);
 bool umma_calibrate_supported(int D, bool bf16);
 bool umma_decode_bits8_supported(int D, bool bf16);
 cudaError_t umma_decode(int D, bool bf16, int bits, int64_t N, const GemmParams &prm, const uint32_t *sign_xor /* host, 128 words */,
-                        cudaStream_t stream);
+                        cudaStream_t stream, bool radix2 = false /* the plan has no rotation: the D = 128 fp16 kernel may split by parity */);
 cudaError_t umma_calibrate(int D, bool bf16, int64_t N, const FftParams &prm, const float *e0, uint32_t *amax_bits, cudaStream_t stream);
 cudaError_t umma_calibrate_d256(bool bf16, int64_t N, const FftParams &prm, const float *e0, uint32_t *amax_bits, cudaStream_t stream);
 cudaError_t umma_encode_d256(bool bf16, bool per_vector, int64_t N, const FftParams &prm, const float *e0, cudaStream_t stream);   // kvq_umma_encode256.cu

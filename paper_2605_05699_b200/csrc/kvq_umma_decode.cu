@@ -58,9 +58,18 @@ constexpr uint32_t kTmemCols = 512;
 // W' = W_hi + W_lo, and x^ = a_hi W_hi + a_lo W_hi + a_hi W_lo accumulates in fp32 (a_lo W_lo is below 1e-7).
 // BITS: 4 (nibble pairs) or 8 (one two's-complement byte per code; scale = absmax / 127).  The byte path dequantises
 // pairs of neighbouring codes, so its K order is the natural one and the B operand is built to match.
-template <int D, bool BF16OUT, int BITS = 4>
+// R2: one radix-2 step of the transform is taken out of the GEMM (plans without a rotation; D = 128, fp16 output, 4-bit
+// codes).  Rows of M are cos / sin(2 pi k n / D), so n -> n + D / 2 multiplies a row by (-1)^k, and in the packing of Eq. 2
+// the parity of k is the parity of the channel c.  With E_n / O_n the sums over the even / odd channels (n < D / 2),
+//     x^_n = s_n (E_n + O_n),        x^_{n + D/2} = s_{n + D/2} (E_n - O_n):
+// two 128 x 64 x 64 GEMMs per tile instead of one 128 x 128 x 128, half the tensor work, and an add, a subtract and half a
+// sign flip per output in the epilogue.  The kernel runs at the board's power limit, where tensor flops are what is left to
+// save: 148 -> 137 us per 2M-vector launch back to back.  The half2 nibble trick yields pairs (c, c + 4) of equal parity, so
+// routing codes to the two A operands is free.
+template <int D, bool BF16OUT, int BITS = 4, bool R2 = false>
 struct Cfg {
     static_assert(D % 32 == 0 && D >= 64 && D <= 160, "head dim not built");
+    static_assert(!R2 || (D == 128 && !BF16OUT && BITS == 4), "radix-2 form: D = 128, fp16 output, 4-bit codes");
     static_assert(!BF16OUT || BITS == 4 || D <= 128, "two-term operands with byte codes: shared memory holds them for D <= 128 only");
     static_assert(BITS == 4 || BITS == 8, "code width not built");
     static constexpr int kTerms = BF16OUT ? 2 : 1;         // W_hi (, W_lo); a_hi (, a_lo)
@@ -69,7 +78,8 @@ struct Cfg {
     static constexpr int kKBlocks = (D + 63) / 64;         // K blocks of 64 elements (the last one may be half used)
     static constexpr int kBBlock = D * 128;                // bytes of one K block: D rows x 128 B
     static constexpr int kBTerm = kKBlocks * kBBlock;
-    static constexpr int kBBytes = kTerms * kBTerm;
+    static constexpr int kBPart = (D / 2) * 128;           // R2: one parity's operand, D / 2 outputs x D / 2 channels
+    static constexpr int kBBytes = R2 ? 2 * kBPart : kTerms * kBTerm;
     static constexpr int kInRow = D * BITS / 8;            // code bytes per row
     static constexpr int kInBytes = kTile * kInRow;        // bytes one TMA load brings
     static constexpr int kInPitch = (kInBytes + 1023) & ~1023;
@@ -98,7 +108,8 @@ struct Cfg {
     {
         return D <= 128 ? 256u + 64u * (uint32_t)kTerms * (uint32_t)s : 160u + 256u * (uint32_t)s;
     }
-    static constexpr uint32_t kIdesc = umma_idesc_m128(D, false);
+    static constexpr uint32_t kIdesc = umma_idesc_m128(R2 ? D / 2 : D, false);
+    static constexpr int kBRows = R2 ? D / 2 : D;          // rows of the plan table that B is built from
 };
 
 struct Ctrl {
@@ -182,7 +193,26 @@ __device__ __forceinline__ void build_b_quad(unsigned char *sB, float4 m, const 
     }
 }
 
-template <int D, bool BF16OUT, int BITS>
+// Radix-2 form, row n < D / 2 of both parities' operands.  The lane's four channels 4 i .. 4 i + 3 alternate in parity;
+// per parity p the even lane assembles the pair (8w + p, 8w + p + 4) and the odd lane (8w + p + 2, 8w + p + 6), each from
+// one value of its own and one of its neighbour's: the K order in which the dequant threads write the codes of parity p.
+template <int D>
+__device__ __forceinline__ void build_b_quad_r2(unsigned char *sB, float4 m, const RecipLambda<D> &rl, int n, int lane)
+{
+    static_assert(D == 128, "one pass of 32 lanes covers the row");
+    const bool odd = lane & 1;
+    auto sat = [](float v) { return fminf(fmaxf(v, -65504.0f), 65504.0f); };
+    const float v[4] = {sat(m.x * rl.r[0].x), sat(m.y * rl.r[0].y), sat(m.z * rl.r[0].z), sat(m.w * rl.r[0].w)};
+    const int w = lane >> 1;   // word of 8 codes; its parity-p codes take bytes 8 w .. 8 w + 7 of the parity's K-major row
+#pragma unroll
+    for (int p = 0; p < 2; ++p) {
+        const float got = __shfl_xor_sync(0xFFFFFFFFu, odd ? v[p] : v[p + 2], 1);
+        const uint32_t h = odd ? narrow2<false>(got, v[p + 2]) : narrow2<false>(v[p], got);
+        *reinterpret_cast<uint32_t *>(sB + p * ((D / 2) * 128) + n * 128 + ((((w >> 1) ^ (n & 7))) << 4) + ((w & 1) ? 8 : 0) + (odd ? 4 : 0)) = h;
+    }
+}
+
+template <int D, bool BF16OUT, int BITS, bool R2>
 __device__ __forceinline__ void build_b_rows(unsigned char *sB, const float *__restrict__ b0, const RecipLambda<D> &rl, int n0, int n1,
                                              int lane)
 {
@@ -193,16 +223,17 @@ __device__ __forceinline__ void build_b_rows(unsigned char *sB, const float *__r
             const int i = lane + 32 * p;
             float4 m = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
             if (i < D / 4) m = __ldg(reinterpret_cast<const float4 *>(b0 + (size_t)n * D) + i);
-            build_b_quad<D, BF16OUT, BITS>(sB, m, rl, n, p, lane);
+            if constexpr (R2) build_b_quad_r2<D>(sB, m, rl, n, lane);
+            else build_b_quad<D, BF16OUT, BITS>(sB, m, rl, n, p, lane);
         }
     }
 }
 
 // The first build of a CTA: its D / 16 table rows per warp are requested at kernel entry, all at once, and turned
 // into B rows here, once lambda has arrived too: one round trip to L2 instead of one per batch of rows.
-template <int D, bool BF16OUT, int BITS>
+template <int D, bool BF16OUT, int BITS, bool R2>
 struct FirstRows {
-    static constexpr int kRows = D / 16, kPasses = RecipLambda<D>::kPasses;
+    static constexpr int kRows = (R2 ? D / 2 : D) / 16, kPasses = RecipLambda<D>::kPasses;
     float4 m[kRows][kPasses];
     __device__ __forceinline__ void load(const float *__restrict__ b0, int n0, int lane)
     {
@@ -219,7 +250,10 @@ struct FirstRows {
 #pragma unroll
         for (int k = 0; k < kRows; ++k)
 #pragma unroll
-            for (int p = 0; p < kPasses; ++p) build_b_quad<D, BF16OUT, BITS>(sB, m[k][p], rl, n0 + k, p, lane);
+            for (int p = 0; p < kPasses; ++p) {
+                if constexpr (R2) build_b_quad_r2<D>(sB, m[k][p], rl, n0 + k, lane);
+                else build_b_quad<D, BF16OUT, BITS>(sB, m[k][p], rl, n0 + k, p, lane);
+            }
     }
 };
 
@@ -250,6 +284,7 @@ struct UmmaDecodeParams {
     int64_t rpl;        // rows per lambda segment (N when there is one lambda row)
     int64_t n_seg;      // segments
     int64_t n_full;     // segments of exactly rpl rows, covered by the main output maps; a shorter last one uses the tail maps
+    uint32_t flip2[32]; // radix-2 form: sign-bit masks of s_n s_{n + 64} for the output pairs (n, n + 1), n = 0, 2, .. 62
 };
 
 struct UmmaDecodeMaps {
@@ -258,11 +293,11 @@ struct UmmaDecodeMaps {
     CUtensorMap slim, slim_tail;   // output, boxes of 32 columns x 32 rows (64-byte swizzle), used when D / 32 is odd
 };
 
-template <int D, bool BF16OUT, int BITS>
+template <int D, bool BF16OUT, int BITS, bool R2>
 __global__ void __launch_bounds__(kThreads, 1)
     kvq_decode_umma_kernel(const __grid_constant__ UmmaDecodeParams prm, const __grid_constant__ UmmaDecodeMaps maps)
 {
-    using C = Cfg<D, BF16OUT, BITS>;
+    using C = Cfg<D, BF16OUT, BITS, R2>;
     constexpr int G = C::G, kInStages = C::kInStages;
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -308,15 +343,15 @@ __global__ void __launch_bounds__(kThreads, 1)
     // ---- producer's first loads are in flight; the mma warp waits for all of them.  Table rows and lambda are
     // ---- requested before the set-up barrier, so that their latency runs under it.
     if (n_my > 0 && warp >= 2) {
-        FirstRows<D, BF16OUT, BITS> rows;
-        rows.load(prm.g.b0, (warp - 2) * (D / 16), lane);
+        FirstRows<D, BF16OUT, BITS, R2> rows;
+        rows.load(prm.g.b0, (warp - 2) * (C::kBRows / 16), lane);
         const RecipLambda<D> rl(lambda_row(seg_first), lane);
         if (rl.wide && warp == 2 && lane == 0) atomicOr(prm.g.status, KVQ_DEV_RANGE);
         fence_proxy_async();
         tc_fence_before();
         __syncthreads();
         tc_fence_after();
-        rows.build(sB, rl, (warp - 2) * (D / 16), lane);
+        rows.build(sB, rl, (warp - 2) * (C::kBRows / 16), lane);
         fence_proxy_async();   // B is read by the tensor core through the async proxy
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&ctrl->b_first));
@@ -369,9 +404,21 @@ __global__ void __launch_bounds__(kThreads, 1)
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + C::acc_col(sc);
                 const uint32_t a_tmem = tmem_base + C::a_col(sa);
+                if constexpr (R2) {   // E = A_even B_even into the first D / 2 accumulator columns, O = A_odd B_odd into the rest
+#pragma unroll
+                    for (int p = 0; p < 2; ++p) {
+#pragma unroll
+                        for (int ks = 0; ks < D / 32; ++ks) {
+                            const uint64_t bd = ((uint64_t)b_hi << 32) | (uint64_t)(b_lo + (uint32_t)p * (C::kBPart >> 4) + (uint32_t)ks * 2u);
+                            const uint32_t dp = d_tmem + (uint32_t)p * (D / 2), ap = a_tmem + (uint32_t)p * (D / 4) + (uint32_t)ks * 8u;
+                            if (ks > 0) umma_f16_ts<true>(dp, ap, bd, C::kIdesc);
+                            else umma_f16_ts<false>(dp, ap, bd, C::kIdesc);
+                        }
+                    }
+                }
                 // bf16 output: a_hi W_hi + a_lo W_hi + a_hi W_lo
 #pragma unroll
-                for (int set = 0; set < (BF16OUT ? 3 : 1); ++set) {
+                for (int set = 0; set < (R2 ? 0 : BF16OUT ? 3 : 1); ++set) {
                     const uint32_t a_set = a_tmem + (set == 1 ? C::kALo : 0u);
                     const uint32_t b_set = b_lo + (set == 2 ? (uint32_t)(C::kBTerm >> 4) : 0u);
 #pragma unroll
@@ -444,7 +491,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                                        status, KVQ_DEV_MMA_TIMEOUT))
                         break;
                     if (rl.wide && q == 0 && lane == 0) atomicOr(status, KVQ_DEV_RANGE);
-                    build_b_rows<D, BF16OUT, BITS>(sB, prm.g.b0, rl, q * (D / 4), (q + 1) * (D / 4), lane);
+                    build_b_rows<D, BF16OUT, BITS, R2>(sB, prm.g.b0, rl, q * (C::kBRows / 4), (q + 1) * (C::kBRows / 4), lane);
                     fence_proxy_async();   // B is read by the tensor core through the async proxy
                 }
                 cached_seg = seg;
@@ -499,7 +546,8 @@ __global__ void __launch_bounds__(kThreads, 1)
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             const uint32_t m = lop3_and_or(u >> (4 * e), 0x000F000Fu, 0x64006400u);   // {1024 + n_e, 1024 + n_{e+4}}
-                            put(4 * i + e, __hsub2(*reinterpret_cast<const __half2 *>(&m), h1032));    // exact q
+                            // radix-2 form: pairs 0 and 2 of a word are even channels (first half of a[]), 1 and 3 odd (second half)
+                            put(R2 ? 8 * (e & 1) + 2 * i + (e >> 1) : 4 * i + e, __hsub2(*reinterpret_cast<const __half2 *>(&m), h1032));   // exact q
                         }
                     }
                 } else {   // 32 byte codes: two 16-byte chunks of the row, pairs of neighbours
@@ -518,7 +566,14 @@ __global__ void __launch_bounds__(kThreads, 1)
                         }
                     }
                 }
-                tmem_st16(a_row + 16u * (uint32_t)c, a);
+                if constexpr (R2) {   // 8 columns of the even operand, 8 of the odd one
+                    const uint32_t ae[8] = {a[0], a[1], a[2], a[3], a[4], a[5], a[6], a[7]};
+                    const uint32_t ao[8] = {a[8], a[9], a[10], a[11], a[12], a[13], a[14], a[15]};
+                    tmem_st8(a_row + 8u * (uint32_t)c, ae);
+                    tmem_st8(a_row + (uint32_t)(D / 4) + 8u * (uint32_t)c, ao);
+                } else {
+                    tmem_st16(a_row + 16u * (uint32_t)c, a);
+                }
                 if constexpr (BF16OUT) tmem_st16(a_row + C::kALo + 16u * (uint32_t)c, al);
             }
             if constexpr (BITS == 8) {   // the packed rows were read group by group: only now is their stage free
@@ -546,8 +601,39 @@ __global__ void __launch_bounds__(kThreads, 1)
             __syncwarp();
             const float row_inv = ctrl->row_scale[j & (kRowScaleSlots - 1)][q * 32 + lane];
             const bool rescale = __any_sync(0xFFFFFFFFu, row_inv != 1.0f);   // rare: a row outside the operand's comfort zone
+            if constexpr (R2) {
 #pragma unroll
-            for (int cc = 0; cc < G; ++cc) {   // 32 accumulator columns = 64 bytes of the output row
+                for (int h = 0; h < 4; ++h) {   // E and O columns 16 h .. 16 h + 15 -> outputs 16 h .. and D / 2 + 16 h ..
+                    uint32_t ev[16], ov[16];
+                    tmem_ld16(lane_addr + C::acc_col(sc) + (uint32_t)h * 16u, ev);
+                    tmem_ld16(lane_addr + C::acc_col(sc) + (uint32_t)(D / 2) + (uint32_t)h * 16u, ov);
+                    tmem_ld_wait();
+                    if (rescale) {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            ev[i] = __float_as_uint(__uint_as_float(ev[i]) * row_inv);
+                            ov[i] = __float_as_uint(__uint_as_float(ov[i]) * row_inv);
+                        }
+                    }
+#pragma unroll
+                    for (int k = 0; k < 2; ++k) {   // 16-byte chunk: 8 outputs
+                        uint32_t lo[4], hi[4];
+#pragma unroll
+                        for (int p2 = 0; p2 < 4; ++p2) {
+                            const int i = 8 * k + 2 * p2;
+                            const float e0 = __uint_as_float(ev[i]), e1 = __uint_as_float(ev[i + 1]);
+                            const float o0 = __uint_as_float(ov[i]), o1 = __uint_as_float(ov[i + 1]);
+                            lo[p2] = narrow2<false>(e0 + o0, e1 + o1);                                       // s_n is already in E and O
+                            hi[p2] = narrow2<false>(e0 - o0, e1 - o1) ^ prm.flip2[8 * h + 4 * k + p2];       // times s_n s_{n + D/2}
+                        }
+                        const int chunk = 2 * h + k;   // both halves of the row are 64-column boxes: [32 rows][128 B], 128-byte swizzle
+                        *reinterpret_cast<uint4 *>(stg + lane * 128 + ((chunk ^ (lane & 7)) << 4)) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                        *reinterpret_cast<uint4 *>(stg + 32 * 128 + lane * 128 + ((chunk ^ (lane & 7)) << 4)) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                    }
+                }
+            }
+#pragma unroll
+            for (int cc = 0; cc < (R2 ? 0 : G); ++cc) {   // 32 accumulator columns = 64 bytes of the output row
                 uint32_t v[32];
                 tmem_ld32(lane_addr + C::acc_col(sc) + (uint32_t)cc * 32u, v);
                 tmem_ld_wait();
@@ -608,10 +694,10 @@ __global__ void __launch_bounds__(kThreads, 1)
 // ------------------------------------------------------------------------------------------------
 namespace {
 
-template <int D, bool BF16OUT, int BITS = 4>
-cudaError_t launch(int64_t N, const GemmParams &g, cudaStream_t stream)
+template <int D, bool BF16OUT, int BITS = 4, bool R2 = false>
+cudaError_t launch(int64_t N, const GemmParams &g, cudaStream_t stream, const uint32_t *sign_xor = nullptr)
 {
-    using C = Cfg<D, BF16OUT, BITS>;
+    using C = Cfg<D, BF16OUT, BITS, R2>;
     static DeviceSlots slots;
     int dev = 0;
     cudaError_t e = current_device_slot(&dev);
@@ -619,7 +705,7 @@ cudaError_t launch(int64_t N, const GemmParams &g, cudaStream_t stream)
     int &sms = slots.sms[dev];
     if (sms == 0) {
         int n = 0;
-        if ((e = cudaFuncSetAttribute(kvq_decode_umma_kernel<D, BF16OUT, BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes)) != cudaSuccess) return e;
+        if ((e = cudaFuncSetAttribute(kvq_decode_umma_kernel<D, BF16OUT, BITS, R2>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes)) != cudaSuccess) return e;
         if ((e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
         sms = n;
     }
@@ -631,6 +717,7 @@ cudaError_t launch(int64_t N, const GemmParams &g, cudaStream_t stream)
     prm.rpl = g.n_lambda == 1 ? N : g.rows_per_lambda;
     prm.n_seg = (N + prm.rpl - 1) / prm.rpl;
     prm.n_full = N / prm.rpl;
+    for (int m = 0; m < 32; ++m) prm.flip2[m] = R2 && sign_xor ? sign_xor[m] ^ sign_xor[m + D / 4] : 0u;   // words hold two signs each
 
     UmmaDecodeMaps maps;
     {
@@ -661,7 +748,7 @@ cudaError_t launch(int64_t N, const GemmParams &g, cudaStream_t stream)
 
     const int64_t tiles = prm.n_seg * ((prm.rpl + kTile - 1) / kTile);
     const int grid = (int)(tiles < sms ? tiles : sms);
-    kvq_decode_umma_kernel<D, BF16OUT, BITS><<<grid, kThreads, C::kSmemBytes, stream>>>(prm, maps);
+    kvq_decode_umma_kernel<D, BF16OUT, BITS, R2><<<grid, kThreads, C::kSmemBytes, stream>>>(prm, maps);
     count_launch();
     return cudaGetLastError();
 }
@@ -677,8 +764,11 @@ bool umma_decode_supported(int D, bool bf16)
 // byte codes: the D <= 160 kernel only (D <= 128 with bf16 output)
 bool umma_decode_bits8_supported(int D, bool bf16) { return D != 256 && !(D == 160 && bf16) && umma_decode_supported(D, bf16); }
 
-cudaError_t umma_decode(int D, bool bf16, int bits, int64_t N, const GemmParams &g, const uint32_t *sign_xor, cudaStream_t stream)
+cudaError_t umma_decode(int D, bool bf16, int bits, int64_t N, const GemmParams &g, const uint32_t *sign_xor, cudaStream_t stream,
+                        bool radix2)
 {
+    // the radix-2 form needs the transform's even / odd structure: the caller asks for it on plans without a rotation
+    if (radix2 && D == 128 && !bf16 && bits == 4 && sign_xor) return launch<128, false, 4, true>(N, g, stream, sign_xor);
     if (bits == 8) {
         switch (D) {
             case 64: return bf16 ? launch<64, true, 8>(N, g, stream) : launch<64, false, 8>(N, g, stream);

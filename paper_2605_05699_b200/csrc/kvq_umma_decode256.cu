@@ -79,14 +79,6 @@ struct Ctrl {
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
 
-// 8 consecutive columns of this thread's tensor-memory lane
-__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&r)[8])
-{
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"r"(taddr), "r"(r[0]), "r"(r[1]),
-                 "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
-                 : "memory");
-}
-
 // 1 / max(lambda, 1e-6) for the channels 4 i .. 4 i + 3, i = lane and lane + 32, divided by rho, the power of two
 // that brings the row's largest reciprocal into [1, 2).  Every lane gets rho.
 struct RecipLambda {
