@@ -69,7 +69,7 @@ constexpr uint32_t kTmemCols = 512;
 template <int D, bool BF16OUT, int BITS = 4, bool R2 = false>
 struct Cfg {
     static_assert(D % 32 == 0 && D >= 64 && D <= 160, "head dim not built");
-    static_assert(!R2 || (D == 128 && !BF16OUT && BITS == 4), "radix-2 form: D = 128, fp16 output, 4-bit codes");
+    static_assert(!R2 || (D == 128 && BITS == 4), "radix-2 form: D = 128, 4-bit codes");
     static_assert(!BF16OUT || BITS == 4 || D <= 128, "two-term operands with byte codes: shared memory holds them for D <= 128 only");
     static_assert(BITS == 4 || BITS == 8, "code width not built");
     static constexpr int kTerms = BF16OUT ? 2 : 1;         // W_hi (, W_lo); a_hi (, a_lo)
@@ -79,7 +79,7 @@ struct Cfg {
     static constexpr int kBBlock = D * 128;                // bytes of one K block: D rows x 128 B
     static constexpr int kBTerm = kKBlocks * kBBlock;
     static constexpr int kBPart = (D / 2) * 128;           // R2: one parity's operand, D / 2 outputs x D / 2 channels
-    static constexpr int kBBytes = R2 ? 2 * kBPart : kTerms * kBTerm;
+    static constexpr int kBBytes = R2 ? kTerms * 2 * kBPart : kTerms * kBTerm;   // R2: [term][parity]
     static constexpr int kInRow = D * BITS / 8;            // code bytes per row
     static constexpr int kInBytes = kTile * kInRow;        // bytes one TMA load brings
     static constexpr int kInPitch = (kInBytes + 1023) & ~1023;
@@ -196,10 +196,11 @@ __device__ __forceinline__ void build_b_quad(unsigned char *sB, float4 m, const 
 // Radix-2 form, row n < D / 2 of both parities' operands.  The lane's four channels 4 i .. 4 i + 3 alternate in parity;
 // per parity p the even lane assembles the pair (8w + p, 8w + p + 4) and the odd lane (8w + p + 2, 8w + p + 6), each from
 // one value of its own and one of its neighbour's: the K order in which the dequant threads write the codes of parity p.
-template <int D>
+template <int D, int TERMS>
 __device__ __forceinline__ void build_b_quad_r2(unsigned char *sB, float4 m, const RecipLambda<D> &rl, int n, int lane)
 {
     static_assert(D == 128, "one pass of 32 lanes covers the row");
+    constexpr int kPart = (D / 2) * 128;
     const bool odd = lane & 1;
     auto sat = [](float v) { return fminf(fmaxf(v, -65504.0f), 65504.0f); };
     const float v[4] = {sat(m.x * rl.r[0].x), sat(m.y * rl.r[0].y), sat(m.z * rl.r[0].z), sat(m.w * rl.r[0].w)};
@@ -207,8 +208,17 @@ __device__ __forceinline__ void build_b_quad_r2(unsigned char *sB, float4 m, con
 #pragma unroll
     for (int p = 0; p < 2; ++p) {
         const float got = __shfl_xor_sync(0xFFFFFFFFu, odd ? v[p] : v[p + 2], 1);
-        const uint32_t h = odd ? narrow2<false>(got, v[p + 2]) : narrow2<false>(v[p], got);
-        *reinterpret_cast<uint32_t *>(sB + p * ((D / 2) * 128) + n * 128 + ((((w >> 1) ^ (n & 7))) << 4) + ((w & 1) ? 8 : 0) + (odd ? 4 : 0)) = h;
+        float w0 = odd ? got : v[p], w1 = odd ? v[p + 2] : got;
+        unsigned char *dst = sB + p * kPart + n * 128 + ((((w >> 1) ^ (n & 7))) << 4) + ((w & 1) ? 8 : 0) + (odd ? 4 : 0);
+#pragma unroll
+        for (int t = 0; t < TERMS; ++t) {
+            const uint32_t h = narrow2<false>(w0, w1);
+            *reinterpret_cast<uint32_t *>(dst + t * (2 * kPart)) = h;
+            if (t + 1 < TERMS) {   // what the fp16 term left behind (exact in fp32)
+                const float2 a = widen2<false>(h);
+                w0 -= a.x, w1 -= a.y;
+            }
+        }
     }
 }
 
@@ -223,7 +233,7 @@ __device__ __forceinline__ void build_b_rows(unsigned char *sB, const float *__r
             const int i = lane + 32 * p;
             float4 m = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
             if (i < D / 4) m = __ldg(reinterpret_cast<const float4 *>(b0 + (size_t)n * D) + i);
-            if constexpr (R2) build_b_quad_r2<D>(sB, m, rl, n, lane);
+            if constexpr (R2) build_b_quad_r2<D, Cfg<D, BF16OUT, BITS, R2>::kTerms>(sB, m, rl, n, lane);
             else build_b_quad<D, BF16OUT, BITS>(sB, m, rl, n, p, lane);
         }
     }
@@ -251,7 +261,7 @@ struct FirstRows {
         for (int k = 0; k < kRows; ++k)
 #pragma unroll
             for (int p = 0; p < kPasses; ++p) {
-                if constexpr (R2) build_b_quad_r2<D>(sB, m[k][p], rl, n0 + k, lane);
+                if constexpr (R2) build_b_quad_r2<D, Cfg<D, BF16OUT, BITS, R2>::kTerms>(sB, m[k][p], rl, n0 + k, lane);
                 else build_b_quad<D, BF16OUT, BITS>(sB, m[k][p], rl, n0 + k, p, lane);
             }
     }
@@ -408,11 +418,16 @@ __global__ void __launch_bounds__(kThreads, 1)
 #pragma unroll
                     for (int p = 0; p < 2; ++p) {
 #pragma unroll
-                        for (int ks = 0; ks < D / 32; ++ks) {
-                            const uint64_t bd = ((uint64_t)b_hi << 32) | (uint64_t)(b_lo + (uint32_t)p * (C::kBPart >> 4) + (uint32_t)ks * 2u);
-                            const uint32_t dp = d_tmem + (uint32_t)p * (D / 2), ap = a_tmem + (uint32_t)p * (D / 4) + (uint32_t)ks * 8u;
-                            if (ks > 0) umma_f16_ts<true>(dp, ap, bd, C::kIdesc);
-                            else umma_f16_ts<false>(dp, ap, bd, C::kIdesc);
+                        for (int set = 0; set < (BF16OUT ? 3 : 1); ++set) {   // bf16 output: a_hi W_hi + a_lo W_hi + a_hi W_lo
+#pragma unroll
+                            for (int ks = 0; ks < D / 32; ++ks) {
+                                const uint32_t b_set = b_lo + (set == 2 ? (uint32_t)((2 * C::kBPart) >> 4) : 0u) + (uint32_t)p * (C::kBPart >> 4);
+                                const uint64_t bd = ((uint64_t)b_hi << 32) | (uint64_t)(b_set + (uint32_t)ks * 2u);
+                                const uint32_t dp = d_tmem + (uint32_t)p * (D / 2);
+                                const uint32_t ap = a_tmem + (set == 1 ? C::kALo : 0u) + (uint32_t)p * (D / 4) + (uint32_t)ks * 8u;
+                                if (set > 0 || ks > 0) umma_f16_ts<true>(dp, ap, bd, C::kIdesc);
+                                else umma_f16_ts<false>(dp, ap, bd, C::kIdesc);
+                            }
                         }
                     }
                 }
@@ -571,10 +586,16 @@ __global__ void __launch_bounds__(kThreads, 1)
                     const uint32_t ao[8] = {a[8], a[9], a[10], a[11], a[12], a[13], a[14], a[15]};
                     tmem_st8(a_row + 8u * (uint32_t)c, ae);
                     tmem_st8(a_row + (uint32_t)(D / 4) + 8u * (uint32_t)c, ao);
+                    if constexpr (BF16OUT) {
+                        const uint32_t le[8] = {al[0], al[1], al[2], al[3], al[4], al[5], al[6], al[7]};
+                        const uint32_t lo[8] = {al[8], al[9], al[10], al[11], al[12], al[13], al[14], al[15]};
+                        tmem_st8(a_row + C::kALo + 8u * (uint32_t)c, le);
+                        tmem_st8(a_row + C::kALo + (uint32_t)(D / 4) + 8u * (uint32_t)c, lo);
+                    }
                 } else {
                     tmem_st16(a_row + 16u * (uint32_t)c, a);
+                    if constexpr (BF16OUT) tmem_st16(a_row + C::kALo + 16u * (uint32_t)c, al);
                 }
-                if constexpr (BF16OUT) tmem_st16(a_row + C::kALo + 16u * (uint32_t)c, al);
             }
             if constexpr (BITS == 8) {   // the packed rows were read group by group: only now is their stage free
                 __syncwarp();
@@ -623,8 +644,8 @@ __global__ void __launch_bounds__(kThreads, 1)
                             const int i = 8 * k + 2 * p2;
                             const float e0 = __uint_as_float(ev[i]), e1 = __uint_as_float(ev[i + 1]);
                             const float o0 = __uint_as_float(ov[i]), o1 = __uint_as_float(ov[i + 1]);
-                            lo[p2] = narrow2<false>(e0 + o0, e1 + o1);                                       // s_n is already in E and O
-                            hi[p2] = narrow2<false>(e0 - o0, e1 - o1) ^ prm.flip2[8 * h + 4 * k + p2];       // times s_n s_{n + D/2}
+                            lo[p2] = narrow2<BF16OUT>(e0 + o0, e1 + o1);                                     // s_n is already in E and O
+                            hi[p2] = narrow2<BF16OUT>(e0 - o0, e1 - o1) ^ prm.flip2[8 * h + 4 * k + p2];     // times s_n s_{n + D/2}
                         }
                         const int chunk = 2 * h + k;   // both halves of the row are 64-column boxes: [32 rows][128 B], 128-byte swizzle
                         *reinterpret_cast<uint4 *>(stg + lane * 128 + ((chunk ^ (lane & 7)) << 4)) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
@@ -768,7 +789,8 @@ cudaError_t umma_decode(int D, bool bf16, int bits, int64_t N, const GemmParams 
                         bool radix2)
 {
     // the radix-2 form needs the transform's even / odd structure: the caller asks for it on plans without a rotation
-    if (radix2 && D == 128 && !bf16 && bits == 4 && sign_xor) return launch<128, false, 4, true>(N, g, stream, sign_xor);
+    if (radix2 && D == 128 && bits == 4 && sign_xor)
+        return bf16 ? launch<128, true, 4, true>(N, g, stream, sign_xor) : launch<128, false, 4, true>(N, g, stream, sign_xor);
     if (bits == 8) {
         switch (D) {
             case 64: return bf16 ? launch<64, true, 8>(N, g, stream) : launch<64, false, 8>(N, g, stream);
