@@ -551,7 +551,7 @@ def measure_append_dispatch(kb, wl, dev, dtype, S, layers=80, T=1024, iters=20):
 # DRAM bytes per full launch (2,097,152 vectors, the bench's launch size) from ncu: dram__bytes_read.sum +
 # dram__bytes_write.sum, one-pass capture; see profiles/dram_traffic_d128_n2097152.md.  Reads match the algorithmic
 # bytes; writes are short of them by what is still in the 126 MB L2 when the kernel ends.
-TRAFFIC = {"decode": 151166464 + 476459776, "encode": 537959424 + 128567040}
+TRAFFIC = {"decode": 151190784 + 476806656, "encode": 538161152 + 128756736}
 
 
 # --------------------------------------------------------------------------------------------

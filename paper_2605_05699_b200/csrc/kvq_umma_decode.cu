@@ -64,7 +64,7 @@ constexpr uint32_t kTmemCols = 512;
 //     x^_n = s_n (E_n + O_n),        x^_{n + D/2} = s_{n + D/2} (E_n - O_n):
 // two 128 x 64 x 64 GEMMs per tile instead of one 128 x 128 x 128, half the tensor work, and an add, a subtract and half a
 // sign flip per output in the epilogue.  The kernel runs at the board's power limit, where tensor flops are what is left to
-// save: 148 -> 137 us per 2M-vector launch back to back.  The half2 nibble trick yields pairs (c, c + 4) of equal parity, so
+// save: 147 -> 134 us per 2M-vector launch back to back (bf16 output: 215 -> 192 us).  The half2 nibble trick yields pairs (c, c + 4) of equal parity, so
 // routing codes to the two A operands is free.
 template <int D, bool BF16OUT, int BITS = 4, bool R2 = false>
 struct Cfg {
