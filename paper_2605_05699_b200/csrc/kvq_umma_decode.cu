@@ -58,14 +58,14 @@ constexpr uint32_t kTmemCols = 512;
 // W' = W_hi + W_lo, and x^ = a_hi W_hi + a_lo W_hi + a_hi W_lo accumulates in fp32 (a_lo W_lo is below 1e-7).
 // BITS: 4 (nibble pairs) or 8 (one two's-complement byte per code; scale = absmax / 127).  The byte path dequantises
 // pairs of neighbouring codes, so its K order is the natural one and the B operand is built to match.
-// R2: one radix-2 step of the transform is taken out of the GEMM (plans without a rotation; D = 128, fp16 output, 4-bit
-// codes).  Rows of M are cos / sin(2 pi k n / D), so n -> n + D / 2 multiplies a row by (-1)^k, and in the packing of Eq. 2
+// R2: one radix-2 step of the transform is taken out of the GEMM (plans without a rotation; D = 128, 4-bit codes, either
+// output type).  Rows of M are cos / sin(2 pi k n / D), so n -> n + D / 2 multiplies a row by (-1)^k, and in the packing of Eq. 2
 // the parity of k is the parity of the channel c.  With E_n / O_n the sums over the even / odd channels (n < D / 2),
 //     x^_n = s_n (E_n + O_n),        x^_{n + D/2} = s_{n + D/2} (E_n - O_n):
 // two 128 x 64 x 64 GEMMs per tile instead of one 128 x 128 x 128, half the tensor work, and an add, a subtract and half a
 // sign flip per output in the epilogue.  The kernel runs at the board's power limit, where tensor flops are what is left to
-// save: 147 -> 134 us per 2M-vector launch back to back (bf16 output: 215 -> 192 us).  The half2 nibble trick yields pairs (c, c + 4) of equal parity, so
-// routing codes to the two A operands is free.
+// save: 147 -> 134 us per 2M-vector launch back to back (bf16 output: 215 -> 192 us).  The half2 nibble trick yields pairs
+// (c, c + 4) of equal parity, so routing codes to the two A operands is free.
 template <int D, bool BF16OUT, int BITS = 4, bool R2 = false>
 struct Cfg {
     static_assert(D % 32 == 0 && D >= 64 && D <= 160, "head dim not built");
