@@ -293,14 +293,14 @@ def run_ours(args):
     enc_gbs = N * BYTES_PER_VEC / (enc_avg * 1e-3) / 1e9
     # The two large kernels take about the same time; the graded one is the full-prefix decode.  2 D^2 = 32768 flops per
     # vector at the measured sustained tensor rate are ~0.023 ns/vec, below the 0.051 ns/vec of bytes: HBM is the roof.
-    roofline = {"bound": "hbm", "kernel": "kvq_decode_umma_d128_kernel (full-prefix read, %d vectors per launch)" % N,
+    roofline = {"bound": "hbm", "kernel": "kvq_decode_umma_kernel<128, fp16 out, 4-bit, radix-2> (full-prefix read, %d vectors per launch)" % N,
                 "achieved": dec_gbs, "peak": peak, "unit": "GB/s", "frac": dec_gbs / peak,
                 "peak_source": peak_src, "algorithmic_bytes_per_launch": N * BYTES_PER_VEC,
                 "avg_launch_ms": dec_avg, "traffic": TRAFFIC.get("decode"),
                 "sustained_copy_GBps": copy_gbs, "frac_of_sustained_copy": dec_gbs / copy_gbs,
                 "sustained_copy_note": "a plain device copy of one layer buffer, back to back for 0.3 s in this run: the same "
                                        "power-capped regime as the timed region (peak above is the driver's burst copy)",
-                "encode": {"kernel": "kvq_encode_umma_d128_kernel (%d vectors per launch)" % N, "achieved": enc_gbs,
+                "encode": {"kernel": "kvq_encode_umma_kernel<128, fp16 in> (%d vectors per launch)" % N, "achieved": enc_gbs,
                            "frac": enc_gbs / peak, "avg_launch_ms": enc_avg, "traffic": TRAFFIC.get("encode")}}
     cpu = cpu_baseline_sample(target_seconds=12.0)
     line = {
