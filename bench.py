@@ -291,8 +291,9 @@ def run_ours(args):
     enc_avg = sum(enc_ms) / len(enc_ms)
     dec_gbs = N * BYTES_PER_VEC / (dec_avg * 1e-3) / 1e9
     enc_gbs = N * BYTES_PER_VEC / (enc_avg * 1e-3) / 1e9
-    # The two large kernels take about the same time; the graded one is the full-prefix decode.  2 D^2 = 32768 flops per
-    # vector at the measured sustained tensor rate are ~0.023 ns/vec, below the 0.051 ns/vec of bytes: HBM is the roof.
+    # The graded kernel is the full-prefix decode.  Its contraction is D^2 = 16384 flops per vector (one radix-2 step is taken
+    # out of the 2 D^2 dense form; the encode runs two dense terms): ~0.012 ns/vec at the measured sustained tensor rate,
+    # below the 0.051 ns/vec of bytes: HBM is the roof.
     roofline = {"bound": "hbm", "kernel": "kvq_decode_umma_kernel<128, fp16 out, 4-bit, radix-2> (full-prefix read, %d vectors per launch)" % N,
                 "achieved": dec_gbs, "peak": peak, "unit": "GB/s", "frac": dec_gbs / peak,
                 "peak_source": peak_src, "algorithmic_bytes_per_launch": N * BYTES_PER_VEC,
