@@ -20,8 +20,9 @@
  *   - every data pointer is a DEVICE pointer owned by the caller unless it says "host".
  *     The library owns only the plan and the small device tables hanging off it.
  *   - calls are asynchronous on the given CUDA stream (a cudaStream_t passed as void*,
- *     NULL = default stream); they do not synchronize.  kvq_encode / kvq_decode /
- *     kvq_append allocate nothing after the plan's first use on a device.
+ *     NULL = default stream).  The first use of a plan on a device allocates its small tables and
+ *     copies them with a blocking copy; kvq_plan_prepare does that, and the per-kernel set-up,
+ *     ahead of time, after which the compute calls allocate nothing and never synchronize.
  *   - every function returns a kvq_status_t; nothing throws across the boundary.
  *     Arguments are validated on the host before any CUDA call is made.
  *   - there is no CPU fallback: without a CUDA device the compute calls return KVQ_ERR_CUDA.
@@ -69,8 +70,8 @@ typedef enum {
 } kvq_impl_t;
 
 /*
- * kvq_plan_create -- "kvq_plan(D, group, seed)": draws the sign diagonal s (Sec. 3.1: "a fixed
- * random sign vector drawn at initialization") and fixes the radix plan of the length-D/2
+ * kvq_plan_create -- "kvq_plan(D, group, seed)": draws the sign diagonal s (Sec. 3.1: one random
+ * sign per coordinate, fixed for the life of the plan) and fixes the radix plan of the length-D/2
  * complex FFT (Sec. 3.2 step 2; mixed radix 3 / 5 for D = 96 / 160).
  *   D      head dimension; supported: 64, 96, 128, 160, 256.
  *   group  coordinates per scale; supported: 32, or D (one scale per vector).
@@ -128,6 +129,35 @@ kvq_status_t kvq_plan_describe(const kvq_plan_t *plan, int *radices, int *n_radi
  * (decode_impl) calls on this plan.  Default: AUTO for both. */
 kvq_status_t kvq_plan_set_impl(kvq_plan_t *plan, kvq_impl_t encode_impl, kvq_impl_t decode_impl);
 
+/*
+ * kvq_plan_prepare -- everything a compute call would otherwise do on its first use, done now, on the
+ * device that is current: allocates the plan's device tables (a status word; two [D, D] fp32 tables
+ * where a tensor-core or matrix-vector kernel serves the plan), fills them with blocking copies, and
+ * sets the launch attributes (shared-memory size, occupancy look-ups) of every kernel that a call with
+ * this plan and this 16-bit type can take, whichever family kvq_plan_set_impl or AUTO picks later.
+ *   dtype   the type of x / out in the calls that follow; call once per type that will be used.
+ * After it, kvq_encode, kvq_decode, kvq_append[_at], kvq_flush_block[_at] and kvq_calibrate_lambda on
+ * this plan and type make no CUDA call besides their kernel launches (kvq_calibrate_lambda: and one
+ * cudaMemsetAsync) and a query of the current device: nothing allocates, nothing blocks, and the
+ * calls can be recorded into a CUDA graph without a warm call first.  Call it again after
+ * kvq_plan_set_rotation (a rotated D = 256 plan decodes with another kernel).  Idempotent.
+ * Errors: INVALID_ARG (null plan, unknown dtype, plan already bound to another device), NOMEM, CUDA
+ * (no device: arguments are checked first).
+ */
+kvq_status_t kvq_plan_prepare(kvq_plan_t *plan, kvq_dtype_t dtype);
+
+/*
+ * kvq_plan_set_wait_limit -- how long the tensor-core encode kernel (D <= 160) lets its first wait run.
+ * Every device-side wait in the library is bounded (about 2^22 polls, seconds of wall time) and ends in
+ * a status bit instead of a hang.  This knob shortens ONE of them, the wait of the role that issues the
+ * tensor-core instructions for the kernel's first operand build, a point at which that role has
+ * nothing in flight: with a limit of a few polls the launch gives up at once, writes nothing, frees
+ * what it holds and raises bit 2 of the status word, so that an integration can see KVQ_ERR_TIMEOUT
+ * reported and cleared without a fault.
+ *   polls   0 restores the default.  Takes effect for later kvq_encode / kvq_append calls on this plan.
+ */
+kvq_status_t kvq_plan_set_wait_limit(kvq_plan_t *plan, uint32_t polls);
+
 /* Synchronizes the current device and returns the plan's device status word through *word
  * (host): 0 when no kernel using this plan ever gave up a bounded wait or left its number
  * range.  Bits 0-2: a bounded wait ran out (load, tensor-core commit, pipeline slot): returns
@@ -168,7 +198,7 @@ kvq_status_t kvq_encode(kvq_plan_t *plan, const void *x, kvq_dtype_t dtype, int6
                         uint8_t *packed, void *scales, void *cuda_stream);
 
 /*
- * kvq_decode -- inverse path ("unpack, irfft, apply s", Sec. 3.1; lambda clamped at 1e-6,
+ * kvq_decode -- inverse path (Sec. 3.1: Eq. 2 undone, inverse real DFT, signs last; lambda clamped at 1e-6,
  * Sec. 5.1 item 1) on N stored vectors: the per-step full-prefix read.
  *   packed, scales, lambda as in kvq_encode (inputs here);
  *   out      device out, [N, D] row-major, fp16 or bf16 per `dtype` (round to nearest even);
@@ -251,8 +281,8 @@ kvq_status_t kvq_calibrate_lambda(kvq_plan_t *plan, const void *x, kvq_dtype_t d
  * kvq_decode calls cudaMalloc the first time a plan is used on a device (a status word, and the
  * [D, D] fp32 table of the tensor-core kernel).  A server that gave all of HBM to its own pool, a
  * decode loop that cannot take cudaMalloc's device-wide synchronisation, or a plug-in restricted to
- * the buffers it was handed cannot make that call.  This variant runs the same tensor-core kernel
- * with those two objects in a fixed 65,792-byte block that is part of the library image (every GPU
+ * the buffers it was handed cannot make that call.  This variant runs the D = 128 fp16 tensor-core kernel in its dense
+ * 128 x 128 form (kvq_decode takes one radix-2 step out of it) with those two objects in a fixed 65,792-byte block that is part of the library image (every GPU
  * context that loads the library holds it until the process exits).  It calls no cudaMalloc,
  * cudaFree or other allocating routine, on any call.
  *
@@ -265,7 +295,11 @@ kvq_status_t kvq_calibrate_lambda(kvq_plan_t *plan, const void *x, kvq_dtype_t d
  *                inside the block, where this library version does not expose it.
  *
  * The first call on a device looks up the block's device address; make that call before any
- * stream capture begins.  The block is shared: it keeps the last call's table, which belongs to
+ * stream capture begins.  A call made while its stream is being captured records the table
+ * fill in front of the decode every time, so a replayed graph never depends on what other
+ * calls left in the block; and since a replay changes the block behind the host's back, every
+ * call on that device after the first captured one refills the table too (a few microseconds).  N must be below 2^31 (INVALID_ARG otherwise, before anything is
+ * enqueued).  The block is shared: it keeps the last call's table, which belongs to
  * one plan, and a call with a different plan rewrites it on the caller's stream before decoding.
  * Calls that can overlap on the GPU (different streams, no ordering between them) race on the
  * block and on the table: order them, or use kvq_decode.

@@ -19,7 +19,7 @@
  *     q_c = clamp(rint(v_c / sigma_j), -7, 7)       round half to even
  *     byte_i = (q_{2i+1} << 4) | (q_{2i} & 0xF)     nibble pack (Sec. 3.2)
  *
- *   inverse  (Sec. 3.1 "unpack, irfft, apply s"; Sec. 5.1 item 1 for the clamp)
+ *   inverse  (Sec. 3.1: undo the packing of Eq. 2, inverse real DFT, signs last; Sec. 5.1 item 1 for the clamp)
  *     q -> v^ = q sigma_j -> z^ = v^ / max(lambda_c, 1e-6)
  *     Y^ from z^ by undoing Eq. 2, u = unitary inverse real DFT, x^ = s (.) u
  *
@@ -151,8 +151,8 @@ static uint16_t narrow(double v, int dtype)
 }
 
 /* ------------------------------------------------------------------ */
-/* sign diagonal (Sec. 3.1: "a fixed random sign vector drawn at       */
-/* initialization"; the generator itself is this build's reading)      */
+/* sign diagonal (Sec. 3.1: one +-1 per coordinate, drawn once when    */
+/* the plan is made; the generator itself is this build's reading)     */
 /* ------------------------------------------------------------------ */
 
 uint64_t kvqo_splitmix64_mix(uint64_t z)

@@ -40,7 +40,7 @@ KVQ_IMPL_MATVEC = 3
 # every symbol include/kvq.h declares
 EXPORTS = (
     "kvq_plan_create", "kvq_plan_create_ex", "kvq_plan_set_rotation", "kvq_plan_clear_device_status", "kvq_plan_destroy", "kvq_plan_get_signs", "kvq_plan_describe", "kvq_plan_set_impl",
-    "kvq_plan_device_status", "kvq_encode", "kvq_decode", "kvq_append", "kvq_decode_static", "kvq_calibrate_lambda", "kvq_flush_block", "kvq_append_at", "kvq_flush_block_at",
+    "kvq_plan_device_status", "kvq_plan_prepare", "kvq_plan_set_wait_limit", "kvq_encode", "kvq_decode", "kvq_append", "kvq_decode_static", "kvq_calibrate_lambda", "kvq_flush_block", "kvq_append_at", "kvq_flush_block_at",
     "kvq_status_string",
     "kvq_launch_count",
 )
@@ -79,6 +79,10 @@ def lib() -> ctypes.CDLL:
         L.kvq_plan_describe.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_size_t)]
         L.kvq_plan_set_impl.restype = i32
         L.kvq_plan_set_impl.argtypes = [vp, i32, i32]
+        L.kvq_plan_prepare.restype = i32
+        L.kvq_plan_prepare.argtypes = [vp, i32]
+        L.kvq_plan_set_wait_limit.restype = i32
+        L.kvq_plan_set_wait_limit.argtypes = [vp, ctypes.c_uint32]
         L.kvq_plan_device_status.restype = i32
         L.kvq_plan_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
         L.kvq_encode.restype = i32
@@ -233,6 +237,19 @@ def kvq_plan_device_status(plan: int) -> int:
     return int(w.value)
 
 
+def kvq_plan_prepare(plan: int, dtype: torch.dtype, device=None) -> None:
+    """Allocates the plan's device tables and sets every kernel's launch attributes now, on ``device`` (default: the
+    current one), so that later calls with tensors of ``dtype`` allocate nothing and never block."""
+    code = KVQ_F16 if dtype == torch.float16 else KVQ_BF16 if dtype == torch.bfloat16 else -1
+    dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+    with _on_device(dev):
+        _check(lib().kvq_plan_prepare(plan, code), "kvq_plan_prepare")
+
+
+def kvq_plan_set_wait_limit(plan: int, polls: int) -> None:
+    _check(lib().kvq_plan_set_wait_limit(plan, polls), "kvq_plan_set_wait_limit")
+
+
 def kvq_plan_clear_device_status(plan: int) -> None:
     _check(lib().kvq_plan_clear_device_status(plan), "kvq_plan_clear_device_status")
 
@@ -356,6 +373,10 @@ class Plan:
 
     def set_rotation(self, R) -> None:
         kvq_plan_set_rotation(self.handle, R, self.D)
+
+    def describe(self):
+        """(radices of the length-D/2 complex FFT, bytes of device tables the plan holds: 0 until its first use on a device)"""
+        return kvq_plan_describe(self.handle)
 
     def close(self):
         if getattr(self, "handle", None):

@@ -142,6 +142,41 @@ static kvq_status_t ensure_device(kvq_plan *p)
         p->d_e0 = de;
         p->table_bytes += 2 * bytes;
     }
+    if (p->D == 256) {   // the radix-2 encode kernel's B operand, one image per input type, from the table without a rotation
+        std::vector<float> b0, e0;
+        std::vector<unsigned char> img;
+        unsigned char *dr = nullptr;
+        double *rot = p->rot;
+        const float tmax = p->table_max;
+        p->rot = nullptr;
+        bool ok = make_tables(p, b0, e0);
+        const float lift = r2_encode_lift(p->table_max);
+        p->rot = rot;
+        p->table_max = tmax;
+        if (ok) {
+            try {
+                img.resize(2 * (size_t)kR2ImageBytes);
+            } catch (...) {
+                ok = false;
+            }
+        }
+        if (ok) {
+            r2_encode_b_image(e0.data(), lift, false, img.data());
+            r2_encode_b_image(e0.data(), lift, true, img.data() + kR2ImageBytes);
+            ok = cudaMalloc(&dr, img.size()) == cudaSuccess && cudaMemcpy(dr, img.data(), img.size(), cudaMemcpyHostToDevice) == cudaSuccess;
+        }
+        if (!ok) {
+            (void)cudaGetLastError();
+            if (dr) cudaFree(dr);
+            if (p->d_b0) cudaFree(p->d_b0);
+            if (p->d_e0) cudaFree(p->d_e0);
+            cudaFree(st);
+            p->d_status = nullptr, p->d_b0 = nullptr, p->d_e0 = nullptr;
+            return KVQ_ERR_NOMEM;
+        }
+        p->d_r2 = dr;
+        p->table_bytes += img.size();
+    }
     p->device = dev;
     return KVQ_OK;
 }
@@ -182,6 +217,7 @@ static void fill_params(const kvq_plan *p, FftParams &prm, int64_t N, const floa
     prm.in_map = RowMap{1, 1, 0};
     prm.status = p->d_status;
     prm.table_max = p->table_max;
+    prm.first_wait_polls = p->first_wait_polls;
     prm.bits = p->bits;
     std::memcpy(prm.sign_xor, p->sign_xor, sizeof(prm.sign_xor));
 }
@@ -209,9 +245,11 @@ kvq_status_t kvq_plan_create_ex(int D, int group, int bits, uint64_t seed, kvq_p
     p->d_status = nullptr;
     p->d_b0 = nullptr;
     p->d_e0 = nullptr;
+    p->d_r2 = nullptr;
     p->table_bytes = 0;
     p->rot = nullptr;
     p->table_max = (float)std::sqrt(2.0 / D);
+    p->first_wait_polls = 0;
     std::memset(p->signs, 0, sizeof(p->signs));
     std::memset(p->sign_xor, 0, sizeof(p->sign_xor));
     for (int n = 0; n < D; ++n) {
@@ -234,6 +272,9 @@ kvq_status_t kvq_plan_destroy(kvq_plan_t *plan)
     }
     if (plan->d_e0) {
         if (cudaFree(plan->d_e0) != cudaSuccess) (void)cudaGetLastError();
+    }
+    if (plan->d_r2) {
+        if (cudaFree(plan->d_r2) != cudaSuccess) (void)cudaGetLastError();
     }
     delete[] plan->rot;
     delete plan;
@@ -309,6 +350,54 @@ kvq_status_t kvq_plan_set_impl(kvq_plan_t *plan, kvq_impl_t encode_impl, kvq_imp
     return KVQ_OK;
 }
 
+kvq_status_t kvq_plan_set_wait_limit(kvq_plan_t *plan, uint32_t polls)
+{
+    if (!plan) return KVQ_ERR_INVALID_ARG;
+    plan->first_wait_polls = polls;
+    return KVQ_OK;
+}
+
+// Device tables and launch attributes of every kernel a call with this plan and this 16-bit type can take: each
+// launcher is entered with N = 0, sets its kernel's attributes for the current device and returns before its launch.
+kvq_status_t kvq_plan_prepare(kvq_plan_t *plan, kvq_dtype_t dtype)
+{
+    if (!plan) return KVQ_ERR_INVALID_ARG;
+    if (dtype != KVQ_F16 && dtype != KVQ_BF16) return KVQ_ERR_INVALID_ARG;
+    kvq_status_t st = ensure_device(plan);
+    if (st != KVQ_OK) return st;
+    const bool bf16 = dtype == KVQ_BF16, per_vector = plan->group == plan->D;
+    FftParams prm;
+    fill_params(plan, prm, 0, nullptr, 1, 1);
+    GemmParams g;
+    std::memset(&g, 0, sizeof(g));
+    g.n_lambda = g.rows_per_lambda = 1;
+    g.per_vector = per_vector;
+    g.status = plan->d_status;
+    g.b0 = plan->d_b0;
+    if (plan->d_r2 && !plan->rot) prm.r2_image = plan->d_r2 + (bf16 ? kR2ImageBytes : 0);
+    cudaError_t e = cudaSuccess;
+    auto also = [&e](cudaError_t r) {
+        if (e == cudaSuccess) e = r;
+    };
+    if (gemm_encode_ok(plan, bf16)) also(umma_encode(plan->D, bf16, per_vector, 0, prm, plan->d_e0, nullptr));
+    if (gemm_decode_ok(plan, bf16))
+        also(plan->rot && plan->D == 256 ? umma_decode_d256_dense(bf16, 0, g, nullptr)
+                                         : umma_decode(plan->D, bf16, plan->bits, 0, g, plan->sign_xor, nullptr, !plan->rot));
+    if (umma_calibrate_supported(plan->D, bf16)) also(umma_calibrate(plan->D, bf16, 0, prm, plan->d_e0, nullptr, nullptr));
+    also(matvec_encode(plan->D, plan->group, plan->bits, bf16, 0, prm, plan->d_b0, nullptr));
+    also(matvec_decode(plan->D, plan->group, plan->bits, bf16, 0, prm, plan->d_e0, nullptr));
+    also(matvec_flush(plan->D, plan->group, plan->bits, bf16, 0, prm, plan->d_b0, plan->d_e0, nullptr));
+    if (!plan->rot) {
+        also(fft_encode(plan->D, plan->group, plan->bits, bf16, 0, prm, nullptr));
+        also(fft_decode(plan->D, plan->group, plan->bits, bf16, 0, prm, nullptr));
+    }
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        return KVQ_ERR_CUDA;
+    }
+    return KVQ_OK;
+}
+
 kvq_status_t kvq_plan_device_status(kvq_plan_t *plan, uint32_t *word)
 {
     if (!plan || !word) return KVQ_ERR_INVALID_ARG;
@@ -374,6 +463,7 @@ static kvq_status_t encode_common(kvq_plan_t *plan, const void *x, kvq_dtype_t d
     prm.packed = packed;
     prm.scales = scales;
     prm.out_map = out_map;
+    if (plan->d_r2 && !plan->rot) prm.r2_image = plan->d_r2 + (bf16 ? kR2ImageBytes : 0);
     // AUTO: the matrix-vector kernel for small calls (latency), beyond that the tensor-core kernel (measured faster than
     // the register FFT at every size above the matrix-vector limit), the register FFT where no tensor-core kernel is
     // built.  A rotated plan has no FFT path: matrix-vector wherever the tensor-core kernel does not apply.

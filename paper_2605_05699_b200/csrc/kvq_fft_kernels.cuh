@@ -225,7 +225,7 @@ __device__ __forceinline__ void encode_row(const uint4 *__restrict__ row, const 
 }
 
 // ------------------------------------------------------------------------------------------
-// inverse path of one row (Sec. 3.1: "unpack, irfft, apply s"; 1 / max(lambda, 1e-6) of Sec. 5.1)
+// inverse path of one row (Sec. 3.1: Eq. 2 undone, inverse real DFT, signs last; 1 / max(lambda, 1e-6) of Sec. 5.1)
 //   row      this lane's D BITS / 8 code bytes in shared memory
 //   sig      this row's D/GRP scales, already widened
 //   rl       1 / max(lambda, 1e-6) in shared memory (warp-shared)
@@ -559,6 +559,7 @@ static cudaError_t launch_persistent(Kern kern, int warps, size_t smem, int64_t 
         *cached_blocks_per_sm = nb;
         *cached_sms = sms;
     }
+    if (N == 0) return cudaSuccess;   // kvq_plan_prepare: the launch attributes are set, there is nothing to run
     const int64_t tiles = (N + 31) / 32;
     const int64_t want = (tiles + warps - 1) / warps;
     const int64_t cap = (int64_t)(*cached_blocks_per_sm) * (*cached_sms);

@@ -304,7 +304,7 @@ __global__ void __launch_bounds__(kWarps * 32) kvq_encode_matvec_kernel(const __
 }
 
 // ------------------------------------------------------------------------------------------------
-// decode: codes and scales -> x^  (Sec. 3.1 "unpack, irfft, apply s"; 1 / max(lambda, 1e-6) of Sec. 5.1)
+// decode: codes and scales -> x^  (Sec. 3.1: Eq. 2 undone, inverse real DFT, signs last; 1 / max(lambda, 1e-6) of Sec. 5.1)
 // ------------------------------------------------------------------------------------------------
 template <int D, bool BF16>
 __device__ __forceinline__ void decode_batch(const MatvecParams &prm, float4 (&t)[Geo<D>::CH][Geo<D>::P], float *zs, float *red, int warp,
@@ -393,6 +393,7 @@ cudaError_t launch(const MatvecParams &prm, cudaStream_t stream)
         if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kWarps * 32, Geo<D>::kSmemBytes)) != cudaSuccess) return e;
         slots.sms[dev] = sms * (per_sm > 0 ? per_sm : 1);
     }
+    if (prm.N == 0) return cudaSuccess;   // kvq_plan_prepare: the launch attributes are set, there is nothing to run
     const int64_t batches = (prm.N + kV - 1) / kV;
     if (batches > 0x7FFFFFFF) return cudaErrorInvalidValue;
     // one resident wave of CTAs that loop over batches where the kernel does; else a CTA per batch

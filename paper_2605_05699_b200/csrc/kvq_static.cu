@@ -6,11 +6,17 @@
 // to its own pool at start-up (cudaMalloc then fails), a latency-critical decode loop (cudaMalloc
 // synchronises the whole device), a plug-in that is only allowed to touch memory it was given.
 // For them this file keeps the same two objects in one fixed block of device memory that is part
-// of the library image, and runs the same D = 128 fp16 tensor-core kernel on it.
+// of the library image, and runs the D = 128 fp16 tensor-core kernel on it (the dense 128 x 128 form; kvq_decode
+// takes one radix-2 step out of it on plans without a rotation).
 //
 // The block is shared by every call on a device and keeps what the last call left in it:
 //   - the table belongs to ONE plan at a time; a call with another plan rewrites it first, with a
 //     small kernel on the caller's stream;
+//   - a call made while its stream is being captured always records that rewrite in front of the
+//     decode and leaves the host's note of "whose table is in the block" alone: what the block holds
+//     when the graph is replayed is not known at capture time.  A replay rewrites the table without
+//     the host seeing it, so once a call has been captured on a device every later call there,
+//     captured or not, rewrites the table first (a 128-CTA kernel of a few microseconds);
 //   - the status word is cleared on the caller's stream before every launch;
 //   - two calls that overlap on the GPU (different streams, no ordering between them) race on the
 //     block.  Serialise them, or use kvq_decode.
@@ -52,6 +58,7 @@ __global__ void kvq_static_fill_kernel(float *table, int D, const __grid_constan
 struct DeviceSlot {
     float *block = nullptr;   // device address of kvq_static_scratch on this device
     bool table_valid = false;
+    bool replays_possible = false;   // a call was recorded into a graph: replays rewrite the table when the host is not looking
     int table_D = 0;
     uint64_t table_seed = 0;
 };
@@ -74,6 +81,7 @@ extern "C" kvq_status_t kvq_decode_static(kvq_plan_t *plan, const uint8_t *packe
     if (plan->D != 128 || dtype != KVQ_F16 || plan->group != 32 || plan->bits != 4 || plan->rot)
         return KVQ_ERR_UNSUPPORTED_DIM;   // the kernel behind it: D = 128, fp16, groups of 32, 4-bit codes, no rotation
     if (N == 0) return KVQ_OK;
+    if (N >= ((int64_t)1 << 31)) return KVQ_ERR_INVALID_ARG;   // the kernel addresses rows through 32-bit tensor-map coordinates
     if (!packed || !scales || !out || !lambda || n_lambda < 1) return KVQ_ERR_INVALID_ARG;
     if (n_lambda > 1) {
         if (rows_per_lambda < 1) return KVQ_ERR_INVALID_ARG;
@@ -105,16 +113,27 @@ extern "C" kvq_status_t kvq_decode_static(kvq_plan_t *plan, const uint8_t *packe
     uint32_t *own_status = reinterpret_cast<uint32_t *>(slot.block + kTableFloats);
     uint32_t *status = status_word ? status_word : own_status;
 
-    if (!slot.table_valid || slot.table_D != plan->D || slot.table_seed != plan->seed) {
+    // A captured call runs later, possibly many times, after calls this host code never sees in that order: it carries
+    // its own table fill, and the host's note of what the block holds is neither trusted nor updated.
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &cap) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return KVQ_ERR_CUDA;
+    }
+    const bool capturing = cap != cudaStreamCaptureStatusNone;
+    if (capturing) slot.replays_possible = true;   // from now on no eager call on this device can know what the block holds
+    if (capturing || slot.replays_possible || !slot.table_valid || slot.table_D != plan->D || slot.table_seed != plan->seed) {
         SignWords sw;
         for (int i = 0; i < 128; ++i) sw.w[i] = plan->sign_xor[i];
-        slot.table_valid = false;
+        if (!capturing) slot.table_valid = false;
         kvq_static_fill_kernel<<<plan->D, plan->D, 0, stream>>>(table, plan->D, sw);
         count_launch();
         if (cudaGetLastError() != cudaSuccess) return KVQ_ERR_CUDA;
-        slot.table_valid = true;
-        slot.table_D = plan->D;
-        slot.table_seed = plan->seed;
+        if (!capturing) {
+            slot.table_valid = true;
+            slot.table_D = plan->D;
+            slot.table_seed = plan->seed;
+        }
     }
     if (cudaMemsetAsync(status, 0, sizeof(uint32_t), stream) != cudaSuccess) {
         (void)cudaGetLastError();

@@ -115,7 +115,7 @@ __device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&r)[8])
 
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-// TMA tensor load, two coordinates, completion on an mbarrier (never multicast)
+// TMA tensor load, two coordinates, completion on an mbarrier: a per-CTA load of this GPU's own memory
 __device__ __forceinline__ void tma_load_2d(uint32_t dst_smem, const CUtensorMap *tm, int c0, int c1, uint32_t bar)
 {
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
@@ -159,10 +159,12 @@ __device__ __forceinline__ float operand_rescue(const uint32_t (&sc)[(G + 1) / 2
 
 // Bounded wait that also gives up when another role of the CTA has raised the abort flag.  On a
 // time-out it raises the flag itself and records `reason` in the status word.
+constexpr uint32_t kWaitPolls = 1u << 22;   // polls of a bounded wait before it gives up (seconds of wall time)
+
 __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *status,
-                                              uint32_t reason)
+                                              uint32_t reason, uint32_t limit = kWaitPolls)
 {
-    for (uint32_t it = 0; it < (1u << 22); ++it) {
+    for (uint32_t it = 0; it < limit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if (it > 32) {
             if (*abort_flag) return false;
@@ -181,18 +183,16 @@ typedef CUresult (*TensorMapEncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, c
 
 inline TensorMapEncodeTiledFn tensor_map_encode_fn()
 {
-    static TensorMapEncodeTiledFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
+    // looked up once; the initialisation of a function-local static is thread-safe
+    static const TensorMapEncodeTiledFn fn = [] {
         void *p = nullptr;
         cudaDriverEntryPointQueryResult qres;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
             qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<TensorMapEncodeTiledFn>(p);
-        else
-            (void)cudaGetLastError();
-    }
+            return reinterpret_cast<TensorMapEncodeTiledFn>(p);
+        (void)cudaGetLastError();
+        return static_cast<TensorMapEncodeTiledFn>(nullptr);
+    }();
     return fn;
 }
 

@@ -1,7 +1,7 @@
 // Warp-specialised tcgen05 DFT-as-GEMM decode kernel of libkvq (sm_100a): D = 64, 96, 128, 160, fp16 or bf16 output.
 //
-// The inverse path x^ = diag(s) M^T diag(1 / max(lambda, 1e-6)) (q (.) sigma) (Sec. 3.1 "unpack, irfft,
-// apply s"; Sec. 5.1 item 1) is a dense D x D contraction per vector, for any even D (the mixed-radix
+// The inverse path x^ = diag(s) M^T diag(1 / max(lambda, 1e-6)) (q (.) sigma) (Sec. 3.1: the packing of
+// Eq. 2 undone, inverse real DFT, signs last; Sec. 5.1 item 1) is a dense D x D contraction per vector, for any even D (the mixed-radix
 // head dims need no special case here).  A tile of 128 vectors is one 128 x D x D GEMM on the
 // 5th-generation tensor core, a fraction of the time the tile's bytes need to cross HBM, so the kernel's
 // job is to keep HBM busy: one persistent CTA per SM runs four roles that hand tiles to one another
@@ -731,6 +731,7 @@ cudaError_t launch(int64_t N, const GemmParams &g, cudaStream_t stream, const ui
         sms = n;
     }
     if (!tensor_map_encode_fn()) return cudaErrorNotSupported;
+    if (N == 0) return cudaSuccess;   // kvq_plan_prepare: the launch attributes are set, there is nothing to run
     if (N >= (int64_t)1 << 31) return cudaErrorInvalidValue;   // tensor-map coordinates are 32-bit
 
     UmmaDecodeParams prm;

@@ -482,6 +482,7 @@ cudaError_t launch(int64_t N, const GemmParams &g, cudaStream_t stream)
         sms = n;
     }
     if (!tensor_map_encode_fn()) return cudaErrorNotSupported;
+    if (N == 0) return cudaSuccess;   // kvq_plan_prepare: the launch attributes are set, there is nothing to run
     if (N >= (int64_t)1 << 31) return cudaErrorInvalidValue;   // tensor-map coordinates are 32-bit
 
     UmmaDecode256DenseParams prm;

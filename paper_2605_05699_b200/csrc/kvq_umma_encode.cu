@@ -178,6 +178,19 @@ struct FirstRows {
     }
 };
 
+// The mma role's wait for the CTA's first B operand: the one wait whose limit the host may shorten
+// (kvq_plan_set_wait_limit), because the waiting thread has issued nothing yet and can leave at once.  A shortened limit
+// counts looks at the barrier that do not block, so that "one poll" is over before the operand can possibly be there.
+__device__ __forceinline__ bool wait_first_operand(uint32_t bar, volatile uint32_t *abort_flag, uint32_t *status, uint32_t limit)
+{
+    if (limit >= kWaitPolls) return wait_or_abort(bar, 0u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT);
+    for (uint32_t it = 0; it < limit; ++it)
+        if (mbar_test_wait(bar, 0u)) return true;
+    *abort_flag = 1u;
+    atomicOr(status, (uint32_t)KVQ_DEV_SLOT_TIMEOUT);
+    return false;
+}
+
 }  // namespace
 
 struct UmmaEncodeParams {
@@ -194,6 +207,7 @@ struct UmmaEncodeParams {
     int bits;              // 4: nibble pairs; 8: one two's-complement byte per code, scale = absmax / 127
     uint32_t *status;
     uint32_t *amax_bits;        // calibration only: [D] running column maxima as fp32 bit patterns (start at zero)
+    uint32_t first_wait_polls;  // polls the mma role gives the first B build before it gives up (kvq_plan_set_wait_limit)
 };
 
 // PERVEC: one scale per vector (group = D; Sec. 3.2 step 3, Sec. 4.1) instead of one per 32 channels.
@@ -263,11 +277,11 @@ __global__ void __launch_bounds__(kThreads, 1)
     const uint32_t tmem_base = ctrl->tmem_base;
     volatile uint32_t *abort_flag = &ctrl->abort;
     uint32_t *status = prm.status;
+    int issued = 0;   // producer thread: x tiles whose loads have been issued
 
     if (warp == 0) {
         // =========================== producer ===========================
         if (lane == 0) {
-            int issued = 0;
             bool ok = true;
             TileCursor cur(tile_begin, tps);
             for (int j = 0; j < n_my; ++j, cur.advance(1)) {
@@ -310,7 +324,8 @@ __global__ void __launch_bounds__(kThreads, 1)
             for (int j = 0; j < n_my; ++j, cur.advance(1)) {
                 const int s = j % kInStages, sc = j % kAccStages;
                 if (j == 0) {   // all epilogue warps build the first B while the first x tiles are in flight
-                    if (!wait_or_abort(smem_u32(&ctrl->b_first), 0u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT)) break;
+                    // (this thread has issued nothing yet: the one wait whose limit the host may shorten, to see a time-out reported)
+                    if (!wait_first_operand(smem_u32(&ctrl->b_first), abort_flag, status, prm.first_wait_polls)) break;
                 } else if (cur.first_of_segment()) {   // an epilogue set rebuilds B for this lambda row
                     if (!wait_or_abort(smem_u32(&ctrl->b_ready), builds & 1u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT)) break;
                     ++builds;
@@ -514,7 +529,16 @@ __global__ void __launch_bounds__(kThreads, 1)
     tc_fence_before();
     __syncthreads();
     if (warp == 0) {
-        if (*abort_flag) __nanosleep(20000);   // let tensor-core work that was already issued drain
+        if (*abort_flag) {
+            // Every role has left its loop.  The x tiles whose loads are still in flight were this thread's to issue: give
+            // each a bounded chance to land (nobody else may have waited for them), then let tensor-core work that was
+            // already issued drain, before the shared and tensor memory go back.
+            if (lane == 0)
+                for (int j = issued > kInStages ? issued - kInStages : 0; j < issued; ++j)
+                    (void)mbar_wait_bounded(smem_u32(&ctrl->in_full[j % kInStages]), (uint32_t)(j / kInStages) & 1u, 1u << 16);
+            __nanosleep(20000);
+            __syncwarp();
+        }
         tmem_dealloc(tmem_base, kTmemCols);
     }
 }
@@ -539,6 +563,7 @@ cudaError_t launch(int64_t N, const FftParams &f, const float *e0, cudaStream_t 
         if ((e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
         sms = n;
     }
+    if (N == 0) return cudaSuccess;   // kvq_plan_prepare: the launch attributes are set, there is nothing to run
     if (N >= (int64_t)1 << 31) return cudaErrorInvalidValue;   // tensor-map coordinates are 32-bit
 
     UmmaEncodeParams prm;
@@ -555,6 +580,7 @@ cudaError_t launch(int64_t N, const FftParams &f, const float *e0, cudaStream_t 
     prm.bits = f.bits;
     prm.status = f.status;
     prm.amax_bits = amax_bits;
+    prm.first_wait_polls = f.first_wait_polls ? f.first_wait_polls : kWaitPolls;
 
     CUtensorMap tm_x;
     const cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)N};

@@ -520,6 +520,30 @@ cudaError_t launch(int64_t N, const FftParams &f, const float *e0, cudaStream_t 
         if ((e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
         sms = n;
     }
+    // one scale per vector: the pair is a cluster of two CTAs, as many pairs as the device holds at once (SMs of a
+    // cluster share a GPC); looked up once per device
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    if constexpr (PERVEC) {
+        cfg.gridDim = dim3((unsigned)sms, 1, 1);
+        cfg.blockDim = dim3(kThreads, 1, 1);
+        cfg.dynamicSmemBytes = C::kSmemBytes;
+        cfg.stream = stream;
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int &fit = slots.blocks_per_sm[dev];
+        if (fit == 0) {
+            int n = 0;
+            if ((e = cudaOccupancyMaxActiveClusters(&n, kern, &cfg)) != cudaSuccess) return e;
+            if (n < 1) return cudaErrorLaunchOutOfResources;
+            fit = n;
+        }
+    }
+    if (N == 0) return cudaSuccess;   // kvq_plan_prepare: the launch attributes are set, there is nothing to run
     if (N >= (int64_t)1 << 31) return cudaErrorInvalidValue;   // tensor-map coordinates are 32-bit
 
     UmmaEncode256Params prm;
@@ -547,26 +571,7 @@ cudaError_t launch(int64_t N, const FftParams &f, const float *e0, cudaStream_t 
     const int64_t tiles = prm.n_seg * ((prm.rpl + kTile - 1) / kTile);
     int64_t pairs = tiles < sms / 2 ? tiles : sms / 2;
     if constexpr (PERVEC) {
-        // the pair is a cluster of two CTAs: as many pairs as the device holds at once (SMs of a cluster share a GPC)
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)sms, 1, 1);
-        cfg.blockDim = dim3(kThreads, 1, 1);
-        cfg.dynamicSmemBytes = C::kSmemBytes;
-        cfg.stream = stream;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = 2;
-        attr[0].val.clusterDim.y = 1;
-        attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        int &fit = slots.blocks_per_sm[dev];   // clusters resident at once, looked up once per device
-        if (fit == 0) {
-            int n = 0;
-            if ((e = cudaOccupancyMaxActiveClusters(&n, kern, &cfg)) != cudaSuccess) return e;
-            if (n < 1) return cudaErrorLaunchOutOfResources;
-            fit = n;
-        }
+        const int fit = slots.blocks_per_sm[dev];   // clusters resident at once
         if (pairs > fit) pairs = fit;
         cfg.gridDim = dim3((unsigned)(2 * pairs), 1, 1);
         e = cudaLaunchKernelEx(&cfg, kern, prm, tm_x);
@@ -584,6 +589,7 @@ cudaError_t umma_encode_d256(bool bf16, bool per_vector, int64_t N, const FftPar
 {
     if (!tensor_map_encode_fn()) return cudaErrorNotSupported;
     if (per_vector) return bf16 ? launch<true, false, true>(N, f, e0, stream) : launch<false, false, true>(N, f, e0, stream);
+    if (f.r2_image && f.bits == 4) return umma_encode_d256_r2(bf16, N, f, stream);   // no rotation: half the tensor work, one CTA per tile
     return bf16 ? launch<true>(N, f, e0, stream) : launch<false>(N, f, e0, stream);
 }
 

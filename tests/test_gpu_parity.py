@@ -295,7 +295,7 @@ def test_config4_mixed_radix(D, impl):
 
 def test_config2_qwen_shaped_prefill_append_decode():
     shp = wl.QWEN25_1P5B
-    D, T0, steps = shp.head_dim, shp.prefix, 4
+    D, T0, steps = shp.head_dim, shp.prefix, 128      # the configuration's 128 decode steps
     S = shp.streams  # 112 streams: (layer, K/V, head)
     T_max = T0 + steps
     per_lambda = shp.kv_heads  # one lambda row per (layer, K/V): 56 rows
@@ -346,11 +346,17 @@ def test_append_touches_only_row_pos():
     torch.cuda.synchronize()
     keep = [t for t in range(T) if t != 4]
     assert bool((packed[:, keep] == 0xAB).all()) and bool((scales[:, keep] == 1.25).all())
+    # the oracle's append leaves the same rows alone and writes, at row 4, what its encode of the 37 vectors gives
     pc = np.full((S, T, D // 2), 0xAB, dtype=np.uint8)
     sc = np.full((S, T, D // G), np.float16(1.25).view(np.uint16), dtype=np.uint16)
     ko.append(bits(x), ko.F16, plan.signs(), lam.cpu().numpy(), G, pc, sc, 4, 1)
-    assert (packed.cpu().numpy() == pc).mean() > 0.999
-    assert np.abs(bits(scales).astype(np.int64) - sc.astype(np.int64)).max() <= 1
+    assert (pc[:, keep] == 0xAB).all() and (sc[:, keep] == np.float16(1.25).view(np.uint16)).all()
+    ora = ko.encode(bits(x), ko.F16, plan.signs(), lam.cpu().numpy(), G, 1, want_v=True)
+    assert np.array_equal(pc[:, 4], ora["packed"]) and np.array_equal(sc[:, 4], ora["scales"])
+    # and the library's row 4 against it, under the code, tie and scale rules (4736 codes: one mismatch at a tie would
+    # already be 2e-4 of them, so the share rule of the sampled tests applies; in practice they are identical)
+    enc = parity.check_encode(packed[:, 4].contiguous().cpu().numpy(), bits(scales[:, 4].contiguous()), ora, G, "append row", min_agree=0.9995)
+    assert enc["mismatches"] <= 1
     plan.close()
 
 
@@ -918,7 +924,12 @@ def test_degenerate_lambda(D, dtype, impl, wild):
     sg = plan.signs()
     packed, scales = gpu_encode(plan, x.cuda(), lam.cuda(), 1500)
     ora = ko.encode(bits(x), odt, sg, lam.numpy(), G, 1500, want_v=True)
-    parity.check_encode(packed.cpu().numpy(), bits(scales), ora, G, "odd lambda encode (%s)" % impl)
+    # bf16 input on the tensor cores carries the table in two bf16 terms (16 bits): an error of 1e-5 of the vector's norm in
+    # every coefficient.  The wild row lifts ONE channel 3000 times above its neighbours, so a group's maximum can be a
+    # coefficient near zero seen through that gain, and its stored scale then moves by 2 fp16 ulps (1e-3) in about one
+    # group in 20,000; the 1e-3 relative L2 per vector on the scales holds regardless.
+    ulps = 2 if (wild and impl == "gemm" and dtype == "bf16") else 1
+    parity.check_encode(packed.cpu().numpy(), bits(scales), ora, G, "odd lambda encode (%s)" % impl, max_scale_ulps=ulps)
     ob, o64 = ko.decode(ora["packed"], ora["scales"], sg, lam.numpy(), G, odt, 1500, want_f64=True)
     out = gpu_decode_raw(plan, torch.from_numpy(ora["packed"]).cuda(),
                          torch.from_numpy(ora["scales"].view(np.int16)).view(torch.float16).cuda(), lam.cuda(), dtype, 1500)
@@ -1006,12 +1017,17 @@ def test_row_offsets_beyond_four_gigabytes(impl):
     idx_d = idx.cuda()
     xs, pk, sc, od = x[idx_d].cpu(), packed[idx_d].cpu().numpy(), bits(scales[idx_d]), bits(out[idx_d])
     lrow = (idx // rpl).numpy()
+    mismatches = codes = 0
     for l in np.unique(lrow):
         m = lrow == l
         ora = ko.encode(bits(xs)[m], ko.F16, sg, lam.numpy()[l], G, want_v=True)
-        parity.check_encode(pk[m], sc[m], ora, G, "rows past 4 GB, encode, lambda row %d" % l, min_agree=0.9995)
+        # per lambda row: ties, scales, byte layout; the 99.99 % rule is applied to the whole sample below
+        enc = parity.check_encode(pk[m], sc[m], ora, G, "rows past 4 GB, encode, lambda row %d" % l, min_agree=0.9995)
+        mismatches += enc["mismatches"]
+        codes += enc["codes"]
         ob, o64 = ko.decode(pk[m], sc[m], sg, lam.numpy()[l], G, ko.F16, want_f64=True)
         parity.check_decode(od[m], ob, o64, ko.F16, "rows past 4 GB, decode, lambda row %d" % l)
+    assert mismatches <= (1.0 - parity.CODE_AGREEMENT) * codes, "only %.6f of the sampled codes agree" % (1.0 - mismatches / codes)
     plan.close()
 
 
@@ -1033,6 +1049,8 @@ def _full_size_sampled(D, dtype, N, kind, seed, n_lambda, rows_per_lambda, n_ran
     lrow = (idx // rows_per_lambda).numpy() if n_lambda > 1 else np.zeros(len(idx), dtype=np.int64)
     xs, pk, sc, od = x[idx_d].cpu(), packed[idx_d].cpu().numpy(), bits(scales[idx_d]), bits(out[idx_d])
     mismatches = codes = 0
+    tie_rows = n_rows = 0.0
+    worst = 0.0
     for l in np.unique(lrow):
         m = lrow == l
         ora = ko.encode(bits(xs)[m], DT[dtype], sg, lam_h[l], G, want_v=True)
@@ -1042,8 +1060,15 @@ def _full_size_sampled(D, dtype, N, kind, seed, n_lambda, rows_per_lambda, n_ran
         mismatches += enc["mismatches"]
         codes += enc["codes"]
         ob, o64 = ko.decode(pk[m], sc[m], sg, lam_h[l], G, DT[dtype], want_f64=True)
-        parity.check_decode(od[m], ob, o64, DT[dtype], "full-size decode lambda row %d" % l)
+        dec = parity.check_decode(od[m], ob, o64, DT[dtype], "full-size decode lambda row %d" % l)
+        tie_rows += dec["rows_needing_tie_rule"] * int(m.sum())
+        n_rows += int(m.sum())
+        worst = max(worst, dec["rel_l2_plain_max"])
     assert mismatches <= (1.0 - parity.CODE_AGREEMENT) * codes, "only %.6f of the sampled codes agree" % (1.0 - mismatches / codes)
+    # how much of the decode's agreement rests on the output-rounding tie rule: little (fp16 output: none expected)
+    print("full-size sampled D=%d %s dec=%s: code agreement %.6f, decode rel-L2 max %.3g, rows needing the tie rule %.4f"
+          % (D, dtype, dec_impl, 1.0 - mismatches / codes, worst, tie_rows / n_rows))
+    assert tie_rows / n_rows < (0.001 if dtype == "f16" else 0.02)
     # properties that hold at any size: codes in range everywhere, scales finite and non-negative
     assert bool(torch.isfinite(scales).all()) and bool((scales >= 0).all())
     lo, hi = packed & 0xF, packed >> 4

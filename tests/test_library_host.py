@@ -101,6 +101,21 @@ def test_rotation_is_validated_on_the_host():
     assert torch.allclose(near @ near.T, torch.eye(64), atol=1e-5) and float((near - torch.eye(64)).abs().max()) < 0.5
 
 
+def test_prepare_and_wait_limit_check_their_arguments_before_cuda():
+    L = kb.lib()
+    p = kb.Plan(128, 32, 1)
+    assert L.kvq_plan_prepare(None, kb.KVQ_F16) == kb.KVQ_ERR_INVALID_ARG
+    assert L.kvq_plan_prepare(p.handle, 2) == kb.KVQ_ERR_INVALID_ARG           # dtype
+    assert L.kvq_plan_set_wait_limit(None, 4) == kb.KVQ_ERR_INVALID_ARG
+    assert L.kvq_plan_set_wait_limit(p.handle, 4) == kb.KVQ_OK
+    assert L.kvq_plan_set_wait_limit(p.handle, 0) == kb.KVQ_OK
+    if not torch.cuda.is_available():
+        # valid arguments, no device: the failing CUDA call is reported, nothing is computed on the host
+        assert L.kvq_plan_prepare(p.handle, kb.KVQ_F16) == kb.KVQ_ERR_CUDA
+        assert kb.kvq_plan_describe(p.handle)[1] == 0
+    p.close()
+
+
 def test_bad_arguments_are_rejected_on_the_host():
     L = kb.lib()
     p = kb.Plan(128, 32, 1)
