@@ -2,6 +2,7 @@
 """Benchmark of the fused int4 KV-cache quantizer hot path on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py --op decode --D 256 --dtype bf16 --n 524288 [--family gemm] [--sustain 4]     one kernel, one case
 
 Workload: the Llama-3-70B-shaped cache (80 layers x 8 KV heads x D=128 fp16,
 batch 4, prefix 32768).  One STEP is one pass of the whole hot path over one layer of that cache:
@@ -279,9 +280,16 @@ def run_ours(args):
         return
 
     copy_gbs = measure_sustained_copy(slots, dev)
-    d256 = incr = sweep = None
+    d256 = incr = sweep = c1 = c2 = c4 = sustained = None
     if not args.no_side:
+        # the timed region of a short run (the default of the graded run is 20 steps, 6 ms) never reaches the board's power
+        # cap: the same two kernels back to back for 0.6 s each show the capped regime
+        if ms_total < 500.0:
+            sustained = measure_sustained(kb, wl, dev, slots, plan, lam, rpl)
         d256 = measure_d256(kb, wl, dev)
+        c1 = measure_config1(kb, wl, dev)
+        c2 = measure_config2(kb, wl, dev)
+        c4 = measure_config4(kb, wl, dev)
         incr = measure_incremental(kb, wl, dev, dec_avg_ms=sum(dec_ms) / len(dec_ms))
         sweep = measure_model_sweep(kb, wl, dev, shp.dtype, S, T)
     step_bytes = (2 * N + S) * BYTES_PER_VEC
@@ -297,12 +305,12 @@ def run_ours(args):
     roofline = {"bound": "hbm", "kernel": "kvq_decode_umma_kernel<128, fp16 out, 4-bit, radix-2> (full-prefix read, %d vectors per launch)" % N,
                 "achieved": dec_gbs, "peak": peak, "unit": "GB/s", "frac": dec_gbs / peak,
                 "peak_source": peak_src, "algorithmic_bytes_per_launch": N * BYTES_PER_VEC,
-                "avg_launch_ms": dec_avg, "traffic": TRAFFIC.get("decode"),
+                "avg_launch_ms": dec_avg, "traffic": dram_traffic("decode"), "sustained": sustained,
                 "sustained_copy_GBps": copy_gbs, "frac_of_sustained_copy": dec_gbs / copy_gbs,
                 "sustained_copy_note": "a plain device copy of one layer buffer, back to back for 0.3 s in this run: the same "
                                        "power-capped regime as the timed region (peak above is the driver's burst copy)",
                 "encode": {"kernel": "kvq_encode_umma_kernel<128, fp16 in> (%d vectors per launch)" % N, "achieved": enc_gbs,
-                           "frac": enc_gbs / peak, "avg_launch_ms": enc_avg, "traffic": TRAFFIC.get("encode")}}
+                           "frac": enc_gbs / peak, "avg_launch_ms": enc_avg, "traffic": dram_traffic("encode")}}
     cpu = cpu_baseline_sample(target_seconds=12.0)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -319,13 +327,16 @@ def run_ours(args):
             "prefix_decode_frac_of_hbm_peak": dec_gbs / peak, "prefix_decode_frac_of_8TBps": dec_gbs / 8000.0,
             "append_us": 1e3 * sum(app_ms) / len(app_ms),
             "value_first_%d_steps_GBps" % n_first: n_first * step_bytes / (ms_first * 1e-3) / 1e9,
-            "power_note": "back to back the step runs at the board's 1000 W cap (sw_power_cap) with the SM clock lowered "
-                          "to fit; a plain device copy under the same cap moves 6245 GB/s (profiles/sustained_power_cap)",
+            "power_note": "back to back for more than a few milliseconds the step runs at the board's 1000 W cap (sw_power_cap) "
+                          "with the SM clock lowered to fit; roofline.sustained holds the two kernels in that regime",
             "encode_ms_min": min(enc_ms), "decode_ms_min": min(dec_ms),
             "model_sweep_decode_ms_80_layers": 80 * dec_avg,
             "model_sweep_measured": sweep,
             "paper_context": "paper: 24.6 ns/vec encode at D=128, ~50 ns/vec at D=256 on an Apple M1 GPU (fp32 in, Sec. 7.1)",
             "d256_bf16_gemma_shaped": d256,
+            "config1": c1,
+            "config2_qwen_shaped": c2,
+            "config4": c4,
             "incremental_decode": incr,
         },
         "roofline": roofline,
@@ -359,41 +370,176 @@ def measure_sustained_copy(slots, dev, seconds=0.3):
     return reps * nbytes / (e0.elapsed_time(e1) * 1e-3) / 1e9
 
 
-def measure_d256(kb, wl, dev, iters=10):
-    """Outside the timed region: the Gemma-3-1B-shaped cache (config 3: 26 layers x K,V x 4096 tokens, D=256 bf16) in one
-    encode and one decode launch over all layers (52 lambda rows), device-timed, two buffer sets in rotation."""
+def bytes_per_vector(Dh: int) -> int:
+    return 2 * Dh + Dh // 2 + 2 * (Dh // GROUP)
+
+
+def time_case(kb, wl, dev, Dh, dtype, Nv, kind, n_lambda=1, rpl=0, iters=20, warm=3, cold=False, seed=35):
+    """Device time of one kvq_encode and one kvq_decode launch of Nv vectors (events on the launching stream, one launch
+    per measurement): medians and minima over `iters` launches after `warm`.  cold=False: the same buffers every time (what
+    fits stays in L2).  cold=True: a 256 MB buffer is rewritten before every launch, so nothing of the case is left in L2."""
     import torch
 
-    Dh, T, L = 256, 4096, 52
-    Nv = L * T
-    bpv = 2 * Dh + Dh // 2 + 2 * (Dh // GROUP)
     plan = kb.Plan(Dh, GROUP, 33)
-    lam = wl.make_lambda(L, Dh, 34, device=dev)
-    sets = []
-    for i in range(2):
-        x = wl.make_vectors(Nv, Dh, "bf16", "c1", 35 + i, device=dev)
-        sets.append((x, plan.empty_packed(Nv, dev), plan.empty_scales(Nv, dev), torch.empty_like(x)))
+    lam = wl.make_lambda(n_lambda, Dh, seed - 1, device=dev)
+    x = wl.make_vectors(Nv, Dh, dtype, kind, seed, device=dev)
+    pk, sc, out = plan.empty_packed(Nv, dev), plan.empty_scales(Nv, dev), torch.empty_like(x)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if cold else None
     enc, dec = [], []
-    for i in range(iters + 2):
-        x, pk, sc, out = sets[i % 2]
-        e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+    for i in range(iters + warm):
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        if flush is not None:
+            flush.fill_(i & 255)
         e[0].record()
-        kb.kvq_encode(plan.handle, x, lam, pk, sc, T)
+        kb.kvq_encode(plan.handle, x, lam, pk, sc, rpl)
         e[1].record()
-        kb.kvq_decode(plan.handle, pk, sc, lam, out, T)
+        if flush is not None:
+            flush.fill_((i + 1) & 255)
         e[2].record()
+        kb.kvq_decode(plan.handle, pk, sc, lam, out, rpl)
+        e[3].record()
         torch.cuda.synchronize()
-        if i >= 2:
+        if i >= warm:
             enc.append(e[0].elapsed_time(e[1]))
-            dec.append(e[1].elapsed_time(e[2]))
+            dec.append(e[2].elapsed_time(e[3]))
     assert kb.kvq_plan_device_status(plan.handle) == 0
     plan.close()
-    em, dm = statistics.median(enc), statistics.median(dec)
     peak, _ = measured_peak()
-    return {"vectors": Nv, "bytes_per_vector": bpv, "encode_ns_per_vec": em * 1e6 / Nv, "encode_GBps": Nv * bpv / (em * 1e-3) / 1e9,
-            "decode_ns_per_vec": dm * 1e6 / Nv, "prefix_decode_GBps": Nv * bpv / (dm * 1e-3) / 1e9,
-            "prefix_decode_frac_of_hbm_peak": Nv * bpv / (dm * 1e-3) / 1e9 / peak,
-            "note": "working set 140 MB per launch, about the size of L2: not a roofline number"}
+    bpv = bytes_per_vector(Dh)
+
+    def stats(ms):
+        med, mn = statistics.median(ms), min(ms)
+        return {"us_median": 1e3 * med, "us_min": 1e3 * mn, "ns_per_vec": med * 1e6 / Nv, "GBps": Nv * bpv / (med * 1e-3) / 1e9,
+                "frac_of_hbm_peak": Nv * bpv / (med * 1e-3) / 1e9 / peak}
+
+    return {"encode": stats(enc), "decode": stats(dec)}
+
+
+def hot_and_cold(kb, wl, dev, Dh, dtype, Nv, kind, n_lambda=1, rpl=0, iters=20):
+    bpv = bytes_per_vector(Dh)
+    return {"vectors": Nv, "D": Dh, "io_dtype": dtype, "bytes_per_vector": bpv, "working_set_MB": Nv * bpv / 1e6,
+            "hot_l2": time_case(kb, wl, dev, Dh, dtype, Nv, kind, n_lambda, rpl, iters, cold=False),
+            "cold": time_case(kb, wl, dev, Dh, dtype, Nv, kind, n_lambda, rpl, iters, cold=True)}
+
+
+def measure_config1(kb, wl, dev):
+    """Config 1: one tensor of 4096 x 128 fp16 (1.3 MB in all): a launch-bound size, reported, not held to the roofline."""
+    r = hot_and_cold(kb, wl, dev, 128, "f16", 4096, "c1")
+    r["note"] = "4096 vectors: latency of one launch (the matrix-vector kernels serve calls of this size), not bandwidth"
+    return r
+
+
+def measure_config4(kb, wl, dev):
+    """Config 4: the mixed-radix head dims, 65,536 vectors each, fp16, lognormal channel scales."""
+    return {"D96": hot_and_cold(kb, wl, dev, 96, "f16", 65536, "lognormal"),
+            "D160": hot_and_cold(kb, wl, dev, 160, "f16", 65536, "lognormal"),
+            "note": "16-27 MB per launch: fits L2 when hot; cold = a 256 MB buffer rewritten before every launch"}
+
+
+def measure_config2(kb, wl, dev, steps=128):
+    """Config 2, the Qwen2.5-1.5B-shaped decode loop: 28 layers x 2 KV heads x (K, V) = 112 streams of D=128 fp16, prefix 1024.
+    Prefill encode of all streams in one call, then `steps` decode steps, each one kvq_append of 112 vectors (one launch, a
+    lambda row per (layer, K/V)) and one full-prefix kvq_decode of the whole cache.  Device time per step between events."""
+    import torch
+
+    shp = wl.QWEN25_1P5B
+    Dh, S, T0 = shp.head_dim, shp.streams, shp.prefix
+    T_max = T0 + steps
+    spl = shp.kv_heads
+    plan = kb.Plan(Dh, GROUP, 77)
+    lam = wl.make_lambda(S // spl, Dh, 21, device=dev)
+    x = wl.make_vectors(S * T_max, Dh, shp.dtype, "k_outlier", 500, device=dev).view(S, T_max, Dh)
+    packed = torch.zeros(S, T_max, Dh // 2, dtype=torch.uint8, device=dev)
+    scales = torch.zeros(S, T_max, Dh // GROUP, dtype=torch.float16, device=dev)
+    out = torch.empty(S * T_max, Dh, dtype=torch.float16, device=dev)
+    xs = [x[:, T0 + t].contiguous() for t in range(steps)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    xp = x[:, :T0].contiguous()
+    pp, sp = plan.empty_packed(S * T0, dev), plan.empty_scales(S * T0, dev)
+    for rep in range(3):
+        e0.record()
+        kb.kvq_encode(plan.handle, xp.view(-1, Dh), lam, pp, sp, spl * T0)
+        e1.record()
+        torch.cuda.synchronize()
+    prefill_ms = e0.elapsed_time(e1)
+    packed[:, :T0] = pp.view(S, T0, -1)
+    scales[:, :T0] = sp.view(S, T0, -1)
+    ms = []
+    for t in range(steps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        kb.kvq_append(plan.handle, xs[t], lam, packed, scales, T0 + t, spl)
+        kb.kvq_decode(plan.handle, packed.view(-1, Dh // 2), scales.view(-1, Dh // GROUP), lam, out, spl * T_max)
+        b.record()
+        ms.append((a, b))
+    torch.cuda.synchronize()
+    assert kb.kvq_plan_device_status(plan.handle) == 0
+    plan.close()
+    per = [a.elapsed_time(b) for a, b in ms][3:]
+    peak, _ = measured_peak()
+    bpv = bytes_per_vector(Dh)
+    step_bytes = (S + S * T_max) * bpv
+    med = statistics.median(per)
+    return {"streams": S, "prefix": T0, "steps": steps, "vectors_decoded_per_step": S * T_max,
+            "prefill_encode_us": 1e3 * prefill_ms, "prefill_encode_GBps": S * T0 * bpv / (prefill_ms * 1e-3) / 1e9,
+            "step_us_median": 1e3 * med, "step_us_min": 1e3 * min(per), "step_bytes": step_bytes,
+            "step_us_at_hbm_peak": step_bytes / (peak * 1e9) * 1e6, "step_GBps": step_bytes / (med * 1e-3) / 1e9,
+            "note": "steps queued back to back on one stream; the 42 MB a step touches stay in L2 (hot), so the step is bound by two "
+                    "launches, not by HBM; the whole [112, prefix + steps] cache is decoded every step, rows not yet written included"}
+
+
+def measure_d256(kb, wl, dev):
+    """Config 3, the Gemma-3-1B-shaped cache (26 layers x K,V, D=256 bf16): one encode and one decode launch over all layers
+    (52 lambda rows) at prefix 256 / 1024 / 4096, and a launch of a million vectors that no cache can hold."""
+    L = 2 * wl.GEMMA3_1B.layers
+    res = {}
+    for T in (256, 1024, 4096):
+        res["prefix_%d" % T] = hot_and_cold(kb, wl, dev, 256, "bf16", L * T, "c1", L, T)
+    big = L * 20480                                   # 1,064,960 vectors, 699 MB per launch
+    res["hbm_bound_%d" % big] = {"vectors": big, "working_set_MB": big * bytes_per_vector(256) / 1e6,
+                                 "cold": time_case(kb, wl, dev, 256, "bf16", big, "c1", L, 20480, iters=10, cold=True)}
+    res["note"] = ("prefix sweep: 9-140 MB per launch, at or below the size of L2, and 9-70 us of device time of which 5-8 us are the "
+                   "launch's fixed cost: not roofline numbers; the last entry is the D=256 roofline point")
+    return res
+
+
+def measure_sustained(kb, wl, dev, slots, plan, lam, rpl, seconds=0.6):
+    """Outside the timed region: the step's two large kernels launched back to back for `seconds` each, with the SM clock
+    sampled meanwhile: the power-capped regime that a short timed region never reaches."""
+    import torch
+
+    peak, _ = measured_peak()
+    Nv = slots[0]["x"].shape[0]
+    nbytes = Nv * BYTES_PER_VEC
+    res = {}
+    for name in ("decode", "encode"):
+        def launch(i):
+            sl = slots[i % len(slots)]
+            if name == "decode":
+                kb.kvq_decode(plan.handle, sl["packed"], sl["scales"], lam, sl["out"], rpl)
+            else:
+                kb.kvq_encode(plan.handle, sl["x"], lam, sl["packed"], sl["scales"], rpl)
+        for i in range(3):
+            launch(i)
+        torch.cuda.synchronize()
+        reps = max(100, int(seconds / 1.4e-4))
+        sampler = ClockSampler(dev.index or 0)
+        sampler.start()
+        time.sleep(0.15)
+        w0 = time.time()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(reps):
+            launch(i)
+        e1.record()
+        torch.cuda.synchronize()
+        w1 = time.time()
+        clk = sampler.stop(w0, w1)
+        us = 1e3 * e0.elapsed_time(e1) / reps
+        res[name] = {"launches": reps, "us_per_launch": us, "GBps": nbytes / (us * 1e-6) / 1e9, "frac": nbytes / (us * 1e-6) / 1e9 / peak,
+                     "sm_mhz_median": clk.get("sm_mhz"), "power_w_max": clk.get("power_w_max"), "reasons": clk.get("reasons"),
+                     "us_times_mhz": None if clk.get("sm_mhz") is None else us * clk["sm_mhz"]}
+    return res
 
 
 def measure_model_sweep(kb, wl, dev, dtype, S, T, layers=80, sweeps=5):
@@ -549,10 +695,21 @@ def measure_append_dispatch(kb, wl, dev, dtype, S, layers=80, T=1024, iters=20):
                     "kvq_append_at reads the row from device memory, so the graph is replayed as is for every position"}
 
 
-# DRAM bytes per full launch (2,097,152 vectors, the bench's launch size) from ncu: dram__bytes_read.sum +
-# dram__bytes_write.sum, one-pass capture; see profiles/dram_traffic_d128_n2097152.md.  Reads match the algorithmic
-# bytes; writes are short of them by what is still in the 126 MB L2 when the kernel ends.
-TRAFFIC = {"decode": 151190784 + 476806656, "encode": 538161152 + 128756736}
+def dram_traffic(which: str):
+    """DRAM bytes of one full launch (dram__bytes_read.sum + dram__bytes_write.sum from a one-pass ncu capture of the bench's own
+    launch size), as recorded by `python -m paper_2605_05699_b200.traffic`.  None when there is no record, or when the kernel's
+    source file has changed since the counters were taken."""
+    import hashlib
+
+    try:
+        with open(os.path.join(ROOT, "profiles", "dram_traffic.json")) as f:
+            rec = json.load(f)[which]
+        with open(os.path.join(ROOT, "paper_2605_05699_b200", "csrc", rec["source"]), "rb") as f:
+            if hashlib.sha256(f.read()).hexdigest()[:16] != rec["source_sha16"]:
+                return None
+        return int(rec["dram_bytes_read"]) + int(rec["dram_bytes_write"])
+    except Exception:
+        return None
 
 
 # --------------------------------------------------------------------------------------------
@@ -626,6 +783,101 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+# --------------------------------------------------------------------------------------------
+# one kernel, one case: the command that goes under a profiler, and the back-to-back (power-capped) probe
+# --------------------------------------------------------------------------------------------
+
+FAMILY = {"auto": 0, "fft": 1, "gemm": 2, "matvec": 3}
+
+
+def run_case(args):
+    """`--op encode|decode|append|flush|copy`: runs ONE kernel on one fixed case a few times and prints one JSON line with the
+    CUDA-event time of the last launch (never quote a time taken under a profiler).  With `--sustain SECONDS` the op is
+    launched back to back for that long over three buffer sets, timed in chunks of 200 launches, while nvidia-smi is sampled:
+    the board's power cap bounds the large kernels in steady state (`--op copy` is a plain device copy, the reference)."""
+    import torch
+
+    from paper_2605_05699_b200 import binding as kb
+    from paper_2605_05699_b200 import workloads as wl
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the product path")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    Dh, Nv, fam = args.D, args.n, FAMILY[args.family]
+    n_lambda = max(1, args.n_lambda)
+    rpl = (Nv + n_lambda - 1) // n_lambda if n_lambda > 1 else 0
+    bpv = bytes_per_vector(Dh)
+    plan = kb.Plan(Dh, GROUP, 3)
+    lam = wl.make_lambda(n_lambda, Dh, 12, device=dev)
+    n_sets = 3 if args.sustain > 0 else 1
+    sets = []
+    for i in range(n_sets):
+        x = wl.make_vectors(Nv, Dh, args.dtype, args.kind, 11 + i, device=dev)
+        sets.append((x, plan.empty_packed(Nv, dev), plan.empty_scales(Nv, dev), torch.empty_like(x)))
+    # the compressed input of decode comes from the fp32 register-FFT encoder
+    kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_FFT, fam)
+    for x, pk, sc, out in sets:
+        kb.kvq_encode(plan.handle, x, lam, pk, sc, rpl)
+    kb.kvq_plan_set_impl(plan.handle, fam, fam)
+    torch.cuda.synchronize()
+
+    def launch(i):
+        x, pk, sc, out = sets[i % n_sets]
+        if args.op == "encode":
+            kb.kvq_encode(plan.handle, x, lam, pk, sc, rpl)
+        elif args.op == "decode":
+            kb.kvq_decode(plan.handle, pk, sc, lam, out, rpl)
+        elif args.op == "append":
+            kb.kvq_append(plan.handle, x[:4096], lam[:1], pk.view(4096, -1, Dh // 2), sc.view(4096, -1, Dh // GROUP), 1)
+        elif args.op == "flush":   # the window flush: 64 streams x 16 new tokens into caches of n / 64 rows per stream, one launch
+            kb.kvq_flush_block(plan.handle, x[:1024].view(64, 16, Dh), lam[:1], pk.view(64, -1, Dh // 2), sc.view(64, -1, Dh // GROUP),
+                               out.view(64, -1, Dh), 16)
+        else:
+            out.copy_(sets[(i + 1) % n_sets][0])
+
+    base = {"op": args.op, "D": Dh, "io_dtype": args.dtype, "family": args.family, "n_lambda": n_lambda}
+    if args.sustain > 0:
+        if args.op in ("append", "flush"):
+            raise SystemExit("--sustain takes encode, decode or copy")
+        time.sleep(1.0)
+        sampler = ClockSampler(0)
+        sampler.start()
+        chunks = []
+        w0 = time.time()
+        while time.time() < w0 + args.sustain:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for i in range(200):
+                launch(i)
+            e1.record()
+            torch.cuda.synchronize()
+            chunks.append(1e3 * e0.elapsed_time(e1) / 200)
+        w1 = time.time()
+        clk = sampler.stop(w0 + 0.5 * (w1 - w0), w1)
+        assert kb.kvq_plan_device_status(plan.handle) == 0
+        nbytes = Nv * bpv if args.op != "copy" else 2 * Nv * 2 * Dh
+        tail = sorted(chunks[len(chunks) // 2:])
+        steady = tail[len(tail) // 2]
+        base.update({"n": Nv, "seconds": args.sustain, "us_per_launch_first_chunk": chunks[0], "us_per_launch_steady": steady,
+                     "GBps_steady": nbytes / (steady * 1e-6) / 1e9, "bytes_per_launch": nbytes, "clocks_second_half": clk})
+        print(json.dumps(base))
+        return
+    if args.op == "copy":
+        raise SystemExit("--op copy is for --sustain")
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for i in range(max(1, args.reps)):
+        e0.record()
+        launch(0)
+        e1.record()
+        torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    assert kb.kvq_plan_device_status(plan.handle) == 0
+    n_eff = 4096 if args.op == "append" else 1024 if args.op == "flush" else Nv
+    base.update({"n": n_eff, "ms_last": ms, "ns_per_vec": ms * 1e6 / n_eff, "algorithmic_GBps": n_eff * bpv / (ms * 1e-3) / 1e9})
+    print(json.dumps(base))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -634,7 +886,19 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-side", action="store_true",
                     help="leave out the measurements beside the timed region (D=256, window flush, 80-layer sweep): for a launch list")
+    # one kernel on one case (see run_case): a profiler's command line
+    ap.add_argument("--op", choices=["encode", "decode", "append", "flush", "copy"], default=None)
+    ap.add_argument("--D", type=int, default=128)
+    ap.add_argument("--dtype", choices=["f16", "bf16"], default="f16")
+    ap.add_argument("--n", type=int, default=1 << 20)
+    ap.add_argument("--n-lambda", type=int, default=1)
+    ap.add_argument("--family", choices=["auto", "fft", "gemm", "matvec"], default="auto")
+    ap.add_argument("--kind", default="k_outlier")
+    ap.add_argument("--reps", type=int, default=3)
+    ap.add_argument("--sustain", type=float, default=0.0, help="with --op: seconds of back-to-back launches with nvidia-smi sampling")
     args = ap.parse_args()
+    if args.op is not None:
+        return run_case(args)
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     if args.impl == "reference":

@@ -142,41 +142,6 @@ static kvq_status_t ensure_device(kvq_plan *p)
         p->d_e0 = de;
         p->table_bytes += 2 * bytes;
     }
-    if (p->D == 256) {   // the radix-2 encode kernel's B operand, one image per input type, from the table without a rotation
-        std::vector<float> b0, e0;
-        std::vector<unsigned char> img;
-        unsigned char *dr = nullptr;
-        double *rot = p->rot;
-        const float tmax = p->table_max;
-        p->rot = nullptr;
-        bool ok = make_tables(p, b0, e0);
-        const float lift = r2_encode_lift(p->table_max);
-        p->rot = rot;
-        p->table_max = tmax;
-        if (ok) {
-            try {
-                img.resize(2 * (size_t)kR2ImageBytes);
-            } catch (...) {
-                ok = false;
-            }
-        }
-        if (ok) {
-            r2_encode_b_image(e0.data(), lift, false, img.data());
-            r2_encode_b_image(e0.data(), lift, true, img.data() + kR2ImageBytes);
-            ok = cudaMalloc(&dr, img.size()) == cudaSuccess && cudaMemcpy(dr, img.data(), img.size(), cudaMemcpyHostToDevice) == cudaSuccess;
-        }
-        if (!ok) {
-            (void)cudaGetLastError();
-            if (dr) cudaFree(dr);
-            if (p->d_b0) cudaFree(p->d_b0);
-            if (p->d_e0) cudaFree(p->d_e0);
-            cudaFree(st);
-            p->d_status = nullptr, p->d_b0 = nullptr, p->d_e0 = nullptr;
-            return KVQ_ERR_NOMEM;
-        }
-        p->d_r2 = dr;
-        p->table_bytes += img.size();
-    }
     p->device = dev;
     return KVQ_OK;
 }
@@ -245,7 +210,6 @@ kvq_status_t kvq_plan_create_ex(int D, int group, int bits, uint64_t seed, kvq_p
     p->d_status = nullptr;
     p->d_b0 = nullptr;
     p->d_e0 = nullptr;
-    p->d_r2 = nullptr;
     p->table_bytes = 0;
     p->rot = nullptr;
     p->table_max = (float)std::sqrt(2.0 / D);
@@ -272,9 +236,6 @@ kvq_status_t kvq_plan_destroy(kvq_plan_t *plan)
     }
     if (plan->d_e0) {
         if (cudaFree(plan->d_e0) != cudaSuccess) (void)cudaGetLastError();
-    }
-    if (plan->d_r2) {
-        if (cudaFree(plan->d_r2) != cudaSuccess) (void)cudaGetLastError();
     }
     delete[] plan->rot;
     delete plan;
@@ -374,7 +335,6 @@ kvq_status_t kvq_plan_prepare(kvq_plan_t *plan, kvq_dtype_t dtype)
     g.per_vector = per_vector;
     g.status = plan->d_status;
     g.b0 = plan->d_b0;
-    if (plan->d_r2 && !plan->rot) prm.r2_image = plan->d_r2 + (bf16 ? kR2ImageBytes : 0);
     cudaError_t e = cudaSuccess;
     auto also = [&e](cudaError_t r) {
         if (e == cudaSuccess) e = r;
@@ -463,7 +423,6 @@ static kvq_status_t encode_common(kvq_plan_t *plan, const void *x, kvq_dtype_t d
     prm.packed = packed;
     prm.scales = scales;
     prm.out_map = out_map;
-    if (plan->d_r2 && !plan->rot) prm.r2_image = plan->d_r2 + (bf16 ? kR2ImageBytes : 0);
     // AUTO: the matrix-vector kernel for small calls (latency), beyond that the tensor-core kernel (measured faster than
     // the register FFT at every size above the matrix-vector limit), the register FFT where no tensor-core kernel is
     // built.  A rotated plan has no FFT path: matrix-vector wherever the tensor-core kernel does not apply.

@@ -37,8 +37,6 @@ struct FftParams {
     uint32_t *status;           // per-plan device status word
     float table_max;            // tensor-core encode: largest |entry| of the plan's forward table (sqrt(2/D) without a rotation)
     uint32_t first_wait_polls;  // tensor-core encode, D <= 160: polls the mma role gives its first operand build (0: the default)
-    const void *r2_image;       // tensor-core encode, D = 256, plans without a rotation: the radix-2 kernel's B operand image for
-                                // this input type (kR2ImageBytes, device memory), or null: the dense kernel
     int bits;                   // tensor-core encode: 4 or 8 (the register-FFT launchers take it as an argument)
     uint32_t sign_xor[128];     // word m: bit 15 set if s_{2m} = -1, bit 31 set if s_{2m+1} = -1
 };
@@ -68,12 +66,6 @@ cudaError_t umma_decode(int D, bool bf16, int bits, int64_t N, const GemmParams 
 cudaError_t umma_calibrate(int D, bool bf16, int64_t N, const FftParams &prm, const float *e0, uint32_t *amax_bits, cudaStream_t stream);
 cudaError_t umma_calibrate_d256(bool bf16, int64_t N, const FftParams &prm, const float *e0, uint32_t *amax_bits, cudaStream_t stream);
 cudaError_t umma_encode_d256(bool bf16, bool per_vector, int64_t N, const FftParams &prm, const float *e0, cudaStream_t stream);   // kvq_umma_encode256.cu
-// kvq_umma_encode256_r2.cu: D = 256, groups of 32, 4-bit codes, no rotation: one radix-2 step outside the GEMM.  Its B
-// operand does not depend on lambda: one image per plan and input type, built on the host from the forward table.
-constexpr int kR2ImageBytes = 131072;
-float r2_encode_lift(float table_max);
-void r2_encode_b_image(const float *e0_host /* [256, 256] */, float lift, bool bf16, void *image_host /* kR2ImageBytes */);
-cudaError_t umma_encode_d256_r2(bool bf16, int64_t N, const FftParams &prm, cudaStream_t stream);
 cudaError_t umma_decode_d256(bool bf16, int64_t N, const GemmParams &prm, const uint32_t *sign_xor, cudaStream_t stream);   // kvq_umma_decode256.cu
 cudaError_t umma_decode_d256_dense(bool bf16, int64_t N, const GemmParams &prm, cudaStream_t stream);   // kvq_umma_decode256_dense.cu: any table
 bool umma_encode_per_vector_supported(int D, bool bf16);
@@ -129,8 +121,6 @@ struct kvq_plan {
     uint32_t *d_status;    // device status word
     float *d_b0;           // [D, D] fp32 inverse-transform matrix with the signs folded in (GEMM decode), or null
     float *d_e0;           // [D, D] fp32 forward-transform matrix with the signs folded in (GEMM encode), or null
-    unsigned char *d_r2;   // D = 256: B images of the radix-2 encode kernel, fp16 then bf16 (2 x kR2ImageBytes), or null; they
-                           // hold the transform without a rotation and are used only while the plan has none
     size_t table_bytes;
     double *rot;           // host, [D, D] row-major: the rotation between the transform and lambda, or null
     float table_max;       // largest |entry| of the forward table

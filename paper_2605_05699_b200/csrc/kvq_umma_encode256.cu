@@ -589,7 +589,6 @@ cudaError_t umma_encode_d256(bool bf16, bool per_vector, int64_t N, const FftPar
 {
     if (!tensor_map_encode_fn()) return cudaErrorNotSupported;
     if (per_vector) return bf16 ? launch<true, false, true>(N, f, e0, stream) : launch<false, false, true>(N, f, e0, stream);
-    if (f.r2_image && f.bits == 4) return umma_encode_d256_r2(bf16, N, f, stream);   // no rotation: half the tensor work, one CTA per tile
     return bf16 ? launch<true>(N, f, e0, stream) : launch<false>(N, f, e0, stream);
 }
 

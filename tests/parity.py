@@ -8,10 +8,7 @@ Tolerances (the project's stated ones, with the readings the design notes list):
     rounding tie: with t = v_oracle / sigma in fp64, |t - boundary| <= 1e-3 for sigma = the GPU's or the
     oracle's stored scale; or, when the two stored scales differ (by one fp16 ulp at most), the GPU code is
     the correctly rounded code for the GPU's own stored scale.
-  * group scales: |sigma_gpu - sigma_oracle| <= 1 fp16 ulp everywhere, and relative L2 per vector <= 1e-3.  (One test
-    hands a lambda row to the bf16 tensor-core encode that lifts a single channel 3000 times above its neighbours; there the
-    group maximum can be a near-zero coefficient seen through that gain, its error is relative to the vector and not to
-    itself, and the test allows 2 ulps on top of the 1e-3 rule, which stands.)
+  * group scales: |sigma_gpu - sigma_oracle| <= 1 fp16 ulp everywhere, and relative L2 per vector <= 1e-3.
   * reconstruction: relative L2 per vector <= 1e-3 against the oracle's output rounded to the same dtype,
     not counting elements where the two outputs are format neighbours and the exact value sits at the
     midpoint between them (within 1e-3 of the vector's rms): the output format's own rounding tie.
@@ -31,7 +28,7 @@ def f16_bits_to_f64(b):
     return np.ascontiguousarray(b).view(np.uint16).view(np.float16).astype(np.float64)
 
 
-def check_encode(gpu_packed, gpu_scales_bits, ora, group, label="", bits=4, min_agree=CODE_AGREEMENT, max_scale_ulps=1):
+def check_encode(gpu_packed, gpu_scales_bits, ora, group, label="", bits=4, min_agree=CODE_AGREEMENT):
     """gpu_packed [N, D bits/8] uint8, gpu_scales_bits [N,G] uint16, ora = oracle.encode(..., want_v=True, bits=bits).
     The rules are those of the 4-bit codes with 7 read as 2^(bits-1) - 1; 8-bit codes are one byte each."""
     gpu_packed = np.ascontiguousarray(gpu_packed).view(np.uint8)
@@ -58,7 +55,7 @@ def check_encode(gpu_packed, gpu_scales_bits, ora, group, label="", bits=4, min_
     # scales
     bg = gpu_scales_bits.astype(np.int64)
     bo = ora["scales"].astype(np.int64)
-    assert np.abs(bg - bo).max(initial=0) <= max_scale_ulps, label + ": a scale differs by more than %d fp16 ulp" % max_scale_ulps
+    assert np.abs(bg - bo).max(initial=0) <= 1, label + ": a scale differs by more than one fp16 ulp"
     sg, so = f16_bits_to_f64(gpu_scales_bits), f16_bits_to_f64(ora["scales"])
     den = np.linalg.norm(so, axis=1)
     rel = np.linalg.norm(sg - so, axis=1) / np.where(den > 0, den, 1.0)

@@ -924,12 +924,7 @@ def test_degenerate_lambda(D, dtype, impl, wild):
     sg = plan.signs()
     packed, scales = gpu_encode(plan, x.cuda(), lam.cuda(), 1500)
     ora = ko.encode(bits(x), odt, sg, lam.numpy(), G, 1500, want_v=True)
-    # bf16 input on the tensor cores carries the table in two bf16 terms (16 bits): an error of 1e-5 of the vector's norm in
-    # every coefficient.  The wild row lifts ONE channel 3000 times above its neighbours, so a group's maximum can be a
-    # coefficient near zero seen through that gain, and its stored scale then moves by 2 fp16 ulps (1e-3) in about one
-    # group in 20,000; the 1e-3 relative L2 per vector on the scales holds regardless.
-    ulps = 2 if (wild and impl == "gemm" and dtype == "bf16") else 1
-    parity.check_encode(packed.cpu().numpy(), bits(scales), ora, G, "odd lambda encode (%s)" % impl, max_scale_ulps=ulps)
+    parity.check_encode(packed.cpu().numpy(), bits(scales), ora, G, "odd lambda encode (%s)" % impl)
     ob, o64 = ko.decode(ora["packed"], ora["scales"], sg, lam.numpy(), G, odt, 1500, want_f64=True)
     out = gpu_decode_raw(plan, torch.from_numpy(ora["packed"]).cuda(),
                          torch.from_numpy(ora["scales"].view(np.int16)).view(torch.float16).cuda(), lam.cuda(), dtype, 1500)
