@@ -183,7 +183,6 @@ struct FirstRows {
 // counts looks at the barrier that do not block, so that "one poll" is over before the operand can possibly be there.
 __device__ __forceinline__ bool wait_first_operand(uint32_t bar, volatile uint32_t *abort_flag, uint32_t *status, uint32_t limit)
 {
-    if (limit >= kWaitPolls) return wait_or_abort(bar, 0u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT);
     for (uint32_t it = 0; it < limit; ++it)
         if (mbar_test_wait(bar, 0u)) return true;
     *abort_flag = 1u;
@@ -312,6 +311,11 @@ __global__ void __launch_bounds__(kThreads, 1)
     } else if (warp == 1) {
         // =========================== mma issuer ===========================
         if (lane == 0) {
+            // A limit shortened by the host (kvq_plan_set_wait_limit) is spent here, straight after the set-up barrier, when
+            // the builders have only just begun to store: this thread has issued nothing yet and can leave at once.
+            bool first_ok = true;
+            if (n_my > 0 && prm.first_wait_polls < kWaitPolls)
+                first_ok = wait_first_operand(smem_u32(&ctrl->b_first), abort_flag, status, prm.first_wait_polls);
             // Descriptors differ only in their 14-bit start-address field (bytes >> 4): one base per operand, one add per MMA.
             // The issuing thread is a single instruction stream: what it spends per MMA beyond the issue itself is time
             // the tensor core idles.
@@ -321,11 +325,10 @@ __global__ void __launch_bounds__(kThreads, 1)
             const uint32_t a_lo = (uint32_t)a_desc, a_hi = (uint32_t)(a_desc >> 32);
             uint32_t builds = 0;
             TileCursor cur(tile_begin, tps);
-            for (int j = 0; j < n_my; ++j, cur.advance(1)) {
+            for (int j = 0; j < n_my && first_ok; ++j, cur.advance(1)) {
                 const int s = j % kInStages, sc = j % kAccStages;
                 if (j == 0) {   // all epilogue warps build the first B while the first x tiles are in flight
-                    // (this thread has issued nothing yet: the one wait whose limit the host may shorten, to see a time-out reported)
-                    if (!wait_first_operand(smem_u32(&ctrl->b_first), abort_flag, status, prm.first_wait_polls)) break;
+                    if (!wait_or_abort(smem_u32(&ctrl->b_first), 0u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT)) break;
                 } else if (cur.first_of_segment()) {   // an epilogue set rebuilds B for this lambda row
                     if (!wait_or_abort(smem_u32(&ctrl->b_ready), builds & 1u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT)) break;
                     ++builds;
