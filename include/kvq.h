@@ -48,8 +48,8 @@ typedef enum {
     KVQ_ERR_TIMEOUT = 5,         /* a bounded device-side wait ran out (see kvq_plan_device_status) */
     KVQ_ERR_NOMEM = 6,
     KVQ_ERR_SCRATCH_LIMIT = 7,   /* the plan needs more fixed scratch than kvq_decode_static holds */
-    KVQ_ERR_RANGE = 8            /* a tensor-core decode met a lambda row or a stored scale outside its operand
-                                    range (see kvq_plan_device_status) */
+    KVQ_ERR_RANGE = 8            /* reserved (earlier: a tensor-core decode met numbers outside its operands' range;
+                                    such tiles are now decoded in fp32 by the same launch) */
 } kvq_status_t;
 
 typedef enum { KVQ_F16 = 0, KVQ_BF16 = 1 } kvq_dtype_t;
@@ -161,20 +161,19 @@ kvq_status_t kvq_plan_set_wait_limit(kvq_plan_t *plan, uint32_t polls);
 /* Synchronizes the current device and returns the plan's device status word through *word
  * (host): 0 when no kernel using this plan ever gave up a bounded wait or left its number
  * range.  Bits 0-2: a bounded wait ran out (load, tensor-core commit, pipeline slot): returns
- * KVQ_ERR_TIMEOUT.  Bit 3: a tensor-core kvq_decode met data outside its operand range; the rows
- * concerned are wrong, decode them with KVQ_IMPL_MATVEC or KVQ_IMPL_FFT (fp32 throughout).
- * Those kernels carry q sigma / lambda and the table entries divided by lambda as fp16 operands:
+ * KVQ_ERR_TIMEOUT.  Bit 3 is reserved: no kernel raises it any longer.  The tensor-core decode kernels
+ * carry q sigma / lambda and the table entries divided by lambda as fp16 operands, which cannot hold
  *   - a lambda row whose reciprocals 1 / max(lambda, 1e-6) span more than a factor of 2^8
- *     (entries at or below the 1e-6 clamp next to ordinary ones, for instance) loses bits on the
- *     channels with the small reciprocals: every tensor-core decode kernel reports it;
- *   - a non-zero stored scale sigma with sigma rho outside [2^-14, 9357] (rho: the power of two at
- *     or below the row's largest reciprocal; very small or very large vectors): all kernels but
- *     one rescale such rows by a power of two and are exact for them; the dense D = 256 kernel
- *     of ROTATED plans reports them instead.
+ *     (entries at or below the 1e-6 clamp of Sec. 5.1 item 1 next to ordinary ones, for instance), or
+ *   - in the dense D = 256 kernel of ROTATED plans, which has no room for the other kernels' per-row
+ *     power-of-two rescue, a non-zero stored scale sigma with sigma rho outside [2^-14, 9357]
+ *     (rho: the power of two at or below the row's largest reciprocal);
+ * a CTA that met either decodes the tiles concerned once more at the end of the same launch, in
+ * fp32 on the CUDA cores (about a hundred times slower per row), so kvq_decode is exact for every
+ * lambda row and scale whichever kernel serves it, and nothing is reported.
  * Bit 4: kvq_append_at or kvq_flush_block_at found a position outside the cache in device memory and
  * wrote nothing: returns KVQ_ERR_INVALID_ARG (unless bits 0-2 are set too).
- * Returns KVQ_ERR_RANGE if bit 3 is the only bit set.  The word is sticky until
- * kvq_plan_clear_device_status. */
+ * The word is sticky until kvq_plan_clear_device_status. */
 kvq_status_t kvq_plan_device_status(kvq_plan_t *plan, uint32_t *word);
 
 /* Synchronizes the current device and clears the plan's device status word (after the caller has dealt with what it

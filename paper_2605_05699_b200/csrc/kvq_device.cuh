@@ -17,7 +17,7 @@ enum : uint32_t {
     KVQ_DEV_LOAD_TIMEOUT = 1u,   // a bounded wait for a bulk load ran out
     KVQ_DEV_MMA_TIMEOUT = 2u,    // a bounded wait for a tensor-core commit ran out
     KVQ_DEV_SLOT_TIMEOUT = 4u,   // a bounded wait for a free pipeline slot ran out
-    KVQ_DEV_RANGE = 8u,          // a tensor-core decode met a lambda row or a stored scale outside its fp16 operands' range
+    KVQ_DEV_RANGE = 8u,          // reserved: tiles outside the fp16 operands' range are redone in fp32 by the decode kernels themselves
     KVQ_DEV_POSITION = 16u,      // a cache position read from device memory was outside the cache: nothing was written
 };
 

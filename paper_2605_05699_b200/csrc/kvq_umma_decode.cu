@@ -37,6 +37,7 @@
 // vector before the output rounding.  Every wait on an mbarrier is bounded: on a time-out the role
 // records the reason in the status word, raises the CTA's abort flag and leaves its loop; the CTA
 // then frees its tensor memory and returns.
+#include "kvq_decode_fp32.cuh"
 #include "kvq_internal.h"
 #include "kvq_umma.cuh"
 
@@ -119,6 +120,7 @@ struct Ctrl {
     uint64_t b_first;
     uint32_t tmem_base;
     volatile uint32_t abort;
+    volatile uint32_t any_wide;   // some lambda row of this CTA's tiles is too wide for the fp16 B operand: redone in fp32 at the end
     float row_scale[kRowScaleSlots][kTile];   // what the epilogue multiplies a row by (1 unless its scales left fp16's comfort zone)
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
@@ -333,6 +335,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
         mbar_init(smem_u32(&ctrl->b_first), 16);   // first B: the sixteen dequant and epilogue warps build it
         ctrl->abort = 0u;
+        ctrl->any_wide = 0u;
         mbar_init_fence();
     }
     if (warp == 0) tmem_alloc(smem_u32(&ctrl->tmem_base), kTmemCols);
@@ -356,11 +359,11 @@ __global__ void __launch_bounds__(kThreads, 1)
         FirstRows<D, BF16OUT, BITS, R2> rows;
         rows.load(prm.g.b0, (warp - 2) * (C::kBRows / 16), lane);
         const RecipLambda<D> rl(lambda_row(seg_first), lane);
-        if (rl.wide && warp == 2 && lane == 0) atomicOr(prm.g.status, KVQ_DEV_RANGE);
         fence_proxy_async();
         tc_fence_before();
         __syncthreads();
         tc_fence_after();
+        if (rl.wide) ctrl->any_wide = 1u;
         rows.build(sB, rl, (warp - 2) * (C::kBRows / 16), lane);
         fence_proxy_async();   // B is read by the tensor core through the async proxy
         __syncwarp();
@@ -493,6 +496,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             if (seg != cached_seg) {
                 const RecipLambda<D> rl(lambda_row(seg), lane);
                 rho = rl.rho;
+                if (rl.wide) ctrl->any_wide = 1u;
                 if (cur.first_of_segment()) {
                     // Every MMA issued so far has read B: the commit of the previous tile (the other group's) covers them
                     // all.  A parity wait can only tell a phase from its neighbours, and the other group may lag by more
@@ -505,7 +509,6 @@ __global__ void __launch_bounds__(kThreads, 1)
                     if (!wait_or_abort(smem_u32(&ctrl->a_empty[(j - 1) % C::kABars]), (uint32_t)((j - 1) / C::kABars) & 1u, abort_flag,
                                        status, KVQ_DEV_MMA_TIMEOUT))
                         break;
-                    if (rl.wide && q == 0 && lane == 0) atomicOr(status, KVQ_DEV_RANGE);
                     build_b_rows<D, BF16OUT, BITS, R2>(sB, prm.g.b0, rl, q * (C::kBRows / 4), (q + 1) * (C::kBRows / 4), lane);
                     fence_proxy_async();   // B is read by the tensor core through the async proxy
                 }
@@ -708,6 +711,9 @@ __global__ void __launch_bounds__(kThreads, 1)
         if (*abort_flag) __nanosleep(20000);   // let tensor-core work that was already issued drain
         tmem_dealloc(tmem_base, kTmemCols);
     }
+    // ---- tiles of a lambda row too wide for the fp16 B operand: decoded again in fp32, over what the pipeline stored
+    if (ctrl->any_wide && !*abort_flag)
+        redo_tiles_fp32<D, BF16OUT, BITS, kTile>(prm.g, tile_begin, n_my, tps, rpl, reinterpret_cast<float *>(smem));
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -32,6 +32,7 @@
 //
 // Every wait is bounded: on a time-out the role records the reason in the status word, raises the CTA's abort
 // flag and leaves its loop; the CTA then frees its tensor memory and returns.
+#include "kvq_decode_fp32.cuh"
 #include "kvq_internal.h"
 #include "kvq_umma.cuh"
 
@@ -74,7 +75,8 @@ struct Ctrl {
     uint64_t b_first;
     uint32_t tmem_base;
     volatile uint32_t abort;
-    uint32_t pad[2];
+    volatile uint32_t any_wide;   // some lambda row of this CTA's tiles is too wide for the fp16 B operand: redone in fp32 at the end
+    uint32_t pad;
     uint4 flip[16];   // sign-bit masks of s_n s_{n+128} for the output pairs (n, n + 1), n = 0, 2, .. 126
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
@@ -192,6 +194,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         mbar_init(smem_u32(&ctrl->acc_empty), 8);
         mbar_init(smem_u32(&ctrl->b_first), 16);
         ctrl->abort = 0u;
+        ctrl->any_wide = 0u;
         mbar_init_fence();
     }
     if (threadIdx.x >= 32 && threadIdx.x < 96) {   // sign of s_n s_{n+128}: the xor of the two sign bits
@@ -223,7 +226,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     // ---- and eight the O operand, sixteen rows each
     if (n_my > 0 && warp >= 2) {
         const RecipLambda rl(lambda_row(seg_first), lane);
-        if (rl.wide && warp == 2 && lane == 0) atomicOr(prm.g.status, KVQ_DEV_RANGE);
+        if (rl.wide) ctrl->any_wide = 1u;
         const int bp = ((warp - 2) >> 2) & 1, bw = ((warp - 2) & 3) + 4 * ((warp - 2) >> 3);   // parity, position among its eight
         build_b_rows<kTerms>(sB, prm.g.b0, rl, bp, bw * 16, bw * 16 + 16, lane);
         fence_proxy_async();   // B is read by the tensor core through the async proxy
@@ -326,7 +329,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             // ---- GEMM issued so far is complete: the previous tile's, on this group's own barriers (it sees every phase)
             if (seg != cached_seg) {
                 const RecipLambda rl(lambda_row(seg), lane);
-                if (rl.wide && q == 0 && lane == 0) atomicOr(status, KVQ_DEV_RANGE);
+                if (rl.wide) ctrl->any_wide = 1u;
                 rho = rl.rho;
                 if (!wait_or_abort(smem_u32(&ctrl->a_empty[p][(j - 1) % C::kAStages]), (uint32_t)((j - 1) / C::kAStages) & 1u, abort_flag,
                                    status, KVQ_DEV_MMA_TIMEOUT))
@@ -466,6 +469,9 @@ __global__ void __launch_bounds__(kThreads, 1)
         if (*abort_flag) __nanosleep(20000);   // let tensor-core work that was already issued drain
         tmem_dealloc(tmem_base, kTmemCols);
     }
+    // ---- tiles of a lambda row too wide for the fp16 B operand: decoded again in fp32, over what the pipeline stored
+    if (ctrl->any_wide && !*abort_flag)
+        redo_tiles_fp32<kD, BF16OUT, 4, kTile>(prm.g, tile_begin, n_my, tps, rpl, reinterpret_cast<float *>(smem));
 }
 
 // ------------------------------------------------------------------------------------------------

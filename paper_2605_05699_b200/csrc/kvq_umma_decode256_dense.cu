@@ -19,6 +19,7 @@
 // The A operand lives in tensor memory by K halves (128 codes: 64 columns, twice that with a_lo), two
 // stages; the accumulator (128 columns) has two stages.  Roles as in kvq_umma_decode.cu: producer (TMA),
 // two dequant groups, one mma thread, two epilogue groups; every wait is bounded.
+#include "kvq_decode_fp32.cuh"
 #include "kvq_internal.h"
 #include "kvq_umma.cuh"
 
@@ -56,6 +57,7 @@ struct Ctrl {
     uint64_t b_first;
     uint32_t tmem_base;
     volatile uint32_t abort;
+    volatile uint32_t any_wide;  // a lambda row too wide for the fp16 B operand, or a scale outside A's range: tiles redone in fp32 at the end
     volatile uint32_t b_epoch;   // lambda rows whose last MMA is complete, counted from the CTA's first one
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
@@ -172,6 +174,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
         mbar_init(smem_u32(&ctrl->b_first), 16);
         ctrl->abort = 0u;
+        ctrl->any_wide = 0u;
         ctrl->b_epoch = 0u;
         mbar_init_fence();
     }
@@ -199,7 +202,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     // ---- B for the first tile's lambda row: the sixteen dequant and epilogue warps build eight rows each
     if (n_my > 0 && warp >= 2) {
         const RecipLambda rl(lambda_row(seg_first), lane);
-        if (rl.wide && warp == 2 && lane == 0) atomicOr(prm.g.status, KVQ_DEV_RANGE);
+        if (rl.wide) ctrl->any_wide = 1u;
         build_b_rows<C::kBTerms>(sB, prm.g.b0, rl, half, (warp - 2) * 8, (warp - 1) * 8, lane);
         fence_proxy_async();   // B is read by the tensor core through the async proxy
         __syncwarp();
@@ -315,7 +318,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             // ---- a new lambda row: this group needs its rho; the group that meets the row's first tile rebuilds B
             if (seg != cached_seg) {
                 const RecipLambda rl(lambda_row(seg), lane);
-                if (rl.wide && q == 0 && lane == 0) atomicOr(status, KVQ_DEV_RANGE);
+                if (rl.wide) ctrl->any_wide = 1u;
                 rho = rl.rho;
                 if (cur.first_of_segment()) {
                     // every MMA issued so far must have read B: the mma thread says so by raising b_epoch to this row's index
@@ -377,7 +380,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                     const float sr = sig * rho;
                 const __half2 s2 = __float2half2_rn(sr);
                 // the A operand q sigma rho is fp16: it overflows beyond 7 sr = 65504 and loses bits once sr is subnormal
-                if (sr != 0.0f && (sr > 9357.0f || sr < 6.1035156e-5f)) atomicOr(status, KVQ_DEV_RANGE);
+                if (sr != 0.0f && (sr > 9357.0f || sr < 6.1035156e-5f)) ctrl->any_wide = 1u;   // the tile is redone in fp32 at the end
                     const uint32_t words[4] = {pk[c].x, pk[c].y, pk[c].z, pk[c].w};
                     uint32_t a_hi[16], a_lo[16];
 #pragma unroll
@@ -459,6 +462,10 @@ __global__ void __launch_bounds__(kThreads, 1)
         if (*abort_flag) __nanosleep(20000);   // let tensor-core work that was already issued drain
         tmem_dealloc(tmem_base, kTmemCols);
     }
+    // ---- tiles of a lambda row too wide for the fp16 B operand, or with a scale outside the A operand's range: this CTA's
+    // ---- output columns decoded again in fp32
+    if (ctrl->any_wide && !*abort_flag)
+        redo_tiles_fp32<kD, BF16OUT, 4, kTile, kHalfN, true>(prm.g, tile_begin, n_my, tps, rpl, reinterpret_cast<float *>(smem), half * kHalfN);
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -131,6 +131,33 @@ def test_a_captured_static_decode_brings_its_own_table():
     plan_b.close()
 
 
+def test_static_decode_of_a_lambda_row_no_fp16_operand_can_carry():
+    """An entry at the 1e-6 clamp (Sec. 5.1 item 1) beside ordinary ones: the kernel redoes such a row's tiles in fp32 inside
+    the same launch, with the table in the fixed block, and still allocates nothing."""
+    N, rpl = 3000, 1000
+    helper = kb.Plan(D, G, 41)
+    x = wl.make_vectors(N, D, "f16", "k_outlier", 600, device="cuda")
+    lam = wl.make_lambda(3, D, 601, device="cuda")
+    lam[1, 9] = 1e-6
+    packed, scales = helper.empty_packed(N), helper.empty_scales(N)
+    kb.kvq_encode(helper.handle, x, lam, packed, scales, rpl)
+    torch.cuda.synchronize()
+    helper.close()
+    plan = kb.Plan(D, G, 41)
+    got = torch.empty(N, D, dtype=torch.float16, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    kb.kvq_decode_static(plan.handle, packed, scales, lam, got, rpl, status_word=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    sg = ko.signs(D, 41)
+    ob, o64 = ko.decode(packed.cpu().numpy(), wl.raw_bits(scales), sg, lam.cpu().numpy(), G, ko.F16, rpl, want_f64=True)
+    ok = np.abs(o64).max(axis=1) < 0.25 * 65504.0
+    assert ok[:rpl].all() and ok[2 * rpl:].all() and ok[rpl:2 * rpl].mean() > 0.3
+    parity.check_decode(wl.raw_bits(got)[ok], ob[ok], o64[ok], ko.F16, "static decode, wide lambda row")
+    assert plan.describe()[1] == 0
+    plan.close()
+
+
 def test_static_decode_refuses_what_does_not_fit():
     lam256 = torch.ones(256, device="cuda")
     big = kb.Plan(256, G, 1)
