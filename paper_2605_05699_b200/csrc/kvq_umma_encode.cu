@@ -50,6 +50,10 @@ constexpr int kBlockBytes = kTile * 128;   // one K block of the x tile: 128 row
 constexpr int kCtrlBytes = 4608;            // barriers and flags, then the row maxima the two half-row threads trade
 constexpr int kSmemLimit = 232448;         // 227 KB of dynamic shared memory per CTA
 constexpr uint32_t kTmemCols = 512;
+// "Accumulator full" barriers form a ring of four indexed by TILE, whatever the number of accumulator stages: the producer
+// takes tile j - kInStages's as "x stage free", and a parity wait only tells a phase from its neighbours, so the barrier it
+// waits on must not be able to complete another phase before the producer has loaded tile j.
+constexpr int kFullBars = 4;
 
 
 // THREE: a third bf16 term of W.  The calibration pass takes it (it runs once; its result is compared at 1e-6 of the
@@ -62,22 +66,29 @@ struct Cfg {
     static constexpr int kKSteps = D / 16;
     static constexpr int kKBlocks = (D + 63) / 64;              // K blocks of 64 elements (the last one may be half used)
     static constexpr int kXBytes = kKBlocks * kBlockBytes;      // one x tile
-    static constexpr int kBBlock = D * 128;                     // one K block of one split term: D rows x 128 B
-    static constexpr int kBTerm = kKBlocks * kBBlock;           // one split term
-    static constexpr int kBBytes = kSplit * kBTerm;
+    // Two terms and D <= 128: the terms are STACKED along N, rows [0, D) of a K block the first term's, rows [D, 2 D) the
+    // second's, and one MMA of N = 2 D computes x W_hi into accumulator columns [0, D) and x W_lo into [D, 2 D); the
+    // epilogue adds the two.  An MMA of M 128, N 128, K 16 costs about 120 cycles here, one of N = 256 about 176 (measured,
+    // both operands in shared memory, accumulating into one tile; the nominal rates are 68 and 135): the per-instruction
+    // overhead is paid once for both terms, and the x tile is read from shared memory once instead of twice.
+    static constexpr bool kStack = kSplit == 2 && D <= 128;
+    static constexpr int kNmma = kStack ? 2 * D : D;            // N of one MMA
+    static constexpr int kBBlock = kNmma * 128;                 // one K block of B: kNmma rows x 128 B
+    static constexpr int kBTerm = kStack ? D * 128 : kKBlocks * kBBlock;   // from one term's row c to the next term's
+    static constexpr int kBBytes = kSplit * kKBlocks * D * 128;
     static constexpr int kRoom = (kSmemLimit - 1024 - kCtrlBytes - kBBytes) / kXBytes;
     static constexpr int kInStages = kRoom < 4 ? kRoom : 4;     // x tiles in flight
-    static_assert(kInStages >= 2, "this head dim and input type do not fit shared memory");
+    static_assert(kInStages >= 2 && kInStages <= kFullBars, "this head dim and input type do not fit shared memory");
     static constexpr int kSmemBytes = kBBytes + kInStages * kXBytes + kCtrlBytes + 1024;
-    static constexpr int kAccStages = D <= 128 ? 4 : 3;         // accumulators in tensor memory
-    static constexpr uint32_t kAccStride = D <= 128 ? 128 : 160;
-    static constexpr uint32_t kIdesc = umma_idesc_m128(D, BF16);
+    static constexpr uint32_t kAccStride = kStack ? 2 * D : D <= 128 ? 128 : 160;
+    static constexpr int kAccStages = 512 / (int)kAccStride < 4 ? 512 / (int)kAccStride : 4;   // accumulators in tensor memory
+    static constexpr uint32_t kIdesc = umma_idesc_m128(kNmma, BF16);
     static constexpr int kGroupsPerPart = (G + 1) / 2;          // groups of the first half row; the second takes the rest
 };
 
 struct Ctrl {
     uint64_t in_full[4];
-    uint64_t acc_full[4], acc_empty[4];
+    uint64_t acc_full[kFullBars], acc_empty[4];
     uint64_t b_first, b_ready;
     uint64_t pair[2][4];        // one scale per vector: the two warps that share 32 rows of a set meet here, once per tile
     uint32_t tmem_base;
@@ -227,10 +238,8 @@ __global__ void __launch_bounds__(kThreads, 1)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kInStages; ++s) mbar_init(smem_u32(&ctrl->in_full[s]), 1);
-        for (int s = 0; s < kAccStages; ++s) {
-            mbar_init(smem_u32(&ctrl->acc_full[s]), 1);
-            mbar_init(smem_u32(&ctrl->acc_empty[s]), kEpiWarps / 2);
-        }
+        for (int s = 0; s < kFullBars; ++s) mbar_init(smem_u32(&ctrl->acc_full[s]), 1);
+        for (int s = 0; s < kAccStages; ++s) mbar_init(smem_u32(&ctrl->acc_empty[s]), kEpiWarps / 2);
         mbar_init(smem_u32(&ctrl->b_first), kEpiWarps);       // first B: all epilogue warps build it
         mbar_init(smem_u32(&ctrl->b_ready), kEpiWarps / 2);   // later rebuilds: the set that owns the tile
         for (int s = 0; s < 2; ++s)
@@ -286,11 +295,10 @@ __global__ void __launch_bounds__(kThreads, 1)
             for (int j = 0; j < n_my; ++j, cur.advance(1)) {
                 const int s = j % kInStages;
                 // The x stage is free once the MMAs of the tile that used it last are complete: that tile's accumulator
-                // barrier.  (MMAs complete in order and this thread waited for the tile before, so the barrier is at most
-                // one phase behind and the parity test cannot be fooled.)
+                // barrier.  (Its next phase is tile j's own, which cannot complete before this load: the parity test holds.)
                 if (j >= kInStages) {
                     const int jp = j - kInStages;
-                    ok = wait_or_abort(smem_u32(&ctrl->acc_full[jp % kAccStages]), (uint32_t)(jp / kAccStages) & 1u, abort_flag, status,
+                    ok = wait_or_abort(smem_u32(&ctrl->acc_full[jp % kFullBars]), (uint32_t)(jp / kFullBars) & 1u, abort_flag, status,
                                        KVQ_DEV_SLOT_TIMEOUT);
                 }
                 if (!ok) break;
@@ -341,7 +349,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                 const uint32_t d_tmem = tmem_base + (uint32_t)sc * C::kAccStride;
                 const uint32_t a_lo_s = a_lo + (uint32_t)s * (C::kXBytes >> 4);
 #pragma unroll
-                for (int t = 0; t < C::kSplit; ++t) {
+                for (int t = 0; t < (C::kStack ? 1 : C::kSplit); ++t) {   // stacked terms: one MMA per K-step computes both
 #pragma unroll
                     for (int ks = 0; ks < C::kKSteps; ++ks) {
                         // (bytes >> 4) of K-step ks inside the x tile and inside a split term
@@ -353,7 +361,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                         else umma_f16_ss<false>(d_tmem, ad, bd, C::kIdesc);
                     }
                 }
-                umma_commit(smem_u32(&ctrl->acc_full[sc]));   // to the epilogue; the producer takes it as "x stage free"
+                umma_commit(smem_u32(&ctrl->acc_full[j % kFullBars]));   // to the epilogue; the producer takes it as "x stage free"
             }
         }
     } else {
@@ -370,6 +378,19 @@ __global__ void __launch_bounds__(kThreads, 1)
         const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16);
         int64_t cached_seg = first_seg;           // B holds this row's table (built above)
         float unlift = 1.0f / first_lift;
+        // Group g of this thread's row of accumulator stage sc; with stacked terms the sum of the two terms' columns.
+        auto load_group = [&](int sc, int g, uint32_t (&vb)[32]) {
+            tmem_ld32(t_addr + (uint32_t)sc * C::kAccStride + (uint32_t)(g * kGroup), vb);
+            if constexpr (C::kStack) {
+                uint32_t lo[32];
+                tmem_ld32(t_addr + (uint32_t)sc * C::kAccStride + (uint32_t)(D + g * kGroup), lo);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) vb[i] = __float_as_uint(__uint_as_float(vb[i]) + __uint_as_float(lo[i]));
+            } else {
+                tmem_ld_wait();
+            }
+        };
         float colmax[C::kGroupsPerPart] = {};   // calibration: lane i keeps the running maximum of column i of each of this thread's groups
         TileCursor cur(tile_begin + set, tps);
         for (int j = set; j < n_my; j += 2, cur.advance(2)) {
@@ -384,7 +405,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                 const float *lam = CALIB ? nullptr : prm.lambda + (prm.n_lambda == 1 ? 0 : seg) * D;
                 const float lift = lift_of<D>(lam, prm.table_max, lane);
                 if (j > 0 && cur.first_of_segment()) {
-                    if (!wait_or_abort(smem_u32(&ctrl->acc_full[(j - 1) % kAccStages]), (uint32_t)((j - 1) / kAccStages) & 1u,
+                    if (!wait_or_abort(smem_u32(&ctrl->acc_full[(j - 1) % kFullBars]), (uint32_t)((j - 1) / kFullBars) & 1u,
                                        abort_flag, status, KVQ_DEV_MMA_TIMEOUT))
                         break;
                     build_b_rows<D, BF16, CALIB || WIDE>(sB, prm.e0, lam, lift, bw * (D / 8), (bw + 1) * (D / 8), lane);
@@ -397,7 +418,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             }
 
             const int sc = j % kAccStages;
-            if (!wait_or_abort(smem_u32(&ctrl->acc_full[sc]), (uint32_t)(j / kAccStages) & 1u, abort_flag, status, KVQ_DEV_MMA_TIMEOUT)) break;
+            if (!wait_or_abort(smem_u32(&ctrl->acc_full[j % kFullBars]), (uint32_t)(j / kFullBars) & 1u, abort_flag, status, KVQ_DEV_MMA_TIMEOUT)) break;
             tc_fence_after();
 
             // ---- rows of the tile that exist: the segment (and with it the tensor) may end inside the tile
@@ -417,8 +438,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                     const int g = g0 + gi;
                     if (g < g1) {
                         uint32_t vb[32];
-                        tmem_ld32(t_addr + (uint32_t)sc * C::kAccStride + (uint32_t)(g * kGroup), vb);
-                        tmem_ld_wait();
+                        load_group(sc, g, vb);
 #pragma unroll
                         for (int i = 0; i < 32; ++i) m = fmaxf(m, fabsf(__uint_as_float(vb[i])));
                     }
@@ -443,8 +463,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                 const int g = g0 + gi;       // warp-uniform
                 if (g < g1) {
                     uint32_t vb[32];
-                    tmem_ld32(t_addr + (uint32_t)sc * C::kAccStride + (uint32_t)(g * kGroup), vb);
-                    tmem_ld_wait();
+                    load_group(sc, g, vb);
                     if (g == g1 - 1) {   // this thread's last group is in registers: hand the accumulator back
                         tc_fence_before();
                         __syncwarp();
