@@ -35,9 +35,7 @@ constexpr int kD = 256;
 constexpr int kG = kD / kGroup;            // 8 scales per row
 constexpr int kHalfN = 128;                // channels per CTA = MMA N
 constexpr int kKBlocks = kD / 64;          // 4 K blocks per tile
-constexpr int kBBlock = kHalfN * 128;      // one K block of one split term: 128 rows x 128 B
-constexpr int kBTerm = kKBlocks * kBBlock; // 64 KB
-constexpr int kAccStages = 4;
+constexpr int kBTermBytes = kKBlocks * kHalfN * 128;   // one split term of B: 128 rows x K = 256, 64 KB
 constexpr int kMaxRing = 6;
 
 // CALIB: the calibration pass keeps a third bf16 term (it runs once; its result is compared at 1e-6 of the vector norm)
@@ -46,13 +44,23 @@ constexpr int kMaxRing = 6;
 template <bool BF16, bool CALIB = false, bool PERVEC = false>
 struct Cfg {
     static constexpr int kSplit = (BF16 && CALIB) ? 3 : 2;
-    static constexpr int kBBytes = kSplit * kBTerm;
+    static constexpr int kBBytes = kSplit * kBTermBytes;
+    // Two terms: STACKED along N, rows [0, 128) of a K block the first term's, rows [128, 256) the second's, so that one
+    // MMA of N = 256 computes x W_hi into accumulator columns [0, 128) and x W_lo into [128, 256); the epilogue adds the
+    // two.  An MMA of M 128, N 128, K 16 costs about 120 cycles here, one of N = 256 about 176 (measured, operands in
+    // shared memory): the per-instruction overhead is paid once for both terms and x is read once instead of twice.
+    static constexpr bool kStack = kSplit == 2;
+    static constexpr int kNmma = kStack ? 2 * kHalfN : kHalfN;
+    static constexpr int kBBlock = kNmma * 128;                          // one K block of B: kNmma rows x 128 B
+    static constexpr int kBTerm = kStack ? kHalfN * 128 : kBTermBytes;   // from one term's row c to the next term's
+    static constexpr uint32_t kAccStride = kNmma;                        // tensor-memory columns per accumulator
+    static constexpr int kAccStages = 512 / kNmma;                       // 2 (stacked) or 4
     static constexpr int kMaxBytes = PERVEC ? 2 * 2 * 4 * kTile * (int)sizeof(float) : 0;   // [tile parity][set][party][row]
     static constexpr int kRoom = (kSmemLimit - 1024 - kCtrlBytes - kMaxBytes - kBBytes) / kBlockBytes;
     static constexpr int kRing = kRoom < kMaxRing ? kRoom : kMaxRing;   // K blocks of x in flight: 6 (2 next to a three-term B)
     static_assert(kRing >= 2, "no room for the x ring");
     static constexpr int kSmemBytes = kBBytes + kRing * kBlockBytes + kCtrlBytes + kMaxBytes + 1024;
-    static constexpr uint32_t kIdesc = umma_idesc_m128(kHalfN, BF16);
+    static constexpr uint32_t kIdesc = umma_idesc_m128(kNmma, BF16);
 };
 
 struct Ctrl {
@@ -152,11 +160,11 @@ __device__ __forceinline__ void build_b_rows(unsigned char *sB, const float *__r
             const float4 m = __ldg(reinterpret_cast<const float4 *>(e0 + (size_t)cg * kD) + i);
             float w[4] = {m.x * f, m.y * f, m.z * f, m.w * f};
             const int ch = i >> 1;   // 16-byte chunk of the K-major row: K block ch / 8, chunk ch % 8
-            const uint32_t off = (uint32_t)((ch >> 3) * kBBlock + c * 128 + (((ch & 7) ^ (c & 7)) << 4) + ((i & 1) ? 8 : 0));
+            const uint32_t off = (uint32_t)((ch >> 3) * C::kBBlock + c * 128 + (((ch & 7) ^ (c & 7)) << 4) + ((i & 1) ? 8 : 0));
 #pragma unroll
             for (int t = 0; t < C::kSplit; ++t) {
                 const uint32_t lo = narrow2<BF16>(w[0], w[1]), hi = narrow2<BF16>(w[2], w[3]);
-                *reinterpret_cast<uint2 *>(sB + t * kBTerm + off) = make_uint2(lo, hi);
+                *reinterpret_cast<uint2 *>(sB + t * C::kBTerm + off) = make_uint2(lo, hi);
                 if (t + 1 < C::kSplit) {   // what the 16-bit term left behind (exact in fp32)
                     const float2 a = widen2<BF16>(lo), b = widen2<BF16>(hi);
                     w[0] -= a.x, w[1] -= a.y, w[2] -= b.x, w[3] -= b.y;
@@ -204,7 +212,7 @@ __device__ __forceinline__ void encode_d256_body(const UmmaEncode256Params &prm,
             mbar_init(smem_u32(&ctrl->in_full[s]), 1);
             mbar_init(smem_u32(&ctrl->in_empty[s]), 1);
         }
-        for (int s = 0; s < kAccStages; ++s) {
+        for (int s = 0; s < C::kAccStages; ++s) {
             mbar_init(smem_u32(&ctrl->acc_full[s]), 1);
             mbar_init(smem_u32(&ctrl->acc_empty[s]), kEpiWarps / 2);
         }
@@ -271,17 +279,17 @@ __device__ __forceinline__ void encode_d256_body(const UmmaEncode256Params &prm,
             bool ok = true;
             TileCursor cur(tile_begin, tps);
             for (int j = 0; j < n_my && ok; ++j, cur.advance(1)) {
-                const int sc = j % kAccStages;
+                const int sc = j % C::kAccStages;
                 if (j == 0) {   // all epilogue warps build the first B while the first x blocks are in flight
                     if (!wait_or_abort(smem_u32(&ctrl->b_first), 0u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT)) break;
                 } else if (cur.first_of_segment()) {   // an epilogue set rebuilds B for this lambda row
                     if (!wait_or_abort(smem_u32(&ctrl->b_ready), builds & 1u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT)) break;
                     ++builds;
                 }
-                if (!wait_or_abort(smem_u32(&ctrl->acc_empty[sc]), ((uint32_t)(j / kAccStages) & 1u) ^ 1u, abort_flag, status,
+                if (!wait_or_abort(smem_u32(&ctrl->acc_empty[sc]), ((uint32_t)(j / C::kAccStages) & 1u) ^ 1u, abort_flag, status,
                                    KVQ_DEV_SLOT_TIMEOUT))
                     break;
-                const uint32_t d_tmem = tmem_base + (uint32_t)sc * kHalfN;
+                const uint32_t d_tmem = tmem_base + (uint32_t)sc * C::kAccStride;
 #pragma unroll
                 for (int kb = 0; kb < kKBlocks; ++kb) {
                     const int u = kKBlocks * j + kb, s = u % kRing;
@@ -292,12 +300,12 @@ __device__ __forceinline__ void encode_d256_body(const UmmaEncode256Params &prm,
                     tc_fence_after();
                     const uint32_t a_lo_s = a_lo + (uint32_t)s * (kBlockBytes >> 4);
 #pragma unroll
-                    for (int t = 0; t < C::kSplit; ++t) {
+                    for (int t = 0; t < (C::kStack ? 1 : C::kSplit); ++t) {   // stacked terms: one MMA per K-step computes both
 #pragma unroll
                         for (int ks = 0; ks < 4; ++ks) {   // the four K steps of this block
                             const uint64_t ad = ((uint64_t)a_hi << 32) | (uint64_t)(a_lo_s + (uint32_t)ks * 2u);
                             const uint64_t bd = ((uint64_t)b_hi << 32) |
-                                                (uint64_t)(b_lo + (uint32_t)t * (kBTerm >> 4) + (uint32_t)kb * (kBBlock >> 4) + (uint32_t)ks * 2u);
+                                                (uint64_t)(b_lo + (uint32_t)t * (C::kBTerm >> 4) + (uint32_t)kb * (C::kBBlock >> 4) + (uint32_t)ks * 2u);
                             if (kb > 0 || t > 0 || ks > 0) umma_f16_ss<true>(d_tmem, ad, bd, C::kIdesc);
                             else umma_f16_ss<false>(d_tmem, ad, bd, C::kIdesc);
                         }
@@ -318,6 +326,20 @@ __device__ __forceinline__ void encode_d256_body(const UmmaEncode256Params &prm,
         const int bw = (warp - 2) & 7;          // position within the set: 16 rows of B per warp when the set rebuilds B
         const int g0 = 2 * h;                   // this thread's groups within the CTA's four: g0, g0 + 1
         const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16);
+        // Group g (of this CTA's four) of this thread's row of accumulator stage sc; with stacked terms the sum of the two
+        // terms' columns.
+        auto load_group = [&](int sc, int g, uint32_t (&vb)[32]) {
+            tmem_ld32(t_addr + (uint32_t)sc * C::kAccStride + (uint32_t)(g * kGroup), vb);
+            if constexpr (C::kStack) {
+                uint32_t lo[32];
+                tmem_ld32(t_addr + (uint32_t)sc * C::kAccStride + (uint32_t)(kHalfN + g * kGroup), lo);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) vb[i] = __float_as_uint(__uint_as_float(vb[i]) + __uint_as_float(lo[i]));
+            } else {
+                tmem_ld_wait();
+            }
+        };
         int64_t cached_seg = -1;
         float unlift = 1.0f;
         if (n_my > 0) {   // B for the CTA's first lambda row: D / 16 rows per warp, all sixteen warps
@@ -345,7 +367,7 @@ __device__ __forceinline__ void encode_d256_body(const UmmaEncode256Params &prm,
                 const float *lam = CALIB ? nullptr : prm.lambda + (prm.n_lambda == 1 ? 0 : seg) * kD;
                 const float lift = lift_of<kD>(lam, prm.table_max, lane);
                 if (j > 0 && cur.first_of_segment()) {
-                    if (!wait_or_abort(smem_u32(&ctrl->acc_full[(j - 1) % kAccStages]), (uint32_t)((j - 1) / kAccStages) & 1u,
+                    if (!wait_or_abort(smem_u32(&ctrl->acc_full[(j - 1) % C::kAccStages]), (uint32_t)((j - 1) / C::kAccStages) & 1u,
                                        abort_flag, status, KVQ_DEV_MMA_TIMEOUT))
                         break;
                     build_b_rows<BF16, CALIB>(sB, prm.e0, lam, lift, half, bw * 16, (bw + 1) * 16, lane);
@@ -357,8 +379,8 @@ __device__ __forceinline__ void encode_d256_body(const UmmaEncode256Params &prm,
                 cached_seg = seg;
             }
 
-            const int sc = j % kAccStages;
-            if (!wait_or_abort(smem_u32(&ctrl->acc_full[sc]), (uint32_t)(j / kAccStages) & 1u, abort_flag, status, KVQ_DEV_MMA_TIMEOUT)) break;
+            const int sc = j % C::kAccStages;
+            if (!wait_or_abort(smem_u32(&ctrl->acc_full[sc]), (uint32_t)(j / C::kAccStages) & 1u, abort_flag, status, KVQ_DEV_MMA_TIMEOUT)) break;
             tc_fence_after();
 
             // ---- rows of the tile that exist: the segment (and with it the tensor) may end inside the tile
@@ -376,8 +398,7 @@ __device__ __forceinline__ void encode_d256_body(const UmmaEncode256Params &prm,
 #pragma unroll
                 for (int gi = 0; gi < 2; ++gi) {
                     uint32_t vb[32];
-                    tmem_ld32(t_addr + (uint32_t)sc * kHalfN + (uint32_t)((g0 + gi) * kGroup), vb);
-                    tmem_ld_wait();
+                    load_group(sc, g0 + gi, vb);
 #pragma unroll
                     for (int i = 0; i < 32; ++i) m = fmaxf(m, fabsf(__uint_as_float(vb[i])));
                 }
@@ -408,8 +429,7 @@ __device__ __forceinline__ void encode_d256_body(const UmmaEncode256Params &prm,
                 const int g = g0 + gi;       // warp-uniform; group within this CTA's half
                 {
                     uint32_t vb[32];
-                    tmem_ld32(t_addr + (uint32_t)sc * kHalfN + (uint32_t)(g * kGroup), vb);
-                    tmem_ld_wait();
+                    load_group(sc, g, vb);
                     if (gi == 1) {   // this thread's last group is in registers: hand the accumulator back
                         tc_fence_before();
                         __syncwarp();
