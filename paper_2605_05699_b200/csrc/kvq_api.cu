@@ -587,8 +587,32 @@ static kvq_status_t flush_common(kvq_plan_t *plan, const void *x_block, kvq_dtyp
     prm.out_map = map;
     const bool mv = flush_decode_is_matvec(plan, N);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const cudaError_t e = mv ? matvec_decode(plan->D, plan->group, plan->bits, dtype == KVQ_BF16, N, prm, plan->d_e0, stream)
-                             : fft_decode(plan->D, plan->group, plan->bits, dtype == KVQ_BF16, N, prm, stream);
+    const bool bf16 = dtype == KVQ_BF16;
+    // A large block of a plan without a rotation: the tensor-core decode, reading and writing the window [pos0, pos0 + rows)
+    // of every stream's cache in place through a cache view (tiles of 128 rows per stream, so blocks of 64 rows and more;
+    // the whole cache must fit 32-bit tensor-map coordinates).
+    if (!mv && plan->dec_impl != KVQ_IMPL_FFT && gemm_decode_ok(plan, bf16) && (rows >= 64 || plan->dec_impl == KVQ_IMPL_GEMM) &&
+        S <= (((int64_t)1 << 31) - 1) / T_max) {
+        GemmParams g;
+        g.packed = packed_cache;
+        g.scales = scales_cache;
+        g.lambda = lambda;
+        g.out = dq_cache;
+        g.b0 = plan->d_b0;
+        g.N = N;
+        g.n_lambda = n_lambda;
+        g.rows_per_lambda = rpl;
+        g.per_vector = plan->group == plan->D;
+        g.status = plan->d_status;
+        g.view = CacheView{rows, T_max, pos0, streams_per_lambda < 1 ? 1 : streams_per_lambda};
+        if (umma_decode(plan->D, bf16, plan->bits, N, g, plan->sign_xor, stream, true) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return KVQ_ERR_CUDA;
+        }
+        return KVQ_OK;
+    }
+    const cudaError_t e = mv ? matvec_decode(plan->D, plan->group, plan->bits, bf16, N, prm, plan->d_e0, stream)
+                             : fft_decode(plan->D, plan->group, plan->bits, bf16, N, prm, stream);
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
         return KVQ_ERR_CUDA;

@@ -39,7 +39,7 @@ __device__ __forceinline__ bool lambda_row_is_wide(const float *__restrict__ lam
 // the CTA calls it with the same arguments; `su` is shared-memory scratch of 32 * D floats.  A thread owns one output
 // channel n and eight rows at a time; the table row b0[n][.] streams from L2.
 template <int D, bool BF16OUT, int BITS, int NCOLS>
-__device__ __noinline__ void decode_rows_fp32(const GemmParams &g, const float *__restrict__ lam, int64_t row0, int rows, int n0, float *su)
+__device__ __noinline__ void decode_rows_fp32(const GemmParams &g, const float *__restrict__ lam, int64_t row0 /* in memory */, int rows, int n0, float *su)
 {
     constexpr int G = D / 32, kPerThread = 8;
     const int T = (int)blockDim.x, tid = (int)threadIdx.x;
@@ -113,14 +113,14 @@ __device__ __forceinline__ void redo_tiles_fp32(const GemmParams &g, int64_t til
     float rho = 1.0f;
     for (int j = 0; j < n_my; ++j) {
         const int64_t t = tile_begin + j, seg = t / tps, off = (t - seg * tps) * TILE;
-        const float *lam = g.lambda + (g.n_lambda == 1 ? 0 : seg) * D;
+        const float *lam = g.lambda + g.lambda_index(seg) * D;
         if (seg != seen) {
             seen = seg;
             wide = lambda_row_is_wide<D>(lam, lane, &rho);
         }
-        const int64_t row0 = seg * rpl + off;
+        const int64_t row0 = g.phys_row(seg, off, rpl);   // where the tile's first row lives
         int64_t rows = rpl - off < TILE ? rpl - off : TILE;
-        if (row0 + rows > g.N) rows = g.N - row0;
+        if (seg * rpl + off + rows > g.N) rows = g.N - (seg * rpl + off);   // the call's last segment may be short
         if (rows <= 0) continue;
         bool redo = wide;
         if (CHECK_SCALES && !wide) {

@@ -41,6 +41,13 @@ struct FftParams {
     uint32_t sign_xor[128];     // word m: bit 15 set if s_{2m} = -1, bit 31 set if s_{2m+1} = -1
 };
 
+// A decode whose rows live in a cache laid out [stream][T][...]: the call's N = S * rows logical rows are rows
+// [base, base + rows) of each of S streams, `stride` cache rows apart, in packed, scales and out alike; the lambda row of
+// stream s is s / streams_per_lambda.  rows == 0: the flat layout, row r at row r.
+struct CacheView {
+    int64_t rows, stride, base, streams_per_lambda;
+};
+
 // Arguments of the tcgen05 DFT-as-GEMM decode kernel (kvq_umma_decode.cu).
 struct GemmParams {
     const void *packed;    // [N, D/2] bytes
@@ -52,6 +59,16 @@ struct GemmParams {
     int64_t n_lambda, rows_per_lambda;
     int per_vector;        // one scale per vector (group = D) instead of one per 32 channels
     uint32_t *status;
+    CacheView view = {0, 0, 0, 1};   // where the rows live (the block flush decodes a window of every stream's cache)
+    // row of packed / scales / out that holds row `off` of segment `seg` (flat: segments of rows_per_segment rows back to back)
+    __host__ __device__ __forceinline__ int64_t phys_row(int64_t seg, int64_t off, int64_t rows_per_segment) const
+    {
+        return view.rows ? seg * view.stride + view.base + off : seg * rows_per_segment + off;
+    }
+    __host__ __device__ __forceinline__ int64_t lambda_index(int64_t seg) const
+    {
+        return n_lambda == 1 ? 0 : view.rows ? seg / view.streams_per_lambda : seg;
+    }
 };
 
 // tcgen05 DFT-as-GEMM kernels (kvq_umma_decode.cu, kvq_umma_encode.cu): which (D, 16-bit type) pairs are built, and the

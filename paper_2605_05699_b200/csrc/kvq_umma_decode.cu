@@ -296,6 +296,7 @@ struct UmmaDecodeParams {
     int64_t rpl;        // rows per lambda segment (N when there is one lambda row)
     int64_t n_seg;      // segments
     int64_t n_full;     // segments of exactly rpl rows, covered by the main output maps; a shorter last one uses the tail maps
+    int64_t phys_rows;  // rows of the packed / scales arrays (N, or the whole cache for a cache view)
     uint32_t flip2[32]; // radix-2 form: sign-bit masks of s_n s_{n + 64} for the output pairs (n, n + 1), n = 0, 2, .. 62
 };
 
@@ -350,7 +351,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     const int64_t tile_end = tile_begin + per_cta < n_tiles ? tile_begin + per_cta : n_tiles;
     const int n_my = tile_end > tile_begin ? (int)(tile_end - tile_begin) : 0;
     const int64_t seg_first = n_my > 0 ? tile_begin / tps : 0;
-    auto lambda_row = [&](int64_t seg) -> const float * { return prm.g.lambda + (prm.g.n_lambda == 1 ? 0 : seg) * D; };
+    auto lambda_row = [&](int64_t seg) -> const float * { return prm.g.lambda + prm.g.lambda_index(seg) * D; };
 
     // ---- B for the first tile's lambda row: the sixteen dequant and epilogue warps build D / 16 rows each while the
     // ---- producer's first loads are in flight; the mma warp waits for all of them.  Table rows and lambda are
@@ -389,7 +390,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                 const uint32_t use = (uint32_t)(j / kInStages);
                 ok = wait_or_abort(smem_u32(&ctrl->in_empty[s]), (use & 1u) ^ 1u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT);
                 if (!ok) break;
-                const int64_t row0 = cur.seg * rpl + cur.row_in_segment();
+                const int64_t row0 = prm.g.phys_row(cur.seg, cur.row_in_segment(), rpl);   // rows past the segment are read and never stored
                 const uint32_t bar = smem_u32(&ctrl->in_full[s]);
                 mbar_arrive_expect_tx(bar, C::kInBytes);
                 tma_load_2d(smem_u32(sIn + s * C::kInPitch), &maps.packed, 0, (int)row0, bar);
@@ -470,8 +471,8 @@ __global__ void __launch_bounds__(kThreads, 1)
 #pragma unroll
             for (int i = 0; i < (G + 1) / 2; ++i) sc_next[i] = 0u;
             if (j < n_my) {
-                const int64_t row = ahead.seg * rpl + ahead.row_in_segment() + r;
-                if (row < N) {
+                const int64_t row = prm.g.phys_row(ahead.seg, ahead.row_in_segment(), rpl) + r;
+                if (row < prm.phys_rows) {
                     if (prm.g.per_vector) {   // one scale per vector: the same value in every group's slot
                         const uint32_t s1 = (uint32_t)__ldg(scales + row);
 #pragma unroll
@@ -742,14 +743,18 @@ cudaError_t launch(int64_t N, const GemmParams &g, cudaStream_t stream, const ui
 
     UmmaDecodeParams prm;
     prm.g = g;
-    prm.rpl = g.n_lambda == 1 ? N : g.rows_per_lambda;
+    prm.rpl = g.view.rows ? g.view.rows : g.n_lambda == 1 ? N : g.rows_per_lambda;   // a cache view: one segment per stream
     prm.n_seg = (N + prm.rpl - 1) / prm.rpl;
     prm.n_full = N / prm.rpl;
+    prm.phys_rows = g.view.rows ? prm.n_seg * g.view.stride : N;
+    if (prm.phys_rows >= (int64_t)1 << 31) return cudaErrorInvalidValue;
+    const int64_t seg_stride = g.view.rows ? g.view.stride : prm.rpl;   // rows from one segment's first row to the next's
+    unsigned char *out0 = static_cast<unsigned char *>(g.out) + (size_t)(g.view.rows ? g.view.base : 0) * (2 * D);
     for (int m = 0; m < 32; ++m) prm.flip2[m] = R2 && sign_xor ? sign_xor[m] ^ sign_xor[m + D / 4] : 0u;   // words hold two signs each
 
     UmmaDecodeMaps maps;
     {
-        const cuuint64_t dims[2] = {(cuuint64_t)C::kInRow, (cuuint64_t)N};
+        const cuuint64_t dims[2] = {(cuuint64_t)C::kInRow, (cuuint64_t)prm.phys_rows};
         const cuuint64_t strides[1] = {(cuuint64_t)C::kInRow};
         const cuuint32_t box[2] = {(cuuint32_t)C::kInRow, (cuuint32_t)kTile};
         const CUtensorMapSwizzle sw = C::kInSwizzleBits == 3   ? CU_TENSOR_MAP_SWIZZLE_128B
@@ -760,14 +765,14 @@ cudaError_t launch(int64_t N, const GemmParams &g, cudaStream_t stream, const ui
     }
     auto out_map = [&](CUtensorMap *tm, void *base, int64_t rows, int64_t segs, bool wide) -> bool {
         const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)rows, (cuuint64_t)segs};
-        const cuuint64_t strides[2] = {(cuuint64_t)(2 * D), (cuuint64_t)(2 * D) * (cuuint64_t)rows};
+        const cuuint64_t strides[2] = {(cuuint64_t)(2 * D), (cuuint64_t)(2 * D) * (cuuint64_t)(segs > 1 ? seg_stride : rows)};
         const cuuint32_t box[3] = {wide ? 64u : 32u, 32u, 1u};
         return make_tensor_map(tm, BF16OUT ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, base, dims, strides, box,
                                wide ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B);
     };
     const int64_t tail_rows = N - prm.n_full * prm.rpl;
-    unsigned char *tail_base = static_cast<unsigned char *>(g.out) + (size_t)prm.n_full * prm.rpl * (2 * D);
-    if (prm.n_full > 0 && (!out_map(&maps.wide, g.out, prm.rpl, prm.n_full, true) || !out_map(&maps.slim, g.out, prm.rpl, prm.n_full, false)))
+    unsigned char *tail_base = out0 + (size_t)prm.n_full * seg_stride * (2 * D);
+    if (prm.n_full > 0 && (!out_map(&maps.wide, out0, prm.rpl, prm.n_full, true) || !out_map(&maps.slim, out0, prm.rpl, prm.n_full, false)))
         return cudaErrorInvalidValue;
     if (tail_rows > 0 && (!out_map(&maps.wide_tail, tail_base, tail_rows, 1, true) || !out_map(&maps.slim_tail, tail_base, tail_rows, 1, false)))
         return cudaErrorInvalidValue;

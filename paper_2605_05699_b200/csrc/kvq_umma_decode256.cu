@@ -156,6 +156,7 @@ struct UmmaDecode256Params {
     int64_t rpl;        // rows per lambda segment (N when there is one lambda row)
     int64_t n_seg;      // segments
     int64_t n_full;     // segments of exactly rpl rows, covered by the main output map; a shorter last one uses the tail map
+    int64_t phys_rows;  // rows of the packed / scales arrays (N, or the whole cache for a cache view)
     uint32_t sign_xor[128];   // word m: bit 15 set if s_{2m} = -1, bit 31 set if s_{2m+1} = -1
 };
 
@@ -212,7 +213,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     const int64_t tile_end = tile_begin + per_cta < n_tiles ? tile_begin + per_cta : n_tiles;
     const int n_my = tile_end > tile_begin ? (int)(tile_end - tile_begin) : 0;
     const int64_t seg_first = n_my > 0 ? tile_begin / tps : 0;
-    auto lambda_row = [&](int64_t seg) -> const float * { return prm.g.lambda + (prm.g.n_lambda == 1 ? 0 : seg) * kD; };
+    auto lambda_row = [&](int64_t seg) -> const float * { return prm.g.lambda + prm.g.lambda_index(seg) * kD; };
 
     fence_proxy_async();
     tc_fence_before();
@@ -244,7 +245,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                 const int s = j % kInStages;
                 ok = wait_or_abort(smem_u32(&ctrl->in_empty[s]), ((uint32_t)(j / kInStages) & 1u) ^ 1u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT);
                 if (!ok) break;
-                const int64_t row0 = cur.seg * rpl + cur.row_in_segment();
+                const int64_t row0 = prm.g.phys_row(cur.seg, cur.row_in_segment(), rpl);   // rows past the segment are read and never stored
                 const uint32_t bar = smem_u32(&ctrl->in_full[s]);
                 mbar_arrive_expect_tx(bar, kInBytes);
                 tma_load_2d(smem_u32(sIn + s * kInBytes), &maps.packed, 0, (int)row0, bar);
@@ -307,8 +308,8 @@ __global__ void __launch_bounds__(kThreads, 1)
         TileCursor cur(tile_begin, tps), ahead(tile_begin, tps);
         auto fetch_scales = [&](int j) -> uint4 {
             if (j >= n_my) return make_uint4(0u, 0u, 0u, 0u);
-            const int64_t row = ahead.seg * rpl + ahead.row_in_segment() + r;
-            if (row >= N) return make_uint4(0u, 0u, 0u, 0u);
+            const int64_t row = prm.g.phys_row(ahead.seg, ahead.row_in_segment(), rpl) + r;
+            if (row >= prm.phys_rows) return make_uint4(0u, 0u, 0u, 0u);
             if (prm.g.per_vector) {   // one scale per vector: the same value in every group's slot
                 const uint32_t s1 = (uint32_t)__ldg(reinterpret_cast<const uint16_t *>(prm.g.scales) + row);
                 const uint32_t s2 = s1 | (s1 << 16);
@@ -500,14 +501,18 @@ cudaError_t launch(int64_t N, const GemmParams &g, const uint32_t *sign_xor, cud
 
     UmmaDecode256Params prm;
     prm.g = g;
-    prm.rpl = g.n_lambda == 1 ? N : g.rows_per_lambda;
+    prm.rpl = g.view.rows ? g.view.rows : g.n_lambda == 1 ? N : g.rows_per_lambda;   // a cache view: one segment per stream
     prm.n_seg = (N + prm.rpl - 1) / prm.rpl;
     prm.n_full = N / prm.rpl;
+    prm.phys_rows = g.view.rows ? prm.n_seg * g.view.stride : N;
+    if (prm.phys_rows >= (int64_t)1 << 31) return cudaErrorInvalidValue;
+    const int64_t seg_stride = g.view.rows ? g.view.stride : prm.rpl;   // rows from one segment's first row to the next's
+    unsigned char *out0 = static_cast<unsigned char *>(g.out) + (size_t)(g.view.rows ? g.view.base : 0) * (2 * kD);
     for (int i = 0; i < 128; ++i) prm.sign_xor[i] = sign_xor[i];
 
     UmmaDecode256Maps maps;
     {
-        const cuuint64_t dims[2] = {(cuuint64_t)(kD / 2), (cuuint64_t)N};
+        const cuuint64_t dims[2] = {(cuuint64_t)(kD / 2), (cuuint64_t)prm.phys_rows};
         const cuuint64_t strides[1] = {(cuuint64_t)(kD / 2)};
         const cuuint32_t box[2] = {(cuuint32_t)(kD / 2), (cuuint32_t)kTile};
         if (!make_tensor_map(&maps.packed, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, g.packed, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B))
@@ -515,14 +520,14 @@ cudaError_t launch(int64_t N, const GemmParams &g, const uint32_t *sign_xor, cud
     }
     auto out_map = [&](CUtensorMap *tm, void *base, int64_t rows, int64_t segs) -> bool {
         const cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)rows, (cuuint64_t)segs};
-        const cuuint64_t strides[2] = {(cuuint64_t)(2 * kD), (cuuint64_t)(2 * kD) * (cuuint64_t)rows};
+        const cuuint64_t strides[2] = {(cuuint64_t)(2 * kD), (cuuint64_t)(2 * kD) * (cuuint64_t)(segs > 1 ? seg_stride : rows)};
         const cuuint32_t box[3] = {32u, 32u, 1u};
         return make_tensor_map(tm, BF16OUT ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, base, dims, strides, box,
                                CU_TENSOR_MAP_SWIZZLE_64B);
     };
     const int64_t tail_rows = N - prm.n_full * prm.rpl;
-    unsigned char *tail_base = static_cast<unsigned char *>(g.out) + (size_t)prm.n_full * prm.rpl * (2 * kD);
-    if (prm.n_full > 0 && !out_map(&maps.out, g.out, prm.rpl, prm.n_full)) return cudaErrorInvalidValue;
+    unsigned char *tail_base = out0 + (size_t)prm.n_full * seg_stride * (2 * kD);
+    if (prm.n_full > 0 && !out_map(&maps.out, out0, prm.rpl, prm.n_full)) return cudaErrorInvalidValue;
     if (tail_rows > 0 && !out_map(&maps.tail, tail_base, tail_rows, 1)) return cudaErrorInvalidValue;
     if (tail_rows == 0) maps.tail = maps.out;
     if (prm.n_full == 0) maps.out = maps.tail;

@@ -391,6 +391,13 @@ def test_append_touches_only_row_pos():
     (128, "f16", 3, 9000, 1, (8192, 64)),              # blocks long enough for the tensor-core encode
     (256, "bf16", 26, 80, 1, (33, 32, 15)),
     (96, "f16", 7, 40, 7, (5, 35)),
+    # blocks of 64 rows and more on plans without a rotation: the tensor-core decode reads and writes the window of every
+    # stream's cache in place (tiles that end inside a stream's window, lambda rows shared by several streams, a window
+    # that starts past row 0)
+    (256, "bf16", 20, 400, 3, (200, 130, 70)),
+    (160, "f16", 9, 500, 2, (300, 129)),
+    (64, "bf16", 40, 200, 5, (128, 65)),
+    (128, "bf16", 33, 260, 4, (64, 196)),
 ])
 def test_flush_block_fills_the_int4_and_the_dequantized_caches(D, dtype, S, T_max, spl, blocks):
     odt = ko.F16 if dtype == "f16" else ko.BF16
