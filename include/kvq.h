@@ -231,7 +231,8 @@ kvq_status_t kvq_append(kvq_plan_t *plan, const void *x_new /* [S, D] */, kvq_dt
  * Requires 0 <= pos0 and pos0 + rows <= T_max.  S == 0 or rows == 0 is a no-op.  One launch on the stream when
  * S * rows <= 2048 (1024 for D > 128): the matrix-vector kernel quantizes a vector, dequantizes it from the values it
  * stored and transforms it back in the same CTA.  Larger blocks take two launches (the encode as kvq_encode picks it,
- * then a decode of the stored rows).  The
+ * then a decode of the stored rows, in place on the caches: the tensor-core kernel for blocks of 64 rows and more on a
+ * plan without a rotation, the matrix-vector kernel on rotated plans, else the register FFT).  The
  * window itself (holding the not yet flushed tokens in fp16) is the caller's buffer: this call is its flush.
  */
 kvq_status_t kvq_flush_block(kvq_plan_t *plan, const void *x_block, kvq_dtype_t dtype, int64_t S, int64_t rows,
