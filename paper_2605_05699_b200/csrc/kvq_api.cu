@@ -154,6 +154,7 @@ static bool gemm_encode_ok(const kvq_plan *p, bool bf16)
 }
 static bool gemm_decode_ok(const kvq_plan *p, bool bf16)
 {
+    if (p->bits == 8 && p->D == 256 && p->rot) return false;   // the dense D = 256 kernel of rotated plans has no byte-code form
     return p->bits == 8 ? umma_decode_bits8_supported(p->D, bf16) : umma_decode_supported(p->D, bf16);
 }
 

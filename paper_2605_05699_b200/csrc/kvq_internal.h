@@ -83,7 +83,7 @@ cudaError_t umma_decode(int D, bool bf16, int bits, int64_t N, const GemmParams 
 cudaError_t umma_calibrate(int D, bool bf16, int64_t N, const FftParams &prm, const float *e0, uint32_t *amax_bits, cudaStream_t stream);
 cudaError_t umma_calibrate_d256(bool bf16, int64_t N, const FftParams &prm, const float *e0, uint32_t *amax_bits, cudaStream_t stream);
 cudaError_t umma_encode_d256(bool bf16, bool per_vector, int64_t N, const FftParams &prm, const float *e0, cudaStream_t stream);   // kvq_umma_encode256.cu
-cudaError_t umma_decode_d256(bool bf16, int64_t N, const GemmParams &prm, const uint32_t *sign_xor, cudaStream_t stream);   // kvq_umma_decode256.cu
+cudaError_t umma_decode_d256(bool bf16, int bits, int64_t N, const GemmParams &prm, const uint32_t *sign_xor, cudaStream_t stream);   // kvq_umma_decode256.cu
 cudaError_t umma_decode_d256_dense(bool bf16, int64_t N, const GemmParams &prm, cudaStream_t stream);   // kvq_umma_decode256_dense.cu: any table
 bool umma_encode_per_vector_supported(int D, bool bf16);
 bool umma_encode_bits8_supported(int D, bool bf16);

@@ -794,8 +794,8 @@ bool umma_decode_supported(int D, bool bf16)
     return D == 256 || D == 64 || D == 96 || D == 128 || D == 160;
 }
 
-// byte codes: the D <= 160 kernel only (D <= 128 with bf16 output)
-bool umma_decode_bits8_supported(int D, bool bf16) { return D != 256 && !(D == 160 && bf16) && umma_decode_supported(D, bf16); }
+// byte codes: every kernel but the D = 160 bf16 form (and the dense D = 256 kernel of rotated plans, which the caller excludes)
+bool umma_decode_bits8_supported(int D, bool bf16) { return !(D == 160 && bf16) && umma_decode_supported(D, bf16); }
 
 cudaError_t umma_decode(int D, bool bf16, int bits, int64_t N, const GemmParams &g, const uint32_t *sign_xor, cudaStream_t stream,
                         bool radix2)
@@ -803,6 +803,7 @@ cudaError_t umma_decode(int D, bool bf16, int bits, int64_t N, const GemmParams 
     // the radix-2 form needs the transform's even / odd structure: the caller asks for it on plans without a rotation
     if (radix2 && D == 128 && bits == 4 && sign_xor)
         return bf16 ? launch<128, true, 4, true>(N, g, stream, sign_xor) : launch<128, false, 4, true>(N, g, stream, sign_xor);
+    if (D == 256 && sign_xor) return umma_decode_d256(bf16, bits, N, g, sign_xor, stream);   // its own kernel: radix-2 split, split operands for bf16
     if (bits == 8) {
         switch (D) {
             case 64: return bf16 ? launch<64, true, 8>(N, g, stream) : launch<64, false, 8>(N, g, stream);
@@ -812,7 +813,6 @@ cudaError_t umma_decode(int D, bool bf16, int bits, int64_t N, const GemmParams 
         }
         return cudaErrorInvalidValue;
     }
-    if (D == 256) return umma_decode_d256(bf16, N, g, sign_xor, stream);   // its own kernel: radix-2 split, split operands for bf16
     switch (D) {
         case 64: return bf16 ? launch<64, true>(N, g, stream) : launch<64, false>(N, g, stream);
         case 96: return bf16 ? launch<96, true>(N, g, stream) : launch<96, false>(N, g, stream);

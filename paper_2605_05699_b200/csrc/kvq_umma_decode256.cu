@@ -46,7 +46,6 @@ constexpr int kTile = 128;       // vectors per tile = MMA M
 constexpr int kHalf = 128;       // outputs n < 128 per GEMM = MMA N; also K of each GEMM (channels of one parity)
 constexpr int kThreads = 576;    // producer, mma, 2 x 4 dequant, 8 epilogue warps
 constexpr int kMaxInStages = 4;
-constexpr int kInBytes = kTile * (kD / 2);             // 16 KB
 constexpr int kBBlock = kHalf * 128;                   // one K block of 64: 128 rows x 128 B
 constexpr int kBPart = 2 * kBBlock;                    // 32 KB: one parity of one term, K = 128
 constexpr int kOutWarpBytes = 2 * 2 * 32 * 64;         // per epilogue warp: two chunks x two [32 rows][64 B] boxes
@@ -55,12 +54,17 @@ constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kACol0 = 256;                       // accumulator E at 0, O at 128; A of parity p at 256 + 128 p (hi, then lo)
 constexpr uint32_t kIdesc = umma_idesc_m128(kHalf, false);
 
-template <bool BF16OUT>
+// BITS = 8: byte codes (Sec. 3.2 step 4's int8 output).  A packed row is then 256 B, loaded as two boxes of 128 B.
+template <bool BF16OUT, int BITS = 4>
 struct Cfg {
+    static constexpr int kInRow = kD * BITS / 8;       // bytes of a packed row
+    static constexpr int kInBytes = kTile * kInRow;    // 16 KB (32 KB for byte codes)
     static constexpr int kTerms = BF16OUT ? 2 : 1;     // fp16 terms per operand
     static constexpr int kAStages = BF16OUT ? 1 : 2;   // per parity: 128 columns hold a_hi | a_lo, or two stages of a_hi
     static constexpr int kBBytes = kTerms * 2 * kBPart;
-    static constexpr int kInStages = BF16OUT ? 2 : 4;  // packed tiles in flight (16 KB each): what the split B leaves room for
+    // packed tiles in flight: what the split B and the 64 KB of output staging leave room for (byte codes with bf16 output:
+    // one 32 KB tile, reloaded while the MMAs and the epilogue of the tile before run)
+    static constexpr int kInStages = BITS == 8 ? (BF16OUT ? 1 : 2) : BF16OUT ? 2 : 4;
     // per-row output scales of the tiles between a dequant group and the epilogue: as many slots as a group can run ahead
     static constexpr int kScaleSlots = 2 * kAStages;
     static constexpr int kScaleBytes = kScaleSlots * kTile * (int)sizeof(float);
@@ -165,12 +169,12 @@ struct UmmaDecode256Maps {
     CUtensorMap out, tail;    // output, boxes of 32 columns x 32 rows (64-byte swizzle)
 };
 
-template <bool BF16OUT>
+template <bool BF16OUT, int BITS>
 __global__ void __launch_bounds__(kThreads, 1)
     kvq_decode_umma_d256_kernel(const __grid_constant__ UmmaDecode256Params prm, const __grid_constant__ UmmaDecode256Maps maps)
 {
-    using C = Cfg<BF16OUT>;
-    constexpr int kTerms = C::kTerms, kInStages = C::kInStages;
+    using C = Cfg<BF16OUT, BITS>;
+    constexpr int kTerms = C::kTerms, kInStages = C::kInStages, kInBytes = C::kInBytes;
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     unsigned char *sB = smem;                           // [term][parity][2 K blocks][128 rows][128 B]
@@ -249,6 +253,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                 const uint32_t bar = smem_u32(&ctrl->in_full[s]);
                 mbar_arrive_expect_tx(bar, kInBytes);
                 tma_load_2d(smem_u32(sIn + s * kInBytes), &maps.packed, 0, (int)row0, bar);
+                if constexpr (BITS == 8) tma_load_2d(smem_u32(sIn + s * kInBytes + kInBytes / 2), &maps.packed, 128, (int)row0, bar);   // bytes 128 .. 255 of the rows
                 issued = j + 1;
             }
             if (!ok) {
@@ -343,14 +348,14 @@ __global__ void __launch_bounds__(kThreads, 1)
             // ---- this tile's packed rows have landed
             const int s = j % kInStages;
             if (!wait_or_abort(smem_u32(&ctrl->in_full[s]), (uint32_t)(j / kInStages) & 1u, abort_flag, status, KVQ_DEV_LOAD_TIMEOUT)) break;
-            uint4 pk[kG];
-            {
-                const unsigned char *row = sIn + s * kInBytes + r * 128;
+            uint4 pk[BITS == 4 ? kG : 1];
+            const unsigned char *row = sIn + s * kInBytes + r * 128;
+            if constexpr (BITS == 4) {
 #pragma unroll
                 for (int c = 0; c < kG; ++c) pk[c] = *reinterpret_cast<const uint4 *>(row + ((c ^ (r & 7)) << 4));
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctrl->in_empty[s]));   // the values are in registers
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&ctrl->in_empty[s]));   // the values are in registers
 
             // ---- the operand stage is free again (the MMAs of the tile that used it last are complete)
             if (!wait_or_abort(smem_u32(&ctrl->a_empty[p][sa]), ((uint32_t)(j / C::kAStages) & 1u) ^ 1u, abort_flag, status, KVQ_DEV_MMA_TIMEOUT))
@@ -361,7 +366,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             // ---- in fp32; every other row has the factor 1 and costs the epilogue nothing.  Both parity groups see the
             // ---- same scales and take the same factor; group 0 posts it.
             float inv;
-            const float pw = operand_rescue<kG>(sc, rho, 9000.0f, inv);
+            const float pw = operand_rescue<kG>(sc, rho, BITS == 4 ? 9000.0f : 500.0f, inv);   // 7 (127) times this stays inside fp16
             if (p == 0) row_scale[(j % C::kScaleSlots) * kTile + r] = inv;
             const uint32_t a_row = tmem_base + ((uint32_t)(q * 32) << 16) + kACol0 + (uint32_t)p * 128u + (uint32_t)sa * 64u;
             const __half2 h1032 = __float2half2_rn(1032.0f);
@@ -369,26 +374,55 @@ __global__ void __launch_bounds__(kThreads, 1)
             for (int c = 0; c < kG; ++c) {   // group c: 16 codes of this parity, 8 tensor-memory columns
                 const float sig = __half2float(__ushort_as_half((unsigned short)((sc[c >> 1] >> (16 * (c & 1))) & 0xFFFFu)));
                 const __half2 s2 = __float2half2_rn(sig * rho * pw);
-                const uint32_t words[4] = {pk[c].x, pk[c].y, pk[c].z, pk[c].w};
                 uint32_t a_hi[8], a_lo[8];
+                auto put = [&](int k, __half2 qq) {   // K pair k of the group: one rounding, and what it left behind
+                    const __half2 hi = __hmul2(qq, s2);
+                    a_hi[k] = *reinterpret_cast<const uint32_t *>(&hi);
+                    if constexpr (kTerms == 2) {
+                        const __half2 lo = __hfma2(qq, s2, __hneg2(hi));   // q s - hi: exact, the product has 15 (byte codes: 18) bits
+                        a_lo[k] = *reinterpret_cast<const uint32_t *>(&lo);
+                    }
+                };
+                if constexpr (BITS == 4) {
+                    const uint32_t words[4] = {pk[c].x, pk[c].y, pk[c].z, pk[c].w};
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const uint32_t w = (words[i] ^ 0x88888888u) >> (4 * p);   // nibbles hold q + 8; parity p starts at nibble p
+                    for (int i = 0; i < 4; ++i) {
+                        const uint32_t w = (words[i] ^ 0x88888888u) >> (4 * p);   // nibbles hold q + 8; parity p starts at nibble p
 #pragma unroll
-                    for (int t = 0; t < 2; ++t) {
-                        // nibbles 2t + p and 2t + p + 4 of the word: channels 8w + 2t + p and + 4, both of parity p
-                        const uint32_t m = lop3_and_or(w >> (8 * t), 0x000F000Fu, 0x64006400u);   // {1024 + n, 1024 + n'}
-                        const __half2 qq = __hsub2(*reinterpret_cast<const __half2 *>(&m), h1032);       // exact codes
-                        const __half2 hi = __hmul2(qq, s2);                                               // one rounding
-                        a_hi[2 * i + t] = *reinterpret_cast<const uint32_t *>(&hi);
-                        if constexpr (kTerms == 2) {
-                            const __half2 lo = __hfma2(qq, s2, __hneg2(hi));   // q s - hi: exact, the product has 15 bits
-                            a_lo[2 * i + t] = *reinterpret_cast<const uint32_t *>(&lo);
+                        for (int t = 0; t < 2; ++t) {
+                            // nibbles 2t + p and 2t + p + 4 of the word: channels 8w + 2t + p and + 4, both of parity p
+                            const uint32_t m = lop3_and_or(w >> (8 * t), 0x000F000Fu, 0x64006400u);   // {1024 + n, 1024 + n'}
+                            put(2 * i + t, __hsub2(*reinterpret_cast<const __half2 *>(&m), h1032));       // exact codes
+                        }
+                    }
+                } else {
+                    // group c = bytes 32 c .. 32 c + 31 of the row: two 16-byte chunks of the box that holds this half of the row.
+                    // Eight channels 8w .. 8w + 7 are two words; the pairs of parity p are bytes (p, p + 4) and (p + 2, p + 6):
+                    // the K order of the B operand.
+                    const __half2 h1152 = __float2half2_rn(1152.0f);
+                    const unsigned char *half_row = row + (c >> 2) * (kInBytes / 2);
+#pragma unroll
+                    for (int hc = 0; hc < 2; ++hc) {
+                        const uint4 pc = *reinterpret_cast<const uint4 *>(half_row + ((uint32_t)((2 * (c & 3) + hc) ^ (r & 7)) << 4));
+                        const uint32_t words[4] = {pc.x ^ 0x80808080u, pc.y ^ 0x80808080u, pc.z ^ 0x80808080u, pc.w ^ 0x80808080u};   // bytes hold q + 128
+#pragma unroll
+                        for (int i = 0; i < 2; ++i) {   // eight channels: words 2 i and 2 i + 1
+#pragma unroll
+                            for (int t = 0; t < 2; ++t) {
+                                const uint32_t sel = (uint32_t)(p + 2 * t) | ((uint32_t)(4 + p + 2 * t) << 8);   // byte p + 2t of each word, to bytes 0 and 2
+                                const uint32_t two = __byte_perm(words[2 * i], words[2 * i + 1], sel);
+                                const uint32_t m = lop3_and_or(two, 0x00FF00FFu, 0x64006400u);                  // {1024 + b, 1024 + b'}
+                                put(4 * hc + 2 * i + t, __hsub2(*reinterpret_cast<const __half2 *>(&m), h1152));   // exact codes
+                            }
                         }
                     }
                 }
                 tmem_st8(a_row + 8u * (uint32_t)c, a_hi);
                 if constexpr (kTerms == 2) tmem_st8(a_row + 64u + 8u * (uint32_t)c, a_lo);
+            }
+            if constexpr (BITS == 8) {   // the packed rows were read group by group: only now is their stage free
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctrl->in_empty[s]));
             }
             tmem_st_wait();
             tc_fence_before();
@@ -472,7 +506,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     }
     // ---- tiles of a lambda row too wide for the fp16 B operand: decoded again in fp32, over what the pipeline stored
     if (ctrl->any_wide && !*abort_flag)
-        redo_tiles_fp32<kD, BF16OUT, 4, kTile>(prm.g, tile_begin, n_my, tps, rpl, reinterpret_cast<float *>(smem));
+        redo_tiles_fp32<kD, BF16OUT, BITS, kTile>(prm.g, tile_begin, n_my, tps, rpl, reinterpret_cast<float *>(smem));
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -480,10 +514,10 @@ __global__ void __launch_bounds__(kThreads, 1)
 // ------------------------------------------------------------------------------------------------
 namespace {
 
-template <bool BF16OUT>
+template <bool BF16OUT, int BITS>
 cudaError_t launch(int64_t N, const GemmParams &g, const uint32_t *sign_xor, cudaStream_t stream)
 {
-    using C = Cfg<BF16OUT>;
+    using C = Cfg<BF16OUT, BITS>;
     static DeviceSlots slots;
     int dev = 0;
     cudaError_t e = current_device_slot(&dev);
@@ -491,7 +525,7 @@ cudaError_t launch(int64_t N, const GemmParams &g, const uint32_t *sign_xor, cud
     int &sms = slots.sms[dev];
     if (sms == 0) {
         int n = 0;
-        if ((e = cudaFuncSetAttribute(kvq_decode_umma_d256_kernel<BF16OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes)) != cudaSuccess) return e;
+        if ((e = cudaFuncSetAttribute(kvq_decode_umma_d256_kernel<BF16OUT, BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes)) != cudaSuccess) return e;
         if ((e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
         sms = n;
     }
@@ -512,9 +546,9 @@ cudaError_t launch(int64_t N, const GemmParams &g, const uint32_t *sign_xor, cud
 
     UmmaDecode256Maps maps;
     {
-        const cuuint64_t dims[2] = {(cuuint64_t)(kD / 2), (cuuint64_t)prm.phys_rows};
-        const cuuint64_t strides[1] = {(cuuint64_t)(kD / 2)};
-        const cuuint32_t box[2] = {(cuuint32_t)(kD / 2), (cuuint32_t)kTile};
+        const cuuint64_t dims[2] = {(cuuint64_t)C::kInRow, (cuuint64_t)prm.phys_rows};
+        const cuuint64_t strides[1] = {(cuuint64_t)C::kInRow};
+        const cuuint32_t box[2] = {128u, (cuuint32_t)kTile};   // 128 bytes of 128 rows: a whole nibble row, half a byte row
         if (!make_tensor_map(&maps.packed, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, g.packed, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B))
             return cudaErrorInvalidValue;
     }
@@ -534,16 +568,17 @@ cudaError_t launch(int64_t N, const GemmParams &g, const uint32_t *sign_xor, cud
 
     const int64_t tiles = prm.n_seg * ((prm.rpl + kTile - 1) / kTile);
     const int grid = (int)(tiles < sms ? tiles : sms);
-    kvq_decode_umma_d256_kernel<BF16OUT><<<grid, kThreads, C::kSmemBytes, stream>>>(prm, maps);
+    kvq_decode_umma_d256_kernel<BF16OUT, BITS><<<grid, kThreads, C::kSmemBytes, stream>>>(prm, maps);
     count_launch();
     return cudaGetLastError();
 }
 
 }  // namespace
 
-cudaError_t umma_decode_d256(bool bf16, int64_t N, const GemmParams &g, const uint32_t *sign_xor, cudaStream_t stream)
+cudaError_t umma_decode_d256(bool bf16, int bits, int64_t N, const GemmParams &g, const uint32_t *sign_xor, cudaStream_t stream)
 {
-    return bf16 ? launch<true>(N, g, sign_xor, stream) : launch<false>(N, g, sign_xor, stream);
+    if (bits == 8) return bf16 ? launch<true, 8>(N, g, sign_xor, stream) : launch<false, 8>(N, g, sign_xor, stream);
+    return bf16 ? launch<true, 4>(N, g, sign_xor, stream) : launch<false, 4>(N, g, sign_xor, stream);
 }
 
 }  // namespace kvq

@@ -157,7 +157,7 @@ def test_gemm_encode_serves_large_appends():
 
 
 def test_gemm_kernels_are_refused_where_they_are_not_built():
-    for D, dtype, nbits in [(160, torch.bfloat16, 8), (256, torch.float16, 8)]:
+    for D, dtype, nbits in [(160, torch.bfloat16, 8)]:
         plan = kb.Plan(D, G, 1, nbits)
         kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_AUTO, kb.KVQ_IMPL_GEMM)
         pk, sc = plan.empty_packed(8), plan.empty_scales(8)
@@ -697,9 +697,10 @@ def test_small_calls_take_the_matvec_kernels_and_agree_with_the_fft():
 ])
 @pytest.mark.parametrize("impl", ["fft", "matvec", "gemm"])
 def test_base_variants_per_vector_scale_and_byte_codes(D, dtype, per_vector, nbits, impl):
-    if impl == "gemm" and ((D == 256 and nbits == 8) or (D == 160 and dtype == "bf16")):
+    if impl == "gemm" and D == 160 and dtype == "bf16":
         pytest.skip("no tensor-core kernel for this layout: covered by the refusal test")
-    enc_impl = impl
+    # byte codes at D = 256: the tensor cores decode them, the encode stays on the register FFT
+    enc_impl = "fft" if impl == "gemm" and D == 256 and nbits == 8 else impl
     N, n_lambda, rpl = 5003, 3, 1700          # ragged, lambda rows straddle the warps' tiles
     group = D if per_vector else G
     odt = ko.F16 if dtype == "f16" else ko.BF16
@@ -721,6 +722,30 @@ def test_base_variants_per_vector_scale_and_byte_codes(D, dtype, per_vector, nbi
     parity.check_encode(pk, sb, ora, group, "variant encode", bits=nbits)
     ob, o64 = ko.decode(pk, sb, sg, lam.numpy(), group, odt, rpl, want_f64=True, bits=nbits)
     parity.check_decode(bits(out), ob, o64, odt, "variant decode")
+    plan.close()
+
+
+@pytest.mark.parametrize("dtype,per_vector", [("f16", False), ("bf16", False), ("bf16", True)])
+def test_byte_codes_at_d256_decode_on_the_tensor_cores(dtype, per_vector):
+    """8-bit codes (Sec. 3.2 step 4's int8 output) at D = 256 through the radix-2 tensor-core decode: rows of 256 bytes loaded
+    as two boxes, bytes routed by channel parity; several CTAs, lambda rows that end inside tiles, AUTO and forced."""
+    D, N, n_lambda, rpl = 256, 21000, 5, 4300
+    group = D if per_vector else G
+    odt = DT[dtype]
+    plan = kb.Plan(D, group, 300, bits=8)
+    sg = plan.signs()
+    lam = wl.make_lambda(n_lambda, D, 301)
+    x = wl.make_vectors(N, D, dtype, "k_outlier", 302)
+    ora = ko.encode(bits(x), odt, sg, lam.numpy(), group, rpl, want_v=True, bits=8)
+    ob, o64 = ko.decode(ora["packed"], ora["scales"], sg, lam.numpy(), group, odt, rpl, want_f64=True, bits=8)
+    pk = torch.from_numpy(ora["packed"]).cuda()
+    sc = torch.from_numpy(ora["scales"].view(np.int16)).view(torch.float16).cuda()
+    for impl in (kb.KVQ_IMPL_GEMM, kb.KVQ_IMPL_AUTO):
+        kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_AUTO, impl)
+        n0 = kb.kvq_launch_count()
+        out = gpu_decode_raw(plan, pk, sc, lam.cuda(), dtype, rpl)
+        assert kb.kvq_launch_count() - n0 == 1
+        parity.check_decode(bits(out), ob, o64, odt, "byte codes, D = 256, tensor-core decode")
     plan.close()
 
 
@@ -771,11 +796,14 @@ def test_base_variants_append_and_flush_and_refusals():
     pk32, sb32 = packed[:, :32].reshape(-1, D).cpu().numpy(), bits(scales[:, :32].reshape(-1, 1))
     ob, o64 = ko.decode(pk32, sb32, sg, lam.numpy(), D, ko.F16, 32, want_f64=True, bits=8)
     parity.check_decode(bits(dq[:, :32].reshape(-1, D)), ob, o64, ko.F16, "variant dequantized cache")
-    # the tensor-core kernels do not serve byte codes at D = 256
+    # byte codes at D = 256: the tensor cores decode them (the flushed rows: the same values as the dequantized cache up to
+    # the families' rounding), but have no encode for them
     kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_GEMM, kb.KVQ_IMPL_GEMM)
-    o = torch.empty(S * T, D, dtype=torch.float16, device="cuda")
-    with pytest.raises(kb.KvqError):
-        kb.kvq_decode(plan.handle, packed.view(-1, D), scales.view(-1, 1), lamd, o, T)
+    o = torch.empty(S * 32, D, dtype=torch.float16, device="cuda")
+    kb.kvq_decode(plan.handle, packed[:, :32].reshape(-1, D).contiguous(), scales[:, :32].reshape(-1, 1).contiguous(), lamd, o, 32)
+    torch.cuda.synchronize()
+    assert kb.kvq_plan_device_status(plan.handle) == 0
+    parity.check_decode(bits(o), ob, o64, ko.F16, "variant cache, tensor-core decode")
     with pytest.raises(kb.KvqError):
         kb.kvq_encode(plan.handle, x.reshape(-1, D).cuda(), lamd, packed.view(-1, D), scales.view(-1, 1), T)
     plan.close()
