@@ -62,8 +62,8 @@ typedef enum {
     KVQ_IMPL_FFT = 1,   /* fp32 register FFT, one thread per vector: every D, dtype and layout; no rotation */
     KVQ_IMPL_GEMM = 2,  /* tcgen05 DFT-as-GEMM.  bits = 4: encode / append and decode: D = 64, 96, 128, 160, 256 in fp16
                            and bf16; either group size.  bits = 8:
-                           D <= 160 in fp16, D <= 128 in bf16; at D = 256 the decode only (both types, plans
-                           without a rotation).  At most 2^31 - 1 rows per call (AUTO falls back
+                           D <= 160 in fp16, D <= 128 in bf16; at D = 256 the decode (both types, plans without
+                           a rotation) and the encode from fp16.  At most 2^31 - 1 rows per call (AUTO falls back
                            to the register FFT beyond).
                            Elsewhere the compute calls return KVQ_ERR_UNSUPPORTED_DIM. */
     KVQ_IMPL_MATVEC = 3 /* fp32 matrix-vector product with the plan's D x D table, a CTA per 8 vectors: every D, dtype
@@ -91,7 +91,7 @@ kvq_status_t kvq_plan_create(int D, int group, uint64_t seed, kvq_plan_t **out);
  *          two's-complement byte per value: `packed` rows are D bytes).
  * Everything else is as for kvq_plan_create, which is (group, bits = 4).  Wherever a comment of this header says
  * "[*, D/2] bytes" a plan with bits = 8 takes [*, D] bytes.  The tensor-core kernels serve either group size, and
- * bits = 8 up to D = 160 and for the decode at D = 256 (see KVQ_IMPL_GEMM); elsewhere such plans run on the register-FFT and matrix-vector kernels
+ * bits = 8 up to D = 160 and, encode from bf16 apart, at D = 256 (see KVQ_IMPL_GEMM); elsewhere such plans run on the register-FFT and matrix-vector kernels
  * (KVQ_IMPL_GEMM is refused with UNSUPPORTED_DIM); kvq_decode_static serves group = 32, bits = 4 only.
  */
 kvq_status_t kvq_plan_create_ex(int D, int group, int bits, uint64_t seed, kvq_plan_t **out);

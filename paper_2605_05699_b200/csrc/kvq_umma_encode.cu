@@ -633,9 +633,10 @@ bool umma_calibrate_supported(int D, bool bf16) { return umma_encode_supported(D
 // one scale per vector: the row maximum is traded inside a CTA, or across the cluster pair of the D = 256 kernel
 bool umma_encode_per_vector_supported(int D, bool bf16) { return umma_encode_supported(D, bf16); }
 
-// byte codes: the D <= 160 kernel (the code step is 18 times finer than with 4 bits: two bf16 terms of W would leave 2e-4
-// of the codes on the wrong side of a rounding, so bf16 input takes the three-term instantiation)
-bool umma_encode_bits8_supported(int D, bool bf16) { return D != 256 && !(D == 160 && bf16) && umma_encode_supported(D, bf16); }
+// byte codes: the code step is 18 times finer than with 4 bits: two bf16 terms of W would leave 2e-4 of the codes on the
+// wrong side of a rounding, so bf16 input takes the three-term instantiation (D <= 128: at D = 160 and 256 three terms leave
+// no room for x); fp16 input keeps its two terms at every D
+bool umma_encode_bits8_supported(int D, bool bf16) { return !(D == 256 && bf16) && !(D == 160 && bf16) && umma_encode_supported(D, bf16); }
 
 cudaError_t umma_encode(int D, bool bf16, bool per_vector, int64_t N, const FftParams &f, const float *e0, cudaStream_t stream)
 {

@@ -189,6 +189,7 @@ struct UmmaEncode256Params {
     float table_max;       // largest |entry| of e0
     uint32_t *status;
     uint32_t *amax_bits;        // calibration only: [D] running column maxima as fp32 bit patterns (start at zero)
+    int bits;                   // 4: nibble pairs; 8 (fp16 input): one two's-complement byte per code, scale = absmax / 127
 };
 
 template <bool BF16, bool CALIB, bool PERVEC>
@@ -388,6 +389,7 @@ __device__ __forceinline__ void encode_d256_body(const UmmaEncode256Params &prm,
             if (seg_rows > rpl) seg_rows = rpl;
             const bool live = off + r < seg_rows;
             const int64_t orow = prm.out_map(seg * rpl + off + r);
+            const float Q = prm.bits == 4 ? 7.0f : 127.0f;   // largest code (warp-uniform)
             // ---- one scale per vector: this thread's maximum over its 64 channels goes to both CTAs of the pair; the four
             // ---- parties of a row (two half-row threads in each CTA) meet on a four-arrival barrier in each CTA, once per
             // ---- tile; buffers alternate with the tile parity, so a party cannot overwrite what another still reads
@@ -416,11 +418,11 @@ __device__ __forceinline__ void encode_d256_body(const UmmaEncode256Params &prm,
                 if (!wait_cluster_or_abort(smem_u32(&ctrl->quad[set][q]), (uint32_t)it & 1u, abort_flag, status, KVQ_DEV_SLOT_TIMEOUT)) break;
                 m = fmaxf(fmaxf(slot[r], slot[kTile + r]), fmaxf(slot[2 * kTile + r], slot[3 * kTile + r]));
                 const float amax = m * unlift;
-                const float sig = fminf(__fdiv_rn(amax, 7.0f), 65504.0f);
+                const float sig = fminf(__fdiv_rn(amax, Q), 65504.0f);
                 const __half hs = __float2half_rn(sig);
                 const float sg = __half2float(hs);
                 const float rs1 = sg > 0.0f ? __frcp_rn(sg) : 0.0f;
-                row_clamp = !(amax * rs1 < 7.25f);
+                row_clamp = !(amax * rs1 < Q + 0.25f);
                 row_rs = rs1 * unlift;
                 if (live && party == 0) prm.scales[orow] = __half_as_ushort(hs);
             }
@@ -453,14 +455,39 @@ __device__ __forceinline__ void encode_d256_body(const UmmaEncode256Params &prm,
 #pragma unroll
                         for (int i = 0; i < 32; ++i) amax = fmaxf(amax, fabsf(__uint_as_float(vb[i])));
                         amax *= unlift;
-                        const float sig = fminf(__fdiv_rn(amax, 7.0f), 65504.0f);
+                        const float sig = fminf(__fdiv_rn(amax, Q), 65504.0f);
                         hs = __float2half_rn(sig);
                         const float sg = __half2float(hs);
                         const float rs1 = sg > 0.0f ? __frcp_rn(sg) : 0.0f;
-                        clamp = !(amax * rs1 < 7.25f);   // saturated or subnormal scale: codes could leave [-7, 7]
+                        clamp = !(amax * rs1 < Q + 0.25f);   // saturated or subnormal scale: codes could leave [-Q, Q]
                         rs = rs1 * unlift;               // applies to the lifted accumulator values
                     }
 
+                    const int gg = 4 * half + g;   // group within the row
+                    if (prm.bits == 8) {   // ---- round, bias to unsigned bytes, pack 4 codes per word
+                        uint32_t words[8];
+#pragma unroll
+                        for (int w = 0; w < 8; ++w) {
+                            uint32_t acc = 0;
+                            if (!clamp) {
+#pragma unroll
+                                for (int e = 0; e < 4; ++e)
+                                    acc += __float_as_uint(fmaf(__uint_as_float(vb[4 * w + e]), rs, kMagicRound8)) << (8 * e);
+                            } else {
+#pragma unroll
+                                for (int e = 0; e < 4; ++e)
+                                    acc += __float_as_uint(fminf(fmaxf(__uint_as_float(vb[4 * w + e]) * rs, -127.0f), 127.0f) + kMagicRound8) << (8 * e);
+                            }
+                            words[w] = (acc - kMagicSum8) ^ 0x80808080u;
+                        }
+                        if (live) {
+                            uint4 *dst = reinterpret_cast<uint4 *>(prm.packed + orow * kD + gg * 32);
+                            dst[0] = make_uint4(words[0], words[1], words[2], words[3]);
+                            dst[1] = make_uint4(words[4], words[5], words[6], words[7]);
+                            if constexpr (!PERVEC) prm.scales[orow * kG + gg] = __half_as_ushort(hs);
+                        }
+                        continue;
+                    }
                     // ---- round, bias to unsigned nibbles, pack 8 codes per word
                     uint32_t words[4];
 #pragma unroll
@@ -478,7 +505,6 @@ __device__ __forceinline__ void encode_d256_body(const UmmaEncode256Params &prm,
                         words[w] = (acc - kMagicSum) ^ 0x88888888u;
                     }
                     if (live) {
-                        const int gg = 4 * half + g;   // group within the row
                         *reinterpret_cast<uint4 *>(prm.packed + orow * (kD / 2) + gg * 16) = make_uint4(words[0], words[1], words[2], words[3]);
                         if constexpr (!PERVEC) prm.scales[orow * kG + gg] = __half_as_ushort(hs);
                     }
@@ -579,6 +605,7 @@ cudaError_t launch(int64_t N, const FftParams &f, const float *e0, cudaStream_t 
     prm.table_max = f.table_max;
     prm.status = f.status;
     prm.amax_bits = amax_bits;
+    prm.bits = f.bits;
 
     CUtensorMap tm_x;
     const cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)N};

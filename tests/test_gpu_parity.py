@@ -166,7 +166,7 @@ def test_gemm_kernels_are_refused_where_they_are_not_built():
             kb.kvq_decode(plan.handle, pk, sc, torch.ones(D, device="cuda"), out)
         assert e.value.status == kb.KVQ_ERR_UNSUPPORTED_DIM
         plan.close()
-    for D, dtype, nbits in [(160, torch.bfloat16, 8), (256, torch.float16, 8)]:     # byte codes: three-term B does not fit
+    for D, dtype, nbits in [(160, torch.bfloat16, 8), (256, torch.bfloat16, 8)]:     # byte codes from bf16: a three-term B does not fit
         plan = kb.Plan(D, G, 1, nbits)
         kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_GEMM, kb.KVQ_IMPL_AUTO)
         x = torch.zeros(8, D, dtype=dtype, device="cuda")
@@ -699,8 +699,8 @@ def test_small_calls_take_the_matvec_kernels_and_agree_with_the_fft():
 def test_base_variants_per_vector_scale_and_byte_codes(D, dtype, per_vector, nbits, impl):
     if impl == "gemm" and D == 160 and dtype == "bf16":
         pytest.skip("no tensor-core kernel for this layout: covered by the refusal test")
-    # byte codes at D = 256: the tensor cores decode them, the encode stays on the register FFT
-    enc_impl = "fft" if impl == "gemm" and D == 256 and nbits == 8 else impl
+    # byte codes at D = 256: the tensor cores decode them and encode them from fp16; from bf16 the encode stays on the register FFT
+    enc_impl = "fft" if impl == "gemm" and D == 256 and nbits == 8 and dtype == "bf16" else impl
     N, n_lambda, rpl = 5003, 3, 1700          # ragged, lambda rows straddle the warps' tiles
     group = D if per_vector else G
     odt = ko.F16 if dtype == "f16" else ko.BF16
@@ -746,6 +746,10 @@ def test_byte_codes_at_d256_decode_on_the_tensor_cores(dtype, per_vector):
         out = gpu_decode_raw(plan, pk, sc, lam.cuda(), dtype, rpl)
         assert kb.kvq_launch_count() - n0 == 1
         parity.check_decode(bits(out), ob, o64, odt, "byte codes, D = 256, tensor-core decode")
+    if dtype == "f16":   # the tensor-core encode takes byte codes from fp16 input (two fp16 terms of W carry 22 bits)
+        kb.kvq_plan_set_impl(plan.handle, kb.KVQ_IMPL_GEMM, kb.KVQ_IMPL_AUTO)
+        packed, scales = gpu_encode(plan, x.cuda(), lam.cuda(), rpl)
+        parity.check_encode(packed.cpu().numpy(), bits(scales), ora, group, "byte codes, D = 256, tensor-core encode", bits=8)
     plan.close()
 
 
@@ -804,8 +808,15 @@ def test_base_variants_append_and_flush_and_refusals():
     torch.cuda.synchronize()
     assert kb.kvq_plan_device_status(plan.handle) == 0
     parity.check_decode(bits(o), ob, o64, ko.F16, "variant cache, tensor-core decode")
+    # ... and encode them from fp16 (the whole cache again, as one flat call), but not from bf16
+    p2, s2 = torch.empty(S * T, D, dtype=torch.uint8, device="cuda"), torch.empty(S * T, 1, dtype=torch.float16, device="cuda")
+    kb.kvq_encode(plan.handle, x.reshape(-1, D).cuda(), lamd, p2, s2, T)
+    torch.cuda.synchronize()
+    assert kb.kvq_plan_device_status(plan.handle) == 0
+    ora_all = ko.encode(bits(x.reshape(-1, D)), ko.F16, sg, lam.numpy(), D, T, want_v=True, bits=8)
+    parity.check_encode(p2.cpu().numpy(), bits(s2), ora_all, D, "byte codes, D = 256, tensor-core encode", bits=8, min_agree=0.9995)
     with pytest.raises(kb.KvqError):
-        kb.kvq_encode(plan.handle, x.reshape(-1, D).cuda(), lamd, packed.view(-1, D), scales.view(-1, 1), T)
+        kb.kvq_encode(plan.handle, x.reshape(-1, D).to(torch.bfloat16).cuda(), lamd, packed.view(-1, D), scales.view(-1, 1), T)
     plan.close()
     with pytest.raises(kb.KvqError):
         kb.Plan(128, 64, 1)           # groups other than 32 or D
