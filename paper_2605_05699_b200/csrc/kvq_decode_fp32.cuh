@@ -13,26 +13,17 @@
 #include <cstdint>
 
 #include "kvq_internal.h"
+#include "kvq_umma.cuh"
 
 namespace kvq {
 
-// Is the lambda row too wide for the fp16 B operand?  The same test the B builders apply, on the whole row, by one warp.
+// Is the lambda row too wide for the fp16 B operand?  The B builders' own test (RecipLambda), by one warp.
 template <int D>
 __device__ __forceinline__ bool lambda_row_is_wide(const float *__restrict__ lam, int lane, float *rho_out = nullptr)
 {
-    float mx = 0.0f, mn = 3.0e38f;
-    for (int c = lane; c < D; c += 32) {
-        const float r = __frcp_rn(fmaxf(__ldg(lam + c), 1e-6f));
-        mx = fmaxf(mx, r), mn = fminf(mn, r);
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
-        mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, o));
-    }
-    const float rho = __uint_as_float(__float_as_uint(mx) & 0x7F800000u);   // what the B builders divide the reciprocals by
-    if (rho_out) *rho_out = rho;
-    return mn < rho * 0.00390625f;
+    const RecipLambda<D> rl(lam, lane);
+    if (rho_out) *rho_out = rl.rho;   // what the B builders divide the reciprocals by
+    return rl.wide;
 }
 
 // Output channels [n0, n0 + NCOLS) of rows [row0, row0 + rows) of the call, all of one lambda row `lam`.  Every thread of

@@ -202,6 +202,24 @@ struct TileCursor {
     __device__ __forceinline__ int64_t row_in_segment() const { return tin * 128; }
 };
 
+// The contiguous share of a call's tiles that one CTA (or one CTA pair) of a persistent kernel takes: lambda segments of rpl
+// rows are cut into tiles of 128 rows (a segment's last tile may be short), n_seg * tps tiles in all, `parts` equal shares.
+// Contiguous, so that the B operand of a lambda row is rebuilt as rarely as possible.
+struct TileShare {
+    int64_t tps;     // tiles per segment
+    int64_t begin;   // first tile of this share
+    int n;           // tiles in this share
+    __device__ __forceinline__ TileShare(int64_t n_seg, int64_t rpl, unsigned part, unsigned parts)
+    {
+        tps = (rpl + 127) / 128;
+        const int64_t n_tiles = n_seg * tps;
+        const int64_t per = (n_tiles + parts - 1) / parts;
+        begin = (int64_t)part * per;
+        const int64_t end = begin + per < n_tiles ? begin + per : n_tiles;
+        n = end > begin ? (int)(end - begin) : 0;
+    }
+};
+
 // ---------------------------------------------------------------------------
 // half-precision words: two 16-bit values per 32-bit word, low half first
 // ---------------------------------------------------------------------------

@@ -157,6 +157,41 @@ __device__ __forceinline__ float operand_rescue(const uint32_t (&sc)[(G + 1) / 2
     return __uint_as_float((uint32_t)(127 + 7 - e) << 23);
 }
 
+// 1 / max(lambda, 1e-6) for the channels this lane covers (4 i .. 4 i + 3, i = lane and, for D > 128, lane + 32),
+// divided by rho, the power of two that brings the row's largest reciprocal into [1, 2).  Every lane gets rho.
+template <int D>
+struct RecipLambda {
+    static constexpr int kPasses = (D / 4 + 31) / 32;
+    float4 r[kPasses];
+    float rho;
+    bool wide;   // the reciprocals span more than 2^8: B, which carries them in fp16 next to each other, loses bits on the small ones
+    __device__ __forceinline__ RecipLambda(const float *__restrict__ lam, int lane)
+    {
+        float mx = 0.0f, mn = 3.0e38f;
+#pragma unroll
+        for (int p = 0; p < kPasses; ++p) {
+            const int i = lane + 32 * p;
+            r[p] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            if (i < D / 4) {
+                const float4 l = __ldg(reinterpret_cast<const float4 *>(lam) + i);
+                r[p] = make_float4(__frcp_rn(fmaxf(l.x, 1e-6f)), __frcp_rn(fmaxf(l.y, 1e-6f)), __frcp_rn(fmaxf(l.z, 1e-6f)),
+                                   __frcp_rn(fmaxf(l.w, 1e-6f)));
+            }
+            mx = fmaxf(mx, fmaxf(fmaxf(r[p].x, r[p].y), fmaxf(r[p].z, r[p].w)));
+            if (i < D / 4) mn = fminf(mn, fminf(fminf(r[p].x, r[p].y), fminf(r[p].z, r[p].w)));
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+            mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, o));
+        }
+        rho = __uint_as_float(__float_as_uint(mx) & 0x7F800000u);   // 2^floor(log2 max): exact to divide by
+        wide = mn < rho * 0.00390625f;
+#pragma unroll
+        for (int p = 0; p < kPasses; ++p) r[p].x /= rho, r[p].y /= rho, r[p].z /= rho, r[p].w /= rho;
+    }
+};
+
 // Bounded wait that also gives up when another role of the CTA has raised the abort flag.  On a
 // time-out it raises the flag itself and records `reason` in the status word.
 constexpr uint32_t kWaitPolls = 1u << 22;   // polls of a bounded wait before it gives up (seconds of wall time)

@@ -125,41 +125,6 @@ struct Ctrl {
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
 
-// 1 / max(lambda, 1e-6) for the channels this lane covers (4 i .. 4 i + 3, i = lane and, for D > 128, lane + 32),
-// divided by rho, the power of two that brings the row's largest reciprocal into [1, 2).  Every lane gets rho.
-template <int D>
-struct RecipLambda {
-    static constexpr int kPasses = (D / 4 + 31) / 32;
-    float4 r[kPasses];
-    float rho;
-    bool wide;   // the reciprocals span more than 2^8: B, which carries them in fp16 next to each other, loses bits on the small ones
-    __device__ __forceinline__ RecipLambda(const float *__restrict__ lam, int lane)
-    {
-        float mx = 0.0f, mn = 3.0e38f;
-#pragma unroll
-        for (int p = 0; p < kPasses; ++p) {
-            const int i = lane + 32 * p;
-            r[p] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-            if (i < D / 4) {
-                const float4 l = __ldg(reinterpret_cast<const float4 *>(lam) + i);
-                r[p] = make_float4(__frcp_rn(fmaxf(l.x, 1e-6f)), __frcp_rn(fmaxf(l.y, 1e-6f)), __frcp_rn(fmaxf(l.z, 1e-6f)),
-                                   __frcp_rn(fmaxf(l.w, 1e-6f)));
-            }
-            mx = fmaxf(mx, fmaxf(fmaxf(r[p].x, r[p].y), fmaxf(r[p].z, r[p].w)));
-            if (i < D / 4) mn = fminf(mn, fminf(fminf(r[p].x, r[p].y), fminf(r[p].z, r[p].w)));
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
-            mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, o));
-        }
-        rho = __uint_as_float(__float_as_uint(mx) & 0x7F800000u);   // 2^floor(log2 max): exact to divide by
-        wide = mn < rho * 0.00390625f;
-#pragma unroll
-        for (int p = 0; p < kPasses; ++p) r[p].x /= rho, r[p].y /= rho, r[p].z /= rho, r[p].w /= rho;
-    }
-};
-
 // Rows [n0, n1) of the B operand, by one warp: a lane reads four table entries b0[n][4 i .. 4 i + 3] (coalesced
 // rows), scales them, trades two values with its neighbour so that each lane holds two K-ordered pairs, and
 // writes 8 bytes of the swizzled row.
@@ -344,12 +309,9 @@ __global__ void __launch_bounds__(kThreads, 1)
     // ---- tiles: lambda segments of rpl rows, cut into tiles of 128 rows; a contiguous range of tiles
     // ---- per CTA, so that the B operand is rebuilt as rarely as possible
     const int64_t N = prm.g.N, rpl = prm.rpl;
-    const int64_t tps = (rpl + kTile - 1) / kTile;                 // tiles per segment
-    const int64_t n_tiles = prm.n_seg * tps;
-    const int64_t per_cta = (n_tiles + gridDim.x - 1) / gridDim.x;
-    const int64_t tile_begin = (int64_t)blockIdx.x * per_cta;
-    const int64_t tile_end = tile_begin + per_cta < n_tiles ? tile_begin + per_cta : n_tiles;
-    const int n_my = tile_end > tile_begin ? (int)(tile_end - tile_begin) : 0;
+    const TileShare share(prm.n_seg, rpl, blockIdx.x, gridDim.x);
+    const int64_t tps = share.tps, tile_begin = share.begin;
+    const int n_my = share.n;
     const int64_t seg_first = n_my > 0 ? tile_begin / tps : 0;
     auto lambda_row = [&](int64_t seg) -> const float * { return prm.g.lambda + prm.g.lambda_index(seg) * D; };
 

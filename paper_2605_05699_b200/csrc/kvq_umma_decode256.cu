@@ -85,42 +85,13 @@ struct Ctrl {
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
 
-// 1 / max(lambda, 1e-6) for the channels 4 i .. 4 i + 3, i = lane and lane + 32, divided by rho, the power of two
-// that brings the row's largest reciprocal into [1, 2).  Every lane gets rho.
-struct RecipLambda {
-    float4 r[2];
-    float rho;
-    bool wide;   // the reciprocals span more than 2^8: B, which carries them in fp16 next to each other, loses bits on the small ones
-    __device__ __forceinline__ RecipLambda(const float *__restrict__ lam, int lane)
-    {
-        float mx = 0.0f, mn = 3.0e38f;
-#pragma unroll
-        for (int p = 0; p < 2; ++p) {
-            const float4 l = __ldg(reinterpret_cast<const float4 *>(lam) + lane + 32 * p);
-            r[p] = make_float4(__frcp_rn(fmaxf(l.x, 1e-6f)), __frcp_rn(fmaxf(l.y, 1e-6f)), __frcp_rn(fmaxf(l.z, 1e-6f)),
-                               __frcp_rn(fmaxf(l.w, 1e-6f)));
-            mx = fmaxf(mx, fmaxf(fmaxf(r[p].x, r[p].y), fmaxf(r[p].z, r[p].w)));
-            mn = fminf(mn, fminf(fminf(r[p].x, r[p].y), fminf(r[p].z, r[p].w)));
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
-            mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, o));
-        }
-        rho = __uint_as_float(__float_as_uint(mx) & 0x7F800000u);   // 2^floor(log2 max): exact to divide by
-        wide = mn < rho * 0.00390625f;
-#pragma unroll
-        for (int p = 0; p < 2; ++p) r[p].x /= rho, r[p].y /= rho, r[p].z /= rho, r[p].w /= rho;
-    }
-};
-
 // Rows [n0, n1) (outputs n < 128) of the B operand of parity p (0: E GEMM, even channels; 1: O GEMM), by one warp.
 // The table row b0[n][c] = s_n M[c][n] is used as it is: the accumulators then hold s_n E_n and s_n O_n.  Lanes 2w and 2w + 1 hold
 // channels 8w .. 8w + 7; the K order inside a word is the one the nibble trick produces, pairs (c, c + 4): the even
 // lane assembles the pair (8w + p, 8w + p + 4), the odd lane (8w + p + 2, 8w + p + 6), each from one value of its
 // own and one of its neighbour's.  Terms: fp16(W'), then what that left behind.
 template <int TERMS>
-__device__ __forceinline__ void build_b_rows(unsigned char *sB, const float *__restrict__ b0, const RecipLambda &rl, int p, int n0, int n1, int lane)
+__device__ __forceinline__ void build_b_rows(unsigned char *sB, const float *__restrict__ b0, const RecipLambda<kD> &rl, int p, int n0, int n1, int lane)
 {
     const bool odd = lane & 1;
 #pragma unroll 8   // 16 row quads in flight per lane: the build is a chain of L2 round trips, not arithmetic
@@ -210,12 +181,9 @@ __global__ void __launch_bounds__(kThreads, 1)
 
     // ---- tiles: lambda segments of rpl rows, cut into tiles of 128 rows; a contiguous range of tiles per CTA
     const int64_t N = prm.g.N, rpl = prm.rpl;
-    const int64_t tps = (rpl + kTile - 1) / kTile;
-    const int64_t n_tiles = prm.n_seg * tps;
-    const int64_t per_cta = (n_tiles + gridDim.x - 1) / gridDim.x;
-    const int64_t tile_begin = (int64_t)blockIdx.x * per_cta;
-    const int64_t tile_end = tile_begin + per_cta < n_tiles ? tile_begin + per_cta : n_tiles;
-    const int n_my = tile_end > tile_begin ? (int)(tile_end - tile_begin) : 0;
+    const TileShare share(prm.n_seg, rpl, blockIdx.x, gridDim.x);
+    const int64_t tps = share.tps, tile_begin = share.begin;
+    const int n_my = share.n;
     const int64_t seg_first = n_my > 0 ? tile_begin / tps : 0;
     auto lambda_row = [&](int64_t seg) -> const float * { return prm.g.lambda + prm.g.lambda_index(seg) * kD; };
 
@@ -230,7 +198,7 @@ __global__ void __launch_bounds__(kThreads, 1)
     // ---- B for the first tile's lambda row: of the sixteen dequant and epilogue warps, eight build the E operand
     // ---- and eight the O operand, sixteen rows each
     if (n_my > 0 && warp >= 2) {
-        const RecipLambda rl(lambda_row(seg_first), lane);
+        const RecipLambda<kD> rl(lambda_row(seg_first), lane);
         if (rl.wide) ctrl->any_wide = 1u;
         const int bp = ((warp - 2) >> 2) & 1, bw = ((warp - 2) & 3) + 4 * ((warp - 2) >> 3);   // parity, position among its eight
         build_b_rows<kTerms>(sB, prm.g.b0, rl, bp, bw * 16, bw * 16 + 16, lane);
@@ -308,7 +276,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         const int r = q * 32 + lane;            // tile row and tensor-memory lane of this thread
         const uint4 *scales = static_cast<const uint4 *>(prm.g.scales);   // 8 fp16 scales per row
         int64_t cached_seg = n_my > 0 ? seg_first : -1;   // B holds this row's table (built above)
-        float rho = RecipLambda(lambda_row(seg_first), lane).rho;
+        float rho = RecipLambda<kD>(lambda_row(seg_first), lane).rho;
 
         TileCursor cur(tile_begin, tps), ahead(tile_begin, tps);
         auto fetch_scales = [&](int j) -> uint4 {
@@ -334,7 +302,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             // ---- a new lambda row: new rho, and this group rebuilds the B operand of its own GEMM once every MMA of that
             // ---- GEMM issued so far is complete: the previous tile's, on this group's own barriers (it sees every phase)
             if (seg != cached_seg) {
-                const RecipLambda rl(lambda_row(seg), lane);
+                const RecipLambda<kD> rl(lambda_row(seg), lane);
                 if (rl.wide) ctrl->any_wide = 1u;
                 rho = rl.rho;
                 if (!wait_or_abort(smem_u32(&ctrl->a_empty[p][(j - 1) % C::kAStages]), (uint32_t)((j - 1) / C::kAStages) & 1u, abort_flag,

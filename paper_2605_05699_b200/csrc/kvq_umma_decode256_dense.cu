@@ -62,41 +62,12 @@ struct Ctrl {
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block too large");
 
-// 1 / max(lambda, 1e-6) for the channels 4 i .. 4 i + 3, i = lane and lane + 32, divided by rho, the power of two
-// that brings the row's largest reciprocal into [1, 2).  Every lane gets rho.
-struct RecipLambda {
-    float4 r[2];
-    float rho;
-    bool wide;   // the reciprocals span more than 2^8: B, which carries them in fp16 next to each other, loses bits on the small ones
-    __device__ __forceinline__ RecipLambda(const float *__restrict__ lam, int lane)
-    {
-        float mx = 0.0f, mn = 3.0e38f;
-#pragma unroll
-        for (int p = 0; p < 2; ++p) {
-            const float4 l = __ldg(reinterpret_cast<const float4 *>(lam) + lane + 32 * p);
-            r[p] = make_float4(__frcp_rn(fmaxf(l.x, 1e-6f)), __frcp_rn(fmaxf(l.y, 1e-6f)), __frcp_rn(fmaxf(l.z, 1e-6f)),
-                               __frcp_rn(fmaxf(l.w, 1e-6f)));
-            mx = fmaxf(mx, fmaxf(fmaxf(r[p].x, r[p].y), fmaxf(r[p].z, r[p].w)));
-            mn = fminf(mn, fminf(fminf(r[p].x, r[p].y), fminf(r[p].z, r[p].w)));
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
-            mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, o));
-        }
-        rho = __uint_as_float(__float_as_uint(mx) & 0x7F800000u);   // 2^floor(log2 max): exact to divide by
-        wide = mn < rho * 0.00390625f;
-#pragma unroll
-        for (int p = 0; p < 2; ++p) r[p].x /= rho, r[p].y /= rho, r[p].z /= rho, r[p].w /= rho;
-    }
-};
-
 // Rows [n0, n1) of this CTA's half of the B operand (output column 128 half + n), by one warp.  A lane reads four
 // table entries per pass, scales them, trades two values with its neighbour so that each lane holds two K-ordered
 // pairs (the K order of a word of 8 codes is (0,4,1,5,2,6,3,7)), peels off fp16 terms and writes 8 bytes of each
 // term's swizzled row.
 template <int TERMS>
-__device__ __forceinline__ void build_b_rows(unsigned char *sB, const float *__restrict__ b0, const RecipLambda &rl, int half, int n0,
+__device__ __forceinline__ void build_b_rows(unsigned char *sB, const float *__restrict__ b0, const RecipLambda<kD> &rl, int half, int n0,
                                              int n1, int lane)
 {
     const bool odd = lane & 1;
@@ -182,14 +153,11 @@ __global__ void __launch_bounds__(kThreads, 1)
 
     // ---- tiles: lambda segments of rpl rows, cut into tiles of 128 rows; a contiguous range of tiles per CTA pair
     const int64_t N = prm.g.N, rpl = prm.rpl;
-    const int64_t tps = (rpl + kTile - 1) / kTile;
-    const int64_t n_tiles = prm.n_seg * tps;
-    const int64_t per_pair = (n_tiles + n_pairs - 1) / n_pairs;
-    const int64_t tile_begin = (int64_t)pair * per_pair;
-    const int64_t tile_end = tile_begin + per_pair < n_tiles ? tile_begin + per_pair : n_tiles;
-    const int n_my = tile_end > tile_begin ? (int)(tile_end - tile_begin) : 0;
+    const TileShare share(prm.n_seg, rpl, (unsigned)pair, (unsigned)n_pairs);
+    const int64_t tps = share.tps, tile_begin = share.begin;
+    const int n_my = share.n;
     const int64_t seg_first = n_my > 0 ? tile_begin / tps : 0;
-    auto lambda_row = [&](int64_t seg) -> const float * { return prm.g.lambda + (prm.g.n_lambda == 1 ? 0 : seg) * kD; };
+    auto lambda_row = [&](int64_t seg) -> const float * { return prm.g.lambda + prm.g.lambda_index(seg) * kD; };
 
     fence_proxy_async();
     tc_fence_before();
@@ -201,7 +169,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 
     // ---- B for the first tile's lambda row: the sixteen dequant and epilogue warps build eight rows each
     if (n_my > 0 && warp >= 2) {
-        const RecipLambda rl(lambda_row(seg_first), lane);
+        const RecipLambda<kD> rl(lambda_row(seg_first), lane);
         if (rl.wide) ctrl->any_wide = 1u;
         build_b_rows<C::kBTerms>(sB, prm.g.b0, rl, half, (warp - 2) * 8, (warp - 1) * 8, lane);
         fence_proxy_async();   // B is read by the tensor core through the async proxy
@@ -292,7 +260,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         const int r = q * 32 + lane;            // tile row and tensor-memory lane of this thread
         const uint4 *scales = static_cast<const uint4 *>(prm.g.scales);   // 8 fp16 scales per row
         int64_t cached_seg = n_my > 0 ? seg_first : -1;   // B holds this row's table (built above)
-        float rho = RecipLambda(lambda_row(seg_first), lane).rho;
+        float rho = RecipLambda<kD>(lambda_row(seg_first), lane).rho;
 
         TileCursor cur(tile_begin + grp, tps), ahead(tile_begin + grp, tps);
         auto fetch_scales = [&](int j) -> uint4 {
@@ -317,7 +285,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 
             // ---- a new lambda row: this group needs its rho; the group that meets the row's first tile rebuilds B
             if (seg != cached_seg) {
-                const RecipLambda rl(lambda_row(seg), lane);
+                const RecipLambda<kD> rl(lambda_row(seg), lane);
                 if (rl.wide) ctrl->any_wide = 1u;
                 rho = rl.rho;
                 if (cur.first_of_segment()) {

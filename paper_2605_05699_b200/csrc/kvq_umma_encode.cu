@@ -251,12 +251,9 @@ __global__ void __launch_bounds__(kThreads, 1)
 
     // ---- tiles: lambda segments of rpl rows, cut into tiles of 128 rows; a contiguous range per CTA
     const int64_t N = prm.N, rpl = prm.rpl;
-    const int64_t tps = (rpl + kTile - 1) / kTile;                 // tiles per segment
-    const int64_t n_tiles = prm.n_seg * tps;
-    const int64_t per_cta = (n_tiles + gridDim.x - 1) / gridDim.x;
-    const int64_t tile_begin = (int64_t)blockIdx.x * per_cta;
-    const int64_t tile_end = tile_begin + per_cta < n_tiles ? tile_begin + per_cta : n_tiles;
-    const int n_my = tile_end > tile_begin ? (int)(tile_end - tile_begin) : 0;
+    const TileShare share(prm.n_seg, rpl, blockIdx.x, gridDim.x);
+    const int64_t tps = share.tps, tile_begin = share.begin;
+    const int n_my = share.n;
 
     // ---- B for the CTA's first lambda row: D / 16 rows per epilogue warp.  Table rows and lambda are requested before
     // ---- the set-up barrier, so that their latency runs under it and under the first x loads.

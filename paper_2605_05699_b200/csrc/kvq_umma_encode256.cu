@@ -236,12 +236,9 @@ __device__ __forceinline__ void encode_d256_body(const UmmaEncode256Params &prm,
 
     // ---- tiles: lambda segments of rpl rows, cut into tiles of 128 rows; a contiguous range per CTA pair
     const int64_t N = prm.N, rpl = prm.rpl;
-    const int64_t tps = (rpl + kTile - 1) / kTile;                 // tiles per segment
-    const int64_t n_tiles = prm.n_seg * tps;
-    const int64_t per_pair = (n_tiles + n_pairs - 1) / n_pairs;
-    const int64_t tile_begin = (int64_t)pair * per_pair;
-    const int64_t tile_end = tile_begin + per_pair < n_tiles ? tile_begin + per_pair : n_tiles;
-    const int n_my = tile_end > tile_begin ? (int)(tile_end - tile_begin) : 0;
+    const TileShare share(prm.n_seg, rpl, (unsigned)pair, (unsigned)n_pairs);
+    const int64_t tps = share.tps, tile_begin = share.begin;
+    const int n_my = share.n;
 
     if (warp == 0) {
         // =========================== producer ===========================
