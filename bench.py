@@ -374,45 +374,57 @@ def bytes_per_vector(Dh: int) -> int:
     return 2 * Dh + Dh // 2 + 2 * (Dh // GROUP)
 
 
-def time_case(kb, wl, dev, Dh, dtype, Nv, kind, n_lambda=1, rpl=0, iters=20, warm=3, cold=False, seed=35):
-    """Device time of one kvq_encode and one kvq_decode launch of Nv vectors (events on the launching stream, one launch
-    per measurement): medians and minima over `iters` launches after `warm`.  cold=False: the same buffers every time (what
-    fits stays in L2).  cold=True: a 256 MB buffer is rewritten before every launch, so nothing of the case is left in L2."""
+def time_case(kb, wl, dev, Dh, dtype, Nv, kind, n_lambda=1, rpl=0, iters=12, warm=2, cold=False, seed=35):
+    """Device time per kvq_encode and per kvq_decode launch of Nv vectors: `reps` launches queued back to back between two
+    events on the launching stream, behind one more launch of the same call, so that neither the host's work for a launch
+    (binding, tensor maps, the launch itself: 15-25 us that an event recorded on an idle stream would count as device time)
+    nor an idle gap sits between the events; medians and minima over `iters` such measurements after `warm`.
+    cold=False: the same buffers every launch (what fits stays in L2).  cold=True: the launches rotate over enough buffer
+    sets to exceed 300 MB, more than twice the L2, so every launch reads from and writes to HBM."""
     import torch
 
+    bpv = bytes_per_vector(Dh)
+    n_sets = max(2, min(256, -(-300_000_000 // (Nv * bpv)))) if cold else 1
+    reps = max(4, n_sets)
     plan = kb.Plan(Dh, GROUP, 33)
     lam = wl.make_lambda(n_lambda, Dh, seed - 1, device=dev)
-    x = wl.make_vectors(Nv, Dh, dtype, kind, seed, device=dev)
-    pk, sc, out = plan.empty_packed(Nv, dev), plan.empty_scales(Nv, dev), torch.empty_like(x)
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if cold else None
+    sets = []
+    for k in range(n_sets):
+        x = wl.make_vectors(Nv, Dh, dtype, kind, seed + k, device=dev)
+        sets.append((x, plan.empty_packed(Nv, dev), plan.empty_scales(Nv, dev), torch.empty_like(x)))
+    for x, pk, sc, out in sets:                      # the codes every decode reads
+        kb.kvq_encode(plan.handle, x, lam, pk, sc, rpl)
+
+    def encode(k):
+        x, pk, sc, out = sets[k % n_sets]
+        kb.kvq_encode(plan.handle, x, lam, pk, sc, rpl)
+
+    def decode(k):
+        x, pk, sc, out = sets[k % n_sets]
+        kb.kvq_decode(plan.handle, pk, sc, lam, out, rpl)
+
     enc, dec = [], []
     for i in range(iters + warm):
-        e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
-        if flush is not None:
-            flush.fill_(i & 255)
-        e[0].record()
-        kb.kvq_encode(plan.handle, x, lam, pk, sc, rpl)
-        e[1].record()
-        if flush is not None:
-            flush.fill_((i + 1) & 255)
-        e[2].record()
-        kb.kvq_decode(plan.handle, pk, sc, lam, out, rpl)
-        e[3].record()
-        torch.cuda.synchronize()
-        if i >= warm:
-            enc.append(e[0].elapsed_time(e[1]))
-            dec.append(e[2].elapsed_time(e[3]))
+        for fn, acc in ((encode, enc), (decode, dec)):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            fn(n_sets - 1)                           # in front: the stream is busy while the host queues the timed launches
+            e0.record()
+            for k in range(reps):
+                fn(k)
+            e1.record()
+            torch.cuda.synchronize()
+            if i >= warm:
+                acc.append(e0.elapsed_time(e1) / reps)
     assert kb.kvq_plan_device_status(plan.handle) == 0
     plan.close()
     peak, _ = measured_peak()
-    bpv = bytes_per_vector(Dh)
 
     def stats(ms):
         med, mn = statistics.median(ms), min(ms)
         return {"us_median": 1e3 * med, "us_min": 1e3 * mn, "ns_per_vec": med * 1e6 / Nv, "GBps": Nv * bpv / (med * 1e-3) / 1e9,
                 "frac_of_hbm_peak": Nv * bpv / (med * 1e-3) / 1e9 / peak}
 
-    return {"encode": stats(enc), "decode": stats(dec)}
+    return {"encode": stats(enc), "decode": stats(dec), "launches_per_measurement": reps, "buffer_sets": n_sets}
 
 
 def hot_and_cold(kb, wl, dev, Dh, dtype, Nv, kind, n_lambda=1, rpl=0, iters=20):
@@ -433,7 +445,7 @@ def measure_config4(kb, wl, dev):
     """Config 4: the mixed-radix head dims, 65,536 vectors each, fp16, lognormal channel scales."""
     return {"D96": hot_and_cold(kb, wl, dev, 96, "f16", 65536, "lognormal"),
             "D160": hot_and_cold(kb, wl, dev, 160, "f16", 65536, "lognormal"),
-            "note": "16-27 MB per launch: fits L2 when hot; cold = a 256 MB buffer rewritten before every launch"}
+            "note": "16-27 MB per launch: fits L2 when hot; cold = the launches rotate over more than 300 MB of buffer sets"}
 
 
 def measure_config2(kb, wl, dev, steps=128):
