@@ -17,7 +17,8 @@
 //     a_hi + a_lo (one half2 FMA), W' = W_hi + W_lo, and a_hi W_hi + a_lo W_hi + a_hi W_lo accumulates in fp32
 //     (the a_lo W_lo term is below 1e-7).  fp16 output needs one term.
 //
-//   warp 0        producer   one TMA tensor load per tile: 128 packed rows x 128 B, 128-byte swizzle, 4 stages (2 for bf16)
+//   warp 0        producer   one TMA tensor load per tile: 128 packed rows x 128 B, 128-byte swizzle, 4 stages (2 for bf16);
+//                            byte codes (template BITS = 8): rows of 256 B as two such boxes, 2 stages (1 for bf16)
 //   warps 2-9     dequant    two groups of four warps, thread = row, both on every tile: group 0 turns the even
 //                            channels of the row's packed words into the A operand of the E GEMM, group 1 the
 //                            odd ones into that of the O GEMM (tensor memory; two stages each for fp16 output,

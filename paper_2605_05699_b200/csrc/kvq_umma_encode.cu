@@ -10,16 +10,18 @@
 //      bf16 input:  W 2^k = W1 + W2          (two bf16 terms: 16 bits; 6e-6 of the codes and 0.2 % of the stored
 //                                             scales then differ from the fp64 evaluation, all at rounding ties;
 //                                             the calibration pass adds a third term)
-// every product x_n W_i[c, n] is exact in fp32, and all terms accumulate in one fp32 accumulator in
-// tensor memory.  A term costs as much energy as the same GEMM in a library (0.6 pJ per flop), and the kernel runs
+// every product x_n W_i[c, n] is exact in fp32, and the terms are summed in fp32: for D <= 128 the two terms are stacked
+// along N (one MMA of N = 2 D per K-step fills two halves of the accumulator, which the epilogue adds: an MMA
+// instruction costs about 117 cycles whatever N <= 128 it carries and 176 at N = 256, so half the instructions is
+// worth more than the flops); D = 160 and the three-term forms accumulate all terms in one accumulator.  A term costs as much energy as the same GEMM in a library (0.6 pJ per flop), and the kernel runs
 // at the board's power cap, so a term more is 20 % less throughput.  2^k lifts the small terms clear of fp16's subnormal range; the epilogue undoes it in
 // the scale computation, at no cost per element.
 //
 //   warp 0        producer   one TMA tensor load per K block of 64 elements and tile of 128 vectors (128-byte
 //                            swizzle): x lands in shared memory in the tensor core's canonical K-major
 //                            layout, several tiles in flight, no thread touches it
-//   warp 1        mma        one thread issues D / 16 K-steps per split term into one accumulator stage, then
-//                            commits once: the epilogue reads it as "accumulator full", the producer as
+//   warp 1        mma        one thread issues D / 16 K-steps (per split term where the terms are not stacked) into
+//                            one accumulator stage, then commits once: the epilogue reads it as "accumulator full", the producer as
 //                            "x stage free"
 //   warps 2-17    epilogue   two sets of eight warps on alternate tiles; thread = (row, half row).  Per group
 //                            of 32 channels: tcgen05.ld of the 32 accumulator columns, abs-max, fp16 scale,
@@ -30,8 +32,9 @@
 //                            row rebuilds the B operand (the mma warp waits for it on an mbarrier).
 //
 //   A [128 vectors, K = D]     x in shared memory (TMA), K-major, 128-byte swizzle, K blocks of 64
-//   B [N = D channels, K]      split terms of W 2^k in shared memory, same layout, one region per term
-//   D [128, D]                 fp32 accumulator in tensor memory, three or four stages
+//   B [N = D channels, K]      split terms of W 2^k in shared memory, same layout: one region per term, or the
+//                              terms stacked as rows [0, D) and [D, 2 D) of every K block (D <= 128, two terms)
+//   D [128, D or 2 D]          fp32 accumulator in tensor memory, two to four stages
 //
 // Every wait on an mbarrier is bounded: on a time-out the role records the reason in the status word,
 // raises the CTA's abort flag and leaves its loop; the CTA then frees its tensor memory and returns.

@@ -13,7 +13,10 @@
 //     as soon as the block has landed and releases it with a commit of its own.
 //
 // Roles as in kvq_umma_encode.cu: producer (TMA), one mma thread, two epilogue sets of eight warps on
-// alternate tiles (thread = (row, two groups)); four accumulator stages of 128 columns; every wait is bounded.
+// alternate tiles (thread = (row, two groups)).  With two terms they are stacked along N as there (one MMA of
+// N = 256 per K-step and CTA, two accumulator stages of 256 columns, the epilogue adds the halves); the three-term
+// calibration form keeps four stages of 128 columns.  Byte codes (fp16 input) are a run-time switch of the epilogue.
+// Every wait is bounded.
 #include "kvq_internal.h"
 #include "kvq_umma.cuh"
 
