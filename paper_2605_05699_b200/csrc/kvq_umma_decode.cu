@@ -318,10 +318,31 @@ __global__ void __launch_bounds__(kThreads, 1)
     // ---- B for the first tile's lambda row: the sixteen dequant and epilogue warps build D / 16 rows each while the
     // ---- producer's first loads are in flight; the mma warp waits for all of them.  Table rows and lambda are
     // ---- requested before the set-up barrier, so that their latency runs under it.
+    // ---- The dequant warps also request the scales of their first tile here and keep rho, so that neither costs a round
+    // ---- trip to L2 after the build.
+    float rho_first = 1.0f;
+    uint32_t sc_first[(G + 1) / 2];
+#pragma unroll
+    for (int i = 0; i < (G + 1) / 2; ++i) sc_first[i] = 0u;
     if (n_my > 0 && warp >= 2) {
         FirstRows<D, BF16OUT, BITS, R2> rows;
         rows.load(prm.g.b0, (warp - 2) * (C::kBRows / 16), lane);
+        if (warp < 10 && ((warp - 2) >> 2) < n_my) {   // dequant group g's first tile is tile_begin + g
+            const TileCursor first(tile_begin + ((warp - 2) >> 2), tps);
+            const int64_t row = prm.g.phys_row(first.seg, first.row_in_segment(), rpl) + (warp & 3) * 32 + lane;
+            const uint16_t *scales = static_cast<const uint16_t *>(prm.g.scales);
+            if (row < prm.phys_rows) {
+                if (prm.g.per_vector) {
+                    const uint32_t s1 = (uint32_t)__ldg(scales + row);
+#pragma unroll
+                    for (int i = 0; i < (G + 1) / 2; ++i) sc_first[i] = s1 | (s1 << 16);
+                } else {
+                    load_row_scales<G>(scales + row * G, sc_first);
+                }
+            }
+        }
         const RecipLambda<D> rl(lambda_row(seg_first), lane);
+        rho_first = rl.rho;
         fence_proxy_async();
         tc_fence_before();
         __syncthreads();
@@ -425,7 +446,7 @@ __global__ void __launch_bounds__(kThreads, 1)
                              : C::kInSwizzleBits == 1 ? (uint32_t)((r >> 2) & 1)
                                                       : 0u;
         int64_t cached_seg = n_my > 0 ? seg_first : -1;   // B holds this row's table (built above)
-        float rho = RecipLambda<D>(lambda_row(seg_first), lane).rho;
+        float rho = rho_first;
 
         TileCursor cur(tile_begin + grp, tps), ahead(tile_begin + grp, tps);   // this tile; the tile whose scales are fetched
         uint32_t sc_next[(G + 1) / 2];
@@ -446,7 +467,8 @@ __global__ void __launch_bounds__(kThreads, 1)
             }
         };
 
-        fetch_scales(grp);
+#pragma unroll
+        for (int i = 0; i < (G + 1) / 2; ++i) sc_next[i] = sc_first[i];   // requested before the first B build
         for (int j = grp; j < n_my; j += 2, cur.advance(2)) {
             uint32_t sc[(G + 1) / 2];
 #pragma unroll

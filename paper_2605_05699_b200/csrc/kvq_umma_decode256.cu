@@ -198,8 +198,25 @@ __global__ void __launch_bounds__(kThreads, 1)
 
     // ---- B for the first tile's lambda row: of the sixteen dequant and epilogue warps, eight build the E operand
     // ---- and eight the O operand, sixteen rows each
+    // ---- (the dequant warps request their first tile's scales before the build and keep rho from it, so that neither
+    // ---- costs a round trip to L2 after it)
+    float rho_first = 1.0f;
+    uint4 sc_first = make_uint4(0u, 0u, 0u, 0u);
     if (n_my > 0 && warp >= 2) {
+        if (warp < 10) {
+            const TileCursor first(tile_begin, tps);
+            const int64_t row = prm.g.phys_row(first.seg, first.row_in_segment(), rpl) + (warp & 3) * 32 + lane;
+            if (row < prm.phys_rows) {
+                if (prm.g.per_vector) {
+                    const uint32_t s1 = (uint32_t)__ldg(static_cast<const uint16_t *>(prm.g.scales) + row);
+                    sc_first = make_uint4(s1 | (s1 << 16), s1 | (s1 << 16), s1 | (s1 << 16), s1 | (s1 << 16));
+                } else {
+                    sc_first = __ldg(static_cast<const uint4 *>(prm.g.scales) + row);
+                }
+            }
+        }
         const RecipLambda<kD> rl(lambda_row(seg_first), lane);
+        rho_first = rl.rho;
         if (rl.wide) ctrl->any_wide = 1u;
         const int bp = ((warp - 2) >> 2) & 1, bw = ((warp - 2) & 3) + 4 * ((warp - 2) >> 3);   // parity, position among its eight
         build_b_rows<kTerms>(sB, prm.g.b0, rl, bp, bw * 16, bw * 16 + 16, lane);
@@ -277,7 +294,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         const int r = q * 32 + lane;            // tile row and tensor-memory lane of this thread
         const uint4 *scales = static_cast<const uint4 *>(prm.g.scales);   // 8 fp16 scales per row
         int64_t cached_seg = n_my > 0 ? seg_first : -1;   // B holds this row's table (built above)
-        float rho = RecipLambda<kD>(lambda_row(seg_first), lane).rho;
+        float rho = rho_first;
 
         TileCursor cur(tile_begin, tps), ahead(tile_begin, tps);
         auto fetch_scales = [&](int j) -> uint4 {
@@ -291,7 +308,7 @@ __global__ void __launch_bounds__(kThreads, 1)
             }
             return __ldg(scales + row);
         };
-        uint4 sc_next = fetch_scales(0);
+        uint4 sc_next = sc_first;   // requested before the first B build
         for (int j = 0; j < n_my; ++j, cur.advance(1)) {
             const uint4 sc4 = sc_next;
             const uint32_t sc[4] = {sc4.x, sc4.y, sc4.z, sc4.w};

@@ -153,7 +153,7 @@ __device__ __forceinline__ void build_b_rows(unsigned char *sB, const float *__r
                                              int half, int c0, int c1, int lane)
 {
     using C = Cfg<BF16, CALIB>;
-#pragma unroll 2
+#pragma unroll 2   // (eight rows in flight were tried: slower, 60.3 against 55.9 us at 212,992 vectors and 52 lambda rows)
     for (int c = c0; c < c1; ++c) {
         const int cg = half * kHalfN + c;
         const float f = lam ? __ldg(lam + cg) * lift : lift;
