@@ -203,8 +203,11 @@ struct TileCursor {
 };
 
 // The contiguous share of a call's tiles that one CTA (or one CTA pair) of a persistent kernel takes: lambda segments of rpl
-// rows are cut into tiles of 128 rows (a segment's last tile may be short), n_seg * tps tiles in all, `parts` equal shares.
-// Contiguous, so that the B operand of a lambda row is rebuilt as rarely as possible.
+// rows are cut into tiles of 128 rows (a segment's last tile may be short), n_seg * tps tiles in all, `parts` shares.
+// Contiguous, so that the B operand of a lambda row is rebuilt as rarely as possible.  A share that crosses into another
+// lambda row pays a rebuild of B, about one tile's time, so with several rows and at least eight tiles per share the shares
+// are equal in COST, each segment counting one unit more than its tiles (a share that would begin inside that unit begins
+// at the segment's first tile); otherwise they are equal in tiles.
 struct TileShare {
     int64_t tps;     // tiles per segment
     int64_t begin;   // first tile of this share
@@ -213,9 +216,16 @@ struct TileShare {
     {
         tps = (rpl + 127) / 128;
         const int64_t n_tiles = n_seg * tps;
-        const int64_t per = (n_tiles + parts - 1) / parts;
-        begin = (int64_t)part * per;
-        const int64_t end = begin + per < n_tiles ? begin + per : n_tiles;
+        const int64_t R = (n_seg > 1 && n_tiles >= 8 * (int64_t)parts) ? 1 : 0;   // cost units of a rebuild
+        const int64_t C = tps + R, total = n_seg * C;
+        const int64_t per = (total + parts - 1) / parts;
+        auto tile_of = [&](int64_t u) -> int64_t {
+            if (u >= total) return n_tiles;
+            const int64_t seg = u / C, w = u - seg * C;
+            return seg * tps + (w > R ? w - R : 0);
+        };
+        begin = tile_of((int64_t)part * per);
+        const int64_t end = tile_of(((int64_t)part + 1) * per);
         n = end > begin ? (int)(end - begin) : 0;
     }
 };
